@@ -1,0 +1,204 @@
+/*
+ * bigcn.h - C ABI of the binarized Bi-GCN forward layer for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the forward path of "Binary Graph Convolutional Network with Capacity
+ * Exploration" (Bi-GCN): feature / weight binarization with bit packing (Sec. 4.2.1, 4.2.2), the
+ * XNOR + bit-count contraction with its beta_i alpha_j rescale (Sec. 4.2.3, Eq. "cdot-op" and
+ * "bi-op"), and the floating-point aggregation with A_tilde = D_hat^-1/2 (A + I) D_hat^-1/2
+ * (Eq. 1; last equation of Sec. 4.2.3), whose output can be re-binarized for the next layer.
+ *
+ * General rules
+ *   - Every data pointer is a DEVICE pointer owned by the caller unless a comment says "host".
+ *     The library allocates no data buffers: scratch comes from the workspace the caller attaches
+ *     with bigcn_set_workspace().  A context owns only a few hundred bytes of device status words
+ *     and some CUDA events.
+ *   - All work is enqueued on the stream given to bigcn_create() (borrowed, not owned).  Calls are
+ *     asynchronous unless stated; results are ready once that stream has been synchronised.
+ *   - Matrices are row-major; leading dimensions ("ld") are in elements, packed strides in 32-bit
+ *     words.  Outputs must not alias inputs.  n = 0 is a valid no-op.
+ *   - Arguments are validated on the host before anything is launched; a failing call launches
+ *     nothing, returns a status other than BIGCN_OK and leaves a message in bigcn_last_error().
+ *   - There is no CPU fallback: without a CUDA device every compute entry point fails.
+ *
+ * Packed layout (the paper fixes "1 bit per element plus one 32-bit float per bucket", Sec. 5.1-5.2,
+ * not the bit order; this is the order used here): element 32*w + k of a bucket is bit k (bit 0 =
+ * least significant) of 32-bit word w; +1 is stored as 1 and -1 as 0; bits past the bucket length
+ * and words past ceil(len/32) are 0.  A packed row occupies bigcn_packed_stride_words(len) words:
+ * ceil(len/32) rounded up to a multiple of 4, so that every row starts on a 16-byte boundary.
+ * sign(x) = +1 iff x >= 0 (both zeros give +1; a NaN gives -1).
+ */
+#ifndef BIGCN_H
+#define BIGCN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define BIGCN_MAX_LAYERS 16
+
+typedef enum {
+    BIGCN_OK = 0,
+    BIGCN_ERR_NULL = 1,        /* a required pointer is null */
+    BIGCN_ERR_SHAPE = 2,       /* a size, leading dimension or stride is out of range */
+    BIGCN_ERR_ALIGN = 3,       /* a pointer is not aligned as documented */
+    BIGCN_ERR_GRAPH = 4,       /* the sparse structure is malformed */
+    BIGCN_ERR_WORKSPACE = 5,   /* no workspace attached, or it is too small */
+    BIGCN_ERR_CUDA = 6,        /* a CUDA runtime call failed (message in bigcn_last_error) */
+    BIGCN_ERR_UNSUPPORTED = 7, /* a valid request this build does not implement */
+    BIGCN_ERR_INTERNAL = 8     /* a device-side self-check tripped */
+} bigcn_status;
+
+typedef struct bigcn_ctx bigcn_ctx;
+
+/* Options for bigcn_set_option(). */
+enum {
+    /* Storage of the rescaled contraction zeta between the bit-GEMM and the aggregation.
+     * 0 = choose per layer (default); 1 = fp32 zeta_ij = (beta_i alpha_j) dot_ij, exactly Eq. "cdot-op";
+     * 2 = the integer dot products as int16, with beta folded into the edge weights and alpha
+     *     applied once per output element (same sum, different rounding order);
+     * 3 = as 2 but int8 (layers with d_in <= 127 only; others fall back to 2). */
+    BIGCN_OPT_ZETA_FORMAT = 1,
+    /* Rows of the sparse matrix with more entries than this are split across thread blocks. 0 = default. */
+    BIGCN_OPT_LONG_ROW = 2
+};
+
+/* Context: binds a device and a stream.  `cuda_stream` is a cudaStream_t (0 = default stream). */
+bigcn_status bigcn_create(bigcn_ctx** out, int device, void* cuda_stream);
+bigcn_status bigcn_destroy(bigcn_ctx* ctx);
+/* Message of the last failing call on this context ("" if none).  Host string owned by ctx. */
+const char* bigcn_last_error(const bigcn_ctx* ctx);
+const char* bigcn_status_string(bigcn_status s);
+bigcn_status bigcn_set_option(bigcn_ctx* ctx, int32_t option, int64_t value);
+/* Number of kernels this context has launched so far. */
+int64_t bigcn_launch_count(const bigcn_ctx* ctx);
+/* Synchronises the stream and reports a pending CUDA error or a tripped device self-check. */
+bigcn_status bigcn_sync_check(bigcn_ctx* ctx);
+
+/* Words per packed row of `len` elements: ceil(len/32) rounded up to a multiple of 4. */
+int64_t bigcn_packed_stride_words(int32_t len);
+
+/* Scratch.  bigcn_workspace_bytes() bounds what bigcn_forward()/bigcn_layer_forward() need for a
+ * graph of n nodes and nnz stored entries and the layer widths dims[0..n_layers];
+ * with host_io != 0 it adds the staging buffers of bigcn_forward_host().
+ * bigcn_set_workspace() attaches caller-owned device memory (256-byte aligned) until replaced. */
+size_t bigcn_workspace_bytes(int64_t n, int64_t nnz, const int32_t* dims /*host*/, int32_t n_layers,
+                             int32_t host_io);
+bigcn_status bigcn_set_workspace(bigcn_ctx* ctx, void* workspace, size_t bytes);
+
+/* Sparse normalised adjacency in CSR (Eq. 1: A_tilde = D_hat^-1/2 (A + I) D_hat^-1/2, "a sparse
+ * matrix").  rowptr[n+1] int64, colidx[nnz] int32 ascending within a row and including the
+ * diagonal, val[nnz] fp32 = dinv[i] * dinv[j], dinv[n] fp32 = D_hat_ii^-1/2.  n < 2^31. */
+typedef struct {
+    int64_t n;
+    int64_t nnz;
+    const int64_t* rowptr;
+    const int32_t* colidx;
+    const float* val;
+    const float* dinv;
+} bigcn_graph;
+
+/* Set-up step, once per graph (Sec. 3.1, Eq. 1).  Input: CSR of the adjacency A of an undirected
+ * graph: symmetric pattern, columns ascending and unique within a row; diagonal entries in the
+ * input are ignored and exactly one self-loop per node is added (A_hat = A + I).
+ * Output arrays must hold nnz_in + n entries (colidx, val), n + 1 (rowptr) and n (dinv).
+ * D_hat_ii = number of stored entries of row i of A_hat; dinv = 1/sqrt(D_hat_ii) evaluated in
+ * double and rounded to fp32; val = fp32 product dinv[i] * dinv[j].
+ * The input is checked on the device (ascending unique columns in [0, n), symmetry); a violation
+ * gives BIGCN_ERR_GRAPH.  Needs 16 * (n/1024 + 2) + 64 bytes of workspace.  SYNCHRONOUS: returns after the
+ * stream has drained; *nnz_out (host) receives the number of stored entries. */
+bigcn_status bigcn_normalize_adjacency(bigcn_ctx* ctx, int64_t n, int64_t nnz_in,
+                                       const int64_t* rowptr_A, const int32_t* colidx_A,
+                                       int64_t* rowptr, int32_t* colidx, float* val, float* dinv,
+                                       int64_t* nnz_out /*host*/);
+
+/* Feature binarization (Sec. 4.2.2, Eq. "beta" and "F"; batch normalisation of the input as in
+ * Sec. 4.4).  H fp32 [n x d], leading dimension ld >= d.  With col_shift/col_scale (fp32 [d], both
+ * or neither) x_hat_ij = (H_ij - shift_j) * scale_j in fp32, else x_hat = H.
+ * bits_out u32 [n x stride_words] gets F_i = sign(x_hat_i,:) in the packed layout (stride_words >=
+ * bigcn_packed_stride_words(d), multiple of 4; every word of the row is written); beta_out fp32 [n]
+ * gets ||x_hat_i,:||_1 / d (the bucket length; Eq. "beta" prints 1/N, see the generic rule of
+ * Sec. 4.1).  bits_out must be 16-byte aligned. */
+bigcn_status bigcn_pack_features(bigcn_ctx* ctx, const float* H, int64_t n, int32_t d, int64_t ld,
+                                 const float* col_shift, const float* col_scale,
+                                 uint32_t* bits_out, int64_t stride_words, float* beta_out);
+
+/* Weight binarization (Sec. 4.2.1, Eq. "B" and "alpha").  W fp32 [d_in x d_out], leading dimension
+ * ldw >= d_out.  bitsT_out u32 [d_out x stride_words]: row j holds B_j = sign(W_:,j) packed along
+ * d_in; alpha_out fp32 [d_out] = ||W_:,j||_1 / d_in. */
+bigcn_status bigcn_pack_weights(bigcn_ctx* ctx, const float* W, int32_t d_in, int32_t d_out, int64_t ldw,
+                                uint32_t* bitsT_out, int64_t stride_words, float* alpha_out);
+
+/* One binarized layer's parameters: packed weights from bigcn_pack_weights() with
+ * stride bigcn_packed_stride_words(d_in), and the optional batch-norm constants of the layer's
+ * INPUT (fp32 [d_in], both or neither; Sec. 4.4). */
+typedef struct {
+    int32_t d_in;
+    int32_t d_out;
+    const uint32_t* w_bitsT;
+    const float* alpha;
+    const float* in_shift;
+    const float* in_scale;
+} bigcn_layer;
+
+/* One layer (Sec. 4.2.3): dot_ij = F_i (*) B_j = d_in - 2 popc(F_i XOR B_j) (Eq. "bi-op"),
+ * zeta_ij = beta_i alpha_j dot_ij (Eq. "cdot-op"), H' = A_tilde zeta.  No bias, no activation.
+ *   in_bits  u32 [n x bigcn_packed_stride_words(d_in)], in_beta fp32 [n]: the packed input.
+ *   h_out    fp32 [n x ldh] or null: H'.
+ *   next     null, or the following layer: then next_bits [n x bigcn_packed_stride_words(d_out)] and
+ *            next_beta [n] receive the binarization of H' under next->in_shift/in_scale
+ *            (next->d_in must equal layer->d_out).  h_out and next may both be given.
+ *   dbg_dot  int32 [n x d_out] or null, dbg_zeta fp32 [n x d_out] or null: taps on the contraction
+ *            for testing (dbg_zeta always in the fp32 form of Eq. "cdot-op").
+ * Needs workspace (bigcn_workspace_bytes with n_layers = 1). */
+bigcn_status bigcn_layer_forward(bigcn_ctx* ctx, const bigcn_graph* graph, const bigcn_layer* layer,
+                                 const uint32_t* in_bits, const float* in_beta,
+                                 float* h_out, int64_t ldh,
+                                 const bigcn_layer* next, uint32_t* next_bits, float* next_beta,
+                                 int32_t* dbg_dot, float* dbg_zeta);
+
+/* Per-step device times of one bigcn_forward() call, in milliseconds (CUDA events). */
+typedef struct {
+    int32_t n_layers;
+    int32_t launches;
+    float ms_total;
+    float ms_pack;                       /* binarize + pack of X */
+    float ms_gemm[BIGCN_MAX_LAYERS];     /* XNOR/bit-count contraction + rescale */
+    float ms_spmm[BIGCN_MAX_LAYERS];     /* aggregation (+ re-binarization) */
+} bigcn_stats;
+
+/* L stacked layers from fp32 features to logits (H^(0) = X, Sec. 3.2; every layer binarized, the
+ * last one's H' returned as logits [n x ldo]).  `layers` is a HOST array of n_layers structs whose
+ * pointers are device pointers.  With stats != null the call records events around every step and
+ * synchronises before returning; otherwise it is asynchronous. */
+bigcn_status bigcn_forward(bigcn_ctx* ctx, const bigcn_graph* graph, const bigcn_layer* layers /*host*/,
+                           int32_t n_layers, const float* X, int64_t ldx,
+                           float* logits_out, int64_t ldo, bigcn_stats* stats /*host, nullable*/);
+
+/* As bigcn_forward() from features that are already binarized ("loaded data is binary", Sec. 5.2):
+ * x_bits [n x bigcn_packed_stride_words(dims[0])], x_beta [n]. */
+bigcn_status bigcn_forward_packed(bigcn_ctx* ctx, const bigcn_graph* graph, const bigcn_layer* layers /*host*/,
+                                  int32_t n_layers, const uint32_t* x_bits, const float* x_beta,
+                                  float* logits_out, int64_t ldo, bigcn_stats* stats /*host, nullable*/);
+
+/* As bigcn_forward() with HOST buffers for the per-call data: X_host fp32 [n x ldx] (ldx = d_0
+ * required) is copied to the device, the forward runs, logits_host fp32 [n x ldo] (ldo = classes)
+ * is copied back, and the call returns after the stream has drained.  Graph and layer arrays
+ * stay device-resident.  Page-locked host memory makes the copies asynchronous and faster but is
+ * not required.  Needs a workspace sized with host_io = 1. */
+bigcn_status bigcn_forward_host(bigcn_ctx* ctx, const bigcn_graph* graph, const bigcn_layer* layers /*host*/,
+                                int32_t n_layers, const float* X_host, int64_t ldx,
+                                float* logits_host, int64_t ldo);
+
+/* Batch statistics for the batch normalisation of a layer's input (Sec. 4.4: zero mean, unit
+ * variance per feature over the nodes): shift_out[j] = mean_j, scale_out[j] = 1/sqrt(var_j + eps),
+ * biased variance.  H fp32 [n x d], ld >= d.  Needs 16 * d * 1024 bytes of workspace. */
+bigcn_status bigcn_col_stats(bigcn_ctx* ctx, const float* H, int64_t n, int32_t d, int64_t ld,
+                             float eps, float* shift_out, float* scale_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BIGCN_H */

@@ -16,6 +16,7 @@ from __future__ import annotations
 
 import ctypes
 import os
+import platform
 import subprocess
 from dataclasses import dataclass
 from typing import List, Optional, Sequence
@@ -40,6 +41,8 @@ def build(force: bool = False) -> str:
     tmp = _LIB + ".%d.tmp" % os.getpid()
     cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off",
            "-fno-fast-math", "-o", tmp, _SRC, "-lm"]
+    if platform.machine() in ("x86_64", "AMD64"):
+        cmd.insert(1, "-mpopcnt")
     subprocess.run(cmd, check=True)
     os.replace(tmp, _LIB)
     return _LIB

@@ -249,12 +249,8 @@ void oracle_dot_pm1(const int8_t* F, const int8_t* B, int64_t n, int32_t d_in, i
         }
 }
 
-static inline int32_t count_ones(uint32_t x)
-{
-    int32_t c = 0;
-    while (x) { x &= x - 1u; ++c; }      /* clears the lowest set bit each turn */
-    return c;
-}
+/* bit count of a word (the compiler's population-count primitive) */
+static inline int32_t count_ones(uint32_t x) { return (int32_t)__builtin_popcount(x); }
 
 /* ------------------------------------------------------------------------- */
 /* Eq. "bi-op": the same inner product by XNOR and bit count.  Over the d_in  */

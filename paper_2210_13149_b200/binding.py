@@ -1,0 +1,321 @@
+"""ctypes binding of libbigcn (``include/bigcn.h``).
+
+Argument marshalling only: every step of the forward path runs in the library's CUDA kernels.
+torch is used for device memory (inputs, outputs, the workspace) and for the current stream.
+There is no CPU fallback: if the shared library cannot be loaded or no CUDA device is present,
+creating a :class:`BiGCN` raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbigcn.so")
+
+MAX_LAYERS = 16
+OPT_ZETA_FORMAT = 1
+OPT_LONG_ROW = 2
+ZETA_AUTO, ZETA_F32, ZETA_I16, ZETA_I8 = 0, 1, 2, 3
+
+_i32, _i64, _vp, _sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_size_t
+
+
+class bigcn_graph(ctypes.Structure):
+    _fields_ = [("n", _i64), ("nnz", _i64), ("rowptr", _vp), ("colidx", _vp), ("val", _vp), ("dinv", _vp)]
+
+
+class bigcn_layer(ctypes.Structure):
+    _fields_ = [("d_in", _i32), ("d_out", _i32), ("w_bitsT", _vp), ("alpha", _vp),
+                ("in_shift", _vp), ("in_scale", _vp)]
+
+
+class bigcn_stats(ctypes.Structure):
+    _fields_ = [("n_layers", _i32), ("launches", _i32), ("ms_total", ctypes.c_float),
+                ("ms_pack", ctypes.c_float), ("ms_gemm", ctypes.c_float * MAX_LAYERS),
+                ("ms_spmm", ctypes.c_float * MAX_LAYERS)]
+
+
+# name -> (restype, argtypes); every symbol include/bigcn.h declares
+SIGNATURES = {
+    "bigcn_create": (ctypes.c_int, [ctypes.POINTER(_vp), ctypes.c_int, _vp]),
+    "bigcn_destroy": (ctypes.c_int, [_vp]),
+    "bigcn_last_error": (ctypes.c_char_p, [_vp]),
+    "bigcn_status_string": (ctypes.c_char_p, [ctypes.c_int]),
+    "bigcn_set_option": (ctypes.c_int, [_vp, _i32, _i64]),
+    "bigcn_launch_count": (_i64, [_vp]),
+    "bigcn_sync_check": (ctypes.c_int, [_vp]),
+    "bigcn_packed_stride_words": (_i64, [_i32]),
+    "bigcn_workspace_bytes": (_sz, [_i64, _i64, ctypes.POINTER(_i32), _i32, _i32]),
+    "bigcn_set_workspace": (ctypes.c_int, [_vp, _vp, _sz]),
+    "bigcn_normalize_adjacency": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp,
+                                                 ctypes.POINTER(_i64)]),
+    "bigcn_pack_features": (ctypes.c_int, [_vp, _vp, _i64, _i32, _i64, _vp, _vp, _vp, _i64, _vp]),
+    "bigcn_pack_weights": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i64, _vp, _i64, _vp]),
+    "bigcn_layer_forward": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer),
+                                           _vp, _vp, _vp, _i64, ctypes.POINTER(bigcn_layer), _vp, _vp, _vp, _vp]),
+    "bigcn_forward": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer), _i32,
+                                     _vp, _i64, _vp, _i64, ctypes.POINTER(bigcn_stats)]),
+    "bigcn_forward_packed": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer), _i32,
+                                            _vp, _vp, _vp, _i64, ctypes.POINTER(bigcn_stats)]),
+    "bigcn_forward_host": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer), _i32,
+                                          _vp, _i64, _vp, _i64]),
+    "bigcn_col_stats": (ctypes.c_int, [_vp, _vp, _i64, _i32, _i64, ctypes.c_float, _vp, _vp]),
+}
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Loads libbigcn.so from the package directory (build it with ``python -m
+    paper_2210_13149_b200.build`` or ``__graft_entry__.build()``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libbigcn.so is not built (%s): run paper_2210_13149_b200/build.py; "
+                               "there is no fallback path" % LIB_PATH)
+        lib = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = lib
+    return _lib
+
+
+class BigcnError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__("bigcn status %d: %s" % (status, message))
+        self.status = status
+
+
+def packed_stride_words(length: int) -> int:
+    return int(load().bigcn_packed_stride_words(int(length)))
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+@dataclass
+class Graph:
+    """Device-resident CSR of A_tilde plus the C struct that points at it."""
+    n: int
+    nnz: int
+    rowptr: torch.Tensor
+    colidx: torch.Tensor
+    val: torch.Tensor
+    dinv: Optional[torch.Tensor]
+    c: bigcn_graph
+
+
+def make_graph(rowptr: torch.Tensor, colidx: torch.Tensor, val: torch.Tensor,
+               dinv: Optional[torch.Tensor] = None) -> Graph:
+    assert rowptr.dtype == torch.int64 and colidx.dtype == torch.int32 and val.dtype == torch.float32
+    n = rowptr.numel() - 1
+    nnz = colidx.numel()
+    c = bigcn_graph(n, nnz, rowptr.data_ptr(), colidx.data_ptr(), val.data_ptr(),
+                    dinv.data_ptr() if dinv is not None else None)
+    return Graph(n, nnz, rowptr, colidx, val, dinv, c)
+
+
+@dataclass
+class Layer:
+    """Device-resident packed weights of one layer plus the C struct that points at them."""
+    d_in: int
+    d_out: int
+    w_bitsT: torch.Tensor
+    alpha: torch.Tensor
+    in_shift: Optional[torch.Tensor]
+    in_scale: Optional[torch.Tensor]
+    c: bigcn_layer
+
+
+def make_layer(d_in: int, d_out: int, w_bitsT: torch.Tensor, alpha: torch.Tensor,
+               in_shift: Optional[torch.Tensor] = None, in_scale: Optional[torch.Tensor] = None) -> Layer:
+    c = bigcn_layer(d_in, d_out, w_bitsT.data_ptr(), alpha.data_ptr(),
+                    in_shift.data_ptr() if in_shift is not None else None,
+                    in_scale.data_ptr() if in_scale is not None else None)
+    return Layer(d_in, d_out, w_bitsT, alpha, in_shift, in_scale, c)
+
+
+def _layer_array(layers: Sequence[Layer]):
+    arr = (bigcn_layer * len(layers))()
+    for i, l in enumerate(layers):
+        arr[i] = l.c
+    return arr
+
+
+class BiGCN:
+    """One library context bound to a device and to torch's current stream on it."""
+
+    def __init__(self, device: int = 0, stream: Optional[torch.cuda.Stream] = None):
+        self.lib = load()
+        if not torch.cuda.is_available():
+            raise RuntimeError("no CUDA device: the bigcn library has no CPU path")
+        self.device = torch.device("cuda", device)
+        with torch.cuda.device(self.device):
+            self.stream = stream if stream is not None else torch.cuda.current_stream()
+        h = _vp()
+        st = self.lib.bigcn_create(ctypes.byref(h), device, ctypes.c_void_p(self.stream.cuda_stream))
+        if st != 0:
+            raise BigcnError(st, self.lib.bigcn_status_string(st).decode())
+        self.h = h
+        self.workspace: Optional[torch.Tensor] = None
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.lib.bigcn_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- helpers
+    def _check(self, st: int):
+        if st != 0:
+            raise BigcnError(st, self.lib.bigcn_last_error(self.h).decode())
+
+    def _empty(self, shape, dtype):
+        return torch.empty(shape, dtype=dtype, device=self.device)
+
+    def set_option(self, option: int, value: int):
+        self._check(self.lib.bigcn_set_option(self.h, option, value))
+
+    def launch_count(self) -> int:
+        return int(self.lib.bigcn_launch_count(self.h))
+
+    def sync_check(self):
+        self._check(self.lib.bigcn_sync_check(self.h))
+
+    def workspace_bytes(self, n: int, nnz: int, dims: Sequence[int], host_io: bool = False) -> int:
+        arr = (_i32 * len(dims))(*[int(d) for d in dims])
+        return int(self.lib.bigcn_workspace_bytes(n, nnz, arr, len(dims) - 1, 1 if host_io else 0))
+
+    def ensure_workspace(self, nbytes: int):
+        if self.workspace is None or self.workspace.numel() < nbytes:
+            self.workspace = None
+            self.workspace = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=self.device)
+            self._check(self.lib.bigcn_set_workspace(self.h, _ptr(self.workspace), self.workspace.numel()))
+
+    # -- the ABI calls
+    def normalize_adjacency(self, rowptr_A: torch.Tensor, colidx_A: torch.Tensor) -> Graph:
+        n = rowptr_A.numel() - 1
+        nnz_in = colidx_A.numel()
+        self.ensure_workspace(16 * (n // 1024 + 2) + 64)
+        rowptr = self._empty(n + 1, torch.int64)
+        colidx = self._empty(nnz_in + n, torch.int32)
+        val = self._empty(nnz_in + n, torch.float32)
+        dinv = self._empty(n, torch.float32)
+        nnz = _i64(0)
+        self._check(self.lib.bigcn_normalize_adjacency(self.h, n, nnz_in, _ptr(rowptr_A), _ptr(colidx_A),
+                                                       _ptr(rowptr), _ptr(colidx), _ptr(val), _ptr(dinv),
+                                                       ctypes.byref(nnz)))
+        k = int(nnz.value)
+        return make_graph(rowptr, colidx[:k], val[:k], dinv)
+
+    def pack_features(self, H: torch.Tensor, shift: Optional[torch.Tensor] = None,
+                      scale: Optional[torch.Tensor] = None, stride_words: Optional[int] = None):
+        n, d = H.shape
+        ld = H.stride(0) if n > 1 else d
+        assert H.dtype == torch.float32 and (d == 1 or H.stride(1) == 1)
+        stride = packed_stride_words(d) if stride_words is None else stride_words
+        bits = self._empty((n, stride), torch.int32)
+        beta = self._empty(n, torch.float32)
+        self._check(self.lib.bigcn_pack_features(self.h, _ptr(H), n, d, ld, _ptr(shift), _ptr(scale),
+                                                 _ptr(bits), stride, _ptr(beta)))
+        return bits, beta
+
+    def pack_weights(self, W: torch.Tensor):
+        d_in, d_out = W.shape
+        assert W.dtype == torch.float32 and W.is_contiguous()
+        stride = packed_stride_words(d_in)
+        bitsT = self._empty((d_out, stride), torch.int32)
+        alpha = self._empty(d_out, torch.float32)
+        self._check(self.lib.bigcn_pack_weights(self.h, _ptr(W), d_in, d_out, d_out, _ptr(bitsT), stride, _ptr(alpha)))
+        return bitsT, alpha
+
+    def layer_forward(self, graph: Graph, layer: Layer, in_bits: torch.Tensor, in_beta: torch.Tensor,
+                      want_h: bool = True, next_layer: Optional[Layer] = None, debug: bool = False):
+        """Returns dict with h, next_bits, next_beta, dot, zeta (those requested)."""
+        n = graph.n
+        self.ensure_workspace(self.workspace_bytes(n, graph.nnz, [layer.d_in, layer.d_out]))
+        out = {}
+        h = self._empty((n, layer.d_out), torch.float32) if want_h else None
+        nb = nbeta = None
+        if next_layer is not None:
+            nb = self._empty((n, packed_stride_words(layer.d_out)), torch.int32)
+            nbeta = self._empty(n, torch.float32)
+        dot = self._empty((n, layer.d_out), torch.int32) if debug else None
+        zeta = self._empty((n, layer.d_out), torch.float32) if debug else None
+        self._check(self.lib.bigcn_layer_forward(
+            self.h, ctypes.byref(graph.c), ctypes.byref(layer.c), _ptr(in_bits), _ptr(in_beta),
+            _ptr(h), layer.d_out, ctypes.byref(next_layer.c) if next_layer is not None else None,
+            _ptr(nb), _ptr(nbeta), _ptr(dot), _ptr(zeta)))
+        out.update(h=h, next_bits=nb, next_beta=nbeta, dot=dot, zeta=zeta)
+        return out
+
+    def _prep_forward(self, graph: Graph, layers: Sequence[Layer], host_io: bool = False):
+        dims = [layers[0].d_in] + [l.d_out for l in layers]
+        self.ensure_workspace(self.workspace_bytes(graph.n, graph.nnz, dims, host_io))
+        return _layer_array(layers), dims
+
+    def forward(self, graph: Graph, layers: Sequence[Layer], X: torch.Tensor,
+                logits: Optional[torch.Tensor] = None, stats: bool = False):
+        arr, dims = self._prep_forward(graph, layers)
+        if logits is None:
+            logits = self._empty((graph.n, dims[-1]), torch.float32)
+        st = bigcn_stats() if stats else None
+        ldx = X.stride(0) if graph.n > 1 else dims[0]
+        self._check(self.lib.bigcn_forward(self.h, ctypes.byref(graph.c), arr, len(layers), _ptr(X), ldx,
+                                           _ptr(logits), logits.stride(0) if graph.n > 1 else dims[-1],
+                                           ctypes.byref(st) if stats else None))
+        return (logits, st) if stats else logits
+
+    def forward_packed(self, graph: Graph, layers: Sequence[Layer], x_bits: torch.Tensor, x_beta: torch.Tensor,
+                       logits: Optional[torch.Tensor] = None, stats: bool = False):
+        arr, dims = self._prep_forward(graph, layers)
+        if logits is None:
+            logits = self._empty((graph.n, dims[-1]), torch.float32)
+        st = bigcn_stats() if stats else None
+        self._check(self.lib.bigcn_forward_packed(self.h, ctypes.byref(graph.c), arr, len(layers), _ptr(x_bits),
+                                                  _ptr(x_beta), _ptr(logits),
+                                                  logits.stride(0) if graph.n > 1 else dims[-1],
+                                                  ctypes.byref(st) if stats else None))
+        return (logits, st) if stats else logits
+
+    def forward_host(self, graph: Graph, layers: Sequence[Layer], X_host: torch.Tensor,
+                     logits_host: torch.Tensor):
+        """X_host / logits_host are CPU tensors (pinned for speed); synchronous."""
+        arr, dims = self._prep_forward(graph, layers, host_io=True)
+        assert X_host.device.type == "cpu" and logits_host.device.type == "cpu"
+        assert X_host.is_contiguous() and logits_host.is_contiguous()
+        self._check(self.lib.bigcn_forward_host(self.h, ctypes.byref(graph.c), arr, len(layers), _ptr(X_host),
+                                                dims[0], _ptr(logits_host), dims[-1]))
+        return logits_host
+
+    def col_stats(self, H: torch.Tensor, eps: float = 1e-5):
+        n, d = H.shape
+        self.ensure_workspace(16 * d * 1024)
+        shift = self._empty(d, torch.float32)
+        scale = self._empty(d, torch.float32)
+        self._check(self.lib.bigcn_col_stats(self.h, _ptr(H), n, d, H.stride(0) if n > 1 else d, eps,
+                                             _ptr(shift), _ptr(scale)))
+        return shift, scale
+
+    # -- convenience built only from the calls above
+    def prepare_layers(self, weights: Sequence[torch.Tensor], shifts=None, scales=None) -> List[Layer]:
+        layers = []
+        for l, W in enumerate(weights):
+            bitsT, alpha = self.pack_weights(W)
+            sh = shifts[l] if shifts is not None else None
+            sc = scales[l] if scales is not None else None
+            layers.append(make_layer(W.shape[0], W.shape[1], bitsT, alpha, sh, sc))
+        return layers

@@ -1,0 +1,539 @@
+// C ABI of libbigcn: contexts, argument validation, workspace carving and the launch sequences.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "bigcn_internal.cuh"
+
+using namespace bigcn;
+
+struct bigcn_ctx {
+    int device;
+    cudaStream_t stream;
+    char err[512];
+    void* ws;
+    size_t ws_bytes;
+    int* d_flag;                 // device status words (owned)
+    int launches_i;              // launches of the call in progress
+    int64_t launches;
+    int zeta_format;             // 0 = auto
+    int64_t long_row;            // 0 = default
+    cudaEvent_t ev[2 * BIGCN_MAX_LAYERS + 2];
+    bool ev_ready;
+};
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int64_t kDefaultLongRow = 2048;
+
+bigcn_status fail(bigcn_ctx* ctx, bigcn_status s, const char* fmt, ...)
+{
+    if (ctx) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(ctx->err, sizeof(ctx->err), fmt, ap);
+        va_end(ap);
+    }
+    return s;
+}
+
+bigcn_status cuda_fail(bigcn_ctx* ctx, cudaError_t e, const char* what)
+{
+    return fail(ctx, BIGCN_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+#define BIGCN_CUDA(ctx, call)                                        \
+    do {                                                             \
+        cudaError_t e__ = (call);                                    \
+        if (e__ != cudaSuccess) return cuda_fail(ctx, e__, #call);   \
+    } while (0)
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+// Storage format of zeta for a layer under the context's option.
+int pick_format(const bigcn_ctx* ctx, int d_in)
+{
+    int f = ctx->zeta_format;
+    if (f == 0) f = kZetaI16;
+    if (f == kZetaI8 && d_in > 127) f = kZetaI16;
+    if (f == kZetaI16 && d_in > 32767) f = kZetaF32;
+    return f;
+}
+
+struct Carver {
+    char* base;
+    size_t size, off;
+    void* take(size_t bytes)
+    {
+        off = up(off);
+        if (off + bytes > size) return nullptr;
+        void* p = base + off;
+        off += bytes;
+        return p;
+    }
+};
+
+bigcn_status bind_device(bigcn_ctx* ctx)
+{
+    if (!ctx) return BIGCN_ERR_NULL;
+    BIGCN_CUDA(ctx, cudaSetDevice(ctx->device));
+    return BIGCN_OK;
+}
+
+bigcn_status check_graph(bigcn_ctx* ctx, const bigcn_graph* g)
+{
+    if (!g) return fail(ctx, BIGCN_ERR_NULL, "graph is null");
+    if (g->n < 0 || g->n >= (int64_t(1) << 31) || g->nnz < 0) return fail(ctx, BIGCN_ERR_SHAPE, "graph: n=%lld nnz=%lld out of range", (long long)g->n, (long long)g->nnz);
+    if (g->n > 0 && (!g->rowptr || (g->nnz > 0 && (!g->colidx || !g->val))))
+        return fail(ctx, BIGCN_ERR_NULL, "graph: rowptr/colidx/val must be given");
+    return BIGCN_OK;
+}
+
+bigcn_status check_layer(bigcn_ctx* ctx, const bigcn_layer* l, const char* name)
+{
+    if (!l) return fail(ctx, BIGCN_ERR_NULL, "%s is null", name);
+    if (l->d_in < 1 || l->d_out < 1) return fail(ctx, BIGCN_ERR_SHAPE, "%s: d_in=%d d_out=%d must be >= 1", name, l->d_in, l->d_out);
+    if (l->d_out > 512) return fail(ctx, BIGCN_ERR_UNSUPPORTED, "%s: d_out=%d > 512 is not supported", name, l->d_out);
+    if (!l->w_bitsT || !l->alpha) return fail(ctx, BIGCN_ERR_NULL, "%s: w_bitsT/alpha are null", name);
+    if ((l->in_shift == nullptr) != (l->in_scale == nullptr)) return fail(ctx, BIGCN_ERR_NULL, "%s: in_shift and in_scale go together", name);
+    if (!aligned(l->w_bitsT, 16)) return fail(ctx, BIGCN_ERR_ALIGN, "%s: w_bitsT must be 16-byte aligned", name);
+    return BIGCN_OK;
+}
+
+// One layer on already validated arguments.  `zeta` is scratch for n * zeta_ld(d_out) elements.
+bigcn_status run_layer(bigcn_ctx* ctx, const bigcn_graph* g, const bigcn_layer* layer,
+                       const uint32_t* in_bits, const float* in_beta, void* zeta,
+                       float* h_out, int64_t ldh, const bigcn_layer* next, uint32_t* next_bits,
+                       float* next_beta, int32_t* dbg_dot, float* dbg_zeta,
+                       cudaEvent_t ev_mid /*nullable*/)
+{
+    const int fmt = pick_format(ctx, layer->d_in);
+    const int64_t ldz = zeta_ld(layer->d_out, fmt);
+    const int64_t stride_in = bigcn_packed_stride_words(layer->d_in);
+    cudaError_t e = launch_bitgemm(ctx->stream, in_bits, stride_in, layer->w_bitsT, stride_in, g->n,
+                                   layer->d_in, layer->d_out, in_beta, layer->alpha, fmt, zeta, ldz,
+                                   dbg_dot, dbg_zeta, &ctx->launches_i);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "bit-GEMM launch");
+    if (ev_mid) BIGCN_CUDA(ctx, cudaEventRecord(ev_mid, ctx->stream));
+    SpmmArgs a;
+    a.n = g->n;
+    a.rowptr = g->rowptr;
+    a.colidx = g->colidx;
+    a.val = g->val;
+    a.fmt = fmt;
+    a.zeta = zeta;
+    a.ldz = ldz;
+    a.d_out = layer->d_out;
+    a.node_w = in_beta;
+    a.col_w = layer->alpha;
+    a.h_out = h_out;
+    a.ldh = ldh;
+    a.next_bits = next ? next_bits : nullptr;
+    a.next_stride = next ? bigcn_packed_stride_words(layer->d_out) : 0;
+    a.next_beta = next ? next_beta : nullptr;
+    a.next_shift = next ? next->in_shift : nullptr;
+    a.next_scale = next ? next->in_scale : nullptr;
+    a.long_row = ctx->long_row > 0 ? ctx->long_row : kDefaultLongRow;
+    a.scratch = nullptr;
+    a.scratch_bytes = 0;
+    e = launch_spmm(ctx->stream, a, &ctx->launches_i);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "SpMM launch");
+    return BIGCN_OK;
+}
+
+size_t zeta_bytes_max(int64_t n, const int32_t* dims, int n_layers)
+{
+    size_t m = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const size_t b = (size_t)n * (size_t)zeta_ld(dims[l + 1], kZetaF32) * 4;   // fp32 is the widest form
+        if (b > m) m = b;
+    }
+    return m;
+}
+
+void finish_call(bigcn_ctx* ctx)
+{
+    ctx->launches += ctx->launches_i;
+    ctx->launches_i = 0;
+}
+
+bigcn_status forward_impl(bigcn_ctx* ctx, const bigcn_graph* graph, const bigcn_layer* layers,
+                          int32_t n_layers, const float* X, int64_t ldx, const uint32_t* x_bits,
+                          const float* x_beta, float* logits_out, int64_t ldo, bigcn_stats* stats,
+                          Carver& ws)
+{
+    const int64_t n = graph->n;
+    int32_t dims[BIGCN_MAX_LAYERS + 1];
+    dims[0] = layers[0].d_in;
+    for (int l = 0; l < n_layers; ++l) dims[l + 1] = layers[l].d_out;
+    int64_t stride_max = 0;
+    for (int l = 0; l < n_layers; ++l) stride_max = stride_max > bigcn_packed_stride_words(dims[l]) ? stride_max : bigcn_packed_stride_words(dims[l]);
+    void* zeta = ws.take(zeta_bytes_max(n, dims, n_layers));
+    uint32_t* bits[2];
+    float* beta[2];
+    for (int i = 0; i < 2; ++i) {
+        bits[i] = static_cast<uint32_t*>(ws.take((size_t)n * stride_max * 4));
+        beta[i] = static_cast<float*>(ws.take((size_t)n * 4));
+    }
+    if (!zeta || !bits[0] || !beta[0] || !bits[1] || !beta[1])
+        return fail(ctx, BIGCN_ERR_WORKSPACE, "workspace of %zu bytes is too small (see bigcn_workspace_bytes)", ws.size);
+
+    cudaEvent_t* ev = ctx->ev;
+    if (stats) BIGCN_CUDA(ctx, cudaEventRecord(ev[0], ctx->stream));
+    const uint32_t* cur_bits = x_bits;
+    const float* cur_beta = x_beta;
+    if (X) {
+        cudaError_t e = launch_pack_rows(ctx->stream, X, n, dims[0], ldx, layers[0].in_shift, layers[0].in_scale,
+                                         bits[0], bigcn_packed_stride_words(dims[0]), beta[0], &ctx->launches_i);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "pack launch");
+        cur_bits = bits[0];
+        cur_beta = beta[0];
+    }
+    if (stats) BIGCN_CUDA(ctx, cudaEventRecord(ev[1], ctx->stream));
+    for (int l = 0; l < n_layers; ++l) {
+        const bool last = (l == n_layers - 1);
+        const int o = (l + 1) & 1;
+        bigcn_status st = run_layer(ctx, graph, &layers[l], cur_bits, cur_beta, zeta,
+                                    last ? logits_out : nullptr, ldo, last ? nullptr : &layers[l + 1],
+                                    bits[o], beta[o], nullptr, nullptr, stats ? ev[2 + 2 * l] : nullptr);
+        if (st != BIGCN_OK) return st;
+        if (stats) BIGCN_CUDA(ctx, cudaEventRecord(ev[3 + 2 * l], ctx->stream));
+        cur_bits = bits[o];
+        cur_beta = beta[o];
+    }
+    if (stats) {
+        BIGCN_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+        memset(stats, 0, sizeof(*stats));
+        stats->n_layers = n_layers;
+        stats->launches = ctx->launches_i;
+        cudaEventElapsedTime(&stats->ms_pack, ev[0], ev[1]);
+        for (int l = 0; l < n_layers; ++l) {
+            cudaEventElapsedTime(&stats->ms_gemm[l], ev[1 + 2 * l], ev[2 + 2 * l]);
+            cudaEventElapsedTime(&stats->ms_spmm[l], ev[2 + 2 * l], ev[3 + 2 * l]);
+        }
+        cudaEventElapsedTime(&stats->ms_total, ev[0], ev[1 + 2 * n_layers]);
+    }
+    return BIGCN_OK;
+}
+
+bigcn_status check_forward(bigcn_ctx* ctx, const bigcn_graph* graph, const bigcn_layer* layers,
+                           int32_t n_layers, const void* logits, int64_t ldo)
+{
+    bigcn_status st = check_graph(ctx, graph);
+    if (st != BIGCN_OK) return st;
+    if (!layers) return fail(ctx, BIGCN_ERR_NULL, "layers is null");
+    if (n_layers < 1 || n_layers > BIGCN_MAX_LAYERS) return fail(ctx, BIGCN_ERR_SHAPE, "n_layers=%d not in [1, %d]", n_layers, BIGCN_MAX_LAYERS);
+    for (int l = 0; l < n_layers; ++l) {
+        if ((st = check_layer(ctx, &layers[l], "layer")) != BIGCN_OK) return st;
+        if (l > 0 && layers[l].d_in != layers[l - 1].d_out)
+            return fail(ctx, BIGCN_ERR_SHAPE, "layer %d: d_in=%d does not match the previous d_out=%d", l, layers[l].d_in, layers[l - 1].d_out);
+    }
+    if (graph->n > 0 && !logits) return fail(ctx, BIGCN_ERR_NULL, "logits output is null");
+    if (ldo < layers[n_layers - 1].d_out) return fail(ctx, BIGCN_ERR_SHAPE, "ldo=%lld < classes=%d", (long long)ldo, layers[n_layers - 1].d_out);
+    if (graph->n > 0 && !ctx->ws) return fail(ctx, BIGCN_ERR_WORKSPACE, "no workspace attached");
+    return BIGCN_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------
+
+extern "C" {
+
+const char* bigcn_status_string(bigcn_status s)
+{
+    switch (s) {
+        case BIGCN_OK: return "ok";
+        case BIGCN_ERR_NULL: return "null pointer";
+        case BIGCN_ERR_SHAPE: return "bad shape";
+        case BIGCN_ERR_ALIGN: return "misaligned pointer";
+        case BIGCN_ERR_GRAPH: return "malformed graph";
+        case BIGCN_ERR_WORKSPACE: return "workspace missing or too small";
+        case BIGCN_ERR_CUDA: return "CUDA error";
+        case BIGCN_ERR_UNSUPPORTED: return "unsupported";
+        case BIGCN_ERR_INTERNAL: return "device self-check failed";
+    }
+    return "unknown status";
+}
+
+bigcn_status bigcn_create(bigcn_ctx** out, int device, void* cuda_stream)
+{
+    if (!out) return BIGCN_ERR_NULL;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || count == 0 || device < 0 || device >= count) {
+        cudaGetLastError();
+        return BIGCN_ERR_CUDA;          // no CUDA device: there is no CPU fallback
+    }
+    if (cudaSetDevice(device) != cudaSuccess) return BIGCN_ERR_CUDA;
+    bigcn_ctx* ctx = new (std::nothrow) bigcn_ctx();
+    if (!ctx) return BIGCN_ERR_INTERNAL;
+    memset(ctx, 0, sizeof(*ctx));
+    ctx->device = device;
+    ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMalloc(reinterpret_cast<void**>(&ctx->d_flag), 256) != cudaSuccess ||
+        cudaMemset(ctx->d_flag, 0, 256) != cudaSuccess) {
+        delete ctx;
+        return BIGCN_ERR_CUDA;
+    }
+    for (auto& e : ctx->ev)
+        if (cudaEventCreate(&e) != cudaSuccess) { bigcn_destroy(ctx); return BIGCN_ERR_CUDA; }
+    ctx->ev_ready = true;
+    *out = ctx;
+    return BIGCN_OK;
+}
+
+bigcn_status bigcn_destroy(bigcn_ctx* ctx)
+{
+    if (!ctx) return BIGCN_OK;
+    cudaSetDevice(ctx->device);
+    for (auto& e : ctx->ev)
+        if (e) cudaEventDestroy(e);
+    if (ctx->d_flag) cudaFree(ctx->d_flag);
+    delete ctx;
+    return BIGCN_OK;
+}
+
+const char* bigcn_last_error(const bigcn_ctx* ctx) { return ctx ? ctx->err : "context is null"; }
+
+bigcn_status bigcn_set_option(bigcn_ctx* ctx, int32_t option, int64_t value)
+{
+    if (!ctx) return BIGCN_ERR_NULL;
+    switch (option) {
+        case BIGCN_OPT_ZETA_FORMAT:
+            if (value < 0 || value > 3) return fail(ctx, BIGCN_ERR_SHAPE, "zeta format %lld not in [0, 3]", (long long)value);
+            ctx->zeta_format = (int)value;
+            return BIGCN_OK;
+        case BIGCN_OPT_LONG_ROW:
+            if (value < 0) return fail(ctx, BIGCN_ERR_SHAPE, "long-row threshold must be >= 0");
+            ctx->long_row = value;
+            return BIGCN_OK;
+    }
+    return fail(ctx, BIGCN_ERR_UNSUPPORTED, "unknown option %d", option);
+}
+
+int64_t bigcn_launch_count(const bigcn_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+bigcn_status bigcn_sync_check(bigcn_ctx* ctx)
+{
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    BIGCN_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    BIGCN_CUDA(ctx, cudaGetLastError());
+    return BIGCN_OK;
+}
+
+int64_t bigcn_packed_stride_words(int32_t len)
+{
+    if (len < 0) return 0;
+    return round_up(ceil_div(len, 32), 4);
+}
+
+size_t bigcn_workspace_bytes(int64_t n, int64_t nnz, const int32_t* dims, int32_t n_layers, int32_t host_io)
+{
+    (void)nnz;
+    if (n < 0 || !dims || n_layers < 1 || n_layers > BIGCN_MAX_LAYERS) return 0;
+    int64_t stride_max = 0;
+    int32_t d_max = 0;
+    for (int l = 0; l <= n_layers; ++l) {
+        if (dims[l] < 1) return 0;
+        if (l < n_layers && bigcn_packed_stride_words(dims[l]) > stride_max) stride_max = bigcn_packed_stride_words(dims[l]);
+        if (dims[l] > d_max) d_max = dims[l];
+    }
+    size_t total = up(zeta_bytes_max(n, dims, n_layers));
+    total += 2 * (up((size_t)n * stride_max * 4) + up((size_t)n * 4));
+    size_t aux = up(normalize_scratch_bytes(n));
+    if (up(col_stats_scratch_bytes(d_max)) > aux) aux = up(col_stats_scratch_bytes(d_max));
+    if (host_io) {
+        total += up((size_t)n * dims[0] * 4) + up((size_t)n * dims[n_layers] * 4);
+    }
+    if (aux > total) total = aux;
+    return total + kAlign;
+}
+
+bigcn_status bigcn_set_workspace(bigcn_ctx* ctx, void* workspace, size_t bytes)
+{
+    if (!ctx) return BIGCN_ERR_NULL;
+    if (workspace && !aligned(workspace, kAlign)) return fail(ctx, BIGCN_ERR_ALIGN, "workspace must be 256-byte aligned");
+    ctx->ws = workspace;
+    ctx->ws_bytes = workspace ? bytes : 0;
+    return BIGCN_OK;
+}
+
+bigcn_status bigcn_normalize_adjacency(bigcn_ctx* ctx, int64_t n, int64_t nnz_in,
+                                       const int64_t* rowptr_A, const int32_t* colidx_A,
+                                       int64_t* rowptr, int32_t* colidx, float* val, float* dinv,
+                                       int64_t* nnz_out)
+{
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    if (n < 0 || n >= (int64_t(1) << 31) || nnz_in < 0) return fail(ctx, BIGCN_ERR_SHAPE, "n=%lld nnz_in=%lld out of range", (long long)n, (long long)nnz_in);
+    if (!nnz_out) return fail(ctx, BIGCN_ERR_NULL, "nnz_out is null");
+    if (!rowptr) return fail(ctx, BIGCN_ERR_NULL, "rowptr output is null");
+    *nnz_out = 0;
+    if (n == 0) {
+        BIGCN_CUDA(ctx, cudaMemsetAsync(rowptr, 0, sizeof(int64_t), ctx->stream));
+        BIGCN_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+        return BIGCN_OK;
+    }
+    if (!rowptr_A || (nnz_in > 0 && !colidx_A) || !colidx || !val || !dinv) return fail(ctx, BIGCN_ERR_NULL, "an input or output array is null");
+    if (!ctx->ws || ctx->ws_bytes < normalize_scratch_bytes(n)) return fail(ctx, BIGCN_ERR_WORKSPACE, "needs %zu bytes of workspace", normalize_scratch_bytes(n));
+    cudaError_t e = launch_normalize_adjacency(ctx->stream, n, nnz_in, rowptr_A, colidx_A, rowptr, colidx, val, dinv,
+                                               ctx->ws, ctx->d_flag, &ctx->launches_i);
+    finish_call(ctx);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "normalize_adjacency launch");
+    int flag = 0;
+    int64_t total = 0;
+    BIGCN_CUDA(ctx, cudaMemcpyAsync(&flag, ctx->d_flag, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+    BIGCN_CUDA(ctx, cudaMemcpyAsync(&total, rowptr + n, sizeof(int64_t), cudaMemcpyDeviceToHost, ctx->stream));
+    BIGCN_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (flag)
+        return fail(ctx, BIGCN_ERR_GRAPH, "adjacency input rejected:%s%s%s%s",
+                    (flag & 8) ? " rowptr not monotone from 0 to nnz;" : "",
+                    (flag & 2) ? " column index outside [0, n);" : "",
+                    (flag & 1) ? " columns not ascending and unique within a row;" : "",
+                    (flag & 4) ? " pattern not symmetric;" : "");
+    *nnz_out = total;
+    return BIGCN_OK;
+}
+
+bigcn_status bigcn_pack_features(bigcn_ctx* ctx, const float* H, int64_t n, int32_t d, int64_t ld,
+                                 const float* col_shift, const float* col_scale,
+                                 uint32_t* bits_out, int64_t stride_words, float* beta_out)
+{
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    if (n < 0 || d < 1 || ld < d) return fail(ctx, BIGCN_ERR_SHAPE, "n=%lld d=%d ld=%lld", (long long)n, d, (long long)ld);
+    if (stride_words < bigcn_packed_stride_words(d) || stride_words % 4 != 0)
+        return fail(ctx, BIGCN_ERR_SHAPE, "stride_words=%lld must be a multiple of 4 and >= %lld", (long long)stride_words, (long long)bigcn_packed_stride_words(d));
+    if ((col_shift == nullptr) != (col_scale == nullptr)) return fail(ctx, BIGCN_ERR_NULL, "col_shift and col_scale go together");
+    if (n == 0) return BIGCN_OK;
+    if (!H || !bits_out || !beta_out) return fail(ctx, BIGCN_ERR_NULL, "H, bits_out or beta_out is null");
+    if (!aligned(bits_out, 16)) return fail(ctx, BIGCN_ERR_ALIGN, "bits_out must be 16-byte aligned");
+    cudaError_t e = launch_pack_rows(ctx->stream, H, n, d, ld, col_shift, col_scale, bits_out, stride_words, beta_out, &ctx->launches_i);
+    finish_call(ctx);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "pack_features launch");
+    return BIGCN_OK;
+}
+
+bigcn_status bigcn_pack_weights(bigcn_ctx* ctx, const float* W, int32_t d_in, int32_t d_out, int64_t ldw,
+                                uint32_t* bitsT_out, int64_t stride_words, float* alpha_out)
+{
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    if (d_in < 1 || d_out < 1 || ldw < d_out) return fail(ctx, BIGCN_ERR_SHAPE, "d_in=%d d_out=%d ldw=%lld", d_in, d_out, (long long)ldw);
+    if (stride_words < bigcn_packed_stride_words(d_in) || stride_words % 4 != 0 || stride_words > 65535)
+        return fail(ctx, BIGCN_ERR_SHAPE, "stride_words=%lld must be a multiple of 4 in [%lld, 65535]", (long long)stride_words, (long long)bigcn_packed_stride_words(d_in));
+    if (!W || !bitsT_out || !alpha_out) return fail(ctx, BIGCN_ERR_NULL, "W, bitsT_out or alpha_out is null");
+    if (!aligned(bitsT_out, 16)) return fail(ctx, BIGCN_ERR_ALIGN, "bitsT_out must be 16-byte aligned");
+    cudaError_t e = launch_pack_weights(ctx->stream, W, d_in, d_out, ldw, bitsT_out, stride_words, alpha_out, &ctx->launches_i);
+    finish_call(ctx);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "pack_weights launch");
+    return BIGCN_OK;
+}
+
+bigcn_status bigcn_layer_forward(bigcn_ctx* ctx, const bigcn_graph* graph, const bigcn_layer* layer,
+                                 const uint32_t* in_bits, const float* in_beta,
+                                 float* h_out, int64_t ldh,
+                                 const bigcn_layer* next, uint32_t* next_bits, float* next_beta,
+                                 int32_t* dbg_dot, float* dbg_zeta)
+{
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    if ((st = check_graph(ctx, graph)) != BIGCN_OK) return st;
+    if ((st = check_layer(ctx, layer, "layer")) != BIGCN_OK) return st;
+    if (next) {
+        if (next->d_in != layer->d_out) return fail(ctx, BIGCN_ERR_SHAPE, "next->d_in=%d != layer->d_out=%d", next->d_in, layer->d_out);
+        if ((next->in_shift == nullptr) != (next->in_scale == nullptr)) return fail(ctx, BIGCN_ERR_NULL, "next: in_shift and in_scale go together");
+    }
+    if (h_out && ldh < layer->d_out) return fail(ctx, BIGCN_ERR_SHAPE, "ldh=%lld < d_out=%d", (long long)ldh, layer->d_out);
+    if (graph->n == 0) return BIGCN_OK;
+    if (!in_bits || !in_beta) return fail(ctx, BIGCN_ERR_NULL, "in_bits or in_beta is null");
+    if (!aligned(in_bits, 16)) return fail(ctx, BIGCN_ERR_ALIGN, "in_bits must be 16-byte aligned");
+    if (next && (!next_bits || !next_beta)) return fail(ctx, BIGCN_ERR_NULL, "next_bits or next_beta is null");
+    if (!h_out && !next) return fail(ctx, BIGCN_ERR_NULL, "neither h_out nor next is given: nothing to compute");
+    const int32_t dims[2] = {layer->d_in, layer->d_out};
+    const size_t need = up(zeta_bytes_max(graph->n, dims, 1));
+    if (!ctx->ws || ctx->ws_bytes < need) return fail(ctx, BIGCN_ERR_WORKSPACE, "needs %zu bytes of workspace, has %zu", need, ctx->ws_bytes);
+    st = run_layer(ctx, graph, layer, in_bits, in_beta, ctx->ws, h_out, ldh, next, next_bits, next_beta,
+                   dbg_dot, dbg_zeta, nullptr);
+    finish_call(ctx);
+    return st;
+}
+
+bigcn_status bigcn_forward(bigcn_ctx* ctx, const bigcn_graph* graph, const bigcn_layer* layers,
+                           int32_t n_layers, const float* X, int64_t ldx,
+                           float* logits_out, int64_t ldo, bigcn_stats* stats)
+{
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    if ((st = check_forward(ctx, graph, layers, n_layers, logits_out, ldo)) != BIGCN_OK) return st;
+    if (ldx < layers[0].d_in) return fail(ctx, BIGCN_ERR_SHAPE, "ldx=%lld < d_0=%d", (long long)ldx, layers[0].d_in);
+    if (graph->n == 0) return BIGCN_OK;
+    if (!X) return fail(ctx, BIGCN_ERR_NULL, "X is null");
+    Carver ws{static_cast<char*>(ctx->ws), ctx->ws_bytes, 0};
+    st = forward_impl(ctx, graph, layers, n_layers, X, ldx, nullptr, nullptr, logits_out, ldo, stats, ws);
+    finish_call(ctx);
+    return st;
+}
+
+bigcn_status bigcn_forward_packed(bigcn_ctx* ctx, const bigcn_graph* graph, const bigcn_layer* layers,
+                                  int32_t n_layers, const uint32_t* x_bits, const float* x_beta,
+                                  float* logits_out, int64_t ldo, bigcn_stats* stats)
+{
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    if ((st = check_forward(ctx, graph, layers, n_layers, logits_out, ldo)) != BIGCN_OK) return st;
+    if (graph->n == 0) return BIGCN_OK;
+    if (!x_bits || !x_beta) return fail(ctx, BIGCN_ERR_NULL, "x_bits or x_beta is null");
+    if (!aligned(x_bits, 16)) return fail(ctx, BIGCN_ERR_ALIGN, "x_bits must be 16-byte aligned");
+    Carver ws{static_cast<char*>(ctx->ws), ctx->ws_bytes, 0};
+    st = forward_impl(ctx, graph, layers, n_layers, nullptr, 0, x_bits, x_beta, logits_out, ldo, stats, ws);
+    finish_call(ctx);
+    return st;
+}
+
+bigcn_status bigcn_forward_host(bigcn_ctx* ctx, const bigcn_graph* graph, const bigcn_layer* layers,
+                                int32_t n_layers, const float* X_host, int64_t ldx,
+                                float* logits_host, int64_t ldo)
+{
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    if ((st = check_forward(ctx, graph, layers, n_layers, logits_host, ldo)) != BIGCN_OK) return st;
+    const int32_t d0 = layers[0].d_in, classes = layers[n_layers - 1].d_out;
+    if (ldx != d0 || ldo != classes) return fail(ctx, BIGCN_ERR_SHAPE, "host buffers must be dense: ldx=%lld (d_0=%d), ldo=%lld (classes=%d)", (long long)ldx, d0, (long long)ldo, classes);
+    const int64_t n = graph->n;
+    if (n == 0) return BIGCN_OK;
+    if (!X_host) return fail(ctx, BIGCN_ERR_NULL, "X_host is null");
+    Carver ws{static_cast<char*>(ctx->ws), ctx->ws_bytes, 0};
+    float* x_dev = static_cast<float*>(ws.take((size_t)n * d0 * 4));
+    float* out_dev = static_cast<float*>(ws.take((size_t)n * classes * 4));
+    if (!x_dev || !out_dev) return fail(ctx, BIGCN_ERR_WORKSPACE, "workspace too small for the host staging buffers (size it with host_io = 1)");
+    BIGCN_CUDA(ctx, cudaMemcpyAsync(x_dev, X_host, (size_t)n * d0 * 4, cudaMemcpyHostToDevice, ctx->stream));
+    st = forward_impl(ctx, graph, layers, n_layers, x_dev, d0, nullptr, nullptr, out_dev, classes, nullptr, ws);
+    finish_call(ctx);
+    if (st != BIGCN_OK) return st;
+    BIGCN_CUDA(ctx, cudaMemcpyAsync(logits_host, out_dev, (size_t)n * classes * 4, cudaMemcpyDeviceToHost, ctx->stream));
+    BIGCN_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return BIGCN_OK;
+}
+
+bigcn_status bigcn_col_stats(bigcn_ctx* ctx, const float* H, int64_t n, int32_t d, int64_t ld,
+                             float eps, float* shift_out, float* scale_out)
+{
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    if (n < 0 || d < 1 || ld < d || !(eps >= 0.f)) return fail(ctx, BIGCN_ERR_SHAPE, "n=%lld d=%d ld=%lld eps=%g", (long long)n, d, (long long)ld, (double)eps);
+    if (!shift_out || !scale_out || (n > 0 && !H)) return fail(ctx, BIGCN_ERR_NULL, "H, shift_out or scale_out is null");
+    if (!ctx->ws || ctx->ws_bytes < col_stats_scratch_bytes(d)) return fail(ctx, BIGCN_ERR_WORKSPACE, "needs %zu bytes of workspace", col_stats_scratch_bytes(d));
+    cudaError_t e = launch_col_stats(ctx->stream, H, n, d, ld, eps, shift_out, scale_out, ctx->ws, &ctx->launches_i);
+    finish_call(ctx);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "col_stats launch");
+    return BIGCN_OK;
+}
+
+}  // extern "C"

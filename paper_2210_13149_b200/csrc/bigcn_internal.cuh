@@ -1,0 +1,76 @@
+// Internal declarations shared by the translation units of libbigcn (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "bigcn.h"
+
+namespace bigcn {
+
+constexpr int kWarp = 32;
+
+// Storage of the contraction result between the bit-GEMM and the aggregation.
+enum ZetaFormat : int { kZetaF32 = 1, kZetaI16 = 2, kZetaI8 = 3 };
+
+inline __host__ __device__ int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline __host__ __device__ int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
+
+// Elements per row of the zeta buffer: d_out rounded up so that a row is a whole number of 16-byte vectors.
+inline int64_t zeta_ld(int d_out, int fmt)
+{
+    const int per16 = fmt == kZetaF32 ? 4 : (fmt == kZetaI16 ? 8 : 16);
+    return round_up(d_out, per16);
+}
+inline int zeta_elt_bytes(int fmt) { return fmt == kZetaF32 ? 4 : (fmt == kZetaI16 ? 2 : 1); }
+
+// ---- launchers (each returns the launch status; all asynchronous on `s`) ------------------------
+
+cudaError_t launch_pack_rows(cudaStream_t s, const float* H, int64_t n, int d, int64_t ld,
+                             const float* shift, const float* scale,
+                             uint32_t* bits, int64_t stride, float* beta, int* launches);
+
+cudaError_t launch_pack_weights(cudaStream_t s, const float* W, int d_in, int d_out, int64_t ldw,
+                                uint32_t* bitsT, int64_t stride, float* alpha, int* launches);
+
+cudaError_t launch_bitgemm(cudaStream_t s, const uint32_t* A, int64_t stride_a,
+                           const uint32_t* BT, int64_t stride_b, int64_t n, int d_in, int d_out,
+                           const float* beta, const float* alpha, int fmt, void* zeta, int64_t ldz,
+                           int32_t* dbg_dot, float* dbg_zeta, int* launches);
+
+struct SpmmArgs {
+    int64_t n;
+    const int64_t* rowptr;
+    const int32_t* colidx;
+    const float* val;
+    int fmt;                 // ZetaFormat of `zeta`
+    const void* zeta;        // [n x ldz] of float / int16 / int8
+    int64_t ldz;
+    int d_out;
+    const float* node_w;     // integer formats: per-source-node factor (beta), multiplied into the edge weight
+    const float* col_w;      // integer formats: per-column factor (alpha), applied once per output
+    float* h_out;            // nullable
+    int64_t ldh;
+    uint32_t* next_bits;     // nullable: fused re-binarization of the output
+    int64_t next_stride;
+    float* next_beta;
+    const float* next_shift; // nullable
+    const float* next_scale;
+    int64_t long_row;        // rows with more entries are split (0 = never)
+    void* scratch;           // partial sums of split rows
+    size_t scratch_bytes;
+};
+cudaError_t launch_spmm(cudaStream_t s, const SpmmArgs& a, int* launches);
+size_t spmm_scratch_bytes(int64_t n, int64_t nnz, int d_out);
+
+cudaError_t launch_normalize_adjacency(cudaStream_t s, int64_t n, int64_t nnz_in,
+                                       const int64_t* rowptr_A, const int32_t* colidx_A,
+                                       int64_t* rowptr, int32_t* colidx, float* val, float* dinv,
+                                       void* scratch, int* d_flag, int* launches);
+size_t normalize_scratch_bytes(int64_t n);
+
+cudaError_t launch_col_stats(cudaStream_t s, const float* H, int64_t n, int d, int64_t ld, float eps,
+                             float* shift, float* scale, void* scratch, int* launches);
+size_t col_stats_scratch_bytes(int d);
+
+}  // namespace bigcn
