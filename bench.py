@@ -1,0 +1,366 @@
+#!/usr/bin/env python
+"""Benchmark of the Bi-GCN binarized forward path: nodes/s of a full L-layer forward on one B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c5] [--impl ours|reference]
+
+A step is one pass of the whole hot path (binarize+pack of the fp32 features, then per layer the
+XNOR/bit-count contraction with rescale and the CSR aggregation with fused re-binarization) over one
+seeded synthetic graph.  With N > 1 every rank runs an independent replica on its own GPU (the path
+has no exchange step); the reported value is the sum over replicas divided by the slowest rank's time.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "bigcn_forward_nodes_per_s"
+UNIT = "nodes/s"
+DTYPE = "u32-xor-popc+f32"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="c5", help="workload c1..c5 (default: the largest, c5)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--zeta-format", type=int, default=0, help="0 auto, 1 fp32, 2 int16, 3 int8")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--cpu-sample-scale", type=float, default=None)
+    return ap.parse_args()
+
+
+def workload_description(spec, n, nnz):
+    return ("%s: %d-layer Bi-GCN forward, synthetic power-law graph, %d nodes, %d stored entries of A_tilde, "
+            "widths %s, %s features" % (spec.name, len(spec.dims) - 1, n, nnz, "-".join(str(d) for d in spec.dims),
+                                        spec.features))
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            with open(path) as f:
+                p = json.load(f)
+            return float(p["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1]))
+                    mx.append(float(parts[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(names, parts[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------------- oracle arm
+
+def time_oracle(spec_name: str, scale: float, steps: int, warmup: int):
+    """Times the CPU oracle, as it stands, on a scaled-down draw of the workload (same recipe, same
+    widths and mean degree).  Returns (nodes/s, threads, sample description, ms per step)."""
+    import oracle
+    from paper_2210_13149_b200 import synth
+    wl = synth.make_workload(spec_name, scale=scale if scale < 1.0 else None, device="cpu")
+    src, dst = synth.edge_list(wl.rowptr, wl.colidx)
+    g = oracle.normalize_adjacency(wl.n, src, dst)
+    X = wl.X.numpy()
+    layers = oracle.calibrate_bn(g, [w.numpy() for w in wl.W], X, wl.bn_layers())
+    times = []
+    for it in range(warmup + steps):
+        t0 = time.perf_counter()
+        oracle.forward(g, layers, X, keep_trace=False)
+        t1 = time.perf_counter()
+        if it >= warmup:
+            times.append(t1 - t0)
+    ms = 1e3 * sum(times) / len(times)
+    sample = ("%s recipe at %g of its nodes and edges (%d nodes, %d stored entries, same widths and mean degree): "
+              "full %d-layer oracle forward, set-up excluded" % (spec_name, scale, wl.n, g.nnz, len(layers)))
+    return wl.n / (ms * 1e-3), oracle.num_threads(), sample, ms
+
+
+def default_cpu_scale(spec) -> float:
+    # roughly 1e10 multiply-adds of aggregation per oracle forward keeps a run at a few seconds
+    work = sum(spec.e_dir * d for d in spec.dims[1:]) + sum(spec.n * a * b / 32 for a, b in zip(spec.dims[:-1], spec.dims[1:]))
+    return min(1.0, 6e9 / max(work, 1.0))
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2210_13149_b200 import synth
+    spec = synth.WORKLOADS[args.config]
+    scale = args.cpu_sample_scale or default_cpu_scale(spec)
+    value, threads, sample, ms = time_oracle(args.config, scale, args.steps, args.warmup)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64-accumulate (CPU oracle)", "data": "synthetic",
+            "config": {"workload": "CPU oracle on a sample of " + args.config, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------------- our arm
+
+def spmm_bytes_model(n, nnz, d_out, row_bytes, out_bytes, l2_bytes=126e6):
+    """Algorithmic HBM bytes of one aggregation launch: the CSR stream, the per-node vectors, the
+    output, and the gathered operand rows.  Lower bound: every operand row once.  No-reuse bound:
+    one row per stored entry.  Expected: rows are re-read from HBM except for the share of the
+    operand matrix the L2 can hold (node ids carry no locality)."""
+    fixed = nnz * 8.0 + 8.0 * (n + 1) + 4.0 * n + out_bytes
+    z = n * row_bytes
+    lower = fixed + z
+    upper = fixed + nnz * row_bytes
+    miss = max(0.0, 1.0 - l2_bytes / z) if z > 0 else 0.0
+    expected = fixed + z + max(0.0, (nnz - n)) * row_bytes * miss
+    return lower, upper, expected
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2210_13149_b200 import binding, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+
+    spec = synth.WORKLOADS[args.config]
+    wl = synth.make_workload(args.config, device=dev)
+    ctx = binding.BiGCN(local)
+    if args.zeta_format:
+        ctx.set_option(binding.OPT_ZETA_FORMAT, args.zeta_format)
+    G = ctx.normalize_adjacency(wl.rowptr, wl.colidx)
+    n, nnz = G.n, G.nnz
+    del wl.rowptr, wl.colidx
+    dims = list(spec.dims)
+    L = len(dims) - 1
+
+    # Set-up (untimed): pack the weights; freeze the batch-norm constants of every layer input that
+    # has them from the library's own column statistics, layer after layer.
+    bn = wl.bn_layers()
+    packed = [ctx.pack_weights(W) for W in wl.W]
+    layers, shifts, scales = [], [], []
+    bits = beta = None
+    for l in range(L):
+        if l == 0:
+            sh, sc = ctx.col_stats(wl.X) if bn[0] else (None, None)
+            bits, beta = ctx.pack_features(wl.X, sh, sc)
+        else:
+            prev = layers[-1]
+            out = ctx.layer_forward(G, prev, bits, beta, want_h=True)
+            sh, sc = ctx.col_stats(out["h"]) if bn[l] else (None, None)
+            bits, beta = ctx.pack_features(out["h"], sh, sc)
+            del out
+        layers.append(binding.make_layer(dims[l], dims[l + 1], packed[l][0], packed[l][1], sh, sc))
+    del bits, beta
+    ctx.workspace = None
+    torch.cuda.empty_cache()
+
+    X = wl.X
+    logits = torch.empty((n, dims[-1]), dtype=torch.float32, device=dev)
+    ctx._prep_forward(G, layers, host_io=not args.no_e2e)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        ctx.forward(G, layers, X, logits)
+    barrier()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    launches0 = ctx.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    per_kernel = {"pack": [], "gemm": [[] for _ in range(L)], "spmm": [[] for _ in range(L)]}
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        _, st = ctx.forward(G, layers, X, logits, stats=True)
+        per_kernel["pack"].append(st.ms_pack)
+        for l in range(L):
+            per_kernel["gemm"][l].append(st.ms_gemm[l])
+            per_kernel["spmm"][l].append(st.ms_spmm[l])
+    ev1.record()
+    barrier()
+    elapsed_ms = ev0.elapsed_time(ev1)
+    launches = ctx.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    if world > 1:
+        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / args.steps
+    value = world * n / (ms_per_step * 1e-3)
+
+    # end to end through the host-buffer entry point: pinned X in, logits out, every step
+    e2e = None
+    if not args.no_e2e:
+        xh = torch.empty((n, dims[0]), dtype=torch.float32).pin_memory()
+        xh.copy_(X)
+        oh = torch.empty((n, dims[-1]), dtype=torch.float32).pin_memory()
+        e_steps = max(3, min(args.steps, 10))
+        for _ in range(2):
+            ctx.forward_host(G, layers, xh, oh)
+        barrier()
+        ev0.record()
+        for _ in range(e_steps):
+            ctx.forward_host(G, layers, xh, oh)
+        ev1.record()
+        barrier()
+        e_ms = ev0.elapsed_time(ev1) / e_steps
+        if world > 1:
+            t = torch.tensor([e_ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        e2e = {"value": world * n / (e_ms * 1e-3), "unit": UNIT, "ms_per_step": e_ms, "steps": e_steps,
+               "h2d_bytes_per_step": n * dims[0] * 4, "d2h_bytes_per_step": n * dims[-1] * 4,
+               "api": "bigcn_forward_host (pinned host X in, host logits out)"}
+        del xh, oh
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # roofline of the dominant kernel: the aggregation of the layer that takes longest
+    peak, peak_kind = load_peaks()
+    mean = lambda v: sum(v) / len(v)
+    spmm_ms = [mean(v) for v in per_kernel["spmm"]]
+    gemm_ms = [mean(v) for v in per_kernel["gemm"]]
+    pack_ms = mean(per_kernel["pack"])
+    fmt = args.zeta_format or binding.ZETA_I16
+    kernels = {}
+    dom = max(range(L), key=lambda l: spmm_ms[l])
+    for l in range(L):
+        f = fmt
+        if f == binding.ZETA_I8 and dims[l] > 127:
+            f = binding.ZETA_I16
+        elt = {1: 4, 2: 2, 3: 1}[f]
+        per16 = 16 // elt
+        ldz = (dims[l + 1] + per16 - 1) // per16 * per16
+        last = (l == L - 1)
+        out_bytes = n * dims[l + 1] * 4.0 if last else n * (binding.packed_stride_words(dims[l + 1]) * 4.0 + 4.0)
+        lower, upper, expected = spmm_bytes_model(n, nnz, dims[l + 1], ldz * elt, out_bytes)
+        t = spmm_ms[l] * 1e-3
+        kernels["spmm_l%d" % l] = {"ms": spmm_ms[l], "GBps_expected_model": expected / t / 1e9,
+                                   "GBps_lower_model": lower / t / 1e9, "GBps_no_reuse_model": upper / t / 1e9,
+                                   "bytes_expected": expected, "zeta_format": {1: "f32", 2: "i16", 3: "i8"}[f]}
+        ops = 2.0 * n * dims[l] * dims[l + 1]
+        kernels["bitgemm_l%d" % l] = {"ms": gemm_ms[l], "binary_TOPS": ops / (gemm_ms[l] * 1e-3) / 1e12,
+                                      "out_GBps": n * ldz * elt / (gemm_ms[l] * 1e-3) / 1e9}
+    pack_bytes = n * (dims[0] * 4.0 + binding.packed_stride_words(dims[0]) * 4.0 + 4.0)
+    kernels["pack_features"] = {"ms": pack_ms, "GBps": pack_bytes / (pack_ms * 1e-3) / 1e9,
+                                "frac_of_hbm_peak": pack_bytes / (pack_ms * 1e-3) / 1e9 / peak}
+    achieved = kernels["spmm_l%d" % dom]["GBps_expected_model"]
+    roofline = {"kernel": "spmm_kernel (layer %d: %d -> %d columns)" % (dom, dims[dom], dims[dom + 1]),
+                "bound": "hbm", "achieved": achieved, "peak": peak, "peak_kind": "%s copy bandwidth" % peak_kind,
+                "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                "model": "CSR stream + per-node vectors + output + operand rows re-read per stored entry except the "
+                         "share of the operand matrix that fits the 126 MB L2"}
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        try:
+            scale = args.cpu_sample_scale or default_cpu_scale(spec)
+            v, threads, sample, ms = time_oracle(args.config, scale, 2, 1)
+            cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample, "ms_per_step": ms}
+        except Exception as exc:      # the oracle is optional equipment for the bench
+            cpu = {"value": None, "unit": UNIT, "cores": 0, "kind": "oracle", "sample": "failed: %r" % (exc,)}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": DTYPE, "data": "synthetic",
+            "config": {"workload": workload_description(spec, n, nnz), "l2": "inputs_exceed_l2",
+                       "parallelism": "replicas" if world > 1 else "single-gpu",
+                       "zeta_format": {0: "auto(i16)", 1: "f32", 2: "i16", 3: "i8"}[args.zeta_format]},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
+            "kernels": kernels}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,94 @@
+"""Shared helpers of the GPU parity tests: build a workload, run the CPU oracle on it, move arrays
+to the device.  The oracle side and the CUDA side only meet here, through plain arrays."""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import List, Optional
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2210_13149_b200 import synth
+
+ATOL, RTOL = 1e-4, 1e-5          # |gpu - oracle| <= ATOL + RTOL * |oracle| per fp32 element
+
+
+def dev(a, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if dtype is not None:
+        t = t.to(dtype)
+    return t.cuda()
+
+
+def bits_to_dev(bits_u32: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(bits_u32).view(np.int32)).cuda()
+
+
+def bits_from_dev(t: torch.Tensor) -> np.ndarray:
+    return t.cpu().numpy().view(np.uint32)
+
+
+def within_tol(got: torch.Tensor, ref: torch.Tensor):
+    """Returns (ok, worst ratio of error to allowance, max abs error), computed where `got` lives."""
+    ref = ref.to(got.device)
+    err = (got.double() - ref.double()).abs()
+    allow = ATOL + RTOL * ref.double().abs()
+    ratio = (err / allow).max().item() if err.numel() else 0.0
+    return ratio <= 1.0, ratio, (err.max().item() if err.numel() else 0.0)
+
+
+def assert_close(got: torch.Tensor, ref, what=""):
+    if isinstance(ref, np.ndarray):
+        ref = torch.from_numpy(ref)
+    assert got.shape == ref.shape, (what, got.shape, ref.shape)
+    ok, ratio, mx = within_tol(got, ref)
+    assert ok, "%s: error / allowance = %.3g (max abs err %.3g)" % (what, ratio, mx)
+
+
+@dataclass
+class OracleRun:
+    wl: synth.Workload
+    graph: oracle.Graph
+    layers: List[oracle.Layer]
+    traces: Optional[List[oracle.LayerTrace]]
+    logits: np.ndarray
+
+
+def oracle_run(wl: synth.Workload, keep_trace=True) -> OracleRun:
+    src, dst = synth.edge_list(wl.rowptr, wl.colidx)
+    g = oracle.normalize_adjacency(wl.n, src, dst)
+    X = wl.X.cpu().numpy()
+    W = [w.cpu().numpy() for w in wl.W]
+    layers = oracle.calibrate_bn(g, W, X, wl.bn_layers())
+    logits, traces = oracle.forward(g, layers, X, keep_trace=keep_trace)
+    return OracleRun(wl, g, layers, traces if keep_trace else None, logits)
+
+
+def device_graph(binding, g: oracle.Graph):
+    return binding.make_graph(dev(g.rowptr), dev(g.colidx), dev(g.val), dev(g.dinv))
+
+
+def device_layers_from_oracle(binding, run: OracleRun):
+    """Layers whose packed weights, alpha and batch-norm constants are the oracle's own arrays."""
+    out = []
+    for l, layer in enumerate(run.layers):
+        B, alpha = oracle.binarize_cols(layer.W)
+        bitsT = oracle.pack_cols(B)
+        sh = dev(layer.in_shift) if layer.in_shift is not None else None
+        sc = dev(layer.in_scale) if layer.in_scale is not None else None
+        out.append(binding.make_layer(layer.W.shape[0], layer.W.shape[1], bits_to_dev(bitsT), dev(alpha), sh, sc))
+    return out
+
+
+def flip_report(gpu_bits: np.ndarray, ref_F: np.ndarray, ref_H: np.ndarray, shift: Optional[np.ndarray]):
+    """Compares re-binarized bits with the oracle's signs.  A disagreement is admissible only where
+    the oracle's pre-sign value lies within the fp32 tolerance of the threshold.
+    Returns (flips, inadmissible flips, total)."""
+    d = ref_F.shape[1]
+    got_F = oracle.unpack_rows(gpu_bits, d)
+    diff = got_F != ref_F
+    centred = ref_H.astype(np.float64) - (shift.astype(np.float64)[None, :] if shift is not None else 0.0)
+    near = np.abs(centred) <= ATOL + RTOL * np.abs(ref_H.astype(np.float64))
+    bad = diff & ~near
+    return int(diff.sum()), int(bad.sum()), int(diff.size)

@@ -1,0 +1,364 @@
+"""GPU parity: every step of the CUDA path against the CPU oracle, through the C ABI.
+
+Packed bits and integer dot products must match exactly; fp32 outputs within
+|gpu - oracle| <= 1e-4 + 1e-5 |oracle| when the layer is fed the oracle's own input.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2210_13149_b200 import synth
+from parity_util import (ATOL, RTOL, assert_close, bits_from_dev, bits_to_dev, dev, device_graph,
+                         device_layers_from_oracle, flip_report, oracle_run)
+
+pytestmark = pytest.mark.gpu
+
+FORMATS = [1, 2, 3]          # fp32 zeta, int16 dots, int8 dots (falls back to int16 when d_in > 127)
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2210_13149_b200 import binding
+    return binding
+
+
+@pytest.fixture()
+def ctx(B):
+    c = B.BiGCN(0)
+    yield c
+    c.sync_check()
+    c.close()
+
+
+def small_graph(n, e_dir, seed):
+    rp, ci = synth.power_law_graph(n, e_dir, seed)
+    src, dst = synth.edge_list(rp, ci)
+    return rp, ci, oracle.normalize_adjacency(n, src, dst)
+
+
+# --------------------------------------------------------------------------- set-up step
+
+@pytest.mark.parametrize("n,e,seed", [(1, 0, 1), (7, 0, 2), (50, 200, 3), (2708, 10556, 1001), (5000, 400000, 5)])
+def test_normalize_adjacency_is_bit_exact(ctx, n, e, seed):
+    rp, ci, g = small_graph(n, e, seed)
+    got = ctx.normalize_adjacency(rp.cuda(), ci.cuda())
+    assert got.nnz == g.nnz
+    assert np.array_equal(got.rowptr.cpu().numpy(), g.rowptr)
+    assert np.array_equal(got.colidx.cpu().numpy(), g.colidx)
+    assert np.array_equal(got.dinv.cpu().numpy(), g.dinv)
+    assert np.array_equal(got.val.cpu().numpy(), g.val)
+
+
+def test_normalize_adjacency_drops_input_diagonal(ctx):
+    # path 0-1-2 with self-loops already present on 0 and 2
+    rp = torch.tensor([0, 2, 4, 6], dtype=torch.int64)
+    ci = torch.tensor([0, 1, 0, 2, 1, 2], dtype=torch.int32)
+    g = oracle.normalize_adjacency(3, np.array([0, 1], np.int32), np.array([1, 2], np.int32))
+    got = ctx.normalize_adjacency(rp.cuda(), ci.cuda())
+    assert np.array_equal(got.colidx.cpu().numpy(), g.colidx)
+    assert np.array_equal(got.val.cpu().numpy(), g.val)
+
+
+@pytest.mark.parametrize("rp,ci", [
+    ([0, 1, 1], [1]),                 # (0,1) without (1,0)
+    ([0, 2, 3, 4], [2, 1, 0, 0]),     # columns not ascending
+    ([0, 1, 2], [1, 5]),              # column out of range
+    ([0, 2, 1], [1, 0]),              # rowptr not monotone
+])
+def test_normalize_adjacency_rejects_malformed_input(ctx, B, rp, ci):
+    with pytest.raises(B.BigcnError) as e:
+        ctx.normalize_adjacency(torch.tensor(rp, dtype=torch.int64).cuda(), torch.tensor(ci, dtype=torch.int32).cuda())
+    assert e.value.status == 4
+    ctx.sync_check()                  # the context stays usable
+
+
+# --------------------------------------------------------------------------- binarize + pack
+
+@pytest.mark.parametrize("n,d", [(1, 1), (5, 31), (9, 32), (13, 33), (300, 100), (77, 602), (40, 1433), (11, 3703), (1000, 256)])
+@pytest.mark.parametrize("norm", [False, True])
+def test_pack_features(ctx, n, d, norm):
+    rng = np.random.default_rng(n * 7919 + d)
+    H = rng.standard_normal((n, d)).astype(np.float32)
+    H[rng.random((n, d)) < 0.2] = 0.0
+    shift = scale = None
+    if norm:
+        shift, scale = oracle.col_stats(H)
+    F, beta = oracle.binarize_rows(H, shift, scale)
+    bits = oracle.pack_rows(F)
+    gb, gbeta = ctx.pack_features(dev(H), dev(shift) if norm else None, dev(scale) if norm else None)
+    assert np.array_equal(bits_from_dev(gb), bits)
+    np.testing.assert_allclose(gbeta.cpu().numpy(), beta, rtol=2e-6, atol=1e-30)
+
+
+def test_pack_features_strided_input_and_wide_output(ctx):
+    rng = np.random.default_rng(5)
+    n, d, ld = 33, 70, 96
+    buf = rng.standard_normal((n, ld)).astype(np.float32)
+    H = buf[:, :d]
+    F, beta = oracle.binarize_rows(np.ascontiguousarray(H))
+    bits = oracle.pack_rows(F, stride=8)
+    gb, gbeta = ctx.pack_features(dev(buf)[:, :d], stride_words=8)
+    assert np.array_equal(bits_from_dev(gb), bits)
+    np.testing.assert_allclose(gbeta.cpu().numpy(), beta, rtol=2e-6)
+
+
+def test_pack_features_sign_convention(ctx):
+    tiny = np.float32(1e-45)
+    H = np.array([[0.0, -0.0, tiny, -tiny, 1.0, -1.0, np.inf, -np.inf, np.nan]], np.float32)
+    F, _ = oracle.binarize_rows(H)
+    gb, _ = ctx.pack_features(dev(H))
+    assert np.array_equal(bits_from_dev(gb), oracle.pack_rows(F))
+    assert bits_from_dev(gb)[0, 0] == 0b001010111
+
+
+@pytest.mark.parametrize("d_in,d_out", [(1, 1), (33, 7), (100, 256), (602, 256), (1433, 64), (3703, 64), (256, 47), (64, 3)])
+def test_pack_weights(ctx, d_in, d_out):
+    rng = np.random.default_rng(d_in * 31 + d_out)
+    W = (rng.standard_normal((d_in, d_out)) * d_in ** -0.5).astype(np.float32)
+    W[rng.random((d_in, d_out)) < 0.05] = 0.0
+    Bm, alpha = oracle.binarize_cols(W)
+    bitsT = oracle.pack_cols(Bm)
+    gb, ga = ctx.pack_weights(dev(W))
+    assert np.array_equal(bits_from_dev(gb), bitsT)
+    np.testing.assert_allclose(ga.cpu().numpy(), alpha, rtol=1e-6)
+
+
+def test_col_stats(ctx):
+    rng = np.random.default_rng(9)
+    H = (rng.standard_normal((5000, 77)) * 3 + 1.5).astype(np.float32)
+    shift, scale = oracle.col_stats(H)
+    gs, gc = ctx.col_stats(dev(H))
+    np.testing.assert_allclose(gs.cpu().numpy(), shift, rtol=1e-6, atol=1e-7)
+    np.testing.assert_allclose(gc.cpu().numpy(), scale, rtol=1e-6)
+
+
+# --------------------------------------------------------------------------- one layer, oracle-fed
+
+LAYER_SHAPES = [(200, 1500, 1, 1), (300, 2500, 33, 7), (500, 6000, 100, 256), (400, 5000, 602, 256),
+                (350, 3000, 1433, 64), (250, 2000, 3703, 64), (600, 9000, 256, 47), (600, 9000, 256, 41),
+                (700, 5000, 64, 3), (450, 4000, 64, 6), (300, 3000, 256, 256), (260, 3000, 127, 100),
+                (260, 3000, 128, 512)]
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+@pytest.mark.parametrize("n,e,d_in,d_out", LAYER_SHAPES)
+def test_layer_forward_against_oracle(ctx, B, fmt, n, e, d_in, d_out):
+    rng = np.random.default_rng(n + 3 * d_in + 7 * d_out)
+    _, _, g = small_graph(n, e, 100 + n)
+    H = rng.standard_normal((n, d_in)).astype(np.float32)
+    W = (rng.standard_normal((d_in, d_out)) * d_in ** -0.5).astype(np.float32)
+    W2 = rng.standard_normal((d_out, 4)).astype(np.float32)
+    t = oracle.layer_forward(g, oracle.Layer(W), H)
+    nshift, nscale = oracle.col_stats(t.H_out)
+    Fn, beta_n = oracle.binarize_rows(t.H_out, nshift, nscale)
+
+    ctx.set_option(B.OPT_ZETA_FORMAT, fmt)
+    G = device_graph(B, g)
+    layer = B.make_layer(d_in, d_out, bits_to_dev(t.bitsT), dev(t.alpha))
+    nxt = B.make_layer(d_out, 4, bits_to_dev(oracle.pack_cols(oracle.binarize_cols(W2)[0])), dev(np.ones(4, np.float32)),
+                       dev(nshift), dev(nscale))
+    out = ctx.layer_forward(G, layer, bits_to_dev(t.bits), dev(t.beta), want_h=True, next_layer=nxt, debug=True)
+    ctx.sync_check()
+    assert np.array_equal(out["dot"].cpu().numpy(), t.dot)                 # integers: exact
+    assert np.array_equal(out["zeta"].cpu().numpy(), t.zeta)               # same two fp32 products: exact
+    assert_close(out["h"], t.H_out, "H'")
+    flips, bad, total = flip_report(bits_from_dev(out["next_bits"]), Fn, t.H_out, nshift)
+    assert bad == 0, "%d sign flips away from the threshold (of %d flips, %d bits)" % (bad, flips, total)
+    assert flips <= max(2, total // 2000)
+    # pad bits of the re-binarized rows are zero
+    nb = bits_from_dev(out["next_bits"])
+    if d_out % 32:
+        assert (nb[:, d_out // 32] >> (d_out % 32) == 0).all()
+    assert (nb[:, (d_out + 31) // 32:] == 0).all()
+    np.testing.assert_allclose(out["next_beta"].cpu().numpy(), beta_n, rtol=1e-4, atol=1e-5)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_layer_forward_hub_rows_split_across_the_block(ctx, B, fmt):
+    """A star plus a random graph: one row holds n entries.  With a tiny long-row threshold every
+    moderately long row takes the block-cooperative path; results must not change."""
+    n, d_in, d_out = 3000, 100, 256
+    rng = np.random.default_rng(77)
+    rp, ci = synth.power_law_graph(n, 30000, 77)
+    src, dst = synth.edge_list(rp, ci)
+    src = np.concatenate([src, np.zeros(n - 1, np.int32)])
+    dst = np.concatenate([dst, np.arange(1, n, dtype=np.int32)])
+    g = oracle.normalize_adjacency(n, src, dst)
+    assert (np.diff(g.rowptr)).max() == n
+    H = rng.standard_normal((n, d_in)).astype(np.float32)
+    W = (rng.standard_normal((d_in, d_out)) * 0.1).astype(np.float32)
+    t = oracle.layer_forward(g, oracle.Layer(W), H)
+    ctx.set_option(B.OPT_ZETA_FORMAT, fmt)
+    G = device_graph(B, g)
+    layer = B.make_layer(d_in, d_out, bits_to_dev(t.bitsT), dev(t.alpha))
+    outs = []
+    for thr in (0, 8, 100000):       # default threshold, nearly every row long, no row long
+        ctx.set_option(B.OPT_LONG_ROW, thr)
+        out = ctx.layer_forward(G, layer, bits_to_dev(t.bits), dev(t.beta), want_h=True)
+        assert_close(out["h"], t.H_out, "H' (threshold %d)" % thr)
+        outs.append(out["h"].clone())
+    again = ctx.layer_forward(G, layer, bits_to_dev(t.bits), dev(t.beta), want_h=True)["h"]
+    assert torch.equal(again, outs[-1])          # run-to-run deterministic
+
+
+def test_layer_on_pm1_inputs_is_the_gcn_layer(ctx, B):
+    """H, W in {+-1}: the scalars are 1 and the layer is exactly A_tilde (H W) (Eq. 1, no activation)."""
+    rng = np.random.default_rng(21)
+    n, d, c = 300, 45, 5
+    _, _, g = small_graph(n, 2000, 21)
+    H = rng.choice(np.array([-1.0, 1.0], np.float32), size=(n, d))
+    W = rng.choice(np.array([-1.0, 1.0], np.float32), size=(d, c))
+    G = device_graph(B, g)
+    bits, beta = ctx.pack_features(dev(H))
+    bitsT, alpha = ctx.pack_weights(dev(W))
+    assert (beta == 1).all() and (alpha == 1).all()
+    out = ctx.layer_forward(G, B.make_layer(d, c, bitsT, alpha), bits, beta)
+    A = torch.sparse_csr_tensor(dev(g.rowptr), dev(g.colidx).long(), dev(g.val).double(), size=(n, n))
+    ref = (A.to_dense() @ (dev(H).double() @ dev(W).double()))
+    assert_close(out["h"], ref.float().cpu(), "GCN special case")
+
+
+def test_isolated_nodes_and_empty_graph(ctx, B):
+    n, d_in, d_out = 37, 50, 9
+    rng = np.random.default_rng(3)
+    e = np.zeros(0, np.int32)
+    g = oracle.normalize_adjacency(n, e, e)                        # A_tilde = I  =>  H' = zeta
+    H = rng.standard_normal((n, d_in)).astype(np.float32)
+    W = rng.standard_normal((d_in, d_out)).astype(np.float32)
+    t = oracle.layer_forward(g, oracle.Layer(W), H)
+    G = device_graph(B, g)
+    out = ctx.layer_forward(G, B.make_layer(d_in, d_out, bits_to_dev(t.bitsT), dev(t.alpha)), bits_to_dev(t.bits),
+                            dev(t.beta), debug=True)
+    assert_close(out["h"], t.H_out, "identity adjacency")
+    assert_close(out["h"], out["zeta"].cpu(), "H' = zeta")
+    # n = 0 is a no-op
+    G0 = B.make_graph(torch.zeros(1, dtype=torch.int64).cuda(), torch.zeros(0, dtype=torch.int32).cuda(),
+                      torch.zeros(0).cuda())
+    lay = B.make_layer(d_in, d_out, bits_to_dev(t.bitsT), dev(t.alpha))
+    logits = ctx.forward(G0, [lay], torch.zeros((0, d_in)).cuda())
+    assert logits.shape == (0, d_out)
+
+
+def test_argument_errors_are_reported_not_launched(ctx, B):
+    import ctypes
+    n, d_in, d_out = 10, 40, 5
+    _, _, g = small_graph(n, 30, 1)
+    G = device_graph(B, g)
+    bitsT = torch.zeros((d_out, 4), dtype=torch.int32).cuda()
+    alpha = torch.ones(d_out).cuda()
+    lay = B.make_layer(d_in, d_out, bitsT, alpha)
+    before = ctx.launch_count()
+    with pytest.raises(B.BigcnError) as e:                      # no workspace large enough: shrink it
+        ctx.lib.bigcn_set_workspace(ctx.h, None, 0)
+        ctx._check(ctx.lib.bigcn_forward(ctx.h, ctypes.byref(G.c), B._layer_array([lay]), 1,
+                                         ctypes.c_void_p(alpha.data_ptr()), d_in, ctypes.c_void_p(alpha.data_ptr()), d_out, None))
+    assert e.value.status == 5
+    ctx.workspace = None
+    bad = B.make_layer(d_in, 0, bitsT, alpha)
+    with pytest.raises(B.BigcnError) as e:
+        ctx.forward(G, [bad], torch.zeros((n, d_in)).cuda())
+    assert e.value.status == 2
+    two = [lay, B.make_layer(d_out + 1, 3, bitsT, alpha)]          # widths do not chain
+    with pytest.raises(B.BigcnError) as e:
+        ctx.forward(G, two, torch.zeros((n, d_in)).cuda())
+    assert e.value.status == 2
+    with pytest.raises(B.BigcnError) as e:                      # misaligned packed input
+        ctx._check(ctx.lib.bigcn_pack_features(ctx.h, ctypes.c_void_p(alpha.data_ptr()), 1, 4, 4, None, None,
+                                               ctypes.c_void_p(bitsT.data_ptr() + 4), 4, ctypes.c_void_p(alpha.data_ptr())))
+    assert e.value.status == 3
+    assert ctx.launch_count() == before
+
+
+# --------------------------------------------------------------------------- whole networks
+
+NETS = [("c1", None), ("c2", None), ("c3", None), ("c4", 0.01), ("c5", 0.004)]
+
+
+@pytest.fixture(scope="module", params=NETS, ids=lambda p: p[0] if p[1] is None else "%s@%g" % p)
+def net(request):
+    name, scale = request.param
+    wl = synth.make_workload(name, scale=scale, device="cuda")
+    return oracle_run(wl)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_network_layer_by_layer_oracle_fed(B, net, fmt):
+    """Each layer is fed the oracle's own input (packed bits and beta); bits and dots exact, fp32
+    within tolerance, re-binarized bits equal up to threshold-adjacent flips."""
+    ctx = B.BiGCN(0)
+    ctx.set_option(B.OPT_ZETA_FORMAT, fmt)
+    G = device_graph(B, net.graph)
+    layers = device_layers_from_oracle(B, net)
+    L = len(layers)
+    for l in range(L):
+        t = net.traces[l]
+        nxt = layers[l + 1] if l + 1 < L else None
+        out = ctx.layer_forward(G, layers[l], bits_to_dev(t.bits), dev(t.beta), want_h=True, next_layer=nxt, debug=True)
+        assert torch.equal(out["dot"].cpu(), torch.from_numpy(t.dot))
+        assert torch.equal(out["zeta"].cpu(), torch.from_numpy(t.zeta))
+        assert_close(out["h"], t.H_out, "layer %d output" % l)
+        if nxt is not None:
+            tn = net.traces[l + 1]
+            flips, bad, total = flip_report(bits_from_dev(out["next_bits"]), tn.F, t.H_out, net.layers[l + 1].in_shift)
+            assert bad == 0 and flips <= max(2, total // 2000), (flips, bad, total)
+            np.testing.assert_allclose(out["next_beta"].cpu().numpy(), tn.beta, rtol=1e-4, atol=1e-5)
+    ctx.sync_check()
+    ctx.close()
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_network_end_to_end(B, net, fmt):
+    """From fp32 features and fp32 weights through the library's own packers to logits."""
+    wl = net.wl
+    ctx = B.BiGCN(0)
+    ctx.set_option(B.OPT_ZETA_FORMAT, fmt)
+    G = ctx.normalize_adjacency(wl.rowptr.cuda(), wl.colidx.cuda())
+    shifts = [dev(l.in_shift) if l.in_shift is not None else None for l in net.layers]
+    scales = [dev(l.in_scale) if l.in_scale is not None else None for l in net.layers]
+    layers = ctx.prepare_layers([w.cuda() for w in wl.W], shifts, scales)
+    X = wl.X.cuda()
+    # first-layer bits must be exact (sign(x - mu) is decided in the same fp32 arithmetic)
+    xb, xbeta = ctx.pack_features(X, shifts[0], scales[0])
+    assert np.array_equal(bits_from_dev(xb), net.traces[0].bits)
+    logits, st = ctx.forward(G, layers, X, stats=True)
+    ref = torch.from_numpy(net.logits)
+    err = (logits.cpu().double() - ref.double()).abs()
+    allow = ATOL + RTOL * ref.double().abs()
+    frac_out = (err > allow).double().mean().item()
+    agree = (logits.cpu().argmax(1) == ref.argmax(1)).double().mean().item()
+    print("\n[%s fmt %d] max|err| %.3g, share outside tolerance %.3g, argmax agreement %.6f, launches %d, %.3f ms"
+          % (wl.spec.name, fmt, err.max().item(), frac_out, agree, st.launches, st.ms_total))
+    # sign flips at a re-binarization may move a few logits beyond the per-element tolerance; they
+    # must stay rare and the predictions must agree
+    assert frac_out <= 2e-3 and agree >= 0.995
+    assert st.launches == 1 + 2 * len(layers)
+    # same result from pre-packed input and from host buffers
+    l2 = ctx.forward_packed(G, layers, xb, xbeta)
+    assert torch.equal(l2, logits)
+    xh = wl.X.cpu().pin_memory()
+    oh = torch.empty((wl.n, wl.spec.dims[-1]), dtype=torch.float32).pin_memory()
+    ctx.forward_host(G, layers, xh, oh)
+    assert torch.equal(oh, logits.cpu())
+    # deterministic from run to run
+    assert torch.equal(ctx.forward(G, layers, X), logits)
+    ctx.sync_check()
+    ctx.close()
+
+
+def test_network_flip_rate_report(B, net):
+    """End to end with the GPU's own intermediate results: how many re-binarized bits differ from the
+    oracle's (reported; they can only sit next to the threshold)."""
+    wl = net.wl
+    ctx = B.BiGCN(0)
+    G = device_graph(B, net.graph)
+    layers = device_layers_from_oracle(B, net)
+    bits, beta = bits_to_dev(net.traces[0].bits), dev(net.traces[0].beta)
+    for l in range(len(layers) - 1):
+        out = ctx.layer_forward(G, layers[l], bits, beta, want_h=False, next_layer=layers[l + 1])
+        bits, beta = out["next_bits"], out["next_beta"]
+        got = oracle.unpack_rows(bits_from_dev(bits), layers[l].d_out)
+        flips = int((got != net.traces[l + 1].F).sum())
+        print("\n[%s] layer %d -> %d: %d of %d bits flipped (%.3g)" % (wl.spec.name, l, l + 1, flips, got.size, flips / got.size))
+        assert flips <= max(4, got.size // 1000)
+    ctx.close()
