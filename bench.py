@@ -40,6 +40,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-sample-scale", type=float, default=None)
+    ap.add_argument("--scale", type=float, default=None,
+                    help="shrink nodes and edges of the workload by this factor (profiling on a small case)")
     return ap.parse_args()
 
 
@@ -194,8 +196,8 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
 
-    spec = synth.WORKLOADS[args.config]
-    wl = synth.make_workload(args.config, device=dev)
+    wl = synth.make_workload(args.config, scale=args.scale, device=dev)
+    spec = wl.spec
     ctx = binding.BiGCN(local)
     if args.zeta_format:
         ctx.set_option(binding.OPT_ZETA_FORMAT, args.zeta_format)
@@ -335,7 +337,7 @@ def run_ours(args):
     cpu = None
     if not args.no_cpu_baseline:
         try:
-            scale = args.cpu_sample_scale or default_cpu_scale(spec)
+            scale = args.cpu_sample_scale or min(1.0, default_cpu_scale(synth.WORKLOADS[args.config]))
             v, threads, sample, ms = time_oracle(args.config, scale, 2, 1)
             cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample, "ms_per_step": ms}
         except Exception as exc:      # the oracle is optional equipment for the bench
