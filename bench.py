@@ -36,7 +36,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default="c5", help="workload c1..c5 (default: the largest, c5)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--zeta-format", type=int, default=0, help="0 auto, 1 fp32, 2 int16, 3 int8")
+    ap.add_argument("--zeta-format", type=int, default=0, help="0 auto, 1 fp32, 2 int16, 3 int8, 4 fp16")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-sample-scale", type=float, default=None)
@@ -304,14 +304,16 @@ def run_ours(args):
     spmm_ms = [mean(v) for v in per_kernel["spmm"]]
     gemm_ms = [mean(v) for v in per_kernel["gemm"]]
     pack_ms = mean(per_kernel["pack"])
-    fmt = args.zeta_format or binding.ZETA_I16
+    fmt = args.zeta_format or binding.ZETA_F16
     kernels = {}
     dom = max(range(L), key=lambda l: spmm_ms[l])
     for l in range(L):
         f = fmt
         if f == binding.ZETA_I8 and dims[l] > 127:
+            f = binding.ZETA_F16
+        if f == binding.ZETA_F16 and dims[l] > 2048:
             f = binding.ZETA_I16
-        elt = {1: 4, 2: 2, 3: 1}[f]
+        elt = {1: 4, 2: 2, 3: 1, 4: 2}[f]
         per16 = 16 // elt
         ldz = (dims[l + 1] + per16 - 1) // per16 * per16
         last = (l == L - 1)
@@ -320,7 +322,7 @@ def run_ours(args):
         t = spmm_ms[l] * 1e-3
         kernels["spmm_l%d" % l] = {"ms": spmm_ms[l], "GBps_expected_model": expected / t / 1e9,
                                    "GBps_lower_model": lower / t / 1e9, "GBps_no_reuse_model": upper / t / 1e9,
-                                   "bytes_expected": expected, "zeta_format": {1: "f32", 2: "i16", 3: "i8"}[f]}
+                                   "bytes_expected": expected, "zeta_format": {1: "f32", 2: "i16", 3: "i8", 4: "f16"}[f]}
         ops = 2.0 * n * dims[l] * dims[l + 1]
         kernels["bitgemm_l%d" % l] = {"ms": gemm_ms[l], "binary_TOPS": ops / (gemm_ms[l] * 1e-3) / 1e12,
                                       "out_GBps": n * ldz * elt / (gemm_ms[l] * 1e-3) / 1e9}
@@ -348,7 +350,7 @@ def run_ours(args):
             "vs_baseline": None, "dtype": DTYPE, "data": "synthetic",
             "config": {"workload": workload_description(spec, n, nnz), "l2": "inputs_exceed_l2",
                        "parallelism": "replicas" if world > 1 else "single-gpu",
-                       "zeta_format": {0: "auto(i16)", 1: "f32", 2: "i16", 3: "i8"}[args.zeta_format]},
+                       "zeta_format": {0: "auto(f16)", 1: "f32", 2: "i16", 3: "i8", 4: "f16"}[args.zeta_format]},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
             "kernels": kernels}
     print(json.dumps(line), flush=True)

@@ -56,10 +56,13 @@ typedef struct bigcn_ctx bigcn_ctx;
 /* Options for bigcn_set_option(). */
 enum {
     /* Storage of the rescaled contraction zeta between the bit-GEMM and the aggregation.
-     * 0 = choose per layer (default); 1 = fp32 zeta_ij = (beta_i alpha_j) dot_ij, exactly Eq. "cdot-op";
+     * 0 = choose per layer (default: 4 when d_in <= 2048, else 2);
+     * 1 = fp32 zeta_ij = (beta_i alpha_j) dot_ij, exactly Eq. "cdot-op";
      * 2 = the integer dot products as int16, with beta folded into the edge weights and alpha
      *     applied once per output element (same sum, different rounding order);
-     * 3 = as 2 but int8 (layers with d_in <= 127 only; others fall back to 2). */
+     * 3 = as 2 but int8 (layers with d_in <= 127 only; others fall back to 4);
+     * 4 = as 2 but the integers held as fp16, which is exact for |dot| <= 2048 (layers with
+     *     d_in <= 2048 only; others fall back to 2). */
     BIGCN_OPT_ZETA_FORMAT = 1,
     /* Rows of the sparse matrix with more entries than this are split across thread blocks. 0 = default. */
     BIGCN_OPT_LONG_ROW = 2

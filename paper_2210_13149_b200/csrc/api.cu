@@ -58,8 +58,9 @@ size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 int pick_format(const bigcn_ctx* ctx, int d_in)
 {
     int f = ctx->zeta_format;
-    if (f == 0) f = kZetaI16;
-    if (f == kZetaI8 && d_in > 127) f = kZetaI16;
+    if (f == 0) f = kZetaF16;
+    if (f == kZetaI8 && d_in > 127) f = kZetaF16;      // |dot| must fit the element type exactly
+    if (f == kZetaF16 && d_in > 2048) f = kZetaI16;
     if (f == kZetaI16 && d_in > 32767) f = kZetaF32;
     return f;
 }
@@ -305,7 +306,7 @@ bigcn_status bigcn_set_option(bigcn_ctx* ctx, int32_t option, int64_t value)
     if (!ctx) return BIGCN_ERR_NULL;
     switch (option) {
         case BIGCN_OPT_ZETA_FORMAT:
-            if (value < 0 || value > 3) return fail(ctx, BIGCN_ERR_SHAPE, "zeta format %lld not in [0, 3]", (long long)value);
+            if (value < 0 || value > 4) return fail(ctx, BIGCN_ERR_SHAPE, "zeta format %lld not in [0, 4]", (long long)value);
             ctx->zeta_format = (int)value;
             return BIGCN_OK;
         case BIGCN_OPT_LONG_ROW:

@@ -11,7 +11,7 @@ namespace bigcn {
 constexpr int kWarp = 32;
 
 // Storage of the contraction result between the bit-GEMM and the aggregation.
-enum ZetaFormat : int { kZetaF32 = 1, kZetaI16 = 2, kZetaI8 = 3 };
+enum ZetaFormat : int { kZetaF32 = 1, kZetaI16 = 2, kZetaI8 = 3, kZetaF16 = 4 };
 
 inline __host__ __device__ int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline __host__ __device__ int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
@@ -19,10 +19,9 @@ inline __host__ __device__ int64_t round_up(int64_t a, int64_t b) { return ceil_
 // Elements per row of the zeta buffer: d_out rounded up so that a row is a whole number of 16-byte vectors.
 inline int64_t zeta_ld(int d_out, int fmt)
 {
-    const int per16 = fmt == kZetaF32 ? 4 : (fmt == kZetaI16 ? 8 : 16);
-    return round_up(d_out, per16);
+    return round_up(d_out, 16 / (fmt == kZetaF32 ? 4 : (fmt == kZetaI8 ? 1 : 2)));
 }
-inline int zeta_elt_bytes(int fmt) { return fmt == kZetaF32 ? 4 : (fmt == kZetaI16 ? 2 : 1); }
+inline int zeta_elt_bytes(int fmt) { return fmt == kZetaF32 ? 4 : (fmt == kZetaI8 ? 1 : 2); }
 
 // ---- launchers (each returns the launch status; all asynchronous on `s`) ------------------------
 

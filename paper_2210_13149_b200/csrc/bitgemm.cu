@@ -1,6 +1,8 @@
 // XNOR / bit-count contraction fused with the beta_i alpha_j rescale.
 // Bi-GCN Sec. 4.2.3: dot_ij = F_i (*) B_j = d_in - 2 popc(F_i XOR B_j)   (Eq. "bi-op"),
 //                    zeta_ij = beta_i alpha_j dot_ij                     (Eq. "cdot-op").
+#include <cuda_fp16.h>
+
 #include <algorithm>
 
 #include "bigcn_internal.cuh"
@@ -96,14 +98,15 @@ bitgemm_kernel(const uint32_t* __restrict__ A, int64_t stride_a,
                     if (j < d_out) {
                         const float z = __fmul_rn(__fmul_rn(be, al[t]), (float)dot);
                         if (fmt == kZetaF32) reinterpret_cast<float*>(zeta)[row * ldz + j] = z;
+                        else if (fmt == kZetaF16) reinterpret_cast<__half*>(zeta)[row * ldz + j] = __int2half_rn(dot);   // exact: |dot| <= 2048
                         else if (fmt == kZetaI16) reinterpret_cast<int16_t*>(zeta)[row * ldz + j] = (int16_t)dot;
                         else reinterpret_cast<int8_t*>(zeta)[row * ldz + j] = (int8_t)dot;
                         if (dbg_dot) dbg_dot[row * (int64_t)d_out + j] = dot;
                         if (dbg_zeta) dbg_zeta[row * (int64_t)d_out + j] = z;
                     } else if (j < ldz) {                  // padding columns of the zeta row: keep them zero
                         if (fmt == kZetaF32) reinterpret_cast<float*>(zeta)[row * ldz + j] = 0.f;
-                        else if (fmt == kZetaI16) reinterpret_cast<int16_t*>(zeta)[row * ldz + j] = 0;
-                        else reinterpret_cast<int8_t*>(zeta)[row * ldz + j] = 0;
+                        else if (fmt == kZetaI8) reinterpret_cast<int8_t*>(zeta)[row * ldz + j] = 0;
+                        else reinterpret_cast<int16_t*>(zeta)[row * ldz + j] = 0;          // int16 and fp16 zero alike
                     }
                 }
             }

@@ -2,12 +2,25 @@
 // optional re-binarization of H' for the next layer (Sec. 4.2.2 applied to the layer output, after
 // the next layer's batch-norm constants of Sec. 4.4) fused into the epilogue.
 //
-// One warp owns one output row.  A row of zeta is read as 16-byte vectors: LPR lanes cover one row
-// (NCH vectors per lane when a row has more than 32 vectors) and the 32/LPR lane groups of a warp
-// work on different neighbours at the same time; their partial sums are combined with shuffles.
-// Rows with more stored entries than `long_row` are processed by all warps of the thread block
-// together (each warp a contiguous slice of the row, partial sums combined through shared memory in
-// warp order), so results never depend on scheduling.
+// The kernel is bound by the random gather of zeta rows, so it is built around keeping many row
+// fetches in flight at a low instruction cost per stored entry.  A warp owns a run of consecutive
+// output rows and treats their stored entries as one stream.  Each stream position is fetched with
+// one warp-wide asynchronous copy (cp.async, 16 bytes per lane, global -> shared, bypassing L1 and
+// the register file) into a ring of slots private to the warp; positions are issued and retired in
+// groups of PB, and NG groups are in flight per warp, across row boundaries.  A row of zeta is nv
+// 16-byte vectors: LPR lanes cover one row (NCH vectors per lane when nv > 32) and the G = 32/LPR
+// lane groups of a warp fetch G consecutive entries per position; their partial sums are combined
+// with shuffles when a row ends.  Column indices and edge weights are prefetched three 32-entry
+// chunks ahead in registers.  There is no waiting on other warps or blocks anywhere:
+// cp.async.wait_group only waits for the calling thread's own copies.
+//
+// Rows with more stored entries than `long_row` are left out of the streams and processed afterwards
+// by all warps of the thread block together (each warp a contiguous slice, partial sums combined
+// through shared memory in warp order), so results never depend on scheduling.
+#include <cuda_fp16.h>
+
+#include <algorithm>
+
 #include "bigcn_internal.cuh"
 
 namespace bigcn {
@@ -16,8 +29,9 @@ namespace {
 
 constexpr int kSpmmWarps = 8;
 constexpr int kSpmmThreads = kSpmmWarps * kWarp;
-constexpr int kEdgesInFlight = 4;        // independent 16-byte gathers per lane group
+constexpr int kMaxRowsPerWarp = 16;      // consecutive rows streamed by one warp
 
+// Element types of a zeta row and their conversion to fp32 (one 16-byte vector at a time).
 template <typename T> struct Elt;
 template <> struct Elt<float> {
     static constexpr int kPerVec = 4;
@@ -25,6 +39,19 @@ template <> struct Elt<float> {
     {
         f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
         f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+    }
+};
+template <> struct Elt<__half> {
+    static constexpr int kPerVec = 8;
+    static __device__ __forceinline__ void unpack(const uint4& v, float (&f)[8])
+    {
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 t = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+            f[2 * i] = t.x;
+            f[2 * i + 1] = t.y;
+        }
     }
 };
 template <> struct Elt<int16_t> {
@@ -75,57 +102,28 @@ struct SpmmDev {
     int64_t long_row;
 };
 
-// acc += sum over stored entries [start, end) of weight * zeta row, for the calling warp.
-template <typename T, int NCH, int LPR>
-__device__ __forceinline__ void accumulate(const SpmmDev& p, int64_t start, int64_t end, int lane,
-                                           float (&acc)[NCH][Elt<T>::kPerVec])
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
 {
-    constexpr int EPV = Elt<T>::kPerVec;
-    constexpr int G = kWarp / LPR;
-    constexpr int U = kEdgesInFlight;
-    const int g = lane / LPR, l = lane % LPR;
-    bool active[NCH];
-#pragma unroll
-    for (int c = 0; c < NCH; ++c) active[c] = (c * 32 + l) < p.nv;
+    const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 
-    for (int64_t base = start; base < end; base += 32) {
-        const int cnt = (int)min((int64_t)32, end - base);
-        int my_col = 0;
-        float my_w = 0.f;
-        if (lane < cnt) {
-            my_col = __ldg(p.colidx + base + lane);
-            my_w = __ldg(p.val + base + lane);
-            if (p.node_w) my_w *= __ldg(p.node_w + my_col);
-        }
-        for (int e = 0; e < cnt; e += G * U) {
-            uint4 v[U][NCH];
-            float w[U];
+template <int NCH, int EPV>
+__device__ __forceinline__ void zero_acc(float (&acc)[NCH][EPV])
+{
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int idx = e + u * G + g;
-                const int k = __shfl_sync(0xffffffffu, my_col, idx & 31);
-                w[u] = __shfl_sync(0xffffffffu, my_w, idx & 31);
-                const bool ok = idx < cnt;
-                if (!ok) w[u] = 0.f;
-                const uint4* zrow = p.zeta + (int64_t)k * p.nv + l;
+    for (int c = 0; c < NCH; ++c)
 #pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    if (ok && active[c]) v[u][c] = __ldg(zrow + c * 32);
-                    else v[u][c] = make_uint4(0u, 0u, 0u, 0u);
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < U; ++u)
-#pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    float f[EPV];
-                    Elt<T>::unpack(v[u][c], f);
-#pragma unroll
-                    for (int i = 0; i < EPV; ++i) acc[c][i] = fmaf(w[u], f[i], acc[c][i]);
-                }
-        }
-    }
-    // combine the lane groups: afterwards every lane holds the sum for its vector(s)
+        for (int i = 0; i < EPV; ++i) acc[c][i] = 0.f;
+}
+
+// Sum over the lane groups: afterwards every lane holds the total for its vector(s).
+template <int NCH, int EPV, int LPR>
+__device__ __forceinline__ void reduce_groups(float (&acc)[NCH][EPV])
+{
 #pragma unroll
     for (int o = LPR; o < kWarp; o <<= 1)
 #pragma unroll
@@ -194,58 +192,223 @@ __device__ __forceinline__ void finish_row(const SpmmDev& p, int64_t row, int la
     }
 }
 
-template <typename T, int NCH, int LPR>
-__global__ void __launch_bounds__(kSpmmThreads)
-spmm_kernel(const SpmmDev p)
+template <int NCH, int LPR>
+struct Pipe {
+    static constexpr int G = kWarp / LPR;                       // entries per position
+    static constexpr int PB = (4 * G <= 32) ? 4 : 32 / G;       // positions per group (PB * G divides 32)
+    static constexpr int NG = NCH == 1 ? 3 : 2;                 // groups in flight per warp
+    static constexpr int RING = PB * NG;                        // slots of NCH * 512 bytes
+    static constexpr size_t kWarpBytes = (size_t)RING * (NCH * 512 + G * 4);
+};
+
+// Streams the stored entries [e0, e0 + n_ent) through the warp's ring.
+//   kPartial = false: the entries are those of rows [row_lo, row_hi); `rp_rel` holds, in lane j, the
+//                     end of local row j - 1 relative to e0 (shuffled out as rows complete); every
+//                     row is written as its last entry is consumed.
+//   kPartial = true : the entries are a slice of one long row; the slice's sum is left in `acc`
+//                     (already combined over the lane groups).
+template <typename T, int NCH, int LPR, bool kPartial>
+__device__ __forceinline__ void stream_entries(const SpmmDev& p, uint4* ring, float* wfifo, int lane,
+                                               int64_t e0, int n_ent, int64_t warp_row0, int row_lo,
+                                               int row_hi, int rp_rel,
+                                               float (&acc)[NCH][Elt<T>::kPerVec])
 {
+    using P = Pipe<NCH, LPR>;
     constexpr int EPV = Elt<T>::kPerVec;
-    __shared__ float part[kSpmmWarps][(LPR < 32 ? LPR : NCH * 32) * EPV];
-    __shared__ int long_mask;
+    constexpr int G = P::G, PB = P::PB, NG = P::NG;
+    const int g = lane / LPR, l = lane % LPR;
+    bool active[NCH];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) active[c] = (c * 32 + l) < p.nv;
+    const int32_t* cols = p.colidx + e0;
+    const float* vals = p.val + e0;
+
+    // metadata chunks of 32 entries: A = ready (column, weight), B = column/value/node factor in
+    // flight, C = column/value in flight
+    auto load_col = [&](int e) { return e < n_ent ? __ldg(cols + e) : 0; };
+    auto load_val = [&](int e) { return e < n_ent ? __ldg(vals + e) : 0.f; };
+    int a_col = load_col(lane);
+    float a_w = load_val(lane);
+    int b_col = load_col(32 + lane);
+    float b_val = load_val(32 + lane);
+    int c_col = load_col(64 + lane);
+    float c_val = load_val(64 + lane);
+    if (p.node_w) a_w *= __ldg(p.node_w + a_col);
+    float b_nw = p.node_w ? __ldg(p.node_w + b_col) : 1.f;
+    int chunk = 0;
+
+    const int n_groups = (n_ent + PB * G - 1) / (PB * G);
+    int rt = row_lo;                                          // row being accumulated (local index)
+    int row_end = kPartial ? n_ent : __shfl_sync(0xffffffffu, rp_rel, rt + 1);
+    zero_acc<NCH, EPV>(acc);
+
+    for (int it = 0; it < n_groups + NG; ++it) {
+        const int gslot = (it % NG) * PB;                     // first slot of the group handled now
+        if (it >= NG) {
+            // ---- retire group it - NG (its copies are the oldest outstanding cp.async group)
+            cp_async_wait<NG - 1>();
+            __syncwarp();
+            const int off0 = (it - NG) * (PB * G);            // first entry of the group
+            uint4 v[PB][NCH];
+            float w[PB];
+#pragma unroll
+            for (int b = 0; b < PB; ++b) {
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) v[b][c] = ring[(gslot + b) * (NCH * 32) + c * 32 + lane];
+                w[b] = wfifo[(gslot + b) * G + g];
+            }
+            if (off0 + PB * G < row_end) {
+                // the whole group lies inside the current row: no boundary logic
+#pragma unroll
+                for (int b = 0; b < PB; ++b)
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) {
+                        float f[EPV];
+                        Elt<T>::unpack(v[b][c], f);
+                        if (NCH == 1 || active[c]) {
+#pragma unroll
+                            for (int i = 0; i < EPV; ++i) acc[c][i] = fmaf(w[b], f[i], acc[c][i]);
+                        }
+                    }
+            } else {
+#pragma unroll
+                for (int b = 0; b < PB; ++b) {
+                    const int eb = off0 + b * G;              // first entry of the position
+                    if (eb >= n_ent) break;
+                    const int nb = min(G, n_ent - eb);
+                    float f[NCH][EPV];
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) Elt<T>::unpack(v[b][c], f[c]);
+                    int done = 0;
+                    for (;;) {
+                        const int rem = row_end - eb;         // entries of the position before the row's end
+                        const int upto = rem < nb ? rem : nb;
+                        if (g >= done && g < upto) {
+#pragma unroll
+                            for (int c = 0; c < NCH; ++c)
+                                if (active[c]) {
+#pragma unroll
+                                    for (int i = 0; i < EPV; ++i) acc[c][i] = fmaf(w[b], f[c][i], acc[c][i]);
+                                }
+                        }
+                        if (rem > nb) break;                  // the row continues in a later position
+                        reduce_groups<NCH, EPV, LPR>(acc);
+                        if (kPartial) return;                 // slice complete (only at the last position)
+                        finish_row<T, NCH, LPR>(p, warp_row0 + rt, lane, acc);
+                        zero_acc<NCH, EPV>(acc);
+                        if (upto > done) done = upto;
+                        ++rt;
+                        if (rt == row_hi) break;
+                        row_end = __shfl_sync(0xffffffffu, rp_rel, rt + 1);
+                    }
+                }
+            }
+            __syncwarp();                                     // all lanes are done with these slots
+        }
+        if (it < n_groups) {
+            // ---- issue group `it` into the slots just freed
+            const int off0 = it * (PB * G);
+            if ((off0 >> 5) != chunk) {                       // rotate the metadata chunks
+                a_col = b_col;
+                a_w = b_val * b_nw;
+                b_col = c_col;
+                b_val = c_val;
+                b_nw = p.node_w ? __ldg(p.node_w + b_col) : 1.f;
+                ++chunk;
+                c_col = load_col(((chunk + 2) << 5) + lane);
+                c_val = load_val(((chunk + 2) << 5) + lane);
+            }
+            const bool whole = off0 + PB * G <= n_ent;        // no entry of the group is past the end
+#pragma unroll
+            for (int b = 0; b < PB; ++b) {
+                const int idx = (off0 & 31) + b * G + g;
+                const int k = __shfl_sync(0xffffffffu, a_col, idx);
+                const float wv = __shfl_sync(0xffffffffu, a_w, idx);
+                if (whole || off0 + b * G + g < n_ent) {
+                    const uint4* src = p.zeta + (int64_t)k * p.nv + l;
+                    uint4* dst = ring + (gslot + b) * (NCH * 32) + lane;
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c)
+                        if (active[c]) cp_async16(dst + c * 32, src + c * 32);
+                }
+                if (l == 0) wfifo[(gslot + b) * G + g] = wv;  // padding entries carry weight 0
+            }
+        }
+        cp_async_commit();                                    // one group per iteration, possibly empty
+    }
+    cp_async_wait<0>();
+    if (kPartial) {                                           // empty slice
+        reduce_groups<NCH, EPV, LPR>(acc);
+        return;
+    }
+    while (rt < row_hi) {                                     // rows without entries at the end of the run
+        reduce_groups<NCH, EPV, LPR>(acc);
+        finish_row<T, NCH, LPR>(p, warp_row0 + rt, lane, acc);
+        zero_acc<NCH, EPV>(acc);
+        ++rt;
+    }
+}
+
+template <typename T, int NCH, int LPR>
+__global__ void __launch_bounds__(kSpmmThreads, NCH == 1 ? 4 : (NCH == 2 ? 2 : 1))
+spmm_kernel(const SpmmDev p, int rows_per_warp)
+{
+    using P = Pipe<NCH, LPR>;
+    constexpr int EPV = Elt<T>::kPerVec;
+    constexpr int G = P::G;
+    constexpr int kCols = (LPR < 32 ? LPR : NCH * 32) * EPV;  // accumulator columns of one warp
+    extern __shared__ __align__(128) unsigned char dsmem[];
+    __shared__ int long_rows[kSpmmWarps * kMaxRowsPerWarp];
+    __shared__ int n_long;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const int64_t row = (int64_t)blockIdx.x * kSpmmWarps + warp;
-    if (threadIdx.x == 0) long_mask = 0;
+    uint4* ring = reinterpret_cast<uint4*>(dsmem + (size_t)warp * P::RING * NCH * 512);
+    float* wfifo = reinterpret_cast<float*>(dsmem + (size_t)kSpmmWarps * P::RING * NCH * 512) + warp * P::RING * G;
+    float* part = reinterpret_cast<float*>(dsmem);           // [kSpmmWarps][kCols], reuses the rings (see below)
+    static_assert((size_t)kSpmmWarps * kCols * 4 <= (size_t)kSpmmWarps * P::RING * NCH * 512, "partials must fit the rings");
+    if (threadIdx.x == 0) n_long = 0;
     __syncthreads();
 
-    int64_t start = 0, end = 0;
-    if (row < p.n) {
-        start = __ldg(p.rowptr + row);
-        end = __ldg(p.rowptr + row + 1);
+    const int64_t block_row0 = (int64_t)blockIdx.x * kSpmmWarps * rows_per_warp;
+    const int64_t warp_row0 = block_row0 + (int64_t)warp * rows_per_warp;
+    const int n_rows = (int)max((int64_t)0, min((int64_t)rows_per_warp, p.n - warp_row0));
+    float acc[NCH][EPV];
+    if (n_rows > 0) {
+        const int64_t rp_reg = __ldg(p.rowptr + warp_row0 + min(lane, n_rows));
+        const int64_t rp_next = __shfl_down_sync(0xffffffffu, rp_reg, 1);
+        const bool is_long = lane < n_rows && p.long_row > 0 && (rp_next - rp_reg) > p.long_row;
+        const unsigned long_mask = __ballot_sync(0xffffffffu, is_long);
+        if (is_long) long_rows[atomicAdd(&n_long, 1)] = (int)(warp_row0 + lane - block_row0);
+        int ra = 0;
+        while (ra < n_rows) {                                 // runs of rows between the long ones
+            const unsigned rest = long_mask >> ra;
+            const int rl = rest ? ra + (__ffs(rest) - 1) : n_rows;
+            if (rl > ra) {
+                const int64_t e0 = __shfl_sync(0xffffffffu, rp_reg, ra);
+                const int64_t e1 = __shfl_sync(0xffffffffu, rp_reg, rl);
+                // a run holds at most kMaxRowsPerWarp * long_row entries
+                stream_entries<T, NCH, LPR, false>(p, ring, wfifo, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
+                                                   (int)(rp_reg - e0), acc);
+            }
+            ra = rl + 1;
+        }
     }
-    const bool is_long = p.long_row > 0 && (end - start) > p.long_row;
-    if (row < p.n && !is_long) {
-        float acc[NCH][EPV];
-#pragma unroll
-        for (int c = 0; c < NCH; ++c)
-#pragma unroll
-            for (int i = 0; i < EPV; ++i) acc[c][i] = 0.f;
-        accumulate<T, NCH, LPR>(p, start, end, lane, acc);
-        finish_row<T, NCH, LPR>(p, row, lane, acc);
-    }
-    if (is_long && lane == 0) atomicOr(&long_mask, 1 << warp);
     __syncthreads();
-    const int mask = long_mask;
-    if (mask == 0) return;
-
+    const int nl = n_long;
     // Long rows of this block, one after the other, each by all warps together.
-    for (int wr = 0; wr < kSpmmWarps; ++wr) {
-        if (!((mask >> wr) & 1)) continue;
-        const int64_t lrow = (int64_t)blockIdx.x * kSpmmWarps + wr;
+    for (int q = 0; q < nl; ++q) {
+        const int64_t lrow = block_row0 + long_rows[q];
         const int64_t ls = __ldg(p.rowptr + lrow), le = __ldg(p.rowptr + lrow + 1);
         const int64_t slice = round_up(ceil_div(le - ls, kSpmmWarps), 32);
         const int64_t s0 = min(le, ls + warp * slice), s1 = min(le, s0 + slice);
-        float acc[NCH][EPV];
-#pragma unroll
-        for (int c = 0; c < NCH; ++c)
-#pragma unroll
-            for (int i = 0; i < EPV; ++i) acc[c][i] = 0.f;
-        accumulate<T, NCH, LPR>(p, s0, s1, lane, acc);
+        stream_entries<T, NCH, LPR, true>(p, ring, wfifo, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
+        __syncthreads();                                      // every ring is idle: reuse them for the partial sums
         const int l = lane % LPR;
         if (lane < LPR) {
 #pragma unroll
             for (int c = 0; c < NCH; ++c)
 #pragma unroll
-                for (int i = 0; i < EPV; ++i) part[warp][(c * 32 + l) * EPV + i] = acc[c][i];
+                for (int i = 0; i < EPV; ++i) part[warp * kCols + (c * 32 + l) * EPV + i] = acc[c][i];
         }
         __syncthreads();
         if (warp == 0) {
@@ -254,7 +417,7 @@ spmm_kernel(const SpmmDev p)
 #pragma unroll
                 for (int i = 0; i < EPV; ++i) {
                     float t = 0.f;
-                    for (int w = 0; w < kSpmmWarps; ++w) t += part[w][(c * 32 + l) * EPV + i];
+                    for (int w = 0; w < kSpmmWarps; ++w) t += part[w * kCols + (c * 32 + l) * EPV + i];
                     acc[c][i] = t;
                 }
             finish_row<T, NCH, LPR>(p, lrow, lane, acc);
@@ -266,8 +429,15 @@ spmm_kernel(const SpmmDev p)
 template <typename T, int NCH, int LPR>
 cudaError_t launch_one(cudaStream_t s, const SpmmDev& p)
 {
-    const unsigned grid = (unsigned)ceil_div(p.n, kSpmmWarps);
-    spmm_kernel<T, NCH, LPR><<<grid, kSpmmThreads, 0, s>>>(p);
+    constexpr size_t smem = kSpmmWarps * Pipe<NCH, LPR>::kWarpBytes;
+    // enough thread blocks to fill the machine on small graphs, long runs of rows on large ones
+    const int rows_per_warp = (int)std::min<int64_t>(kMaxRowsPerWarp, std::max<int64_t>(1, p.n / (kSpmmWarps * 148 * 8)));
+    if (smem > 40 * 1024) {                                   // above the default limit: opt in
+        cudaError_t e = cudaFuncSetAttribute(spmm_kernel<T, NCH, LPR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    const unsigned grid = (unsigned)ceil_div(p.n, (int64_t)kSpmmWarps * rows_per_warp);
+    spmm_kernel<T, NCH, LPR><<<grid, kSpmmThreads, smem, s>>>(p, rows_per_warp);
     return cudaGetLastError();
 }
 
@@ -281,7 +451,7 @@ cudaError_t dispatch(cudaStream_t s, const SpmmDev& p)
     if (nv <= 8) return launch_one<T, 1, 8>(s, p);
     if (nv <= 16) return launch_one<T, 1, 16>(s, p);
     if (nv <= 32) return launch_one<T, 1, 32>(s, p);
-    // wider rows: up to 512 columns in any format (128 / 64 / 32 vectors of fp32 / int16 / int8)
+    // wider rows: up to 512 columns in any format (128 / 64 / 32 vectors of 4- / 2- / 1-byte elements)
     if constexpr (sizeof(T) >= 2) {
         if (nv <= 64) return launch_one<T, 2, 32>(s, p);
     }
@@ -320,6 +490,7 @@ cudaError_t launch_spmm(cudaStream_t s, const SpmmArgs& a, int* launches)
     ++*launches;
     switch (a.fmt) {
         case kZetaF32: return dispatch<float>(s, p);
+        case kZetaF16: return dispatch<__half>(s, p);
         case kZetaI16: return dispatch<int16_t>(s, p);
         case kZetaI8: return dispatch<int8_t>(s, p);
         default: return cudaErrorInvalidValue;

@@ -14,7 +14,7 @@ from parity_util import (ATOL, RTOL, assert_close, bits_from_dev, bits_to_dev, d
 
 pytestmark = pytest.mark.gpu
 
-FORMATS = [1, 2, 3]          # fp32 zeta, int16 dots, int8 dots (falls back to int16 when d_in > 127)
+FORMATS = [1, 2, 3, 4]       # fp32 zeta; integer dots as int16 / int8 (d_in <= 127) / fp16 (d_in <= 2048)
 
 
 @pytest.fixture(scope="module")
