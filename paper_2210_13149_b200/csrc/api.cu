@@ -107,7 +107,7 @@ bigcn_status check_layer(bigcn_ctx* ctx, const bigcn_layer* l, const char* name)
 
 // One layer on already validated arguments.  `zeta` is scratch for n * zeta_ld(d_out) elements.
 bigcn_status run_layer(bigcn_ctx* ctx, const bigcn_graph* g, const bigcn_layer* layer,
-                       const uint32_t* in_bits, const float* in_beta, void* zeta,
+                       const uint32_t* in_bits, const float* in_beta, void* zeta, void* scratch,
                        float* h_out, int64_t ldh, const bigcn_layer* next, uint32_t* next_bits,
                        float* next_beta, int32_t* dbg_dot, float* dbg_zeta,
                        cudaEvent_t ev_mid /*nullable*/)
@@ -139,8 +139,8 @@ bigcn_status run_layer(bigcn_ctx* ctx, const bigcn_graph* g, const bigcn_layer* 
     a.next_shift = next ? next->in_shift : nullptr;
     a.next_scale = next ? next->in_scale : nullptr;
     a.long_row = ctx->long_row > 0 ? ctx->long_row : kDefaultLongRow;
-    a.scratch = nullptr;
-    a.scratch_bytes = 0;
+    a.scratch = scratch;
+    a.scratch_bytes = spmm_scratch_bytes(g->n, g->nnz, layer->d_out);
     e = launch_spmm(ctx->stream, a, &ctx->launches_i);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "SpMM launch");
     return BIGCN_OK;
@@ -174,13 +174,14 @@ bigcn_status forward_impl(bigcn_ctx* ctx, const bigcn_graph* graph, const bigcn_
     int64_t stride_max = 0;
     for (int l = 0; l < n_layers; ++l) stride_max = stride_max > bigcn_packed_stride_words(dims[l]) ? stride_max : bigcn_packed_stride_words(dims[l]);
     void* zeta = ws.take(zeta_bytes_max(n, dims, n_layers));
+    void* scratch = ws.take(spmm_scratch_bytes(n, graph->nnz, 0));
     uint32_t* bits[2];
     float* beta[2];
     for (int i = 0; i < 2; ++i) {
         bits[i] = static_cast<uint32_t*>(ws.take((size_t)n * stride_max * 4));
         beta[i] = static_cast<float*>(ws.take((size_t)n * 4));
     }
-    if (!zeta || !bits[0] || !beta[0] || !bits[1] || !beta[1])
+    if (!zeta || !scratch || !bits[0] || !beta[0] || !bits[1] || !beta[1])
         return fail(ctx, BIGCN_ERR_WORKSPACE, "workspace of %zu bytes is too small (see bigcn_workspace_bytes)", ws.size);
 
     cudaEvent_t* ev = ctx->ev;
@@ -198,7 +199,7 @@ bigcn_status forward_impl(bigcn_ctx* ctx, const bigcn_graph* graph, const bigcn_
     for (int l = 0; l < n_layers; ++l) {
         const bool last = (l == n_layers - 1);
         const int o = (l + 1) & 1;
-        bigcn_status st = run_layer(ctx, graph, &layers[l], cur_bits, cur_beta, zeta,
+        bigcn_status st = run_layer(ctx, graph, &layers[l], cur_bits, cur_beta, zeta, scratch,
                                     last ? logits_out : nullptr, ldo, last ? nullptr : &layers[l + 1],
                                     bits[o], beta[o], nullptr, nullptr, stats ? ev[2 + 2 * l] : nullptr);
         if (st != BIGCN_OK) return st;
@@ -336,7 +337,6 @@ int64_t bigcn_packed_stride_words(int32_t len)
 
 size_t bigcn_workspace_bytes(int64_t n, int64_t nnz, const int32_t* dims, int32_t n_layers, int32_t host_io)
 {
-    (void)nnz;
     if (n < 0 || !dims || n_layers < 1 || n_layers > BIGCN_MAX_LAYERS) return 0;
     int64_t stride_max = 0;
     int32_t d_max = 0;
@@ -345,7 +345,7 @@ size_t bigcn_workspace_bytes(int64_t n, int64_t nnz, const int32_t* dims, int32_
         if (l < n_layers && bigcn_packed_stride_words(dims[l]) > stride_max) stride_max = bigcn_packed_stride_words(dims[l]);
         if (dims[l] > d_max) d_max = dims[l];
     }
-    size_t total = up(zeta_bytes_max(n, dims, n_layers));
+    size_t total = up(zeta_bytes_max(n, dims, n_layers)) + up(spmm_scratch_bytes(n, nnz, 0));
     total += 2 * (up((size_t)n * stride_max * 4) + up((size_t)n * 4));
     size_t aux = up(normalize_scratch_bytes(n));
     if (up(col_stats_scratch_bytes(d_max)) > aux) aux = up(col_stats_scratch_bytes(d_max));
@@ -458,9 +458,10 @@ bigcn_status bigcn_layer_forward(bigcn_ctx* ctx, const bigcn_graph* graph, const
     if (next && (!next_bits || !next_beta)) return fail(ctx, BIGCN_ERR_NULL, "next_bits or next_beta is null");
     if (!h_out && !next) return fail(ctx, BIGCN_ERR_NULL, "neither h_out nor next is given: nothing to compute");
     const int32_t dims[2] = {layer->d_in, layer->d_out};
-    const size_t need = up(zeta_bytes_max(graph->n, dims, 1));
+    const size_t zbytes = up(zeta_bytes_max(graph->n, dims, 1));
+    const size_t need = zbytes + up(spmm_scratch_bytes(graph->n, graph->nnz, layer->d_out));
     if (!ctx->ws || ctx->ws_bytes < need) return fail(ctx, BIGCN_ERR_WORKSPACE, "needs %zu bytes of workspace, has %zu", need, ctx->ws_bytes);
-    st = run_layer(ctx, graph, layer, in_bits, in_beta, ctx->ws, h_out, ldh, next, next_bits, next_beta,
+    st = run_layer(ctx, graph, layer, in_bits, in_beta, ctx->ws, static_cast<char*>(ctx->ws) + zbytes, h_out, ldh, next, next_bits, next_beta,
                    dbg_dot, dbg_zeta, nullptr);
     finish_call(ctx);
     return st;

@@ -14,9 +14,13 @@
 // chunks ahead in registers.  There is no waiting on other warps or blocks anywhere:
 // cp.async.wait_group only waits for the calling thread's own copies.
 //
+// Runs of rows are handed out to warps through an atomic counter in global memory (zeroed by the
+// launcher), so that warps with heavy rows do not hold back the others; which warp computes a row
+// does not change how the row is computed, so results never depend on scheduling.
+//
 // Rows with more stored entries than `long_row` are left out of the streams and processed afterwards
 // by all warps of the thread block together (each warp a contiguous slice, partial sums combined
-// through shared memory in warp order), so results never depend on scheduling.
+// through shared memory in warp order).
 #include <cuda_fp16.h>
 
 #include <algorithm>
@@ -29,7 +33,8 @@ namespace {
 
 constexpr int kSpmmWarps = 8;
 constexpr int kSpmmThreads = kSpmmWarps * kWarp;
-constexpr int kMaxRowsPerWarp = 16;      // consecutive rows streamed by one warp
+constexpr int kMaxRowsPerWarp = 16;      // consecutive rows handed to a warp at a time
+constexpr int kLongQueue = 96;           // long rows a thread block can queue for cooperative processing
 
 // Element types of a zeta row and their conversion to fp32 (one 16-byte vector at a time).
 template <typename T> struct Elt;
@@ -100,6 +105,7 @@ struct SpmmDev {
     const float* next_shift;
     const float* next_scale;
     int64_t long_row;
+    int* run_counter;        // zeroed before the launch: next run of rows to hand out
 };
 
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
@@ -337,15 +343,15 @@ __device__ __forceinline__ void stream_entries(const SpmmDev& p, uint4* ring, fl
         cp_async_commit();                                    // one group per iteration, possibly empty
     }
     cp_async_wait<0>();
-    if (kPartial) {                                           // empty slice
+    if constexpr (kPartial) {                                 // empty slice
         reduce_groups<NCH, EPV, LPR>(acc);
-        return;
-    }
-    while (rt < row_hi) {                                     // rows without entries at the end of the run
-        reduce_groups<NCH, EPV, LPR>(acc);
-        finish_row<T, NCH, LPR>(p, warp_row0 + rt, lane, acc);
-        zero_acc<NCH, EPV>(acc);
-        ++rt;
+    } else {
+        while (rt < row_hi) {                                 // rows without entries at the end of the run
+            reduce_groups<NCH, EPV, LPR>(acc);
+            finish_row<T, NCH, LPR>(p, warp_row0 + rt, lane, acc);
+            zero_acc<NCH, EPV>(acc);
+            ++rt;
+        }
     }
 }
 
@@ -358,7 +364,7 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
     constexpr int G = P::G;
     constexpr int kCols = (LPR < 32 ? LPR : NCH * 32) * EPV;  // accumulator columns of one warp
     extern __shared__ __align__(128) unsigned char dsmem[];
-    __shared__ int long_rows[kSpmmWarps * kMaxRowsPerWarp];
+    __shared__ int64_t long_rows[kLongQueue];
     __shared__ int n_long;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -369,16 +375,24 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
     if (threadIdx.x == 0) n_long = 0;
     __syncthreads();
 
-    const int64_t block_row0 = (int64_t)blockIdx.x * kSpmmWarps * rows_per_warp;
-    const int64_t warp_row0 = block_row0 + (int64_t)warp * rows_per_warp;
-    const int n_rows = (int)max((int64_t)0, min((int64_t)rows_per_warp, p.n - warp_row0));
+    const int64_t n_runs = ceil_div(p.n, rows_per_warp);
     float acc[NCH][EPV];
-    if (n_rows > 0) {
+    for (;;) {
+        int64_t run = 0;
+        if (lane == 0) run = atomicAdd(p.run_counter, 1);
+        run = __shfl_sync(0xffffffffu, run, 0);
+        if (run >= n_runs) break;
+        const int64_t warp_row0 = run * rows_per_warp;
+        const int n_rows = (int)min((int64_t)rows_per_warp, p.n - warp_row0);
         const int64_t rp_reg = __ldg(p.rowptr + warp_row0 + min(lane, n_rows));
         const int64_t rp_next = __shfl_down_sync(0xffffffffu, rp_reg, 1);
-        const bool is_long = lane < n_rows && p.long_row > 0 && (rp_next - rp_reg) > p.long_row;
+        bool is_long = lane < n_rows && p.long_row > 0 && (rp_next - rp_reg) > p.long_row;
+        if (is_long) {                                        // queue it for the block; if the queue is full, stream it here
+            const int slot = atomicAdd(&n_long, 1);
+            if (slot < kLongQueue) long_rows[slot] = warp_row0 + lane;
+            else is_long = false;
+        }
         const unsigned long_mask = __ballot_sync(0xffffffffu, is_long);
-        if (is_long) long_rows[atomicAdd(&n_long, 1)] = (int)(warp_row0 + lane - block_row0);
         int ra = 0;
         while (ra < n_rows) {                                 // runs of rows between the long ones
             const unsigned rest = long_mask >> ra;
@@ -386,7 +400,6 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
             if (rl > ra) {
                 const int64_t e0 = __shfl_sync(0xffffffffu, rp_reg, ra);
                 const int64_t e1 = __shfl_sync(0xffffffffu, rp_reg, rl);
-                // a run holds at most kMaxRowsPerWarp * long_row entries
                 stream_entries<T, NCH, LPR, false>(p, ring, wfifo, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
                                                    (int)(rp_reg - e0), acc);
             }
@@ -394,10 +407,10 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
         }
     }
     __syncthreads();
-    const int nl = n_long;
+    const int nl = min(n_long, kLongQueue);
     // Long rows of this block, one after the other, each by all warps together.
     for (int q = 0; q < nl; ++q) {
-        const int64_t lrow = block_row0 + long_rows[q];
+        const int64_t lrow = long_rows[q];
         const int64_t ls = __ldg(p.rowptr + lrow), le = __ldg(p.rowptr + lrow + 1);
         const int64_t slice = round_up(ceil_div(le - ls, kSpmmWarps), 32);
         const int64_t s0 = min(le, ls + warp * slice), s1 = min(le, s0 + slice);
@@ -436,7 +449,11 @@ cudaError_t launch_one(cudaStream_t s, const SpmmDev& p)
         cudaError_t e = cudaFuncSetAttribute(spmm_kernel<T, NCH, LPR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    const unsigned grid = (unsigned)ceil_div(p.n, (int64_t)kSpmmWarps * rows_per_warp);
+    cudaError_t e = cudaMemsetAsync(p.run_counter, 0, sizeof(int), s);
+    if (e != cudaSuccess) return e;
+    // one wave of resident blocks; the warps pull runs of rows until none are left
+    const int64_t wanted = ceil_div(ceil_div(p.n, rows_per_warp), kSpmmWarps);
+    const unsigned grid = (unsigned)std::min<int64_t>(wanted, 148 * (NCH == 1 ? 4 : (NCH == 2 ? 2 : 1)));
     spmm_kernel<T, NCH, LPR><<<grid, kSpmmThreads, smem, s>>>(p, rows_per_warp);
     return cudaGetLastError();
 }
@@ -463,7 +480,7 @@ cudaError_t dispatch(cudaStream_t s, const SpmmDev& p)
 
 }  // namespace
 
-size_t spmm_scratch_bytes(int64_t, int64_t, int) { return 0; }
+size_t spmm_scratch_bytes(int64_t, int64_t, int) { return 256; }
 
 cudaError_t launch_spmm(cudaStream_t s, const SpmmArgs& a, int* launches)
 {
@@ -487,6 +504,8 @@ cudaError_t launch_spmm(cudaStream_t s, const SpmmArgs& a, int* launches)
     p.next_shift = a.next_shift;
     p.next_scale = a.next_scale;
     p.long_row = a.long_row;
+    if (!a.scratch || a.scratch_bytes < sizeof(int)) return cudaErrorInvalidValue;
+    p.run_counter = static_cast<int*>(a.scratch);
     ++*launches;
     switch (a.fmt) {
         case kZetaF32: return dispatch<float>(s, p);
