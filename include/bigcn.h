@@ -201,6 +201,34 @@ bigcn_status bigcn_forward_host(bigcn_ctx* ctx, const bigcn_graph* graph, const 
 bigcn_status bigcn_col_stats(bigcn_ctx* ctx, const float* H, int64_t n, int32_t d, int64_t ld,
                              float eps, float* shift_out, float* scale_out);
 
+/* One layer without any allocation (the paper has no counterpart of this call; it is a packaging of
+ * bigcn_layer_forward() for callers that must not allocate device memory: a process whose own pool
+ * took the whole GPU at start-up, so that cudaMalloc would fail, or a latency-critical loop that
+ * cannot afford the device-wide synchronisation an allocation implies).
+ * It needs no context and no workspace: the scratch between the bit-GEMM and the aggregation
+ * lives in a fixed array of BIGCN_NOALLOC_SCRATCH_BYTES inside the library's device image (held by
+ * every GPU that loads the library until the process exits).  It never calls cudaMalloc, cudaFree
+ * or any allocating routine.
+ *   cuda_stream  the cudaStream_t to enqueue on (0 = default stream); the device that owns it
+ *                must be the calling thread's current device.
+ *   other arguments and results: exactly as bigcn_layer_forward(), default option values, without
+ *   the debug taps.  Results are the same as that call's.
+ * Limits and rules:
+ *   - n * round_up(d_out, 8) * 2 bytes (4 bytes per element and round_up(d_out, 4) when d_in > 32767)
+ *     must not exceed BIGCN_NOALLOC_SCRATCH_BYTES - 256; a larger problem is refused with
+ *     BIGCN_ERR_WORKSPACE before anything is launched.
+ *   - The first call on a device looks up the array's device address (once per device); make that
+ *     first call before starting any stream capture on that device.
+ *   - All calls in a process share the one array, and it keeps what the previous call left; the call
+ *     itself rewrites everything it later reads, so a stale content is harmless, but two calls whose
+ *     GPU work overlaps (different streams, or different threads) race on it: keep them ordered.
+ * Returns a status only (there is no context to hold a message). */
+#define BIGCN_NOALLOC_SCRATCH_BYTES (8u * 1024u * 1024u)
+bigcn_status bigcn_layer_forward_noalloc(void* cuda_stream, const bigcn_graph* graph, const bigcn_layer* layer,
+                                         const uint32_t* in_bits, const float* in_beta,
+                                         float* h_out, int64_t ldh,
+                                         const bigcn_layer* next, uint32_t* next_bits, float* next_beta);
+
 #ifdef __cplusplus
 }
 #endif

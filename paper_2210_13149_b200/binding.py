@@ -65,7 +65,11 @@ SIGNATURES = {
     "bigcn_forward_host": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer), _i32,
                                           _vp, _i64, _vp, _i64]),
     "bigcn_col_stats": (ctypes.c_int, [_vp, _vp, _i64, _i32, _i64, ctypes.c_float, _vp, _vp]),
+    "bigcn_layer_forward_noalloc": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer),
+                                                   _vp, _vp, _vp, _i64, ctypes.POINTER(bigcn_layer), _vp, _vp]),
 }
+
+NOALLOC_SCRATCH_BYTES = 8 * 1024 * 1024
 
 _lib = None
 
@@ -148,6 +152,24 @@ def _layer_array(layers: Sequence[Layer]):
     for i, l in enumerate(layers):
         arr[i] = l.c
     return arr
+
+
+def layer_forward_noalloc(graph: "Graph", layer: "Layer", in_bits: torch.Tensor, in_beta: torch.Tensor,
+                          h_out: Optional[torch.Tensor] = None, next_layer: Optional["Layer"] = None,
+                          next_bits: Optional[torch.Tensor] = None, next_beta: Optional[torch.Tensor] = None,
+                          stream: Optional[torch.cuda.Stream] = None) -> int:
+    """bigcn_layer_forward_noalloc(): one layer for callers that must not allocate device memory.
+
+    Needs no context and no workspace (the scratch is a fixed array inside the library) and this
+    wrapper allocates nothing either: every output tensor is passed in by the caller.  Returns the
+    status code (0 = ok; 5 = the problem does not fit the built-in scratch).  Calls must not overlap
+    on the GPU: they share the one scratch array."""
+    lib = load()
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(lib.bigcn_layer_forward_noalloc(
+        ctypes.c_void_p(s.cuda_stream), ctypes.byref(graph.c), ctypes.byref(layer.c), _ptr(in_bits), _ptr(in_beta),
+        _ptr(h_out), h_out.stride(0) if h_out is not None else 0,
+        ctypes.byref(next_layer.c) if next_layer is not None else None, _ptr(next_bits), _ptr(next_beta)))
 
 
 class BiGCN:
