@@ -208,18 +208,14 @@ def traffic_record(kernel_key):
 
 def run_ours(args):
     import torch
-    import torch.distributed as dist
-    from paper_2210_13149_b200 import binding, synth
+    from paper_2210_13149_b200 import binding, replicas, synth
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, local, world = replicas.env_rank()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
+    replicas.init("nccl", dev)
 
     wl = synth.make_workload(args.config, scale=args.scale, device=dev)
     spec = wl.spec
@@ -261,8 +257,7 @@ def run_ours(args):
     ctx._prep_forward(G, layers, host_io=not args.no_e2e)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
 
     for _ in range(max(args.warmup, 3)):
@@ -289,12 +284,7 @@ def run_ours(args):
     elapsed_ms = ev0.elapsed_time(ev1)
     launches = ctx.launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
-    if world > 1:
-        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
-    ms_per_step = elapsed_ms / args.steps
-    value = world * n / (ms_per_step * 1e-3)
+    value, ms_per_step = replicas.throughput(elapsed_ms / args.steps, n, dev)
 
     # end to end through the host-buffer entry point: pinned X in, logits out, every step
     e2e = None
@@ -311,19 +301,14 @@ def run_ours(args):
             ctx.forward_host(G, layers, xh, oh)
         ev1.record()
         barrier()
-        e_ms = ev0.elapsed_time(ev1) / e_steps
-        if world > 1:
-            t = torch.tensor([e_ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
-        e2e = {"value": world * n / (e_ms * 1e-3), "unit": UNIT, "ms_per_step": e_ms, "steps": e_steps,
+        e_value, e_ms = replicas.throughput(ev0.elapsed_time(ev1) / e_steps, n, dev)
+        e2e = {"value": e_value, "unit": UNIT, "ms_per_step": e_ms, "steps": e_steps,
                "h2d_bytes_per_step": n * dims[0] * 4, "d2h_bytes_per_step": n * dims[-1] * 4,
                "api": "bigcn_forward_host (pinned host X in, host logits out)"}
         del xh, oh
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        replicas.finish()
         return
 
     # roofline of the dominant kernel: the aggregation of the layer that takes longest
@@ -385,8 +370,7 @@ def run_ours(args):
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
             "kernels": kernels}
     print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.finish()
 
 
 def main():
