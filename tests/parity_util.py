@@ -92,3 +92,59 @@ def flip_report(gpu_bits: np.ndarray, ref_F: np.ndarray, ref_H: np.ndarray, shif
     near = np.abs(centred) <= ATOL + RTOL * np.abs(ref_H.astype(np.float64))
     bad = diff & ~near
     return int(diff.sum()), int(bad.sum()), int(diff.size)
+
+
+def unpack_signs_dev(bits: torch.Tensor, d: int) -> torch.Tensor:
+    """bool [n, d] from packed int32 words [n, stride] (bit k of word w is element 32 w + k)."""
+    n = bits.shape[0]
+    shifts = torch.arange(32, device=bits.device, dtype=torch.int32)
+    b = (bits.unsqueeze(-1) >> shifts) & 1
+    return b.reshape(n, -1)[:, :d].bool()
+
+
+def end_to_end_with_flip_accounting(ctx, G, layers, run: OracleRun, X: torch.Tensor):
+    """Runs the network layer by layer on the GPU's own intermediate results and checks it against
+    the oracle: every fp32 output row that is not downstream of a re-binarization disagreement must be
+    within tolerance, and every disagreement that is not itself downstream of an earlier one must sit
+    at the threshold (the oracle's pre-sign value within the fp32 tolerance of it).
+
+    Returns a dict with the counts that are reported: threshold flips per layer, share of output rows
+    downstream of a flip, share of logits outside tolerance overall, argmax agreement."""
+    n = G.n
+    A = torch.sparse_csr_tensor(G.rowptr, G.colidx.long(), torch.ones_like(G.val), size=(n, n))
+    L = len(layers)
+    bits, beta = ctx.pack_features(X, layers[0].in_shift, layers[0].in_scale)
+    assert torch.equal(bits, bits_to_dev(run.traces[0].bits)), "first-layer packed bits differ from the oracle"
+    dirty = torch.zeros(n, dtype=torch.bool, device=X.device)          # rows whose packed input differs
+    report = {"origin_flips": [], "dirty_rows": []}
+    for l in range(L):
+        t = run.traces[l]
+        nxt = layers[l + 1] if l + 1 < L else None
+        out = ctx.layer_forward(G, layers[l], bits, beta, want_h=True, next_layer=nxt)
+        tainted = (A @ dirty.to(torch.float32).unsqueeze(1)).squeeze(1) > 0    # rows that gather a differing row
+        ref = dev(t.H_out)
+        err = (out["h"].double() - ref.double()).abs()
+        allow = ATOL + RTOL * ref.double().abs()
+        clean_bad = ((err > allow).any(1) & ~tainted).sum().item()
+        assert clean_bad == 0, "layer %d: %d rows outside tolerance that no sign flip explains" % (l, clean_bad)
+        if nxt is None:
+            report["logit_rows_downstream_of_flips"] = float(tainted.double().mean())
+            report["logits_outside_tolerance"] = float((err > allow).double().mean())
+            report["max_abs_err"] = float(err.max())
+            report["argmax_agreement"] = float((out["h"].argmax(1) == ref.argmax(1)).double().mean())
+            break
+        tn = run.traces[l + 1]
+        got = unpack_signs_dev(out["next_bits"], layers[l].d_out)
+        want = dev(tn.F) > 0
+        diff = got != want
+        mu = dev(run.layers[l + 1].in_shift).double() if run.layers[l + 1].in_shift is not None else 0.0
+        near = (ref.double() - mu).abs() <= allow
+        origin = diff & ~tainted.unsqueeze(1)
+        bad = int((origin & ~near).sum())
+        assert bad == 0, "layer %d: %d sign flips away from the threshold" % (l, bad)
+        report["origin_flips"].append(int(origin.sum()))
+        dirty = diff.any(1) | (err > allow).any(1)       # rows whose packed bits or scale are no longer the oracle's
+        report["dirty_rows"].append(int(dirty.sum()))
+        bits, beta = out["next_bits"], out["next_beta"]
+        del out, got, want, diff, near, origin, err, allow, ref
+    return report
