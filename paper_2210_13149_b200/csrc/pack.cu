@@ -1,5 +1,7 @@
 // Binarization + bit packing of node features (rows) and weights (columns).
 // Bi-GCN Sec. 4.2.1 (Eq. "B", "alpha"), Sec. 4.2.2 (Eq. "F", "beta"), Sec. 4.4 (batch-normalised input).
+#include <algorithm>
+
 #include "bigcn_internal.cuh"
 
 namespace bigcn {
@@ -8,43 +10,79 @@ namespace {
 
 constexpr int kPackWarpsPerBlock = 8;
 
-// One warp per row.  Lane l reads element 32 w + l of the row (128 contiguous bytes per warp load,
-// whatever the row's alignment), so the ballot of "x >= 0" IS packed word w.  Up to 32 words are
-// kept one per lane and stored with a single coalesced write.
-template <bool kNorm>
+// A warp packs R rows at a time.  Lane l reads element 32 w + l of a row (128 contiguous bytes per
+// warp load, whatever the row's alignment), so the ballot of "x >= 0" IS packed word w.  The loads of
+// a chunk of WC words of all R rows are issued before any of them is used (R * WC loads of 128 bytes
+// in flight per warp), and warps loop over the rows of the matrix (persistent grid).  Up to 32 words
+// per row are kept one per lane and stored with a single coalesced write.  The R row sums of |x| are
+// reduced together: each exchange step halves the rows a lane still carries.
+template <bool kNorm, int R, int WC>
 __global__ void __launch_bounds__(kPackWarpsPerBlock* kWarp)
 pack_rows_kernel(const float* __restrict__ H, int64_t n, int d, int64_t ld,
                  const float* __restrict__ shift, const float* __restrict__ scale,
                  uint32_t* __restrict__ bits, int64_t stride, float* __restrict__ beta)
 {
     const int lane = threadIdx.x & 31;
-    const int64_t row = (int64_t)blockIdx.x * kPackWarpsPerBlock + (threadIdx.x >> 5);
-    if (row >= n) return;
-    const float* __restrict__ h = H + row * ld;
-    uint32_t* __restrict__ out = bits + row * stride;
+    const int64_t warp_id = (int64_t)blockIdx.x * kPackWarpsPerBlock + (threadIdx.x >> 5);
+    const int64_t n_warps = (int64_t)gridDim.x * kPackWarpsPerBlock;
     const int kw = (d + 31) >> 5;
-    float l1 = 0.f;
-    for (int w0 = 0; w0 < stride; w0 += 32) {
-        uint32_t mine = 0u;
-        const int wend = min(32, kw - w0);
-#pragma unroll 4
-        for (int ww = 0; ww < wend; ++ww) {
-            const int j = ((w0 + ww) << 5) + lane;
-            bool pos = false;
-            if (j < d) {
-                float x = __ldg(h + j);
-                if (kNorm) x = __fmul_rn(__fsub_rn(x, __ldg(shift + j)), __ldg(scale + j));
-                pos = x >= 0.f;
-                l1 += fabsf(x);
-            }
-            const uint32_t word = __ballot_sync(0xffffffffu, pos);
-            if (lane == ww) mine = word;
-        }
-        if (w0 + lane < stride) out[w0 + lane] = mine;
-    }
+    const float inv_d = 1.f / (float)d;
+    for (int64_t row0 = warp_id * R; row0 < n; row0 += n_warps * R) {
+        float l1[R];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) l1 += __shfl_xor_sync(0xffffffffu, l1, o);
-    if (lane == 0) beta[row] = l1 / (float)d;
+        for (int r = 0; r < R; ++r) l1[r] = 0.f;
+        for (int w0 = 0; w0 < stride; w0 += 32) {
+            uint32_t mine[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) mine[r] = 0u;
+            const int wlast = min(w0 + 32, kw);
+            for (int c0 = w0; c0 < wlast; c0 += WC) {
+                float x[R][WC];
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+#pragma unroll
+                    for (int q = 0; q < WC; ++q) {
+                        const int j = ((c0 + q) << 5) + lane;
+                        x[r][q] = (row0 + r < n && j < d) ? __ldg(H + (row0 + r) * ld + j) : 0.f;
+                    }
+#pragma unroll
+                for (int q = 0; q < WC; ++q) {
+                    const int j = ((c0 + q) << 5) + lane;
+                    const bool in = j < d;
+                    float sh = 0.f, sc = 1.f;
+                    if (kNorm && in) { sh = __ldg(shift + j); sc = __ldg(scale + j); }
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        float v = x[r][q];
+                        if (kNorm) v = __fmul_rn(__fsub_rn(v, sh), sc);
+                        const bool pos = in && (v >= 0.f);
+                        if (in) l1[r] += fabsf(v);
+                        const uint32_t word = __ballot_sync(0xffffffffu, pos);
+                        if (lane == c0 + q - w0) mine[r] = word;
+                    }
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+                if (row0 + r < n && w0 + lane < stride) bits[(row0 + r) * stride + w0 + lane] = mine[r];
+        }
+        // reduce the R row sums: after the halving steps lane L carries row L / (32 / R)
+        int off = 16;
+#pragma unroll
+        for (int half = R / 2; half >= 1; half /= 2, off /= 2) {
+            const bool upper = (lane & off) != 0;
+#pragma unroll
+            for (int i = 0; i < half; ++i) {
+                const float send = upper ? l1[i] : l1[i + half];
+                const float keep = upper ? l1[i + half] : l1[i];
+                l1[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+            }
+        }
+        for (int o = off; o >= 1; o /= 2) l1[0] += __shfl_xor_sync(0xffffffffu, l1[0], o);
+        constexpr int kLanesPerRow = 32 / R;
+        const int64_t row = row0 + lane / kLanesPerRow;
+        if (lane % kLanesPerRow == 0 && row < n) beta[row] = l1[0] * inv_d;
+    }
 }
 
 // Weights: W is [d_in x d_out] row-major and the packed output is transposed (one row per output
@@ -95,12 +133,24 @@ cudaError_t launch_pack_rows(cudaStream_t s, const float* H, int64_t n, int d, i
                              uint32_t* bits, int64_t stride, float* beta, int* launches)
 {
     if (n == 0) return cudaSuccess;
-    const unsigned grid = (unsigned)ceil_div(n, kPackWarpsPerBlock);
+    const int kw = (d + 31) / 32;
+    const int rows = kw <= 4 ? 8 : (kw <= 8 ? 4 : (kw <= 32 ? 2 : 1));     // rows a warp packs at a time
+    const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, (int64_t)kPackWarpsPerBlock * rows), 148 * 8);
     const dim3 block(kPackWarpsPerBlock * kWarp);
-    if (shift)
-        pack_rows_kernel<true><<<grid, block, 0, s>>>(H, n, d, ld, shift, scale, bits, stride, beta);
-    else
-        pack_rows_kernel<false><<<grid, block, 0, s>>>(H, n, d, ld, nullptr, nullptr, bits, stride, beta);
+#define BIGCN_PACK_LAUNCH(NORM, R, WC) \
+    pack_rows_kernel<NORM, R, WC><<<grid, block, 0, s>>>(H, n, d, ld, shift, scale, bits, stride, beta)
+    if (shift) {
+        if (rows == 8) BIGCN_PACK_LAUNCH(true, 8, 4);
+        else if (rows == 4) BIGCN_PACK_LAUNCH(true, 4, 8);
+        else if (rows == 2) BIGCN_PACK_LAUNCH(true, 2, 8);
+        else BIGCN_PACK_LAUNCH(true, 1, 8);
+    } else {
+        if (rows == 8) BIGCN_PACK_LAUNCH(false, 8, 4);
+        else if (rows == 4) BIGCN_PACK_LAUNCH(false, 4, 8);
+        else if (rows == 2) BIGCN_PACK_LAUNCH(false, 2, 8);
+        else BIGCN_PACK_LAUNCH(false, 1, 8);
+    }
+#undef BIGCN_PACK_LAUNCH
     ++*launches;
     return cudaGetLastError();
 }
