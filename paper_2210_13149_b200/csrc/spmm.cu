@@ -105,6 +105,8 @@ struct SpmmDev {
     const float* next_shift;
     const float* next_scale;
     int64_t long_row;
+    int covered_words;       // packed words of the next layer that the zeta columns cover
+    float inv_d_out;
     int* run_counter;        // zeroed before the launch: next run of rows to hand out
 };
 
@@ -190,11 +192,10 @@ __device__ __forceinline__ void finish_row(const SpmmDev& p, int64_t row, int la
         }
     }
     if (p.next_bits) {
-        const int covered = (int)ceil_div((int64_t)p.nv * EPV, 32);
-        for (int w = covered + lane; w < p.next_stride; w += 32) p.next_bits[row * p.next_stride + w] = 0u;
+        for (int w = p.covered_words + lane; w < p.next_stride; w += 32) p.next_bits[row * p.next_stride + w] = 0u;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) l1 += __shfl_xor_sync(0xffffffffu, l1, o);
-        if (lane == 0) p.next_beta[row] = l1 / (float)p.d_out;
+        if (lane == 0) p.next_beta[row] = l1 * p.inv_d_out;
     }
 }
 
@@ -202,7 +203,7 @@ template <int NCH, int LPR>
 struct Pipe {
     static constexpr int G = kWarp / LPR;                       // entries per position
     static constexpr int PB = (4 * G <= 32) ? 4 : 32 / G;       // positions per group (PB * G divides 32)
-    static constexpr int NG = NCH == 1 ? 3 : 2;                 // groups in flight per warp
+    static constexpr int NG = NCH > 1 ? 2 : (LPR == 32 ? 4 : 3);  // groups in flight per warp (a power of two for wide rows)
     static constexpr int RING = PB * NG;                        // slots of NCH * 512 bytes
     static constexpr size_t kWarpBytes = (size_t)RING * (NCH * 512 + G * 4);
 };
@@ -355,8 +356,183 @@ __device__ __forceinline__ void stream_entries(const SpmmDev& p, uint4* ring, fl
     }
 }
 
+// acc[0..EPV) += w * (the EPV elements of one 16-byte vector), using the packed two-lane fp32 FMA
+// of sm_100 where the element type converts pairwise.
+template <typename T>
+__device__ __forceinline__ void fma_vec(float w, const uint4& v, float (&acc)[Elt<T>::kPerVec])
+{
+    constexpr int EPV = Elt<T>::kPerVec;
+    if constexpr (sizeof(T) == 1) {
+        float f[EPV];
+        Elt<T>::unpack(v, f);
+#pragma unroll
+        for (int i = 0; i < EPV; ++i) acc[i] = fmaf(w, f[i], acc[i]);
+    } else {
+        float f[EPV];
+        Elt<T>::unpack(v, f);
+        const float2 ww = make_float2(w, w);
+#pragma unroll
+        for (int i = 0; i < EPV; i += 2) {
+            const float2 r = __ffma2_rn(ww, make_float2(f[i], f[i + 1]), make_float2(acc[i], acc[i + 1]));
+            acc[i] = r.x;
+            acc[i + 1] = r.y;
+        }
+    }
+}
+
+__device__ __forceinline__ void cp_async16_s(uint32_t smem_dst, const void* gmem_src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
+
+// The same stream for wide rows (LPR = 32: one stored entry per position, the common hot case), laid
+// out so that the inner loop carries no row-boundary logic: a group of PB positions never straddles a
+// row.  A row with `deg` entries takes ceil(deg / PB) groups (at least one, so that rows without
+// entries are still written); the unused positions of a row's last group are simply not copied and
+// not accumulated.  The issue cursor and the retire cursor walk the rows in the same way, NG groups
+// apart.  Column indices and weights of the next entries sit in two ready 32-entry chunks (A, B) so
+// that a group may reach past a chunk boundary; two more chunks (C, D) are in flight behind them.
+// Full groups (the usual case) take straight-line code on both sides.
+template <typename T, int NCH, bool kPartial>
+__device__ __forceinline__ void stream_rows_wide(const SpmmDev& p, uint4* ring, float* wfifo, int lane,
+                                                 int64_t e0, int n_ent, int64_t warp_row0, int row_lo,
+                                                 int row_hi, int rp_rel,
+                                                 float (&acc)[NCH][Elt<T>::kPerVec])
+{
+    using P = Pipe<NCH, 32>;
+    constexpr int EPV = Elt<T>::kPerVec;
+    constexpr int PB = P::PB, NG = P::NG;
+    static_assert(PB == 4 && (NG & (NG - 1)) == 0, "float4 weight reads; power-of-two group ring");
+    constexpr int kSlotVecs = NCH * 32;                       // 16-byte vectors per slot
+    bool active[NCH];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) active[c] = (c * 32 + lane) < p.nv;
+    const int32_t* cols = p.colidx + e0;
+    const float* vals = p.val + e0;
+    auto load_col = [&](int e) { return e < n_ent ? __ldg(cols + e) : 0; };
+    auto load_val = [&](int e) { return e < n_ent ? __ldg(vals + e) : 0.f; };
+    auto load_nw = [&](int col) { return p.node_w ? __ldg(p.node_w + col) : 1.f; };
+    auto row_end_of = [&](int r) { return kPartial ? n_ent : __shfl_sync(0xffffffffu, rp_rel, r + 1); };
+    const uint4* ring_l = ring + lane;                        // this lane's vector of slot 0
+    const uint32_t ring_sa = (uint32_t)__cvta_generic_to_shared(ring_l);
+    const char* zeta_l = reinterpret_cast<const char*>(p.zeta + lane);
+    const uint32_t row_bytes = (uint32_t)p.nv * 16u;
+
+    int a_col = load_col(lane), b_col = load_col(32 + lane), c_col = load_col(64 + lane), d_col = load_col(96 + lane);
+    float a_w = load_val(lane), b_w = load_val(32 + lane), c_val = load_val(64 + lane), d_val = load_val(96 + lane);
+    a_w *= load_nw(a_col);
+    b_w *= load_nw(b_col);
+    float c_nw = load_nw(c_col);
+    int cbase = 0;                                            // first entry of chunk A
+
+    int ie = 0, ir = row_lo, iend = row_end_of(row_lo);       // issue cursor: entry, row, end of that row
+    int re = 0, rr = row_lo, rend = iend;                     // retire cursor
+    bool more = row_lo < row_hi;
+    int issued = 0, goff = 0;                                 // groups issued; ring position of the current group
+    zero_acc<NCH, EPV>(acc);
+
+    for (int it = 0;; ++it) {
+        if (it >= NG) {
+            if (it - NG >= issued) break;
+            // ---- retire the oldest group
+            cp_async_wait<NG - 1>();
+            __syncwarp();
+            const uint4* gp = ring_l + goff * (PB * kSlotVecs);
+            uint4 v[PB][NCH];
+#pragma unroll
+            for (int b = 0; b < PB; ++b)
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) v[b][c] = gp[b * kSlotVecs + c * 32];
+            const float4 w4 = *reinterpret_cast<const float4*>(wfifo + goff * PB);
+            const float w[PB] = {w4.x, w4.y, w4.z, w4.w};
+            const int left = rend - re;
+            if (left >= PB) {
+#pragma unroll
+                for (int b = 0; b < PB; ++b)
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c)
+                        if (NCH == 1 || active[c]) fma_vec<T>(w[b], v[b][c], acc[c]);
+                re += PB;
+            } else {
+#pragma unroll
+                for (int b = 0; b < PB - 1; ++b)
+                    if (b < left) {
+#pragma unroll
+                        for (int c = 0; c < NCH; ++c)
+                            if (NCH == 1 || active[c]) fma_vec<T>(w[b], v[b][c], acc[c]);
+                    }
+                re = rend;
+            }
+            if (re == rend) {                                 // the row is complete
+                if (kPartial) return;
+                finish_row<T, NCH, 32>(p, warp_row0 + rr, lane, acc);
+                zero_acc<NCH, EPV>(acc);
+                ++rr;
+                if (rr < row_hi) rend = row_end_of(rr);
+            }
+            __syncwarp();                                     // all lanes are done with these slots
+        }
+        if (more) {
+            // ---- issue the next group of the row under the issue cursor
+            const int left = iend - ie;
+            const int base = ie - cbase;                      // position of the group in chunk A (< 32)
+            const uint32_t dsta = ring_sa + goff * (PB * kSlotVecs * 16);
+            if (left >= PB && base <= 32 - PB) {
+#pragma unroll
+                for (int b = 0; b < PB; ++b) {
+                    const uint32_t k = (uint32_t)__shfl_sync(0xffffffffu, a_col, base + b);
+                    const char* src = zeta_l + (uint64_t)k * row_bytes;
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c)
+                        if (NCH == 1 || active[c]) cp_async16_s(dsta + (b * kSlotVecs + c * 32) * 16, src + c * 512);
+                }
+                if ((unsigned)(lane - base) < (unsigned)PB) wfifo[goff * PB + lane - base] = a_w;
+                ie += PB;
+            } else {
+                const int cnt = min(PB, left);
+#pragma unroll
+                for (int b = 0; b < PB; ++b)
+                    if (b < cnt) {
+                        const int idx = base + b;
+                        const uint32_t k = (uint32_t)(idx < 32 ? __shfl_sync(0xffffffffu, a_col, idx)
+                                                               : __shfl_sync(0xffffffffu, b_col, idx - 32));
+                        const char* src = zeta_l + (uint64_t)k * row_bytes;
+#pragma unroll
+                        for (int c = 0; c < NCH; ++c)
+                            if (NCH == 1 || active[c]) cp_async16_s(dsta + (b * kSlotVecs + c * 32) * 16, src + c * 512);
+                    }
+                const int rel = lane - base;                  // the lanes that hold these entries write their weights
+                if (rel >= 0 && rel < cnt) wfifo[goff * PB + rel] = a_w;
+                if (rel + 32 < cnt) wfifo[goff * PB + rel + 32] = b_w;
+                ie += cnt;
+            }
+            ++issued;
+            if (ie == iend) {
+                ++ir;
+                if (ir == row_hi) more = false;
+                else iend = row_end_of(ir);
+            }
+            if (ie - cbase >= 32) {                           // rotate the metadata chunks
+                a_col = b_col;
+                a_w = b_w;
+                b_col = c_col;
+                b_w = c_val * c_nw;
+                c_col = d_col;
+                c_val = d_val;
+                c_nw = load_nw(c_col);
+                cbase += 32;
+                d_col = load_col(cbase + 96 + lane);
+                d_val = load_val(cbase + 96 + lane);
+            }
+        }
+        cp_async_commit();                                    // one group per iteration, possibly empty
+        goff = (goff + 1) & (NG - 1);
+    }
+    cp_async_wait<0>();
+}
+
 template <typename T, int NCH, int LPR>
-__global__ void __launch_bounds__(kSpmmThreads, NCH == 1 ? 4 : (NCH == 2 ? 2 : 1))
+__global__ void __launch_bounds__(kSpmmThreads, NCH == 1 ? (LPR == 32 ? 3 : 4) : (NCH == 2 ? 2 : 1))
 spmm_kernel(const SpmmDev p, int rows_per_warp)
 {
     using P = Pipe<NCH, LPR>;
@@ -400,8 +576,12 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
             if (rl > ra) {
                 const int64_t e0 = __shfl_sync(0xffffffffu, rp_reg, ra);
                 const int64_t e1 = __shfl_sync(0xffffffffu, rp_reg, rl);
-                stream_entries<T, NCH, LPR, false>(p, ring, wfifo, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
-                                                   (int)(rp_reg - e0), acc);
+                if constexpr (LPR == 32)
+                    stream_rows_wide<T, NCH, false>(p, ring, wfifo, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
+                                                    (int)(rp_reg - e0), acc);
+                else
+                    stream_entries<T, NCH, LPR, false>(p, ring, wfifo, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
+                                                       (int)(rp_reg - e0), acc);
             }
             ra = rl + 1;
         }
@@ -414,7 +594,10 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
         const int64_t ls = __ldg(p.rowptr + lrow), le = __ldg(p.rowptr + lrow + 1);
         const int64_t slice = round_up(ceil_div(le - ls, kSpmmWarps), 32);
         const int64_t s0 = min(le, ls + warp * slice), s1 = min(le, s0 + slice);
-        stream_entries<T, NCH, LPR, true>(p, ring, wfifo, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
+        if constexpr (LPR == 32)
+            stream_rows_wide<T, NCH, true>(p, ring, wfifo, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
+        else
+            stream_entries<T, NCH, LPR, true>(p, ring, wfifo, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
         __syncthreads();                                      // every ring is idle: reuse them for the partial sums
         const int l = lane % LPR;
         if (lane < LPR) {
@@ -453,7 +636,7 @@ cudaError_t launch_one(cudaStream_t s, const SpmmDev& p)
     if (e != cudaSuccess) return e;
     // one wave of resident blocks; the warps pull runs of rows until none are left
     const int64_t wanted = ceil_div(ceil_div(p.n, rows_per_warp), kSpmmWarps);
-    const unsigned grid = (unsigned)std::min<int64_t>(wanted, 148 * (NCH == 1 ? 4 : (NCH == 2 ? 2 : 1)));
+    const unsigned grid = (unsigned)std::min<int64_t>(wanted, 148 * (NCH == 1 ? (LPR == 32 ? 3 : 4) : (NCH == 2 ? 2 : 1)));
     spmm_kernel<T, NCH, LPR><<<grid, kSpmmThreads, smem, s>>>(p, rows_per_warp);
     return cudaGetLastError();
 }
@@ -504,6 +687,8 @@ cudaError_t launch_spmm(cudaStream_t s, const SpmmArgs& a, int* launches)
     p.next_shift = a.next_shift;
     p.next_scale = a.next_scale;
     p.long_row = a.long_row;
+    p.covered_words = (int)ceil_div(a.ldz, 32);
+    p.inv_d_out = 1.f / (float)a.d_out;
     if (!a.scratch || a.scratch_bytes < sizeof(int)) return cudaErrorInvalidValue;
     p.run_counter = static_cast<int*>(a.scratch);
     ++*launches;
