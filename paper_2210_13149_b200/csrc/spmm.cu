@@ -392,8 +392,9 @@ __device__ __forceinline__ void cp_async16_s(uint32_t smem_dst, const void* gmem
 // not accumulated.  The issue cursor and the retire cursor walk the rows in the same way, NG groups
 // apart.  Column indices and weights of the next entries sit in two ready 32-entry chunks (A, B) so
 // that a group may reach past a chunk boundary; two more chunks (C, D) are in flight behind them.
-// Full groups (the usual case) take straight-line code on both sides.
-template <typename T, int NCH, bool kPartial>
+// Full groups (the usual case) take straight-line code on both sides.  kFull: every lane of a position
+// holds a vector of the row (nv = 32 * NCH), so no lane needs masking.
+template <typename T, int NCH, bool kFull, bool kPartial>
 __device__ __forceinline__ void stream_rows_wide(const SpmmDev& p, uint4* ring, float* wfifo, int lane,
                                                  int64_t e0, int n_ent, int64_t warp_row0, int row_lo,
                                                  int row_hi, int rp_rel,
@@ -451,7 +452,7 @@ __device__ __forceinline__ void stream_rows_wide(const SpmmDev& p, uint4* ring, 
                 for (int b = 0; b < PB; ++b)
 #pragma unroll
                     for (int c = 0; c < NCH; ++c)
-                        if (NCH == 1 || active[c]) fma_vec<T>(w[b], v[b][c], acc[c]);
+                        if (kFull || active[c]) fma_vec<T>(w[b], v[b][c], acc[c]);
                 re += PB;
             } else {
 #pragma unroll
@@ -459,7 +460,7 @@ __device__ __forceinline__ void stream_rows_wide(const SpmmDev& p, uint4* ring, 
                     if (b < left) {
 #pragma unroll
                         for (int c = 0; c < NCH; ++c)
-                            if (NCH == 1 || active[c]) fma_vec<T>(w[b], v[b][c], acc[c]);
+                            if (kFull || active[c]) fma_vec<T>(w[b], v[b][c], acc[c]);
                     }
                 re = rend;
             }
@@ -484,7 +485,7 @@ __device__ __forceinline__ void stream_rows_wide(const SpmmDev& p, uint4* ring, 
                     const char* src = zeta_l + (uint64_t)k * row_bytes;
 #pragma unroll
                     for (int c = 0; c < NCH; ++c)
-                        if (NCH == 1 || active[c]) cp_async16_s(dsta + (b * kSlotVecs + c * 32) * 16, src + c * 512);
+                        if (kFull || active[c]) cp_async16_s(dsta + (b * kSlotVecs + c * 32) * 16, src + c * 512);
                 }
                 if ((unsigned)(lane - base) < (unsigned)PB) wfifo[goff * PB + lane - base] = a_w;
                 ie += PB;
@@ -499,7 +500,7 @@ __device__ __forceinline__ void stream_rows_wide(const SpmmDev& p, uint4* ring, 
                         const char* src = zeta_l + (uint64_t)k * row_bytes;
 #pragma unroll
                         for (int c = 0; c < NCH; ++c)
-                            if (NCH == 1 || active[c]) cp_async16_s(dsta + (b * kSlotVecs + c * 32) * 16, src + c * 512);
+                            if (kFull || active[c]) cp_async16_s(dsta + (b * kSlotVecs + c * 32) * 16, src + c * 512);
                     }
                 const int rel = lane - base;                  // the lanes that hold these entries write their weights
                 if (rel >= 0 && rel < cnt) wfifo[goff * PB + rel] = a_w;
@@ -531,7 +532,7 @@ __device__ __forceinline__ void stream_rows_wide(const SpmmDev& p, uint4* ring, 
     cp_async_wait<0>();
 }
 
-template <typename T, int NCH, int LPR>
+template <typename T, int NCH, int LPR, bool kFull>
 __global__ void __launch_bounds__(kSpmmThreads, NCH == 1 ? (LPR == 32 ? 3 : 4) : (NCH == 2 ? 2 : 1))
 spmm_kernel(const SpmmDev p, int rows_per_warp)
 {
@@ -577,7 +578,7 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
                 const int64_t e0 = __shfl_sync(0xffffffffu, rp_reg, ra);
                 const int64_t e1 = __shfl_sync(0xffffffffu, rp_reg, rl);
                 if constexpr (LPR == 32)
-                    stream_rows_wide<T, NCH, false>(p, ring, wfifo, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
+                    stream_rows_wide<T, NCH, kFull, false>(p, ring, wfifo, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
                                                     (int)(rp_reg - e0), acc);
                 else
                     stream_entries<T, NCH, LPR, false>(p, ring, wfifo, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
@@ -595,7 +596,7 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
         const int64_t slice = round_up(ceil_div(le - ls, kSpmmWarps), 32);
         const int64_t s0 = min(le, ls + warp * slice), s1 = min(le, s0 + slice);
         if constexpr (LPR == 32)
-            stream_rows_wide<T, NCH, true>(p, ring, wfifo, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
+            stream_rows_wide<T, NCH, kFull, true>(p, ring, wfifo, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
         else
             stream_entries<T, NCH, LPR, true>(p, ring, wfifo, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
         __syncthreads();                                      // every ring is idle: reuse them for the partial sums
@@ -622,14 +623,14 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
     }
 }
 
-template <typename T, int NCH, int LPR>
+template <typename T, int NCH, int LPR, bool kFull = false>
 cudaError_t launch_one(cudaStream_t s, const SpmmDev& p)
 {
     constexpr size_t smem = kSpmmWarps * Pipe<NCH, LPR>::kWarpBytes;
     // enough thread blocks to fill the machine on small graphs, long runs of rows on large ones
     const int rows_per_warp = (int)std::min<int64_t>(kMaxRowsPerWarp, std::max<int64_t>(1, p.n / (kSpmmWarps * 148 * 8)));
     if (smem > 40 * 1024) {                                   // above the default limit: opt in
-        cudaError_t e = cudaFuncSetAttribute(spmm_kernel<T, NCH, LPR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(spmm_kernel<T, NCH, LPR, kFull>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
     cudaError_t e = cudaMemsetAsync(p.run_counter, 0, sizeof(int), s);
@@ -637,7 +638,7 @@ cudaError_t launch_one(cudaStream_t s, const SpmmDev& p)
     // one wave of resident blocks; the warps pull runs of rows until none are left
     const int64_t wanted = ceil_div(ceil_div(p.n, rows_per_warp), kSpmmWarps);
     const unsigned grid = (unsigned)std::min<int64_t>(wanted, 148 * (NCH == 1 ? (LPR == 32 ? 3 : 4) : (NCH == 2 ? 2 : 1)));
-    spmm_kernel<T, NCH, LPR><<<grid, kSpmmThreads, smem, s>>>(p, rows_per_warp);
+    spmm_kernel<T, NCH, LPR, kFull><<<grid, kSpmmThreads, smem, s>>>(p, rows_per_warp);
     return cudaGetLastError();
 }
 
@@ -650,6 +651,7 @@ cudaError_t dispatch(cudaStream_t s, const SpmmDev& p)
     if (nv <= 4) return launch_one<T, 1, 4>(s, p);
     if (nv <= 8) return launch_one<T, 1, 8>(s, p);
     if (nv <= 16) return launch_one<T, 1, 16>(s, p);
+    if (nv == 32) return launch_one<T, 1, 32, true>(s, p);
     if (nv <= 32) return launch_one<T, 1, 32>(s, p);
     // wider rows: up to 512 columns in any format (128 / 64 / 32 vectors of 4- / 2- / 1-byte elements)
     if constexpr (sizeof(T) >= 2) {

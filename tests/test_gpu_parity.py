@@ -138,7 +138,7 @@ def test_col_stats(ctx):
 LAYER_SHAPES = [(200, 1500, 1, 1), (300, 2500, 33, 7), (500, 6000, 100, 256), (400, 5000, 602, 256),
                 (350, 3000, 1433, 64), (250, 2000, 3703, 64), (600, 9000, 256, 47), (600, 9000, 256, 41),
                 (700, 5000, 64, 3), (450, 4000, 64, 6), (300, 3000, 256, 256), (260, 3000, 127, 100),
-                (260, 3000, 128, 512)]
+                (260, 3000, 128, 512), (300, 3000, 64, 200)]
 
 
 @pytest.mark.parametrize("fmt", FORMATS)
