@@ -21,13 +21,13 @@ constexpr int kTM = 4;                                  // rows held in register
 // the 32 lanes of a warp - 32 consecutive channels - hit 32 different banks) and one tile of packed
 // feature rows (read as warp-wide broadcasts).  Each lane owns channels lane, lane+32, ... (TN of
 // them) and kTM rows at a time: kTM x TN integer accumulators of popc(a XOR b).
-template <int TN>
+template <int TN, int FMT, bool DBG>
 __global__ void __launch_bounds__(kGemmThreads)
 bitgemm_kernel(const uint32_t* __restrict__ A, int64_t stride_a,
                const uint32_t* __restrict__ BT, int64_t stride_b,
                int64_t n, int d_in, int d_out, int kw, int ldb,
                const float* __restrict__ beta, const float* __restrict__ alpha,
-               int fmt, void* __restrict__ zeta, int64_t ldz,
+               void* __restrict__ zeta, int64_t ldz,
                int32_t* __restrict__ dbg_dot, float* __restrict__ dbg_zeta)
 {
     extern __shared__ __align__(16) uint32_t smem[];
@@ -51,6 +51,7 @@ bitgemm_kernel(const uint32_t* __restrict__ A, int64_t stride_a,
 
     const int64_t n_tiles = ceil_div(n, kTileRows);
     const int sa4 = (int)(stride_a >> 2);
+    const bool small_k = d_in <= 511;
     for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
         const int64_t r0 = tile * kTileRows;
         const int rows_here = (int)min((int64_t)kTileRows, n - r0);
@@ -96,16 +97,27 @@ bitgemm_kernel(const uint32_t* __restrict__ A, int64_t stride_a,
                     const int j = jblock + lane + 32 * t;
                     const int dot = d_in - 2 * acc[m][t];
                     if (j < d_out) {
-                        const float z = __fmul_rn(__fmul_rn(be, al[t]), (float)dot);
-                        if (fmt == kZetaF32) reinterpret_cast<float*>(zeta)[row * ldz + j] = z;
-                        else if (fmt == kZetaF16) reinterpret_cast<__half*>(zeta)[row * ldz + j] = __int2half_rn(dot);   // exact: |dot| <= 2048
-                        else if (fmt == kZetaI16) reinterpret_cast<int16_t*>(zeta)[row * ldz + j] = (int16_t)dot;
-                        else reinterpret_cast<int8_t*>(zeta)[row * ldz + j] = (int8_t)dot;
-                        if (dbg_dot) dbg_dot[row * (int64_t)d_out + j] = dot;
-                        if (dbg_zeta) dbg_zeta[row * (int64_t)d_out + j] = z;
+                        if constexpr (FMT == kZetaF16) {
+                            // exact integer -> fp16; for |dot| <= 511 without the conversion unit (which the bit
+                            // counts keep busy): the bit pattern 0x6600 + dot IS the half 1536 + dot
+                            __half h;
+                            if (small_k) h = __hsub(__ushort_as_half((unsigned short)(0x6600 + dot)), __ushort_as_half((unsigned short)0x6600));
+                            else h = __int2half_rn(dot);                                   // exact: |dot| <= 2048
+                            reinterpret_cast<__half*>(zeta)[row * ldz + j] = h;
+                        } else if constexpr (FMT == kZetaF32) {
+                            reinterpret_cast<float*>(zeta)[row * ldz + j] = __fmul_rn(__fmul_rn(be, al[t]), (float)dot);
+                        } else if constexpr (FMT == kZetaI16) {
+                            reinterpret_cast<int16_t*>(zeta)[row * ldz + j] = (int16_t)dot;
+                        } else {
+                            reinterpret_cast<int8_t*>(zeta)[row * ldz + j] = (int8_t)dot;
+                        }
+                        if constexpr (DBG) {
+                            if (dbg_dot) dbg_dot[row * (int64_t)d_out + j] = dot;
+                            if (dbg_zeta) dbg_zeta[row * (int64_t)d_out + j] = __fmul_rn(__fmul_rn(be, al[t]), (float)dot);
+                        }
                     } else if (j < ldz) {                  // padding columns of the zeta row: keep them zero
-                        if (fmt == kZetaF32) reinterpret_cast<float*>(zeta)[row * ldz + j] = 0.f;
-                        else if (fmt == kZetaI8) reinterpret_cast<int8_t*>(zeta)[row * ldz + j] = 0;
+                        if constexpr (FMT == kZetaF32) reinterpret_cast<float*>(zeta)[row * ldz + j] = 0.f;
+                        else if constexpr (FMT == kZetaI8) reinterpret_cast<int8_t*>(zeta)[row * ldz + j] = 0;
                         else reinterpret_cast<int16_t*>(zeta)[row * ldz + j] = 0;          // int16 and fp16 zero alike
                     }
                 }
@@ -114,24 +126,43 @@ bitgemm_kernel(const uint32_t* __restrict__ A, int64_t stride_a,
     }
 }
 
-template <int TN>
-cudaError_t launch_tn(cudaStream_t s, const uint32_t* A, int64_t stride_a, const uint32_t* BT,
-                      int64_t stride_b, int64_t n, int d_in, int d_out, const float* beta,
-                      const float* alpha, int fmt, void* zeta, int64_t ldz, int32_t* dbg_dot,
-                      float* dbg_zeta, size_t smem_bytes, int ldb)
+template <int TN, int FMT, bool DBG>
+cudaError_t launch_inst(cudaStream_t s, const uint32_t* A, int64_t stride_a, const uint32_t* BT,
+                        int64_t stride_b, int64_t n, int d_in, int d_out, const float* beta,
+                        const float* alpha, void* zeta, int64_t ldz, int32_t* dbg_dot,
+                        float* dbg_zeta, size_t smem_bytes, int ldb)
 {
     const int kw = (d_in + 31) / 32;
     if (smem_bytes > 48 * 1024) {                          // opt in to large dynamic shared memory
-        cudaError_t e = cudaFuncSetAttribute(bitgemm_kernel<TN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(bitgemm_kernel<TN, FMT, DBG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)smem_bytes);
         if (e != cudaSuccess) return e;
     }
     const int64_t n_tiles = ceil_div(n, kTileRows);
     const unsigned gy = (unsigned)ceil_div(d_out, TN * 32);
     const unsigned gx = (unsigned)std::min<int64_t>(n_tiles, 148 * 8);
-    bitgemm_kernel<TN><<<dim3(gx, gy), kGemmThreads, smem_bytes, s>>>(
-        A, stride_a, BT, stride_b, n, d_in, d_out, kw, ldb, beta, alpha, fmt, zeta, ldz, dbg_dot, dbg_zeta);
+    bitgemm_kernel<TN, FMT, DBG><<<dim3(gx, gy), kGemmThreads, smem_bytes, s>>>(
+        A, stride_a, BT, stride_b, n, d_in, d_out, kw, ldb, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta);
     return cudaGetLastError();
+}
+
+template <int TN>
+cudaError_t launch_tn(cudaStream_t s, const uint32_t* A, int64_t stride_a, const uint32_t* BT,
+                      int64_t stride_b, int64_t n, int d_in, int d_out, const float* beta,
+                      const float* alpha, int fmt, void* zeta, int64_t ldz, int32_t* dbg_dot,
+                      float* dbg_zeta, size_t smem_bytes, int ldb)
+{
+#define BIGCN_GEMM_CALL(FMT, DBG) \
+    launch_inst<TN, FMT, DBG>(s, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, smem_bytes, ldb)
+    const bool dbg = dbg_dot || dbg_zeta;
+    switch (fmt) {
+        case kZetaF32: return dbg ? BIGCN_GEMM_CALL(kZetaF32, true) : BIGCN_GEMM_CALL(kZetaF32, false);
+        case kZetaF16: return dbg ? BIGCN_GEMM_CALL(kZetaF16, true) : BIGCN_GEMM_CALL(kZetaF16, false);
+        case kZetaI16: return dbg ? BIGCN_GEMM_CALL(kZetaI16, true) : BIGCN_GEMM_CALL(kZetaI16, false);
+        case kZetaI8: return dbg ? BIGCN_GEMM_CALL(kZetaI8, true) : BIGCN_GEMM_CALL(kZetaI8, false);
+        default: return cudaErrorInvalidValue;
+    }
+#undef BIGCN_GEMM_CALL
 }
 
 }  // namespace
