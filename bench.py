@@ -39,6 +39,7 @@ def parse_args():
     ap.add_argument("--zeta-format", type=int, default=0, help="0 auto, 1 fp32, 2 int16, 3 int8, 4 fp16")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--graph", action="store_true", help="also time the forward replayed as one CUDA graph")
     ap.add_argument("--cpu-sample-scale", type=float, default=None)
     ap.add_argument("--scale", type=float, default=None,
                     help="shrink nodes and edges of the workload by this factor (profiling on a small case)")
@@ -270,12 +271,13 @@ def run_ours(args):
         time.sleep(0.25)
     launches0 = ctx.launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    per_kernel = {"pack": [], "gemm": [[] for _ in range(L)], "spmm": [[] for _ in range(L)]}
+    per_kernel = {"pack": [], "gemm": [[] for _ in range(L)], "spmm": [[] for _ in range(L)], "step": []}
     barrier()
     ev0.record()
     for _ in range(args.steps):
         _, st = ctx.forward(G, layers, X, logits, stats=True)
         per_kernel["pack"].append(st.ms_pack)
+        per_kernel["step"].append(st.ms_total)
         for l in range(L):
             per_kernel["gemm"][l].append(st.ms_gemm[l])
             per_kernel["spmm"][l].append(st.ms_spmm[l])
@@ -285,6 +287,54 @@ def run_ours(args):
     launches = ctx.launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
     value, ms_per_step = replicas.throughput(elapsed_ms / args.steps, n, dev)
+
+    # side measurements (not part of `value`): the same forward from already-binary input (Sec. 5.2 of
+    # the paper: the loaded data is binary), and replayed as one CUDA graph (the small workloads are
+    # bound by launch latency)
+    extras = {}
+    if rank == 0:
+        xb, xbeta = ctx.pack_features(X, layers[0].in_shift, layers[0].in_scale)
+        for _ in range(3):
+            ctx.forward_packed(G, layers, xb, xbeta, logits)
+        barrier_local = torch.cuda.synchronize
+        barrier_local()
+        ev0.record()
+        for _ in range(args.steps):
+            ctx.forward_packed(G, layers, xb, xbeta, logits)
+        ev1.record()
+        barrier_local()
+        extras["packed_input_ms_per_step"] = ev0.elapsed_time(ev1) / args.steps
+        del xb, xbeta
+        if args.graph or ms_per_step < 2.0:
+            try:
+                side = torch.cuda.Stream()
+                gctx = binding.BiGCN(local, stream=side)
+                gctx._prep_forward(G, layers)
+                with torch.cuda.stream(side):
+                    for _ in range(3):
+                        gctx.forward(G, layers, X, logits)
+                side.synchronize()
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    gctx.forward(G, layers, X, logits)
+                for _ in range(3):
+                    graph.replay()
+                torch.cuda.synchronize()
+                reps = max(args.steps, 50)
+                ev0.record()
+                for _ in range(reps):
+                    graph.replay()
+                ev1.record()
+                torch.cuda.synchronize()
+                extras["cuda_graph_ms_per_step"] = ev0.elapsed_time(ev1) / reps
+                del graph
+                gctx.close()
+            except Exception as exc:
+                extras["cuda_graph_ms_per_step"] = "failed: %r" % (exc,)
+        try:
+            extras["popc_word_steps_per_s"] = ctx.measure_popc_peak()
+        except Exception as exc:
+            extras["popc_word_steps_per_s"] = None
 
     # end to end through the host-buffer entry point: pinned X in, logits out, every step
     e2e = None
@@ -337,7 +387,11 @@ def run_ours(args):
                                    "GBps_lower_model": lower / t / 1e9, "GBps_no_reuse_model": upper / t / 1e9,
                                    "bytes_cached_model": expected, "row_bytes": ldz * elt, "zeta_format": {1: "f32", 2: "i16", 3: "i8", 4: "f16"}[f]}
         ops = 2.0 * n * dims[l] * dims[l + 1]
+        words = n * dims[l + 1] * ((dims[l] + 31) // 32)                  # XOR + bit-count + add steps
+        popc_peak = extras.get("popc_word_steps_per_s")
         kernels["bitgemm_l%d" % l] = {"ms": gemm_ms[l], "binary_TOPS": ops / (gemm_ms[l] * 1e-3) / 1e12,
+                                      "word_steps_per_s": words / (gemm_ms[l] * 1e-3),
+                                      "frac_of_popc_peak": (words / (gemm_ms[l] * 1e-3) / popc_peak) if popc_peak else None,
                                       "out_GBps": n * ldz * elt / (gemm_ms[l] * 1e-3) / 1e9}
     pack_bytes = n * (dims[0] * 4.0 + binding.packed_stride_words(dims[0]) * 4.0 + 4.0)
     kernels["pack_features"] = {"ms": pack_ms, "GBps": pack_bytes / (pack_ms * 1e-3) / 1e9,
@@ -368,7 +422,8 @@ def run_ours(args):
                        "parallelism": "replicas" if world > 1 else "single-gpu",
                        "zeta_format": {0: "auto(f16)", 1: "f32", 2: "i16", 3: "i8", 4: "f16"}[args.zeta_format]},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
-            "kernels": kernels}
+            "step_ms_median": statistics.median(per_kernel["step"]), "step_ms_min": min(per_kernel["step"]),
+            "extras": extras, "kernels": kernels}
     print(json.dumps(line), flush=True)
     replicas.finish()
 

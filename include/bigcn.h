@@ -201,6 +201,12 @@ bigcn_status bigcn_forward_host(bigcn_ctx* ctx, const bigcn_graph* graph, const 
 bigcn_status bigcn_col_stats(bigcn_ctx* ctx, const float* H, int64_t n, int32_t d, int64_t ld,
                              float eps, float* shift_out, float* scale_out);
 
+/* Measurement aid: the rate at which this GPU retires the step the contraction of Eq. "bi-op" is made
+ * of (XOR, bit count and add on one 32-bit word per lane), from a register-only loop; the result, in
+ * word steps per second, is the denominator of the bit-GEMM's roofline fraction (x 64 = binary ops/s).
+ * Needs 1.2 MB of workspace.  SYNCHRONOUS. */
+bigcn_status bigcn_measure_popc_peak(bigcn_ctx* ctx, double* word_steps_per_s /*host*/);
+
 /* One layer without any allocation (the paper has no counterpart of this call; it is a packaging of
  * bigcn_layer_forward() for callers that must not allocate device memory: a process whose own pool
  * took the whole GPU at start-up, so that cudaMalloc would fail, or a latency-critical loop that

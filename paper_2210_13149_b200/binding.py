@@ -65,6 +65,7 @@ SIGNATURES = {
     "bigcn_forward_host": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer), _i32,
                                           _vp, _i64, _vp, _i64]),
     "bigcn_col_stats": (ctypes.c_int, [_vp, _vp, _i64, _i32, _i64, ctypes.c_float, _vp, _vp]),
+    "bigcn_measure_popc_peak": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_double)]),
     "bigcn_layer_forward_noalloc": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer),
                                                    _vp, _vp, _vp, _i64, ctypes.POINTER(bigcn_layer), _vp, _vp]),
 }
@@ -331,6 +332,13 @@ class BiGCN:
         self._check(self.lib.bigcn_col_stats(self.h, _ptr(H), n, d, H.stride(0) if n > 1 else d, eps,
                                              _ptr(shift), _ptr(scale)))
         return shift, scale
+
+    def measure_popc_peak(self) -> float:
+        """32-bit XOR + bit-count + add steps per second of this GPU (register-only probe)."""
+        self.ensure_workspace(2 << 20)
+        out = ctypes.c_double(0.0)
+        self._check(self.lib.bigcn_measure_popc_peak(self.h, ctypes.byref(out)))
+        return float(out.value)
 
     # -- convenience built only from the calls above
     def prepare_layers(self, weights: Sequence[torch.Tensor], shifts=None, scales=None) -> List[Layer]:

@@ -538,4 +538,16 @@ bigcn_status bigcn_col_stats(bigcn_ctx* ctx, const float* H, int64_t n, int32_t 
     return BIGCN_OK;
 }
 
+bigcn_status bigcn_measure_popc_peak(bigcn_ctx* ctx, double* word_steps_per_s)
+{
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    if (!word_steps_per_s) return fail(ctx, BIGCN_ERR_NULL, "word_steps_per_s is null");
+    if (!ctx->ws || ctx->ws_bytes < popc_peak_scratch_bytes()) return fail(ctx, BIGCN_ERR_WORKSPACE, "needs %zu bytes of workspace", popc_peak_scratch_bytes());
+    cudaError_t e = measure_popc_peak(ctx->stream, ctx->ws, word_steps_per_s, &ctx->launches_i);
+    finish_call(ctx);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "popcount peak measurement");
+    return BIGCN_OK;
+}
+
 }  // extern "C"

@@ -72,4 +72,7 @@ cudaError_t launch_col_stats(cudaStream_t s, const float* H, int64_t n, int d, i
                              float* shift, float* scale, void* scratch, int* launches);
 size_t col_stats_scratch_bytes(int d);
 
+cudaError_t measure_popc_peak(cudaStream_t s, void* scratch, double* word_steps_per_s, int* launches);
+size_t popc_peak_scratch_bytes();
+
 }  // namespace bigcn
