@@ -70,6 +70,9 @@ def lib() -> ctypes.CDLL:
         L.oracle_rescale.argtypes = [_vp, _vp, _vp, _c_i64, _c_i32, _vp, _c_i64]
         L.oracle_spmm.argtypes = [_c_i64, _vp, _vp, _vp, _vp, _c_i32, _c_i64, _vp, _c_i64]
         L.oracle_cost_model.argtypes = [_c_f64, _c_f64, _vp, _c_i32, _vp]
+        L.oracle_mean_adjacency.restype = _c_i64
+        L.oracle_mean_adjacency.argtypes = [_c_i64, _c_i64, _vp, _vp, _vp, _vp, _vp, _vp]
+        L.oracle_spmm_add.argtypes = [_c_i64, _vp, _vp, _vp, _vp, _c_i32, _c_i64, _vp, _c_i64, _vp, _c_i64]
         _lib = L
     return _lib
 
@@ -307,3 +310,73 @@ def calibrate_bn(g: Graph, weights: List[np.ndarray], X: np.ndarray, bn_layers: 
         if l + 1 < len(weights):
             H = layer_forward(g, layer, H).H_out
     return layers
+
+
+# --------------------------------------------------------------------------- Bi-GraphSAGE (Sec. 4.4.2)
+
+def mean_adjacency(n: int, src, dst) -> Graph:
+    """CSR of the mean aggregator: row i holds 1/|N_i| on its distinct neighbours (no self-loop).
+    The returned Graph's ``dinv`` field holds 1/|N_i| (0 for isolated nodes)."""
+    src = _arr(src, np.int32)
+    dst = _arr(dst, np.int32)
+    m = int(src.shape[0])
+    rowptr = np.zeros(n + 1, dtype=np.int64)
+    colidx = np.zeros(max(2 * m, 1), dtype=np.int32)
+    val = np.zeros(max(2 * m, 1), dtype=np.float32)
+    inv_deg = np.zeros(n, dtype=np.float32)
+    nnz = lib().oracle_mean_adjacency(n, m, _p(src), _p(dst), _p(rowptr), _p(colidx), _p(val), _p(inv_deg))
+    if nnz < 0:
+        raise ValueError("edge list has a node id outside [0, n)")
+    return Graph(n, rowptr, colidx[:nnz].copy(), val[:nnz].copy(), inv_deg)
+
+
+def spmm_add(g: Graph, z: np.ndarray, self_term: Optional[np.ndarray]) -> np.ndarray:
+    """self_term + g @ z, both terms added in double, rounded once."""
+    z = _arr(z, np.float32)
+    d_out = z.shape[1]
+    if self_term is not None:
+        self_term = _arr(self_term, np.float32)
+        assert self_term.shape == (g.n, d_out)
+    out = np.zeros((g.n, d_out), np.float32)
+    lib().oracle_spmm_add(g.n, _p(g.rowptr), _p(g.colidx), _p(g.val), _p(z), d_out, d_out,
+                          _p(self_term), d_out, _p(out), d_out)
+    return out
+
+
+@dataclass
+class SageLayer:
+    """One binarized GraphSAGE layer (mean aggregator): weights of the node itself and of its
+    neighbours, and the optional batch-norm constants of the layer input."""
+    W_self: np.ndarray
+    W_nbr: np.ndarray
+    in_shift: Optional[np.ndarray] = None
+    in_scale: Optional[np.ndarray] = None
+
+
+@dataclass
+class SageTrace:
+    F: np.ndarray
+    beta: np.ndarray
+    bits: np.ndarray
+    bitsT_self: np.ndarray
+    alpha_self: np.ndarray
+    bitsT_nbr: np.ndarray
+    alpha_nbr: np.ndarray
+    zeta_self: np.ndarray
+    zeta_nbr: np.ndarray
+    H_out: np.ndarray
+
+
+def sage_layer_forward(g_mean: Graph, layer: SageLayer, H: np.ndarray) -> SageTrace:
+    """Eq. "bisage-conv": h_i' = W_theta (*) h_i + (1/|N_i|) sum_j W_n (*) h_j, both products by XNOR and
+    bit count on the same binarized input, no activation."""
+    d_in = layer.W_self.shape[0]
+    F, beta = binarize_rows(H, layer.in_shift, layer.in_scale)
+    bits = pack_rows(F)
+    Bs, a_s = binarize_cols(layer.W_self)
+    Bn, a_n = binarize_cols(layer.W_nbr)
+    bT_s, bT_n = pack_cols(Bs), pack_cols(Bn)
+    z_s = rescale(dot_popc(bits, bT_s, d_in), beta, a_s)
+    z_n = rescale(dot_popc(bits, bT_n, d_in), beta, a_n)
+    H_out = spmm_add(g_mean, z_n, z_s)
+    return SageTrace(F, beta, bits, bT_s, a_s, bT_n, a_n, z_s, z_n, H_out)

@@ -28,7 +28,8 @@
  * XNOR/bit-count contraction; dense N x N products and hand-worked star/path
  * graphs for the adjacency and the aggregation; the fp32 GCN layer of Eq. 1 on
  * +-1 inputs for the whole layer; Table 1 and the C.O./M.S./D.S. columns of
- * the result tables for the cost model.  The numerical value of a full forward
+ * the result tables for the cost model; the GraphSAGE mean layer on +-1 inputs
+ * for the Bi-GraphSAGE layer.  The numerical value of a full forward
  * on the paper's datasets is "parity unpinned": the paper prints no worked
  * numerical example and the datasets are not available.
  */
@@ -302,6 +303,82 @@ void oracle_spmm(int64_t n_rows, const int64_t* rowptr, const int32_t* colidx, c
                 double a = (double)val[p];
                 const float* z = zeta + (int64_t)colidx[p] * ldz;
                 for (int32_t j = 0; j < d_out; ++j) acc[j] += a * (double)z[j];
+            }
+            for (int32_t j = 0; j < d_out; ++j) out[i * ldo + j] = (float)acc[j];
+        }
+        free(acc);
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Bi-GraphSAGE (Sec. 4.4.2, Eq. "bisage-conv"): the mean aggregator           */
+/*   h_i' = W_theta (*) h_i + (1/|N_i|) sum_{j in N_i} W_n (*) h_j             */
+/* needs the neighbourhood matrix with rows scaled by 1/|N_i|: N_i is the set  */
+/* of distinct neighbours of i (no self-loop); a node without neighbours gets  */
+/* an empty row (its neighbour term is 0).                                     */
+/* Same input convention as oracle_normalize_adjacency.  colidx/val need room  */
+/* for 2*m entries; inv_deg[i] = (float)(1.0/|N_i|), 0 for isolated nodes;     */
+/* val = inv_deg[i] on every entry of row i.  Returns nnz or -1.               */
+/* ------------------------------------------------------------------------- */
+int64_t oracle_mean_adjacency(int64_t n, int64_t m, const int32_t* src, const int32_t* dst,
+                              int64_t* rowptr, int32_t* colidx, float* val, float* inv_deg)
+{
+    int64_t* start = (int64_t*)calloc((size_t)n + 1, sizeof(int64_t));
+    if (!start) return -1;
+    for (int64_t e = 0; e < m; ++e) {
+        int32_t u = src[e], v = dst[e];
+        if (u < 0 || u >= n || v < 0 || v >= n) { free(start); return -1; }
+        if (u == v) continue;
+        start[u + 1] += 1;
+        start[v + 1] += 1;
+    }
+    for (int64_t i = 0; i < n; ++i) start[i + 1] += start[i];
+    int64_t total = start[n];
+    int32_t* tmp = (int32_t*)malloc((size_t)(total > 0 ? total : 1) * sizeof(int32_t));
+    int64_t* fill = (int64_t*)malloc((size_t)(n > 0 ? n : 1) * sizeof(int64_t));
+    if (!tmp || !fill) { free(start); free(tmp); free(fill); return -1; }
+    for (int64_t i = 0; i < n; ++i) fill[i] = start[i];
+    for (int64_t e = 0; e < m; ++e) {
+        int32_t u = src[e], v = dst[e];
+        if (u == v) continue;
+        tmp[fill[u]++] = v;
+        tmp[fill[v]++] = u;
+    }
+    rowptr[0] = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        int64_t a = start[i], b = start[i + 1];
+        qsort(tmp + a, (size_t)(b - a), sizeof(int32_t), cmp_i32);
+        int64_t kept = 0;
+        for (int64_t p = a; p < b; ++p)
+            if (p == a || tmp[p] != tmp[p - 1]) tmp[a + kept++] = tmp[p];
+        rowptr[i + 1] = rowptr[i] + kept;
+    }
+    for (int64_t i = 0; i < n; ++i) {
+        int64_t deg = rowptr[i + 1] - rowptr[i];                  /* |N_i| */
+        inv_deg[i] = deg > 0 ? (float)(1.0 / (double)deg) : 0.0f;
+        memcpy(colidx + rowptr[i], tmp + start[i], (size_t)deg * sizeof(int32_t));
+        for (int64_t p = rowptr[i]; p < rowptr[i + 1]; ++p) val[p] = inv_deg[i];
+    }
+    free(start); free(tmp); free(fill);
+    return rowptr[n];
+}
+
+/* out_i,: = self_i,: + sum_{k in row i} val_ik * z_k,:   -- the two terms of Eq. "bisage-conv"      */
+/* added in double and rounded once (self may be NULL: then this is oracle_spmm).                   */
+void oracle_spmm_add(int64_t n_rows, const int64_t* rowptr, const int32_t* colidx, const float* val,
+                     const float* z, int32_t d_out, int64_t ldz, const float* self, int64_t lds,
+                     float* out, int64_t ldo)
+{
+#pragma omp parallel
+    {
+        double* acc = (double*)malloc((size_t)(d_out > 0 ? d_out : 1) * sizeof(double));
+#pragma omp for schedule(dynamic, 64)
+        for (int64_t i = 0; i < n_rows; ++i) {
+            for (int32_t j = 0; j < d_out; ++j) acc[j] = self ? (double)self[i * lds + j] : 0.0;
+            for (int64_t p = rowptr[i]; p < rowptr[i + 1]; ++p) {
+                double a = (double)val[p];
+                const float* zr = z + (int64_t)colidx[p] * ldz;
+                for (int32_t j = 0; j < d_out; ++j) acc[j] += a * (double)zr[j];
             }
             for (int32_t j = 0; j < d_out; ++j) out[i * ldo + j] = (float)acc[j];
         }

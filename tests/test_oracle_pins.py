@@ -373,3 +373,64 @@ def test_cost_model_ratios_of_table_1_and_sec_5_3():
     for d_in, quoted in ((1433, 59), (64, 21)):
         one = oracle.cost_model(1000, 0, [d_in, 16])
         assert round(one["ops_gcn"] / one["ops_bigcn"]) == quoted
+
+
+# ------------------------------------------------------------------ Sec. 4.4.2: Bi-GraphSAGE
+
+def test_mean_adjacency_rows_average_the_neighbours():
+    rng = np.random.default_rng(61)
+    n = 30
+    pairs = random_pairs(rng, n, 60)
+    pairs = np.concatenate([pairs, pairs[:10, ::-1], np.stack([np.arange(4)] * 2, 1).astype(np.int32)])
+    keep = (pairs != 7).all(1)                       # node 7 stays isolated
+    pairs = pairs[keep]
+    g = oracle.mean_adjacency(n, pairs[:, 0], pairs[:, 1])
+    A = np.zeros((n, n))
+    for u, v in pairs.tolist():
+        if u != v:
+            A[u, v] = A[v, u] = 1.0
+    deg = A.sum(1)
+    M = to_dense(g)
+    expect = np.divide(A, deg[:, None], out=np.zeros_like(A), where=deg[:, None] > 0)
+    np.testing.assert_allclose(M, expect, rtol=1e-7, atol=0)
+    assert M[7].sum() == 0 and g.rowptr[8] == g.rowptr[7]
+    rows = M.sum(1)
+    assert np.allclose(rows[deg > 0], 1.0, rtol=1e-6) and (np.diag(M) == 0).all()
+
+
+def test_sage_layer_on_pm1_inputs_is_the_graphsage_mean_layer():
+    """H, W_theta, W_n in {+-1}: scalars are 1 and the layer is W_theta h_i + mean_j W_n h_j exactly
+    (Eq. "sage-conv" without the ReLU, which the binarized layer drops)."""
+    rng = np.random.default_rng(62)
+    n, d, c = 24, 37, 5
+    pairs = random_pairs(rng, n, 50)
+    g = oracle.mean_adjacency(n, pairs[:, 0], pairs[:, 1])
+    H = rng.choice(np.array([-1.0, 1.0], np.float32), size=(n, d))
+    Ws = rng.choice(np.array([-1.0, 1.0], np.float32), size=(d, c))
+    Wn = rng.choice(np.array([-1.0, 1.0], np.float32), size=(d, c))
+    t = oracle.sage_layer_forward(g, oracle.SageLayer(Ws, Wn), H)
+    A = np.zeros((n, n))
+    for u, v in pairs.tolist():
+        if u != v:
+            A[u, v] = A[v, u] = 1.0
+    deg = A.sum(1)
+    mean = np.divide(A, deg[:, None], out=np.zeros_like(A), where=deg[:, None] > 0)
+    ref = H.astype(np.float64) @ Ws + mean @ (H.astype(np.float64) @ Wn)
+    np.testing.assert_allclose(t.H_out, ref, rtol=1e-6, atol=1e-6)
+
+
+def test_sage_layer_general_inputs_and_distinct_weights():
+    """General inputs: the two terms use their own weights (a swap or a shared alpha would show)."""
+    rng = np.random.default_rng(63)
+    n, d, c = 15, 41, 6
+    pairs = random_pairs(rng, n, 40)
+    g = oracle.mean_adjacency(n, pairs[:, 0], pairs[:, 1])
+    H = rng.standard_normal((n, d)).astype(np.float32)
+    Ws = rng.standard_normal((d, c)).astype(np.float32)
+    Wn = (3.0 * rng.standard_normal((d, c))).astype(np.float32)
+    t = oracle.sage_layer_forward(g, oracle.SageLayer(Ws, Wn), H)
+    Ht = np.abs(H).astype(np.float64).mean(1, keepdims=True) * np.where(H >= 0, 1.0, -1.0)
+    Wst = np.abs(Ws).astype(np.float64).mean(0, keepdims=True) * np.where(Ws >= 0, 1.0, -1.0)
+    Wnt = np.abs(Wn).astype(np.float64).mean(0, keepdims=True) * np.where(Wn >= 0, 1.0, -1.0)
+    ref = Ht @ Wst + to_dense(g) @ (Ht @ Wnt)
+    np.testing.assert_allclose(t.H_out, ref, rtol=1e-5, atol=1e-6)
