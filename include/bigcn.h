@@ -201,6 +201,30 @@ bigcn_status bigcn_forward_host(bigcn_ctx* ctx, const bigcn_graph* graph, const 
 bigcn_status bigcn_col_stats(bigcn_ctx* ctx, const float* H, int64_t n, int32_t d, int64_t ld,
                              float eps, float* shift_out, float* scale_out);
 
+/* Bi-GraphSAGE with the mean aggregator (Sec. 4.4.2, Eq. "bisage-conv"):
+ *   h_i' = W_theta (*) h_i + (1/|N_i|) sum_{j in N_i} W_n (*) h_j,   no activation,
+ * both products by XNOR and bit count on the same binarized input.
+ *
+ * bigcn_mean_adjacency(): set-up, once per graph.  Same input and checks as
+ * bigcn_normalize_adjacency(); the output CSR holds, for row i, its distinct neighbours (no
+ * self-loop) with val = 1/|N_i| (computed in double, rounded to fp32); inv_deg[n] receives 1/|N_i|
+ * (0 for a node without neighbours, whose row is empty).  Outputs need nnz_in entries.  SYNCHRONOUS.
+ *
+ * bigcn_sage_layer_forward(): one layer.  mean_graph from bigcn_mean_adjacency(); self_layer and
+ * nbr_layer hold the packed W_theta and W_n (same d_in and d_out; the batch-norm fields of these two
+ * structs are not used: the input arrives already binarized); in_bits / in_beta, h_out, next,
+ * next_bits, next_beta as in bigcn_layer_forward().  Needs twice the workspace of
+ * bigcn_layer_forward() for the same sizes (bigcn_workspace_bytes with n_layers = 1, times two). */
+bigcn_status bigcn_mean_adjacency(bigcn_ctx* ctx, int64_t n, int64_t nnz_in,
+                                  const int64_t* rowptr_A, const int32_t* colidx_A,
+                                  int64_t* rowptr, int32_t* colidx, float* val, float* inv_deg,
+                                  int64_t* nnz_out /*host*/);
+bigcn_status bigcn_sage_layer_forward(bigcn_ctx* ctx, const bigcn_graph* mean_graph,
+                                      const bigcn_layer* self_layer, const bigcn_layer* nbr_layer,
+                                      const uint32_t* in_bits, const float* in_beta,
+                                      float* h_out, int64_t ldh,
+                                      const bigcn_layer* next, uint32_t* next_bits, float* next_beta);
+
 /* Measurement aid: the rate at which this GPU retires the step the contraction of Eq. "bi-op" is made
  * of (XOR, bit count and add on one 32-bit word per lane), from a register-only loop; the result, in
  * word steps per second, is the denominator of the bit-GEMM's roofline fraction (x 64 = binary ops/s).

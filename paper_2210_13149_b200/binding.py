@@ -65,6 +65,11 @@ SIGNATURES = {
     "bigcn_forward_host": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer), _i32,
                                           _vp, _i64, _vp, _i64]),
     "bigcn_col_stats": (ctypes.c_int, [_vp, _vp, _i64, _i32, _i64, ctypes.c_float, _vp, _vp]),
+    "bigcn_mean_adjacency": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp,
+                                            ctypes.POINTER(_i64)]),
+    "bigcn_sage_layer_forward": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer),
+                                                ctypes.POINTER(bigcn_layer), _vp, _vp, _vp, _i64,
+                                                ctypes.POINTER(bigcn_layer), _vp, _vp]),
     "bigcn_measure_popc_peak": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_double)]),
     "bigcn_layer_forward_noalloc": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer),
                                                    _vp, _vp, _vp, _i64, ctypes.POINTER(bigcn_layer), _vp, _vp]),
@@ -332,6 +337,38 @@ class BiGCN:
         self._check(self.lib.bigcn_col_stats(self.h, _ptr(H), n, d, H.stride(0) if n > 1 else d, eps,
                                              _ptr(shift), _ptr(scale)))
         return shift, scale
+
+    def mean_adjacency(self, rowptr_A: torch.Tensor, colidx_A: torch.Tensor) -> Graph:
+        n = rowptr_A.numel() - 1
+        nnz_in = colidx_A.numel()
+        self.ensure_workspace(16 * (n // 1024 + 2) + 64)
+        rowptr = self._empty(n + 1, torch.int64)
+        colidx = self._empty(max(nnz_in, 1), torch.int32)
+        val = self._empty(max(nnz_in, 1), torch.float32)
+        inv_deg = self._empty(n, torch.float32)
+        nnz = _i64(0)
+        self._check(self.lib.bigcn_mean_adjacency(self.h, n, nnz_in, _ptr(rowptr_A), _ptr(colidx_A),
+                                                  _ptr(rowptr), _ptr(colidx), _ptr(val), _ptr(inv_deg),
+                                                  ctypes.byref(nnz)))
+        k = int(nnz.value)
+        return make_graph(rowptr, colidx[:k], val[:k], inv_deg)
+
+    def sage_layer_forward(self, mean_graph: Graph, self_layer: Layer, nbr_layer: Layer, in_bits: torch.Tensor,
+                           in_beta: torch.Tensor, want_h: bool = True, next_layer: Optional[Layer] = None):
+        """Returns dict with h, next_bits, next_beta (those requested)."""
+        n = mean_graph.n
+        self.ensure_workspace(2 * self.workspace_bytes(n, mean_graph.nnz, [self_layer.d_in, self_layer.d_out]))
+        d_out = self_layer.d_out
+        h = self._empty((n, d_out), torch.float32) if want_h else None
+        nb = nbeta = None
+        if next_layer is not None:
+            nb = self._empty((n, packed_stride_words(d_out)), torch.int32)
+            nbeta = self._empty(n, torch.float32)
+        self._check(self.lib.bigcn_sage_layer_forward(
+            self.h, ctypes.byref(mean_graph.c), ctypes.byref(self_layer.c), ctypes.byref(nbr_layer.c),
+            _ptr(in_bits), _ptr(in_beta), _ptr(h), d_out,
+            ctypes.byref(next_layer.c) if next_layer is not None else None, _ptr(nb), _ptr(nbeta)))
+        return {"h": h, "next_bits": nb, "next_beta": nbeta}
 
     def measure_popc_peak(self) -> float:
         """32-bit XOR + bit-count + add steps per second of this GPU (register-only probe)."""

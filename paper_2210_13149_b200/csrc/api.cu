@@ -550,4 +550,113 @@ bigcn_status bigcn_measure_popc_peak(bigcn_ctx* ctx, double* word_steps_per_s)
     return BIGCN_OK;
 }
 
+bigcn_status bigcn_mean_adjacency(bigcn_ctx* ctx, int64_t n, int64_t nnz_in,
+                                  const int64_t* rowptr_A, const int32_t* colidx_A,
+                                  int64_t* rowptr, int32_t* colidx, float* val, float* inv_deg,
+                                  int64_t* nnz_out)
+{
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    if (n < 0 || n >= (int64_t(1) << 31) || nnz_in < 0) return fail(ctx, BIGCN_ERR_SHAPE, "n=%lld nnz_in=%lld out of range", (long long)n, (long long)nnz_in);
+    if (!nnz_out) return fail(ctx, BIGCN_ERR_NULL, "nnz_out is null");
+    if (!rowptr) return fail(ctx, BIGCN_ERR_NULL, "rowptr output is null");
+    *nnz_out = 0;
+    if (n == 0) {
+        BIGCN_CUDA(ctx, cudaMemsetAsync(rowptr, 0, sizeof(int64_t), ctx->stream));
+        BIGCN_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+        return BIGCN_OK;
+    }
+    if (!rowptr_A || (nnz_in > 0 && (!colidx_A || !colidx || !val)) || !inv_deg) return fail(ctx, BIGCN_ERR_NULL, "an input or output array is null");
+    if (!ctx->ws || ctx->ws_bytes < normalize_scratch_bytes(n)) return fail(ctx, BIGCN_ERR_WORKSPACE, "needs %zu bytes of workspace", normalize_scratch_bytes(n));
+    cudaError_t e = launch_normalize_adjacency(ctx->stream, n, nnz_in, rowptr_A, colidx_A, rowptr, colidx, val, inv_deg,
+                                               ctx->ws, ctx->d_flag, &ctx->launches_i, /*mean=*/true);
+    finish_call(ctx);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "mean_adjacency launch");
+    int flag = 0;
+    int64_t total = 0;
+    BIGCN_CUDA(ctx, cudaMemcpyAsync(&flag, ctx->d_flag, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+    BIGCN_CUDA(ctx, cudaMemcpyAsync(&total, rowptr + n, sizeof(int64_t), cudaMemcpyDeviceToHost, ctx->stream));
+    BIGCN_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (flag)
+        return fail(ctx, BIGCN_ERR_GRAPH, "adjacency input rejected:%s%s%s%s",
+                    (flag & 8) ? " rowptr not monotone from 0 to nnz;" : "",
+                    (flag & 2) ? " column index outside [0, n);" : "",
+                    (flag & 1) ? " columns not ascending and unique within a row;" : "",
+                    (flag & 4) ? " pattern not symmetric;" : "");
+    *nnz_out = total;
+    return BIGCN_OK;
+}
+
+bigcn_status bigcn_sage_layer_forward(bigcn_ctx* ctx, const bigcn_graph* mean_graph,
+                                      const bigcn_layer* self_layer, const bigcn_layer* nbr_layer,
+                                      const uint32_t* in_bits, const float* in_beta,
+                                      float* h_out, int64_t ldh,
+                                      const bigcn_layer* next, uint32_t* next_bits, float* next_beta)
+{
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    if ((st = check_graph(ctx, mean_graph)) != BIGCN_OK) return st;
+    if ((st = check_layer(ctx, self_layer, "self_layer")) != BIGCN_OK) return st;
+    if ((st = check_layer(ctx, nbr_layer, "nbr_layer")) != BIGCN_OK) return st;
+    if (self_layer->d_in != nbr_layer->d_in || self_layer->d_out != nbr_layer->d_out)
+        return fail(ctx, BIGCN_ERR_SHAPE, "self and neighbour weights differ in shape (%dx%d vs %dx%d)", self_layer->d_in, self_layer->d_out, nbr_layer->d_in, nbr_layer->d_out);
+    const int d_in = self_layer->d_in, d_out = self_layer->d_out;
+    if (next) {
+        if (next->d_in != d_out) return fail(ctx, BIGCN_ERR_SHAPE, "next->d_in=%d != d_out=%d", next->d_in, d_out);
+        if ((next->in_shift == nullptr) != (next->in_scale == nullptr)) return fail(ctx, BIGCN_ERR_NULL, "next: in_shift and in_scale go together");
+    }
+    if (h_out && ldh < d_out) return fail(ctx, BIGCN_ERR_SHAPE, "ldh=%lld < d_out=%d", (long long)ldh, d_out);
+    const int64_t n = mean_graph->n;
+    if (n == 0) return BIGCN_OK;
+    if (!in_bits || !in_beta) return fail(ctx, BIGCN_ERR_NULL, "in_bits or in_beta is null");
+    if (!aligned(in_bits, 16)) return fail(ctx, BIGCN_ERR_ALIGN, "in_bits must be 16-byte aligned");
+    if (next && (!next_bits || !next_beta)) return fail(ctx, BIGCN_ERR_NULL, "next_bits or next_beta is null");
+    if (!h_out && !next) return fail(ctx, BIGCN_ERR_NULL, "neither h_out nor next is given: nothing to compute");
+    const int32_t dims[2] = {d_in, d_out};
+    const size_t zbytes = up(zeta_bytes_max(n, dims, 1));                 // fp32 size: room for either form
+    const size_t need = 2 * zbytes + up(spmm_scratch_bytes(n, mean_graph->nnz, d_out));
+    if (!ctx->ws || ctx->ws_bytes < need) return fail(ctx, BIGCN_ERR_WORKSPACE, "needs %zu bytes of workspace, has %zu", need, ctx->ws_bytes);
+    char* base = static_cast<char*>(ctx->ws);
+    float* zeta_self = reinterpret_cast<float*>(base);                   // literal fp32 zeta of the node's own term
+    void* zeta_nbr = base + zbytes;
+    void* counter = base + 2 * zbytes;
+    const int64_t stride_in = bigcn_packed_stride_words(d_in);
+    const int64_t ld_self = zeta_ld(d_out, kZetaF32);
+    cudaError_t e = launch_bitgemm(ctx->stream, in_bits, stride_in, self_layer->w_bitsT, stride_in, n, d_in, d_out,
+                                   in_beta, self_layer->alpha, kZetaF32, zeta_self, ld_self, nullptr, nullptr, &ctx->launches_i);
+    if (e != cudaSuccess) { finish_call(ctx); return cuda_fail(ctx, e, "bit-GEMM (self term) launch"); }
+    const int fmt = pick_format(ctx, d_in);
+    const int64_t ldz = zeta_ld(d_out, fmt);
+    e = launch_bitgemm(ctx->stream, in_bits, stride_in, nbr_layer->w_bitsT, stride_in, n, d_in, d_out,
+                       in_beta, nbr_layer->alpha, fmt, zeta_nbr, ldz, nullptr, nullptr, &ctx->launches_i);
+    if (e != cudaSuccess) { finish_call(ctx); return cuda_fail(ctx, e, "bit-GEMM (neighbour term) launch"); }
+    SpmmArgs a;
+    a.n = n;
+    a.rowptr = mean_graph->rowptr;
+    a.colidx = mean_graph->colidx;
+    a.val = mean_graph->val;
+    a.fmt = fmt;
+    a.zeta = zeta_nbr;
+    a.ldz = ldz;
+    a.d_out = d_out;
+    a.node_w = in_beta;
+    a.col_w = nbr_layer->alpha;
+    a.add = zeta_self;
+    a.ld_add = ld_self;
+    a.h_out = h_out;
+    a.ldh = ldh;
+    a.next_bits = next ? next_bits : nullptr;
+    a.next_stride = next ? bigcn_packed_stride_words(d_out) : 0;
+    a.next_beta = next ? next_beta : nullptr;
+    a.next_shift = next ? next->in_shift : nullptr;
+    a.next_scale = next ? next->in_scale : nullptr;
+    a.long_row = ctx->long_row > 0 ? ctx->long_row : kDefaultLongRow;
+    a.scratch = counter;
+    a.scratch_bytes = spmm_scratch_bytes(n, mean_graph->nnz, d_out);
+    e = launch_spmm(ctx->stream, a, &ctx->launches_i);
+    finish_call(ctx);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "SpMM launch");
+    return BIGCN_OK;
+}
+
 }  // extern "C"

@@ -48,6 +48,8 @@ struct SpmmArgs {
     int d_out;
     const float* node_w;     // integer formats: per-source-node factor (beta), multiplied into the edge weight
     const float* col_w;      // integer formats: per-column factor (alpha), applied once per output
+    const float* add = nullptr;   // optional fp32 [n x ld_add] added to every aggregated row (Bi-GraphSAGE self term)
+    int64_t ld_add = 0;
     float* h_out;            // nullable
     int64_t ldh;
     uint32_t* next_bits;     // nullable: fused re-binarization of the output
@@ -65,7 +67,7 @@ size_t spmm_scratch_bytes(int64_t n, int64_t nnz, int d_out);
 cudaError_t launch_normalize_adjacency(cudaStream_t s, int64_t n, int64_t nnz_in,
                                        const int64_t* rowptr_A, const int32_t* colidx_A,
                                        int64_t* rowptr, int32_t* colidx, float* val, float* dinv,
-                                       void* scratch, int* d_flag, int* launches);
+                                       void* scratch, int* d_flag, int* launches, bool mean = false);
 size_t normalize_scratch_bytes(int64_t n);
 
 cudaError_t launch_col_stats(cudaStream_t s, const float* H, int64_t n, int d, int64_t ld, float eps,

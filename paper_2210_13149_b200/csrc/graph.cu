@@ -18,6 +18,7 @@ constexpr int kFlagSymmetry = 4;          // (i, j) stored without (j, i)
 constexpr int kFlagRowptr = 8;            // rowptr not monotone or not matching nnz
 
 // Pass 1: D_hat_ii = 1 + number of off-diagonal entries of row i; checks order and range.
+template <bool kMean>
 __global__ void __launch_bounds__(kRowsPerBlock* kWarp)
 degree_kernel(int64_t n, int64_t nnz_in, const int64_t* __restrict__ rowptr_A,
               const int32_t* __restrict__ colidx_A, int64_t* __restrict__ rowptr,
@@ -41,9 +42,14 @@ degree_kernel(int64_t n, int64_t nnz_in, const int64_t* __restrict__ rowptr_A,
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) off_diag += __shfl_xor_sync(0xffffffffu, off_diag, o);
         if (lane == 0) {
-            const int64_t deg_hat = (int64_t)off_diag + 1;
-            rowptr[i + 1] = deg_hat;
-            dinv[i] = (float)(1.0 / sqrt((double)deg_hat));
+            if (kMean) {                                   // mean aggregator: |N_i| entries, factor 1/|N_i|
+                rowptr[i + 1] = off_diag;
+                dinv[i] = off_diag > 0 ? (float)(1.0 / (double)off_diag) : 0.f;
+            } else {
+                const int64_t deg_hat = (int64_t)off_diag + 1;
+                rowptr[i + 1] = deg_hat;
+                dinv[i] = (float)(1.0 / sqrt((double)deg_hat));
+            }
         }
     }
     if (i == 0 && lane == 0) rowptr[0] = 0;
@@ -114,6 +120,7 @@ scan_apply_kernel(int64_t* __restrict__ x, int64_t m, const int64_t* __restrict_
 
 // Pass 2: writes row i of A_tilde (off-diagonal entries in order with the diagonal merged in) and
 // checks that every stored (i, c) has its mirror (c, i) by binary search in row c.
+template <bool kMean>
 __global__ void __launch_bounds__(kRowsPerBlock* kWarp)
 fill_kernel(int64_t n, const int64_t* __restrict__ rowptr_A, const int32_t* __restrict__ colidx_A,
             const int64_t* __restrict__ rowptr, int32_t* __restrict__ colidx, float* __restrict__ val,
@@ -131,19 +138,21 @@ fill_kernel(int64_t n, const int64_t* __restrict__ rowptr_A, const int32_t* __re
     for (int64_t q = a + lane; q < b; q += 32) below += (colidx_A[q] < (int32_t)i);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) below += __shfl_xor_sync(0xffffffffu, below, o);
-    if (lane == 0) {
+    if (!kMean && lane == 0) {
         colidx[out0 + below] = (int32_t)i;
         val[out0 + below] = __fmul_rn(di, di);
     }
+    const int n_out = (int)(rowptr[i + 1] - out0);            // stored entries of the output row
+    const int has_self = (int)(b - a) - (kMean ? n_out : n_out - 1);
     int bad = 0;
     for (int64_t q = a + lane; q < b; q += 32) {
         const int32_t c = colidx_A[q];
         if (c == (int32_t)i) continue;
         // entries before the diagonal keep their rank; the diagonal of the input (if any) is skipped
         int64_t rank = q - a;
-        if (c > (int32_t)i) rank = below + 1 + (rank - below - ((b - a) - (rowptr[i + 1] - out0 - 1)));
+        if (c > (int32_t)i) rank = rank - has_self + (kMean ? 0 : 1);
         colidx[out0 + rank] = c;
-        val[out0 + rank] = __fmul_rn(di, dinv[c]);
+        val[out0 + rank] = kMean ? di : __fmul_rn(di, dinv[c]);
         int64_t lo = rowptr_A[c], hi = rowptr_A[c + 1];      // mirror entry (c, i)
         bool found = false;
         while (lo < hi) {
@@ -212,12 +221,13 @@ size_t normalize_scratch_bytes(int64_t n) { return (size_t)(ceil_div(n, kScanBlo
 cudaError_t launch_normalize_adjacency(cudaStream_t s, int64_t n, int64_t nnz_in,
                                        const int64_t* rowptr_A, const int32_t* colidx_A,
                                        int64_t* rowptr, int32_t* colidx, float* val, float* dinv,
-                                       void* scratch, int* d_flag, int* launches)
+                                       void* scratch, int* d_flag, int* launches, bool mean)
 {
     cudaError_t e = cudaMemsetAsync(d_flag, 0, sizeof(int), s);
     if (e != cudaSuccess) return e;
     const unsigned row_blocks = (unsigned)ceil_div(n, kRowsPerBlock);
-    degree_kernel<<<row_blocks, kRowsPerBlock * kWarp, 0, s>>>(n, nnz_in, rowptr_A, colidx_A, rowptr, dinv, d_flag);
+    if (mean) degree_kernel<true><<<row_blocks, kRowsPerBlock * kWarp, 0, s>>>(n, nnz_in, rowptr_A, colidx_A, rowptr, dinv, d_flag);
+    else degree_kernel<false><<<row_blocks, kRowsPerBlock * kWarp, 0, s>>>(n, nnz_in, rowptr_A, colidx_A, rowptr, dinv, d_flag);
     ++*launches;
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     int64_t* totals = reinterpret_cast<int64_t*>(scratch);
@@ -227,7 +237,8 @@ cudaError_t launch_normalize_adjacency(cudaStream_t s, int64_t n, int64_t nnz_in
     scan_apply_kernel<<<(unsigned)nb, kScanBlock, 0, s>>>(rowptr + 1, n, totals);
     *launches += 3;
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    fill_kernel<<<row_blocks, kRowsPerBlock * kWarp, 0, s>>>(n, rowptr_A, colidx_A, rowptr, colidx, val, dinv, d_flag);
+    if (mean) fill_kernel<true><<<row_blocks, kRowsPerBlock * kWarp, 0, s>>>(n, rowptr_A, colidx_A, rowptr, colidx, val, dinv, d_flag);
+    else fill_kernel<false><<<row_blocks, kRowsPerBlock * kWarp, 0, s>>>(n, rowptr_A, colidx_A, rowptr, colidx, val, dinv, d_flag);
     ++*launches;
     return cudaGetLastError();
 }

@@ -96,6 +96,8 @@ struct SpmmDev {
     int d_out;
     const float* node_w;     // nullable
     const float* col_w;      // nullable
+    const float* add;        // nullable: fp32 [n x ld_add] added to the aggregated row (after col_w)
+    int64_t ld_add;
     float* h_out;
     int64_t ldh;
     int h_vec;               // 1: rows of h_out can be stored as float4
@@ -159,6 +161,7 @@ __device__ __forceinline__ void finish_row(const SpmmDev& p, int64_t row, int la
         for (int i = 0; i < EPV; ++i) {
             x[i] = acc[c][i];
             if (p.col_w) x[i] *= (col0 + i < p.d_out) ? __ldg(p.col_w + col0 + i) : 0.f;
+            if (p.add && col0 + i < p.d_out) x[i] += __ldg(p.add + row * p.ld_add + col0 + i);
         }
         if (p.h_out && g == 0 && vec < p.nv) {
             float* dst = p.h_out + row * p.ldh + col0;
@@ -680,6 +683,8 @@ cudaError_t launch_spmm(cudaStream_t s, const SpmmArgs& a, int* launches)
     p.d_out = a.d_out;
     p.node_w = a.fmt == kZetaF32 ? nullptr : a.node_w;
     p.col_w = a.fmt == kZetaF32 ? nullptr : a.col_w;
+    p.add = a.add;
+    p.ld_add = a.ld_add;
     p.h_out = a.h_out;
     p.ldh = a.ldh;
     p.h_vec = (a.h_out && (a.ldh % 4 == 0) && (reinterpret_cast<uintptr_t>(a.h_out) % 16 == 0)) ? 1 : 0;
