@@ -36,6 +36,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default="c5", help="workload c1..c5 (default: the largest, c5)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--model", default="gcn", choices=["gcn", "sage"],
+                    help="gcn: the Bi-GCN forward (the benchmark); sage: side benchmark of the Bi-GraphSAGE layers")
     ap.add_argument("--zeta-format", type=int, default=0, help="0 auto, 1 fp32, 2 int16, 3 int8, 4 fp16")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -428,10 +430,84 @@ def run_ours(args):
     replicas.finish()
 
 
+def run_sage(args):
+    """Side benchmark of the Bi-GraphSAGE layer stack (mean aggregator) on the same workload shapes:
+    L layers called one by one through bigcn_sage_layer_forward, hidden activations passed as packed
+    bits.  Single GPU; prints one JSON line."""
+    import torch
+    from paper_2210_13149_b200 import binding, synth
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    dev = torch.device("cuda", 0)
+    wl = synth.make_workload(args.config, scale=args.scale, device=dev)
+    spec = wl.spec
+    dims = list(spec.dims)
+    L = len(dims) - 1
+    ctx = binding.BiGCN(0)
+    G = ctx.mean_adjacency(wl.rowptr, wl.colidx)
+    n, nnz = G.n, G.nnz
+    W2 = synth.weights(spec.dims, spec.seed + 7, dev)
+    bn = wl.bn_layers()
+    pairs = []
+    for l in range(L):
+        bs, a_s = ctx.pack_weights(wl.W[l])
+        bnb, a_n = ctx.pack_weights(W2[l])
+        pairs.append([bs, a_s, bnb, a_n])
+    # calibrate the batch-norm constants layer after layer with the library's own statistics
+    layers = []
+    sh, sc = ctx.col_stats(wl.X) if bn[0] else (None, None)
+    bits, beta = ctx.pack_features(wl.X, sh, sc)
+    x_shift, x_scale = sh, sc
+    for l in range(L):
+        ls = binding.make_layer(dims[l], dims[l + 1], pairs[l][0], pairs[l][1], sh, sc)
+        ln = binding.make_layer(dims[l], dims[l + 1], pairs[l][2], pairs[l][3])
+        layers.append((ls, ln))
+        if l + 1 < L:
+            out = ctx.sage_layer_forward(G, ls, ln, bits, beta, want_h=True)
+            sh, sc = ctx.col_stats(out["h"]) if bn[l + 1] else (None, None)
+            bits, beta = ctx.pack_features(out["h"], sh, sc)
+            del out
+    del bits, beta
+
+    def step():
+        b, be = ctx.pack_features(wl.X, x_shift, x_scale)
+        for l in range(L):
+            last = l == L - 1
+            o = ctx.sage_layer_forward(G, layers[l][0], layers[l][1], b, be, want_h=last,
+                                       next_layer=None if last else layers[l + 1][0])
+            b, be = o["next_bits"], o["next_beta"]
+        return o["h"]
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.25)
+    launches0 = ctx.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    line = {"metric": "bisage_forward_nodes_per_s", "value": n / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": DTYPE, "data": "synthetic",
+            "config": {"workload": "Bi-GraphSAGE (mean aggregator) on " + workload_description(spec, n, nnz),
+                       "l2": "inputs_exceed_l2", "note": "layer-by-layer calls: pack + per layer 2 bit-GEMMs + 1 aggregation"},
+            "clocks": sampler.stop(), "gpu_launches": ctx.launch_count() - launches0}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.model == "sage":
+        run_sage(args)
     else:
         run_ours(args)
 
