@@ -142,26 +142,48 @@ __device__ __forceinline__ void reduce_groups(float (&acc)[NCH][EPV])
             for (int i = 0; i < EPV; ++i) acc[c][i] += __shfl_xor_sync(0xffffffffu, acc[c][i], o);
 }
 
+// Per-column constants of the row epilogue, staged once per thread block: three arrays of kCols
+// floats -- the column factor (0 for padding columns, 1 when there is none), then the next layer's
+// shift and scale (0 and 1 where there are none, so that applying them changes nothing).
+template <int kCols>
+__device__ __forceinline__ void fill_col_table(const SpmmDev& p, float* ctab)
+{
+    for (int col = threadIdx.x; col < kCols; col += blockDim.x) {
+        const bool in = col < p.d_out;
+        ctab[col] = in ? (p.col_w ? __ldg(p.col_w + col) : 1.f) : 0.f;
+        ctab[kCols + col] = (in && p.next_shift) ? __ldg(p.next_shift + col) : 0.f;
+        ctab[2 * kCols + col] = (in && p.next_shift) ? __ldg(p.next_scale + col) : 1.f;
+    }
+}
+
 // Writes one finished row: optional fp32 store, optional sign/scale packing for the next layer.
 // Called by a full warp; every lane holds the totals of vector(s) c*32 + (lane % LPR).
 template <typename T, int NCH, int LPR>
-__device__ __forceinline__ void finish_row(const SpmmDev& p, int64_t row, int lane,
+__device__ __forceinline__ void finish_row(const SpmmDev& p, const float* ctab, int64_t row, int lane,
                                            float (&acc)[NCH][Elt<T>::kPerVec])
 {
     constexpr int EPV = Elt<T>::kPerVec;
     constexpr int LW = 32 / EPV;                  // lanes that share one packed word
+    constexpr int kCols = (LPR < 32 ? LPR : NCH * 32) * EPV;
     const int g = lane / LPR, l = lane % LPR;
     float l1 = 0.f;
 #pragma unroll
     for (int c = 0; c < NCH; ++c) {
         const int vec = c * 32 + l;
         const int col0 = vec * EPV;
-        float x[EPV];
+        float x[EPV], sh[EPV], sc[EPV];
 #pragma unroll
-        for (int i = 0; i < EPV; ++i) {
-            x[i] = acc[c][i];
-            if (p.col_w) x[i] *= (col0 + i < p.d_out) ? __ldg(p.col_w + col0 + i) : 0.f;
-            if (p.add && col0 + i < p.d_out) x[i] += __ldg(p.add + row * p.ld_add + col0 + i);
+        for (int q = 0; q < EPV / 4; ++q) {
+            const float4 a = *reinterpret_cast<const float4*>(ctab + col0 + 4 * q);
+            x[4 * q] = acc[c][4 * q] * a.x;
+            x[4 * q + 1] = acc[c][4 * q + 1] * a.y;
+            x[4 * q + 2] = acc[c][4 * q + 2] * a.z;
+            x[4 * q + 3] = acc[c][4 * q + 3] * a.w;
+        }
+        if (p.add) {
+#pragma unroll
+            for (int i = 0; i < EPV; ++i)
+                if (col0 + i < p.d_out) x[i] += __ldg(p.add + row * p.ld_add + col0 + i);
         }
         if (p.h_out && g == 0 && vec < p.nv) {
             float* dst = p.h_out + row * p.ldh + col0;
@@ -174,18 +196,24 @@ __device__ __forceinline__ void finish_row(const SpmmDev& p, int64_t row, int la
             }
         }
         if (p.next_bits) {
+#pragma unroll
+            for (int q = 0; q < EPV / 4; ++q) {
+                const float4 a = *reinterpret_cast<const float4*>(ctab + kCols + col0 + 4 * q);
+                const float4 b = *reinterpret_cast<const float4*>(ctab + 2 * kCols + col0 + 4 * q);
+                sh[4 * q] = a.x, sh[4 * q + 1] = a.y, sh[4 * q + 2] = a.z, sh[4 * q + 3] = a.w;
+                sc[4 * q] = b.x, sc[4 * q + 1] = b.y, sc[4 * q + 2] = b.z, sc[4 * q + 3] = b.w;
+            }
             uint32_t bits = 0u;
+            float l1c = 0.f;
 #pragma unroll
             for (int i = 0; i < EPV; ++i) {
-                const int col = col0 + i;
-                if (col < p.d_out) {
-                    float xh = x[i];
-                    if (p.next_shift)
-                        xh = __fmul_rn(__fsub_rn(xh, __ldg(p.next_shift + col)), __ldg(p.next_scale + col));
-                    if (xh >= 0.f) bits |= 1u << i;
-                    if (g == 0) l1 += fabsf(xh);
-                }
+                const float xh = __fmul_rn(__fsub_rn(x[i], sh[i]), sc[i]);   // padding columns: (0 - 0) * 1
+                if (xh >= 0.f) bits |= 1u << i;
+                l1c += fabsf(xh);
             }
+            if (vec < p.nv) l1 += l1c;            // lanes past the last vector accumulated nothing meaningful
+            const int n_valid = min(max(p.d_out - col0, 0), EPV);            // padding columns pack as 0
+            bits &= (n_valid >= 32) ? 0xffffffffu : ((1u << n_valid) - 1u);
             uint32_t word = bits << ((col0) & 31);
 #pragma unroll
             for (int o = 1; o < LW; o <<= 1) word |= __shfl_xor_sync(0xffffffffu, word, o);
@@ -196,6 +224,7 @@ __device__ __forceinline__ void finish_row(const SpmmDev& p, int64_t row, int la
     }
     if (p.next_bits) {
         for (int w = p.covered_words + lane; w < p.next_stride; w += 32) p.next_bits[row * p.next_stride + w] = 0u;
+        if (g != 0) l1 = 0.f;                     // the other lane groups hold copies of the same totals
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) l1 += __shfl_xor_sync(0xffffffffu, l1, o);
         if (lane == 0) p.next_beta[row] = l1 * p.inv_d_out;
@@ -218,7 +247,7 @@ struct Pipe {
 //   kPartial = true : the entries are a slice of one long row; the slice's sum is left in `acc`
 //                     (already combined over the lane groups).
 template <typename T, int NCH, int LPR, bool kPartial>
-__device__ __forceinline__ void stream_entries(const SpmmDev& p, uint4* ring, float* wfifo, int lane,
+__device__ __forceinline__ void stream_entries(const SpmmDev& p, uint4* ring, float* wfifo, const float* ctab, int lane,
                                                int64_t e0, int n_ent, int64_t warp_row0, int row_lo,
                                                int row_hi, int rp_rel,
                                                float (&acc)[NCH][Elt<T>::kPerVec])
@@ -304,7 +333,7 @@ __device__ __forceinline__ void stream_entries(const SpmmDev& p, uint4* ring, fl
                         if (rem > nb) break;                  // the row continues in a later position
                         reduce_groups<NCH, EPV, LPR>(acc);
                         if (kPartial) return;                 // slice complete (only at the last position)
-                        finish_row<T, NCH, LPR>(p, warp_row0 + rt, lane, acc);
+                        finish_row<T, NCH, LPR>(p, ctab, warp_row0 + rt, lane, acc);
                         zero_acc<NCH, EPV>(acc);
                         if (upto > done) done = upto;
                         ++rt;
@@ -352,7 +381,7 @@ __device__ __forceinline__ void stream_entries(const SpmmDev& p, uint4* ring, fl
     } else {
         while (rt < row_hi) {                                 // rows without entries at the end of the run
             reduce_groups<NCH, EPV, LPR>(acc);
-            finish_row<T, NCH, LPR>(p, warp_row0 + rt, lane, acc);
+            finish_row<T, NCH, LPR>(p, ctab, warp_row0 + rt, lane, acc);
             zero_acc<NCH, EPV>(acc);
             ++rt;
         }
@@ -398,7 +427,7 @@ __device__ __forceinline__ void cp_async16_s(uint32_t smem_dst, const void* gmem
 // Full groups (the usual case) take straight-line code on both sides.  kFull: every lane of a position
 // holds a vector of the row (nv = 32 * NCH), so no lane needs masking.
 template <typename T, int NCH, bool kFull, bool kPartial>
-__device__ __forceinline__ void stream_rows_wide(const SpmmDev& p, uint4* ring, float* wfifo, int lane,
+__device__ __forceinline__ void stream_rows_wide(const SpmmDev& p, uint4* ring, float* wfifo, const float* ctab, int lane,
                                                  int64_t e0, int n_ent, int64_t warp_row0, int row_lo,
                                                  int row_hi, int rp_rel,
                                                  float (&acc)[NCH][Elt<T>::kPerVec])
@@ -469,7 +498,7 @@ __device__ __forceinline__ void stream_rows_wide(const SpmmDev& p, uint4* ring, 
             }
             if (re == rend) {                                 // the row is complete
                 if (kPartial) return;
-                finish_row<T, NCH, 32>(p, warp_row0 + rr, lane, acc);
+                finish_row<T, NCH, 32>(p, ctab, warp_row0 + rr, lane, acc);
                 zero_acc<NCH, EPV>(acc);
                 ++rr;
                 if (rr < row_hi) rend = row_end_of(rr);
@@ -552,6 +581,8 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
     float* wfifo = reinterpret_cast<float*>(dsmem + (size_t)kSpmmWarps * P::RING * NCH * 512) + warp * P::RING * G;
     float* part = reinterpret_cast<float*>(dsmem);           // [kSpmmWarps][kCols], reuses the rings (see below)
     static_assert((size_t)kSpmmWarps * kCols * 4 <= (size_t)kSpmmWarps * P::RING * NCH * 512, "partials must fit the rings");
+    float* ctab = reinterpret_cast<float*>(dsmem + (size_t)kSpmmWarps * P::kWarpBytes);   // [3][kCols]
+    fill_col_table<kCols>(p, ctab);
     if (threadIdx.x == 0) n_long = 0;
     __syncthreads();
 
@@ -581,10 +612,10 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
                 const int64_t e0 = __shfl_sync(0xffffffffu, rp_reg, ra);
                 const int64_t e1 = __shfl_sync(0xffffffffu, rp_reg, rl);
                 if constexpr (LPR == 32)
-                    stream_rows_wide<T, NCH, kFull, false>(p, ring, wfifo, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
+                    stream_rows_wide<T, NCH, kFull, false>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
                                                     (int)(rp_reg - e0), acc);
                 else
-                    stream_entries<T, NCH, LPR, false>(p, ring, wfifo, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
+                    stream_entries<T, NCH, LPR, false>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
                                                        (int)(rp_reg - e0), acc);
             }
             ra = rl + 1;
@@ -599,9 +630,9 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
         const int64_t slice = round_up(ceil_div(le - ls, kSpmmWarps), 32);
         const int64_t s0 = min(le, ls + warp * slice), s1 = min(le, s0 + slice);
         if constexpr (LPR == 32)
-            stream_rows_wide<T, NCH, kFull, true>(p, ring, wfifo, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
+            stream_rows_wide<T, NCH, kFull, true>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
         else
-            stream_entries<T, NCH, LPR, true>(p, ring, wfifo, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
+            stream_entries<T, NCH, LPR, true>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
         __syncthreads();                                      // every ring is idle: reuse them for the partial sums
         const int l = lane % LPR;
         if (lane < LPR) {
@@ -620,7 +651,7 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
                     for (int w = 0; w < kSpmmWarps; ++w) t += part[w * kCols + (c * 32 + l) * EPV + i];
                     acc[c][i] = t;
                 }
-            finish_row<T, NCH, LPR>(p, lrow, lane, acc);
+            finish_row<T, NCH, LPR>(p, ctab, lrow, lane, acc);
         }
         __syncthreads();
     }
@@ -629,7 +660,8 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
 template <typename T, int NCH, int LPR, bool kFull = false>
 cudaError_t launch_one(cudaStream_t s, const SpmmDev& p)
 {
-    constexpr size_t smem = kSpmmWarps * Pipe<NCH, LPR>::kWarpBytes;
+    constexpr int kCols = (LPR < 32 ? LPR : NCH * 32) * Elt<T>::kPerVec;
+    constexpr size_t smem = kSpmmWarps * Pipe<NCH, LPR>::kWarpBytes + 3 * kCols * sizeof(float);   // rings, weights, column table
     // enough thread blocks to fill the machine on small graphs, long runs of rows on large ones
     const int rows_per_warp = (int)std::min<int64_t>(kMaxRowsPerWarp, std::max<int64_t>(1, p.n / (kSpmmWarps * 148 * 8)));
     if (smem > 40 * 1024) {                                   // above the default limit: opt in
