@@ -75,7 +75,8 @@ def test_normalize_adjacency_rejects_malformed_input(ctx, B, rp, ci):
 
 # --------------------------------------------------------------------------- binarize + pack
 
-@pytest.mark.parametrize("n,d", [(1, 1), (5, 31), (9, 32), (13, 33), (300, 100), (77, 602), (40, 1433), (11, 3703), (1000, 256)])
+@pytest.mark.parametrize("n,d", [(1, 1), (5, 31), (9, 32), (13, 33), (300, 100), (77, 602), (40, 1433), (11, 3703), (1000, 256),
+                                 (77, 600), (33, 132), (19, 4), (3000, 1436)])   # row lengths that are multiples of 4 take the 16-byte-load kernel
 @pytest.mark.parametrize("norm", [False, True])
 def test_pack_features(ctx, n, d, norm):
     rng = np.random.default_rng(n * 7919 + d)
