@@ -48,7 +48,8 @@ typedef enum {
     BIGCN_ERR_WORKSPACE = 5,   /* no workspace attached, or it is too small */
     BIGCN_ERR_CUDA = 6,        /* a CUDA runtime call failed (message in bigcn_last_error) */
     BIGCN_ERR_UNSUPPORTED = 7, /* a valid request this build does not implement */
-    BIGCN_ERR_INTERNAL = 8     /* a device-side self-check tripped */
+    BIGCN_ERR_INTERNAL = 8,    /* a device-side self-check tripped */
+    BIGCN_ERR_BUSY = 9         /* every slot of a pipeline holds a step that has not been waited for */
 } bigcn_status;
 
 typedef struct bigcn_ctx bigcn_ctx;
@@ -85,7 +86,8 @@ int64_t bigcn_packed_stride_words(int32_t len);
 
 /* Scratch.  bigcn_workspace_bytes() bounds what bigcn_forward()/bigcn_layer_forward() need for a
  * graph of n nodes and nnz stored entries and the layer widths dims[0..n_layers];
- * with host_io != 0 it adds the staging buffers of bigcn_forward_host().
+ * with host_io = 1 it adds the staging buffers of bigcn_forward_host(), with host_io = k > 1 those
+ * of a pipeline with k slots (bigcn_pipeline_open).
  * bigcn_set_workspace() attaches caller-owned device memory (256-byte aligned) until replaced. */
 size_t bigcn_workspace_bytes(int64_t n, int64_t nnz, const int32_t* dims /*host*/, int32_t n_layers,
                              int32_t host_io);
@@ -194,6 +196,33 @@ bigcn_status bigcn_forward_packed(bigcn_ctx* ctx, const bigcn_graph* graph, cons
 bigcn_status bigcn_forward_host(bigcn_ctx* ctx, const bigcn_graph* graph, const bigcn_layer* layers /*host*/,
                                 int32_t n_layers, const float* X_host, int64_t ldx,
                                 float* logits_host, int64_t ldo);
+
+/* Back-to-back forwards from host buffers, overlapped.  bigcn_forward_host() finishes one step (copy
+ * in, forward, copy out) before the next begins, so the link to the host and the GPU take turns.
+ * A pipeline keeps `slots` steps in flight on three streams: while step k computes on the context's
+ * stream, the input of step k+1 is copied in and the logits of step k-1 are copied out.  The paper
+ * has no counterpart of these calls (its measurements start from device-resident data, Sec. 6); each
+ * step computes exactly what bigcn_forward() computes.
+ *   bigcn_pipeline_open   copies the graph and layer descriptions (their device arrays must outlive
+ *                         the pipeline) and creates streams and events; allocates no device memory.
+ *                         1 <= slots <= BIGCN_MAX_PIPELINE_SLOTS; 3 overlaps all three stages.
+ *   bigcn_pipeline_submit enqueues one step and returns without waiting: X_host fp32 [n x d_0] dense,
+ *                         logits_host fp32 [n x classes] dense, both HOST memory that must stay valid
+ *                         (and, for the copies to overlap, page-locked) until the matching wait.
+ *                         BIGCN_ERR_BUSY if `slots` steps are outstanding; BIGCN_ERR_WORKSPACE unless
+ *                         the context's workspace was sized with host_io = slots.  The workspace must
+ *                         not be replaced, and the context not used for other calls, while steps are
+ *                         outstanding.
+ *   bigcn_pipeline_wait   blocks until the OLDEST outstanding step has delivered its logits (steps
+ *                         complete in submission order); BIGCN_OK at once if none is outstanding.
+ *   bigcn_pipeline_close  waits for everything outstanding and frees the streams and events. */
+#define BIGCN_MAX_PIPELINE_SLOTS 8
+typedef struct bigcn_pipeline bigcn_pipeline;
+bigcn_status bigcn_pipeline_open(bigcn_ctx* ctx, const bigcn_graph* graph, const bigcn_layer* layers /*host*/,
+                                 int32_t n_layers, int32_t slots, bigcn_pipeline** out);
+bigcn_status bigcn_pipeline_submit(bigcn_pipeline* pipe, const float* X_host, float* logits_host);
+bigcn_status bigcn_pipeline_wait(bigcn_pipeline* pipe);
+bigcn_status bigcn_pipeline_close(bigcn_pipeline* pipe);
 
 /* Batch statistics for the batch normalisation of a layer's input (Sec. 4.4: zero mean, unit
  * variance per feature over the nodes): shift_out[j] = mean_j, scale_out[j] = 1/sqrt(var_j + eps),

@@ -64,6 +64,11 @@ SIGNATURES = {
                                             _vp, _vp, _vp, _i64, ctypes.POINTER(bigcn_stats)]),
     "bigcn_forward_host": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer), _i32,
                                           _vp, _i64, _vp, _i64]),
+    "bigcn_pipeline_open": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer), _i32, _i32,
+                                           ctypes.POINTER(_vp)]),
+    "bigcn_pipeline_submit": (ctypes.c_int, [_vp, _vp, _vp]),
+    "bigcn_pipeline_wait": (ctypes.c_int, [_vp]),
+    "bigcn_pipeline_close": (ctypes.c_int, [_vp]),
     "bigcn_col_stats": (ctypes.c_int, [_vp, _vp, _i64, _i32, _i64, ctypes.c_float, _vp, _vp]),
     "bigcn_mean_adjacency": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp,
                                             ctypes.POINTER(_i64)]),
@@ -223,9 +228,9 @@ class BiGCN:
     def sync_check(self):
         self._check(self.lib.bigcn_sync_check(self.h))
 
-    def workspace_bytes(self, n: int, nnz: int, dims: Sequence[int], host_io: bool = False) -> int:
+    def workspace_bytes(self, n: int, nnz: int, dims: Sequence[int], host_io: int = 0) -> int:
         arr = (_i32 * len(dims))(*[int(d) for d in dims])
-        return int(self.lib.bigcn_workspace_bytes(n, nnz, arr, len(dims) - 1, 1 if host_io else 0))
+        return int(self.lib.bigcn_workspace_bytes(n, nnz, arr, len(dims) - 1, int(host_io)))
 
     def ensure_workspace(self, nbytes: int):
         if self.workspace is None or self.workspace.numel() < nbytes:
@@ -290,7 +295,7 @@ class BiGCN:
         out.update(h=h, next_bits=nb, next_beta=nbeta, dot=dot, zeta=zeta)
         return out
 
-    def _prep_forward(self, graph: Graph, layers: Sequence[Layer], host_io: bool = False):
+    def _prep_forward(self, graph: Graph, layers: Sequence[Layer], host_io: int = 0):
         dims = [layers[0].d_in] + [l.d_out for l in layers]
         self.ensure_workspace(self.workspace_bytes(graph.n, graph.nnz, dims, host_io))
         return _layer_array(layers), dims
@@ -328,6 +333,13 @@ class BiGCN:
         self._check(self.lib.bigcn_forward_host(self.h, ctypes.byref(graph.c), arr, len(layers), _ptr(X_host),
                                                 dims[0], _ptr(logits_host), dims[-1]))
         return logits_host
+
+    def open_pipeline(self, graph: Graph, layers: Sequence[Layer], slots: int = 3) -> "Pipeline":
+        """Overlapped back-to-back forwards from host buffers (bigcn_pipeline_*)."""
+        arr, dims = self._prep_forward(graph, layers, host_io=slots)
+        h = _vp()
+        self._check(self.lib.bigcn_pipeline_open(self.h, ctypes.byref(graph.c), arr, len(layers), slots, ctypes.byref(h)))
+        return Pipeline(self, h, graph, list(layers), dims)
 
     def col_stats(self, H: torch.Tensor, eps: float = 1e-5):
         n, d = H.shape
@@ -386,3 +398,35 @@ class BiGCN:
             sc = scales[l] if scales is not None else None
             layers.append(make_layer(W.shape[0], W.shape[1], bitsT, alpha, sh, sc))
         return layers
+
+
+class Pipeline:
+    """bigcn_pipeline_*: submit() enqueues a step from pinned host tensors, wait() blocks for the oldest one."""
+
+    def __init__(self, ctx: BiGCN, handle, graph: Graph, layers: List[Layer], dims: List[int]):
+        self.ctx, self.h, self.graph, self.layers, self.dims = ctx, handle, graph, layers, dims
+        self._held = []                     # host tensors of outstanding steps stay referenced
+
+    def submit(self, X_host: torch.Tensor, logits_host: torch.Tensor):
+        assert X_host.device.type == "cpu" and logits_host.device.type == "cpu"
+        assert X_host.is_contiguous() and logits_host.is_contiguous()
+        assert tuple(X_host.shape) == (self.graph.n, self.dims[0]) and X_host.dtype == torch.float32
+        assert tuple(logits_host.shape) == (self.graph.n, self.dims[-1]) and logits_host.dtype == torch.float32
+        self.ctx._check(self.ctx.lib.bigcn_pipeline_submit(self.h, _ptr(X_host), _ptr(logits_host)))
+        self._held.append((X_host, logits_host))
+
+    def wait(self) -> Optional[torch.Tensor]:
+        self.ctx._check(self.ctx.lib.bigcn_pipeline_wait(self.h))
+        return self._held.pop(0)[1] if self._held else None
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.ctx.lib.bigcn_pipeline_close(self.h)
+            self.h = None
+            self._held = []
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -258,6 +258,7 @@ const char* bigcn_status_string(bigcn_status s)
         case BIGCN_ERR_CUDA: return "CUDA error";
         case BIGCN_ERR_UNSUPPORTED: return "unsupported";
         case BIGCN_ERR_INTERNAL: return "device self-check failed";
+        case BIGCN_ERR_BUSY: return "pipeline full";
     }
     return "unknown status";
 }
@@ -349,8 +350,8 @@ size_t bigcn_workspace_bytes(int64_t n, int64_t nnz, const int32_t* dims, int32_
     total += 2 * (up((size_t)n * stride_max * 4) + up((size_t)n * 4));
     size_t aux = up(normalize_scratch_bytes(n));
     if (up(col_stats_scratch_bytes(d_max)) > aux) aux = up(col_stats_scratch_bytes(d_max));
-    if (host_io) {
-        total += up((size_t)n * dims[0] * 4) + up((size_t)n * dims[n_layers] * 4);
+    if (host_io > 0) {                                        // staging buffers: one pair per slot
+        total += (size_t)host_io * (up((size_t)n * dims[0] * 4) + up((size_t)n * dims[n_layers] * 4));
     }
     if (aux > total) total = aux;
     return total + kAlign;
@@ -521,6 +522,129 @@ bigcn_status bigcn_forward_host(bigcn_ctx* ctx, const bigcn_graph* graph, const 
     if (st != BIGCN_OK) return st;
     BIGCN_CUDA(ctx, cudaMemcpyAsync(logits_host, out_dev, (size_t)n * classes * 4, cudaMemcpyDeviceToHost, ctx->stream));
     BIGCN_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return BIGCN_OK;
+}
+
+struct bigcn_pipeline {
+    bigcn_ctx* ctx;
+    bigcn_graph graph;
+    bigcn_layer layers[BIGCN_MAX_LAYERS];
+    int32_t n_layers;
+    int32_t slots;
+    cudaStream_t up;                                  // host -> device copies
+    cudaStream_t down;                                // device -> host copies
+    cudaEvent_t x_ready[BIGCN_MAX_PIPELINE_SLOTS];    // the slot's input has arrived
+    cudaEvent_t computed[BIGCN_MAX_PIPELINE_SLOTS];   // the slot's forward is done (input consumed, logits written)
+    cudaEvent_t delivered[BIGCN_MAX_PIPELINE_SLOTS];  // the slot's logits are in host memory
+    bool used[BIGCN_MAX_PIPELINE_SLOTS];
+    int64_t submitted;
+    int64_t waited;
+};
+
+bigcn_status bigcn_pipeline_open(bigcn_ctx* ctx, const bigcn_graph* graph, const bigcn_layer* layers,
+                                 int32_t n_layers, int32_t slots, bigcn_pipeline** out)
+{
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    if (!out) return fail(ctx, BIGCN_ERR_NULL, "out is null");
+    *out = nullptr;
+    if (slots < 1 || slots > BIGCN_MAX_PIPELINE_SLOTS) return fail(ctx, BIGCN_ERR_SHAPE, "slots=%d not in 1..%d", slots, BIGCN_MAX_PIPELINE_SLOTS);
+    float dummy = 0.f;                                // check_forward only tests the logits pointer for null
+    if ((st = check_forward(ctx, graph, layers, n_layers, &dummy, int64_t(1) << 40)) != BIGCN_OK) return st;
+    bigcn_pipeline* p = new (std::nothrow) bigcn_pipeline();
+    if (!p) return fail(ctx, BIGCN_ERR_INTERNAL, "out of host memory");
+    p->ctx = ctx;
+    p->graph = *graph;
+    for (int l = 0; l < n_layers; ++l) p->layers[l] = layers[l];
+    p->n_layers = n_layers;
+    p->slots = slots;
+    cudaError_t e = cudaStreamCreateWithFlags(&p->up, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->down, cudaStreamNonBlocking);
+    for (int s = 0; s < slots && e == cudaSuccess; ++s) {
+        e = cudaEventCreateWithFlags(&p->x_ready[s], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->computed[s], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->delivered[s], cudaEventDisableTiming);
+    }
+    if (e != cudaSuccess) {
+        bigcn_pipeline_close(p);
+        return cuda_fail(ctx, e, "pipeline streams and events");
+    }
+    *out = p;
+    return BIGCN_OK;
+}
+
+bigcn_status bigcn_pipeline_submit(bigcn_pipeline* p, const float* X_host, float* logits_host)
+{
+    if (!p) return BIGCN_ERR_NULL;
+    bigcn_ctx* ctx = p->ctx;
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    if (p->submitted - p->waited >= p->slots) return fail(ctx, BIGCN_ERR_BUSY, "all %d slots hold steps that have not been waited for", p->slots);
+    const int64_t n = p->graph.n;
+    const int32_t d0 = p->layers[0].d_in, classes = p->layers[p->n_layers - 1].d_out;
+    const int s = (int)(p->submitted % p->slots);
+    if (n == 0) {                                             // nothing to move or compute: the step is complete
+        BIGCN_CUDA(ctx, cudaEventRecord(p->delivered[s], p->down));
+        ++p->submitted;
+        return BIGCN_OK;
+    }
+    if (!X_host || !logits_host) return fail(ctx, BIGCN_ERR_NULL, "X_host or logits_host is null");
+    Carver ws{static_cast<char*>(ctx->ws), ctx->ws_bytes, 0};
+    float* x_dev = nullptr;
+    float* out_dev = nullptr;
+    for (int i = 0; i < p->slots; ++i) {                      // the same carving at every call: slot i keeps its buffers
+        float* x = static_cast<float*>(ws.take((size_t)n * d0 * 4));
+        float* o = static_cast<float*>(ws.take((size_t)n * classes * 4));
+        if (!x || !o) return fail(ctx, BIGCN_ERR_WORKSPACE, "workspace too small for %d pairs of staging buffers (size it with host_io = %d)", p->slots, p->slots);
+        if (i == s) { x_dev = x; out_dev = o; }
+    }
+    // copy in: the slot's input buffer is free once the step that used it last has been computed
+    if (p->used[s]) BIGCN_CUDA(ctx, cudaStreamWaitEvent(p->up, p->computed[s], 0));
+    BIGCN_CUDA(ctx, cudaMemcpyAsync(x_dev, X_host, (size_t)n * d0 * 4, cudaMemcpyHostToDevice, p->up));
+    BIGCN_CUDA(ctx, cudaEventRecord(p->x_ready[s], p->up));
+    // forward: the slot's logits buffer is free because its last step has been waited for (slots bound above)
+    BIGCN_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, p->x_ready[s], 0));
+    st = forward_impl(ctx, &p->graph, p->layers, p->n_layers, x_dev, d0, nullptr, nullptr, out_dev, classes, nullptr, ws);
+    finish_call(ctx);
+    if (st != BIGCN_OK) return st;
+    BIGCN_CUDA(ctx, cudaEventRecord(p->computed[s], ctx->stream));
+    // copy out
+    BIGCN_CUDA(ctx, cudaStreamWaitEvent(p->down, p->computed[s], 0));
+    BIGCN_CUDA(ctx, cudaMemcpyAsync(logits_host, out_dev, (size_t)n * classes * 4, cudaMemcpyDeviceToHost, p->down));
+    BIGCN_CUDA(ctx, cudaEventRecord(p->delivered[s], p->down));
+    p->used[s] = true;
+    ++p->submitted;
+    return BIGCN_OK;
+}
+
+bigcn_status bigcn_pipeline_wait(bigcn_pipeline* p)
+{
+    if (!p) return BIGCN_ERR_NULL;
+    bigcn_ctx* ctx = p->ctx;
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    if (p->waited == p->submitted) return BIGCN_OK;
+    const int s = (int)(p->waited % p->slots);
+    ++p->waited;
+    BIGCN_CUDA(ctx, cudaEventSynchronize(p->delivered[s]));
+    return BIGCN_OK;
+}
+
+bigcn_status bigcn_pipeline_close(bigcn_pipeline* p)
+{
+    if (!p) return BIGCN_ERR_NULL;
+    cudaSetDevice(p->ctx->device);
+    if (p->up) cudaStreamSynchronize(p->up);
+    cudaStreamSynchronize(p->ctx->stream);
+    if (p->down) cudaStreamSynchronize(p->down);
+    for (int s = 0; s < p->slots; ++s) {
+        if (p->x_ready[s]) cudaEventDestroy(p->x_ready[s]);
+        if (p->computed[s]) cudaEventDestroy(p->computed[s]);
+        if (p->delivered[s]) cudaEventDestroy(p->delivered[s]);
+    }
+    if (p->up) cudaStreamDestroy(p->up);
+    if (p->down) cudaStreamDestroy(p->down);
+    delete p;
     return BIGCN_OK;
 }
 
