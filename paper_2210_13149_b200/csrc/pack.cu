@@ -85,129 +85,124 @@ pack_rows_kernel(const float* __restrict__ H, int64_t n, int d, int64_t ld,
     }
 }
 
-// The same packing with 16-byte loads, for matrices whose rows start on 16-byte boundaries
-// (ld a multiple of 4, base aligned): lane l of a warp reads columns 128 c + 4 l .. + 3 of chunk c,
-// so a row of up to 128 columns costs one load instruction instead of four.  The four sign bits of a
-// lane are shifted to their place in the packed word and OR-ed over the 8 lanes that share the word.
-// A warp walks over tiles of R rows x one chunk and always has the NEXT tile's loads in flight while
-// it works on the current one (two register buffers used in turn), so the memory system is never
-// idle behind the arithmetic.  kRagged: d is not a multiple of 4, so one lane of a row holds columns
+// Packing through shared memory, for matrices whose rows start on 16-byte boundaries (ld a multiple
+// of 4, base aligned).  In the kernel above a warp instruction handles one element per lane and most
+// instructions are bookkeeping per row; here a LANE owns a whole packed word: the warp copies a tile
+// of 8 rows x 128 columns into its own shared-memory ring with 16-byte asynchronous copies (coalesced,
+// no registers in between), and then lane 4r + w packs word w of row r from 32 consecutive floats, so
+// the sign bits need no exchange between lanes and every bookkeeping instruction is shared by 32
+// elements.  Three tiles per warp are in flight.  The staged rows are skewed (one 16-byte pad after
+// every 8 units, 36 units per row) so that the 16-byte reads of a quarter warp -- 4 words x 2 rows --
+// fall into 8 different bank groups; the per-column shift and scale sit in shared memory in the same
+// skewed form.  kRagged: d is not a multiple of 4, so the last 16-byte unit of a row holds columns
 // past the end that must not count.
-template <bool kNorm, bool kRagged, int R>
-__global__ void __launch_bounds__(kPackWarpsPerBlock* kWarp, 4)
-pack_rows_vec_kernel(const float* __restrict__ H, int64_t n, int d, int64_t ld,
-                     const float* __restrict__ shift, const float* __restrict__ scale,
-                     uint32_t* __restrict__ bits, int64_t stride, float* __restrict__ beta)
+constexpr int kStageRows = 8;                         // rows per tile
+constexpr int kStageRowUnits = 36;                    // 16-byte units per staged row: 4 words x (8 + 1 pad)
+constexpr int kStageTileUnits = kStageRows * kStageRowUnits;
+constexpr int kStageTiles = 3;                        // tiles in flight per warp
+
+__device__ __forceinline__ void stage_copy16(float4* smem_dst, const float* gmem_src)
 {
+    const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(gmem_src) : "memory");
+}
+
+template <bool kNorm, bool kRagged>
+__global__ void __launch_bounds__(kPackWarpsPerBlock* kWarp, 2)
+pack_rows_staged_kernel(const float* __restrict__ H, int64_t n, int d, int64_t ld,
+                        const float* __restrict__ shift, const float* __restrict__ scale,
+                        uint32_t* __restrict__ bits, int64_t stride, float* __restrict__ beta)
+{
+    extern __shared__ __align__(16) unsigned char pack_smem[];
     const int lane = threadIdx.x & 31;
-    const int64_t warp_id = (int64_t)blockIdx.x * kPackWarpsPerBlock + (threadIdx.x >> 5);
-    const int64_t row_step = (int64_t)gridDim.x * kPackWarpsPerBlock * R;
-    const int n_chunks = (int)(stride >> 2);      // 4 packed words = 128 columns per chunk
-    const int sub = lane & 7;                     // this lane's nibble inside its packed word
-    const int shl = 4 * sub;
-    const float inv_d = 1.f / (float)d;
-
-    struct Tile { int64_t row0; int ch; };
-    auto next_of = [&](Tile t) {
-        Tile u = {t.row0, t.ch + 1};
-        if (u.ch == n_chunks) { u.ch = 0; u.row0 = t.row0 + row_step; }
-        return u;
-    };
-    auto load_tile = [&](Tile t, float4 (&x)[R]) {
-        const int j0 = t.ch * 128 + lane * 4;
-        const float* src = H + t.row0 * ld + j0;
-        const bool lane_in = j0 < d;
-        if (t.row0 + R <= n) {                                    // the usual case: no row checks
-#pragma unroll
-            for (int r = 0; r < R; ++r)
-                x[r] = lane_in ? __ldg(reinterpret_cast<const float4*>(src + r * ld)) : make_float4(0.f, 0.f, 0.f, 0.f);
-        } else {
-#pragma unroll
-            for (int r = 0; r < R; ++r)
-                x[r] = (lane_in && t.row0 + r < n) ? __ldg(reinterpret_cast<const float4*>(src + r * ld))
-                                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+    const int warp = threadIdx.x >> 5;
+    float4* ring = reinterpret_cast<float4*>(pack_smem) + warp * (kStageTiles * kStageTileUnits);
+    float4* tab_shift = reinterpret_cast<float4*>(pack_smem) + kPackWarpsPerBlock * kStageTiles * kStageTileUnits;
+    const int tab_units = (int)stride * 9;            // 8 units of data + 1 pad per packed word
+    float4* tab_scale = tab_shift + tab_units;
+    if (kNorm) {
+        for (int col = threadIdx.x; col < (int)stride * 32; col += blockDim.x) {
+            const int at = (col >> 5) * 36 + (col & 31);          // float index in the skewed table
+            reinterpret_cast<float*>(tab_shift)[at] = col < d ? __ldg(shift + col) : 0.f;
+            reinterpret_cast<float*>(tab_scale)[at] = col < d ? __ldg(scale + col) : 1.f;
         }
-    };
-    float sh[4] = {0.f, 0.f, 0.f, 0.f}, sc[4] = {1.f, 1.f, 1.f, 1.f};
-    auto load_norm = [&](int ch) {
-        const int j0 = ch * 128 + lane * 4;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const bool in = j0 + i < d;
-            sh[i] = in ? __ldg(shift + j0 + i) : 0.f;
-            sc[i] = in ? __ldg(scale + j0 + i) : 1.f;
-        }
-    };
-    float l1[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) l1[r] = 0.f;
-
-    auto process = [&](Tile t, const float4 (&x)[R]) {
-        const int j0 = t.ch * 128 + lane * 4;
-        const int n_valid = min(max(d - j0, 0), 4);               // columns of this lane that exist
-        const uint32_t keep = ((1u << n_valid) - 1u) << shl;      // missing columns pack as 0
-        uint32_t* dst = bits + t.row0 * stride + t.ch * 4 + (lane >> 3);
-        const bool full = t.row0 + R <= n;
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-            float v[4] = {x[r].x, x[r].y, x[r].z, x[r].w};
-            uint32_t word = 0u;
-            float part = 0.f;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                if (kRagged && i >= n_valid) v[i] = 0.f;          // whatever lies between d and ld is not data
-                if (kNorm) v[i] = __fmul_rn(__fsub_rn(v[i], sh[i]), sc[i]);
-                if (v[i] >= 0.f) word |= 1u << i;
-                part += fabsf(v[i]);
-            }
-            l1[r] += part;
-            word = (word << shl) & keep;
-            word |= __shfl_xor_sync(0xffffffffu, word, 1);
-            word |= __shfl_xor_sync(0xffffffffu, word, 2);
-            word |= __shfl_xor_sync(0xffffffffu, word, 4);
-            if (sub == 0 && (full || t.row0 + r < n)) dst[r * stride] = word;
-        }
-        if (t.ch == n_chunks - 1) {
-            // reduce the R row sums: after the halving steps lane L carries row L / (32 / R)
-            int off = 16;
-#pragma unroll
-            for (int half = R / 2; half >= 1; half /= 2, off /= 2) {
-                const bool upper = (lane & off) != 0;
-#pragma unroll
-                for (int i = 0; i < half; ++i) {
-                    const float send = upper ? l1[i] : l1[i + half];
-                    const float keep_v = upper ? l1[i + half] : l1[i];
-                    l1[i] = keep_v + __shfl_xor_sync(0xffffffffu, send, off);
-                }
-            }
-            for (int o = off; o >= 1; o /= 2) l1[0] += __shfl_xor_sync(0xffffffffu, l1[0], o);
-            constexpr int kLanesPerRow = 32 / R;
-            const int64_t row = t.row0 + lane / kLanesPerRow;
-            if (lane % kLanesPerRow == 0 && row < n) beta[row] = l1[0] * inv_d;
-#pragma unroll
-            for (int r = 0; r < R; ++r) l1[r] = 0.f;
-        }
-    };
-
-    Tile ta = {warp_id * R, 0};
-    if (ta.row0 >= n) return;
-    float4 xa[R], xb[R];
-    load_tile(ta, xa);
-    if (kNorm) load_norm(0);
-    for (;;) {
-        const Tile tb = next_of(ta);
-        const bool has_b = tb.row0 < n;
-        if (has_b) load_tile(tb, xb);
-        process(ta, xa);
-        if (!has_b) break;
-        if (kNorm && n_chunks > 1) load_norm(tb.ch);
-        ta = next_of(tb);
-        const bool has_a = ta.row0 < n;
-        if (has_a) load_tile(ta, xa);
-        process(tb, xb);
-        if (!has_a) break;
-        if (kNorm && n_chunks > 1) load_norm(ta.ch);
+        __syncthreads();
     }
+    const int64_t warp_id = (int64_t)blockIdx.x * kPackWarpsPerBlock + warp;
+    const int64_t row_step = (int64_t)gridDim.x * kPackWarpsPerBlock * kStageRows;
+    const int n_chunks = (int)(stride >> 2);          // 4 packed words = 128 columns per chunk
+    const float inv_d = 1.f / (float)d;
+    const int r = lane >> 2, w = lane & 3;            // the (row, word) of a tile this lane packs
+    const int copy_unit = 9 * (lane >> 3) + (lane & 7);   // where this lane's 16 bytes of a staged row go
+
+    // issue cursor and consume cursor walk the same sequence of tiles (row group, chunk)
+    int64_t i_row0 = warp_id * kStageRows, c_row0 = i_row0;
+    int i_ch = 0, c_ch = 0, i_slot = 0, c_slot = 0;
+    float l1 = 0.f;
+    auto issue = [&]() {
+        if (i_row0 < n) {
+            float4* dst = ring + i_slot * kStageTileUnits + copy_unit;
+            const int col = i_ch * 128 + 4 * lane;
+            const float* src = H + i_row0 * ld + col;
+            const bool col_in = col < d;
+            const int rows_in = (int)min((int64_t)kStageRows, n - i_row0);
+#pragma unroll
+            for (int q = 0; q < kStageRows; ++q) {
+                if (col_in && q < rows_in) stage_copy16(dst + q * kStageRowUnits, src + q * ld);
+                else dst[q * kStageRowUnits] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            if (++i_ch == n_chunks) { i_ch = 0; i_row0 += row_step; }
+            i_slot = i_slot + 1 == kStageTiles ? 0 : i_slot + 1;
+        }
+        asm volatile("cp.async.commit_group;\n" ::: "memory");   // one group per call, possibly empty
+    };
+#pragma unroll
+    for (int t = 0; t < kStageTiles - 1; ++t) issue();
+    while (c_row0 < n) {
+        issue();
+        asm volatile("cp.async.wait_group %0;\n" ::"n"(kStageTiles - 1) : "memory");
+        __syncwarp();                                 // the other lanes' copies of this tile are visible
+        const float4* src = ring + c_slot * kStageTileUnits + r * kStageRowUnits + w * 9;
+        const float4* ts = tab_shift + (c_ch * 4 + w) * 9;
+        const float4* tc = tab_scale + (c_ch * 4 + w) * 9;
+        const int n_valid = min(max(d - (c_ch * 128 + w * 32), 0), 32);      // columns of this word that exist
+        uint32_t word = 0u;
+        float part = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const float4 x = src[k];
+            float v[4] = {x.x, x.y, x.z, x.w};
+            float sh[4] = {0.f, 0.f, 0.f, 0.f}, sc[4] = {1.f, 1.f, 1.f, 1.f};
+            if (kNorm) {
+                const float4 a = ts[k], b = tc[k];
+                sh[0] = a.x, sh[1] = a.y, sh[2] = a.z, sh[3] = a.w;
+                sc[0] = b.x, sc[1] = b.y, sc[2] = b.z, sc[3] = b.w;
+            }
+            float quad = 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (kRagged && 4 * k + j >= n_valid) v[j] = 0.f;  // whatever lies between d and ld is not data
+                if (kNorm) v[j] = __fmul_rn(__fsub_rn(v[j], sh[j]), sc[j]);
+                if (v[j] >= 0.f) word |= 1u << (4 * k + j);
+                quad += fabsf(v[j]);
+            }
+            part += quad;
+        }
+        if (n_valid < 32) word &= (1u << n_valid) - 1u;           // columns past d pack as 0 (their staged value is 0)
+        l1 += part;
+        const int64_t row = c_row0 + r;
+        if (row < n) bits[row * stride + c_ch * 4 + w] = word;
+        if (c_ch == n_chunks - 1) {                               // the row is complete: its 4 lanes add up
+            l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+            l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+            if (w == 0 && row < n) beta[row] = l1 * inv_d;
+            l1 = 0.f;
+        }
+        __syncwarp();                                 // all lanes are done with the slot before it is refilled
+        if (++c_ch == n_chunks) { c_ch = 0; c_row0 += row_step; }
+        c_slot = c_slot + 1 == kStageTiles ? 0 : c_slot + 1;
+    }
+    asm volatile("cp.async.wait_group 0;\n" ::: "memory");
 }
 
 // Weights: W is [d_in x d_out] row-major and the packed output is transposed (one row per output
@@ -258,18 +253,19 @@ cudaError_t launch_pack_rows(cudaStream_t s, const float* H, int64_t n, int d, i
                              uint32_t* bits, int64_t stride, float* beta, int* launches)
 {
     if (n == 0) return cudaSuccess;
-    if (ld % 4 == 0 && reinterpret_cast<uintptr_t>(H) % 16 == 0) {          // rows start on 16-byte boundaries
-        constexpr int R = 4;
-        auto kernel = shift ? ((d & 3) ? pack_rows_vec_kernel<true, true, R> : pack_rows_vec_kernel<true, false, R>)
-                            : ((d & 3) ? pack_rows_vec_kernel<false, true, R> : pack_rows_vec_kernel<false, false, R>);
+    const size_t staged_smem = (size_t)kPackWarpsPerBlock * kStageTiles * kStageTileUnits * 16 + (shift ? 2 * (size_t)stride * 9 * 16 : 0);
+    if (ld % 4 == 0 && reinterpret_cast<uintptr_t>(H) % 16 == 0 && staged_smem <= 200 * 1024) {   // rows start on 16-byte boundaries
+        auto kernel = shift ? ((d & 3) ? pack_rows_staged_kernel<true, true> : pack_rows_staged_kernel<true, false>)
+                            : ((d & 3) ? pack_rows_staged_kernel<false, true> : pack_rows_staged_kernel<false, false>);
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)staged_smem);
         // persistent grid: exactly the blocks that are resident at once, so that no block waits for a slot
         int per_sm = 0, n_sm = 0, dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaGetDevice(&dev);
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-        if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kPackWarpsPerBlock * kWarp, 0);
+        if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kPackWarpsPerBlock * kWarp, staged_smem);
         if (e != cudaSuccess) return e;
-        const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, (int64_t)kPackWarpsPerBlock * R), (int64_t)n_sm * std::max(per_sm, 1));
-        kernel<<<grid, kPackWarpsPerBlock * kWarp, 0, s>>>(H, n, d, ld, shift, scale, bits, stride, beta);
+        const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, (int64_t)kPackWarpsPerBlock * kStageRows), (int64_t)n_sm * std::max(per_sm, 1));
+        kernel<<<grid, kPackWarpsPerBlock * kWarp, staged_smem, s>>>(H, n, d, ld, shift, scale, bits, stride, beta);
         ++*launches;
         return cudaGetLastError();
     }
