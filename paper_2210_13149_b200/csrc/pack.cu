@@ -1,6 +1,7 @@
 // Binarization + bit packing of node features (rows) and weights (columns).
 // Bi-GCN Sec. 4.2.1 (Eq. "B", "alpha"), Sec. 4.2.2 (Eq. "F", "beta"), Sec. 4.4 (batch-normalised input).
 #include <algorithm>
+#include <mutex>
 
 #include "bigcn_internal.cuh"
 
@@ -255,15 +256,30 @@ cudaError_t launch_pack_rows(cudaStream_t s, const float* H, int64_t n, int d, i
     if (n == 0) return cudaSuccess;
     const size_t staged_smem = (size_t)kPackWarpsPerBlock * kStageTiles * kStageTileUnits * 16 + (shift ? 2 * (size_t)stride * 9 * 16 : 0);
     if (ld % 4 == 0 && reinterpret_cast<uintptr_t>(H) % 16 == 0 && staged_smem <= 200 * 1024) {   // rows start on 16-byte boundaries
+        const int variant = (shift ? 2 : 0) + ((d & 3) ? 1 : 0);
         auto kernel = shift ? ((d & 3) ? pack_rows_staged_kernel<true, true> : pack_rows_staged_kernel<true, false>)
                             : ((d & 3) ? pack_rows_staged_kernel<false, true> : pack_rows_staged_kernel<false, false>);
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)staged_smem);
-        // persistent grid: exactly the blocks that are resident at once, so that no block waits for a slot
+        // persistent grid: exactly the blocks that are resident at once, so that no block waits for a slot.
+        // The attribute and the occupancy query cost tens of microseconds of host time each, so their
+        // result is kept per kernel variant for the last (device, shared-memory size) seen.
+        struct Cached { int dev = -1; size_t smem = 0; int per_sm = 0; int n_sm = 0; };
+        static Cached cache[4];
+        static std::mutex cache_mutex;
         int per_sm = 0, n_sm = 0, dev = 0;
-        if (e == cudaSuccess) e = cudaGetDevice(&dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-        if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kPackWarpsPerBlock * kWarp, staged_smem);
+        cudaError_t e = cudaGetDevice(&dev);
         if (e != cudaSuccess) return e;
+        {
+            std::lock_guard<std::mutex> lock(cache_mutex);
+            Cached& c = cache[variant];
+            if (c.dev != dev || c.smem != staged_smem) {
+                e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)staged_smem);
+                if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+                if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kPackWarpsPerBlock * kWarp, staged_smem);
+                if (e != cudaSuccess) return e;
+                c.dev = dev, c.smem = staged_smem, c.per_sm = per_sm, c.n_sm = n_sm;
+            }
+            per_sm = c.per_sm, n_sm = c.n_sm;
+        }
         const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, (int64_t)kPackWarpsPerBlock * kStageRows), (int64_t)n_sm * std::max(per_sm, 1));
         kernel<<<grid, kPackWarpsPerBlock * kWarp, staged_smem, s>>>(H, n, d, ld, shift, scale, bits, stride, beta);
         ++*launches;
