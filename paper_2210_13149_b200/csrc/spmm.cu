@@ -231,14 +231,18 @@ __device__ __forceinline__ void finish_row(const SpmmDev& p, const float* ctab, 
     }
 }
 
-template <int NCH, int LPR>
+template <int NCH, int LPR, bool kPair = false>
 struct Pipe {
     static constexpr int G = kWarp / LPR;                       // entries per position
     static constexpr int PB = (4 * G <= 32) ? 4 : 32 / G;       // positions per group (PB * G divides 32)
-    static constexpr int NG = NCH > 1 ? 2 : (LPR == 32 ? 4 : 3);  // groups in flight per warp (a power of two for wide rows)
+    static constexpr int NG = NCH > 1 ? 2 : ((LPR == 32 || kPair) ? 4 : 3);  // groups in flight per warp (a power of two for the row-aligned streams)
     static constexpr int RING = PB * NG;                        // slots of NCH * 512 bytes
     static constexpr size_t kWarpBytes = (size_t)RING * (NCH * 512 + G * 4);
 };
+
+// 256-byte rows of 8-bit elements take the row-aligned stream with two entries per position.
+template <typename T, int NCH, int LPR>
+struct UsesPairStream { static constexpr bool value = (sizeof(T) == 1 && NCH == 1 && LPR == 16); };
 
 // Streams the stored entries [e0, e0 + n_ent) through the warp's ring.
 //   kPartial = false: the entries are those of rows [row_lo, row_hi); `rp_rel` holds, in lane j, the
@@ -510,34 +514,35 @@ __device__ __forceinline__ void stream_rows_wide(const SpmmDev& p, uint4* ring, 
             const int left = iend - ie;
             const int base = ie - cbase;                      // position of the group in chunk A (< 32)
             const uint32_t dsta = ring_sa + goff * (PB * kSlotVecs * 16);
-            if (left >= PB && base <= 32 - PB) {
+            // the window of the next 32 entries: lanes below `base` have handed out their chunk-A entry
+            // already and present their chunk-B entry instead, so entry base + b sits in lane (base + b) % 32
+            const int m_col = lane >= base ? a_col : b_col;
+            const float m_w = lane >= base ? a_w : b_w;
+            const int rel = (lane - base) & 31;               // entry of the window held by this lane
+            if (left >= PB) {
 #pragma unroll
                 for (int b = 0; b < PB; ++b) {
-                    const uint32_t k = (uint32_t)__shfl_sync(0xffffffffu, a_col, base + b);
+                    const uint32_t k = (uint32_t)__shfl_sync(0xffffffffu, m_col, base + b);
                     const char* src = zeta_l + (uint64_t)k * row_bytes;
 #pragma unroll
                     for (int c = 0; c < NCH; ++c)
                         if (kFull || active[c]) cp_async16_s(dsta + (b * kSlotVecs + c * 32) * 16, src + c * 512);
                 }
-                if ((unsigned)(lane - base) < (unsigned)PB) wfifo[goff * PB + lane - base] = a_w;
+                if (rel < PB) wfifo[goff * PB + rel] = m_w;
                 ie += PB;
             } else {
-                const int cnt = min(PB, left);
 #pragma unroll
-                for (int b = 0; b < PB; ++b)
-                    if (b < cnt) {
-                        const int idx = base + b;
-                        const uint32_t k = (uint32_t)(idx < 32 ? __shfl_sync(0xffffffffu, a_col, idx)
-                                                               : __shfl_sync(0xffffffffu, b_col, idx - 32));
-                        const char* src = zeta_l + (uint64_t)k * row_bytes;
+                for (int b = 0; b < PB - 1; ++b) {
+                    const uint32_t k = (uint32_t)__shfl_sync(0xffffffffu, m_col, base + b);
+                    const char* src = zeta_l + (uint64_t)k * row_bytes;
+                    if (b < left) {
 #pragma unroll
                         for (int c = 0; c < NCH; ++c)
                             if (kFull || active[c]) cp_async16_s(dsta + (b * kSlotVecs + c * 32) * 16, src + c * 512);
                     }
-                const int rel = lane - base;                  // the lanes that hold these entries write their weights
-                if (rel >= 0 && rel < cnt) wfifo[goff * PB + rel] = a_w;
-                if (rel + 32 < cnt) wfifo[goff * PB + rel + 32] = b_w;
-                ie += cnt;
+                }
+                if (rel < left) wfifo[goff * PB + rel] = m_w;
+                ie += left;
             }
             ++issued;
             if (ie == iend) {
@@ -564,11 +569,159 @@ __device__ __forceinline__ void stream_rows_wide(const SpmmDev& p, uint4* ring, 
     cp_async_wait<0>();
 }
 
+// acc[0..16) += w * (the 16 signed bytes of one 16-byte vector).  A byte b becomes the float
+// 2^23 + (b + 128) by placing b ^ 0x80 in the low mantissa byte of 0x4B000000 (one byte-permute, no
+// conversion unit); subtracting 2^23 + 128 gives b exactly; both steps and the FMA use the packed
+// two-lane fp32 instructions.
+__device__ __forceinline__ void fma_bytes16(float w, const uint4& v, float (&acc)[16])
+{
+    const uint32_t x[4] = {v.x ^ 0x80808080u, v.y ^ 0x80808080u, v.z ^ 0x80808080u, v.w ^ 0x80808080u};
+    const float2 ww = make_float2(w, w);
+    const float2 bias = make_float2(-8388736.f, -8388736.f);   // -(2^23 + 128)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 lo = make_float2(__uint_as_float(__byte_perm(x[i], 0x4B000000u, 0x7540)),
+                                      __uint_as_float(__byte_perm(x[i], 0x4B000000u, 0x7541)));
+        const float2 hi = make_float2(__uint_as_float(__byte_perm(x[i], 0x4B000000u, 0x7542)),
+                                      __uint_as_float(__byte_perm(x[i], 0x4B000000u, 0x7543)));
+        const float2 r0 = __ffma2_rn(ww, __fadd2_rn(lo, bias), make_float2(acc[4 * i], acc[4 * i + 1]));
+        const float2 r1 = __ffma2_rn(ww, __fadd2_rn(hi, bias), make_float2(acc[4 * i + 2], acc[4 * i + 3]));
+        acc[4 * i] = r0.x, acc[4 * i + 1] = r0.y, acc[4 * i + 2] = r1.x, acc[4 * i + 3] = r1.y;
+    }
+}
+
+// The row-aligned stream for 256-byte rows of 8-bit elements (up to 256 columns): a position holds
+// TWO stored entries, one per half warp (lane = 16 g + l fetches and accumulates the 16 bytes l of
+// entry 2 b + g of position b), so the per-position bookkeeping is shared by two entries and a lane's
+// 16-byte vector still carries 16 columns.  A group is 4 positions = 8 entries and never straddles a
+// row (a row takes ceil(deg / 8) groups, at least one).  The two half-warp sums are added when a row
+// completes.  Cursors, metadata chunks and the weight ring are those of stream_rows_wide; the
+// weights of a group are stored half by half (index 4 g + b) so that a lane reads its four with one
+// 16-byte load.  kFull: the row has exactly 16 vectors, no lane needs masking.
+template <bool kFull, bool kPartial>
+__device__ __forceinline__ void stream_rows_pair(const SpmmDev& p, uint4* ring, float* wfifo, const float* ctab, int lane,
+                                                 int64_t e0, int n_ent, int64_t warp_row0, int row_lo,
+                                                 int row_hi, int rp_rel, float (&acc)[1][16])
+{
+    using P = Pipe<1, 16, true>;
+    constexpr int PB = P::PB, NG = P::NG, EG = 2 * PB;        // positions and entries per group
+    static_assert(PB == 4 && (NG & (NG - 1)) == 0, "float4 weight reads; power-of-two group ring");
+    const int g = lane >> 4, l = lane & 15;
+    const bool active = l < p.nv;
+    const int32_t* cols = p.colidx + e0;
+    const float* vals = p.val + e0;
+    auto load_col = [&](int e) { return e < n_ent ? __ldg(cols + e) : 0; };
+    auto load_val = [&](int e) { return e < n_ent ? __ldg(vals + e) : 0.f; };
+    auto load_nw = [&](int col) { return p.node_w ? __ldg(p.node_w + col) : 1.f; };
+    auto row_end_of = [&](int r) { return kPartial ? n_ent : __shfl_sync(0xffffffffu, rp_rel, r + 1); };
+    const uint4* ring_l = ring + lane;                        // this lane's 16 bytes of slot 0
+    const uint32_t ring_sa = (uint32_t)__cvta_generic_to_shared(ring_l);
+    const char* zeta_l = reinterpret_cast<const char*>(p.zeta + l);
+    const uint32_t row_bytes = (uint32_t)p.nv * 16u;
+
+    int a_col = load_col(lane), b_col = load_col(32 + lane), c_col = load_col(64 + lane), d_col = load_col(96 + lane);
+    float a_w = load_val(lane), b_w = load_val(32 + lane), c_val = load_val(64 + lane), d_val = load_val(96 + lane);
+    a_w *= load_nw(a_col);
+    b_w *= load_nw(b_col);
+    float c_nw = load_nw(c_col);
+    int cbase = 0;                                            // first entry of chunk A
+
+    int ie = 0, ir = row_lo, iend = row_end_of(row_lo);       // issue cursor: entry, row, end of that row
+    int re = 0, rr = row_lo, rend = iend;                     // retire cursor
+    bool more = row_lo < row_hi;
+    int issued = 0, goff = 0;                                 // groups issued; ring position of the current group
+    zero_acc<1, 16>(acc);
+
+    for (int it = 0;; ++it) {
+        if (it >= NG) {
+            if (it - NG >= issued) break;
+            // ---- retire the oldest group
+            cp_async_wait<NG - 1>();
+            __syncwarp();
+            const uint4* gp = ring_l + goff * (PB * 32);
+            uint4 v[PB];
+#pragma unroll
+            for (int b = 0; b < PB; ++b) v[b] = gp[b * 32];
+            const float4 w4 = *reinterpret_cast<const float4*>(wfifo + goff * EG + 4 * g);
+            const float w[PB] = {w4.x, w4.y, w4.z, w4.w};
+            const int left = rend - re;
+            if (left >= EG) {
+#pragma unroll
+                for (int b = 0; b < PB; ++b)
+                    if (kFull || active) fma_bytes16(w[b], v[b], acc[0]);
+                re += EG;
+            } else {
+#pragma unroll
+                for (int b = 0; b < PB; ++b)
+                    if (2 * b + g < left && (kFull || active)) fma_bytes16(w[b], v[b], acc[0]);
+                re = rend;
+            }
+            if (re == rend) {                                 // the row is complete
+                reduce_groups<1, 16, 16>(acc);
+                if (kPartial) return;
+                finish_row<int8_t, 1, 16>(p, ctab, warp_row0 + rr, lane, acc);
+                zero_acc<1, 16>(acc);
+                ++rr;
+                if (rr < row_hi) rend = row_end_of(rr);
+            }
+            __syncwarp();                                     // all lanes are done with these slots
+        }
+        if (more) {
+            // ---- issue the next group of the row under the issue cursor
+            const int left = iend - ie;
+            const int base = ie - cbase;                      // position of the group in chunk A (< 32)
+            const uint32_t dsta = ring_sa + goff * (PB * 512);
+            // the window of the next 32 entries: lanes below `base` present their chunk-B entry, so
+            // entry base + e sits in lane (base + e) % 32
+            const int m_col = lane >= base ? a_col : b_col;
+            const float m_w = lane >= base ? a_w : b_w;
+            const int rel = (lane - base) & 31;               // entry of the window held by this lane
+            const int cnt = min(EG, left);
+#pragma unroll
+            for (int b = 0; b < PB; ++b) {
+                const uint32_t k = (uint32_t)__shfl_sync(0xffffffffu, m_col, base + 2 * b + g);
+                if ((cnt == EG || 2 * b + g < cnt) && (kFull || active)) cp_async16_s(dsta + b * 512, zeta_l + (uint64_t)k * row_bytes);
+            }
+            if (rel < cnt) wfifo[goff * EG + 4 * (rel & 1) + (rel >> 1)] = m_w;
+            ie += cnt;
+            ++issued;
+            if (ie == iend) {
+                ++ir;
+                if (ir == row_hi) more = false;
+                else iend = row_end_of(ir);
+            }
+            if (ie - cbase >= 32) {                           // rotate the metadata chunks
+                a_col = b_col;
+                a_w = b_w;
+                b_col = c_col;
+                b_w = c_val * c_nw;
+                c_col = d_col;
+                c_val = d_val;
+                c_nw = load_nw(c_col);
+                cbase += 32;
+                d_col = load_col(cbase + 96 + lane);
+                d_val = load_val(cbase + 96 + lane);
+            }
+        }
+        cp_async_commit();                                    // one group per iteration, possibly empty
+        goff = (goff + 1) & (NG - 1);
+    }
+    cp_async_wait<0>();
+}
+
+// Thread blocks per SM the kernel is compiled for (register budget) and launched with (grid size).
+template <typename T, int NCH, int LPR>
+constexpr int spmm_blocks_per_sm()
+{
+    return NCH == 1 ? ((LPR == 32 || UsesPairStream<T, NCH, LPR>::value) ? 3 : 4) : (NCH == 2 ? 2 : 1);
+}
+
 template <typename T, int NCH, int LPR, bool kFull>
-__global__ void __launch_bounds__(kSpmmThreads, NCH == 1 ? (LPR == 32 ? 3 : 4) : (NCH == 2 ? 2 : 1))
+__global__ void __launch_bounds__(kSpmmThreads, spmm_blocks_per_sm<T, NCH, LPR>())
 spmm_kernel(const SpmmDev p, int rows_per_warp)
 {
-    using P = Pipe<NCH, LPR>;
+    constexpr bool kPair = UsesPairStream<T, NCH, LPR>::value;
+    using P = Pipe<NCH, LPR, kPair>;
     constexpr int EPV = Elt<T>::kPerVec;
     constexpr int G = P::G;
     constexpr int kCols = (LPR < 32 ? LPR : NCH * 32) * EPV;  // accumulator columns of one warp
@@ -614,6 +767,9 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
                 if constexpr (LPR == 32)
                     stream_rows_wide<T, NCH, kFull, false>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
                                                     (int)(rp_reg - e0), acc);
+                else if constexpr (kPair)
+                    stream_rows_pair<kFull, false>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
+                                                   (int)(rp_reg - e0), acc);
                 else
                     stream_entries<T, NCH, LPR, false>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
                                                        (int)(rp_reg - e0), acc);
@@ -631,6 +787,8 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
         const int64_t s0 = min(le, ls + warp * slice), s1 = min(le, s0 + slice);
         if constexpr (LPR == 32)
             stream_rows_wide<T, NCH, kFull, true>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
+        else if constexpr (kPair)
+            stream_rows_pair<kFull, true>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
         else
             stream_entries<T, NCH, LPR, true>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
         __syncthreads();                                      // every ring is idle: reuse them for the partial sums
@@ -661,7 +819,7 @@ template <typename T, int NCH, int LPR, bool kFull = false>
 cudaError_t launch_one(cudaStream_t s, const SpmmDev& p)
 {
     constexpr int kCols = (LPR < 32 ? LPR : NCH * 32) * Elt<T>::kPerVec;
-    constexpr size_t smem = kSpmmWarps * Pipe<NCH, LPR>::kWarpBytes + 3 * kCols * sizeof(float);   // rings, weights, column table
+    constexpr size_t smem = kSpmmWarps * Pipe<NCH, LPR, UsesPairStream<T, NCH, LPR>::value>::kWarpBytes + 3 * kCols * sizeof(float);   // rings, weights, column table
     // enough thread blocks to fill the machine on small graphs, long runs of rows on large ones
     const int rows_per_warp = (int)std::min<int64_t>(kMaxRowsPerWarp, std::max<int64_t>(1, p.n / (kSpmmWarps * 148 * 8)));
     if (smem > 40 * 1024) {                                   // above the default limit: opt in
@@ -672,7 +830,7 @@ cudaError_t launch_one(cudaStream_t s, const SpmmDev& p)
     if (e != cudaSuccess) return e;
     // one wave of resident blocks; the warps pull runs of rows until none are left
     const int64_t wanted = ceil_div(ceil_div(p.n, rows_per_warp), kSpmmWarps);
-    const unsigned grid = (unsigned)std::min<int64_t>(wanted, 148 * (NCH == 1 ? (LPR == 32 ? 3 : 4) : (NCH == 2 ? 2 : 1)));
+    const unsigned grid = (unsigned)std::min<int64_t>(wanted, 148 * spmm_blocks_per_sm<T, NCH, LPR>());
     spmm_kernel<T, NCH, LPR, kFull><<<grid, kSpmmThreads, smem, s>>>(p, rows_per_warp);
     return cudaGetLastError();
 }
@@ -685,6 +843,9 @@ cudaError_t dispatch(cudaStream_t s, const SpmmDev& p)
     if (nv <= 2) return launch_one<T, 1, 2>(s, p);
     if (nv <= 4) return launch_one<T, 1, 4>(s, p);
     if (nv <= 8) return launch_one<T, 1, 8>(s, p);
+    if constexpr (sizeof(T) == 1) {
+        if (nv == 16) return launch_one<T, 1, 16, true>(s, p);   // 256-byte rows: no lane masking
+    }
     if (nv <= 16) return launch_one<T, 1, 16>(s, p);
     if (nv == 32) return launch_one<T, 1, 32, true>(s, p);
     if (nv <= 32) return launch_one<T, 1, 32>(s, p);
