@@ -405,11 +405,12 @@ def run_ours(args):
     spmm_ms = [mean(v) for v in per_kernel["spmm"]]
     gemm_ms = [mean(v) for v in per_kernel["gemm"]]
     pack_ms = mean(per_kernel["pack"])
-    fmt = args.zeta_format or binding.ZETA_F16
     kernels = {}
     dom = max(range(L), key=lambda l: spmm_ms[l])
     for l in range(L):
-        f = fmt
+        f = args.zeta_format                      # the library's rule for the storage of zeta, layer by layer
+        if f == 0:
+            f = binding.ZETA_I8 if (dims[l] <= 127 and 128 < dims[l + 1] <= 256) else binding.ZETA_F16
         if f == binding.ZETA_I8 and dims[l] > 127:
             f = binding.ZETA_F16
         if f == binding.ZETA_F16 and dims[l] > 2048:
@@ -458,7 +459,7 @@ def run_ours(args):
             "vs_baseline": None, "dtype": DTYPE, "data": "synthetic",
             "config": {"workload": workload_description(spec, n, nnz), "l2": "inputs_exceed_l2",
                        "parallelism": "replicas" if world > 1 else "single-gpu",
-                       "zeta_format": {0: "auto(f16)", 1: "f32", 2: "i16", 3: "i8", 4: "f16"}[args.zeta_format]},
+                       "zeta_format": {0: "auto", 1: "f32", 2: "i16", 3: "i8", 4: "f16"}[args.zeta_format]},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
             "step_ms_median": statistics.median(per_kernel["step"]), "step_ms_min": min(per_kernel["step"]),
             "extras": extras, "kernels": kernels}

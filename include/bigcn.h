@@ -57,7 +57,8 @@ typedef struct bigcn_ctx bigcn_ctx;
 /* Options for bigcn_set_option(). */
 enum {
     /* Storage of the rescaled contraction zeta between the bit-GEMM and the aggregation.
-     * 0 = choose per layer (default: 4 when d_in <= 2048, else 2);
+     * 0 = choose per layer (default: 3 for d_in <= 127 with 129..256 output columns, where the
+     *     aggregation streams 256-byte rows; otherwise 4 when d_in <= 2048, else 2);
      * 1 = fp32 zeta_ij = (beta_i alpha_j) dot_ij, exactly Eq. "cdot-op";
      * 2 = the integer dot products as int16, with beta folded into the edge weights and alpha
      *     applied once per output element (same sum, different rounding order);

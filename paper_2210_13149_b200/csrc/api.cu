@@ -54,11 +54,13 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) %
 
 size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
-// Storage format of zeta for a layer under the context's option.
-int pick_format(const bigcn_ctx* ctx, int d_in)
+// Storage format of zeta for a layer under the context's option.  Automatic choice: integers coded as
+// fp16 (exact up to d_in = 2048); for d_in <= 127 and 129..256 output columns the dots fit signed bytes
+// and the aggregation has a row-aligned stream for 256-byte rows that moves half the bytes.
+int pick_format(const bigcn_ctx* ctx, int d_in, int d_out)
 {
     int f = ctx->zeta_format;
-    if (f == 0) f = kZetaF16;
+    if (f == 0) f = (d_in <= 127 && d_out > 128 && d_out <= 256) ? kZetaI8 : kZetaF16;
     if (f == kZetaI8 && d_in > 127) f = kZetaF16;      // |dot| must fit the element type exactly
     if (f == kZetaF16 && d_in > 2048) f = kZetaI16;
     if (f == kZetaI16 && d_in > 32767) f = kZetaF32;
@@ -112,7 +114,7 @@ bigcn_status run_layer(bigcn_ctx* ctx, const bigcn_graph* g, const bigcn_layer* 
                        float* next_beta, int32_t* dbg_dot, float* dbg_zeta,
                        cudaEvent_t ev_mid /*nullable*/)
 {
-    const int fmt = pick_format(ctx, layer->d_in);
+    const int fmt = pick_format(ctx, layer->d_in, layer->d_out);
     const int64_t ldz = zeta_ld(layer->d_out, fmt);
     const int64_t stride_in = bigcn_packed_stride_words(layer->d_in);
     cudaError_t e = launch_bitgemm(ctx->stream, in_bits, stride_in, layer->w_bitsT, stride_in, g->n,
@@ -749,7 +751,7 @@ bigcn_status bigcn_sage_layer_forward(bigcn_ctx* ctx, const bigcn_graph* mean_gr
     cudaError_t e = launch_bitgemm(ctx->stream, in_bits, stride_in, self_layer->w_bitsT, stride_in, n, d_in, d_out,
                                    in_beta, self_layer->alpha, kZetaF32, zeta_self, ld_self, nullptr, nullptr, &ctx->launches_i);
     if (e != cudaSuccess) { finish_call(ctx); return cuda_fail(ctx, e, "bit-GEMM (self term) launch"); }
-    const int fmt = pick_format(ctx, d_in);
+    const int fmt = pick_format(ctx, d_in, d_out);
     const int64_t ldz = zeta_ld(d_out, fmt);
     e = launch_bitgemm(ctx->stream, in_bits, stride_in, nbr_layer->w_bitsT, stride_in, n, d_in, d_out,
                        in_beta, nbr_layer->alpha, fmt, zeta_nbr, ldz, nullptr, nullptr, &ctx->launches_i);

@@ -69,7 +69,7 @@ extern "C" bigcn_status bigcn_layer_forward_noalloc(void* cuda_stream, const big
     if (next && (!next_bits || !next_beta)) return BIGCN_ERR_NULL;
     if (!aligned16(in_bits) || !aligned16(layer->w_bitsT)) return BIGCN_ERR_ALIGN;
 
-    // same storage choice as the default of bigcn_layer_forward()
+    // zeta as integers coded in fp16 (int16 / fp32 beyond their exact ranges): 2 bytes per element decide the size limit
     const int fmt = layer->d_in <= 2048 ? kZetaF16 : (layer->d_in <= 32767 ? kZetaI16 : kZetaF32);
     const int64_t ldz = zeta_ld(layer->d_out, fmt);
     const size_t zeta_bytes = (size_t)graph->n * (size_t)ldz * zeta_elt_bytes(fmt);

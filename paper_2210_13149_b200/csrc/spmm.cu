@@ -677,10 +677,19 @@ __device__ __forceinline__ void stream_rows_pair(const SpmmDev& p, uint4* ring, 
             const float m_w = lane >= base ? a_w : b_w;
             const int rel = (lane - base) & 31;               // entry of the window held by this lane
             const int cnt = min(EG, left);
+            const int src_lane = base + g;                    // lane of the window that holds entry g of the group
+            if (cnt == EG) {
 #pragma unroll
-            for (int b = 0; b < PB; ++b) {
-                const uint32_t k = (uint32_t)__shfl_sync(0xffffffffu, m_col, base + 2 * b + g);
-                if ((cnt == EG || 2 * b + g < cnt) && (kFull || active)) cp_async16_s(dsta + b * 512, zeta_l + (uint64_t)k * row_bytes);
+                for (int b = 0; b < PB; ++b) {
+                    const uint32_t k = (uint32_t)__shfl_sync(0xffffffffu, m_col, src_lane + 2 * b);
+                    if (kFull || active) cp_async16_s(dsta + b * 512, zeta_l + (uint64_t)k * row_bytes);
+                }
+            } else {
+#pragma unroll
+                for (int b = 0; b < PB; ++b) {
+                    const uint32_t k = (uint32_t)__shfl_sync(0xffffffffu, m_col, src_lane + 2 * b);
+                    if (2 * b + g < cnt && (kFull || active)) cp_async16_s(dsta + b * 512, zeta_l + (uint64_t)k * row_bytes);
+                }
             }
             if (rel < cnt) wfifo[goff * EG + 4 * (rel & 1) + (rel >> 1)] = m_w;
             ie += cnt;
