@@ -202,7 +202,7 @@ bigcn_status bigcn_forward_host(bigcn_ctx* ctx, const bigcn_graph* graph, const 
  * in, forward, copy out) before the next begins, so the link to the host and the GPU take turns.
  * A pipeline keeps `slots` steps in flight on three streams: while step k computes on the context's
  * stream, the input of step k+1 is copied in and the logits of step k-1 are copied out.  The paper
- * has no counterpart of these calls (its measurements start from device-resident data, Sec. 6); each
+ * has no counterpart of these calls (its costs are operation and byte counts, Sec. 5, not transfers); each
  * step computes exactly what bigcn_forward() computes.
  *   bigcn_pipeline_open   copies the graph and layer descriptions (their device arrays must outlive
  *                         the pipeline) and creates streams and events; allocates no device memory.

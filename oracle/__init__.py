@@ -73,6 +73,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_mean_adjacency.restype = _c_i64
         L.oracle_mean_adjacency.argtypes = [_c_i64, _c_i64, _vp, _vp, _vp, _vp, _vp, _vp]
         L.oracle_spmm_add.argtypes = [_c_i64, _vp, _vp, _vp, _vp, _c_i32, _c_i64, _vp, _c_i64, _vp, _c_i64]
+        L.oracle_entropy_bins.argtypes = [_vp, _c_i64, _c_i32, _c_i64, _c_i32, _vp, _vp, _vp, _vp]
+        L.oracle_entropy_bins.restype = _c_f64
         _lib = L
     return _lib
 
@@ -380,3 +382,25 @@ def sage_layer_forward(g_mean: Graph, layer: SageLayer, H: np.ndarray) -> SageTr
     z_n = rescale(dot_popc(bits, bT_n, d_in), beta, a_n)
     H_out = spmm_add(g_mean, z_n, z_s)
     return SageTrace(F, beta, bits, bT_s, a_s, bT_n, a_n, z_s, z_n, H_out)
+
+
+@dataclass
+class EntropyEstimate:
+    """Binning estimate of Sec. 6.2: per-neuron range, interval counts, entropies in bits, and their sum."""
+    col_min: np.ndarray      # [d] float32
+    col_max: np.ndarray      # [d] float32
+    counts: np.ndarray       # [d, M] int64
+    entropy: np.ndarray      # [d] float64, bits
+    total: float             # H_ind = sum of the per-neuron entropies
+
+
+def entropy_bins(H: np.ndarray, n_bins: int) -> EntropyEstimate:
+    """H_hat(h_i) = -sum_m p log2 p over M equal-width intervals of each column's own range (Sec. 6.2)."""
+    H = _arr(H, np.float32)
+    n, d = H.shape
+    lo = np.empty(d, np.float32)
+    hi = np.empty(d, np.float32)
+    counts = np.empty((d, n_bins), np.int64)
+    ent = np.empty(d, np.float64)
+    total = lib().oracle_entropy_bins(_p(H), n, d, H.shape[1], n_bins, _p(lo), _p(hi), _p(counts), _p(ent))
+    return EntropyEstimate(lo, hi, counts, ent, float(total))

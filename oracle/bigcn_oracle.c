@@ -413,3 +413,60 @@ void oracle_cost_model(double n, double e, const int32_t* dims, int32_t n_layers
     out[4] = 32.0 * n * d0 / 8.0;                                    /* Eq. "DC" numerator */
     out[5] = (n * d0 + 32.0 * n) / 8.0;                              /* its denominator */
 }
+
+/* ------------------------------------------------------------------------- */
+/* Sec. 6.2 "Entropy Estimation of Hidden Layers": the binning estimate.      */
+/* For neuron (column) i over the N samples (rows): the value range           */
+/* [min_i, max_i] is cut into M intervals of equal width, p_{i,m} is the      */
+/* fraction of samples in interval m (the empirical distribution), and        */
+/*     H_hat(h_i) = - sum_m p_{i,m} log p_{i,m}.                              */
+/* The layer estimate is the independent sum H_ind(h) = sum_i H_hat(h_i).     */
+/* Readings (the paper fixes neither): equal-width intervals over the         */
+/* column's own range; the largest value falls into the last interval; a      */
+/* constant column has entropy 0; the logarithm is base 2 (bits), which the   */
+/* paper's own table forces (its PubMed value exceeds 16 ln 200).             */
+/* The interval index is decided in fp32, in this order:                      */
+/*     scale = (float)M / (max - min);  m = (int)((x - min) * scale)          */
+/* then clamped to M - 1.  Inputs must be finite.                             */
+/* counts: d x M, entropy: d values in bits.  Returns H_ind.                  */
+/* ------------------------------------------------------------------------- */
+double oracle_entropy_bins(const float* H, int64_t n, int32_t d, int64_t ld, int32_t M,
+                           float* col_min, float* col_max, int64_t* counts, double* entropy)
+{
+    double total = 0.0;
+    for (int32_t j = 0; j < d; ++j) {
+        float lo = INFINITY, hi = -INFINITY;
+        for (int64_t i = 0; i < n; ++i) {
+            const float x = H[i * ld + j];
+            if (x < lo) lo = x;
+            if (x > hi) hi = x;
+        }
+        col_min[j] = lo;
+        col_max[j] = hi;
+        int64_t* c = counts + (int64_t)j * M;
+        for (int32_t m = 0; m < M; ++m) c[m] = 0;
+        if (n > 0) {
+            if (hi > lo) {
+                const float scale = (float)M / (hi - lo);
+                for (int64_t i = 0; i < n; ++i) {
+                    const float t = (H[i * ld + j] - lo) * scale;
+                    int32_t m = (int32_t)t;
+                    if (m > M - 1) m = M - 1;
+                    c[m] += 1;
+                }
+            } else {
+                c[0] = n;                      /* every sample has the same value */
+            }
+        }
+        double h = 0.0;
+        for (int32_t m = 0; m < M; ++m) {
+            if (c[m] > 0) {
+                const double p = (double)c[m] / (double)n;
+                h -= p * log2(p);
+            }
+        }
+        entropy[j] = h;
+        total += h;
+    }
+    return total;
+}

@@ -434,3 +434,83 @@ def test_sage_layer_general_inputs_and_distinct_weights():
     Wnt = np.abs(Wn).astype(np.float64).mean(0, keepdims=True) * np.where(Wn >= 0, 1.0, -1.0)
     ref = Ht @ Wst + to_dense(g) @ (Ht @ Wnt)
     np.testing.assert_allclose(t.H_out, ref, rtol=1e-5, atol=1e-6)
+
+
+# --------------------------------------------------------------------------- entropy estimator (Sec. 6.2)
+
+def test_entropy_uniform_column_is_log2_of_the_interval_count():
+    """N = r * M samples spread evenly over the range fill every interval r times: H = log2 M exactly."""
+    M, r = 64, 5
+    x = np.repeat(np.arange(M, dtype=np.float32) + 0.5, r)        # r samples in the middle of each unit interval
+    x = np.concatenate([x, np.float32([0.0, M])])                  # pin the range to [0, M]: +1 in the first and last
+    rng = np.random.default_rng(1)
+    H = rng.permutation(x)[:, None].astype(np.float32)
+    est = oracle.entropy_bins(H, M)
+    assert est.col_min[0] == 0.0 and est.col_max[0] == M
+    want = np.full(M, r); want[0] += 1; want[-1] += 1              # the maximum falls into the last interval
+    assert np.array_equal(est.counts[0], want)
+    p = want / want.sum()
+    assert est.entropy[0] == pytest.approx(-(p * np.log2(p)).sum(), rel=1e-14)
+    assert est.entropy[0] == pytest.approx(np.log2(M), abs=2e-3) and est.entropy[0] < np.log2(M)
+
+
+def test_entropy_closed_forms():
+    n = 1000
+    H = np.zeros((n, 4), np.float32)
+    H[:, 0] = 3.25                                                 # constant neuron: no information
+    H[: n // 2, 1] = -1.0; H[n // 2:, 1] = 2.0                     # fair coin: one bit
+    H[: n // 4, 2] = 0.0; H[n // 4:, 2] = 1.0                      # 1/4 - 3/4 split
+    H[:, 3] = np.arange(n, dtype=np.float32)                       # n distinct values, M >= n intervals: log2 n bits
+    est = oracle.entropy_bins(H, 4096)
+    assert est.entropy[0] == 0.0 and est.counts[0, 0] == n and est.counts[0, 1:].sum() == 0
+    assert est.entropy[1] == pytest.approx(1.0, abs=1e-15)
+    assert est.entropy[2] == pytest.approx(-(0.25 * np.log2(0.25) + 0.75 * np.log2(0.75)), rel=1e-14)
+    assert est.entropy[3] == pytest.approx(np.log2(n), rel=1e-12)
+    assert est.total == pytest.approx(est.entropy.sum(), rel=1e-15)   # H_ind is the plain sum over the neurons
+    assert (est.counts.sum(axis=1) == n).all()
+
+
+def test_entropy_against_library_histogram():
+    """numpy's histogram over the same M equal-width intervals of [min, max] is the same empirical
+    distribution (up to samples that sit on an interval edge to within fp32 rounding)."""
+    rng = np.random.default_rng(7)
+    n, d, M = 20000, 6, 200
+    H = (rng.standard_normal((n, d)) * rng.uniform(0.5, 3.0, d) + rng.uniform(-2, 2, d)).astype(np.float32)
+    H[:, 1] = np.maximum(H[:, 1], 0)                               # a rectified neuron: a spike in the first interval
+    est = oracle.entropy_bins(H, M)
+    for j in range(d):
+        c, _ = np.histogram(H[:, j].astype(np.float64), bins=M, range=(float(H[:, j].min()), float(H[:, j].max())))
+        assert np.abs(c - est.counts[j]).sum() <= 8                # edge cases only
+        p = c[c > 0] / n
+        assert est.entropy[j] == pytest.approx(-(p * np.log2(p)).sum(), abs=2e-3)
+        assert est.entropy[j] <= np.log2(M)
+    assert est.col_min.tolist() == H.min(axis=0).tolist() and est.col_max.tolist() == H.max(axis=0).tolist()
+
+
+def test_entropy_permutation_and_affine_invariance():
+    """The estimate depends on the empirical distribution only: the order of the samples does not matter,
+    and a power-of-two rescaling plus shift of a neuron (exact in fp32 here) leaves every count unchanged."""
+    rng = np.random.default_rng(11)
+    H = np.round(rng.standard_normal((5000, 3)) * 64).astype(np.float32)     # multiples of 1: shifts stay exact
+    a = oracle.entropy_bins(H, 100)
+    b = oracle.entropy_bins(H[rng.permutation(len(H))], 100)
+    c = oracle.entropy_bins(H * np.float32(4.0) + np.float32(1024.0), 100)
+    assert np.array_equal(a.counts, b.counts) and np.array_equal(a.counts, c.counts)
+    assert np.array_equal(a.entropy, b.entropy) and np.array_equal(a.entropy, c.entropy)
+
+
+def test_entropy_table_of_the_paper_fixes_the_logarithm():
+    """Every printed estimate respects H <= n_h log2 M; the PubMed one exceeds n_h ln M, so the paper's
+    logarithm cannot be the natural one: bits."""
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "paper_entropy_table.txt")) if l.strip() and not l.startswith("#")]
+    assert len(rows) == 4
+    for name, kind, nh, ns, M, h in rows:
+        nh, ns, M, h = int(nh), int(ns), int(M), float(h)
+        assert h <= nh * np.log2(M)
+        assert h <= nh * np.log2(ns)
+    nh, M, h = int(rows[0][2]), int(rows[0][4]), float(rows[0][5])
+    assert h > nh * np.log(M)
+    # and the oracle attains the bound it is held to: M equally likely intervals give log2 M per neuron
+    x = (np.arange(M * 3, dtype=np.float32) % M)[:, None]
+    est = oracle.entropy_bins(np.concatenate([x, np.float32([[M]])]), M)
+    assert est.entropy[0] == pytest.approx(np.log2(M), abs=1e-2)
