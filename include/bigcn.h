@@ -198,6 +198,23 @@ bigcn_status bigcn_forward_host(bigcn_ctx* ctx, const bigcn_graph* graph, const 
                                 int32_t n_layers, const float* X_host, int64_t ldx,
                                 float* logits_host, int64_t ldo);
 
+/* Binning estimate of the entropy of a layer's activations (Sec. 6.2, "Entropy Estimation of Hidden
+ * Layers"): for every neuron (column j of H, fp32 [n x d], ld >= d) over the n samples (rows), the
+ * empirical distribution over n_bins intervals and H_hat(h_j) = -sum_m p_jm log2 p_jm; total =
+ * H_ind(h) = sum_j H_hat(h_j), the lower bound the Entropy Cover Hypothesis puts on the width of a
+ * binary hidden layer.  The paper fixes neither the intervals nor the logarithm; here: n_bins
+ * intervals of equal width over the column's own range [min_j, max_j]; the interval of a value x is
+ * decided in fp32 as m = (int)((x - min_j) * ((float)n_bins / (max_j - min_j))), clamped to
+ * n_bins - 1 (the maximum falls into the last interval); a constant column puts every sample into
+ * interval 0; entropies are in bits.  Values must be finite.
+ * Outputs (device): col_min, col_max [d] fp32; counts [d x n_bins] uint32 (overwritten; n < 2^31);
+ * entropy [d] and total [1] in double.  1 <= n_bins <= 8192 (BIGCN_ERR_UNSUPPORTED above).  With
+ * n = 0 the counts and entropies are zero and col_min / col_max are left untouched.  Needs 8 * d
+ * bytes of workspace.  Four launches, two passes over H. */
+bigcn_status bigcn_entropy_bins(bigcn_ctx* ctx, const float* H, int64_t n, int32_t d, int64_t ld,
+                                int32_t n_bins, float* col_min, float* col_max, uint32_t* counts,
+                                double* entropy, double* total);
+
 /* Back-to-back forwards from host buffers, overlapped.  bigcn_forward_host() finishes one step (copy
  * in, forward, copy out) before the next begins, so the link to the host and the GPU take turns.
  * A pipeline keeps `slots` steps in flight on three streams: while step k computes on the context's

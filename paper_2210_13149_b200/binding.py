@@ -75,6 +75,7 @@ SIGNATURES = {
     "bigcn_sage_layer_forward": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer),
                                                 ctypes.POINTER(bigcn_layer), _vp, _vp, _vp, _i64,
                                                 ctypes.POINTER(bigcn_layer), _vp, _vp]),
+    "bigcn_entropy_bins": (ctypes.c_int, [_vp, _vp, _i64, _i32, _i64, _i32, _vp, _vp, _vp, _vp, _vp]),
     "bigcn_measure_popc_peak": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_double)]),
     "bigcn_layer_forward_noalloc": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer),
                                                    _vp, _vp, _vp, _i64, ctypes.POINTER(bigcn_layer), _vp, _vp]),
@@ -340,6 +341,18 @@ class BiGCN:
         h = _vp()
         self._check(self.lib.bigcn_pipeline_open(self.h, ctypes.byref(graph.c), arr, len(layers), slots, ctypes.byref(h)))
         return Pipeline(self, h, graph, list(layers), dims)
+
+    def entropy_bins(self, H: torch.Tensor, n_bins: int):
+        """Binning entropy estimate (Sec. 6.2): dict of col_min, col_max, counts [d x n_bins], entropy [d] (bits), total."""
+        n, d = H.shape
+        self.ensure_workspace(8 * d)
+        out = dict(col_min=self._empty(d, torch.float32), col_max=self._empty(d, torch.float32),
+                   counts=self._empty((d, n_bins), torch.int32), entropy=self._empty(d, torch.float64),
+                   total=self._empty(1, torch.float64))
+        self._check(self.lib.bigcn_entropy_bins(self.h, _ptr(H), n, d, H.stride(0) if n > 1 else d, n_bins,
+                                                _ptr(out["col_min"]), _ptr(out["col_max"]), _ptr(out["counts"]),
+                                                _ptr(out["entropy"]), _ptr(out["total"])))
+        return out
 
     def col_stats(self, H: torch.Tensor, eps: float = 1e-5):
         n, d = H.shape

@@ -664,6 +664,31 @@ bigcn_status bigcn_col_stats(bigcn_ctx* ctx, const float* H, int64_t n, int32_t 
     return BIGCN_OK;
 }
 
+bigcn_status bigcn_entropy_bins(bigcn_ctx* ctx, const float* H, int64_t n, int32_t d, int64_t ld,
+                                int32_t n_bins, float* col_min, float* col_max, uint32_t* counts,
+                                double* entropy, double* total)
+{
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    if (n < 0 || n >= (int64_t(1) << 31) || d < 1 || ld < d || n_bins < 1)
+        return fail(ctx, BIGCN_ERR_SHAPE, "n=%lld d=%d ld=%lld n_bins=%d", (long long)n, d, (long long)ld, n_bins);
+    if (n_bins > entropy_max_bins()) return fail(ctx, BIGCN_ERR_UNSUPPORTED, "n_bins=%d exceeds %d", n_bins, entropy_max_bins());
+    if (!col_min || !col_max || !counts || !entropy || !total || (n > 0 && !H))
+        return fail(ctx, BIGCN_ERR_NULL, "H or an output is null");
+    if (n == 0) {
+        BIGCN_CUDA(ctx, cudaMemsetAsync(counts, 0, (size_t)d * n_bins * 4, ctx->stream));
+        BIGCN_CUDA(ctx, cudaMemsetAsync(entropy, 0, (size_t)d * 8, ctx->stream));
+        BIGCN_CUDA(ctx, cudaMemsetAsync(total, 0, 8, ctx->stream));
+        return BIGCN_OK;
+    }
+    if (!ctx->ws || ctx->ws_bytes < entropy_scratch_bytes(d)) return fail(ctx, BIGCN_ERR_WORKSPACE, "needs %zu bytes of workspace", entropy_scratch_bytes(d));
+    cudaError_t e = launch_entropy_bins(ctx->stream, H, n, d, ld, n_bins, col_min, col_max, counts, entropy, total,
+                                        ctx->ws, &ctx->launches_i);
+    finish_call(ctx);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "entropy estimate launch");
+    return BIGCN_OK;
+}
+
 bigcn_status bigcn_measure_popc_peak(bigcn_ctx* ctx, double* word_steps_per_s)
 {
     bigcn_status st = bind_device(ctx);

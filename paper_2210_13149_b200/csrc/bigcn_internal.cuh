@@ -77,4 +77,11 @@ size_t col_stats_scratch_bytes(int d);
 cudaError_t measure_popc_peak(cudaStream_t s, void* scratch, double* word_steps_per_s, int* launches);
 size_t popc_peak_scratch_bytes();
 
+// Binning entropy estimate (entropy.cu): scratch = 2 * d uint32.
+cudaError_t launch_entropy_bins(cudaStream_t s, const float* H, int64_t n, int d, int64_t ld, int n_bins,
+                                float* col_min, float* col_max, uint32_t* counts, double* entropy, double* total,
+                                void* scratch, int* launches);
+size_t entropy_scratch_bytes(int d);
+int entropy_max_bins();
+
 }  // namespace bigcn
