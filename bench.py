@@ -36,8 +36,9 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default="c5", help="workload c1..c5 (default: the largest, c5)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--model", default="gcn", choices=["gcn", "sage"],
-                    help="gcn: the Bi-GCN forward (the benchmark); sage: side benchmark of the Bi-GraphSAGE layers")
+    ap.add_argument("--model", default="gcn", choices=["gcn", "sage", "entropy"],
+                    help="gcn: the Bi-GCN forward (the benchmark); sage: side benchmark of the Bi-GraphSAGE layers; "
+                         "entropy: side benchmark of the binning entropy estimator")
     ap.add_argument("--zeta-format", type=int, default=0, help="0 auto, 1 fp32, 2 int16, 3 int8, 4 fp16")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -539,12 +540,68 @@ def run_sage(args):
     print(json.dumps(line), flush=True)
 
 
+def run_entropy(args):
+    """Side benchmark of the binning entropy estimator (Sec. 6.2) on synthetic activations with the shape
+    of the largest row of the paper's entropy table: 2,449,029 samples x 128 neurons, 1000 intervals
+    (scaled by --scale).  Single GPU; prints one JSON line; the oracle is timed on a bounded sample."""
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2210_13149_b200 import binding
+
+    n, d, M = max(1, int(2449029 * (args.scale or 1.0))), 128, 1000
+    dev = torch.device("cuda", 0)
+    g = torch.Generator(device=dev).manual_seed(2210)
+    H = torch.randn((n, d), device=dev, generator=g) * (torch.rand(d, device=dev, generator=g) * 3.8 + 0.2)
+    H[:, ::4].clamp_(min=0)                        # every fourth neuron rectified
+    ctx = binding.BiGCN(0)
+    for _ in range(max(args.warmup, 3)):
+        out = ctx.entropy_bins(H, M)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.25)
+    launches0 = ctx.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        out = ctx.entropy_bins(H, M)
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    peak, peak_kind = load_peaks()
+    algo = 2.0 * n * d * 4                          # the matrix is read twice: range pass, histogram pass
+    cpu = None
+    if not args.no_cpu_baseline:
+        ns = min(n, 200000)
+        Hs = H[:ns].cpu().numpy()
+        t0 = time.perf_counter()
+        ref = oracle.entropy_bins(Hs, M)
+        dt = time.perf_counter() - t0
+        got = ctx.entropy_bins(H[:ns], M)
+        assert np.array_equal(got["counts"].cpu().numpy().astype(np.int64), ref.counts)
+        cpu = {"value": ns / dt, "unit": "samples/s", "cores": 1, "kind": "oracle",
+               "sample": "the first %d samples of the same matrix (counts checked against the GPU's)" % ns}
+    line = {"metric": "entropy_estimate_samples_per_s", "value": n / (ms * 1e-3), "unit": "samples/s", "n_gpus": 1,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32 compare + u32 count + f64 log", "data": "synthetic",
+            "config": {"workload": "binning entropy estimate, %d samples x %d neurons, %d intervals" % (n, d, M),
+                       "l2": "inputs_exceed_l2"},
+            "clocks": sampler.stop(), "gpu_launches": ctx.launch_count() - launches0,
+            "roofline": {"bound": "hbm", "achieved": algo / (ms * 1e-3) / 1e9, "peak": peak, "peak_kind": "%s copy bandwidth" % peak_kind,
+                         "unit": "GB/s", "frac": algo / (ms * 1e-3) / 1e9 / peak, "traffic": None},
+            "cpu_baseline": cpu, "H_ind_bits": out["total"].item()}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
     elif args.model == "sage":
         run_sage(args)
+    elif args.model == "entropy":
+        run_entropy(args)
     else:
         run_ours(args)
 
