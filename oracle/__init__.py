@@ -75,6 +75,7 @@ def lib() -> ctypes.CDLL:
         L.oracle_spmm_add.argtypes = [_c_i64, _vp, _vp, _vp, _vp, _c_i32, _c_i64, _vp, _c_i64, _vp, _c_i64]
         L.oracle_entropy_bins.argtypes = [_vp, _c_i64, _c_i32, _c_i64, _c_i32, _vp, _vp, _vp, _vp]
         L.oracle_entropy_bins.restype = _c_f64
+        L.oracle_layer_backward.argtypes = [_c_i64, _vp, _vp, _vp, _c_i32, _c_i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
         _lib = L
     return _lib
 
@@ -404,3 +405,32 @@ def entropy_bins(H: np.ndarray, n_bins: int) -> EntropyEstimate:
     ent = np.empty(d, np.float64)
     total = lib().oracle_entropy_bins(_p(H), n, d, H.shape[1], n_bins, _p(lo), _p(hi), _p(counts), _p(ent))
     return EntropyEstimate(lo, hi, counts, ent, float(total))
+
+
+@dataclass
+class BackwardTrace:
+    """Algorithm 1 for one layer: the three gradients of step 1, then Eq. bp-H and Eq. bp-W."""
+    G_zeta: np.ndarray       # [n, d_out]   A_tilde^T G'
+    G_Wt: np.ndarray         # [d_in, d_out] gradient of the binarized weights W~
+    G_Ht: np.ndarray         # [n, d_in]    gradient of the binarized input H~
+    G_H: np.ndarray          # [n, d_in]    Eq. bp-H
+    G_W: np.ndarray          # [d_in, d_out] Eq. bp-W
+
+
+def layer_backward(g: Graph, W: np.ndarray, F: np.ndarray, beta: np.ndarray, G_out: np.ndarray) -> BackwardTrace:
+    """Back-propagation through H' = A_tilde ((beta F)(alpha B)) with B, alpha from W (Algorithm 1, Sec. 4.3).
+    F is the +-1 input of the forward pass and beta its row scales."""
+    W = _arr(W, np.float32)
+    d_in, d_out = W.shape
+    Bm, alpha = binarize_cols(W)
+    F = _arr(F, np.int8)
+    beta = _arr(beta, np.float32)
+    G_out = _arr(G_out, np.float32)
+    n = g.n
+    assert F.shape == (n, d_in) and G_out.shape == (n, d_out)
+    out = BackwardTrace(np.empty((n, d_out), np.float32), np.empty((d_in, d_out), np.float32),
+                        np.empty((n, d_in), np.float32), np.empty((n, d_in), np.float32),
+                        np.empty((d_in, d_out), np.float32))
+    lib().oracle_layer_backward(n, _p(g.rowptr), _p(g.colidx), _p(g.val), d_in, d_out, _p(F), _p(beta), _p(Bm), _p(alpha),
+                                _p(W), _p(G_out), _p(out.G_zeta), _p(out.G_Wt), _p(out.G_Ht), _p(out.G_H), _p(out.G_W))
+    return out

@@ -470,3 +470,67 @@ double oracle_entropy_bins(const float* H, int64_t n, int32_t d, int64_t ld, int
     }
     return total;
 }
+
+/* ------------------------------------------------------------------------- */
+/* Algorithm 1 (Sec. 4.3): back-propagation through one binarized graph       */
+/* convolutional layer  H' = A_tilde (H~ W~),  H~_ik = beta_i F_ik,           */
+/* W~_kj = alpha_j B_kj.  Given G' = dL/dH' (n x d_out):                      */
+/*   step 1:  G_zeta = A_tilde^T G'                                           */
+/*            G_W~   = H~^T G_zeta            (d_in x d_out)                  */
+/*            G_H~   = G_zeta W~^T            (n x d_in)                      */
+/*   step 2 (Eq. bp-H):  G_H = G_H~ where |G_H~| < 1, else 0                  */
+/*   step 3 (Eq. bp-W):  G_W_ij = (1/d_in) B_ij sum_k G_W~_kj B_kj            */
+/*                               + alpha_j G_W~_ij [ |W_ij| < 1 ]             */
+/*            (the last factor is the straight-through estimate of            */
+/*             d sign(r)/dr = 1_{|r|<1}).                                     */
+/* Step 4 of the algorithm (the parameter update) belongs to the optimiser    */
+/* and is not part of this function.  A_tilde^T is applied as a true          */
+/* transpose: entry (i, k) of A_tilde sends row i of G' to row k of G_zeta.   */
+/* All sums in double; every output rounded to float once.  g_zeta, g_wt,     */
+/* g_ht are the intermediate results (nullable).                              */
+/* ------------------------------------------------------------------------- */
+void oracle_layer_backward(int64_t n, const int64_t* rowptr, const int32_t* colidx, const float* val,
+                           int32_t d_in, int32_t d_out, const int8_t* F, const float* beta,
+                           const int8_t* B, const float* alpha, const float* W,
+                           const float* G_out, float* g_zeta, float* g_wt, float* g_ht,
+                           float* g_h, float* g_w)
+{
+    double* gz = (double*)calloc((size_t)n * d_out, sizeof(double));
+    double* gwt = (double*)calloc((size_t)d_in * d_out, sizeof(double));
+    /* G_zeta = A_tilde^T G' */
+    for (int64_t i = 0; i < n; ++i)
+        for (int64_t e = rowptr[i]; e < rowptr[i + 1]; ++e) {
+            const int64_t k = colidx[e];
+            for (int32_t j = 0; j < d_out; ++j) gz[k * d_out + j] += (double)val[e] * (double)G_out[i * d_out + j];
+        }
+    /* G_W~ = H~^T G_zeta */
+    for (int64_t i = 0; i < n; ++i)
+        for (int32_t k = 0; k < d_in; ++k) {
+            const double h = (double)beta[i] * (double)F[i * d_in + k];
+            for (int32_t j = 0; j < d_out; ++j) gwt[(int64_t)k * d_out + j] += h * gz[i * d_out + j];
+        }
+    /* G_H~ = G_zeta W~^T, then Eq. bp-H */
+    for (int64_t i = 0; i < n; ++i)
+        for (int32_t k = 0; k < d_in; ++k) {
+            double s = 0.0;
+            for (int32_t j = 0; j < d_out; ++j)
+                s += gz[i * d_out + j] * ((double)alpha[j] * (double)B[(int64_t)k * d_out + j]);
+            if (g_ht) g_ht[i * d_in + k] = (float)s;
+            if (g_h) g_h[i * d_in + k] = (fabs(s) < 1.0) ? (float)s : 0.f;
+        }
+    /* Eq. bp-W */
+    for (int32_t j = 0; j < d_out; ++j) {
+        double col = 0.0;                                  /* sum_k G_W~_kj B_kj */
+        for (int32_t k = 0; k < d_in; ++k) col += gwt[(int64_t)k * d_out + j] * (double)B[(int64_t)k * d_out + j];
+        for (int32_t i = 0; i < d_in; ++i) {
+            const int64_t at = (int64_t)i * d_out + j;
+            double g = (double)B[at] * col / (double)d_in;
+            if (fabsf(W[at]) < 1.0f) g += (double)alpha[j] * gwt[at];
+            if (g_w) g_w[at] = (float)g;
+        }
+    }
+    if (g_zeta) for (int64_t t = 0; t < n * d_out; ++t) g_zeta[t] = (float)gz[t];
+    if (g_wt) for (int64_t t = 0; t < (int64_t)d_in * d_out; ++t) g_wt[t] = (float)gwt[t];
+    free(gz);
+    free(gwt);
+}

@@ -514,3 +514,110 @@ def test_entropy_table_of_the_paper_fixes_the_logarithm():
     x = (np.arange(M * 3, dtype=np.float32) % M)[:, None]
     est = oracle.entropy_bins(np.concatenate([x, np.float32([[M]])]), M)
     assert est.entropy[0] == pytest.approx(np.log2(M), abs=1e-2)
+
+
+# --------------------------------------------------------------------------- back-propagation (Algorithm 1)
+
+def _bw_case(seed, n=23, d_in=11, d_out=7, asym=False):
+    rng = np.random.default_rng(seed)
+    src = rng.integers(0, n, 3 * n); dst = rng.integers(0, n, 3 * n)
+    g = oracle.normalize_adjacency(n, src, dst)
+    if asym:                                   # a non-symmetric sparse matrix on the same pattern: tells A^T from A
+        g = oracle.Graph(g.n, g.rowptr, g.colidx, (g.val * rng.uniform(0.5, 1.5, g.val.shape)).astype(np.float32), g.dinv)
+    W = (rng.standard_normal((d_in, d_out)) * 0.8).astype(np.float32)
+    H = rng.standard_normal((n, d_in)).astype(np.float32)
+    F, beta = oracle.binarize_rows(H)
+    G = (rng.standard_normal((n, d_out)) * 0.3).astype(np.float32)
+    return g, W, F, beta, G
+
+
+def _dense(g):
+    A = np.zeros((g.n, g.n))
+    for i in range(g.n):
+        for e in range(g.rowptr[i], g.rowptr[i + 1]):
+            A[i, g.colidx[e]] += float(g.val[e])
+    return A
+
+
+def test_backward_step1_is_the_gradient_of_the_linear_forward():
+    """H' = A (H~ W~) is linear in H~ and in W~: with L = <G', H'> the gradients are A^T G', H~^T A^T G' and
+    A^T G' W~^T exactly.  Checked against dense matrix algebra on a NON-symmetric A (so that A and A^T, and
+    every other transposition, cannot be confused) and against central differences of the dense forward."""
+    g, W, F, beta, G = _bw_case(1, asym=True)
+    bw = oracle.layer_backward(g, W, F, beta, G)
+    A = _dense(g)
+    Bm, alpha = oracle.binarize_cols(W)
+    Ht = beta[:, None].astype(np.float64) * F
+    Wt = alpha[None, :].astype(np.float64) * Bm
+    Gz = A.T @ G.astype(np.float64)
+    np.testing.assert_allclose(bw.G_zeta, Gz, rtol=1e-6, atol=1e-7)
+    np.testing.assert_allclose(bw.G_Wt, Ht.T @ Gz, rtol=1e-6, atol=1e-6)
+    np.testing.assert_allclose(bw.G_Ht, Gz @ Wt.T, rtol=1e-6, atol=1e-6)
+    assert not np.allclose(bw.G_zeta, A @ G, rtol=1e-3, atol=1e-4)          # the untransposed product is different
+    loss = lambda Hx, Wx: float((G.astype(np.float64) * (A @ (Hx @ Wx))).sum())
+    rng = np.random.default_rng(2)
+    for _ in range(6):
+        i, k, j = rng.integers(g.n), rng.integers(W.shape[0]), rng.integers(W.shape[1])
+        E = np.zeros_like(Wt); E[k, j] = 1.0
+        assert (loss(Ht, Wt + E) - loss(Ht, Wt - E)) / 2 == pytest.approx(bw.G_Wt[k, j], rel=1e-5, abs=1e-6)
+        E = np.zeros_like(Ht); E[i, k] = 1.0
+        assert (loss(Ht + E, Wt) - loss(Ht - E, Wt)) / 2 == pytest.approx(bw.G_Ht[i, k], rel=1e-5, abs=1e-6)
+
+
+def test_backward_eq_bp_H_is_a_strict_clip():
+    g, W, F, beta, G = _bw_case(3)
+    bw = oracle.layer_backward(g, W, F, beta, G * 8)                      # large enough that some |G_H~| exceed 1
+    big = np.abs(bw.G_Ht) >= 1
+    assert big.any() and (~big).any()
+    assert (bw.G_H[big] == 0).all() and np.array_equal(bw.G_H[~big], bw.G_Ht[~big])
+    # the boundary itself is excluded (|r| < 1): one node, one feature, weight 1, gradient exactly 1
+    g1 = oracle.Graph(1, np.array([0, 1], np.int64), np.array([0], np.int32), np.array([1.0], np.float32), np.ones(1, np.float32))
+    one = oracle.layer_backward(g1, np.array([[1.0]], np.float32), np.array([[1]], np.int8), np.ones(1, np.float32), np.array([[1.0]], np.float32))
+    assert one.G_Ht[0, 0] == 1.0 and one.G_H[0, 0] == 0.0
+    half = oracle.layer_backward(g1, np.array([[1.0]], np.float32), np.array([[1]], np.int8), np.ones(1, np.float32), np.array([[0.5]], np.float32))
+    assert half.G_H[0, 0] == 0.5
+
+
+def test_backward_eq_bp_W_terms():
+    """First term: the derivative through alpha_j = ||W_:,j||_1 / d_in with the signs held fixed, checked by
+    central differences.  Second term: alpha_j G_W~_ij where |W_ij| < 1 (straight-through estimate), else 0."""
+    g, W, F, beta, G = _bw_case(5)
+    W[0, 0] = 1.5; W[1, 0] = -1.0; W[2, 0] = 0.999                        # outside, on and inside the STE window
+    bw = oracle.layer_backward(g, W, F, beta, G)
+    Bm, alpha = oracle.binarize_cols(W)
+    d_in = W.shape[0]
+    col = (bw.G_Wt.astype(np.float64) * Bm).sum(axis=0)
+    first = Bm * col[None, :] / d_in
+    second = np.where(np.abs(W) < 1, alpha[None, :].astype(np.float64) * bw.G_Wt, 0.0)
+    # (G_W~ is read back rounded to fp32 here, the oracle carries it in double: 1e-5)
+    np.testing.assert_allclose(bw.G_W, first + second, rtol=1e-5, atol=1e-7)
+    assert bw.G_W[0, 0] == pytest.approx(first[0, 0], rel=1e-5) and bw.G_W[1, 0] == pytest.approx(first[1, 0], rel=1e-5)
+    assert bw.G_W[2, 0] == pytest.approx(first[2, 0] + alpha[0] * bw.G_Wt[2, 0], rel=1e-5)
+    # finite differences of L(W) = <G_W~, alpha(W) B> with B fixed reproduce the first term
+    Gwt = bw.G_Wt.astype(np.float64)
+    L = lambda Wx: float((Gwt * (np.abs(Wx).sum(axis=0, keepdims=True) / d_in * Bm)).sum())
+    for (i, j) in [(0, 0), (3, 2), (7, 6)]:
+        h = 1e-3
+        E = np.zeros(W.shape); E[i, j] = h
+        Wd = W.astype(np.float64)
+        assert (L(Wd + E) - L(Wd - E)) / (2 * h) == pytest.approx(first[i, j], rel=1e-6, abs=1e-9)
+
+
+def test_backward_plain_gcn_special_case():
+    """With +-1 inputs and +-1 weights (beta = alpha = 1) the layer is the plain GCN layer A X W, whose
+    gradients are textbook: dL/dW = X^T A^T G', dL/dX = A^T G' W^T."""
+    rng = np.random.default_rng(9)
+    n, d_in, d_out = 15, 6, 4
+    g = oracle.normalize_adjacency(n, rng.integers(0, n, 30), rng.integers(0, n, 30))
+    X = rng.choice([-1.0, 1.0], (n, d_in)).astype(np.float32)
+    W = rng.choice([-1.0, 1.0], (d_in, d_out)).astype(np.float32)
+    F, beta = oracle.binarize_rows(X)
+    assert (beta == 1).all()
+    G = (rng.standard_normal((n, d_out)) * 0.01).astype(np.float32)
+    bw = oracle.layer_backward(g, W, F, beta, G)
+    A = _dense(g)
+    np.testing.assert_allclose(bw.G_Wt, X.T.astype(np.float64) @ A.T @ G, rtol=1e-6, atol=1e-8)
+    np.testing.assert_allclose(bw.G_H, A.T @ G.astype(np.float64) @ W.T, rtol=1e-6, atol=1e-8)   # all |.| < 1: no clipping
+    # |W_ij| = 1 is outside the STE window: only the alpha-path term of Eq. bp-W remains
+    col = (bw.G_Wt.astype(np.float64) * W).sum(axis=0)
+    np.testing.assert_allclose(bw.G_W, W * col[None, :] / d_in, rtol=1e-5, atol=1e-9)
