@@ -215,6 +215,28 @@ bigcn_status bigcn_entropy_bins(bigcn_ctx* ctx, const float* H, int64_t n, int32
                                 int32_t n_bins, float* col_min, float* col_max, uint32_t* counts,
                                 double* entropy, double* total);
 
+/* Back-propagation through one binarized layer (Algorithm 1, Sec. 4.3).  The forward pass of the
+ * layer was H' = A_tilde (H~ W~) with H~_ik = beta_i F_ik (the packed input in_bits / in_beta of
+ * bigcn_layer_forward) and W~_kj = alpha_j sign(W_kj).  Given g_out = dL/dH' (fp32 [n x d_out],
+ * ldg >= d_out) the call computes, in the algorithm's order,
+ *   G_zeta = A_tilde^T g_out,  G_W~ = H~^T G_zeta,  G_H~ = G_zeta W~^T          (step 1)
+ *   g_in   = G_H~ where |G_H~| < 1, else 0                                       (step 2, Eq. bp-H)
+ *   g_w_ij = (1/d_in) B_ij sum_k G_W~_kj B_kj + alpha_j G_W~_ij [|W_ij| < 1]     (step 3, Eq. bp-W;
+ *            the bracket is the straight-through estimate of the sign's derivative)
+ * and leaves step 4, the parameter update, to the caller's optimiser.  W is the latent fp32 weight
+ * matrix [d_in x d_out] (ldw >= d_out) from which layer->w_bitsT and layer->alpha were packed.
+ * g_in fp32 [n x d_in] (ldgi >= d_in) is nullable (the first layer needs no input gradient);
+ * g_w fp32 [d_in x d_out] (ldgw >= d_out).  g_in is the gradient at the input of the binarization,
+ * i.e. after the layer's batch normalisation if it has one (the algorithm does not cover that step).
+ * A_tilde must be symmetric, as bigcn_normalize_adjacency() produces it: A_tilde^T is applied as
+ * A_tilde.  d_out <= 512.  Needs bigcn_backward_workspace_bytes(n, d_in, d_out) of workspace.
+ * fp32 throughout, sums over the nodes split into slabs that are added in a fixed order. */
+size_t bigcn_backward_workspace_bytes(int64_t n, int32_t d_in, int32_t d_out);
+bigcn_status bigcn_layer_backward(bigcn_ctx* ctx, const bigcn_graph* graph, const bigcn_layer* layer,
+                                  const float* W, int64_t ldw, const uint32_t* in_bits, const float* in_beta,
+                                  const float* g_out, int64_t ldg, float* g_in, int64_t ldgi,
+                                  float* g_w, int64_t ldgw);
+
 /* Back-to-back forwards from host buffers, overlapped.  bigcn_forward_host() finishes one step (copy
  * in, forward, copy out) before the next begins, so the link to the host and the GPU take turns.
  * A pipeline keeps `slots` steps in flight on three streams: while step k computes on the context's

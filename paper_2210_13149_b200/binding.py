@@ -76,6 +76,9 @@ SIGNATURES = {
                                                 ctypes.POINTER(bigcn_layer), _vp, _vp, _vp, _i64,
                                                 ctypes.POINTER(bigcn_layer), _vp, _vp]),
     "bigcn_entropy_bins": (ctypes.c_int, [_vp, _vp, _i64, _i32, _i64, _i32, _vp, _vp, _vp, _vp, _vp]),
+    "bigcn_backward_workspace_bytes": (_sz, [_i64, _i32, _i32]),
+    "bigcn_layer_backward": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer), _vp, _i64,
+                                            _vp, _vp, _vp, _i64, _vp, _i64, _vp, _i64]),
     "bigcn_measure_popc_peak": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_double)]),
     "bigcn_layer_forward_noalloc": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer),
                                                    _vp, _vp, _vp, _i64, ctypes.POINTER(bigcn_layer), _vp, _vp]),
@@ -341,6 +344,19 @@ class BiGCN:
         h = _vp()
         self._check(self.lib.bigcn_pipeline_open(self.h, ctypes.byref(graph.c), arr, len(layers), slots, ctypes.byref(h)))
         return Pipeline(self, h, graph, list(layers), dims)
+
+    def layer_backward(self, graph: Graph, layer: Layer, W: torch.Tensor, in_bits: torch.Tensor,
+                       in_beta: torch.Tensor, g_out: torch.Tensor, want_g_in: bool = True):
+        """Algorithm 1 for one layer: returns (g_in or None, g_w)."""
+        n = graph.n
+        self.ensure_workspace(int(self.lib.bigcn_backward_workspace_bytes(n, layer.d_in, layer.d_out)))
+        g_in = self._empty((n, layer.d_in), torch.float32) if want_g_in else None
+        g_w = self._empty((layer.d_in, layer.d_out), torch.float32)
+        self._check(self.lib.bigcn_layer_backward(
+            self.h, ctypes.byref(graph.c), ctypes.byref(layer.c), _ptr(W), W.stride(0) if layer.d_in > 1 else layer.d_out,
+            _ptr(in_bits), _ptr(in_beta), _ptr(g_out), g_out.stride(0) if n > 1 else layer.d_out,
+            _ptr(g_in), layer.d_in, _ptr(g_w), layer.d_out))
+        return g_in, g_w
 
     def entropy_bins(self, H: torch.Tensor, n_bins: int):
         """Binning entropy estimate (Sec. 6.2): dict of col_min, col_max, counts [d x n_bins], entropy [d] (bits), total."""

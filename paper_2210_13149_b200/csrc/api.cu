@@ -689,6 +689,43 @@ bigcn_status bigcn_entropy_bins(bigcn_ctx* ctx, const float* H, int64_t n, int32
     return BIGCN_OK;
 }
 
+size_t bigcn_backward_workspace_bytes(int64_t n, int32_t d_in, int32_t d_out)
+{
+    if (n < 0 || d_in < 1 || d_out < 1) return 0;
+    return backward_scratch_bytes(n, d_in, d_out) + kAlign;
+}
+
+bigcn_status bigcn_layer_backward(bigcn_ctx* ctx, const bigcn_graph* graph, const bigcn_layer* layer,
+                                  const float* W, int64_t ldw, const uint32_t* in_bits, const float* in_beta,
+                                  const float* g_out, int64_t ldg, float* g_in, int64_t ldgi,
+                                  float* g_w, int64_t ldgw)
+{
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    if ((st = check_graph(ctx, graph)) != BIGCN_OK) return st;
+    if ((st = check_layer(ctx, layer, "layer")) != BIGCN_OK) return st;
+    const int32_t d_in = layer->d_in, d_out = layer->d_out;
+    if (d_out > 512) return fail(ctx, BIGCN_ERR_UNSUPPORTED, "d_out=%d > 512", d_out);
+    if (ldw < d_out || ldg < d_out || ldgw < d_out || (g_in && ldgi < d_in))
+        return fail(ctx, BIGCN_ERR_SHAPE, "leading dimensions: ldw=%lld ldg=%lld ldgw=%lld ldgi=%lld", (long long)ldw, (long long)ldg, (long long)ldgw, (long long)ldgi);
+    if (!W || !g_w) return fail(ctx, BIGCN_ERR_NULL, "W or g_w is null");
+    const int64_t n = graph->n;
+    if (n > 0 && (!in_bits || !in_beta || !g_out)) return fail(ctx, BIGCN_ERR_NULL, "in_bits, in_beta or g_out is null");
+    if (n == 0) {                                             // no nodes: every sum over the nodes is empty
+        BIGCN_CUDA(ctx, cudaMemset2DAsync(g_w, (size_t)ldgw * 4, 0, (size_t)d_out * 4, (size_t)d_in, ctx->stream));
+        return BIGCN_OK;
+    }
+    if (!ctx->ws || ctx->ws_bytes < backward_scratch_bytes(n, d_in, d_out))
+        return fail(ctx, BIGCN_ERR_WORKSPACE, "needs %zu bytes of workspace (bigcn_backward_workspace_bytes)", backward_scratch_bytes(n, d_in, d_out));
+    cudaError_t e = launch_layer_backward(ctx->stream, n, graph->rowptr, graph->colidx, graph->val, d_in, d_out, W, ldw,
+                                          layer->alpha, in_bits, bigcn_packed_stride_words(d_in), in_beta, g_out, ldg,
+                                          g_in, ldgi, g_w, ldgw, ctx->long_row ? ctx->long_row : kDefaultLongRow, ctx->ws,
+                                          &ctx->launches_i);
+    finish_call(ctx);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "backward launch");
+    return BIGCN_OK;
+}
+
 bigcn_status bigcn_measure_popc_peak(bigcn_ctx* ctx, double* word_steps_per_s)
 {
     bigcn_status st = bind_device(ctx);

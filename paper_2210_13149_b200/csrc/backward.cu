@@ -1,0 +1,305 @@
+// Back-propagation through one binarized graph convolutional layer (Bi-GCN Algorithm 1, Sec. 4.3):
+//   G_zeta = A_tilde^T G'            (the aggregation kernel of the forward pass, fp32 rows)
+//   G_W~   = H~^T G_zeta             H~_ik = beta_i F_ik from the packed input bits
+//   G_H~   = G_zeta W~^T             W~_kj = alpha_j sign(W_kj)
+//   G_H    = G_H~ [|G_H~| < 1]       (Eq. bp-H)
+//   G_W_ij = (1/d_in) B_ij sum_k G_W~_kj B_kj + alpha_j G_W~_ij [|W_ij| < 1]   (Eq. bp-W)
+// The two dense products have one +-1 operand that is expanded from bits (or from the sign of W) into
+// shared memory tile by tile; the other operand and the accumulation are fp32.
+#include <algorithm>
+
+#include "bigcn_internal.cuh"
+
+namespace bigcn {
+
+namespace {
+
+constexpr int kBwThreads = 256;       // 16 x 16 threads, each a 4 x 4 block of the 64 x 64 output tile
+constexpr int kBwTile = 64;
+constexpr int kBwStep = 32;           // reduction elements staged per step
+
+// Copies rows of d floats into rows of ld_out floats (ld_out >= d, a multiple of 4), zero-filling the tail.
+__global__ void pad_rows_kernel(const float* __restrict__ src, int64_t n, int d, int64_t ld_in,
+                                float* __restrict__ dst, int64_t ld_out)
+{
+    const int64_t total = n * ld_out;
+    for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t i = t / ld_out;
+        const int j = (int)(t - i * ld_out);
+        dst[t] = j < d ? __ldg(src + i * ld_in + j) : 0.f;
+    }
+}
+
+// G_W~ partial sums.  Block (x, y, z): output tile k in [64 x, +64) x j in [64 y, +64), rows
+// [z * rows_per_split, +rows_per_split).  Per step of 32 rows the tile of H~ (beta_i * (+-1) from the
+// bits) and the tile of G_zeta go to shared memory; thread (ty, tx) accumulates k = 4 ty.., j = 4 tx...
+// Every split writes its own slab: part[z][k][j]; a second kernel adds the slabs in a fixed order.
+__global__ void __launch_bounds__(kBwThreads)
+grad_wt_partial_kernel(const uint32_t* __restrict__ bits, int64_t stride, const float* __restrict__ beta,
+                       const float* __restrict__ gz, int64_t ldz, int64_t n, int d_in, int d_out,
+                       int64_t rows_per_split, float* __restrict__ part)
+{
+    __shared__ __align__(16) float Hs[kBwStep][kBwTile + 4];
+    __shared__ __align__(16) float Gs[kBwStep][kBwTile + 4];
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int k0 = blockIdx.x * kBwTile, j0 = blockIdx.y * kBwTile;
+    const int64_t r_begin = (int64_t)blockIdx.z * rows_per_split;
+    const int64_t r_end = min(n, r_begin + rows_per_split);
+    float acc[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+    for (int64_t r0 = r_begin; r0 < r_end; r0 += kBwStep) {
+        // stage: 32 rows x 64 columns of each operand, 8 elements per thread
+        for (int t = threadIdx.x; t < kBwStep * kBwTile; t += kBwThreads) {
+            const int r = t >> 6, c = t & 63;
+            const int64_t row = r0 + r;
+            float h = 0.f, g = 0.f;
+            if (row < r_end) {
+                const int k = k0 + c;
+                if (k < d_in) {
+                    const uint32_t w = __ldg(bits + row * stride + (k >> 5));
+                    const float be = __ldg(beta + row);
+                    h = ((w >> (k & 31)) & 1u) ? be : -be;
+                }
+                const int j = j0 + c;
+                if (j < d_out) g = __ldg(gz + row * ldz + j);
+            }
+            Hs[r][c] = h;
+            Gs[r][c] = g;
+        }
+        __syncthreads();
+#pragma unroll 8
+        for (int r = 0; r < kBwStep; ++r) {
+            const float4 hv = *reinterpret_cast<const float4*>(&Hs[r][4 * ty]);
+            const float4 gv = *reinterpret_cast<const float4*>(&Gs[r][4 * tx]);
+            const float h[4] = {hv.x, hv.y, hv.z, hv.w};
+            const float g[4] = {gv.x, gv.y, gv.z, gv.w};
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(h[a], g[b], acc[a][b]);
+        }
+        __syncthreads();
+    }
+    float* slab = part + (int64_t)blockIdx.z * d_in * d_out;
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        const int k = k0 + 4 * ty + a;
+        if (k >= d_in) continue;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int j = j0 + 4 * tx + b;
+            if (j < d_out) slab[(int64_t)k * d_out + j] = acc[a][b];
+        }
+    }
+}
+
+// G_W~ = sum of the slabs, in slab order (double accumulation: the slabs can differ by orders of magnitude).
+__global__ void grad_wt_reduce_kernel(const float* __restrict__ part, int n_splits, int64_t elems, float* __restrict__ g_wt)
+{
+    const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (t >= elems) return;
+    double s = 0.0;
+    for (int z = 0; z < n_splits; ++z) s += (double)part[(int64_t)z * elems + t];
+    g_wt[t] = (float)s;
+}
+
+// G_H = clip(G_zeta W~^T).  Block (x, y): rows [64 x, +64) x inputs k in [64 y, +64); per step 32
+// output channels j: tile of G_zeta scaled by alpha_j, and the signs of W[k][j] as +-1.
+__global__ void __launch_bounds__(kBwThreads)
+grad_h_kernel(const float* __restrict__ gz, int64_t ldz, const float* __restrict__ alpha,
+              const float* __restrict__ W, int64_t ldw, int64_t n, int d_in, int d_out,
+              float* __restrict__ g_h, int64_t ldh)
+{
+    __shared__ __align__(16) float Gs[kBwStep][kBwTile + 4];          // [j][row]
+    __shared__ __align__(16) float Bs[kBwStep][kBwTile + 4];          // [j][k]
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int64_t i0 = (int64_t)blockIdx.x * kBwTile;
+    const int k0 = blockIdx.y * kBwTile;
+    float acc[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+    for (int j0 = 0; j0 < d_out; j0 += kBwStep) {
+        for (int t = threadIdx.x; t < kBwStep * kBwTile; t += kBwThreads) {
+            // G tile: consecutive threads read consecutive j of one row (coalesced), stored transposed
+            const int jr = t & 31, rr = t >> 5;
+            const int64_t row = i0 + rr;
+            const int j = j0 + jr;
+            Gs[jr][rr] = (row < n && j < d_out) ? __fmul_rn(__ldg(gz + row * ldz + j), __ldg(alpha + j)) : 0.f;
+            const int k = k0 + rr;
+            Bs[jr][rr] = (k < d_in && j < d_out) ? (__ldg(W + (int64_t)k * ldw + j) >= 0.f ? 1.f : -1.f) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll 8
+        for (int j = 0; j < kBwStep; ++j) {
+            const float4 gv = *reinterpret_cast<const float4*>(&Gs[j][4 * ty]);
+            const float4 bv = *reinterpret_cast<const float4*>(&Bs[j][4 * tx]);
+            const float g[4] = {gv.x, gv.y, gv.z, gv.w};
+            const float b[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) acc[a][c] = fmaf(g[a], b[c], acc[a][c]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        const int64_t row = i0 + 4 * ty + a;
+        if (row >= n) continue;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const int k = k0 + 4 * tx + c;
+            if (k < d_in) g_h[row * ldh + k] = fabsf(acc[a][c]) < 1.f ? acc[a][c] : 0.f;     // Eq. bp-H
+        }
+    }
+}
+
+// Eq. bp-W.  One block per 32 output channels: thread (tx, ty) sums G_W~_kj B_kj over k = ty, ty + 32, ...
+// for channel j0 + tx in double; the 32 partial sums of a channel are added in a fixed order; then
+// every element gets (1/d_in) B_ij col_j + alpha_j G_W~_ij [|W_ij| < 1].
+__global__ void __launch_bounds__(1024)
+grad_w_kernel(const float* __restrict__ g_wt, const float* __restrict__ W, int64_t ldw,
+              const float* __restrict__ alpha, int d_in, int d_out, float* __restrict__ g_w, int64_t ldgw)
+{
+    __shared__ double part[32][33];
+    __shared__ double col[32];
+    const int tx = threadIdx.x, ty = threadIdx.y;
+    const int j = blockIdx.x * 32 + tx;
+    double s = 0.0;
+    if (j < d_out)
+        for (int k = ty; k < d_in; k += 32) {
+            const float w = __ldg(W + (int64_t)k * ldw + j);
+            const double g = (double)__ldg(g_wt + (int64_t)k * d_out + j);
+            s += w >= 0.f ? g : -g;
+        }
+    part[ty][tx] = s;
+    __syncthreads();
+    if (ty == 0) {
+        double t = 0.0;
+        for (int r = 0; r < 32; ++r) t += part[r][tx];
+        col[tx] = t;
+    }
+    __syncthreads();
+    if (j < d_out) {
+        const double c = col[tx] / (double)d_in;
+        const float al = __ldg(alpha + j);
+        for (int i = ty; i < d_in; i += 32) {
+            const float w = __ldg(W + (int64_t)i * ldw + j);
+            double g = w >= 0.f ? c : -c;
+            if (fabsf(w) < 1.f) g += (double)al * (double)__ldg(g_wt + (int64_t)i * d_out + j);
+            g_w[(int64_t)i * ldgw + j] = (float)g;
+        }
+    }
+}
+
+int64_t pad4(int64_t d) { return (d + 3) / 4 * 4; }
+
+int wt_splits(int64_t n, int d_in, int d_out)
+{
+    const int64_t tiles = ceil_div(d_in, kBwTile) * ceil_div(d_out, kBwTile);
+    const int64_t want = std::max<int64_t>(1, (148 * 4) / tiles);               // about four blocks per SM in all
+    return (int)std::max<int64_t>(1, std::min<int64_t>(want, ceil_div(n, 4 * kBwStep)));
+}
+
+}  // namespace
+
+size_t backward_scratch_bytes(int64_t n, int d_in, int d_out)
+{
+    const size_t a = 256;
+    auto up = [&](size_t b) { return (b + a - 1) / a * a; };
+    size_t total = up((size_t)n * pad4(d_out) * 4);                              // G' with rows padded to 16 bytes
+    total += up((size_t)n * pad4(d_out) * 4);                                    // G_zeta
+    total += up((size_t)wt_splits(n, d_in, d_out) * d_in * d_out * 4);           // slabs of G_W~
+    total += up((size_t)d_in * d_out * 4);                                       // G_W~
+    total += up(spmm_scratch_bytes(n, 0, 0));
+    return total;
+}
+
+cudaError_t launch_layer_backward(cudaStream_t s, int64_t n, const int64_t* rowptr, const int32_t* colidx,
+                                  const float* val, int d_in, int d_out, const float* W, int64_t ldw,
+                                  const float* alpha, const uint32_t* in_bits, int64_t stride_in,
+                                  const float* in_beta, const float* g_out, int64_t ldg, float* g_in,
+                                  int64_t ldgi, float* g_w, int64_t ldgw, int64_t long_row, void* scratch,
+                                  int* launches)
+{
+    const size_t a = 256;
+    auto up = [&](size_t b) { return (b + a - 1) / a * a; };
+    char* base = static_cast<char*>(scratch);
+    const int64_t ldz = pad4(d_out);
+    float* g_pad = reinterpret_cast<float*>(base);
+    base += up((size_t)n * ldz * 4);
+    float* gz = reinterpret_cast<float*>(base);
+    base += up((size_t)n * ldz * 4);
+    const int n_splits = wt_splits(n, d_in, d_out);
+    float* part = reinterpret_cast<float*>(base);
+    base += up((size_t)n_splits * d_in * d_out * 4);
+    float* g_wt = reinterpret_cast<float*>(base);
+    base += up((size_t)d_in * d_out * 4);
+    void* counter = base;
+
+    // step 1a: G_zeta = A_tilde^T G' (A_tilde is symmetric: the forward aggregation on fp32 rows)
+    const float* g_src = g_out;
+    if (ldg != ldz || reinterpret_cast<uintptr_t>(g_out) % 16 != 0) {            // rows must be 16-byte vectors
+        pad_rows_kernel<<<(unsigned)std::min<int64_t>(ceil_div(n * ldz, 256), 148 * 16), 256, 0, s>>>(g_out, n, d_out, ldg, g_pad, ldz);
+        ++*launches;
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        g_src = g_pad;
+    }
+    SpmmArgs sa;
+    sa.n = n;
+    sa.rowptr = rowptr;
+    sa.colidx = colidx;
+    sa.val = val;
+    sa.fmt = kZetaF32;
+    sa.zeta = g_src;
+    sa.ldz = ldz;
+    sa.d_out = d_out;
+    sa.node_w = nullptr;
+    sa.col_w = nullptr;
+    sa.add = nullptr;
+    sa.ld_add = 0;
+    sa.h_out = gz;
+    sa.ldh = ldz;
+    sa.next_bits = nullptr;
+    sa.next_stride = 0;
+    sa.next_beta = nullptr;
+    sa.next_shift = nullptr;
+    sa.next_scale = nullptr;
+    sa.long_row = long_row;
+    sa.scratch = counter;
+    sa.scratch_bytes = spmm_scratch_bytes(n, 0, 0);
+    cudaError_t e = launch_spmm(s, sa, launches);
+    if (e != cudaSuccess) return e;
+
+    // step 1b: G_W~ = H~^T G_zeta, split over the rows, slabs added in a fixed order
+    {
+        const int64_t rows_per_split = ceil_div(ceil_div(n, n_splits), kBwStep) * kBwStep;
+        const dim3 grid((unsigned)ceil_div(d_in, kBwTile), (unsigned)ceil_div(d_out, kBwTile), (unsigned)n_splits);
+        grad_wt_partial_kernel<<<grid, kBwThreads, 0, s>>>(in_bits, stride_in, in_beta, gz, ldz, n, d_in, d_out, rows_per_split, part);
+        ++*launches;
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        const int64_t elems = (int64_t)d_in * d_out;
+        grad_wt_reduce_kernel<<<(unsigned)ceil_div(elems, 256), 256, 0, s>>>(part, n_splits, elems, g_wt);
+        ++*launches;
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    // step 1c + 2: G_H = clip(G_zeta W~^T)
+    if (g_in) {
+        const dim3 grid((unsigned)ceil_div(n, kBwTile), (unsigned)ceil_div(d_in, kBwTile));
+        grad_h_kernel<<<grid, kBwThreads, 0, s>>>(gz, ldz, alpha, W, ldw, n, d_in, d_out, g_in, ldgi);
+        ++*launches;
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    // step 3: Eq. bp-W
+    grad_w_kernel<<<(unsigned)ceil_div(d_out, 32), dim3(32, 32), 0, s>>>(g_wt, W, ldw, alpha, d_in, d_out, g_w, ldgw);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace bigcn

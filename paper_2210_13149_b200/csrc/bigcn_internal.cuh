@@ -84,4 +84,13 @@ cudaError_t launch_entropy_bins(cudaStream_t s, const float* H, int64_t n, int d
 size_t entropy_scratch_bytes(int d);
 int entropy_max_bins();
 
+// Back-propagation through one binarized layer (backward.cu).
+size_t backward_scratch_bytes(int64_t n, int d_in, int d_out);
+cudaError_t launch_layer_backward(cudaStream_t s, int64_t n, const int64_t* rowptr, const int32_t* colidx,
+                                  const float* val, int d_in, int d_out, const float* W, int64_t ldw,
+                                  const float* alpha, const uint32_t* in_bits, int64_t stride_in,
+                                  const float* in_beta, const float* g_out, int64_t ldg, float* g_in,
+                                  int64_t ldgi, float* g_w, int64_t ldgw, int64_t long_row, void* scratch,
+                                  int* launches);
+
 }  // namespace bigcn
