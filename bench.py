@@ -36,9 +36,10 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default="c5", help="workload c1..c5 (default: the largest, c5)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--model", default="gcn", choices=["gcn", "sage", "entropy"],
+    ap.add_argument("--model", default="gcn", choices=["gcn", "sage", "entropy", "backward"],
                     help="gcn: the Bi-GCN forward (the benchmark); sage: side benchmark of the Bi-GraphSAGE layers; "
-                         "entropy: side benchmark of the binning entropy estimator")
+                         "entropy: side benchmark of the binning entropy estimator; backward: side benchmark of Algorithm 1 "
+                         "for the hidden layer of the workload")
     ap.add_argument("--zeta-format", type=int, default=0, help="0 auto, 1 fp32, 2 int16, 3 int8, 4 fp16")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -594,6 +595,69 @@ def run_entropy(args):
     print(json.dumps(line), flush=True)
 
 
+def run_backward(args):
+    """Side benchmark of the back-propagation through one binarized layer (Algorithm 1) on the workload's
+    graph: the widest hidden layer (c5: 256 -> 256), input gradient included.  Single GPU; one JSON line;
+    the oracle is timed on a draw of the same recipe at a small scale."""
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2210_13149_b200 import binding, synth
+
+    dev = torch.device("cuda", 0)
+    spec = synth.scaled_spec(args.config, args.scale) if args.scale else synth.WORKLOADS[args.config]
+    wl = synth.make_workload(args.config, scale=args.scale, device=dev)
+    n = wl.n
+    dims = [w.shape[0] for w in wl.W] + [wl.W[-1].shape[1]]
+    l = max(range(1, len(wl.W)), key=lambda i: dims[i] * dims[i + 1]) if len(wl.W) > 1 else 0
+    d_in, d_out = dims[l], dims[l + 1]
+    ctx = binding.BiGCN(0)
+    G = ctx.normalize_adjacency(wl.rowptr, wl.colidx)
+    nnz = G.nnz
+    gen = torch.Generator(device=dev).manual_seed(77)
+    W = wl.W[l]
+    bitsT, alpha = ctx.pack_weights(W)
+    layer = binding.make_layer(d_in, d_out, bitsT, alpha)
+    bits, beta = ctx.pack_features(torch.randn((n, d_in), device=dev, generator=gen))
+    g_out = torch.randn((n, d_out), device=dev, generator=gen) * 0.02
+    for _ in range(max(args.warmup, 3)):
+        ctx.layer_backward(G, layer, W, bits, beta, g_out)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.25)
+    launches0 = ctx.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        ctx.layer_backward(G, layer, W, bits, beta, g_out)
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    cpu = None
+    if not args.no_cpu_baseline:
+        small = synth.make_workload(args.config, scale=min(1.0, 20000.0 / synth.WORKLOADS[args.config].n))
+        src, dst = synth.edge_list(small.rowptr, small.colidx)
+        g = oracle.normalize_adjacency(small.n, src, dst)
+        rng = np.random.default_rng(3)
+        F, be = oracle.binarize_rows(rng.standard_normal((small.n, d_in)).astype(np.float32))
+        go = (rng.standard_normal((small.n, d_out)) * 0.02).astype(np.float32)
+        t0 = time.perf_counter()
+        oracle.layer_backward(g, W.cpu().numpy(), F, be, go)
+        dt = time.perf_counter() - t0
+        cpu = {"value": small.n / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": "the same recipe at %d nodes, same layer widths" % small.n}
+    flops = 2.0 * 2.0 * n * d_in * d_out                 # the two dense products
+    line = {"metric": "bigcn_layer_backward_nodes_per_s", "value": n / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "Algorithm 1 for layer %d (%d -> %d) on " % (l, d_in, d_out) + workload_description(spec, n, nnz),
+                       "l2": "inputs_exceed_l2"},
+            "clocks": sampler.stop(), "gpu_launches": ctx.launch_count() - launches0,
+            "dense_products_TFLOPs_if_alone": flops / (ms * 1e-3) / 1e12, "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
@@ -602,6 +666,8 @@ def main():
         run_sage(args)
     elif args.model == "entropy":
         run_entropy(args)
+    elif args.model == "backward":
+        run_backward(args)
     else:
         run_ours(args)
 
