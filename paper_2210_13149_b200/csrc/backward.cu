@@ -8,6 +8,8 @@
 // shared memory tile by tile; the other operand and the accumulation are fp32.
 #include <algorithm>
 
+#include <cuda_bf16.h>
+
 #include "bigcn_internal.cuh"
 
 namespace bigcn {
@@ -159,6 +161,129 @@ grad_h_kernel(const float* __restrict__ gz, int64_t ldz, const float* __restrict
     }
 }
 
+// ---- tensor-core versions of the two dense products -------------------------------------------------
+// Both products have one operand that is exactly +-1 (exact in bf16) and one fp32 operand.  The fp32
+// operand x is split into three bf16 terms x = hi + mid + lo (each the rounding of what is left:
+// 3 x 8 significant bits cover fp32's 24), so three bf16 tensor-core products with fp32 accumulation
+// reproduce the fp32 product to fp32 accuracy.  mma.sync m16n8k16 (row-major A, column-major B):
+// with g = lane / 4, t = lane % 4 a thread holds A[g | g+8][2t, 2t+1 | +8], B[2t, 2t+1 | +8][g],
+// C[g | g+8][2t, 2t+1].  Tiles are staged in shared memory as bf16 with a row pitch of 40 elements
+// (20 words), which makes the fragment reads of a warp hit 32 different banks.
+constexpr int kMmaPitch = 40;                    // bf16 elements per staged row (32 + 8 pad)
+constexpr int kMmaTile = 128;                    // output tile 128 x 128 per block, 8 warps of 32 x 64
+constexpr int kMmaK = 32;                        // reduction elements per staged step
+
+__device__ __forceinline__ void split3(float x, unsigned short& hi, unsigned short& mid, unsigned short& lo)
+{
+    const __nv_bfloat16 h = __float2bfloat16_rn(x);
+    const float r1 = __fsub_rn(x, __bfloat162float(h));
+    const __nv_bfloat16 m = __float2bfloat16_rn(r1);
+    const float r2 = __fsub_rn(r1, __bfloat162float(m));
+    const __nv_bfloat16 l = __float2bfloat16_rn(r2);
+    hi = __bfloat16_as_ushort(h);
+    mid = __bfloat16_as_ushort(m);
+    lo = __bfloat16_as_ushort(l);
+}
+
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2])
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+
+// One staged step of the block's 128 x 128 tile: As[3][128][pitch] (the three terms of the fp32
+// operand, rows = output rows, k contiguous), Bs[128][pitch] (the +-1 operand, rows = output columns,
+// k contiguous).  Warp (wr, wc) owns rows 32 wr.., columns 64 wc...
+__device__ __forceinline__ void mma_step(const unsigned short* As, const unsigned short* Bs, int wr, int wc, int lane,
+                                         float (&acc)[2][8][4])
+{
+    const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int kk = 0; kk < kMmaK; kk += 16) {
+        uint32_t b[8][2];
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb) {
+            const unsigned short* p = Bs + (wc * 64 + nb * 8 + g) * kMmaPitch + kk + 2 * t;
+            b[nb][0] = *reinterpret_cast<const uint32_t*>(p);
+            b[nb][1] = *reinterpret_cast<const uint32_t*>(p + 8);
+        }
+#pragma unroll
+        for (int sp = 0; sp < 3; ++sp) {
+#pragma unroll
+            for (int mb = 0; mb < 2; ++mb) {
+                const unsigned short* p = As + (sp * kMmaTile + wr * 32 + mb * 16 + g) * kMmaPitch + kk + 2 * t;
+                uint32_t a[4];
+                a[0] = *reinterpret_cast<const uint32_t*>(p);
+                a[1] = *reinterpret_cast<const uint32_t*>(p + 8 * kMmaPitch);
+                a[2] = *reinterpret_cast<const uint32_t*>(p + 8);
+                a[3] = *reinterpret_cast<const uint32_t*>(p + 8 * kMmaPitch + 8);
+#pragma unroll
+                for (int nb = 0; nb < 8; ++nb) mma_bf16(acc[mb][nb], a, b[nb]);
+            }
+        }
+    }
+}
+
+// G_H = clip(G_zeta W~^T) on the tensor cores.  Block (x, y): rows [128 x, +128) x inputs k in
+// [128 y, +128); the reduction runs over the output channels j in steps of 32.  A = G_zeta * alpha_j
+// (split in three), B[k][j] = sign(W[k][j]).
+__global__ void __launch_bounds__(kBwThreads)
+grad_h_mma_kernel(const float* __restrict__ gz, int64_t ldz, const float* __restrict__ alpha,
+                  const float* __restrict__ W, int64_t ldw, int64_t n, int d_in, int d_out,
+                  float* __restrict__ g_h, int64_t ldh)
+{
+    __shared__ __align__(16) unsigned short As[3 * kMmaTile * kMmaPitch];
+    __shared__ __align__(16) unsigned short Bs[kMmaTile * kMmaPitch];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int wr = warp >> 1, wc = warp & 1;
+    const int64_t i0 = (int64_t)blockIdx.x * kMmaTile;
+    const int k0 = blockIdx.y * kMmaTile;
+    float acc[2][8][4];
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+        for (int b = 0; b < 8; ++b)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[a][b][c] = 0.f;
+    for (int j0 = 0; j0 < d_out; j0 += kMmaK) {
+        __syncthreads();                                   // the previous step's tiles are consumed
+        for (int t = threadIdx.x; t < kMmaTile * kMmaK; t += kBwThreads) {
+            const int jr = t & 31, rr = t >> 5;            // consecutive threads: consecutive j of one row
+            const int j = j0 + jr;
+            const int64_t row = i0 + rr;
+            const float x = (row < n && j < d_out) ? __fmul_rn(__ldg(gz + row * ldz + j), __ldg(alpha + j)) : 0.f;
+            unsigned short hi, mid, lo;
+            split3(x, hi, mid, lo);
+            As[(0 * kMmaTile + rr) * kMmaPitch + jr] = hi;
+            As[(1 * kMmaTile + rr) * kMmaPitch + jr] = mid;
+            As[(2 * kMmaTile + rr) * kMmaPitch + jr] = lo;
+            const int k = k0 + rr;
+            unsigned short sgn = 0;
+            if (k < d_in && j < d_out) sgn = __ldg(W + (int64_t)k * ldw + j) >= 0.f ? 0x3F80 : 0xBF80;
+            Bs[rr * kMmaPitch + jr] = sgn;
+        }
+        __syncthreads();
+        mma_step(As, Bs, wr, wc, lane, acc);
+    }
+    const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int mb = 0; mb < 2; ++mb)
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const int64_t row = i0 + wr * 32 + mb * 16 + g + 8 * half;
+            if (row >= n) continue;
+#pragma unroll
+            for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    const int k = k0 + wc * 64 + nb * 8 + 2 * t + q;
+                    const float v = acc[mb][nb][2 * half + q];
+                    if (k < d_in) g_h[row * ldh + k] = fabsf(v) < 1.f ? v : 0.f;            // Eq. bp-H
+                }
+        }
+}
+
 // Eq. bp-W.  One block per 32 output channels: thread (tx, ty) sums G_W~_kj B_kj over k = ty, ty + 32, ...
 // for channel j0 + tx in double; the 32 partial sums of a channel are added in a fixed order; then
 // every element gets (1/d_in) B_ij col_j + alpha_j G_W~_ij [|W_ij| < 1].
@@ -291,8 +416,8 @@ cudaError_t launch_layer_backward(cudaStream_t s, int64_t n, const int64_t* rowp
     }
     // step 1c + 2: G_H = clip(G_zeta W~^T)
     if (g_in) {
-        const dim3 grid((unsigned)ceil_div(n, kBwTile), (unsigned)ceil_div(d_in, kBwTile));
-        grad_h_kernel<<<grid, kBwThreads, 0, s>>>(gz, ldz, alpha, W, ldw, n, d_in, d_out, g_in, ldgi);
+        const dim3 grid((unsigned)ceil_div(n, kMmaTile), (unsigned)ceil_div(d_in, kMmaTile));
+        grad_h_mma_kernel<<<grid, kBwThreads, 0, s>>>(gz, ldz, alpha, W, ldw, n, d_in, d_out, g_in, ldgi);
         ++*launches;
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
