@@ -239,6 +239,7 @@ grad_h_mma_kernel(const float* __restrict__ gz, int64_t ldz, const float* __rest
     const int wr = warp >> 1, wc = warp & 1;
     const int64_t i0 = (int64_t)blockIdx.x * kMmaTile;
     const int k0 = blockIdx.y * kMmaTile;
+    const bool vec_ok = (ldz % 4 == 0) && (reinterpret_cast<uintptr_t>(gz) % 16 == 0);
     float acc[2][8][4];
 #pragma unroll
     for (int a = 0; a < 2; ++a)
@@ -248,20 +249,38 @@ grad_h_mma_kernel(const float* __restrict__ gz, int64_t ldz, const float* __rest
             for (int c = 0; c < 4; ++c) acc[a][b][c] = 0.f;
     for (int j0 = 0; j0 < d_out; j0 += kMmaK) {
         __syncthreads();                                   // the previous step's tiles are consumed
-        for (int t = threadIdx.x; t < kMmaTile * kMmaK; t += kBwThreads) {
-            const int jr = t & 31, rr = t >> 5;            // consecutive threads: consecutive j of one row
-            const int j = j0 + jr;
+        // stage 128 x 32 of each operand: a thread takes 4 consecutive j of one row (16-byte loads where the
+        // row allows it) and writes 8 bytes per term
+        for (int t = threadIdx.x; t < kMmaTile * (kMmaK / 4); t += kBwThreads) {
+            const int jq = (t & 7) * 4, rr = t >> 3;
+            const int j = j0 + jq;
             const int64_t row = i0 + rr;
-            const float x = (row < n && j < d_out) ? __fmul_rn(__ldg(gz + row * ldz + j), __ldg(alpha + j)) : 0.f;
-            unsigned short hi, mid, lo;
-            split3(x, hi, mid, lo);
-            As[(0 * kMmaTile + rr) * kMmaPitch + jr] = hi;
-            As[(1 * kMmaTile + rr) * kMmaPitch + jr] = mid;
-            As[(2 * kMmaTile + rr) * kMmaPitch + jr] = lo;
+            float x[4] = {0.f, 0.f, 0.f, 0.f};
+            if (row < n) {
+                if (j + 3 < d_out && vec_ok) {
+                    const float4 v = __ldg(reinterpret_cast<const float4*>(gz + row * ldz + j));
+                    x[0] = v.x, x[1] = v.y, x[2] = v.z, x[3] = v.w;
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        if (j + q < d_out) x[q] = __ldg(gz + row * ldz + j + q);
+                }
+            }
+            unsigned short hi[4], mid[4], lo[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) split3(j + q < d_out ? __fmul_rn(x[q], __ldg(alpha + j + q)) : 0.f, hi[q], mid[q], lo[q]);
+            auto pack = [](const unsigned short (&h)[4]) { return make_uint2((uint32_t)h[0] | ((uint32_t)h[1] << 16), (uint32_t)h[2] | ((uint32_t)h[3] << 16)); };
+            *reinterpret_cast<uint2*>(&As[(0 * kMmaTile + rr) * kMmaPitch + jq]) = pack(hi);
+            *reinterpret_cast<uint2*>(&As[(1 * kMmaTile + rr) * kMmaPitch + jq]) = pack(mid);
+            *reinterpret_cast<uint2*>(&As[(2 * kMmaTile + rr) * kMmaPitch + jq]) = pack(lo);
             const int k = k0 + rr;
-            unsigned short sgn = 0;
-            if (k < d_in && j < d_out) sgn = __ldg(W + (int64_t)k * ldw + j) >= 0.f ? 0x3F80 : 0xBF80;
-            Bs[rr * kMmaPitch + jr] = sgn;
+            unsigned short sg[4] = {0, 0, 0, 0};
+            if (k < d_in) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    if (j + q < d_out) sg[q] = __ldg(W + (int64_t)k * ldw + j + q) >= 0.f ? 0x3F80 : 0xBF80;
+            }
+            *reinterpret_cast<uint2*>(&Bs[rr * kMmaPitch + jq]) = pack(sg);
         }
         __syncthreads();
         mma_step(As, Bs, wr, wc, lane, acc);
