@@ -5,7 +5,8 @@
 //   G_H    = G_H~ [|G_H~| < 1]       (Eq. bp-H)
 //   G_W_ij = (1/d_in) B_ij sum_k G_W~_kj B_kj + alpha_j G_W~_ij [|W_ij| < 1]   (Eq. bp-W)
 // The two dense products have one +-1 operand that is expanded from bits (or from the sign of W) into
-// shared memory tile by tile; the other operand and the accumulation are fp32.
+// shared memory tile by tile as bf16; the fp32 operand is split into three bf16 terms; the products run
+// on the tensor cores with fp32 accumulation.
 #include <algorithm>
 
 #include <cuda_bf16.h>
@@ -16,9 +17,7 @@ namespace bigcn {
 
 namespace {
 
-constexpr int kBwThreads = 256;       // 16 x 16 threads, each a 4 x 4 block of the 64 x 64 output tile
-constexpr int kBwTile = 64;
-constexpr int kBwStep = 32;           // reduction elements staged per step
+constexpr int kBwThreads = 256;       // 8 warps per block
 
 // Copies rows of d floats into rows of ld_out floats (ld_out >= d, a multiple of 4), zero-filling the tail.
 __global__ void pad_rows_kernel(const float* __restrict__ src, int64_t n, int d, int64_t ld_in,
@@ -32,72 +31,6 @@ __global__ void pad_rows_kernel(const float* __restrict__ src, int64_t n, int d,
     }
 }
 
-// G_W~ partial sums.  Block (x, y, z): output tile k in [64 x, +64) x j in [64 y, +64), rows
-// [z * rows_per_split, +rows_per_split).  Per step of 32 rows the tile of H~ (beta_i * (+-1) from the
-// bits) and the tile of G_zeta go to shared memory; thread (ty, tx) accumulates k = 4 ty.., j = 4 tx...
-// Every split writes its own slab: part[z][k][j]; a second kernel adds the slabs in a fixed order.
-__global__ void __launch_bounds__(kBwThreads)
-grad_wt_partial_kernel(const uint32_t* __restrict__ bits, int64_t stride, const float* __restrict__ beta,
-                       const float* __restrict__ gz, int64_t ldz, int64_t n, int d_in, int d_out,
-                       int64_t rows_per_split, float* __restrict__ part)
-{
-    __shared__ __align__(16) float Hs[kBwStep][kBwTile + 4];
-    __shared__ __align__(16) float Gs[kBwStep][kBwTile + 4];
-    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-    const int k0 = blockIdx.x * kBwTile, j0 = blockIdx.y * kBwTile;
-    const int64_t r_begin = (int64_t)blockIdx.z * rows_per_split;
-    const int64_t r_end = min(n, r_begin + rows_per_split);
-    float acc[4][4];
-#pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
-    for (int64_t r0 = r_begin; r0 < r_end; r0 += kBwStep) {
-        // stage: 32 rows x 64 columns of each operand, 8 elements per thread
-        for (int t = threadIdx.x; t < kBwStep * kBwTile; t += kBwThreads) {
-            const int r = t >> 6, c = t & 63;
-            const int64_t row = r0 + r;
-            float h = 0.f, g = 0.f;
-            if (row < r_end) {
-                const int k = k0 + c;
-                if (k < d_in) {
-                    const uint32_t w = __ldg(bits + row * stride + (k >> 5));
-                    const float be = __ldg(beta + row);
-                    h = ((w >> (k & 31)) & 1u) ? be : -be;
-                }
-                const int j = j0 + c;
-                if (j < d_out) g = __ldg(gz + row * ldz + j);
-            }
-            Hs[r][c] = h;
-            Gs[r][c] = g;
-        }
-        __syncthreads();
-#pragma unroll 8
-        for (int r = 0; r < kBwStep; ++r) {
-            const float4 hv = *reinterpret_cast<const float4*>(&Hs[r][4 * ty]);
-            const float4 gv = *reinterpret_cast<const float4*>(&Gs[r][4 * tx]);
-            const float h[4] = {hv.x, hv.y, hv.z, hv.w};
-            const float g[4] = {gv.x, gv.y, gv.z, gv.w};
-#pragma unroll
-            for (int a = 0; a < 4; ++a)
-#pragma unroll
-                for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(h[a], g[b], acc[a][b]);
-        }
-        __syncthreads();
-    }
-    float* slab = part + (int64_t)blockIdx.z * d_in * d_out;
-#pragma unroll
-    for (int a = 0; a < 4; ++a) {
-        const int k = k0 + 4 * ty + a;
-        if (k >= d_in) continue;
-#pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            const int j = j0 + 4 * tx + b;
-            if (j < d_out) slab[(int64_t)k * d_out + j] = acc[a][b];
-        }
-    }
-}
-
 // G_W~ = sum of the slabs, in slab order (double accumulation: the slabs can differ by orders of magnitude).
 __global__ void grad_wt_reduce_kernel(const float* __restrict__ part, int n_splits, int64_t elems, float* __restrict__ g_wt)
 {
@@ -108,60 +41,7 @@ __global__ void grad_wt_reduce_kernel(const float* __restrict__ part, int n_spli
     g_wt[t] = (float)s;
 }
 
-// G_H = clip(G_zeta W~^T).  Block (x, y): rows [64 x, +64) x inputs k in [64 y, +64); per step 32
-// output channels j: tile of G_zeta scaled by alpha_j, and the signs of W[k][j] as +-1.
-__global__ void __launch_bounds__(kBwThreads)
-grad_h_kernel(const float* __restrict__ gz, int64_t ldz, const float* __restrict__ alpha,
-              const float* __restrict__ W, int64_t ldw, int64_t n, int d_in, int d_out,
-              float* __restrict__ g_h, int64_t ldh)
-{
-    __shared__ __align__(16) float Gs[kBwStep][kBwTile + 4];          // [j][row]
-    __shared__ __align__(16) float Bs[kBwStep][kBwTile + 4];          // [j][k]
-    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-    const int64_t i0 = (int64_t)blockIdx.x * kBwTile;
-    const int k0 = blockIdx.y * kBwTile;
-    float acc[4][4];
-#pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
-    for (int j0 = 0; j0 < d_out; j0 += kBwStep) {
-        for (int t = threadIdx.x; t < kBwStep * kBwTile; t += kBwThreads) {
-            // G tile: consecutive threads read consecutive j of one row (coalesced), stored transposed
-            const int jr = t & 31, rr = t >> 5;
-            const int64_t row = i0 + rr;
-            const int j = j0 + jr;
-            Gs[jr][rr] = (row < n && j < d_out) ? __fmul_rn(__ldg(gz + row * ldz + j), __ldg(alpha + j)) : 0.f;
-            const int k = k0 + rr;
-            Bs[jr][rr] = (k < d_in && j < d_out) ? (__ldg(W + (int64_t)k * ldw + j) >= 0.f ? 1.f : -1.f) : 0.f;
-        }
-        __syncthreads();
-#pragma unroll 8
-        for (int j = 0; j < kBwStep; ++j) {
-            const float4 gv = *reinterpret_cast<const float4*>(&Gs[j][4 * ty]);
-            const float4 bv = *reinterpret_cast<const float4*>(&Bs[j][4 * tx]);
-            const float g[4] = {gv.x, gv.y, gv.z, gv.w};
-            const float b[4] = {bv.x, bv.y, bv.z, bv.w};
-#pragma unroll
-            for (int a = 0; a < 4; ++a)
-#pragma unroll
-                for (int c = 0; c < 4; ++c) acc[a][c] = fmaf(g[a], b[c], acc[a][c]);
-        }
-        __syncthreads();
-    }
-#pragma unroll
-    for (int a = 0; a < 4; ++a) {
-        const int64_t row = i0 + 4 * ty + a;
-        if (row >= n) continue;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const int k = k0 + 4 * tx + c;
-            if (k < d_in) g_h[row * ldh + k] = fabsf(acc[a][c]) < 1.f ? acc[a][c] : 0.f;     // Eq. bp-H
-        }
-    }
-}
-
-// ---- tensor-core versions of the two dense products -------------------------------------------------
+// ---- the two dense products, on the tensor cores ------------------------------------------------------
 // Both products have one operand that is exactly +-1 (exact in bf16) and one fp32 operand.  The fp32
 // operand x is split into three bf16 terms x = hi + mid + lo (each the rounding of what is left:
 // 3 x 8 significant bits cover fp32's 24), so three bf16 tensor-core products with fp32 accumulation
@@ -303,6 +183,109 @@ grad_h_mma_kernel(const float* __restrict__ gz, int64_t ldz, const float* __rest
         }
 }
 
+// G_W~ partial sums on the tensor cores.  The product is taken transposed, C^T[j][k] = sum over nodes
+// of (beta_i G_zeta[i][j]) * F[i][k], so that the fp32 operand is again the row operand: A[j][node]
+// (split in three), B[node][k] = +-1 from the packed bits.  Both operands are stored node-major in
+// global memory and the reduction runs over the nodes, so the staging transposes them: a thread takes
+// two consecutive nodes and writes them as one 32-bit pair.  Block (x, y, z): channels j in
+// [128 x, +128), inputs k in [128 y, +128), nodes [z * rows_per_split, +rows_per_split); slab z of
+// `part` receives the tile as [k][j].
+__global__ void __launch_bounds__(kBwThreads)
+grad_wt_mma_kernel(const uint32_t* __restrict__ bits, int64_t stride, const float* __restrict__ beta,
+                   const float* __restrict__ gz, int64_t ldz, int64_t n, int d_in, int d_out,
+                   int64_t rows_per_split, float* __restrict__ part)
+{
+    __shared__ __align__(16) unsigned short As[3 * kMmaTile * kMmaPitch];   // [term][j][node]
+    __shared__ __align__(16) unsigned short Bs[kMmaTile * kMmaPitch];       // [k][node]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int wr = warp >> 1, wc = warp & 1;
+    const int j0 = blockIdx.x * kMmaTile, k0 = blockIdx.y * kMmaTile;
+    const int64_t r_begin = (int64_t)blockIdx.z * rows_per_split;
+    const int64_t r_end = min(n, r_begin + rows_per_split);
+    const bool vec_ok = (ldz % 4 == 0) && (reinterpret_cast<uintptr_t>(gz) % 16 == 0);
+    float acc[2][8][4];
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+        for (int b = 0; b < 8; ++b)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[a][b][c] = 0.f;
+    for (int64_t r0 = r_begin; r0 < r_end; r0 += kMmaK) {
+        __syncthreads();                                   // the previous step's tiles are consumed
+        // A: 16 node pairs x 32 quads of channels
+        for (int t = threadIdx.x; t < 16 * 32; t += kBwThreads) {
+            const int np = t & 15, jq = (t >> 4) * 4;
+            float x[2][4];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int64_t row = r0 + 2 * np + h;
+                const int j = j0 + jq;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) x[h][q] = 0.f;
+                if (row < r_end) {
+                    const float be = __ldg(beta + row);
+                    if (j + 3 < d_out && vec_ok) {
+                        const float4 v = __ldg(reinterpret_cast<const float4*>(gz + row * ldz + j));
+                        x[h][0] = v.x * be, x[h][1] = v.y * be, x[h][2] = v.z * be, x[h][3] = v.w * be;
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            if (j + q < d_out) x[h][q] = __ldg(gz + row * ldz + j + q) * be;
+                    }
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                unsigned short h0, m0, l0, h1, m1, l1;
+                split3(x[0][q], h0, m0, l0);
+                split3(x[1][q], h1, m1, l1);
+                const int at = (jq + q) * kMmaPitch + 2 * np;
+                *reinterpret_cast<uint32_t*>(&As[0 * kMmaTile * kMmaPitch + at]) = (uint32_t)h0 | ((uint32_t)h1 << 16);
+                *reinterpret_cast<uint32_t*>(&As[1 * kMmaTile * kMmaPitch + at]) = (uint32_t)m0 | ((uint32_t)m1 << 16);
+                *reinterpret_cast<uint32_t*>(&As[2 * kMmaTile * kMmaPitch + at]) = (uint32_t)l0 | ((uint32_t)l1 << 16);
+            }
+        }
+        // B: 16 node pairs x 4 words of 32 inputs, each word in two halves of 16
+        for (int t = threadIdx.x; t < 16 * 8; t += kBwThreads) {
+            const int np = t & 15, wd = (t >> 4) >> 1, half = (t >> 4) & 1;
+            const int kw = k0 + wd * 32;                   // first input of the word
+            uint32_t w0 = 0u, w1 = 0u;
+            const int64_t row = r0 + 2 * np;
+            if (kw < d_in) {
+                if (row < r_end) w0 = __ldg(bits + row * stride + (kw >> 5));
+                if (row + 1 < r_end) w1 = __ldg(bits + (row + 1) * stride + (kw >> 5));
+            }
+            const bool in0 = row < r_end, in1 = row + 1 < r_end;
+#pragma unroll
+            for (int b = 0; b < 16; ++b) {
+                const int kb = half * 16 + b;
+                const bool kin = kw + kb < d_in;
+                const uint32_t lo = (kin && in0) ? (((w0 >> kb) & 1u) ? 0x3F80u : 0xBF80u) : 0u;
+                const uint32_t hi = (kin && in1) ? (((w1 >> kb) & 1u) ? 0x3F80u : 0xBF80u) : 0u;
+                *reinterpret_cast<uint32_t*>(&Bs[(wd * 32 + kb) * kMmaPitch + 2 * np]) = lo | (hi << 16);
+            }
+        }
+        __syncthreads();
+        mma_step(As, Bs, wr, wc, lane, acc);
+    }
+    float* slab = part + (int64_t)blockIdx.z * d_in * d_out;
+    const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int mb = 0; mb < 2; ++mb)
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const int j = j0 + wr * 32 + mb * 16 + g + 8 * half;
+            if (j >= d_out) continue;
+#pragma unroll
+            for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    const int k = k0 + wc * 64 + nb * 8 + 2 * t + q;
+                    if (k < d_in) slab[(int64_t)k * d_out + j] = acc[mb][nb][2 * half + q];
+                }
+        }
+}
+
 // Eq. bp-W.  One block per 32 output channels: thread (tx, ty) sums G_W~_kj B_kj over k = ty, ty + 32, ...
 // for channel j0 + tx in double; the 32 partial sums of a channel are added in a fixed order; then
 // every element gets (1/d_in) B_ij col_j + alpha_j G_W~_ij [|W_ij| < 1].
@@ -345,9 +328,9 @@ int64_t pad4(int64_t d) { return (d + 3) / 4 * 4; }
 
 int wt_splits(int64_t n, int d_in, int d_out)
 {
-    const int64_t tiles = ceil_div(d_in, kBwTile) * ceil_div(d_out, kBwTile);
+    const int64_t tiles = ceil_div(d_in, kMmaTile) * ceil_div(d_out, kMmaTile);
     const int64_t want = std::max<int64_t>(1, (148 * 4) / tiles);               // about four blocks per SM in all
-    return (int)std::max<int64_t>(1, std::min<int64_t>(want, ceil_div(n, 4 * kBwStep)));
+    return (int)std::max<int64_t>(1, std::min<int64_t>(want, ceil_div(n, 4 * kMmaK)));
 }
 
 }  // namespace
@@ -423,9 +406,9 @@ cudaError_t launch_layer_backward(cudaStream_t s, int64_t n, const int64_t* rowp
 
     // step 1b: G_W~ = H~^T G_zeta, split over the rows, slabs added in a fixed order
     {
-        const int64_t rows_per_split = ceil_div(ceil_div(n, n_splits), kBwStep) * kBwStep;
-        const dim3 grid((unsigned)ceil_div(d_in, kBwTile), (unsigned)ceil_div(d_out, kBwTile), (unsigned)n_splits);
-        grad_wt_partial_kernel<<<grid, kBwThreads, 0, s>>>(in_bits, stride_in, in_beta, gz, ldz, n, d_in, d_out, rows_per_split, part);
+        const int64_t rows_per_split = ceil_div(ceil_div(n, n_splits), kMmaK) * kMmaK;
+        const dim3 grid((unsigned)ceil_div(d_out, kMmaTile), (unsigned)ceil_div(d_in, kMmaTile), (unsigned)n_splits);
+        grad_wt_mma_kernel<<<grid, kBwThreads, 0, s>>>(in_bits, stride_in, in_beta, gz, ldz, n, d_in, d_out, rows_per_split, part);
         ++*launches;
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         const int64_t elems = (int64_t)d_in * d_out;
