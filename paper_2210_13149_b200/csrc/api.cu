@@ -124,6 +124,7 @@ bigcn_status run_layer(bigcn_ctx* ctx, const bigcn_graph* g, const bigcn_layer* 
     if (ev_mid) BIGCN_CUDA(ctx, cudaEventRecord(ev_mid, ctx->stream));
     SpmmArgs a;
     a.n = g->n;
+    a.nnz = g->nnz;
     a.rowptr = g->rowptr;
     a.colidx = g->colidx;
     a.val = g->val;
@@ -820,6 +821,7 @@ bigcn_status bigcn_sage_layer_forward(bigcn_ctx* ctx, const bigcn_graph* mean_gr
     if (e != cudaSuccess) { finish_call(ctx); return cuda_fail(ctx, e, "bit-GEMM (neighbour term) launch"); }
     SpmmArgs a;
     a.n = n;
+    a.nnz = mean_graph->nnz;
     a.rowptr = mean_graph->rowptr;
     a.colidx = mean_graph->colidx;
     a.val = mean_graph->val;

@@ -39,6 +39,7 @@ cudaError_t launch_bitgemm(cudaStream_t s, const uint32_t* A, int64_t stride_a,
 
 struct SpmmArgs {
     int64_t n;
+    int64_t nnz = 0;         // stored entries (0 = unknown): the mean row length picks the stream for narrow rows
     const int64_t* rowptr;
     const int32_t* colidx;
     const float* val;

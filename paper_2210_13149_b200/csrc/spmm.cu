@@ -231,18 +231,14 @@ __device__ __forceinline__ void finish_row(const SpmmDev& p, const float* ctab, 
     }
 }
 
-template <int NCH, int LPR, bool kPair = false>
+template <int NCH, int LPR, bool kAligned = false>
 struct Pipe {
     static constexpr int G = kWarp / LPR;                       // entries per position
     static constexpr int PB = (4 * G <= 32) ? 4 : 32 / G;       // positions per group (PB * G divides 32)
-    static constexpr int NG = NCH > 1 ? 2 : ((LPR == 32 || kPair) ? 4 : 3);  // groups in flight per warp (a power of two for the row-aligned streams)
+    static constexpr int NG = NCH > 1 ? 2 : ((LPR == 32 || kAligned) ? 4 : 3);  // groups in flight per warp (a power of two for the row-aligned streams)
     static constexpr int RING = PB * NG;                        // slots of NCH * 512 bytes
     static constexpr size_t kWarpBytes = (size_t)RING * (NCH * 512 + G * 4);
 };
-
-// 256-byte rows of 8-bit elements take the row-aligned stream with two entries per position.
-template <typename T, int NCH, int LPR>
-struct UsesPairStream { static constexpr bool value = (sizeof(T) == 1 && NCH == 1 && LPR == 16); };
 
 // Streams the stored entries [e0, e0 + n_ent) through the warp's ring.
 //   kPartial = false: the entries are those of rows [row_lo, row_hi); `rp_rel` holds, in lane j, the
@@ -590,23 +586,34 @@ __device__ __forceinline__ void fma_bytes16(float w, const uint4& v, float (&acc
     }
 }
 
-// The row-aligned stream for 256-byte rows of 8-bit elements (up to 256 columns): a position holds
-// TWO stored entries, one per half warp (lane = 16 g + l fetches and accumulates the 16 bytes l of
-// entry 2 b + g of position b), so the per-position bookkeeping is shared by two entries and a lane's
-// 16-byte vector still carries 16 columns.  A group is 4 positions = 8 entries and never straddles a
-// row (a row takes ceil(deg / 8) groups, at least one).  The two half-warp sums are added when a row
-// completes.  Cursors, metadata chunks and the weight ring are those of stream_rows_wide; the
-// weights of a group are stored half by half (index 4 g + b) so that a lane reads its four with one
-// 16-byte load.  kFull: the row has exactly 16 vectors, no lane needs masking.
-template <bool kFull, bool kPartial>
-__device__ __forceinline__ void stream_rows_pair(const SpmmDev& p, uint4* ring, float* wfifo, const float* ctab, int lane,
-                                                 int64_t e0, int n_ent, int64_t warp_row0, int row_lo,
-                                                 int row_hi, int rp_rel, float (&acc)[1][16])
+// acc += w * (one 16-byte vector of T), whatever T.
+template <typename T>
+__device__ __forceinline__ void fma_any(float w, const uint4& v, float (&acc)[Elt<T>::kPerVec])
 {
-    using P = Pipe<1, 16, true>;
-    constexpr int PB = P::PB, NG = P::NG, EG = 2 * PB;        // positions and entries per group
+    if constexpr (sizeof(T) == 1) fma_bytes16(w, v, acc);
+    else fma_vec<T>(w, v, acc);
+}
+
+// The row-aligned stream for rows of 8 or 16 vectors (128- and 256-byte rows): a position holds G = 4
+// or 2 stored entries, one per group of LPR = 32 / G lanes (lane = LPR g + l fetches and accumulates
+// vector l of entry G b + g of position b), so the per-position bookkeeping is shared by G entries.
+// A group is 4 positions = 4 G entries and never straddles a row (a row takes ceil(deg / 4G) groups,
+// at least one), which pays when rows are long compared with a group; the launcher picks the general
+// stream otherwise.  The lane groups' sums are added when a row completes.  Cursors, metadata chunks
+// and the weight ring are those of stream_rows_wide; the weights of a group are stored lane group by
+// lane group (index 4 g + b) so that a lane reads its four with one 16-byte load.  kFull: the row has
+// exactly LPR vectors, no lane needs masking.
+template <typename T, int G, bool kFull, bool kPartial>
+__device__ __forceinline__ void stream_rows_multi(const SpmmDev& p, uint4* ring, float* wfifo, const float* ctab, int lane,
+                                                  int64_t e0, int n_ent, int64_t warp_row0, int row_lo,
+                                                  int row_hi, int rp_rel, float (&acc)[1][Elt<T>::kPerVec])
+{
+    constexpr int LPR = kWarp / G;
+    constexpr int EPV = Elt<T>::kPerVec;
+    using P = Pipe<1, LPR, true>;
+    constexpr int PB = P::PB, NG = P::NG, EG = G * PB;        // positions and entries per group
     static_assert(PB == 4 && (NG & (NG - 1)) == 0, "float4 weight reads; power-of-two group ring");
-    const int g = lane >> 4, l = lane & 15;
+    const int g = lane / LPR, l = lane % LPR;
     const bool active = l < p.nv;
     const int32_t* cols = p.colidx + e0;
     const float* vals = p.val + e0;
@@ -630,7 +637,7 @@ __device__ __forceinline__ void stream_rows_pair(const SpmmDev& p, uint4* ring, 
     int re = 0, rr = row_lo, rend = iend;                     // retire cursor
     bool more = row_lo < row_hi;
     int issued = 0, goff = 0;                                 // groups issued; ring position of the current group
-    zero_acc<1, 16>(acc);
+    zero_acc<1, EPV>(acc);
 
     for (int it = 0;; ++it) {
         if (it >= NG) {
@@ -648,19 +655,19 @@ __device__ __forceinline__ void stream_rows_pair(const SpmmDev& p, uint4* ring, 
             if (left >= EG) {
 #pragma unroll
                 for (int b = 0; b < PB; ++b)
-                    if (kFull || active) fma_bytes16(w[b], v[b], acc[0]);
+                    if (kFull || active) fma_any<T>(w[b], v[b], acc[0]);
                 re += EG;
             } else {
 #pragma unroll
                 for (int b = 0; b < PB; ++b)
-                    if (2 * b + g < left && (kFull || active)) fma_bytes16(w[b], v[b], acc[0]);
+                    if (G * b + g < left && (kFull || active)) fma_any<T>(w[b], v[b], acc[0]);
                 re = rend;
             }
             if (re == rend) {                                 // the row is complete
-                reduce_groups<1, 16, 16>(acc);
+                reduce_groups<1, EPV, LPR>(acc);
                 if (kPartial) return;
-                finish_row<int8_t, 1, 16>(p, ctab, warp_row0 + rr, lane, acc);
-                zero_acc<1, 16>(acc);
+                finish_row<T, 1, LPR>(p, ctab, warp_row0 + rr, lane, acc);
+                zero_acc<1, EPV>(acc);
                 ++rr;
                 if (rr < row_hi) rend = row_end_of(rr);
             }
@@ -681,17 +688,17 @@ __device__ __forceinline__ void stream_rows_pair(const SpmmDev& p, uint4* ring, 
             if (cnt == EG) {
 #pragma unroll
                 for (int b = 0; b < PB; ++b) {
-                    const uint32_t k = (uint32_t)__shfl_sync(0xffffffffu, m_col, src_lane + 2 * b);
+                    const uint32_t k = (uint32_t)__shfl_sync(0xffffffffu, m_col, src_lane + G * b);
                     if (kFull || active) cp_async16_s(dsta + b * 512, zeta_l + (uint64_t)k * row_bytes);
                 }
             } else {
 #pragma unroll
                 for (int b = 0; b < PB; ++b) {
-                    const uint32_t k = (uint32_t)__shfl_sync(0xffffffffu, m_col, src_lane + 2 * b);
-                    if (2 * b + g < cnt && (kFull || active)) cp_async16_s(dsta + b * 512, zeta_l + (uint64_t)k * row_bytes);
+                    const uint32_t k = (uint32_t)__shfl_sync(0xffffffffu, m_col, src_lane + G * b);
+                    if (G * b + g < cnt && (kFull || active)) cp_async16_s(dsta + b * 512, zeta_l + (uint64_t)k * row_bytes);
                 }
             }
-            if (rel < cnt) wfifo[goff * EG + 4 * (rel & 1) + (rel >> 1)] = m_w;
+            if (rel < cnt) wfifo[goff * EG + 4 * (rel % G) + rel / G] = m_w;
             ie += cnt;
             ++issued;
             if (ie == iend) {
@@ -719,18 +726,19 @@ __device__ __forceinline__ void stream_rows_pair(const SpmmDev& p, uint4* ring, 
 }
 
 // Thread blocks per SM the kernel is compiled for (register budget) and launched with (grid size).
-template <typename T, int NCH, int LPR>
+template <int NCH, int LPR, bool kAligned>
 constexpr int spmm_blocks_per_sm()
 {
-    return NCH == 1 ? ((LPR == 32 || UsesPairStream<T, NCH, LPR>::value) ? 3 : 4) : (NCH == 2 ? 2 : 1);
+    return NCH == 1 ? ((LPR == 32 || kAligned) ? 3 : 4) : (NCH == 2 ? 2 : 1);
 }
 
-template <typename T, int NCH, int LPR, bool kFull>
-__global__ void __launch_bounds__(kSpmmThreads, spmm_blocks_per_sm<T, NCH, LPR>())
+// kAligned (rows of 8 or 16 vectors only): the row-aligned multi-entry stream instead of the general one.
+template <typename T, int NCH, int LPR, bool kFull, bool kAligned>
+__global__ void __launch_bounds__(kSpmmThreads, spmm_blocks_per_sm<NCH, LPR, kAligned>())
 spmm_kernel(const SpmmDev p, int rows_per_warp)
 {
-    constexpr bool kPair = UsesPairStream<T, NCH, LPR>::value;
-    using P = Pipe<NCH, LPR, kPair>;
+    static_assert(!kAligned || (NCH == 1 && (LPR == 8 || LPR == 16)), "the multi-entry stream covers rows of 8 or 16 vectors");
+    using P = Pipe<NCH, LPR, kAligned>;
     constexpr int EPV = Elt<T>::kPerVec;
     constexpr int G = P::G;
     constexpr int kCols = (LPR < 32 ? LPR : NCH * 32) * EPV;  // accumulator columns of one warp
@@ -776,9 +784,9 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
                 if constexpr (LPR == 32)
                     stream_rows_wide<T, NCH, kFull, false>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
                                                     (int)(rp_reg - e0), acc);
-                else if constexpr (kPair)
-                    stream_rows_pair<kFull, false>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
-                                                   (int)(rp_reg - e0), acc);
+                else if constexpr (kAligned)
+                    stream_rows_multi<T, kWarp / LPR, kFull, false>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
+                                                                    (int)(rp_reg - e0), acc);
                 else
                     stream_entries<T, NCH, LPR, false>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
                                                        (int)(rp_reg - e0), acc);
@@ -796,8 +804,8 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
         const int64_t s0 = min(le, ls + warp * slice), s1 = min(le, s0 + slice);
         if constexpr (LPR == 32)
             stream_rows_wide<T, NCH, kFull, true>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
-        else if constexpr (kPair)
-            stream_rows_pair<kFull, true>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
+        else if constexpr (kAligned)
+            stream_rows_multi<T, kWarp / LPR, kFull, true>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
         else
             stream_entries<T, NCH, LPR, true>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
         __syncthreads();                                      // every ring is idle: reuse them for the partial sums
@@ -824,38 +832,46 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
     }
 }
 
-template <typename T, int NCH, int LPR, bool kFull = false>
+template <typename T, int NCH, int LPR, bool kFull = false, bool kAligned = false>
 cudaError_t launch_one(cudaStream_t s, const SpmmDev& p)
 {
     constexpr int kCols = (LPR < 32 ? LPR : NCH * 32) * Elt<T>::kPerVec;
-    constexpr size_t smem = kSpmmWarps * Pipe<NCH, LPR, UsesPairStream<T, NCH, LPR>::value>::kWarpBytes + 3 * kCols * sizeof(float);   // rings, weights, column table
+    constexpr size_t smem = kSpmmWarps * Pipe<NCH, LPR, kAligned>::kWarpBytes + 3 * kCols * sizeof(float);   // rings, weights, column table
     // enough thread blocks to fill the machine on small graphs, long runs of rows on large ones
     const int rows_per_warp = (int)std::min<int64_t>(kMaxRowsPerWarp, std::max<int64_t>(1, p.n / (kSpmmWarps * 148 * 8)));
     if (smem > 40 * 1024) {                                   // above the default limit: opt in
-        cudaError_t e = cudaFuncSetAttribute(spmm_kernel<T, NCH, LPR, kFull>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(spmm_kernel<T, NCH, LPR, kFull, kAligned>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
     cudaError_t e = cudaMemsetAsync(p.run_counter, 0, sizeof(int), s);
     if (e != cudaSuccess) return e;
     // one wave of resident blocks; the warps pull runs of rows until none are left
     const int64_t wanted = ceil_div(ceil_div(p.n, rows_per_warp), kSpmmWarps);
-    const unsigned grid = (unsigned)std::min<int64_t>(wanted, 148 * spmm_blocks_per_sm<T, NCH, LPR>());
-    spmm_kernel<T, NCH, LPR, kFull><<<grid, kSpmmThreads, smem, s>>>(p, rows_per_warp);
+    const unsigned grid = (unsigned)std::min<int64_t>(wanted, 148 * spmm_blocks_per_sm<NCH, LPR, kAligned>());
+    spmm_kernel<T, NCH, LPR, kFull, kAligned><<<grid, kSpmmThreads, smem, s>>>(p, rows_per_warp);
     return cudaGetLastError();
 }
 
+// mean_row: stored entries per row (0 = unknown).  256-byte rows of signed bytes take the row-aligned
+// multi-entry stream (the general stream has no fast unpack for bytes) unless the rows are known to be
+// much shorter than its groups of 8 entries.  For 2- and 4-byte elements in rows of 8 or 16 vectors the
+// aligned stream was measured level with the general one at best (c5, 96-byte rows: 3.80 vs 3.72 ms; at
+// full size those gathers are bound by DRAM access rate, not by instructions), so they keep the general one.
 template <typename T>
-cudaError_t dispatch(cudaStream_t s, const SpmmDev& p)
+cudaError_t dispatch(cudaStream_t s, const SpmmDev& p, double mean_row)
 {
     const int nv = p.nv;
     if (nv <= 1) return launch_one<T, 1, 1>(s, p);
     if (nv <= 2) return launch_one<T, 1, 2>(s, p);
     if (nv <= 4) return launch_one<T, 1, 4>(s, p);
     if (nv <= 8) return launch_one<T, 1, 8>(s, p);
-    if constexpr (sizeof(T) == 1) {
-        if (nv == 16) return launch_one<T, 1, 16, true>(s, p);   // 256-byte rows: no lane masking
+    if (nv <= 16) {
+        if constexpr (sizeof(T) == 1) {
+            if (!(mean_row > 0.0 && mean_row < 8.0))
+                return nv == 16 ? launch_one<T, 1, 16, true, true>(s, p) : launch_one<T, 1, 16, false, true>(s, p);
+        }
+        return launch_one<T, 1, 16>(s, p);
     }
-    if (nv <= 16) return launch_one<T, 1, 16>(s, p);
     if (nv == 32) return launch_one<T, 1, 32, true>(s, p);
     if (nv <= 32) return launch_one<T, 1, 32>(s, p);
     // wider rows: up to 512 columns in any format (128 / 64 / 32 vectors of 4- / 2- / 1-byte elements)
@@ -901,11 +917,12 @@ cudaError_t launch_spmm(cudaStream_t s, const SpmmArgs& a, int* launches)
     if (!a.scratch || a.scratch_bytes < sizeof(int)) return cudaErrorInvalidValue;
     p.run_counter = static_cast<int*>(a.scratch);
     ++*launches;
+    const double mean_row = (a.nnz > 0 && a.n > 0) ? (double)a.nnz / (double)a.n : 0.0;
     switch (a.fmt) {
-        case kZetaF32: return dispatch<float>(s, p);
-        case kZetaF16: return dispatch<__half>(s, p);
-        case kZetaI16: return dispatch<int16_t>(s, p);
-        case kZetaI8: return dispatch<int8_t>(s, p);
+        case kZetaF32: return dispatch<float>(s, p, mean_row);
+        case kZetaF16: return dispatch<__half>(s, p, mean_row);
+        case kZetaI16: return dispatch<int16_t>(s, p, mean_row);
+        case kZetaI8: return dispatch<int8_t>(s, p, mean_row);
         default: return cudaErrorInvalidValue;
     }
 }
