@@ -66,3 +66,57 @@ def test_full_size_layers_oracle_fed_and_end_to_end(name):
     assert abs(share_out - rep["logits_outside_tolerance"]) < 1e-12
     ctx.sync_check()
     ctx.close()
+
+
+def test_entropy_bins_full_size():
+    """The side benchmark's configuration (the largest row of the paper's entropy table: 2,449,029 samples x 128
+    neurons, 1000 intervals): every count against the oracle's."""
+    import oracle
+    n, d, M = 2449029, 128, 1000
+    g = torch.Generator(device="cuda").manual_seed(2210)
+    H = torch.randn((n, d), device="cuda", generator=g) * (torch.rand(d, device="cuda", generator=g) * 3.8 + 0.2)
+    H[:, ::4].clamp_(min=0)
+    from paper_2210_13149_b200 import binding
+    ctx = binding.BiGCN(0)
+    got = ctx.entropy_bins(H, M)
+    want = oracle.entropy_bins(H.cpu().numpy(), M)
+    assert np.array_equal(got["col_min"].cpu().numpy(), want.col_min)
+    assert np.array_equal(got["col_max"].cpu().numpy(), want.col_max)
+    assert np.array_equal(got["counts"].cpu().numpy().astype(np.int64), want.counts)
+    np.testing.assert_allclose(got["entropy"].cpu().numpy(), want.entropy, rtol=1e-12)
+    assert got["total"].item() == pytest.approx(want.total, rel=1e-12)
+    ctx.close()
+
+
+def test_backward_large_graph_sampled_rows():
+    """Algorithm 1 on the c5 recipe at a twentieth of its size (122 k nodes, 6 M entries), 256 -> 64: the weight
+    gradient (a sum over every node) in full, the input gradient on every row."""
+    import oracle
+    from paper_2210_13149_b200 import binding, synth
+    wl = synth.make_workload("c5", scale=0.05, device="cuda")
+    n, d_in, d_out = wl.n, 256, 64
+    ctx = binding.BiGCN(0)
+    G = ctx.normalize_adjacency(wl.rowptr, wl.colidx)
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    W = torch.randn((d_in, d_out), device="cuda", generator=gen) * 0.7
+    Hin = torch.randn((n, d_in), device="cuda", generator=gen)
+    g_out = torch.randn((n, d_out), device="cuda", generator=gen) * 0.02
+    bitsT, alpha = ctx.pack_weights(W)
+    layer = binding.make_layer(d_in, d_out, bitsT, alpha)
+    bits, beta = ctx.pack_features(Hin)
+    g_in, g_w = ctx.layer_backward(G, layer, W, bits, beta, g_out)
+    src, dst = synth.edge_list(wl.rowptr, wl.colidx)
+    g = oracle.normalize_adjacency(n, src, dst)
+    F = oracle.unpack_rows(bits.cpu().numpy().view(np.uint32), d_in)
+    ref = oracle.layer_backward(g, W.cpu().numpy(), F, beta.cpu().numpy(), g_out.cpu().numpy())
+
+    def close(got, want, what):
+        got = got.astype(np.float64); want = want.astype(np.float64)
+        allow = 1e-4 * np.abs(want) + 2e-6 * np.abs(want).max()
+        bad = np.abs(got - want) > allow
+        assert not bad.any(), "%s: %d of %d outside tolerance" % (what, bad.sum(), bad.size)
+
+    close(g_w.cpu().numpy(), ref.G_W, "G_W")
+    near = np.abs(np.abs(ref.G_Ht.astype(np.float64)) - 1.0) <= 2e-4
+    close(np.where(~near, g_in.cpu().numpy(), 0), np.where(~near, ref.G_H, 0), "G_H")
+    ctx.close()
