@@ -67,7 +67,11 @@ enum {
      *     d_in <= 2048 only; others fall back to 2). */
     BIGCN_OPT_ZETA_FORMAT = 1,
     /* Rows of the sparse matrix with more entries than this are split across thread blocks. 0 = default. */
-    BIGCN_OPT_LONG_ROW = 2
+    BIGCN_OPT_LONG_ROW = 2,
+    /* How the binary contraction runs.  0 = default: as int8 tensor-core products (tcgen05, the packed bits
+     * expanded to +1 / -1 bytes in shared memory; the same integers) for layers with d_in <= 256 and
+     * d_out <= 256, on the XOR / bit-count pipe otherwise; 1 = always on the XOR / bit-count pipe. */
+    BIGCN_OPT_CONTRACTION = 3
 };
 
 /* Context: binds a device and a stream.  `cuda_stream` is a cudaStream_t (0 = default stream). */

@@ -35,7 +35,7 @@ cudaError_t launch_pack_weights(cudaStream_t s, const float* W, int d_in, int d_
 cudaError_t launch_bitgemm(cudaStream_t s, const uint32_t* A, int64_t stride_a,
                            const uint32_t* BT, int64_t stride_b, int64_t n, int d_in, int d_out,
                            const float* beta, const float* alpha, int fmt, void* zeta, int64_t ldz,
-                           int32_t* dbg_dot, float* dbg_zeta, int* launches);
+                           int32_t* dbg_dot, float* dbg_zeta, int* launches, bool tensor_cores = true);
 
 struct SpmmArgs {
     int64_t n;
@@ -77,6 +77,13 @@ size_t col_stats_scratch_bytes(int d);
 
 cudaError_t measure_popc_peak(cudaStream_t s, void* scratch, double* word_steps_per_s, int* launches);
 size_t popc_peak_scratch_bytes();
+
+// The same contraction as tcgen05 int8 products (bitgemm_tc.cu): shapes with d_in, d_out <= 256.
+bool bitgemm_tc_covers(int d_in, int d_out, int64_t stride_a, int64_t stride_b);
+cudaError_t launch_bitgemm_tc(cudaStream_t s, const uint32_t* A, int64_t stride_a, const uint32_t* BT, int64_t stride_b,
+                              int64_t n, int d_in, int d_out, const float* beta, const float* alpha, int fmt, void* zeta,
+                              int64_t ldz, int32_t* dbg_dot, float* dbg_zeta);
+int bitgemm_tc_timeouts();
 
 // Binning entropy estimate (entropy.cu): scratch = 2 * d uint32.
 cudaError_t launch_entropy_bins(cudaStream_t s, const float* H, int64_t n, int d, int64_t ld, int n_bins,
