@@ -97,8 +97,9 @@ __device__ __forceinline__ bool wait_barrier(uint64_t* bar, uint32_t parity)
 }
 
 // N: accumulator columns = N of the instruction (a multiple of 16, at most 256).
-template <int N, int FMT>
-__global__ void __launch_bounds__(kTcThreads, 1)
+// kBuf: feature tiles and accumulators per CTA (2 = the CTA overlaps its own tiles, 1 = two CTAs per SM overlap each other).
+template <int N, int FMT, int kBuf>
+__global__ void __launch_bounds__(kTcThreads, kBuf == 1 ? 2 : 1)
 bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32_t* __restrict__ BT, int64_t stride_b,
                   int64_t n, int d_in, int d_out, const float* __restrict__ beta, const float* __restrict__ alpha,
                   void* __restrict__ zeta, int64_t ldz, int32_t* __restrict__ dbg_dot, float* __restrict__ dbg_zeta)
@@ -116,7 +117,7 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&tmem_base_s)), "r"(2 * kCols) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&tmem_base_s)), "r"(kBuf * kCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
     }
     if (threadIdx.x == 0) {
@@ -130,7 +131,7 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
     const int64_t n_tiles = ceil_div(n, kTcRows);
     const int64_t my_tiles = blockIdx.x < n_tiles ? ceil_div(n_tiles - blockIdx.x, (int64_t)gridDim.x) : 0;
     auto tile_row0 = [&](int64_t i) { return (blockIdx.x + i * gridDim.x) * (int64_t)kTcRows; };
-    if (my_tiles > 0) stage_operand(As0, kTcRows, A + tile_row0(0) * stride_a, stride_a, n - tile_row0(0));
+    if (kBuf == 2 && my_tiles > 0) stage_operand(As0, kTcRows, A + tile_row0(0) * stride_a, stride_a, n - tile_row0(0));
     asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
     __syncthreads();
@@ -151,22 +152,30 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
         }
         asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(smem_u32(&bar[buf])) : "memory");
     };
-    if (my_tiles > 0 && threadIdx.x == 0) issue_tile(0);
+    if (kBuf == 2 && my_tiles > 0 && threadIdx.x == 0) issue_tile(0);
 
     constexpr int kVec = FMT == kZetaF32 ? 4 : (FMT == kZetaI8 ? 16 : 8);     // elements per 16-byte store
     const int lane_base = 32 * (warp & 3);                  // a warp reads tensor-memory lanes 32 (warp % 4) .. + 31
     const int c_begin = (warp >> 2) * (N / 2), c_end = c_begin + N / 2;       // warps 0-3: lower half of the columns
     bool ok = true;
     for (int64_t i = 0; i < my_tiles; ++i) {
-        const int buf = (int)(i & 1);
-        if (i + 1 < my_tiles)                               // next tile's features: its buffer was released by the wait of tile i - 1
-            stage_operand(As0 + (buf ^ 1) * a_bytes, kTcRows, A + tile_row0(i + 1) * stride_a, stride_a, n - tile_row0(i + 1));
+        const int buf = kBuf == 2 ? (int)(i & 1) : 0;
+        if (kBuf == 2) {
+            if (i + 1 < my_tiles)                           // next tile's features: its buffer was released by the wait of tile i - 1
+                stage_operand(As0 + (buf ^ 1) * a_bytes, kTcRows, A + tile_row0(i + 1) * stride_a, stride_a, n - tile_row0(i + 1));
+        } else {
+            stage_operand(As0, kTcRows, A + tile_row0(i) * stride_a, stride_a, n - tile_row0(i));   // the wait of tile i - 1 released it
+        }
         asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
-        __syncthreads();                                    // staging done; everyone is past the reads of accumulator buf ^ 1
+        __syncthreads();                                    // staging done; everyone is past the reads of the accumulator to be overwritten
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-        if (i + 1 < my_tiles && threadIdx.x == 0) issue_tile(buf ^ 1);
-        if (!wait_barrier(&bar[buf], (uint32_t)((i >> 1) & 1))) {
+        if (kBuf == 2) {
+            if (i + 1 < my_tiles && threadIdx.x == 0) issue_tile(buf ^ 1);
+        } else if (threadIdx.x == 0) {
+            issue_tile(0);
+        }
+        if (!wait_barrier(&bar[buf], (uint32_t)((kBuf == 2 ? (i >> 1) : i) & 1))) {
             atomicExch(&g_tc_timeout, 1);
             ok = false;
         }
@@ -242,7 +251,7 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
     }
     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
     __syncthreads();
-    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(2 * kCols) : "memory");
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(kBuf * kCols) : "memory");
 }
 
 template <int N, int FMT>
@@ -250,11 +259,13 @@ cudaError_t launch_tc_inst(cudaStream_t s, const uint32_t* A, int64_t stride_a, 
                            int64_t n, int d_in, int d_out, const float* beta, const float* alpha, void* zeta, int64_t ldz,
                            int32_t* dbg_dot, float* dbg_zeta)
 {
-    const size_t smem = (size_t)(N + 2 * kTcRows) * stride_a * 32;
-    cudaError_t e = cudaFuncSetAttribute(bitgemm_tc_kernel<N, FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    // two CTAs per SM, each with one feature tile and one accumulator (N <= 256 columns each: 512 in all)
+    constexpr int kBuf = 1;
+    const size_t smem = (size_t)(N + kBuf * kTcRows) * stride_a * 32;
+    cudaError_t e = cudaFuncSetAttribute(bitgemm_tc_kernel<N, FMT, kBuf>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, kTcRows), 148);
-    bitgemm_tc_kernel<N, FMT><<<grid, kTcThreads, smem, s>>>(A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta);
+    const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, kTcRows), 148 * (kBuf == 1 ? 2 : 1));
+    bitgemm_tc_kernel<N, FMT, kBuf><<<grid, kTcThreads, smem, s>>>(A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta);
     return cudaGetLastError();
 }
 
