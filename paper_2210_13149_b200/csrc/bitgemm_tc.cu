@@ -8,13 +8,12 @@
 // Padding bits are 0 in both operands and expand to (-1)(-1) = +1 each: the constant K_pad - d_in is
 // subtracted in the epilogue.
 //
-// One CTA per SM walks over tiles of 128 rows.  The expanded weight panel (N x K bytes) stays in
-// shared memory; feature tiles (128 x K bytes) and accumulators (N columns of tensor memory) are
-// double-buffered, so the tensor cores work on tile i + 1 while the warps read tile i's accumulators
-// back (tcgen05.ld), convert them to the storage format of zeta and write them out.  Operands sit in
-// shared memory in the K-major no-swizzle canonical form: core matrices of 8 rows x 16 bytes.
-// Every wait on an mbarrier is bounded; if one runs out the kernel raises a flag, frees its tensor
-// memory and returns.
+// Persistent CTAs (two per SM) walk over tiles of 128 rows.  The expanded weight panel (N x K bytes)
+// stays in shared memory; each tile's features are expanded into one 128 x K operand, multiplied into
+// N columns of tensor memory, read back (tcgen05.ld), converted to the storage format of zeta and
+// written out while the other CTA of the SM is in another phase.  Operands sit in shared memory in the
+// K-major no-swizzle canonical form: core matrices of 8 rows x 16 bytes.  Every wait on an mbarrier is
+// bounded; if one runs out the kernel raises a flag, frees its tensor memory and returns.
 #include <algorithm>
 
 #include <cuda_fp16.h>
@@ -96,33 +95,94 @@ __device__ __forceinline__ bool wait_barrier(uint64_t* bar, uint32_t parity)
     return done != 0;
 }
 
-// N: accumulator columns = N of the instruction (a multiple of 16, at most 256).
-// kBuf: feature tiles and accumulators per CTA (2 = the CTA overlaps its own tiles, 1 = two CTAs per SM overlap each other).
-template <int N, int FMT, int kBuf>
-__global__ void __launch_bounds__(kTcThreads, kBuf == 1 ? 2 : 1)
+// Converts 16 consecutive dots of one row to the storage format: kPieces 16-byte pieces.
+template <int FMT>
+struct TcOut;
+template <> struct TcOut<kZetaF16> {
+    static constexpr int kElt = 2;
+    static __device__ __forceinline__ void pack(const int (&dot)[16], float, const float*, uint4 (&out)[2])
+    {
+        // exact integer -> fp16 without the conversion unit: the bit pattern 0x6600 + dot is the half 1536 + dot (|dot| <= 256 here)
+        uint32_t h[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const __half2 biased = __halves2half2(__ushort_as_half((unsigned short)(0x6600 + dot[2 * q])), __ushort_as_half((unsigned short)(0x6600 + dot[2 * q + 1])));
+            const __half2 r = __hsub2(biased, __half2half2(__ushort_as_half((unsigned short)0x6600)));
+            h[q] = *reinterpret_cast<const uint32_t*>(&r);
+        }
+        out[0] = make_uint4(h[0], h[1], h[2], h[3]);
+        out[1] = make_uint4(h[4], h[5], h[6], h[7]);
+    }
+};
+template <> struct TcOut<kZetaI16> {
+    static constexpr int kElt = 2;
+    static __device__ __forceinline__ void pack(const int (&dot)[16], float, const float*, uint4 (&out)[2])
+    {
+        uint32_t h[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) h[q] = ((uint32_t)dot[2 * q] & 0xffffu) | ((uint32_t)dot[2 * q + 1] << 16);
+        out[0] = make_uint4(h[0], h[1], h[2], h[3]);
+        out[1] = make_uint4(h[4], h[5], h[6], h[7]);
+    }
+};
+template <> struct TcOut<kZetaI8> {
+    static constexpr int kElt = 1;
+    static __device__ __forceinline__ void pack(const int (&dot)[16], float, const float*, uint4 (&out)[1])
+    {
+        uint32_t b[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            b[q] = ((uint32_t)dot[4 * q] & 0xffu) | (((uint32_t)dot[4 * q + 1] & 0xffu) << 8) | (((uint32_t)dot[4 * q + 2] & 0xffu) << 16) | ((uint32_t)dot[4 * q + 3] << 24);
+        out[0] = make_uint4(b[0], b[1], b[2], b[3]);
+    }
+};
+template <> struct TcOut<kZetaF32> {
+    static constexpr int kElt = 4;
+    // zeta_ij = (beta_i alpha_j) dot_ij in this order (Eq. "cdot-op"); al points at the chunk's first column
+    static __device__ __forceinline__ void pack(const int (&dot)[16], float be, const float* al, uint4 (&out)[4])
+    {
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+            float f[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) f[q] = __fmul_rn(__fmul_rn(be, al[4 * q4 + q]), (float)dot[4 * q4 + q]);
+            out[q4] = make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
+        }
+    }
+};
+
+// N: accumulator columns = N of the instruction (64, 128 or 256).  Two CTAs per SM, each with one
+// feature tile and one accumulator; a CTA's steps per tile are: expand the tile's bits (fetched into
+// registers during the previous tile) into shared memory, issue the products, fetch the next tile's
+// bits, wait for the accumulators, convert them and write them out.  The write goes through shared
+// memory (the feature tile's space, free once the products are done): a thread owns one row of the
+// accumulators, and rows are far apart in zeta, so each warp first collects 32 rows x 128 bytes and
+// then stores them as whole 128-byte row segments.
+template <int N, int FMT>
+__global__ void __launch_bounds__(kTcThreads, 2)
 bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32_t* __restrict__ BT, int64_t stride_b,
                   int64_t n, int d_in, int d_out, const float* __restrict__ beta, const float* __restrict__ alpha,
                   void* __restrict__ zeta, int64_t ldz, int32_t* __restrict__ dbg_dot, float* __restrict__ dbg_zeta)
 {
+    using Out = TcOut<FMT>;
+    constexpr int kElt = Out::kElt;                         // bytes per stored element = 16-byte pieces per chunk of 16 columns
     extern __shared__ __align__(128) unsigned char tc_smem[];
-    __shared__ __align__(8) uint64_t bar[2];
+    __shared__ __align__(8) uint64_t bar;
     __shared__ uint32_t tmem_base_s;
     __shared__ float al_s[N];
-    constexpr int kCols = N <= 32 ? 32 : (N <= 64 ? 64 : (N <= 128 ? 128 : 256));   // tensor-memory columns per accumulator
+    constexpr int kCols = N <= 32 ? 32 : (N <= 64 ? 64 : (N <= 128 ? 128 : 256));   // tensor-memory columns of the accumulator
     const int K = (int)stride_a * 32;                       // bytes per expanded row (padding included)
     const int pad = K - d_in;                               // padding positions: each contributes +1
     unsigned char* Bs = tc_smem;                            // [N][K]
-    unsigned char* As0 = tc_smem + (size_t)N * K;           // two tiles of [128][K]
-    const size_t a_bytes = (size_t)kTcRows * K;
+    unsigned char* As = tc_smem + (size_t)N * K;            // [128][K]; at least 32 KB: also the epilogue's scratch
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&tmem_base_s)), "r"(kBuf * kCols) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&tmem_base_s)), "r"(kCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
     }
     if (threadIdx.x == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(smem_u32(&bar[0])) : "memory");
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(smem_u32(&bar[1])) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(smem_u32(&bar)) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     for (int j = threadIdx.x; j < N; j += kTcThreads) al_s[j] = j < d_out ? __ldg(alpha + j) : 0.f;
@@ -131,8 +191,17 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
     const int64_t n_tiles = ceil_div(n, kTcRows);
     const int64_t my_tiles = blockIdx.x < n_tiles ? ceil_div(n_tiles - blockIdx.x, (int64_t)gridDim.x) : 0;
     auto tile_row0 = [&](int64_t i) { return (blockIdx.x + i * gridDim.x) * (int64_t)kTcRows; };
-    if (kBuf == 2 && my_tiles > 0) stage_operand(As0, kTcRows, A + tile_row0(0) * stride_a, stride_a, n - tile_row0(0));
-    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+    // a feature tile is 128 rows x (stride / 4) 16-byte pieces of packed bits: at most one piece per thread
+    const int q = (int)(stride_a >> 2);
+    const int my_r = threadIdx.x / q, my_piece = threadIdx.x - my_r * q;
+    const bool my_item = threadIdx.x < kTcRows * q;
+    auto fetch = [&](int64_t i) {
+        uint4 w = make_uint4(0u, 0u, 0u, 0u);
+        if (my_item && i < my_tiles && tile_row0(i) + my_r < n)
+            w = __ldg(reinterpret_cast<const uint4*>(A + (tile_row0(i) + my_r) * stride_a) + my_piece);
+        return w;
+    };
+    uint4 pre = fetch(0);
     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
@@ -141,117 +210,107 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
     // instruction descriptor: D = s32, A = B = s8, both K-major, N, M = 128
     const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kTcRows >> 4) << 24);
     const uint32_t a_lbo = (kTcRows >> 3) * 128, b_lbo = (N >> 3) * 128, sbo = 128;
-    auto issue_tile = [&](int buf) {                        // one thread: all K steps of a tile, then the commit
-        const uint32_t a_base = smem_u32(As0 + buf * a_bytes), b_base = smem_u32(Bs);
-        for (int ks = 0; ks < K / 32; ++ks) {
-            const uint64_t ad = make_desc(a_base + 2 * ks * a_lbo, a_lbo, sbo);
-            const uint64_t bd = make_desc(b_base + 2 * ks * b_lbo, b_lbo, sbo);
-            const uint32_t accum = ks > 0 ? 1u : 0u;
-            asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}\n"
-                         ::"r"(tmem_base + (uint32_t)(buf * kCols)), "l"(ad), "l"(bd), "r"(idesc), "r"(accum) : "memory");
-        }
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(smem_u32(&bar[buf])) : "memory");
-    };
-    if (kBuf == 2 && my_tiles > 0 && threadIdx.x == 0) issue_tile(0);
-
-    constexpr int kVec = FMT == kZetaF32 ? 4 : (FMT == kZetaI8 ? 16 : 8);     // elements per 16-byte store
     const int lane_base = 32 * (warp & 3);                  // a warp reads tensor-memory lanes 32 (warp % 4) .. + 31
-    const int c_begin = (warp >> 2) * (N / 2), c_end = c_begin + N / 2;       // warps 0-3: lower half of the columns
+    const int c_begin = (warp >> 2) * (N / 2);              // warps 0-3: lower half of the columns, 4-7: upper half
+    constexpr int kRowBytes = (N / 2) * kElt;               // bytes of a row that one warp produces
+    constexpr int kPpr = kRowBytes >= 128 ? 8 : kRowBytes / 16;     // 16-byte pieces per row and pass (128 bytes at most)
+    constexpr int kChunksPerPass = kPpr / kElt > 0 ? kPpr / kElt : 1;
+    static_assert(kPpr % kElt == 0 && kRowBytes % (16 * kPpr) == 0, "a pass is a whole number of 16-column chunks");
+    constexpr int kPasses = kRowBytes / (16 * kPpr);
+    unsigned char* scr = As + warp * 4096;                  // 32 rows x 128 bytes; piece p of row r at r * 128 + ((p ^ (r & 7)) * 16)
     bool ok = true;
     for (int64_t i = 0; i < my_tiles; ++i) {
-        const int buf = kBuf == 2 ? (int)(i & 1) : 0;
-        if (kBuf == 2) {
-            if (i + 1 < my_tiles)                           // next tile's features: its buffer was released by the wait of tile i - 1
-                stage_operand(As0 + (buf ^ 1) * a_bytes, kTcRows, A + tile_row0(i + 1) * stride_a, stride_a, n - tile_row0(i + 1));
-        } else {
-            stage_operand(As0, kTcRows, A + tile_row0(i) * stride_a, stride_a, n - tile_row0(i));   // the wait of tile i - 1 released it
+        // ---- expand this tile's bits (in registers since the previous tile) into the operand
+        if (my_item) {
+            const bool in = tile_row0(i) + my_r < n;
+            const uint32_t ws[4] = {pre.x, pre.y, pre.z, pre.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = lo;
+                if (in) expand_word(ws[u], lo, hi);
+                *reinterpret_cast<uint4*>(As + canon_off(kTcRows, my_r, 2 * (4 * my_piece + u))) = lo;
+                *reinterpret_cast<uint4*>(As + canon_off(kTcRows, my_r, 2 * (4 * my_piece + u) + 1)) = hi;
+            }
         }
         asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
-        __syncthreads();                                    // staging done; everyone is past the reads of the accumulator to be overwritten
+        __syncthreads();                                    // operand complete; everyone is past the previous tile's accumulator reads
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-        if (kBuf == 2) {
-            if (i + 1 < my_tiles && threadIdx.x == 0) issue_tile(buf ^ 1);
-        } else if (threadIdx.x == 0) {
-            issue_tile(0);
+        if (threadIdx.x == 0) {                             // one thread: all K steps of the tile, then the commit
+            const uint32_t a_base = smem_u32(As), b_base = smem_u32(Bs);
+            for (int ks = 0; ks < K / 32; ++ks) {
+                const uint64_t ad = make_desc(a_base + 2 * ks * a_lbo, a_lbo, sbo);
+                const uint64_t bd = make_desc(b_base + 2 * ks * b_lbo, b_lbo, sbo);
+                const uint32_t accum = ks > 0 ? 1u : 0u;
+                asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}\n"
+                             ::"r"(tmem_base), "l"(ad), "l"(bd), "r"(idesc), "r"(accum) : "memory");
+            }
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(smem_u32(&bar)) : "memory");
         }
-        if (!wait_barrier(&bar[buf], (uint32_t)((kBuf == 2 ? (i >> 1) : i) & 1))) {
+        pre = fetch(i + 1);                                 // in flight while the products and the epilogue run
+        if (!wait_barrier(&bar, (uint32_t)(i & 1))) {
             atomicExch(&g_tc_timeout, 1);
             ok = false;
         }
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
         if (__syncthreads_or(!ok)) break;                   // leave together if any wait ran out
-        // ---- epilogue of tile i: a thread owns one row and walks over its half of the columns
-        const int64_t row = tile_row0(i) + lane_base + lane;
+        // ---- epilogue: a thread owns row lane_base + lane and walks over its warp's half of the columns
+        const int64_t row0 = tile_row0(i) + lane_base;
+        const int64_t row = row0 + lane;
         const bool row_in = row < n;
         const float be = (row_in && (FMT == kZetaF32 || dbg_zeta)) ? __ldg(beta + row) : 0.f;
-        for (int c0 = c_begin; c0 < c_end; c0 += 16) {
-            uint32_t v[16];
-            const uint32_t taddr = tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)(buf * kCols + c0);
-            asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
-                         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-                           "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-                         : "r"(taddr) : "memory");
-            asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-            if (!row_in) continue;
-            int dot[16];
+#pragma unroll 1
+        for (int pass = 0; pass < kPasses; ++pass) {
 #pragma unroll
-            for (int q = 0; q < 16; ++q) dot[q] = (c0 + q < d_out) ? (int)v[q] - pad : 0;      // padding columns of zeta stay 0
-            if constexpr (FMT == kZetaF16) {
-                // exact integer -> fp16 without the conversion unit: the bit pattern 0x6600 + dot is the half 1536 + dot (|dot| <= 256 here)
-                uint32_t h[8];
+            for (int ch = 0; ch < kChunksPerPass; ++ch) {
+                const int c0 = c_begin + (pass * kChunksPerPass + ch) * 16;
+                uint32_t v[16];
+                const uint32_t taddr = tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)c0;
+                asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+                             : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                               "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                             : "r"(taddr) : "memory");
+                asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+                int dot[16];
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const __half2 biased = __halves2half2(__ushort_as_half((unsigned short)(0x6600 + dot[2 * q])), __ushort_as_half((unsigned short)(0x6600 + dot[2 * q + 1])));
-                    const __half2 r = __hsub2(biased, __half2half2(__ushort_as_half((unsigned short)0x6600)));
-                    h[q] = *reinterpret_cast<const uint32_t*>(&r);
+                for (int e = 0; e < 16; ++e) dot[e] = (c0 + e < d_out) ? (int)v[e] - pad : 0;   // padding columns of zeta stay 0
+                uint4 out[kElt];
+                Out::pack(dot, be, al_s + c0, out);
+#pragma unroll
+                for (int u = 0; u < kElt; ++u) {
+                    const int piece = ch * kElt + u;
+                    *reinterpret_cast<uint4*>(scr + lane * 128 + ((piece ^ (lane & 7)) * 16)) = out[u];
                 }
-                __half* dst = reinterpret_cast<__half*>(zeta) + row * ldz + c0;
-                if (c0 < ldz) *reinterpret_cast<uint4*>(dst) = make_uint4(h[0], h[1], h[2], h[3]);
-                if (c0 + 8 < ldz) *reinterpret_cast<uint4*>(dst + 8) = make_uint4(h[4], h[5], h[6], h[7]);
-            } else if constexpr (FMT == kZetaI16) {
-                uint32_t h[8];
+                if (row_in && (dbg_dot || dbg_zeta)) {
 #pragma unroll
-                for (int q = 0; q < 8; ++q) h[q] = ((uint32_t)dot[2 * q] & 0xffffu) | ((uint32_t)dot[2 * q + 1] << 16);
-                int16_t* dst = reinterpret_cast<int16_t*>(zeta) + row * ldz + c0;
-                if (c0 < ldz) *reinterpret_cast<uint4*>(dst) = make_uint4(h[0], h[1], h[2], h[3]);
-                if (c0 + 8 < ldz) *reinterpret_cast<uint4*>(dst + 8) = make_uint4(h[4], h[5], h[6], h[7]);
-            } else if constexpr (FMT == kZetaI8) {
-                uint32_t b[4];
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    b[q] = ((uint32_t)dot[4 * q] & 0xffu) | (((uint32_t)dot[4 * q + 1] & 0xffu) << 8) | (((uint32_t)dot[4 * q + 2] & 0xffu) << 16) | ((uint32_t)dot[4 * q + 3] << 24);
-                int8_t* dst = reinterpret_cast<int8_t*>(zeta) + row * ldz + c0;
-                if (c0 < ldz) *reinterpret_cast<uint4*>(dst) = make_uint4(b[0], b[1], b[2], b[3]);
-            } else {
-                float* dst = reinterpret_cast<float*>(zeta) + row * ldz + c0;
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    float f[4];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int c = c0 + 4 * q4 + q;
-                        f[q] = c < d_out ? __fmul_rn(__fmul_rn(be, al_s[c]), (float)dot[4 * q4 + q]) : 0.f;
-                    }
-                    if (c0 + 4 * q4 < ldz) *reinterpret_cast<float4*>(dst + 4 * q4) = make_float4(f[0], f[1], f[2], f[3]);
-                }
-            }
-            if (dbg_dot || dbg_zeta) {
-#pragma unroll
-                for (int q = 0; q < 16; ++q) {
-                    const int c = c0 + q;
-                    if (c < d_out) {
-                        if (dbg_dot) dbg_dot[row * (int64_t)d_out + c] = dot[q];
-                        if (dbg_zeta) dbg_zeta[row * (int64_t)d_out + c] = __fmul_rn(__fmul_rn(be, al_s[c]), (float)dot[q]);
+                    for (int e = 0; e < 16; ++e) {
+                        const int c = c0 + e;
+                        if (c < d_out) {
+                            if (dbg_dot) dbg_dot[row * (int64_t)d_out + c] = dot[e];
+                            if (dbg_zeta) dbg_zeta[row * (int64_t)d_out + c] = __fmul_rn(__fmul_rn(be, al_s[c]), (float)dot[e]);
+                        }
                     }
                 }
             }
+            __syncwarp();
+            // write the 32 rows x kPpr pieces out: a warp instruction covers 32 / kPpr whole row segments
+            const int64_t byte0 = (int64_t)(c_begin + pass * kChunksPerPass * 16) * kElt;       // first byte of the pass inside a row of zeta
+#pragma unroll
+            for (int it = 0; it < kPpr; ++it) {
+                const int r = it * (32 / kPpr) + lane / kPpr, pc = lane % kPpr;
+                const uint4 val = *reinterpret_cast<const uint4*>(scr + r * 128 + ((pc ^ (r & 7)) * 16));
+                const int64_t at = byte0 + pc * 16;
+                if (row0 + r < n && at < ldz * kElt)
+                    *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(zeta) + (row0 + r) * ldz * kElt + at) = val;
+            }
+            __syncwarp();
         }
-        (void)kVec;
+        asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+        __syncthreads();                                    // the scratch is the next tile's operand space
     }
     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
     __syncthreads();
-    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(kBuf * kCols) : "memory");
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(kCols) : "memory");
 }
 
 template <int N, int FMT>
@@ -259,13 +318,12 @@ cudaError_t launch_tc_inst(cudaStream_t s, const uint32_t* A, int64_t stride_a, 
                            int64_t n, int d_in, int d_out, const float* beta, const float* alpha, void* zeta, int64_t ldz,
                            int32_t* dbg_dot, float* dbg_zeta)
 {
-    // two CTAs per SM, each with one feature tile and one accumulator (N <= 256 columns each: 512 in all)
-    constexpr int kBuf = 1;
-    const size_t smem = (size_t)(N + kBuf * kTcRows) * stride_a * 32;
-    cudaError_t e = cudaFuncSetAttribute(bitgemm_tc_kernel<N, FMT, kBuf>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    // operands: weight panel N x K bytes, feature tile 128 x K bytes (at least the 32 KB the epilogue's scratch needs)
+    const size_t smem = (size_t)N * stride_a * 32 + std::max<size_t>((size_t)kTcRows * stride_a * 32, 32 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(bitgemm_tc_kernel<N, FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, kTcRows), 148 * (kBuf == 1 ? 2 : 1));
-    bitgemm_tc_kernel<N, FMT, kBuf><<<grid, kTcThreads, smem, s>>>(A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta);
+    const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, kTcRows), 148 * 2);
+    bitgemm_tc_kernel<N, FMT><<<grid, kTcThreads, smem, s>>>(A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta);
     return cudaGetLastError();
 }
 
