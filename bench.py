@@ -339,6 +339,20 @@ def run_ours(args):
             extras["popc_word_steps_per_s"] = ctx.measure_popc_peak()
         except Exception as exc:
             extras["popc_word_steps_per_s"] = None
+        # the same contraction on the XOR / bit-count pipe (the library's other path), for comparison
+        try:
+            ctx.set_option(binding.OPT_CONTRACTION, 1)
+            pop = [[] for _ in range(L)]
+            for k in range(3 + min(args.steps, 5)):
+                _, st = ctx.forward(G, layers, X, logits, stats=True)
+                if k >= 3:
+                    for l in range(L):
+                        pop[l].append(st.ms_gemm[l])
+            extras["bitgemm_popc_pipe_ms"] = [sum(v) / len(v) for v in pop]
+        except Exception as exc:
+            extras["bitgemm_popc_pipe_ms"] = "failed: %r" % (exc,)
+        finally:
+            ctx.set_option(binding.OPT_CONTRACTION, 0)
 
     # end to end through the host-buffer entry points: every step copies its input from pinned host
     # memory and its logits back to pinned host memory.  Headline: the pipelined entry point (the
@@ -430,10 +444,17 @@ def run_ours(args):
         ops = 2.0 * n * dims[l] * dims[l + 1]
         words = n * dims[l + 1] * ((dims[l] + 31) // 32)                  # XOR + bit-count + add steps
         popc_peak = extras.get("popc_word_steps_per_s")
-        kernels["bitgemm_l%d" % l] = {"ms": gemm_ms[l], "binary_TOPS": ops / (gemm_ms[l] * 1e-3) / 1e12,
+        on_tc = dims[l] <= 256 and dims[l + 1] <= 256       # the library's rule for the tensor-core path
+        k_pad = binding.packed_stride_words(dims[l]) * 32
+        io_bytes = n * (binding.packed_stride_words(dims[l]) * 4.0 + 4.0 + ldz * elt)
+        kernels["bitgemm_l%d" % l] = {"ms": gemm_ms[l], "path": "tcgen05 int8" if on_tc else "xor+popc",
+                                      "binary_TOPS": ops / (gemm_ms[l] * 1e-3) / 1e12,
+                                      "int8_TOPS_issued": (2.0 * n * k_pad * dims[l + 1] / (gemm_ms[l] * 1e-3) / 1e12) if on_tc else None,
                                       "word_steps_per_s": words / (gemm_ms[l] * 1e-3),
                                       "frac_of_popc_peak": (words / (gemm_ms[l] * 1e-3) / popc_peak) if popc_peak else None,
-                                      "out_GBps": n * ldz * elt / (gemm_ms[l] * 1e-3) / 1e9}
+                                      "out_GBps": n * ldz * elt / (gemm_ms[l] * 1e-3) / 1e9,
+                                      "GBps": io_bytes / (gemm_ms[l] * 1e-3) / 1e9,
+                                      "frac_of_hbm_peak": io_bytes / (gemm_ms[l] * 1e-3) / 1e9 / peak}
     pack_bytes = n * (dims[0] * 4.0 + binding.packed_stride_words(dims[0]) * 4.0 + 4.0)
     kernels["pack_features"] = {"ms": pack_ms, "GBps": pack_bytes / (pack_ms * 1e-3) / 1e9,
                                 "frac_of_hbm_peak": pack_bytes / (pack_ms * 1e-3) / 1e9 / peak}

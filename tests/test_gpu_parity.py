@@ -145,6 +145,33 @@ LAYER_SHAPES = [(200, 1500, 1, 1), (300, 2500, 33, 7), (500, 6000, 100, 256), (4
 @pytest.mark.parametrize("fmt", FORMATS)
 @pytest.mark.parametrize("n,e,d_in,d_out", LAYER_SHAPES)
 def test_layer_forward_against_oracle(ctx, B, fmt, n, e, d_in, d_out):
+    check_layer_forward(ctx, B, fmt, n, e, d_in, d_out)
+
+
+# shapes the tensor-core contraction covers (d_in, d_out <= 256): tile tails, one row, several tiles per CTA
+TC_SHAPES = [(5, 6, 256, 256), (127, 900, 256, 256), (128, 900, 100, 256), (129, 900, 256, 47), (1000, 9000, 200, 130),
+             (40000, 200000, 256, 256), (39000, 150000, 100, 64)]
+
+
+@pytest.mark.parametrize("fmt", [1, 4])
+@pytest.mark.parametrize("n,e,d_in,d_out", TC_SHAPES)
+def test_layer_forward_tensor_core_contraction(ctx, B, fmt, n, e, d_in, d_out):
+    check_layer_forward(ctx, B, fmt, n, e, d_in, d_out)
+
+
+@pytest.mark.parametrize("fmt", [1, 3, 4])
+@pytest.mark.parametrize("n,e,d_in,d_out", [s for s in LAYER_SHAPES if s[2] <= 256 and s[3] <= 256])
+def test_layer_forward_on_the_bit_count_pipe(ctx, B, fmt, n, e, d_in, d_out):
+    """The library's other contraction path (XOR + bit count on the integer pipe) for the shapes that take the
+    tensor cores by default."""
+    ctx.set_option(B.OPT_CONTRACTION, 1)
+    try:
+        check_layer_forward(ctx, B, fmt, n, e, d_in, d_out)
+    finally:
+        ctx.set_option(B.OPT_CONTRACTION, 0)
+
+
+def check_layer_forward(ctx, B, fmt, n, e, d_in, d_out):
     rng = np.random.default_rng(n + 3 * d_in + 7 * d_out)
     _, _, g = small_graph(n, e, 100 + n)
     H = rng.standard_normal((n, d_in)).astype(np.float32)
