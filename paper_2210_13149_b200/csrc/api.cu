@@ -336,6 +336,7 @@ bigcn_status bigcn_sync_check(bigcn_ctx* ctx)
     BIGCN_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     BIGCN_CUDA(ctx, cudaGetLastError());
     if (bitgemm_tc_timeouts() != 0) return fail(ctx, BIGCN_ERR_INTERNAL, "a bounded wait on the tensor cores ran out (contraction kernel)");
+    if (backward_tc_timeouts() != 0) return fail(ctx, BIGCN_ERR_INTERNAL, "a bounded wait on the tensor cores ran out (backward kernel)");
     return BIGCN_OK;
 }
 

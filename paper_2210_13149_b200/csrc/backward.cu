@@ -12,6 +12,7 @@
 #include <cuda_bf16.h>
 
 #include "bigcn_internal.cuh"
+#include "tc_common.cuh"
 
 namespace bigcn {
 
@@ -286,6 +287,178 @@ grad_wt_mma_kernel(const uint32_t* __restrict__ bits, int64_t stride, const floa
         }
 }
 
+// ---- G_H on the 5th-generation tensor cores ---------------------------------------------------------------
+// The same product as grad_h_mma_kernel with tcgen05.mma kind::f16 (bf16 operands, fp32 accumulators in
+// tensor memory): M = 128 rows, N = 64 / 128 / 256 >= d_in, the reduction over the output channels in
+// chunks of 64 (128 bytes per operand row: the three terms of the fp32 operand take 48 KB, the +-1
+// operand N x 128 bytes).  Two CTAs per SM overlap each other's staging, products and epilogue.  Operands
+// are K-major no-swizzle (core matrices of 8 rows x 16 bytes).  The epilogue reads the accumulators back
+// (a thread owns one row), clips (Eq. bp-H) and writes through shared memory as 128-byte row segments.
+// Needs d_in a multiple of 4 and 16-byte aligned rows of g_h; every mbarrier wait is bounded.
+__device__ int g_bw_tc_timeout;
+
+template <int N>
+__global__ void __launch_bounds__(kBwThreads, 2)
+grad_h_tc_kernel(const float* __restrict__ gz, int64_t ldz, const float* __restrict__ alpha,
+                 const float* __restrict__ W, int64_t ldw, int64_t n, int d_in, int d_out,
+                 float* __restrict__ g_h, int64_t ldh)
+{
+    constexpr int kRows = 128, kKc = 64;                   // tile rows; reduction elements per chunk
+    constexpr int kCols = N <= 64 ? 64 : (N <= 128 ? 128 : 256);
+    extern __shared__ __align__(128) unsigned char bw_smem[];
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ uint32_t tmem_base_s;
+    unsigned char* As = bw_smem;                            // [3][128][128 bytes]; also the epilogue's scratch (>= 32 KB)
+    unsigned char* Bs = bw_smem + 3 * kRows * 128;          // [N][128 bytes]
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (warp == 0) tc::tmem_alloc(&tmem_base_s, kCols);
+    if (threadIdx.x == 0) tc::barrier_init(&bar);
+    tc::fence_before_sync();
+    __syncthreads();
+    tc::fence_after_sync();
+    const uint32_t tmem_base = tmem_base_s;
+    // instruction descriptor: D = f32, A = B = bf16, both K-major, N, M = 128
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kRows >> 4) << 24);
+    const uint32_t a_lbo = (kRows >> 3) * 128, b_lbo = (N >> 3) * 128, sbo = 128;
+    const bool vec_ok = (ldz % 4 == 0) && (reinterpret_cast<uintptr_t>(gz) % 16 == 0);
+    const bool w_vec_ok = (ldw % 4 == 0) && (reinterpret_cast<uintptr_t>(W) % 16 == 0);
+    const int n_chunks = (d_out + kKc - 1) / kKc;
+    const int64_t n_tiles = ceil_div(n, kRows);
+    const int lane_base = 32 * (warp & 3);
+    const int c_begin = (warp >> 2) * (N / 2);
+    unsigned char* scr = As + warp * 4096;                  // 32 rows x 128 bytes, pieces swizzled by (row & 7)
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const int64_t i0 = tile * kRows;
+        for (int ch = 0; ch < n_chunks; ++ch) {
+            const int j0 = ch * kKc;
+            // A: 128 rows x 16 quads of channels -> three bf16 terms of G_zeta * alpha
+            for (int t = threadIdx.x; t < kRows * (kKc / 4); t += kBwThreads) {
+                const int jq = (t & 15) * 4, r = t >> 4;
+                const int j = j0 + jq;
+                const int64_t row = i0 + r;
+                float x[4] = {0.f, 0.f, 0.f, 0.f};
+                if (row < n) {
+                    if (j + 3 < d_out && vec_ok) {
+                        const float4 v = __ldg(reinterpret_cast<const float4*>(gz + row * ldz + j));
+                        x[0] = v.x, x[1] = v.y, x[2] = v.z, x[3] = v.w;
+                    } else {
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (j + u < d_out) x[u] = __ldg(gz + row * ldz + j + u);
+                    }
+                }
+                unsigned short hi[4], mid[4], lo[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) split3(j + u < d_out ? __fmul_rn(x[u], __ldg(alpha + j + u)) : 0.f, hi[u], mid[u], lo[u]);
+                auto pack = [](const unsigned short (&h)[4]) { return make_uint2((uint32_t)h[0] | ((uint32_t)h[1] << 16), (uint32_t)h[2] | ((uint32_t)h[3] << 16)); };
+                const uint32_t off = tc::canon_off(kRows, r, jq >> 3) + (jq & 7) * 2;
+                *reinterpret_cast<uint2*>(As + 0 * kRows * 128 + off) = pack(hi);
+                *reinterpret_cast<uint2*>(As + 1 * kRows * 128 + off) = pack(mid);
+                *reinterpret_cast<uint2*>(As + 2 * kRows * 128 + off) = pack(lo);
+            }
+            // B: N inputs x 16 quads of channels -> sign of W as +-1
+            for (int t = threadIdx.x; t < N * (kKc / 4); t += kBwThreads) {
+                const int jq = (t & 15) * 4, k = t >> 4;
+                const int j = j0 + jq;
+                unsigned short sg[4] = {0, 0, 0, 0};
+                if (k < d_in) {
+                    if (j + 3 < d_out && w_vec_ok) {
+                        const float4 v = __ldg(reinterpret_cast<const float4*>(W + (int64_t)k * ldw + j));
+                        sg[0] = v.x >= 0.f ? 0x3F80 : 0xBF80, sg[1] = v.y >= 0.f ? 0x3F80 : 0xBF80;
+                        sg[2] = v.z >= 0.f ? 0x3F80 : 0xBF80, sg[3] = v.w >= 0.f ? 0x3F80 : 0xBF80;
+                    } else {
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (j + u < d_out) sg[u] = __ldg(W + (int64_t)k * ldw + j + u) >= 0.f ? 0x3F80 : 0xBF80;
+                    }
+                }
+                const uint32_t off = tc::canon_off(N, k, jq >> 3) + (jq & 7) * 2;
+                *reinterpret_cast<uint2*>(Bs + off) = make_uint2((uint32_t)sg[0] | ((uint32_t)sg[1] << 16), (uint32_t)sg[2] | ((uint32_t)sg[3] << 16));
+            }
+            tc::fence_async_smem();
+            tc::fence_before_sync();
+            __syncthreads();                                // operands complete; previous tile's accumulator reads are over
+            tc::fence_after_sync();
+            if (threadIdx.x == 0) {
+                const uint32_t a_base = tc::smem_u32(As), b_base = tc::smem_u32(Bs);
+                for (int ks = 0; ks < kKc / 16; ++ks) {
+                    const uint64_t bd = tc::make_desc(b_base + 2 * ks * b_lbo, b_lbo, sbo);
+#pragma unroll
+                    for (int sp = 0; sp < 3; ++sp) {
+                        const uint64_t ad = tc::make_desc(a_base + sp * kRows * 128 + 2 * ks * a_lbo, a_lbo, sbo);
+                        const uint32_t accum = (ch > 0 || ks > 0 || sp > 0) ? 1u : 0u;
+                        asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+                                     ::"r"(tmem_base), "l"(ad), "l"(bd), "r"(idesc), "r"(accum) : "memory");
+                    }
+                }
+                tc::commit_to(&bar);
+            }
+            if (!tc::wait_barrier(&bar, phase)) {
+                atomicExch(&g_bw_tc_timeout, 1);
+                ok = false;
+            }
+            phase ^= 1u;
+            tc::fence_after_sync();
+            if (__syncthreads_or(!ok)) { ok = false; break; }   // the operands may be overwritten; leave together on a timeout
+        }
+        if (!ok) break;
+        // ---- epilogue: clip and write the tile (a thread owns row lane_base + lane, its warp's half of the columns)
+        const int64_t row0 = i0 + lane_base;
+        constexpr int kPasses = (N / 2) * 4 / 128 > 0 ? (N / 2) * 4 / 128 : 1;    // 32 columns = 128 bytes per pass
+        constexpr int kPpr = (N / 2) * 4 >= 128 ? 8 : (N / 2) * 4 / 16;
+#pragma unroll 1
+        for (int pass = 0; pass < kPasses; ++pass) {
+#pragma unroll
+            for (int c2 = 0; c2 < kPpr / 4; ++c2) {
+                const int c0 = c_begin + pass * 32 + c2 * 16;
+                uint32_t v[16];
+                tc::tmem_ld16(tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)c0, v);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    float f[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float a = __uint_as_float(v[4 * u + e]);
+                        f[e] = fabsf(a) < 1.f ? a : 0.f;                                  // Eq. bp-H
+                    }
+                    const int piece = c2 * 4 + u;
+                    *reinterpret_cast<uint4*>(scr + lane * 128 + ((piece ^ (lane & 7)) * 16)) =
+                        make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
+                }
+            }
+            __syncwarp();
+            const int col0 = c_begin + pass * 32;
+#pragma unroll
+            for (int it = 0; it < kPpr; ++it) {
+                const int r = it * (32 / kPpr) + lane / kPpr, pc = lane % kPpr;
+                const uint4 val = *reinterpret_cast<const uint4*>(scr + r * 128 + ((pc ^ (r & 7)) * 16));
+                const int col = col0 + pc * 4;
+                if (row0 + r < n && col < d_in) *reinterpret_cast<uint4*>(g_h + (row0 + r) * ldh + col) = val;
+            }
+            __syncwarp();
+        }
+        tc::fence_before_sync();
+        __syncthreads();                                    // the scratch is the next tile's operand space
+    }
+    tc::fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tc::tmem_free(tmem_base, kCols);
+}
+
+template <int N>
+cudaError_t launch_grad_h_tc(cudaStream_t s, const float* gz, int64_t ldz, const float* alpha, const float* W, int64_t ldw,
+                             int64_t n, int d_in, int d_out, float* g_h, int64_t ldh)
+{
+    const size_t smem = 3 * 128 * 128 + (size_t)N * 128;
+    cudaError_t e = cudaFuncSetAttribute(grad_h_tc_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, 128), 148 * 2);
+    grad_h_tc_kernel<N><<<grid, kBwThreads, smem, s>>>(gz, ldz, alpha, W, ldw, n, d_in, d_out, g_h, ldh);
+    return cudaGetLastError();
+}
+
 // Eq. bp-W.  One block per 32 output channels: thread (tx, ty) sums G_W~_kj B_kj over k = ty, ty + 32, ...
 // for channel j0 + tx in double; the 32 partial sums of a channel are added in a fixed order; then
 // every element gets (1/d_in) B_ij col_j + alpha_j G_W~_ij [|W_ij| < 1].
@@ -334,6 +507,13 @@ int wt_splits(int64_t n, int d_in, int d_out)
 }
 
 }  // namespace
+
+int backward_tc_timeouts()
+{
+    int v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_bw_tc_timeout, sizeof(int)) != cudaSuccess) return -1;
+    return v;
+}
 
 size_t backward_scratch_bytes(int64_t n, int d_in, int d_out)
 {
@@ -418,10 +598,17 @@ cudaError_t launch_layer_backward(cudaStream_t s, int64_t n, const int64_t* rowp
     }
     // step 1c + 2: G_H = clip(G_zeta W~^T)
     if (g_in) {
-        const dim3 grid((unsigned)ceil_div(n, kMmaTile), (unsigned)ceil_div(d_in, kMmaTile));
-        grad_h_mma_kernel<<<grid, kBwThreads, 0, s>>>(gz, ldz, alpha, W, ldw, n, d_in, d_out, g_in, ldgi);
         ++*launches;
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        if (d_in <= 256 && d_in % 4 == 0 && ldgi % 4 == 0 && reinterpret_cast<uintptr_t>(g_in) % 16 == 0) {   // tcgen05 version
+            if (d_in <= 64) e = launch_grad_h_tc<64>(s, gz, ldz, alpha, W, ldw, n, d_in, d_out, g_in, ldgi);
+            else if (d_in <= 128) e = launch_grad_h_tc<128>(s, gz, ldz, alpha, W, ldw, n, d_in, d_out, g_in, ldgi);
+            else e = launch_grad_h_tc<256>(s, gz, ldz, alpha, W, ldw, n, d_in, d_out, g_in, ldgi);
+            if (e != cudaSuccess) return e;
+        } else {
+            const dim3 grid((unsigned)ceil_div(n, kMmaTile), (unsigned)ceil_div(d_in, kMmaTile));
+            grad_h_mma_kernel<<<grid, kBwThreads, 0, s>>>(gz, ldz, alpha, W, ldw, n, d_in, d_out, g_in, ldgi);
+            if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        }
     }
     // step 3: Eq. bp-W
     grad_w_kernel<<<(unsigned)ceil_div(d_out, 32), dim3(32, 32), 0, s>>>(g_wt, W, ldw, alpha, d_in, d_out, g_w, ldgw);

@@ -94,6 +94,7 @@ int entropy_max_bins();
 
 // Back-propagation through one binarized layer (backward.cu).
 size_t backward_scratch_bytes(int64_t n, int d_in, int d_out);
+int backward_tc_timeouts();
 cudaError_t launch_layer_backward(cudaStream_t s, int64_t n, const int64_t* rowptr, const int32_t* colidx,
                                   const float* val, int d_in, int d_out, const float* W, int64_t ldw,
                                   const float* alpha, const uint32_t* in_bits, int64_t stride_in,

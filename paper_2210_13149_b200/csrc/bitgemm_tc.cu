@@ -19,6 +19,7 @@
 #include <cuda_fp16.h>
 
 #include "bigcn_internal.cuh"
+#include "tc_common.cuh"
 
 namespace bigcn {
 
@@ -26,11 +27,13 @@ namespace {
 
 constexpr int kTcThreads = 256;
 constexpr int kTcRows = 128;                  // rows per tile = M of the instruction
-constexpr int kTcWaitTries = 1 << 22;         // bound of every mbarrier wait
 
 __device__ int g_tc_timeout;                  // set when a wait ran out
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+using tc::canon_off;
+using tc::make_desc;
+using tc::smem_u32;
+using tc::wait_barrier;
 
 // 4 bits -> 4 bytes of +1 (0x01) / -1 (0xFF): the multiplication spreads bit i to bit 8 i.
 __device__ __forceinline__ uint32_t expand4(uint32_t nib)
@@ -42,26 +45,6 @@ __device__ __forceinline__ void expand_word(uint32_t w, uint4& lo, uint4& hi)
 {
     lo = make_uint4(expand4(w & 15u), expand4((w >> 4) & 15u), expand4((w >> 8) & 15u), expand4((w >> 12) & 15u));
     hi = make_uint4(expand4((w >> 16) & 15u), expand4((w >> 20) & 15u), expand4((w >> 24) & 15u), expand4(w >> 28));
-}
-
-// Byte offset of (row r, 16-byte K chunk) in a K-major no-swizzle operand of `rows` rows: the core
-// matrices (8 rows x 16 bytes = 128 contiguous bytes) of one K chunk follow each other over the row
-// groups; K chunks are rows / 8 * 128 bytes apart.
-__device__ __forceinline__ uint32_t canon_off(int rows, int r, int kchunk)
-{
-    return (uint32_t)((kchunk * (rows >> 3) + (r >> 3)) * 128 + (r & 7) * 16);
-}
-
-// Shared-memory matrix descriptor: start address, leading (K direction) and stride (row-group
-// direction) byte offsets in 16-byte units, descriptor version 1, no swizzle.
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
-    d |= (uint64_t)1 << 46;
-    return d;
 }
 
 // Expands `rows_valid` packed rows (stride words each, read 16 bytes at a time) into the canonical
@@ -84,15 +67,6 @@ __device__ __forceinline__ void stage_operand(unsigned char* dst, int rows, cons
             *reinterpret_cast<uint4*>(dst + canon_off(rows, r, 2 * (4 * piece + i) + 1)) = hi;
         }
     }
-}
-
-__device__ __forceinline__ bool wait_barrier(uint64_t* bar, uint32_t parity)
-{
-    uint32_t done = 0;
-    for (int it = 0; it < kTcWaitTries && !done; ++it)
-        asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
-                     : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return done != 0;
 }
 
 // Converts 16 consecutive dots of one row to the storage format: kPieces 16-byte pieces.
