@@ -444,7 +444,7 @@ def run_ours(args):
         ops = 2.0 * n * dims[l] * dims[l + 1]
         words = n * dims[l + 1] * ((dims[l] + 31) // 32)                  # XOR + bit-count + add steps
         popc_peak = extras.get("popc_word_steps_per_s")
-        on_tc = dims[l] <= 256 and dims[l + 1] <= 256       # the library's rule for the tensor-core path
+        on_tc = dims[l] <= 256 and dims[l + 1] <= 256 and n * dims[l + 1] >= (1 << 20)   # the library's rule for the tensor-core path
         k_pad = binding.packed_stride_words(dims[l]) * 32
         io_bytes = n * (binding.packed_stride_words(dims[l]) * 4.0 + 4.0 + ldz * elt)
         kernels["bitgemm_l%d" % l] = {"ms": gemm_ms[l], "path": "tcgen05 int8" if on_tc else "xor+popc",

@@ -70,7 +70,8 @@ enum {
     BIGCN_OPT_LONG_ROW = 2,
     /* How the binary contraction runs.  0 = default: as int8 tensor-core products (tcgen05, the packed bits
      * expanded to +1 / -1 bytes in shared memory; the same integers) for layers with d_in <= 256 and
-     * d_out <= 256, on the XOR / bit-count pipe otherwise; 1 = always on the XOR / bit-count pipe. */
+     * d_out <= 256 and at least 2^20 outputs, on the XOR / bit-count pipe otherwise; 1 = always on the
+     * XOR / bit-count pipe; 2 = tensor cores for every layer with d_in <= 256 and d_out <= 256. */
     BIGCN_OPT_CONTRACTION = 3
 };
 

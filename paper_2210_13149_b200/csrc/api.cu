@@ -19,7 +19,7 @@ struct bigcn_ctx {
     int64_t launches;
     int zeta_format;             // 0 = auto
     int64_t long_row;            // 0 = default
-    int contraction;             // 0 = tensor cores where covered, 1 = bit-count pipe
+    int contraction;             // 0 = auto, 1 = bit-count pipe, 2 = tensor cores wherever covered
     cudaEvent_t ev[2 * BIGCN_MAX_LAYERS + 2];
     bool ev_ready;
 };
@@ -120,7 +120,7 @@ bigcn_status run_layer(bigcn_ctx* ctx, const bigcn_graph* g, const bigcn_layer* 
     const int64_t stride_in = bigcn_packed_stride_words(layer->d_in);
     cudaError_t e = launch_bitgemm(ctx->stream, in_bits, stride_in, layer->w_bitsT, stride_in, g->n,
                                    layer->d_in, layer->d_out, in_beta, layer->alpha, fmt, zeta, ldz,
-                                   dbg_dot, dbg_zeta, &ctx->launches_i, ctx->contraction == 0);
+                                   dbg_dot, dbg_zeta, &ctx->launches_i, ctx->contraction);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "bit-GEMM launch");
     if (ev_mid) BIGCN_CUDA(ctx, cudaEventRecord(ev_mid, ctx->stream));
     SpmmArgs a;
@@ -320,7 +320,7 @@ bigcn_status bigcn_set_option(bigcn_ctx* ctx, int32_t option, int64_t value)
             ctx->long_row = value;
             return BIGCN_OK;
         case BIGCN_OPT_CONTRACTION:
-            if (value < 0 || value > 1) return fail(ctx, BIGCN_ERR_SHAPE, "contraction path %lld not in 0..1", (long long)value);
+            if (value < 0 || value > 2) return fail(ctx, BIGCN_ERR_SHAPE, "contraction path %lld not in 0..2", (long long)value);
             ctx->contraction = (int)value;
             return BIGCN_OK;
     }
@@ -819,12 +819,12 @@ bigcn_status bigcn_sage_layer_forward(bigcn_ctx* ctx, const bigcn_graph* mean_gr
     const int64_t stride_in = bigcn_packed_stride_words(d_in);
     const int64_t ld_self = zeta_ld(d_out, kZetaF32);
     cudaError_t e = launch_bitgemm(ctx->stream, in_bits, stride_in, self_layer->w_bitsT, stride_in, n, d_in, d_out,
-                                   in_beta, self_layer->alpha, kZetaF32, zeta_self, ld_self, nullptr, nullptr, &ctx->launches_i, ctx->contraction == 0);
+                                   in_beta, self_layer->alpha, kZetaF32, zeta_self, ld_self, nullptr, nullptr, &ctx->launches_i, ctx->contraction);
     if (e != cudaSuccess) { finish_call(ctx); return cuda_fail(ctx, e, "bit-GEMM (self term) launch"); }
     const int fmt = pick_format(ctx, d_in, d_out);
     const int64_t ldz = zeta_ld(d_out, fmt);
     e = launch_bitgemm(ctx->stream, in_bits, stride_in, nbr_layer->w_bitsT, stride_in, n, d_in, d_out,
-                       in_beta, nbr_layer->alpha, fmt, zeta_nbr, ldz, nullptr, nullptr, &ctx->launches_i, ctx->contraction == 0);
+                       in_beta, nbr_layer->alpha, fmt, zeta_nbr, ldz, nullptr, nullptr, &ctx->launches_i, ctx->contraction);
     if (e != cudaSuccess) { finish_call(ctx); return cuda_fail(ctx, e, "bit-GEMM (neighbour term) launch"); }
     SpmmArgs a;
     a.n = n;

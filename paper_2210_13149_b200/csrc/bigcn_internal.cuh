@@ -35,7 +35,7 @@ cudaError_t launch_pack_weights(cudaStream_t s, const float* W, int d_in, int d_
 cudaError_t launch_bitgemm(cudaStream_t s, const uint32_t* A, int64_t stride_a,
                            const uint32_t* BT, int64_t stride_b, int64_t n, int d_in, int d_out,
                            const float* beta, const float* alpha, int fmt, void* zeta, int64_t ldz,
-                           int32_t* dbg_dot, float* dbg_zeta, int* launches, bool tensor_cores = true);
+                           int32_t* dbg_dot, float* dbg_zeta, int* launches, int path = 0 /* 0 auto, 1 bit-count pipe, 2 tensor cores wherever covered */);
 
 struct SpmmArgs {
     int64_t n;

@@ -153,10 +153,14 @@ TC_SHAPES = [(5, 6, 256, 256), (127, 900, 256, 256), (128, 900, 100, 256), (129,
              (40000, 200000, 256, 256), (39000, 150000, 100, 64)]
 
 
-@pytest.mark.parametrize("fmt", [1, 4])
-@pytest.mark.parametrize("n,e,d_in,d_out", TC_SHAPES)
+@pytest.mark.parametrize("fmt", [1, 2, 3, 4])
+@pytest.mark.parametrize("n,e,d_in,d_out", TC_SHAPES + [s for s in LAYER_SHAPES if s[2] <= 256 and s[3] <= 256])
 def test_layer_forward_tensor_core_contraction(ctx, B, fmt, n, e, d_in, d_out):
-    check_layer_forward(ctx, B, fmt, n, e, d_in, d_out)
+    ctx.set_option(B.OPT_CONTRACTION, 2)          # also below the size from which it is the default
+    try:
+        check_layer_forward(ctx, B, fmt, n, e, d_in, d_out)
+    finally:
+        ctx.set_option(B.OPT_CONTRACTION, 0)
 
 
 @pytest.mark.parametrize("fmt", [1, 3, 4])
