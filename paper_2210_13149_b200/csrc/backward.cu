@@ -447,6 +447,155 @@ grad_h_tc_kernel(const float* __restrict__ gz, int64_t ldz, const float* __restr
     if (warp == 0) tc::tmem_free(tmem_base, kCols);
 }
 
+// ---- G_W~ partial sums on the 5th-generation tensor cores -------------------------------------------------
+// The product of grad_wt_mma_kernel (transposed: C^T[j][k] = sum over nodes of (beta_i G_zeta[i][j]) F[i][k])
+// with tcgen05.mma kind::f16: M = 128 channels j, N = 64 / 128 / 256 >= d_in inputs k, the reduction over
+// the CTA's nodes in chunks of 64, all of them accumulated in one fp32 tile of tensor memory that is read
+// back once at the end and written as slab blockIdx.y of `part` ([k][j]: consecutive lanes write consecutive
+// j).  Both operands are node-major in global memory; the staging transposes them, two nodes per 32-bit store.
+template <int N>
+__global__ void __launch_bounds__(kBwThreads, 2)
+grad_wt_tc_kernel(const uint32_t* __restrict__ bits, int64_t stride, const float* __restrict__ beta,
+                  const float* __restrict__ gz, int64_t ldz, int64_t n, int d_in, int d_out,
+                  int64_t rows_per_split, float* __restrict__ part)
+{
+    constexpr int kRows = 128, kKc = 64;                   // channels per tile; nodes per chunk
+    constexpr int kCols = N <= 64 ? 64 : (N <= 128 ? 128 : 256);
+    extern __shared__ __align__(128) unsigned char bw_smem[];
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ uint32_t tmem_base_s;
+    unsigned char* As = bw_smem;                            // [3][128 channels][64 nodes] bf16
+    unsigned char* Bs = bw_smem + 3 * kRows * 128;          // [N inputs][64 nodes] bf16
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (warp == 0) tc::tmem_alloc(&tmem_base_s, kCols);
+    if (threadIdx.x == 0) tc::barrier_init(&bar);
+    tc::fence_before_sync();
+    __syncthreads();
+    tc::fence_after_sync();
+    const uint32_t tmem_base = tmem_base_s;
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kRows >> 4) << 24);
+    const uint32_t a_lbo = (kRows >> 3) * 128, b_lbo = (N >> 3) * 128, sbo = 128;
+    const bool vec_ok = (ldz % 4 == 0) && (reinterpret_cast<uintptr_t>(gz) % 16 == 0);
+    const int j0 = blockIdx.x * kRows;
+    const int64_t r_begin = (int64_t)blockIdx.y * rows_per_split;
+    const int64_t r_end = min(n, r_begin + rows_per_split);
+    uint32_t phase = 0;
+    bool ok = true, any = false;
+    for (int64_t r0 = r_begin; r0 < r_end; r0 += kKc) {
+        // A: 32 node pairs x 32 quads of channels
+        for (int t = threadIdx.x; t < 32 * 32; t += kBwThreads) {
+            const int np = t & 31, jq = (t >> 5) * 4;
+            float x[2][4];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int64_t row = r0 + 2 * np + h;
+                const int j = j0 + jq;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) x[h][u] = 0.f;
+                if (row < r_end) {
+                    const float be = __ldg(beta + row);
+                    if (j + 3 < d_out && vec_ok) {
+                        const float4 v = __ldg(reinterpret_cast<const float4*>(gz + row * ldz + j));
+                        x[h][0] = v.x * be, x[h][1] = v.y * be, x[h][2] = v.z * be, x[h][3] = v.w * be;
+                    } else {
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (j + u < d_out) x[h][u] = __ldg(gz + row * ldz + j + u) * be;
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                unsigned short h0, m0, l0, h1, m1, l1;
+                split3(x[0][u], h0, m0, l0);
+                split3(x[1][u], h1, m1, l1);
+                const uint32_t off = tc::canon_off(kRows, jq + u, (2 * np) >> 3) + ((2 * np) & 7) * 2;
+                *reinterpret_cast<uint32_t*>(As + 0 * kRows * 128 + off) = (uint32_t)h0 | ((uint32_t)h1 << 16);
+                *reinterpret_cast<uint32_t*>(As + 1 * kRows * 128 + off) = (uint32_t)m0 | ((uint32_t)m1 << 16);
+                *reinterpret_cast<uint32_t*>(As + 2 * kRows * 128 + off) = (uint32_t)l0 | ((uint32_t)l1 << 16);
+            }
+        }
+        // B: 32 node pairs x (N / 32) packed words x 4 groups of 8 inputs
+        for (int t = threadIdx.x; t < 32 * (N / 32) * 4; t += kBwThreads) {
+            const int np = t & 31, wd = (t >> 5) >> 2, part8 = (t >> 5) & 3;
+            const int kw = wd * 32;                         // first input of the word
+            const int64_t row = r0 + 2 * np;
+            const bool in0 = row < r_end, in1 = row + 1 < r_end;
+            uint32_t w0 = 0u, w1 = 0u;
+            if (kw < d_in) {
+                if (in0) w0 = __ldg(bits + row * stride + wd);
+                if (in1) w1 = __ldg(bits + (row + 1) * stride + wd);
+            }
+#pragma unroll
+            for (int b = 0; b < 8; ++b) {
+                const int kb = part8 * 8 + b, k = kw + kb;
+                const bool kin = k < d_in;
+                const uint32_t lo = (kin && in0) ? (((w0 >> kb) & 1u) ? 0x3F80u : 0xBF80u) : 0u;
+                const uint32_t hi = (kin && in1) ? (((w1 >> kb) & 1u) ? 0x3F80u : 0xBF80u) : 0u;
+                const uint32_t off = tc::canon_off(N, k, (2 * np) >> 3) + ((2 * np) & 7) * 2;
+                *reinterpret_cast<uint32_t*>(Bs + off) = lo | (hi << 16);
+            }
+        }
+        tc::fence_async_smem();
+        tc::fence_before_sync();
+        __syncthreads();
+        tc::fence_after_sync();
+        if (threadIdx.x == 0) {
+            const uint32_t a_base = tc::smem_u32(As), b_base = tc::smem_u32(Bs);
+            for (int ks = 0; ks < kKc / 16; ++ks) {
+                const uint64_t bd = tc::make_desc(b_base + 2 * ks * b_lbo, b_lbo, sbo);
+#pragma unroll
+                for (int sp = 0; sp < 3; ++sp) {
+                    const uint64_t ad = tc::make_desc(a_base + sp * kRows * 128 + 2 * ks * a_lbo, a_lbo, sbo);
+                    const uint32_t accum = (any || ks > 0 || sp > 0) ? 1u : 0u;
+                    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+                                 ::"r"(tmem_base), "l"(ad), "l"(bd), "r"(idesc), "r"(accum) : "memory");
+                }
+            }
+            tc::commit_to(&bar);
+        }
+        any = true;
+        if (!tc::wait_barrier(&bar, phase)) {
+            atomicExch(&g_bw_tc_timeout, 1);
+            ok = false;
+        }
+        phase ^= 1u;
+        tc::fence_after_sync();
+        if (__syncthreads_or(!ok)) { ok = false; break; }   // the operands may be overwritten; leave together on a timeout
+    }
+    // ---- the slab: thread = channel j (tensor-memory lane), its warp's half of the inputs k
+    if (ok) {
+        float* slab = part + (int64_t)blockIdx.y * d_in * d_out;
+        const int lane_base = 32 * (warp & 3);
+        const int j = j0 + lane_base + lane;
+        const int c_begin = (warp >> 2) * (N / 2);
+        for (int c0 = c_begin; c0 < c_begin + N / 2; c0 += 16) {
+            uint32_t v[16];
+            if (any) tc::tmem_ld16(tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)c0, v);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+                const int k = c0 + e;
+                if (j < d_out && k < d_in) slab[(int64_t)k * d_out + j] = any ? __uint_as_float(v[e]) : 0.f;
+            }
+        }
+    }
+    tc::fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tc::tmem_free(tmem_base, kCols);
+}
+
+template <int N>
+cudaError_t launch_grad_wt_tc(cudaStream_t s, const uint32_t* bits, int64_t stride, const float* beta, const float* gz,
+                              int64_t ldz, int64_t n, int d_in, int d_out, int n_splits, int64_t rows_per_split, float* part)
+{
+    const size_t smem = 3 * 128 * 128 + (size_t)N * 128;
+    cudaError_t e = cudaFuncSetAttribute(grad_wt_tc_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const dim3 grid((unsigned)ceil_div(d_out, 128), (unsigned)n_splits);
+    grad_wt_tc_kernel<N><<<grid, kBwThreads, smem, s>>>(bits, stride, beta, gz, ldz, n, d_in, d_out, rows_per_split, part);
+    return cudaGetLastError();
+}
+
 template <int N>
 cudaError_t launch_grad_h_tc(cudaStream_t s, const float* gz, int64_t ldz, const float* alpha, const float* W, int64_t ldw,
                              int64_t n, int d_in, int d_out, float* g_h, int64_t ldh)
@@ -586,11 +735,18 @@ cudaError_t launch_layer_backward(cudaStream_t s, int64_t n, const int64_t* rowp
 
     // step 1b: G_W~ = H~^T G_zeta, split over the rows, slabs added in a fixed order
     {
-        const int64_t rows_per_split = ceil_div(ceil_div(n, n_splits), kMmaK) * kMmaK;
-        const dim3 grid((unsigned)ceil_div(d_out, kMmaTile), (unsigned)ceil_div(d_in, kMmaTile), (unsigned)n_splits);
-        grad_wt_mma_kernel<<<grid, kBwThreads, 0, s>>>(in_bits, stride_in, in_beta, gz, ldz, n, d_in, d_out, rows_per_split, part);
+        const int64_t rows_per_split = ceil_div(ceil_div(n, n_splits), 64) * 64;
         ++*launches;
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        if (d_in <= 256) {                                  // tcgen05 version: one tile covers all inputs
+            if (d_in <= 64) e = launch_grad_wt_tc<64>(s, in_bits, stride_in, in_beta, gz, ldz, n, d_in, d_out, n_splits, rows_per_split, part);
+            else if (d_in <= 128) e = launch_grad_wt_tc<128>(s, in_bits, stride_in, in_beta, gz, ldz, n, d_in, d_out, n_splits, rows_per_split, part);
+            else e = launch_grad_wt_tc<256>(s, in_bits, stride_in, in_beta, gz, ldz, n, d_in, d_out, n_splits, rows_per_split, part);
+            if (e != cudaSuccess) return e;
+        } else {
+            const dim3 grid((unsigned)ceil_div(d_out, kMmaTile), (unsigned)ceil_div(d_in, kMmaTile), (unsigned)n_splits);
+            grad_wt_mma_kernel<<<grid, kBwThreads, 0, s>>>(in_bits, stride_in, in_beta, gz, ldz, n, d_in, d_out, rows_per_split, part);
+            if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        }
         const int64_t elems = (int64_t)d_in * d_out;
         grad_wt_reduce_kernel<<<(unsigned)ceil_div(elems, 256), 256, 0, s>>>(part, n_splits, elems, g_wt);
         ++*launches;
