@@ -164,12 +164,12 @@ __device__ __forceinline__ void finish_row(const SpmmDev& p, const float* ctab, 
 {
     constexpr int EPV = Elt<T>::kPerVec;
     constexpr int LW = 32 / EPV;                  // lanes that share one packed word
-    constexpr int kCols = (LPR < 32 ? LPR : NCH * 32) * EPV;
+    constexpr int kCols = NCH * (LPR < 32 ? LPR : 32) * EPV;
     const int g = lane / LPR, l = lane % LPR;
     float l1 = 0.f;
 #pragma unroll
     for (int c = 0; c < NCH; ++c) {
-        const int vec = c * 32 + l;
+        const int vec = c * (LPR < 32 ? LPR : 32) + l;
         const int col0 = vec * EPV;
         float x[EPV], sh[EPV], sc[EPV];
 #pragma unroll
@@ -594,27 +594,29 @@ __device__ __forceinline__ void fma_any(float w, const uint4& v, float (&acc)[El
     else fma_vec<T>(w, v, acc);
 }
 
-// The row-aligned stream for rows of 8 or 16 vectors (128- and 256-byte rows): a position holds G = 4
-// or 2 stored entries, one per group of LPR = 32 / G lanes (lane = LPR g + l fetches and accumulates
-// vector l of entry G b + g of position b), so the per-position bookkeeping is shared by G entries.
+// The row-aligned stream for rows of up to NV * LPR vectors: a position holds G = 32 / LPR stored entries,
+// one per group of LPR lanes (lane = LPR g + l fetches and accumulates vectors l, LPR + l, .. (NV of them)
+// of entry G b + g of position b), so the per-position bookkeeping is shared by G entries.
 // A group is 4 positions = 4 G entries and never straddles a row (a row takes ceil(deg / 4G) groups,
 // at least one), which pays when rows are long compared with a group; the launcher picks the general
 // stream otherwise.  The lane groups' sums are added when a row completes.  Cursors, metadata chunks
 // and the weight ring are those of stream_rows_wide; the weights of a group are stored lane group by
 // lane group (index 4 g + b) so that a lane reads its four with one 16-byte load.  kFull: the row has
 // exactly LPR vectors, no lane needs masking.
-template <typename T, int G, bool kFull, bool kPartial>
+template <typename T, int G, int NV, bool kFull, bool kPartial>
 __device__ __forceinline__ void stream_rows_multi(const SpmmDev& p, uint4* ring, float* wfifo, const float* ctab, int lane,
                                                   int64_t e0, int n_ent, int64_t warp_row0, int row_lo,
-                                                  int row_hi, int rp_rel, float (&acc)[1][Elt<T>::kPerVec])
+                                                  int row_hi, int rp_rel, float (&acc)[NV][Elt<T>::kPerVec])
 {
     constexpr int LPR = kWarp / G;
     constexpr int EPV = Elt<T>::kPerVec;
-    using P = Pipe<1, LPR, true>;
+    using P = Pipe<NV, LPR, true>;
     constexpr int PB = P::PB, NG = P::NG, EG = G * PB;        // positions and entries per group
     static_assert(PB == 4 && (NG & (NG - 1)) == 0, "float4 weight reads; power-of-two group ring");
     const int g = lane / LPR, l = lane % LPR;
-    const bool active = l < p.nv;
+    bool active[NV];
+#pragma unroll
+    for (int c = 0; c < NV; ++c) active[c] = (c * LPR + l) < p.nv;
     const int32_t* cols = p.colidx + e0;
     const float* vals = p.val + e0;
     auto load_col = [&](int e) { return e < n_ent ? __ldg(cols + e) : 0; };
@@ -637,7 +639,7 @@ __device__ __forceinline__ void stream_rows_multi(const SpmmDev& p, uint4* ring,
     int re = 0, rr = row_lo, rend = iend;                     // retire cursor
     bool more = row_lo < row_hi;
     int issued = 0, goff = 0;                                 // groups issued; ring position of the current group
-    zero_acc<1, EPV>(acc);
+    zero_acc<NV, EPV>(acc);
 
     for (int it = 0;; ++it) {
         if (it >= NG) {
@@ -645,29 +647,37 @@ __device__ __forceinline__ void stream_rows_multi(const SpmmDev& p, uint4* ring,
             // ---- retire the oldest group
             cp_async_wait<NG - 1>();
             __syncwarp();
-            const uint4* gp = ring_l + goff * (PB * 32);
-            uint4 v[PB];
+            const uint4* gp = ring_l + goff * (PB * 32 * NV);
+            uint4 v[PB][NV];
 #pragma unroll
-            for (int b = 0; b < PB; ++b) v[b] = gp[b * 32];
+            for (int b = 0; b < PB; ++b)
+#pragma unroll
+                for (int c = 0; c < NV; ++c) v[b][c] = gp[(b * NV + c) * 32];
             const float4 w4 = *reinterpret_cast<const float4*>(wfifo + goff * EG + 4 * g);
             const float w[PB] = {w4.x, w4.y, w4.z, w4.w};
             const int left = rend - re;
             if (left >= EG) {
 #pragma unroll
                 for (int b = 0; b < PB; ++b)
-                    if (kFull || active) fma_any<T>(w[b], v[b], acc[0]);
+#pragma unroll
+                    for (int c = 0; c < NV; ++c)
+                        if (kFull || active[c]) fma_any<T>(w[b], v[b][c], acc[c]);
                 re += EG;
             } else {
 #pragma unroll
                 for (int b = 0; b < PB; ++b)
-                    if (G * b + g < left && (kFull || active)) fma_any<T>(w[b], v[b], acc[0]);
+                    if (G * b + g < left) {
+#pragma unroll
+                        for (int c = 0; c < NV; ++c)
+                            if (kFull || active[c]) fma_any<T>(w[b], v[b][c], acc[c]);
+                    }
                 re = rend;
             }
             if (re == rend) {                                 // the row is complete
-                reduce_groups<1, EPV, LPR>(acc);
+                reduce_groups<NV, EPV, LPR>(acc);
                 if (kPartial) return;
-                finish_row<T, 1, LPR>(p, ctab, warp_row0 + rr, lane, acc);
-                zero_acc<1, EPV>(acc);
+                finish_row<T, NV, LPR>(p, ctab, warp_row0 + rr, lane, acc);
+                zero_acc<NV, EPV>(acc);
                 ++rr;
                 if (rr < row_hi) rend = row_end_of(rr);
             }
@@ -677,7 +687,7 @@ __device__ __forceinline__ void stream_rows_multi(const SpmmDev& p, uint4* ring,
             // ---- issue the next group of the row under the issue cursor
             const int left = iend - ie;
             const int base = ie - cbase;                      // position of the group in chunk A (< 32)
-            const uint32_t dsta = ring_sa + goff * (PB * 512);
+            const uint32_t dsta = ring_sa + goff * (PB * 512 * NV);
             // the window of the next 32 entries: lanes below `base` present their chunk-B entry, so
             // entry base + e sits in lane (base + e) % 32
             const int m_col = lane >= base ? a_col : b_col;
@@ -689,13 +699,21 @@ __device__ __forceinline__ void stream_rows_multi(const SpmmDev& p, uint4* ring,
 #pragma unroll
                 for (int b = 0; b < PB; ++b) {
                     const uint32_t k = (uint32_t)__shfl_sync(0xffffffffu, m_col, src_lane + G * b);
-                    if (kFull || active) cp_async16_s(dsta + b * 512, zeta_l + (uint64_t)k * row_bytes);
+                    const char* src = zeta_l + (uint64_t)k * row_bytes;
+#pragma unroll
+                    for (int c = 0; c < NV; ++c)
+                        if (kFull || active[c]) cp_async16_s(dsta + (b * NV + c) * 512, src + c * (LPR * 16));
                 }
             } else {
 #pragma unroll
                 for (int b = 0; b < PB; ++b) {
                     const uint32_t k = (uint32_t)__shfl_sync(0xffffffffu, m_col, src_lane + G * b);
-                    if (G * b + g < cnt && (kFull || active)) cp_async16_s(dsta + b * 512, zeta_l + (uint64_t)k * row_bytes);
+                    const char* src = zeta_l + (uint64_t)k * row_bytes;
+                    if (G * b + g < cnt) {
+#pragma unroll
+                        for (int c = 0; c < NV; ++c)
+                            if (kFull || active[c]) cp_async16_s(dsta + (b * NV + c) * 512, src + c * (LPR * 16));
+                    }
                 }
             }
             if (rel < cnt) wfifo[goff * EG + 4 * (rel % G) + rel / G] = m_w;
@@ -737,11 +755,11 @@ template <typename T, int NCH, int LPR, bool kFull, bool kAligned>
 __global__ void __launch_bounds__(kSpmmThreads, spmm_blocks_per_sm<NCH, LPR, kAligned>())
 spmm_kernel(const SpmmDev p, int rows_per_warp)
 {
-    static_assert(!kAligned || (NCH == 1 && (LPR == 8 || LPR == 16)), "the multi-entry stream covers rows of 8 or 16 vectors");
+    static_assert(!kAligned || ((NCH == 1 || NCH == 2) && (LPR == 8 || LPR == 16)), "the multi-entry stream: 8 or 16 lanes per row, one or two vectors per lane");
     using P = Pipe<NCH, LPR, kAligned>;
     constexpr int EPV = Elt<T>::kPerVec;
     constexpr int G = P::G;
-    constexpr int kCols = (LPR < 32 ? LPR : NCH * 32) * EPV;  // accumulator columns of one warp
+    constexpr int kCols = NCH * (LPR < 32 ? LPR : 32) * EPV;  // accumulator columns of one warp
     extern __shared__ __align__(128) unsigned char dsmem[];
     __shared__ int64_t long_rows[kLongQueue];
     __shared__ int n_long;
@@ -785,7 +803,7 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
                     stream_rows_wide<T, NCH, kFull, false>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
                                                     (int)(rp_reg - e0), acc);
                 else if constexpr (kAligned)
-                    stream_rows_multi<T, kWarp / LPR, kFull, false>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
+                    stream_rows_multi<T, kWarp / LPR, NCH, kFull, false>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
                                                                     (int)(rp_reg - e0), acc);
                 else
                     stream_entries<T, NCH, LPR, false>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
@@ -805,7 +823,7 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
         if constexpr (LPR == 32)
             stream_rows_wide<T, NCH, kFull, true>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
         else if constexpr (kAligned)
-            stream_rows_multi<T, kWarp / LPR, kFull, true>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
+            stream_rows_multi<T, kWarp / LPR, NCH, kFull, true>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
         else
             stream_entries<T, NCH, LPR, true>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
         __syncthreads();                                      // every ring is idle: reuse them for the partial sums
@@ -814,7 +832,7 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
 #pragma unroll
             for (int c = 0; c < NCH; ++c)
 #pragma unroll
-                for (int i = 0; i < EPV; ++i) part[warp * kCols + (c * 32 + l) * EPV + i] = acc[c][i];
+                for (int i = 0; i < EPV; ++i) part[warp * kCols + (c * (LPR < 32 ? LPR : 32) + l) * EPV + i] = acc[c][i];
         }
         __syncthreads();
         if (warp == 0) {
@@ -823,7 +841,7 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
 #pragma unroll
                 for (int i = 0; i < EPV; ++i) {
                     float t = 0.f;
-                    for (int w = 0; w < kSpmmWarps; ++w) t += part[w * kCols + (c * 32 + l) * EPV + i];
+                    for (int w = 0; w < kSpmmWarps; ++w) t += part[w * kCols + (c * (LPR < 32 ? LPR : 32) + l) * EPV + i];
                     acc[c][i] = t;
                 }
             finish_row<T, NCH, LPR>(p, ctab, lrow, lane, acc);
@@ -835,7 +853,7 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
 template <typename T, int NCH, int LPR, bool kFull = false, bool kAligned = false>
 cudaError_t launch_one(cudaStream_t s, const SpmmDev& p)
 {
-    constexpr int kCols = (LPR < 32 ? LPR : NCH * 32) * Elt<T>::kPerVec;
+    constexpr int kCols = NCH * (LPR < 32 ? LPR : 32) * Elt<T>::kPerVec;
     constexpr size_t smem = kSpmmWarps * Pipe<NCH, LPR, kAligned>::kWarpBytes + 3 * kCols * sizeof(float);   // rings, weights, column table
     // enough thread blocks to fill the machine on small graphs, long runs of rows on large ones
     const int rows_per_warp = (int)std::min<int64_t>(kMaxRowsPerWarp, std::max<int64_t>(1, p.n / (kSpmmWarps * 148 * 8)));
@@ -867,6 +885,8 @@ cudaError_t dispatch(cudaStream_t s, const SpmmDev& p, double mean_row)
     if (nv <= 8) return launch_one<T, 1, 8>(s, p);
     if (nv <= 16) {
         if constexpr (sizeof(T) == 1) {
+            // (8 lanes per row with two vectors each, four entries per position -- launch_one<T, 2, 8, .., true> -- halves
+            // the bookkeeping per entry again but needs 123 registers: 7.7 ms against 6.4 ms on c5 layer 0; not used)
             if (!(mean_row > 0.0 && mean_row < 8.0))
                 return nv == 16 ? launch_one<T, 1, 16, true, true>(s, p) : launch_one<T, 1, 16, false, true>(s, p);
         }
