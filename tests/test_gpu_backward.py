@@ -70,7 +70,8 @@ def run_case(B, ctx, n, m, d_in, d_out, seed, g_scale=0.05, want_g_in=True, w_sc
 
 
 @pytest.mark.parametrize("n,m,d_in,d_out", [(1, 0, 1, 1), (23, 60, 11, 7), (300, 2000, 100, 256), (500, 3000, 256, 47),
-                                            (1000, 6000, 64, 64), (777, 5000, 130, 200), (2000, 30000, 256, 256)])
+                                            (1000, 6000, 64, 64), (777, 5000, 130, 200), (2000, 30000, 256, 256),
+                                            (400, 3000, 300, 40), (129, 700, 128, 130), (20000, 100000, 256, 256)])   # d_in > 256: the mma.sync kernels; several chunks and tiles per CTA
 def test_backward_matches_oracle(B, ctx, n, m, d_in, d_out):
     run_case(B, ctx, n, m, d_in, d_out, seed=n + d_in)
 
