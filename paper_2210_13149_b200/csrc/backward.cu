@@ -333,49 +333,83 @@ grad_h_tc_kernel(const float* __restrict__ gz, int64_t ldz, const float* __restr
         const int64_t i0 = tile * kRows;
         for (int ch = 0; ch < n_chunks; ++ch) {
             const int j0 = ch * kKc;
-            // A: 128 rows x 16 quads of channels -> three bf16 terms of G_zeta * alpha
-            for (int t = threadIdx.x; t < kRows * (kKc / 4); t += kBwThreads) {
-                const int jq = (t & 15) * 4, r = t >> 4;
-                const int j = j0 + jq;
-                const int64_t row = i0 + r;
-                float x[4] = {0.f, 0.f, 0.f, 0.f};
-                if (row < n) {
-                    if (j + 3 < d_out && vec_ok) {
-                        const float4 v = __ldg(reinterpret_cast<const float4*>(gz + row * ldz + j));
-                        x[0] = v.x, x[1] = v.y, x[2] = v.z, x[3] = v.w;
-                    } else {
+            // A: 128 rows x 16 quads of channels -> three bf16 terms of G_zeta * alpha.  All of a thread's loads are
+            // issued before the first is used (8 independent 16-byte loads in flight per thread).
+            {
+                constexpr int kItems = kRows * (kKc / 4) / kBwThreads;
+                float4 xv[kItems], av[kItems];
 #pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            if (j + u < d_out) x[u] = __ldg(gz + row * ldz + j + u);
+                for (int it = 0; it < kItems; ++it) {
+                    const int t = threadIdx.x + it * kBwThreads;
+                    const int jq = (t & 15) * 4, r = t >> 4;
+                    const int j = j0 + jq;
+                    const int64_t row = i0 + r;
+                    xv[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    av[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (row < n) {
+                        if (j + 3 < d_out && vec_ok) {
+                            xv[it] = __ldg(reinterpret_cast<const float4*>(gz + row * ldz + j));
+                        } else {
+                            if (j < d_out) xv[it].x = __ldg(gz + row * ldz + j);
+                            if (j + 1 < d_out) xv[it].y = __ldg(gz + row * ldz + j + 1);
+                            if (j + 2 < d_out) xv[it].z = __ldg(gz + row * ldz + j + 2);
+                            if (j + 3 < d_out) xv[it].w = __ldg(gz + row * ldz + j + 3);
+                        }
                     }
+                    if (j < d_out) av[it].x = __ldg(alpha + j);
+                    if (j + 1 < d_out) av[it].y = __ldg(alpha + j + 1);
+                    if (j + 2 < d_out) av[it].z = __ldg(alpha + j + 2);
+                    if (j + 3 < d_out) av[it].w = __ldg(alpha + j + 3);
                 }
-                unsigned short hi[4], mid[4], lo[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) split3(j + u < d_out ? __fmul_rn(x[u], __ldg(alpha + j + u)) : 0.f, hi[u], mid[u], lo[u]);
-                auto pack = [](const unsigned short (&h)[4]) { return make_uint2((uint32_t)h[0] | ((uint32_t)h[1] << 16), (uint32_t)h[2] | ((uint32_t)h[3] << 16)); };
-                const uint32_t off = tc::canon_off(kRows, r, jq >> 3) + (jq & 7) * 2;
-                *reinterpret_cast<uint2*>(As + 0 * kRows * 128 + off) = pack(hi);
-                *reinterpret_cast<uint2*>(As + 1 * kRows * 128 + off) = pack(mid);
-                *reinterpret_cast<uint2*>(As + 2 * kRows * 128 + off) = pack(lo);
+                for (int it = 0; it < kItems; ++it) {
+                    const int t = threadIdx.x + it * kBwThreads;
+                    const int jq = (t & 15) * 4, r = t >> 4;
+                    const float x[4] = {__fmul_rn(xv[it].x, av[it].x), __fmul_rn(xv[it].y, av[it].y), __fmul_rn(xv[it].z, av[it].z), __fmul_rn(xv[it].w, av[it].w)};
+                    unsigned short hi[4], mid[4], lo[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) split3(x[u], hi[u], mid[u], lo[u]);
+                    auto pack = [](const unsigned short (&h)[4]) { return make_uint2((uint32_t)h[0] | ((uint32_t)h[1] << 16), (uint32_t)h[2] | ((uint32_t)h[3] << 16)); };
+                    const uint32_t off = tc::canon_off(kRows, r, jq >> 3) + (jq & 7) * 2;
+                    *reinterpret_cast<uint2*>(As + 0 * kRows * 128 + off) = pack(hi);
+                    *reinterpret_cast<uint2*>(As + 1 * kRows * 128 + off) = pack(mid);
+                    *reinterpret_cast<uint2*>(As + 2 * kRows * 128 + off) = pack(lo);
+                }
             }
-            // B: N inputs x 16 quads of channels -> sign of W as +-1
-            for (int t = threadIdx.x; t < N * (kKc / 4); t += kBwThreads) {
-                const int jq = (t & 15) * 4, k = t >> 4;
-                const int j = j0 + jq;
-                unsigned short sg[4] = {0, 0, 0, 0};
-                if (k < d_in) {
-                    if (j + 3 < d_out && w_vec_ok) {
-                        const float4 v = __ldg(reinterpret_cast<const float4*>(W + (int64_t)k * ldw + j));
-                        sg[0] = v.x >= 0.f ? 0x3F80 : 0xBF80, sg[1] = v.y >= 0.f ? 0x3F80 : 0xBF80;
-                        sg[2] = v.z >= 0.f ? 0x3F80 : 0xBF80, sg[3] = v.w >= 0.f ? 0x3F80 : 0xBF80;
-                    } else {
+            // B: N inputs x 16 quads of channels -> sign of W as +-1 (loads batched in the same way)
+            {
+                constexpr int kItems = N * (kKc / 4) / kBwThreads;
+                float4 wv[kItems];
 #pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            if (j + u < d_out) sg[u] = __ldg(W + (int64_t)k * ldw + j + u) >= 0.f ? 0x3F80 : 0xBF80;
+                for (int it = 0; it < kItems; ++it) {
+                    const int t = threadIdx.x + it * kBwThreads;
+                    const int jq = (t & 15) * 4, k = t >> 4;
+                    const int j = j0 + jq;
+                    wv[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (k < d_in) {
+                        if (j + 3 < d_out && w_vec_ok) {
+                            wv[it] = __ldg(reinterpret_cast<const float4*>(W + (int64_t)k * ldw + j));
+                        } else {
+                            if (j < d_out) wv[it].x = __ldg(W + (int64_t)k * ldw + j);
+                            if (j + 1 < d_out) wv[it].y = __ldg(W + (int64_t)k * ldw + j + 1);
+                            if (j + 2 < d_out) wv[it].z = __ldg(W + (int64_t)k * ldw + j + 2);
+                            if (j + 3 < d_out) wv[it].w = __ldg(W + (int64_t)k * ldw + j + 3);
+                        }
                     }
                 }
-                const uint32_t off = tc::canon_off(N, k, jq >> 3) + (jq & 7) * 2;
-                *reinterpret_cast<uint2*>(Bs + off) = make_uint2((uint32_t)sg[0] | ((uint32_t)sg[1] << 16), (uint32_t)sg[2] | ((uint32_t)sg[3] << 16));
+#pragma unroll
+                for (int it = 0; it < kItems; ++it) {
+                    const int t = threadIdx.x + it * kBwThreads;
+                    const int jq = (t & 15) * 4, k = t >> 4;
+                    const int j = j0 + jq;
+                    const bool kin = k < d_in;
+                    const float w[4] = {wv[it].x, wv[it].y, wv[it].z, wv[it].w};
+                    uint32_t sg[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) sg[u] = (kin && j + u < d_out) ? (w[u] >= 0.f ? 0x3F80u : 0xBF80u) : 0u;
+                    const uint32_t off = tc::canon_off(N, k, jq >> 3) + (jq & 7) * 2;
+                    *reinterpret_cast<uint2*>(Bs + off) = make_uint2(sg[0] | (sg[1] << 16), sg[2] | (sg[3] << 16));
+                }
             }
             tc::fence_async_smem();
             tc::fence_before_sync();
@@ -482,58 +516,83 @@ grad_wt_tc_kernel(const uint32_t* __restrict__ bits, int64_t stride, const float
     uint32_t phase = 0;
     bool ok = true, any = false;
     for (int64_t r0 = r_begin; r0 < r_end; r0 += kKc) {
-        // A: 32 node pairs x 32 quads of channels
-        for (int t = threadIdx.x; t < 32 * 32; t += kBwThreads) {
-            const int np = t & 31, jq = (t >> 5) * 4;
-            float x[2][4];
+        // A: 32 node pairs x 32 quads of channels; all of a thread's loads are issued before the first is used
+        {
+            constexpr int kItems = 32 * 32 / kBwThreads;
+            float4 xv[kItems][2];
+            float bv[kItems][2];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int64_t row = r0 + 2 * np + h;
+            for (int it = 0; it < kItems; ++it) {
+                const int t = threadIdx.x + it * kBwThreads;
+                const int np = t & 31, jq = (t >> 5) * 4;
                 const int j = j0 + jq;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) x[h][u] = 0.f;
-                if (row < r_end) {
-                    const float be = __ldg(beta + row);
-                    if (j + 3 < d_out && vec_ok) {
-                        const float4 v = __ldg(reinterpret_cast<const float4*>(gz + row * ldz + j));
-                        x[h][0] = v.x * be, x[h][1] = v.y * be, x[h][2] = v.z * be, x[h][3] = v.w * be;
-                    } else {
-#pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            if (j + u < d_out) x[h][u] = __ldg(gz + row * ldz + j + u) * be;
+                for (int h = 0; h < 2; ++h) {
+                    const int64_t row = r0 + 2 * np + h;
+                    xv[it][h] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    bv[it][h] = 0.f;
+                    if (row < r_end) {
+                        bv[it][h] = __ldg(beta + row);
+                        if (j + 3 < d_out && vec_ok) {
+                            xv[it][h] = __ldg(reinterpret_cast<const float4*>(gz + row * ldz + j));
+                        } else {
+                            if (j < d_out) xv[it][h].x = __ldg(gz + row * ldz + j);
+                            if (j + 1 < d_out) xv[it][h].y = __ldg(gz + row * ldz + j + 1);
+                            if (j + 2 < d_out) xv[it][h].z = __ldg(gz + row * ldz + j + 2);
+                            if (j + 3 < d_out) xv[it][h].w = __ldg(gz + row * ldz + j + 3);
+                        }
                     }
                 }
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                unsigned short h0, m0, l0, h1, m1, l1;
-                split3(x[0][u], h0, m0, l0);
-                split3(x[1][u], h1, m1, l1);
-                const uint32_t off = tc::canon_off(kRows, jq + u, (2 * np) >> 3) + ((2 * np) & 7) * 2;
-                *reinterpret_cast<uint32_t*>(As + 0 * kRows * 128 + off) = (uint32_t)h0 | ((uint32_t)h1 << 16);
-                *reinterpret_cast<uint32_t*>(As + 1 * kRows * 128 + off) = (uint32_t)m0 | ((uint32_t)m1 << 16);
-                *reinterpret_cast<uint32_t*>(As + 2 * kRows * 128 + off) = (uint32_t)l0 | ((uint32_t)l1 << 16);
+            for (int it = 0; it < kItems; ++it) {
+                const int t = threadIdx.x + it * kBwThreads;
+                const int np = t & 31, jq = (t >> 5) * 4;
+                const float x0[4] = {xv[it][0].x * bv[it][0], xv[it][0].y * bv[it][0], xv[it][0].z * bv[it][0], xv[it][0].w * bv[it][0]};
+                const float x1[4] = {xv[it][1].x * bv[it][1], xv[it][1].y * bv[it][1], xv[it][1].z * bv[it][1], xv[it][1].w * bv[it][1]};
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    unsigned short h0, m0, l0, h1, m1, l1;
+                    split3(x0[u], h0, m0, l0);
+                    split3(x1[u], h1, m1, l1);
+                    const uint32_t off = tc::canon_off(kRows, jq + u, (2 * np) >> 3) + ((2 * np) & 7) * 2;
+                    *reinterpret_cast<uint32_t*>(As + 0 * kRows * 128 + off) = (uint32_t)h0 | ((uint32_t)h1 << 16);
+                    *reinterpret_cast<uint32_t*>(As + 1 * kRows * 128 + off) = (uint32_t)m0 | ((uint32_t)m1 << 16);
+                    *reinterpret_cast<uint32_t*>(As + 2 * kRows * 128 + off) = (uint32_t)l0 | ((uint32_t)l1 << 16);
+                }
             }
         }
-        // B: 32 node pairs x (N / 32) packed words x 4 groups of 8 inputs
-        for (int t = threadIdx.x; t < 32 * (N / 32) * 4; t += kBwThreads) {
-            const int np = t & 31, wd = (t >> 5) >> 2, part8 = (t >> 5) & 3;
-            const int kw = wd * 32;                         // first input of the word
-            const int64_t row = r0 + 2 * np;
-            const bool in0 = row < r_end, in1 = row + 1 < r_end;
-            uint32_t w0 = 0u, w1 = 0u;
-            if (kw < d_in) {
-                if (in0) w0 = __ldg(bits + row * stride + wd);
-                if (in1) w1 = __ldg(bits + (row + 1) * stride + wd);
+        // B: 32 node pairs x (N / 32) packed words x 4 groups of 8 inputs (loads batched in the same way)
+        {
+            constexpr int kItems = 32 * (N / 32) * 4 / kBwThreads;
+            uint32_t w0v[kItems], w1v[kItems];
+#pragma unroll
+            for (int it = 0; it < kItems; ++it) {
+                const int t = threadIdx.x + it * kBwThreads;
+                const int np = t & 31, wd = (t >> 5) >> 2;
+                const int64_t row = r0 + 2 * np;
+                w0v[it] = 0u, w1v[it] = 0u;
+                if (wd * 32 < d_in) {
+                    if (row < r_end) w0v[it] = __ldg(bits + row * stride + wd);
+                    if (row + 1 < r_end) w1v[it] = __ldg(bits + (row + 1) * stride + wd);
+                }
             }
 #pragma unroll
-            for (int b = 0; b < 8; ++b) {
-                const int kb = part8 * 8 + b, k = kw + kb;
-                const bool kin = k < d_in;
-                const uint32_t lo = (kin && in0) ? (((w0 >> kb) & 1u) ? 0x3F80u : 0xBF80u) : 0u;
-                const uint32_t hi = (kin && in1) ? (((w1 >> kb) & 1u) ? 0x3F80u : 0xBF80u) : 0u;
-                const uint32_t off = tc::canon_off(N, k, (2 * np) >> 3) + ((2 * np) & 7) * 2;
-                *reinterpret_cast<uint32_t*>(Bs + off) = lo | (hi << 16);
+            for (int it = 0; it < kItems; ++it) {
+                const int t = threadIdx.x + it * kBwThreads;
+                const int np = t & 31, wd = (t >> 5) >> 2, part8 = (t >> 5) & 3;
+                const int kw = wd * 32;
+                const int64_t row = r0 + 2 * np;
+                const bool in0 = row < r_end, in1 = row + 1 < r_end;
+#pragma unroll
+                for (int b = 0; b < 8; ++b) {
+                    const int kb = part8 * 8 + b, k = kw + kb;
+                    const bool kin = k < d_in;
+                    const uint32_t lo = (kin && in0) ? (((w0v[it] >> kb) & 1u) ? 0x3F80u : 0xBF80u) : 0u;
+                    const uint32_t hi = (kin && in1) ? (((w1v[it] >> kb) & 1u) ? 0x3F80u : 0xBF80u) : 0u;
+                    const uint32_t off = tc::canon_off(N, k, (2 * np) >> 3) + ((2 * np) & 7) * 2;
+                    *reinterpret_cast<uint32_t*>(Bs + off) = lo | (hi << 16);
+                }
             }
         }
         tc::fence_async_smem();
