@@ -4,7 +4,8 @@
  * The library implements the forward path of "Binary Graph Convolutional Network with Capacity
  * Exploration" (Bi-GCN): feature / weight binarization with bit packing (Sec. 4.2.1, 4.2.2), the
  * XNOR + bit-count contraction with its beta_i alpha_j rescale (Sec. 4.2.3, Eq. "cdot-op" and
- * "bi-op"), and the floating-point aggregation with A_tilde = D_hat^-1/2 (A + I) D_hat^-1/2
+ * "bi-op"; computed as int8 tensor-core products on the bits expanded to +1 / -1 where the layer is
+ * narrow enough, see BIGCN_OPT_CONTRACTION: the same integers), and the floating-point aggregation with A_tilde = D_hat^-1/2 (A + I) D_hat^-1/2
  * (Eq. 1; last equation of Sec. 4.2.3), whose output can be re-binarized for the next layer.
  *
  * General rules
@@ -176,7 +177,7 @@ typedef struct {
     int32_t launches;
     float ms_total;
     float ms_pack;                       /* binarize + pack of X */
-    float ms_gemm[BIGCN_MAX_LAYERS];     /* XNOR/bit-count contraction + rescale */
+    float ms_gemm[BIGCN_MAX_LAYERS];     /* binary contraction + rescale */
     float ms_spmm[BIGCN_MAX_LAYERS];     /* aggregation (+ re-binarization) */
 } bigcn_stats;
 
