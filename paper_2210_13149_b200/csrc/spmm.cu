@@ -234,8 +234,9 @@ __device__ __forceinline__ void finish_row(const SpmmDev& p, const float* ctab, 
 template <int NCH, int LPR, bool kAligned = false>
 struct Pipe {
     static constexpr int G = kWarp / LPR;                       // entries per position
-    static constexpr int PB = (4 * G <= 32) ? 4 : 32 / G;       // positions per group (PB * G divides 32)
-    static constexpr int NG = NCH > 1 ? 2 : ((LPR == 32 || kAligned) ? 4 : 3);  // groups in flight per warp (a power of two for the row-aligned streams)
+    // positions per group (PB * G divides 32); the aligned stream with two entries per position takes 8
+    static constexpr int PB = (kAligned && G == 2 && NCH == 1) ? 8 : ((4 * G <= 32) ? 4 : 32 / G);
+    static constexpr int NG = (NCH > 1 || PB == 8) ? 2 : ((LPR == 32 || kAligned) ? 4 : 3);  // groups in flight per warp (a power of two for the row-aligned streams)
     static constexpr int RING = PB * NG;                        // slots of NCH * 512 bytes
     static constexpr size_t kWarpBytes = (size_t)RING * (NCH * 512 + G * 4);
 };
@@ -601,7 +602,7 @@ __device__ __forceinline__ void fma_any(float w, const uint4& v, float (&acc)[El
 // at least one), which pays when rows are long compared with a group; the launcher picks the general
 // stream otherwise.  The lane groups' sums are added when a row completes.  Cursors, metadata chunks
 // and the weight ring are those of stream_rows_wide; the weights of a group are stored lane group by
-// lane group (index 4 g + b) so that a lane reads its four with one 16-byte load.  kFull: the row has
+// lane group (index PB g + b) so that a lane reads four of them with one 16-byte load.  kFull: the row has
 // exactly LPR vectors, no lane needs masking.
 template <typename T, int G, int NV, bool kFull, bool kPartial>
 __device__ __forceinline__ void stream_rows_multi(const SpmmDev& p, uint4* ring, float* wfifo, const float* ctab, int lane,
@@ -612,7 +613,7 @@ __device__ __forceinline__ void stream_rows_multi(const SpmmDev& p, uint4* ring,
     constexpr int EPV = Elt<T>::kPerVec;
     using P = Pipe<NV, LPR, true>;
     constexpr int PB = P::PB, NG = P::NG, EG = G * PB;        // positions and entries per group
-    static_assert(PB == 4 && (NG & (NG - 1)) == 0, "float4 weight reads; power-of-two group ring");
+    static_assert(PB % 4 == 0 && (NG & (NG - 1)) == 0, "float4 weight reads; power-of-two group ring");
     const int g = lane / LPR, l = lane % LPR;
     bool active[NV];
 #pragma unroll
@@ -648,31 +649,33 @@ __device__ __forceinline__ void stream_rows_multi(const SpmmDev& p, uint4* ring,
             cp_async_wait<NG - 1>();
             __syncwarp();
             const uint4* gp = ring_l + goff * (PB * 32 * NV);
-            uint4 v[PB][NV];
-#pragma unroll
-            for (int b = 0; b < PB; ++b)
-#pragma unroll
-                for (int c = 0; c < NV; ++c) v[b][c] = gp[(b * NV + c) * 32];
-            const float4 w4 = *reinterpret_cast<const float4*>(wfifo + goff * EG + 4 * g);
-            const float w[PB] = {w4.x, w4.y, w4.z, w4.w};
             const int left = rend - re;
-            if (left >= EG) {
 #pragma unroll
-                for (int b = 0; b < PB; ++b)
+            for (int q = 0; q < PB / 4; ++q) {                // four positions at a time
+                uint4 v[4][NV];
 #pragma unroll
-                    for (int c = 0; c < NV; ++c)
-                        if (kFull || active[c]) fma_any<T>(w[b], v[b][c], acc[c]);
-                re += EG;
-            } else {
+                for (int b = 0; b < 4; ++b)
 #pragma unroll
-                for (int b = 0; b < PB; ++b)
-                    if (G * b + g < left) {
+                    for (int c = 0; c < NV; ++c) v[b][c] = gp[((4 * q + b) * NV + c) * 32];
+                const float4 w4 = *reinterpret_cast<const float4*>(wfifo + goff * EG + PB * g + 4 * q);
+                const float w[4] = {w4.x, w4.y, w4.z, w4.w};
+                if (left >= EG) {
+#pragma unroll
+                    for (int b = 0; b < 4; ++b)
 #pragma unroll
                         for (int c = 0; c < NV; ++c)
                             if (kFull || active[c]) fma_any<T>(w[b], v[b][c], acc[c]);
-                    }
-                re = rend;
+                } else {
+#pragma unroll
+                    for (int b = 0; b < 4; ++b)
+                        if (G * (4 * q + b) + g < left) {
+#pragma unroll
+                            for (int c = 0; c < NV; ++c)
+                                if (kFull || active[c]) fma_any<T>(w[b], v[b][c], acc[c]);
+                        }
+                }
             }
+            re = left >= EG ? re + EG : rend;
             if (re == rend) {                                 // the row is complete
                 reduce_groups<NV, EPV, LPR>(acc);
                 if (kPartial) return;
@@ -716,7 +719,7 @@ __device__ __forceinline__ void stream_rows_multi(const SpmmDev& p, uint4* ring,
                     }
                 }
             }
-            if (rel < cnt) wfifo[goff * EG + 4 * (rel % G) + rel / G] = m_w;
+            if (rel < cnt) wfifo[goff * EG + PB * (rel % G) + rel / G] = m_w;
             ie += cnt;
             ++issued;
             if (ie == iend) {
