@@ -235,7 +235,7 @@ template <int NCH, int LPR, bool kAligned = false>
 struct Pipe {
     static constexpr int G = kWarp / LPR;                       // entries per position
     // positions per group (PB * G divides 32); the aligned stream with two entries per position takes 8
-    static constexpr int PB = (kAligned && G == 2 && NCH == 1) ? 8 : ((4 * G <= 32) ? 4 : 32 / G);
+    static constexpr int PB = ((kAligned && G == 2 && NCH == 1) || (LPR == 32 && NCH == 1)) ? 8 : ((4 * G <= 32) ? 4 : 32 / G);
     static constexpr int NG = (NCH > 1 || PB == 8) ? 2 : ((LPR == 32 || kAligned) ? 4 : 3);  // groups in flight per warp (a power of two for the row-aligned streams)
     static constexpr int RING = PB * NG;                        // slots of NCH * 512 bytes
     static constexpr size_t kWarpBytes = (size_t)RING * (NCH * 512 + G * 4);
@@ -436,7 +436,7 @@ __device__ __forceinline__ void stream_rows_wide(const SpmmDev& p, uint4* ring, 
     using P = Pipe<NCH, 32>;
     constexpr int EPV = Elt<T>::kPerVec;
     constexpr int PB = P::PB, NG = P::NG;
-    static_assert(PB == 4 && (NG & (NG - 1)) == 0, "float4 weight reads; power-of-two group ring");
+    static_assert(PB % 4 == 0 && (NG & (NG - 1)) == 0, "float4 weight reads; power-of-two group ring");
     constexpr int kSlotVecs = NCH * 32;                       // 16-byte vectors per slot
     bool active[NCH];
 #pragma unroll
@@ -472,31 +472,33 @@ __device__ __forceinline__ void stream_rows_wide(const SpmmDev& p, uint4* ring, 
             cp_async_wait<NG - 1>();
             __syncwarp();
             const uint4* gp = ring_l + goff * (PB * kSlotVecs);
-            uint4 v[PB][NCH];
-#pragma unroll
-            for (int b = 0; b < PB; ++b)
-#pragma unroll
-                for (int c = 0; c < NCH; ++c) v[b][c] = gp[b * kSlotVecs + c * 32];
-            const float4 w4 = *reinterpret_cast<const float4*>(wfifo + goff * PB);
-            const float w[PB] = {w4.x, w4.y, w4.z, w4.w};
             const int left = rend - re;
-            if (left >= PB) {
 #pragma unroll
-                for (int b = 0; b < PB; ++b)
+            for (int q = 0; q < PB / 4; ++q) {                // four positions at a time
+                uint4 v[4][NCH];
 #pragma unroll
-                    for (int c = 0; c < NCH; ++c)
-                        if (kFull || active[c]) fma_vec<T>(w[b], v[b][c], acc[c]);
-                re += PB;
-            } else {
+                for (int b = 0; b < 4; ++b)
 #pragma unroll
-                for (int b = 0; b < PB - 1; ++b)
-                    if (b < left) {
+                    for (int c = 0; c < NCH; ++c) v[b][c] = gp[(4 * q + b) * kSlotVecs + c * 32];
+                const float4 w4 = *reinterpret_cast<const float4*>(wfifo + goff * PB + 4 * q);
+                const float w[4] = {w4.x, w4.y, w4.z, w4.w};
+                if (left >= PB) {
+#pragma unroll
+                    for (int b = 0; b < 4; ++b)
 #pragma unroll
                         for (int c = 0; c < NCH; ++c)
                             if (kFull || active[c]) fma_vec<T>(w[b], v[b][c], acc[c]);
-                    }
-                re = rend;
+                } else {
+#pragma unroll
+                    for (int b = 0; b < 4; ++b)
+                        if (4 * q + b < left) {
+#pragma unroll
+                            for (int c = 0; c < NCH; ++c)
+                                if (kFull || active[c]) fma_vec<T>(w[b], v[b][c], acc[c]);
+                        }
+                }
             }
+            re = left >= PB ? re + PB : rend;
             if (re == rend) {                                 // the row is complete
                 if (kPartial) return;
                 finish_row<T, NCH, 32>(p, ctab, warp_row0 + rr, lane, acc);
