@@ -40,7 +40,7 @@ def parse_args():
                     help="gcn: the Bi-GCN forward (the benchmark); sage: side benchmark of the Bi-GraphSAGE layers; "
                          "entropy: side benchmark of the binning entropy estimator; backward: side benchmark of Algorithm 1 "
                          "for the hidden layer of the workload")
-    ap.add_argument("--zeta-format", type=int, default=0, help="0 auto, 1 fp32, 2 int16, 3 int8, 4 fp16")
+    ap.add_argument("--zeta-format", type=int, default=0, help="0 auto, 1 fp32, 2 int16, 3 int8, 4 fp16, 5 half-dot bytes")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--graph", action="store_true", help="also time the forward replayed as one CUDA graph")
@@ -425,13 +425,22 @@ def run_ours(args):
     dom = max(range(L), key=lambda l: spmm_ms[l])
     for l in range(L):
         f = args.zeta_format                      # the library's rule for the storage of zeta, layer by layer
+        wide = 128 < dims[l + 1] <= 256
+        half_ok = wide and 128 <= dims[l] <= 256 and n >= 64
         if f == 0:
-            f = binding.ZETA_I8 if (dims[l] <= 127 and 128 < dims[l + 1] <= 256) else binding.ZETA_F16
+            if wide and dims[l] <= 127:
+                f = binding.ZETA_I8
+            elif half_ok and n * dims[l + 1] >= (1 << 20):
+                f = binding.ZETA_I8H
+            else:
+                f = binding.ZETA_F16
+        if f == binding.ZETA_I8H and not half_ok:
+            f = binding.ZETA_I8 if (wide and dims[l] <= 127) else binding.ZETA_F16
         if f == binding.ZETA_I8 and dims[l] > 127:
             f = binding.ZETA_F16
         if f == binding.ZETA_F16 and dims[l] > 2048:
             f = binding.ZETA_I16
-        elt = {1: 4, 2: 2, 3: 1, 4: 2}[f]
+        elt = {1: 4, 2: 2, 3: 1, 4: 2, 5: 1}[f]
         per16 = 16 // elt
         ldz = (dims[l + 1] + per16 - 1) // per16 * per16
         last = (l == L - 1)
@@ -440,11 +449,11 @@ def run_ours(args):
         t = spmm_ms[l] * 1e-3
         kernels["spmm_l%d" % l] = {"ms": spmm_ms[l], "GBps_cached_model": expected / t / 1e9,
                                    "GBps_lower_model": lower / t / 1e9, "GBps_no_reuse_model": upper / t / 1e9,
-                                   "bytes_cached_model": expected, "row_bytes": ldz * elt, "zeta_format": {1: "f32", 2: "i16", 3: "i8", 4: "f16"}[f]}
+                                   "bytes_cached_model": expected, "row_bytes": ldz * elt, "zeta_format": {1: "f32", 2: "i16", 3: "i8", 4: "f16", 5: "i8h"}[f]}
         ops = 2.0 * n * dims[l] * dims[l + 1]
         words = n * dims[l + 1] * ((dims[l] + 31) // 32)                  # XOR + bit-count + add steps
         popc_peak = extras.get("popc_word_steps_per_s")
-        on_tc = dims[l] <= 256 and dims[l + 1] <= 256 and n * dims[l + 1] >= (1 << 20)   # the library's rule for the tensor-core path
+        on_tc = dims[l] <= 256 and dims[l + 1] <= 256 and (n * dims[l + 1] >= (1 << 20) or f == binding.ZETA_I8H)   # the library's rule for the tensor-core path
         k_pad = binding.packed_stride_words(dims[l]) * 32
         io_bytes = n * (binding.packed_stride_words(dims[l]) * 4.0 + 4.0 + ldz * elt)
         kernels["bitgemm_l%d" % l] = {"ms": gemm_ms[l], "path": "tcgen05 int8" if on_tc else "xor+popc",
@@ -482,7 +491,7 @@ def run_ours(args):
             "vs_baseline": None, "dtype": DTYPE, "data": "synthetic",
             "config": {"workload": workload_description(spec, n, nnz), "l2": "inputs_exceed_l2",
                        "parallelism": "replicas" if world > 1 else "single-gpu",
-                       "zeta_format": {0: "auto", 1: "f32", 2: "i16", 3: "i8", 4: "f16"}[args.zeta_format]},
+                       "zeta_format": {0: "auto", 1: "f32", 2: "i16", 3: "i8", 4: "f16", 5: "i8h"}[args.zeta_format]},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
             "step_ms_median": statistics.median(per_kernel["step"]), "step_ms_min": min(per_kernel["step"]),
             "extras": extras, "kernels": kernels}

@@ -58,14 +58,19 @@ typedef struct bigcn_ctx bigcn_ctx;
 /* Options for bigcn_set_option(). */
 enum {
     /* Storage of the rescaled contraction zeta between the bit-GEMM and the aggregation.
-     * 0 = choose per layer (default: 3 for d_in <= 127 with 129..256 output columns, where the
-     *     aggregation streams 256-byte rows; otherwise 4 when d_in <= 2048, else 2);
+     * 0 = choose per layer (default: for 129..256 output columns, where the aggregation streams 256-byte
+     *     rows, 3 when d_in <= 127 and 5 when 128 <= d_in <= 256 and the layer has at least 2^20 outputs;
+     *     otherwise 4 when d_in <= 2048, else 2);
      * 1 = fp32 zeta_ij = (beta_i alpha_j) dot_ij, exactly Eq. "cdot-op";
      * 2 = the integer dot products as int16, with beta folded into the edge weights and alpha
      *     applied once per output element (same sum, different rounding order);
      * 3 = as 2 but int8 (layers with d_in <= 127 only; others fall back to 4);
      * 4 = as 2 but the integers held as fp16, which is exact for |dot| <= 2048 (layers with
-     *     d_in <= 2048 only; others fall back to 2). */
+     *     d_in <= 2048 only; others fall back to 2);
+     * 5 = signed bytes for 128 <= d_in <= 256 and 129..256 output columns (other layers as 0): the byte is
+     *     s = (dot' - 1) / 2, dot' the dot without its first position when d_in is even (so that dot' is
+     *     odd and s fits a byte exactly); the aggregation adds back sum_k w_k (1 + f_k0 b_0j), two per-row
+     *     sums that ride along with the edge weights.  Exact in the integers; on the tensor-core contraction. */
     BIGCN_OPT_ZETA_FORMAT = 1,
     /* Rows of the sparse matrix with more entries than this are split across thread blocks. 0 = default. */
     BIGCN_OPT_LONG_ROW = 2,

@@ -21,7 +21,7 @@ MAX_LAYERS = 16
 OPT_ZETA_FORMAT = 1
 OPT_LONG_ROW = 2
 OPT_CONTRACTION = 3     # 0 = auto (default), 1 = XOR / bit-count pipe, 2 = tensor cores wherever the shape is covered
-ZETA_AUTO, ZETA_F32, ZETA_I16, ZETA_I8, ZETA_F16 = 0, 1, 2, 3, 4
+ZETA_AUTO, ZETA_F32, ZETA_I16, ZETA_I8, ZETA_F16, ZETA_I8H = 0, 1, 2, 3, 4, 5
 
 _i32, _i64, _vp, _sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_size_t
 

@@ -56,12 +56,20 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) %
 size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 // Storage format of zeta for a layer under the context's option.  Automatic choice: integers coded as
-// fp16 (exact up to d_in = 2048); for d_in <= 127 and 129..256 output columns the dots fit signed bytes
-// and the aggregation has a row-aligned stream for 256-byte rows that moves half the bytes.
-int pick_format(const bigcn_ctx* ctx, int d_in, int d_out)
+// fp16 (exact up to d_in = 2048); for 129..256 output columns the aggregation has a row-aligned stream for
+// 256-byte rows of signed bytes that moves half the bytes: plain dots for d_in <= 127, half-dots
+// (kZetaI8H, on the tensor-core contraction only: layers of at least 2^20 outputs) for 128 <= d_in <= 256.
+int pick_format(const bigcn_ctx* ctx, int d_in, int d_out, int64_t n, bool allow_half = false)
 {
     int f = ctx->zeta_format;
-    if (f == 0) f = (d_in <= 127 && d_out > 128 && d_out <= 256) ? kZetaI8 : kZetaF16;
+    const bool wide = d_out > 128 && d_out <= 256;
+    const bool half_ok = allow_half && wide && d_in >= 128 && d_in <= 256 && n >= 64 && ctx->contraction != 1;
+    if (f == 0) {
+        if (wide && d_in <= 127) f = kZetaI8;
+        else if (half_ok && n * (int64_t)d_out >= (int64_t(1) << 20)) f = kZetaI8H;
+        else f = kZetaF16;
+    }
+    if (f == kZetaI8H && !half_ok) f = (wide && d_in <= 127) ? kZetaI8 : kZetaF16;
     if (f == kZetaI8 && d_in > 127) f = kZetaF16;      // |dot| must fit the element type exactly
     if (f == kZetaF16 && d_in > 2048) f = kZetaI16;
     if (f == kZetaI16 && d_in > 32767) f = kZetaF32;
@@ -115,12 +123,22 @@ bigcn_status run_layer(bigcn_ctx* ctx, const bigcn_graph* g, const bigcn_layer* 
                        float* next_beta, int32_t* dbg_dot, float* dbg_zeta,
                        cudaEvent_t ev_mid /*nullable*/)
 {
-    const int fmt = pick_format(ctx, layer->d_in, layer->d_out);
+    const int fmt = pick_format(ctx, layer->d_in, layer->d_out, g->n, /*allow_half=*/true);
+    const bool half = fmt == kZetaI8H;
     const int64_t ldz = zeta_ld(layer->d_out, fmt);
     const int64_t stride_in = bigcn_packed_stride_words(layer->d_in);
+    // half-dot bytes: the node factors carrying the first feature sign and the columns' first weight signs follow
+    // the byte rows inside the zeta scratch (which is sized for fp32 rows, four times as much)
+    float* nws = nullptr;
+    float* col_b0 = nullptr;
+    if (half) {
+        char* after = static_cast<char*>(zeta) + up((size_t)g->n * ldz);
+        nws = reinterpret_cast<float*>(after);
+        col_b0 = reinterpret_cast<float*>(after + up((size_t)g->n * 4));
+    }
     cudaError_t e = launch_bitgemm(ctx->stream, in_bits, stride_in, layer->w_bitsT, stride_in, g->n,
                                    layer->d_in, layer->d_out, in_beta, layer->alpha, fmt, zeta, ldz,
-                                   dbg_dot, dbg_zeta, &ctx->launches_i, ctx->contraction);
+                                   dbg_dot, dbg_zeta, &ctx->launches_i, half ? 2 : ctx->contraction, nws, col_b0);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "bit-GEMM launch");
     if (ev_mid) BIGCN_CUDA(ctx, cudaEventRecord(ev_mid, ctx->stream));
     SpmmArgs a;
@@ -129,12 +147,14 @@ bigcn_status run_layer(bigcn_ctx* ctx, const bigcn_graph* g, const bigcn_layer* 
     a.rowptr = g->rowptr;
     a.colidx = g->colidx;
     a.val = g->val;
-    a.fmt = fmt;
+    a.fmt = half ? kZetaI8 : fmt;
     a.zeta = zeta;
     a.ldz = ldz;
     a.d_out = layer->d_out;
-    a.node_w = in_beta;
+    a.node_w = half ? nws : in_beta;
     a.col_w = layer->alpha;
+    a.half_dots = half;
+    a.col_b0 = col_b0;
     a.h_out = h_out;
     a.ldh = ldh;
     a.next_bits = next ? next_bits : nullptr;
@@ -312,7 +332,7 @@ bigcn_status bigcn_set_option(bigcn_ctx* ctx, int32_t option, int64_t value)
     if (!ctx) return BIGCN_ERR_NULL;
     switch (option) {
         case BIGCN_OPT_ZETA_FORMAT:
-            if (value < 0 || value > 4) return fail(ctx, BIGCN_ERR_SHAPE, "zeta format %lld not in [0, 4]", (long long)value);
+            if (value < 0 || value > 5) return fail(ctx, BIGCN_ERR_SHAPE, "zeta format %lld not in [0, 5]", (long long)value);
             ctx->zeta_format = (int)value;
             return BIGCN_OK;
         case BIGCN_OPT_LONG_ROW:
@@ -821,7 +841,7 @@ bigcn_status bigcn_sage_layer_forward(bigcn_ctx* ctx, const bigcn_graph* mean_gr
     cudaError_t e = launch_bitgemm(ctx->stream, in_bits, stride_in, self_layer->w_bitsT, stride_in, n, d_in, d_out,
                                    in_beta, self_layer->alpha, kZetaF32, zeta_self, ld_self, nullptr, nullptr, &ctx->launches_i, ctx->contraction);
     if (e != cudaSuccess) { finish_call(ctx); return cuda_fail(ctx, e, "bit-GEMM (self term) launch"); }
-    const int fmt = pick_format(ctx, d_in, d_out);
+    const int fmt = pick_format(ctx, d_in, d_out, n);
     const int64_t ldz = zeta_ld(d_out, fmt);
     e = launch_bitgemm(ctx->stream, in_bits, stride_in, nbr_layer->w_bitsT, stride_in, n, d_in, d_out,
                        in_beta, nbr_layer->alpha, fmt, zeta_nbr, ldz, nullptr, nullptr, &ctx->launches_i, ctx->contraction);

@@ -11,7 +11,9 @@ namespace bigcn {
 constexpr int kWarp = 32;
 
 // Storage of the contraction result between the bit-GEMM and the aggregation.
-enum ZetaFormat : int { kZetaF32 = 1, kZetaI16 = 2, kZetaI8 = 3, kZetaF16 = 4 };
+// kZetaI8H (128 <= d_in <= 256): signed bytes s = (dot' - 1) / 2 where dot' is the dot without the first position when
+// d_in is even (so that dot' is odd and s fits a byte); the aggregation adds the missing terms back (see spmm.cu).
+enum ZetaFormat : int { kZetaF32 = 1, kZetaI16 = 2, kZetaI8 = 3, kZetaF16 = 4, kZetaI8H = 5 };
 
 inline __host__ __device__ int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline __host__ __device__ int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
@@ -19,9 +21,9 @@ inline __host__ __device__ int64_t round_up(int64_t a, int64_t b) { return ceil_
 // Elements per row of the zeta buffer: d_out rounded up so that a row is a whole number of 16-byte vectors.
 inline int64_t zeta_ld(int d_out, int fmt)
 {
-    return round_up(d_out, 16 / (fmt == kZetaF32 ? 4 : (fmt == kZetaI8 ? 1 : 2)));
+    return round_up(d_out, 16 / (fmt == kZetaF32 ? 4 : ((fmt == kZetaI8 || fmt == kZetaI8H) ? 1 : 2)));
 }
-inline int zeta_elt_bytes(int fmt) { return fmt == kZetaF32 ? 4 : (fmt == kZetaI8 ? 1 : 2); }
+inline int zeta_elt_bytes(int fmt) { return fmt == kZetaF32 ? 4 : ((fmt == kZetaI8 || fmt == kZetaI8H) ? 1 : 2); }
 
 // ---- launchers (each returns the launch status; all asynchronous on `s`) ------------------------
 
@@ -35,7 +37,8 @@ cudaError_t launch_pack_weights(cudaStream_t s, const float* W, int d_in, int d_
 cudaError_t launch_bitgemm(cudaStream_t s, const uint32_t* A, int64_t stride_a,
                            const uint32_t* BT, int64_t stride_b, int64_t n, int d_in, int d_out,
                            const float* beta, const float* alpha, int fmt, void* zeta, int64_t ldz,
-                           int32_t* dbg_dot, float* dbg_zeta, int* launches, int path = 0 /* 0 auto, 1 bit-count pipe, 2 tensor cores wherever covered */);
+                           int32_t* dbg_dot, float* dbg_zeta, int* launches, int path = 0 /* 0 auto, 1 bit-count pipe, 2 tensor cores wherever covered */,
+                           float* nws = nullptr /* kZetaI8H: [n] beta_i times the first sign */, float* col_b0 = nullptr /* kZetaI8H: [d_out] */);
 
 struct SpmmArgs {
     int64_t n;
@@ -49,6 +52,8 @@ struct SpmmArgs {
     int d_out;
     const float* node_w;     // integer formats: per-source-node factor (beta), multiplied into the edge weight
     const float* col_w;      // integer formats: per-column factor (alpha), applied once per output
+    const float* col_b0 = nullptr;   // half-dot bytes (kZetaI8H): per-column first weight sign (0 when d_in is odd)
+    bool half_dots = false;          // zeta holds s = (dot' - 1) / 2 and node_w carries the first feature sign
     const float* add = nullptr;   // optional fp32 [n x ld_add] added to every aggregated row (Bi-GraphSAGE self term)
     int64_t ld_add = 0;
     float* h_out;            // nullable
@@ -82,7 +87,7 @@ size_t popc_peak_scratch_bytes();
 bool bitgemm_tc_covers(int d_in, int d_out, int64_t stride_a, int64_t stride_b);
 cudaError_t launch_bitgemm_tc(cudaStream_t s, const uint32_t* A, int64_t stride_a, const uint32_t* BT, int64_t stride_b,
                               int64_t n, int d_in, int d_out, const float* beta, const float* alpha, int fmt, void* zeta,
-                              int64_t ldz, int32_t* dbg_dot, float* dbg_zeta);
+                              int64_t ldz, int32_t* dbg_dot, float* dbg_zeta, float* nws = nullptr, float* col_b0 = nullptr);
 int bitgemm_tc_timeouts();
 
 // Binning entropy estimate (entropy.cu): scratch = 2 * d uint32.

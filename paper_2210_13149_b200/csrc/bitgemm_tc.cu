@@ -110,6 +110,8 @@ template <> struct TcOut<kZetaI8> {
         out[0] = make_uint4(b[0], b[1], b[2], b[3]);
     }
 };
+// half-dot bytes: the dots are replaced by s = (dot' - 1) / 2 before packing (see the epilogue), then stored as bytes
+template <> struct TcOut<kZetaI8H> : TcOut<kZetaI8> {};
 template <> struct TcOut<kZetaF32> {
     static constexpr int kElt = 4;
     // zeta_ij = (beta_i alpha_j) dot_ij in this order (Eq. "cdot-op"); al points at the chunk's first column
@@ -136,7 +138,8 @@ template <int N, int FMT>
 __global__ void __launch_bounds__(kTcThreads, 2)
 bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32_t* __restrict__ BT, int64_t stride_b,
                   int64_t n, int d_in, int d_out, const float* __restrict__ beta, const float* __restrict__ alpha,
-                  void* __restrict__ zeta, int64_t ldz, int32_t* __restrict__ dbg_dot, float* __restrict__ dbg_zeta)
+                  void* __restrict__ zeta, int64_t ldz, int32_t* __restrict__ dbg_dot, float* __restrict__ dbg_zeta,
+                  float* __restrict__ nws, float* __restrict__ col_b0)
 {
     using Out = TcOut<FMT>;
     constexpr int kElt = Out::kElt;                         // bytes per stored element = 16-byte pieces per chunk of 16 columns
@@ -144,6 +147,7 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
     __shared__ __align__(8) uint64_t bar;
     __shared__ uint32_t tmem_base_s;
     __shared__ float al_s[N];
+    __shared__ int b0_s[FMT == kZetaI8H ? N : 1];          // half-dot bytes: first sign of every weight column (0 when d_in is odd)
     constexpr int kCols = N <= 32 ? 32 : (N <= 64 ? 64 : (N <= 128 ? 128 : 256));   // tensor-memory columns of the accumulator
     const int K = (int)stride_a * 32;                       // bytes per expanded row (padding included)
     const int pad = K - d_in;                               // padding positions: each contributes +1
@@ -160,6 +164,14 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     for (int j = threadIdx.x; j < N; j += kTcThreads) al_s[j] = j < d_out ? __ldg(alpha + j) : 0.f;
+    if constexpr (FMT == kZetaI8H) {
+        const bool even = (d_in & 1) == 0;                  // even d_in: the first position is left out of the stored dot
+        for (int j = threadIdx.x; j < N; j += kTcThreads) {
+            const int b0 = (even && j < d_out) ? ((__ldg(BT + (int64_t)j * stride_b) & 1u) ? 1 : -1) : 0;
+            b0_s[j] = b0;
+            if (blockIdx.x == 0 && j < d_out) col_b0[j] = (float)b0;
+        }
+    }
     stage_operand(Bs, N, BT, stride_b, d_out);
 
     const int64_t n_tiles = ceil_div(n, kTcRows);
@@ -232,7 +244,15 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
         const int64_t row0 = tile_row0(i) + lane_base;
         const int64_t row = row0 + lane;
         const bool row_in = row < n;
-        const float be = (row_in && (FMT == kZetaF32 || dbg_zeta)) ? __ldg(beta + row) : 0.f;
+        const float be = (row_in && (FMT == kZetaF32 || FMT == kZetaI8H || dbg_zeta)) ? __ldg(beta + row) : 0.f;
+        int f0 = 0;                                         // half-dot bytes: the row's first sign (0 when d_in is odd)
+        if constexpr (FMT == kZetaI8H) {
+            if (row_in) {
+                const int sgn = (__ldg(A + row * stride_a) & 1u) ? 1 : -1;
+                f0 = (d_in & 1) ? 0 : sgn;
+                if (warp < 4) nws[row] = (d_in & 1) ? be : be * (float)sgn;      // beta_i carrying the first sign
+            }
+        }
 #pragma unroll 1
         for (int pass = 0; pass < kPasses; ++pass) {
 #pragma unroll
@@ -248,6 +268,14 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
                 int dot[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e) dot[e] = (c0 + e < d_out) ? (int)v[e] - pad : 0;   // padding columns of zeta stay 0
+                int full[16];                               // the true dots, for the debug taps
+#pragma unroll
+                for (int e = 0; e < 16; ++e) full[e] = dot[e];
+                if constexpr (FMT == kZetaI8H) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e)
+                        if (c0 + e < d_out) dot[e] = (dot[e] - f0 * b0_s[c0 + e] - 1) >> 1;       // odd by construction: exact
+                }
                 uint4 out[kElt];
                 Out::pack(dot, be, al_s + c0, out);
 #pragma unroll
@@ -260,8 +288,8 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
                     for (int e = 0; e < 16; ++e) {
                         const int c = c0 + e;
                         if (c < d_out) {
-                            if (dbg_dot) dbg_dot[row * (int64_t)d_out + c] = dot[e];
-                            if (dbg_zeta) dbg_zeta[row * (int64_t)d_out + c] = __fmul_rn(__fmul_rn(be, al_s[c]), (float)dot[e]);
+                            if (dbg_dot) dbg_dot[row * (int64_t)d_out + c] = full[e];
+                            if (dbg_zeta) dbg_zeta[row * (int64_t)d_out + c] = __fmul_rn(__fmul_rn(be, al_s[c]), (float)full[e]);
                         }
                     }
                 }
@@ -290,29 +318,32 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
 template <int N, int FMT>
 cudaError_t launch_tc_inst(cudaStream_t s, const uint32_t* A, int64_t stride_a, const uint32_t* BT, int64_t stride_b,
                            int64_t n, int d_in, int d_out, const float* beta, const float* alpha, void* zeta, int64_t ldz,
-                           int32_t* dbg_dot, float* dbg_zeta)
+                           int32_t* dbg_dot, float* dbg_zeta, float* nws, float* col_b0)
 {
     // operands: weight panel N x K bytes, feature tile 128 x K bytes (at least the 32 KB the epilogue's scratch needs)
     const size_t smem = (size_t)N * stride_a * 32 + std::max<size_t>((size_t)kTcRows * stride_a * 32, 32 * 1024);
     cudaError_t e = cudaFuncSetAttribute(bitgemm_tc_kernel<N, FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, kTcRows), 148 * 2);
-    bitgemm_tc_kernel<N, FMT><<<grid, kTcThreads, smem, s>>>(A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta);
+    bitgemm_tc_kernel<N, FMT><<<grid, kTcThreads, smem, s>>>(A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0);
     return cudaGetLastError();
 }
 
 template <int N>
 cudaError_t launch_tc_n(cudaStream_t s, int fmt, const uint32_t* A, int64_t stride_a, const uint32_t* BT, int64_t stride_b,
                         int64_t n, int d_in, int d_out, const float* beta, const float* alpha, void* zeta, int64_t ldz,
-                        int32_t* dbg_dot, float* dbg_zeta)
+                        int32_t* dbg_dot, float* dbg_zeta, float* nws, float* col_b0)
 {
+#define BIGCN_TC_CALL(FMT) launch_tc_inst<N, FMT>(s, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0)
     switch (fmt) {
-        case kZetaF32: return launch_tc_inst<N, kZetaF32>(s, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta);
-        case kZetaF16: return launch_tc_inst<N, kZetaF16>(s, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta);
-        case kZetaI16: return launch_tc_inst<N, kZetaI16>(s, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta);
-        case kZetaI8: return launch_tc_inst<N, kZetaI8>(s, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta);
+        case kZetaF32: return BIGCN_TC_CALL(kZetaF32);
+        case kZetaF16: return BIGCN_TC_CALL(kZetaF16);
+        case kZetaI16: return BIGCN_TC_CALL(kZetaI16);
+        case kZetaI8: return BIGCN_TC_CALL(kZetaI8);
+        case kZetaI8H: return (nws && col_b0 && d_in <= 256) ? BIGCN_TC_CALL(kZetaI8H) : cudaErrorInvalidValue;
         default: return cudaErrorInvalidValue;
     }
+#undef BIGCN_TC_CALL
 }
 
 }  // namespace
@@ -324,12 +355,12 @@ bool bitgemm_tc_covers(int d_in, int d_out, int64_t stride_a, int64_t stride_b)
 
 cudaError_t launch_bitgemm_tc(cudaStream_t s, const uint32_t* A, int64_t stride_a, const uint32_t* BT, int64_t stride_b,
                               int64_t n, int d_in, int d_out, const float* beta, const float* alpha, int fmt, void* zeta,
-                              int64_t ldz, int32_t* dbg_dot, float* dbg_zeta)
+                              int64_t ldz, int32_t* dbg_dot, float* dbg_zeta, float* nws, float* col_b0)
 {
     // the instruction's N: the output channels rounded up to 64 / 128 / 256 (16 would do; fewer variants to build)
-    if (d_out <= 64) return launch_tc_n<64>(s, fmt, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta);
-    if (d_out <= 128) return launch_tc_n<128>(s, fmt, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta);
-    return launch_tc_n<256>(s, fmt, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta);
+    if (d_out <= 64) return launch_tc_n<64>(s, fmt, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0);
+    if (d_out <= 128) return launch_tc_n<128>(s, fmt, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0);
+    return launch_tc_n<256>(s, fmt, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0);
 }
 
 // Number of waits that ran out since the library was loaded on the current device (0 = none).

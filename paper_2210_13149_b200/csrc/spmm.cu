@@ -96,6 +96,8 @@ struct SpmmDev {
     int d_out;
     const float* node_w;     // nullable
     const float* col_w;      // nullable
+    const float* col_b0;     // half-dot bytes only: per-column first weight sign (0 where none)
+    int half_dots;           // zeta holds s = (dot' - 1) / 2; node_w carries the first feature sign
     const float* add;        // nullable: fp32 [n x ld_add] added to the aggregated row (after col_w)
     int64_t ld_add;
     float* h_out;
@@ -142,9 +144,10 @@ __device__ __forceinline__ void reduce_groups(float (&acc)[NCH][EPV])
             for (int i = 0; i < EPV; ++i) acc[c][i] += __shfl_xor_sync(0xffffffffu, acc[c][i], o);
 }
 
-// Per-column constants of the row epilogue, staged once per thread block: three arrays of kCols
-// floats -- the column factor (0 for padding columns, 1 when there is none), then the next layer's
-// shift and scale (0 and 1 where there are none, so that applying them changes nothing).
+// Per-column constants of the row epilogue, staged once per thread block: four arrays of kCols
+// floats -- the column factor (0 for padding columns, 1 when there is none), the next layer's shift and
+// scale (0 and 1 where there are none, so that applying them changes nothing), and the first weight
+// sign of the column (half-dot bytes only, else 0).
 template <int kCols>
 __device__ __forceinline__ void fill_col_table(const SpmmDev& p, float* ctab)
 {
@@ -153,14 +156,18 @@ __device__ __forceinline__ void fill_col_table(const SpmmDev& p, float* ctab)
         ctab[col] = in ? (p.col_w ? __ldg(p.col_w + col) : 1.f) : 0.f;
         ctab[kCols + col] = (in && p.next_shift) ? __ldg(p.next_shift + col) : 0.f;
         ctab[2 * kCols + col] = (in && p.next_shift) ? __ldg(p.next_scale + col) : 1.f;
+        ctab[3 * kCols + col] = (in && p.col_b0) ? __ldg(p.col_b0 + col) : 0.f;
     }
 }
 
 // Writes one finished row: optional fp32 store, optional sign/scale packing for the next layer.
 // Called by a full warp; every lane holds the totals of vector(s) c*32 + (lane % LPR).
-template <typename T, int NCH, int LPR>
+// kHalf (half-dot bytes): the accumulators hold sum_k w_k s_kj with s = (dot' - 1) / 2; the row's sum of the
+// edge weights `wsum` and their sum signed by the sources' first feature sign `wsgn` give back
+// sum_k w_k dot_kj = 2 acc_j + wsum + b0_j wsgn before the column factor is applied.
+template <typename T, int NCH, int LPR, bool kHalf = false>
 __device__ __forceinline__ void finish_row(const SpmmDev& p, const float* ctab, int64_t row, int lane,
-                                           float (&acc)[NCH][Elt<T>::kPerVec])
+                                           float (&acc)[NCH][Elt<T>::kPerVec], float wsum = 0.f, float wsgn = 0.f)
 {
     constexpr int EPV = Elt<T>::kPerVec;
     constexpr int LW = 32 / EPV;                  // lanes that share one packed word
@@ -175,10 +182,18 @@ __device__ __forceinline__ void finish_row(const SpmmDev& p, const float* ctab, 
 #pragma unroll
         for (int q = 0; q < EPV / 4; ++q) {
             const float4 a = *reinterpret_cast<const float4*>(ctab + col0 + 4 * q);
-            x[4 * q] = acc[c][4 * q] * a.x;
-            x[4 * q + 1] = acc[c][4 * q + 1] * a.y;
-            x[4 * q + 2] = acc[c][4 * q + 2] * a.z;
-            x[4 * q + 3] = acc[c][4 * q + 3] * a.w;
+            float t[4] = {acc[c][4 * q], acc[c][4 * q + 1], acc[c][4 * q + 2], acc[c][4 * q + 3]};
+            if constexpr (kHalf) {
+                const float4 b0 = *reinterpret_cast<const float4*>(ctab + 3 * kCols + col0 + 4 * q);
+                t[0] = fmaf(2.f, t[0], fmaf(b0.x, wsgn, wsum));
+                t[1] = fmaf(2.f, t[1], fmaf(b0.y, wsgn, wsum));
+                t[2] = fmaf(2.f, t[2], fmaf(b0.z, wsgn, wsum));
+                t[3] = fmaf(2.f, t[3], fmaf(b0.w, wsgn, wsum));
+            }
+            x[4 * q] = t[0] * a.x;
+            x[4 * q + 1] = t[1] * a.y;
+            x[4 * q + 2] = t[2] * a.z;
+            x[4 * q + 3] = t[3] * a.w;
         }
         if (p.add) {
 #pragma unroll
@@ -606,7 +621,7 @@ __device__ __forceinline__ void fma_any(float w, const uint4& v, float (&acc)[El
 // and the weight ring are those of stream_rows_wide; the weights of a group are stored lane group by
 // lane group (index PB g + b) so that a lane reads four of them with one 16-byte load.  kFull: the row has
 // exactly LPR vectors, no lane needs masking.
-template <typename T, int G, int NV, bool kFull, bool kPartial>
+template <typename T, int G, int NV, bool kFull, bool kPartial, bool kHalf = false>
 __device__ __forceinline__ void stream_rows_multi(const SpmmDev& p, uint4* ring, float* wfifo, const float* ctab, int lane,
                                                   int64_t e0, int n_ent, int64_t warp_row0, int row_lo,
                                                   int row_hi, int rp_rel, float (&acc)[NV][Elt<T>::kPerVec])
@@ -643,6 +658,7 @@ __device__ __forceinline__ void stream_rows_multi(const SpmmDev& p, uint4* ring,
     bool more = row_lo < row_hi;
     int issued = 0, goff = 0;                                 // groups issued; ring position of the current group
     zero_acc<NV, EPV>(acc);
+    float wsum = 0.f, wsgn = 0.f;                             // half-dot bytes: sum of the row's weights, plain and signed
 
     for (int it = 0;; ++it) {
         if (it >= NG) {
@@ -663,26 +679,50 @@ __device__ __forceinline__ void stream_rows_multi(const SpmmDev& p, uint4* ring,
                 const float w[4] = {w4.x, w4.y, w4.z, w4.w};
                 if (left >= EG) {
 #pragma unroll
-                    for (int b = 0; b < 4; ++b)
+                    for (int b = 0; b < 4; ++b) {
+                        const float wa = kHalf ? fabsf(w[b]) : w[b];      // the sign carries the source's first feature sign
+                        if (kHalf) { wsum += wa; wsgn += w[b]; }
 #pragma unroll
                         for (int c = 0; c < NV; ++c)
-                            if (kFull || active[c]) fma_any<T>(w[b], v[b][c], acc[c]);
+                            if (kFull || active[c]) fma_any<T>(wa, v[b][c], acc[c]);
+                    }
                 } else {
 #pragma unroll
                     for (int b = 0; b < 4; ++b)
                         if (G * (4 * q + b) + g < left) {
+                            const float wa = kHalf ? fabsf(w[b]) : w[b];
+                            if (kHalf) { wsum += wa; wsgn += w[b]; }
 #pragma unroll
                             for (int c = 0; c < NV; ++c)
-                                if (kFull || active[c]) fma_any<T>(w[b], v[b][c], acc[c]);
+                                if (kFull || active[c]) fma_any<T>(wa, v[b][c], acc[c]);
                         }
                 }
             }
             re = left >= EG ? re + EG : rend;
             if (re == rend) {                                 // the row is complete
                 reduce_groups<NV, EPV, LPR>(acc);
-                if (kPartial) return;
-                finish_row<T, NV, LPR>(p, ctab, warp_row0 + rr, lane, acc);
+                if (kHalf) {
+#pragma unroll
+                    for (int o = LPR; o < kWarp; o <<= 1) {
+                        wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
+                        wsgn += __shfl_xor_sync(0xffffffffu, wsgn, o);
+                    }
+                }
+                if (kPartial) {
+                    if (kHalf) {                              // a slice of a long row: hand back the reconstructed partial sums
+                        constexpr int kCols = NV * LPR * EPV;
+#pragma unroll
+                        for (int c = 0; c < NV; ++c)
+#pragma unroll
+                            for (int i = 0; i < EPV; ++i)
+                                acc[c][i] = fmaf(2.f, acc[c][i], fmaf(ctab[3 * kCols + (c * LPR + l) * EPV + i], wsgn, wsum));
+                    }
+                    return;
+                }
+                finish_row<T, NV, LPR, kHalf>(p, ctab, warp_row0 + rr, lane, acc, wsum, wsgn);
                 zero_acc<NV, EPV>(acc);
+                wsum = 0.f;
+                wsgn = 0.f;
                 ++rr;
                 if (rr < row_hi) rend = row_end_of(rr);
             }
@@ -756,10 +796,12 @@ constexpr int spmm_blocks_per_sm()
 }
 
 // kAligned (rows of 8 or 16 vectors only): the row-aligned multi-entry stream instead of the general one.
-template <typename T, int NCH, int LPR, bool kFull, bool kAligned>
+// kHalf: half-dot bytes (aligned byte stream only).
+template <typename T, int NCH, int LPR, bool kFull, bool kAligned, bool kHalf = false>
 __global__ void __launch_bounds__(kSpmmThreads, spmm_blocks_per_sm<NCH, LPR, kAligned>())
 spmm_kernel(const SpmmDev p, int rows_per_warp)
 {
+    static_assert(!kHalf || (kAligned && sizeof(T) == 1), "half-dot bytes take the aligned byte stream");
     static_assert(!kAligned || ((NCH == 1 || NCH == 2) && (LPR == 8 || LPR == 16)), "the multi-entry stream: 8 or 16 lanes per row, one or two vectors per lane");
     using P = Pipe<NCH, LPR, kAligned>;
     constexpr int EPV = Elt<T>::kPerVec;
@@ -808,7 +850,7 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
                     stream_rows_wide<T, NCH, kFull, false>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
                                                     (int)(rp_reg - e0), acc);
                 else if constexpr (kAligned)
-                    stream_rows_multi<T, kWarp / LPR, NCH, kFull, false>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
+                    stream_rows_multi<T, kWarp / LPR, NCH, kFull, false, kHalf>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
                                                                     (int)(rp_reg - e0), acc);
                 else
                     stream_entries<T, NCH, LPR, false>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
@@ -828,7 +870,7 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
         if constexpr (LPR == 32)
             stream_rows_wide<T, NCH, kFull, true>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
         else if constexpr (kAligned)
-            stream_rows_multi<T, kWarp / LPR, NCH, kFull, true>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
+            stream_rows_multi<T, kWarp / LPR, NCH, kFull, true, kHalf>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
         else
             stream_entries<T, NCH, LPR, true>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
         __syncthreads();                                      // every ring is idle: reuse them for the partial sums
@@ -855,15 +897,15 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
     }
 }
 
-template <typename T, int NCH, int LPR, bool kFull = false, bool kAligned = false>
+template <typename T, int NCH, int LPR, bool kFull = false, bool kAligned = false, bool kHalf = false>
 cudaError_t launch_one(cudaStream_t s, const SpmmDev& p)
 {
     constexpr int kCols = NCH * (LPR < 32 ? LPR : 32) * Elt<T>::kPerVec;
-    constexpr size_t smem = kSpmmWarps * Pipe<NCH, LPR, kAligned>::kWarpBytes + 3 * kCols * sizeof(float);   // rings, weights, column table
+    constexpr size_t smem = kSpmmWarps * Pipe<NCH, LPR, kAligned>::kWarpBytes + 4 * kCols * sizeof(float);   // rings, weights, column table
     // enough thread blocks to fill the machine on small graphs, long runs of rows on large ones
     const int rows_per_warp = (int)std::min<int64_t>(kMaxRowsPerWarp, std::max<int64_t>(1, p.n / (kSpmmWarps * 148 * 8)));
     if (smem > 40 * 1024) {                                   // above the default limit: opt in
-        cudaError_t e = cudaFuncSetAttribute(spmm_kernel<T, NCH, LPR, kFull, kAligned>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(spmm_kernel<T, NCH, LPR, kFull, kAligned, kHalf>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
     cudaError_t e = cudaMemsetAsync(p.run_counter, 0, sizeof(int), s);
@@ -871,7 +913,7 @@ cudaError_t launch_one(cudaStream_t s, const SpmmDev& p)
     // one wave of resident blocks; the warps pull runs of rows until none are left
     const int64_t wanted = ceil_div(ceil_div(p.n, rows_per_warp), kSpmmWarps);
     const unsigned grid = (unsigned)std::min<int64_t>(wanted, 148 * spmm_blocks_per_sm<NCH, LPR, kAligned>());
-    spmm_kernel<T, NCH, LPR, kFull, kAligned><<<grid, kSpmmThreads, smem, s>>>(p, rows_per_warp);
+    spmm_kernel<T, NCH, LPR, kFull, kAligned, kHalf><<<grid, kSpmmThreads, smem, s>>>(p, rows_per_warp);
     return cudaGetLastError();
 }
 
@@ -890,6 +932,7 @@ cudaError_t dispatch(cudaStream_t s, const SpmmDev& p, double mean_row)
     if (nv <= 8) return launch_one<T, 1, 8>(s, p);
     if (nv <= 16) {
         if constexpr (sizeof(T) == 1) {
+            if (p.half_dots) return nv == 16 ? launch_one<T, 1, 16, true, true, true>(s, p) : launch_one<T, 1, 16, false, true, true>(s, p);
             // (8 lanes per row with two vectors each, four entries per position -- launch_one<T, 2, 8, .., true> -- halves
             // the bookkeeping per entry again but needs 123 registers: 7.7 ms against 6.4 ms on c5 layer 0; not used)
             if (!(mean_row > 0.0 && mean_row < 8.0))
@@ -927,6 +970,9 @@ cudaError_t launch_spmm(cudaStream_t s, const SpmmArgs& a, int* launches)
     p.node_w = a.fmt == kZetaF32 ? nullptr : a.node_w;
     p.col_w = a.fmt == kZetaF32 ? nullptr : a.col_w;
     p.add = a.add;
+    p.col_b0 = a.half_dots ? a.col_b0 : nullptr;
+    p.half_dots = a.half_dots ? 1 : 0;
+    if (a.half_dots && (a.fmt != kZetaI8 || p.nv > 16 || p.nv <= 8 || !a.col_b0 || !a.node_w)) return cudaErrorInvalidValue;   // 129..256 byte columns only
     p.ld_add = a.ld_add;
     p.h_out = a.h_out;
     p.ldh = a.ldh;

@@ -14,7 +14,7 @@ from parity_util import (ATOL, RTOL, assert_close, bits_from_dev, bits_to_dev, d
 
 pytestmark = pytest.mark.gpu
 
-FORMATS = [1, 2, 3, 4]       # fp32 zeta; integer dots as int16 / int8 (d_in <= 127) / fp16 (d_in <= 2048)
+FORMATS = [1, 2, 3, 4, 5]    # fp32 zeta; integer dots as int16 / int8 (d_in <= 127) / fp16 (d_in <= 2048) / half-dot bytes (128 <= d_in <= 256)
 
 
 @pytest.fixture(scope="module")
@@ -146,6 +146,37 @@ LAYER_SHAPES = [(200, 1500, 1, 1), (300, 2500, 33, 7), (500, 6000, 100, 256), (4
 @pytest.mark.parametrize("n,e,d_in,d_out", LAYER_SHAPES)
 def test_layer_forward_against_oracle(ctx, B, fmt, n, e, d_in, d_out):
     check_layer_forward(ctx, B, fmt, n, e, d_in, d_out)
+
+
+# half-dot bytes: every parity of d_in in range, both ends of the byte range, ragged column counts, several tiles
+HALF_SHAPES = [(64, 300, 128, 129), (500, 6000, 129, 200), (700, 9000, 200, 256), (300, 4000, 255, 130),
+               (300, 3000, 256, 256), (2000, 60000, 256, 200), (40000, 300000, 256, 256), (5000, 60000, 254, 256)]
+
+
+@pytest.mark.parametrize("n,e,d_in,d_out", HALF_SHAPES)
+def test_layer_forward_half_dot_bytes(ctx, B, n, e, d_in, d_out):
+    check_layer_forward(ctx, B, 5, n, e, d_in, d_out)
+
+
+def test_half_dot_bytes_at_the_ends_of_the_byte_range(ctx, B):
+    """Rows equal to a weight column (dot = +256) and to its complement (dot = -256): the stored bytes reach
+    +127 and -128; the reconstructed sums must still be exact."""
+    n, d_in, d_out = 300, 256, 256
+    rng = np.random.default_rng(12)
+    _, _, g = small_graph(n, 3000, 12)
+    W = rng.standard_normal((d_in, d_out)).astype(np.float32)
+    H = rng.standard_normal((n, d_in)).astype(np.float32)
+    H[0] = np.abs(H[0]) * np.where(W[:, 0] >= 0, 1, -1)        # same signs as column 0
+    H[1] = -np.abs(H[1]) * np.where(W[:, 1] >= 0, 1, -1)       # opposite signs to column 1
+    t = oracle.layer_forward(g, oracle.Layer(W), H)
+    assert t.dot[0, 0] == 256 and t.dot[1, 1] == -256
+    ctx.set_option(B.OPT_ZETA_FORMAT, 5)
+    G = device_graph(B, g)
+    layer = B.make_layer(d_in, d_out, bits_to_dev(t.bitsT), dev(t.alpha))
+    out = ctx.layer_forward(G, layer, bits_to_dev(t.bits), dev(t.beta), want_h=True, debug=True)
+    ctx.sync_check()
+    assert np.array_equal(out["dot"].cpu().numpy(), t.dot)
+    assert_close(out["h"], t.H_out, "H' (half-dot bytes, extreme dots)")
 
 
 # shapes the tensor-core contraction covers (d_in, d_out <= 256): tile tails, one row, several tiles per CTA
