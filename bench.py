@@ -339,6 +339,21 @@ def run_ours(args):
             extras["popc_word_steps_per_s"] = ctx.measure_popc_peak()
         except Exception as exc:
             extras["popc_word_steps_per_s"] = None
+        # the same forward with every zeta row in fp16 (the HBM-bound variant of the wide aggregations), for comparison
+        if args.zeta_format == 0:
+            try:
+                ctx.set_option(binding.OPT_ZETA_FORMAT, binding.ZETA_F16)
+                alt = [[] for _ in range(L)]
+                for k in range(3 + min(args.steps, 5)):
+                    _, st = ctx.forward(G, layers, X, logits, stats=True)
+                    if k >= 3:
+                        for l in range(L):
+                            alt[l].append(st.ms_spmm[l])
+                extras["spmm_fp16_rows_ms"] = [sum(v) / len(v) for v in alt]
+            except Exception as exc:
+                extras["spmm_fp16_rows_ms"] = "failed: %r" % (exc,)
+            finally:
+                ctx.set_option(binding.OPT_ZETA_FORMAT, 0)
         # the same contraction on the XOR / bit-count pipe (the library's other path), for comparison
         try:
             ctx.set_option(binding.OPT_CONTRACTION, 1)
@@ -473,6 +488,9 @@ def run_ours(args):
                 "bound": "hbm", "achieved": achieved, "peak": peak, "peak_kind": "%s copy bandwidth" % peak_kind,
                 "unit": "GB/s", "frac": achieved / peak, "traffic": traffic_record(dom_key),
                 "algorithmic_bytes": kernels["spmm_l%d" % dom]["bytes_cached_model"],
+                "note": "byte rows (i8 / i8h) halve the DRAM traffic of the 256-column aggregations and leave them bound by "
+                        "instruction issue, not HBM; with fp16 rows (--zeta-format 4) the same layer is HBM-bound: see "
+                        "extras.spmm_fp16_rows_ms and kernels.*",
                 "model": "per launch: 8 B per stored entry (column, value) + rowptr + node weights + output + every "
                          "operand row once + one operand row per further stored entry whose source is not among the "
                          "highest-degree rows an ideal 126 MB cache would hold"}
