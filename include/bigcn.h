@@ -78,7 +78,13 @@ enum {
      * expanded to +1 / -1 bytes in shared memory; the same integers) for layers with d_in <= 256 and
      * d_out <= 256 and at least 2^20 outputs, on the XOR / bit-count pipe otherwise; 1 = always on the
      * XOR / bit-count pipe; 2 = tensor cores for every layer with d_in <= 256 and d_out <= 256. */
-    BIGCN_OPT_CONTRACTION = 3
+    BIGCN_OPT_CONTRACTION = 3,
+    /* How rows of 129..256 signed bytes (zeta formats 3 and 5) are aggregated.  0 = default and 2: as exact integer
+     * products on the tensor cores (mma.sync s8 x s8 -> s32: the edge weights of up to 32 stored entries of a row
+     * in 28..31-bit fixed point against a common power of two, split into four signed base-256 digits; the digit
+     * sums recombined in fp32 when the row ends); 1 = the fp32 FMA stream (bytes converted to fp32 one by one;
+     * with format 5 this stream takes the edge values as non-negative). */
+    BIGCN_OPT_BYTE_AGGREGATION = 4
 };
 
 /* Context: binds a device and a stream.  `cuda_stream` is a cudaStream_t (0 = default stream). */

@@ -20,6 +20,7 @@ struct bigcn_ctx {
     int zeta_format;             // 0 = auto
     int64_t long_row;            // 0 = default
     int contraction;             // 0 = auto, 1 = bit-count pipe, 2 = tensor cores wherever covered
+    int byte_path;               // aggregation of 129..256 byte columns: 0 / 2 = integer tensor-core products, 1 = fp32 FMA stream
     cudaEvent_t ev[2 * BIGCN_MAX_LAYERS + 2];
     bool ev_ready;
 };
@@ -154,6 +155,7 @@ bigcn_status run_layer(bigcn_ctx* ctx, const bigcn_graph* g, const bigcn_layer* 
     a.node_w = half ? nws : in_beta;
     a.col_w = layer->alpha;
     a.half_dots = half;
+    a.byte_path = ctx->byte_path;
     a.col_b0 = col_b0;
     a.h_out = h_out;
     a.ldh = ldh;
@@ -342,6 +344,10 @@ bigcn_status bigcn_set_option(bigcn_ctx* ctx, int32_t option, int64_t value)
         case BIGCN_OPT_CONTRACTION:
             if (value < 0 || value > 2) return fail(ctx, BIGCN_ERR_SHAPE, "contraction path %lld not in 0..2", (long long)value);
             ctx->contraction = (int)value;
+            return BIGCN_OK;
+        case BIGCN_OPT_BYTE_AGGREGATION:
+            if (value < 0 || value > 2) return fail(ctx, BIGCN_ERR_SHAPE, "byte aggregation path %lld not in 0..2", (long long)value);
+            ctx->byte_path = (int)value;
             return BIGCN_OK;
     }
     return fail(ctx, BIGCN_ERR_UNSUPPORTED, "unknown option %d", option);
@@ -859,6 +865,7 @@ bigcn_status bigcn_sage_layer_forward(bigcn_ctx* ctx, const bigcn_graph* mean_gr
     a.node_w = in_beta;
     a.col_w = nbr_layer->alpha;
     a.add = zeta_self;
+    a.byte_path = ctx->byte_path;
     a.ld_add = ld_self;
     a.h_out = h_out;
     a.ldh = ldh;

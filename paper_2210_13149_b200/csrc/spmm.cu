@@ -93,11 +93,13 @@ struct SpmmDev {
     const float* val;
     const uint4* zeta;       // rows of nv 16-byte vectors
     int nv;                  // vectors per zeta row
+    int nv_fin;              // groups of Elt<T>::kPerVec columns the row epilogue covers (nv, unless the epilogue's element type differs)
     int d_out;
     const float* node_w;     // nullable
     const float* col_w;      // nullable
     const float* col_b0;     // half-dot bytes only: per-column first weight sign (0 where none)
     int half_dots;           // zeta holds s = (dot' - 1) / 2; node_w carries the first feature sign
+    int byte_path;           // 129..256 byte columns: 0 / 2 integer tensor-core products, 1 the FMA stream
     const float* add;        // nullable: fp32 [n x ld_add] added to the aggregated row (after col_w)
     int64_t ld_add;
     float* h_out;
@@ -200,7 +202,7 @@ __device__ __forceinline__ void finish_row(const SpmmDev& p, const float* ctab, 
             for (int i = 0; i < EPV; ++i)
                 if (col0 + i < p.d_out) x[i] += __ldg(p.add + row * p.ld_add + col0 + i);
         }
-        if (p.h_out && g == 0 && vec < p.nv) {
+        if (p.h_out && g == 0 && vec < p.nv_fin) {
             float* dst = p.h_out + row * p.ldh + col0;
             if (EPV == 4 && p.h_vec && col0 + 3 < p.d_out) {
                 *reinterpret_cast<float4*>(dst) = make_float4(x[0], x[1], x[2], x[3]);
@@ -226,14 +228,14 @@ __device__ __forceinline__ void finish_row(const SpmmDev& p, const float* ctab, 
                 if (xh >= 0.f) bits |= 1u << i;
                 l1c += fabsf(xh);
             }
-            if (vec < p.nv) l1 += l1c;            // lanes past the last vector accumulated nothing meaningful
+            if (vec < p.nv_fin) l1 += l1c;            // lanes past the last vector accumulated nothing meaningful
             const int n_valid = min(max(p.d_out - col0, 0), EPV);            // padding columns pack as 0
             bits &= (n_valid >= 32) ? 0xffffffffu : ((1u << n_valid) - 1u);
             uint32_t word = bits << ((col0) & 31);
 #pragma unroll
             for (int o = 1; o < LW; o <<= 1) word |= __shfl_xor_sync(0xffffffffu, word, o);
             const int widx = col0 >> 5;
-            if (g == 0 && (l % LW) == 0 && vec < p.nv && widx < p.next_stride)
+            if (g == 0 && (l % LW) == 0 && vec < p.nv_fin && widx < p.next_stride)
                 p.next_bits[row * p.next_stride + widx] = word;
         }
     }
@@ -788,6 +790,364 @@ __device__ __forceinline__ void stream_rows_multi(const SpmmDev& p, uint4* ring,
     cp_async_wait<0>();
 }
 
+// ---- rows of signed bytes on the integer tensor-core path -------------------------------------------------------
+//
+// For 129..256 byte columns the aggregation of one output row, sum_e w_e s_e[j], is computed as exact integer
+// products: within a segment of a row the weights are written in fixed point against a common power of two S
+// (q_e = trunc(w_e 2^31 / S), |q_e| < 2^30, at least 28 significant bits for the largest weight of the segment's
+// first window), q_e is split into four balanced base-256 digits, and a window of up to 32 stored entries of ONE row
+// becomes one K = 32 step of mma.sync.m16n8k32 (s8 x s8 -> s32): rows 0..3 of the A operand hold the four digits of
+// the 32 weights, the B operand holds the 32 gathered byte rows (8 columns per instruction, 32 instructions per
+// window for 256 columns), rows 0..3 of the accumulator hold the four digit sums.  When a row (or a segment) ends,
+// the digit sums are recombined in fp32 and scaled by S 2^-31.  The gathered rows never pass through a byte -> float
+// conversion: per stored entry the kernel issues about a third of the instructions of the FMA stream.
+//
+// The B fragment wants, in one register, the same column of four consecutive entries; the gathered rows sit in
+// shared memory entry by entry, so a lane reads 16 columns of four entries (4 x 16 bytes) and transposes 4 x 4 bytes
+// with byte permutes.  Which accumulator a column lands in is a fixed permutation that the recombination undoes.
+// A window's slot holds 32 rows of 256 bytes; 16-byte chunk c of entry e sits at chunk c ^ (2 ((e / 4) % 4)), which
+// makes both the asynchronous copies and the fragment reads free of bank conflicts.  A new segment starts with every
+// row, when a window holds a weight too large for the current S, and every 2,048 windows (so that the 32-bit digit
+// sums cannot overflow).
+constexpr int kImmaWarps = 8;
+constexpr int kImmaThreads = kImmaWarps * kWarp;
+constexpr int kImmaNG = 3;                                    // windows in a warp's ring (two in flight while one retires)
+constexpr int kWinData = 32 * 256;                            // gathered rows of a window
+constexpr int kWinQ = kWinData;                               // uint32[32]: the digits of the window's weights
+constexpr int kWinW = kWinData + 128;                         // float[2][32]: the weights, plain and with the first feature sign
+constexpr int kWinInfo = kWinData + 384;                      // int4: descriptor, scale bits
+constexpr int kWinBytes = kWinData + 384 + 32;
+constexpr int kStagePitch = 324;                              // ints per digit in the recombination buffer (16 chunks of 20)
+constexpr int kSegHeadroom = 3;                               // S = 2^(3+1) times the power of two below the first window's largest weight
+constexpr int kSegMaxWindows = 2048;
+enum : int { kWinCnt = 63, kWinLast = 64, kWinFirst = 128, kWinValid = 256, kWinSegEnd = 512 };
+
+__device__ __forceinline__ void mma_s8_k32(int (&c)[2], uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi)
+{
+    int unused0, unused1;                                     // rows 8..15 of the tile: the A operand has zeros there
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %10, %10};\n"
+        : "+r"(c[0]), "+r"(c[1]), "=r"(unused0), "=r"(unused1)
+        : "r"(a_lo), "r"(0), "r"(a_hi), "r"(0), "r"(b_lo), "r"(b_hi), "r"(0));
+}
+
+// out[c] = (r0.byte c, r1.byte c, r2.byte c, r3.byte c)
+__device__ __forceinline__ void transpose_4x4_bytes(uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3, uint32_t* out)
+{
+    const uint32_t t0 = __byte_perm(r0, r1, 0x5140), t1 = __byte_perm(r2, r3, 0x5140);
+    const uint32_t t2 = __byte_perm(r0, r1, 0x7362), t3 = __byte_perm(r2, r3, 0x7362);
+    out[0] = __byte_perm(t0, t1, 0x5410);
+    out[1] = __byte_perm(t0, t1, 0x7632);
+    out[2] = __byte_perm(t2, t3, 0x5410);
+    out[3] = __byte_perm(t2, t3, 0x7632);
+}
+
+// Streams the stored entries [e0, e0 + n_ent) of rows [row_lo, row_hi) (kPartial: a slice of one long row, whose
+// sum is left in `accf`) through the warp's ring of windows.  Lane L ends up with columns 8 L .. 8 L + 7 of a row.
+// Per iteration, oldest first: retire window it - 2 - NG (products, and the row epilogue where a row ends), issue
+// the gathers of window it - 2 into the slot just freed, fetch the node factors of window it - 1, and lay out
+// window `it` (its column indices and values).
+template <bool kFull, bool kPartial, bool kHalf>
+__device__ __forceinline__ void stream_rows_imma(const SpmmDev& p, unsigned char* ring, const float* ctab, int lane,
+                                                 int64_t e0, int n_ent, int64_t warp_row0, int row_lo, int row_hi,
+                                                 int rp_rel, float (&accf)[1][8])
+{
+    constexpr int NG = kImmaNG;
+    const int g = lane >> 2, qq = lane & 3;                   // fragment coordinates
+    const int h = lane >> 4, l = lane & 15;                   // gather coordinates: entry parity, 16-byte chunk
+    const int32_t* cols = p.colidx + e0;
+    const float* vals = p.val + e0;
+    auto row_end_of = [&](int r) { return kPartial ? n_ent : __shfl_sync(0xffffffffu, rp_rel, r + 1); };
+    const uint32_t ring_sa = (uint32_t)__cvta_generic_to_shared(ring);
+    const char* zeta_l = reinterpret_cast<const char*>(p.zeta) + l * 16;
+    const uint32_t row_bytes = (uint32_t)p.nv * 16u;
+    const bool lact = kFull || l < p.nv;
+    const uint32_t frag_off = (uint32_t)(4 * qq) * 256u + (uint32_t)((g ^ (2 * qq)) << 4);   // entry 4 qq, chunk g
+
+    // layout cursor
+    int ie = 0, ir = row_lo, iend = row_end_of(row_lo);
+    bool ifirst = true, more = row_lo < row_hi;
+    int nwin = 0;
+    // windows between the stages
+    int n_desc = 0, n_col = 0, i_desc = 0, i_col = 0;
+    float n_val = 0.f, i_val = 0.f, i_nw = 1.f;
+    // issue side: the current segment
+    int es_lim = 0, seg_windows = 0;
+    // retire side
+    int rr = row_lo;
+    int C[2][16][2];
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+        for (int t = 0; t < 16; ++t) C[a][t][0] = C[a][t][1] = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) accf[0][i] = 0.f;
+    float wsum = 0.f, wsgn = 0.f;
+
+    for (int it = 0;; ++it) {
+        const int kr = it - 2 - NG;
+        if (!more && kr >= nwin) break;
+        const int sl = it % NG;                               // slot retired and refilled in this iteration
+        unsigned char* slot = ring + sl * kWinBytes;
+        if (kr >= 0) {
+            // ---- retire window kr
+            cp_async_wait<NG - 1>();
+            __syncwarp();
+            const int2 info = *reinterpret_cast<const int2*>(slot + kWinInfo);
+            uint32_t a_lo, a_hi;
+            {
+                const uint4 q0 = *reinterpret_cast<const uint4*>(slot + kWinQ + 16 * qq);
+                const uint4 q1 = *reinterpret_cast<const uint4*>(slot + kWinQ + 64 + 16 * qq);
+                const uint32_t sel = (uint32_t)(g & 3) | ((uint32_t)(4 + (g & 3)) << 4);   // digit g of two words
+                a_lo = __byte_perm(__byte_perm(q0.x, q0.y, sel), __byte_perm(q0.z, q0.w, sel), 0x5410);
+                a_hi = __byte_perm(__byte_perm(q1.x, q1.y, sel), __byte_perm(q1.z, q1.w, sel), 0x5410);
+                if (g >= 4) a_lo = a_hi = 0u;
+            }
+#pragma unroll
+            for (int hx = 0; hx < 2; ++hx) {
+                uint32_t bf[2][16];
+#pragma unroll
+                for (int kh = 0; kh < 2; ++kh) {
+                    uint4 r[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        r[j] = *reinterpret_cast<const uint4*>(slot + frag_off + hx * 128 + kh * 4096 + j * 256);
+                    transpose_4x4_bytes(r[0].x, r[1].x, r[2].x, r[3].x, &bf[kh][0]);
+                    transpose_4x4_bytes(r[0].y, r[1].y, r[2].y, r[3].y, &bf[kh][4]);
+                    transpose_4x4_bytes(r[0].z, r[1].z, r[2].z, r[3].z, &bf[kh][8]);
+                    transpose_4x4_bytes(r[0].w, r[1].w, r[2].w, r[3].w, &bf[kh][12]);
+                }
+#pragma unroll
+                for (int t = 0; t < 16; ++t) mma_s8_k32(C[hx][t], a_lo, a_hi, bf[0][t], bf[1][t]);
+            }
+            if (kHalf) {
+                const float* wf = reinterpret_cast<const float*>(slot + kWinW);
+                wsum += wf[lane];
+                wsgn += wf[32 + lane];
+            }
+            if (info.x & (kWinLast | kWinSegEnd)) {
+                // ---- the segment ends: recombine the digit sums (through the window's data area, free now)
+                __syncwarp();
+                int* stage = reinterpret_cast<int*>(slot);
+                if (g < 4) {
+#pragma unroll
+                    for (int hx = 0; hx < 2; ++hx)
+#pragma unroll
+                        for (int b = 0; b < 2; ++b) {
+                            int* dst = stage + g * kStagePitch + (2 * qq + b + 8 * hx) * 20;
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                *reinterpret_cast<int4*>(dst + 4 * i) =
+                                    make_int4(C[hx][4 * i][b], C[hx][4 * i + 1][b], C[hx][4 * i + 2][b], C[hx][4 * i + 3][b]);
+                        }
+                }
+                __syncwarp();
+                const float scale = __int_as_float(info.y);
+                const int* src = stage + (lane >> 1) * 20 + 8 * (lane & 1);
+                int d[4][8];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int4 u0 = *reinterpret_cast<const int4*>(src + k * kStagePitch);
+                    const int4 u1 = *reinterpret_cast<const int4*>(src + k * kStagePitch + 4);
+                    d[k][0] = u0.x, d[k][1] = u0.y, d[k][2] = u0.z, d[k][3] = u0.w;
+                    d[k][4] = u1.x, d[k][5] = u1.y, d[k][6] = u1.z, d[k][7] = u1.w;
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float f = fmaf((float)d[3][i], 16777216.f, (float)d[2][i] * 65536.f) + fmaf((float)d[1][i], 256.f, (float)d[0][i]);
+                    accf[0][i] = fmaf(scale, f, accf[0][i]);
+                }
+#pragma unroll
+                for (int a = 0; a < 2; ++a)
+#pragma unroll
+                    for (int t = 0; t < 16; ++t) C[a][t][0] = C[a][t][1] = 0;
+                if (info.x & kWinLast) {                      // the row is complete
+                    if (kHalf) {
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+                            wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
+                            wsgn += __shfl_xor_sync(0xffffffffu, wsgn, o);
+                        }
+                    }
+                    if (kPartial) {
+                        if (kHalf) {                          // a slice of a long row: hand back the reconstructed partial sums
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                accf[0][i] = fmaf(2.f, accf[0][i], fmaf(ctab[3 * 256 + 8 * lane + i], wsgn, wsum));
+                        }
+                        return;
+                    }
+                    finish_row<__half, 1, 32, kHalf>(p, ctab, warp_row0 + rr, lane, accf, wsum, wsgn);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) accf[0][i] = 0.f;
+                    wsum = 0.f;
+                    wsgn = 0.f;
+                    ++rr;
+                }
+            }
+            __syncwarp();                                     // all lanes are done with this slot
+        }
+        if (i_desc & kWinValid) {
+            // ---- issue window it - 2 into the slot: fixed-point weights, then the gathers
+            const int cnt = i_desc & kWinCnt;
+            const float wa = i_val * (kHalf ? fabsf(i_nw) : i_nw);            // the weight of the byte row
+            const uint32_t mbits = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(wa)));
+            const int ew = (int)(mbits >> 23);                                // biased exponent of the window's largest weight
+            const bool newseg = (i_desc & kWinFirst) || ew >= es_lim || seg_windows >= kSegMaxWindows;
+            if (newseg) {
+                es_lim = min(max(ew + kSegHeadroom, 31), 254);                // S = 2^(es_lim + 1 - 127)
+                seg_windows = 0;
+            }
+            ++seg_windows;
+            const float inv = __int_as_float((284 - es_lim) << 23);           // 2^31 / S
+            const int q = __float2int_rz(wa * inv);                           // |q| < 2^30 (2^28 in a segment's first window)
+            *reinterpret_cast<uint32_t*>(slot + kWinQ + 4 * lane) = ((uint32_t)q + 0x00808080u) ^ 0x00808080u;   // balanced digits
+            if (kHalf) {
+                float* wf = reinterpret_cast<float*>(slot + kWinW);
+                wf[lane] = wa;
+                wf[32 + lane] = i_val * i_nw;                                 // signed by the source's first feature sign
+            }
+            if (lane == 0) {
+                *reinterpret_cast<int2*>(slot + kWinInfo) = make_int2(i_desc, (es_lim - 30) << 23);   // scale = S 2^-31
+                if (newseg && !(i_desc & kWinFirst))                          // the window before this one closes its segment
+                    *reinterpret_cast<int*>(ring + ((it + NG - 1) % NG) * kWinBytes + kWinInfo) |= kWinSegEnd;
+            }
+            const uint32_t dsta = ring_sa + sl * kWinBytes + (uint32_t)h * 256u;
+            if (cnt == 32) {
+#pragma unroll
+                for (int b = 0; b < 16; ++b) {
+                    const uint32_t k = (uint32_t)__shfl_sync(0xffffffffu, i_col, 2 * b + h);
+                    if (lact) cp_async16_s(dsta + b * 512 + ((l ^ (((b >> 1) & 3) << 1)) << 4), zeta_l + (uint64_t)k * row_bytes);
+                }
+            } else {
+#pragma unroll
+                for (int b = 0; b < 16; ++b) {
+                    const uint32_t k = (uint32_t)__shfl_sync(0xffffffffu, i_col, 2 * b + h);
+                    if (lact && 2 * b + h < cnt) cp_async16_s(dsta + b * 512 + ((l ^ (((b >> 1) & 3) << 1)) << 4), zeta_l + (uint64_t)k * row_bytes);
+                }
+            }
+        }
+        cp_async_commit();                                    // one group per iteration, possibly empty
+        // ---- the node factors of window it - 1
+        i_desc = n_desc;
+        i_col = n_col;
+        i_val = n_val;
+        i_nw = (p.node_w && (n_desc & kWinValid)) ? __ldg(p.node_w + n_col) : 1.f;
+        // ---- lay out window `it`
+        n_desc = 0;
+        n_col = 0;
+        n_val = 0.f;
+        if (more) {
+            const int left = iend - ie;
+            const int cnt = min(32, left);
+            n_desc = cnt | (cnt == left ? kWinLast : 0) | (ifirst ? kWinFirst : 0) | kWinValid;
+            if (lane < cnt) {
+                n_col = __ldg(cols + ie + lane);
+                n_val = __ldg(vals + ie + lane);
+            }
+            ie += cnt;
+            ifirst = false;
+            ++nwin;
+            if (ie == iend) {
+                ifirst = true;
+                ++ir;
+                if (ir == row_hi) more = false;
+                else iend = row_end_of(ir);
+            }
+        }
+    }
+    cp_async_wait<0>();
+}
+
+// The kernel around stream_rows_imma: the same hand-out of row runs and the same cooperative treatment of long
+// rows as spmm_kernel.  One thread block of 8 warps per SM (the rings take most of the shared memory).
+template <bool kFull, bool kHalf>
+__global__ void __launch_bounds__(kImmaThreads, 1)
+spmm_imma_kernel(const SpmmDev p, int rows_per_warp)
+{
+    constexpr int kCols = 256;
+    extern __shared__ __align__(128) unsigned char dsmem[];
+    __shared__ int64_t long_rows[kLongQueue];
+    __shared__ int n_long;
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    unsigned char* ring = dsmem + (size_t)warp * kImmaNG * kWinBytes;
+    float* part = reinterpret_cast<float*>(dsmem);           // [kImmaWarps][kCols], reuses the rings
+    float* ctab = reinterpret_cast<float*>(dsmem + (size_t)kImmaWarps * kImmaNG * kWinBytes);   // [4][kCols]
+    fill_col_table<kCols>(p, ctab);
+    if (threadIdx.x == 0) n_long = 0;
+    __syncthreads();
+
+    const int64_t n_runs = ceil_div(p.n, rows_per_warp);
+    float accf[1][8];
+    for (;;) {
+        int64_t run = 0;
+        if (lane == 0) run = atomicAdd(p.run_counter, 1);
+        run = __shfl_sync(0xffffffffu, run, 0);
+        if (run >= n_runs) break;
+        const int64_t warp_row0 = run * rows_per_warp;
+        const int n_rows = (int)min((int64_t)rows_per_warp, p.n - warp_row0);
+        const int64_t rp_reg = __ldg(p.rowptr + warp_row0 + min(lane, n_rows));
+        const int64_t rp_next = __shfl_down_sync(0xffffffffu, rp_reg, 1);
+        bool is_long = lane < n_rows && p.long_row > 0 && (rp_next - rp_reg) > p.long_row;
+        if (is_long) {                                        // queue it for the block; if the queue is full, stream it here
+            const int slot = atomicAdd(&n_long, 1);
+            if (slot < kLongQueue) long_rows[slot] = warp_row0 + lane;
+            else is_long = false;
+        }
+        const unsigned long_mask = __ballot_sync(0xffffffffu, is_long);
+        int ra = 0;
+        while (ra < n_rows) {                                 // runs of rows between the long ones
+            const unsigned rest = long_mask >> ra;
+            const int rl = rest ? ra + (__ffs(rest) - 1) : n_rows;
+            if (rl > ra) {
+                const int64_t e0 = __shfl_sync(0xffffffffu, rp_reg, ra);
+                const int64_t e1 = __shfl_sync(0xffffffffu, rp_reg, rl);
+                stream_rows_imma<kFull, false, kHalf>(p, ring, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl, (int)(rp_reg - e0), accf);
+            }
+            ra = rl + 1;
+        }
+    }
+    __syncthreads();
+    const int nl = min(n_long, kLongQueue);
+    for (int q = 0; q < nl; ++q) {                            // long rows of this block, each by all warps together
+        const int64_t lrow = long_rows[q];
+        const int64_t ls = __ldg(p.rowptr + lrow), le = __ldg(p.rowptr + lrow + 1);
+        const int64_t slice = round_up(ceil_div(le - ls, kImmaWarps), 32);
+        const int64_t s0 = min(le, ls + warp * slice), s1 = min(le, s0 + slice);
+        stream_rows_imma<kFull, true, kHalf>(p, ring, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, accf);
+        __syncthreads();                                      // every ring is idle: reuse them for the partial sums
+#pragma unroll
+        for (int i = 0; i < 8; ++i) part[warp * kCols + 8 * lane + i] = accf[0][i];
+        __syncthreads();
+        if (warp == 0) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float t = 0.f;
+                for (int w = 0; w < kImmaWarps; ++w) t += part[w * kCols + 8 * lane + i];
+                accf[0][i] = t;
+            }
+            finish_row<__half, 1, 32>(p, ctab, lrow, lane, accf);
+        }
+        __syncthreads();
+    }
+}
+
+template <bool kFull, bool kHalf>
+cudaError_t launch_imma(cudaStream_t s, SpmmDev p)
+{
+    constexpr size_t smem = (size_t)kImmaWarps * kImmaNG * kWinBytes + 4 * 256 * sizeof(float);
+    p.nv_fin = 2 * p.nv;                                      // the row epilogue works on groups of 8 columns
+    const int rows_per_warp = (int)std::min<int64_t>(kMaxRowsPerWarp, std::max<int64_t>(1, p.n / (kImmaWarps * 148 * 8)));
+    cudaError_t e = cudaFuncSetAttribute(spmm_imma_kernel<kFull, kHalf>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(p.run_counter, 0, sizeof(int), s);
+    if (e != cudaSuccess) return e;
+    const int64_t wanted = ceil_div(ceil_div(p.n, rows_per_warp), kImmaWarps);
+    const unsigned grid = (unsigned)std::min<int64_t>(wanted, 148);
+    spmm_imma_kernel<kFull, kHalf><<<grid, kImmaThreads, smem, s>>>(p, rows_per_warp);
+    return cudaGetLastError();
+}
+
 // Thread blocks per SM the kernel is compiled for (register budget) and launched with (grid size).
 template <int NCH, int LPR, bool kAligned>
 constexpr int spmm_blocks_per_sm()
@@ -932,6 +1292,10 @@ cudaError_t dispatch(cudaStream_t s, const SpmmDev& p, double mean_row)
     if (nv <= 8) return launch_one<T, 1, 8>(s, p);
     if (nv <= 16) {
         if constexpr (sizeof(T) == 1) {
+            if (nv > 8 && p.byte_path != 1) {                  // integer tensor-core products
+                if (p.half_dots) return nv == 16 ? launch_imma<true, true>(s, p) : launch_imma<false, true>(s, p);
+                return nv == 16 ? launch_imma<true, false>(s, p) : launch_imma<false, false>(s, p);
+            }
             if (p.half_dots) return nv == 16 ? launch_one<T, 1, 16, true, true, true>(s, p) : launch_one<T, 1, 16, false, true, true>(s, p);
             // (8 lanes per row with two vectors each, four entries per position -- launch_one<T, 2, 8, .., true> -- halves
             // the bookkeeping per entry again but needs 123 registers: 7.7 ms against 6.4 ms on c5 layer 0; not used)
@@ -966,12 +1330,14 @@ cudaError_t launch_spmm(cudaStream_t s, const SpmmArgs& a, int* launches)
     p.val = a.val;
     p.zeta = reinterpret_cast<const uint4*>(a.zeta);
     p.nv = (int)(a.ldz * zeta_elt_bytes(a.fmt) / 16);
+    p.nv_fin = p.nv;
     p.d_out = a.d_out;
     p.node_w = a.fmt == kZetaF32 ? nullptr : a.node_w;
     p.col_w = a.fmt == kZetaF32 ? nullptr : a.col_w;
     p.add = a.add;
     p.col_b0 = a.half_dots ? a.col_b0 : nullptr;
     p.half_dots = a.half_dots ? 1 : 0;
+    p.byte_path = a.byte_path;
     if (a.half_dots && (a.fmt != kZetaI8 || p.nv > 16 || p.nv <= 8 || !a.col_b0 || !a.node_w)) return cudaErrorInvalidValue;   // 129..256 byte columns only
     p.ld_add = a.ld_add;
     p.h_out = a.h_out;

@@ -179,6 +179,76 @@ def test_half_dot_bytes_at_the_ends_of_the_byte_range(ctx, B):
     assert_close(out["h"], t.H_out, "H' (half-dot bytes, extreme dots)")
 
 
+BYTE_ROW_SHAPES = [(3, 500, 6000, 100, 200), (3, 300, 3000, 127, 256), (3, 40000, 300000, 64, 130),
+                   (5, 500, 6000, 129, 200), (5, 300, 3000, 256, 256), (5, 40000, 300000, 256, 256)]
+
+
+@pytest.mark.parametrize("fmt,n,e,d_in,d_out", BYTE_ROW_SHAPES)
+def test_byte_rows_on_the_fma_stream(ctx, B, fmt, n, e, d_in, d_out):
+    """The library's other aggregation of 129..256 byte columns (bytes converted to fp32, packed FMAs) beside the
+    default integer tensor-core products."""
+    ctx.set_option(B.OPT_BYTE_AGGREGATION, 1)
+    try:
+        check_layer_forward(ctx, B, fmt, n, e, d_in, d_out)
+    finally:
+        ctx.set_option(B.OPT_BYTE_AGGREGATION, 0)
+
+
+@pytest.mark.parametrize("fmt,d_in", [(3, 100), (5, 256), (5, 201)])
+@pytest.mark.parametrize("span", [0, 12, 40])
+def test_byte_rows_signed_edge_values_of_wide_range(ctx, B, fmt, d_in, span):
+    """Edge values of both signs spread over 2^-span .. 2^span inside every row: the fixed-point weights of the
+    integer products open new segments as larger weights arrive, and the sign rides in the digits."""
+    n, d_out = 600, 256
+    rng = np.random.default_rng(5 + span)
+    _, _, g = small_graph(n, 24000, 31)                      # about 80 entries per row: several windows
+    g.val[:] = (g.val * np.exp2(rng.integers(-span, span + 1, g.val.shape)) * rng.choice([-1.0, 1.0], g.val.shape)).astype(np.float32)
+    H = rng.standard_normal((n, d_in)).astype(np.float32)
+    W = (rng.standard_normal((d_in, d_out)) * d_in ** -0.5).astype(np.float32)
+    t = oracle.layer_forward(g, oracle.Layer(W), H)
+    ctx.set_option(B.OPT_ZETA_FORMAT, fmt)
+    G = device_graph(B, g)
+    layer = B.make_layer(d_in, d_out, bits_to_dev(t.bitsT), dev(t.alpha))
+    out = ctx.layer_forward(G, layer, bits_to_dev(t.bits), dev(t.beta), want_h=True, debug=True)
+    ctx.sync_check()
+    assert np.array_equal(out["dot"].cpu().numpy(), t.dot)
+    ref = t.H_out
+    got = out["h"].cpu().numpy().astype(np.float64)
+    # the sum of one row in fp32 is good to a few ulps of its largest term, whatever the cancellation
+    A = np.zeros((n, n)); 
+    for i in range(n):
+        A[i, g.colidx[g.rowptr[i]:g.rowptr[i + 1]]] = np.abs(g.val[g.rowptr[i]:g.rowptr[i + 1]])
+    bound = (A @ (np.abs(t.dot) * t.beta[:, None].astype(np.float64))) * np.abs(t.alpha)[None, :]
+    assert np.all(np.abs(got - ref) <= 1e-5 * np.abs(ref) + 4e-6 * bound + 1e-30)
+
+
+def test_half_dot_bytes_hub_row_split_across_the_block(ctx, B):
+    """One row with n entries under half-dot bytes: slices of a long row hand back reconstructed partial sums."""
+    n, d_in, d_out = 3000, 256, 256
+    rng = np.random.default_rng(78)
+    rp, ci = synth.power_law_graph(n, 30000, 78)
+    src, dst = synth.edge_list(rp, ci)
+    src = np.concatenate([src, np.zeros(n - 1, np.int32)])
+    dst = np.concatenate([dst, np.arange(1, n, dtype=np.int32)])
+    g = oracle.normalize_adjacency(n, src, dst)
+    H = rng.standard_normal((n, d_in)).astype(np.float32)
+    W = (rng.standard_normal((d_in, d_out)) * 0.1).astype(np.float32)
+    t = oracle.layer_forward(g, oracle.Layer(W), H)
+    ctx.set_option(B.OPT_ZETA_FORMAT, 5)
+    G = device_graph(B, g)
+    layer = B.make_layer(d_in, d_out, bits_to_dev(t.bitsT), dev(t.alpha))
+    for path in (0, 1):
+        ctx.set_option(B.OPT_BYTE_AGGREGATION, path)
+        try:
+            for thr in (0, 8, 100000):
+                ctx.set_option(B.OPT_LONG_ROW, thr)
+                out = ctx.layer_forward(G, layer, bits_to_dev(t.bits), dev(t.beta), want_h=True)
+                assert_close(out["h"], t.H_out, "H' (path %d, threshold %d)" % (path, thr))
+        finally:
+            ctx.set_option(B.OPT_BYTE_AGGREGATION, 0)
+            ctx.set_option(B.OPT_LONG_ROW, 0)
+
+
 # shapes the tensor-core contraction covers (d_in, d_out <= 256): tile tails, one row, several tiles per CTA
 TC_SHAPES = [(5, 6, 256, 256), (127, 900, 256, 256), (128, 900, 100, 256), (129, 900, 256, 47), (1000, 9000, 200, 130),
              (40000, 200000, 256, 256), (39000, 150000, 100, 64)]
