@@ -794,7 +794,7 @@ __device__ __forceinline__ void stream_rows_multi(const SpmmDev& p, uint4* ring,
 //
 // For 129..256 byte columns the aggregation of one output row, sum_e w_e s_e[j], is computed as exact integer
 // products: within a segment of a row the weights are written in fixed point against a common power of two S
-// (q_e = trunc(w_e 2^31 / S), |q_e| < 2^30, at least 28 significant bits for the largest weight of the segment's
+// (q_e = trunc(w_e 2^31 / S), |q_e| < 2^30, at least 29 significant bits for the largest weight of the segment's
 // first window), q_e is split into four balanced base-256 digits, and a window of up to 32 stored entries of ONE row
 // becomes one K = 32 step of mma.sync.m16n8k32 (s8 x s8 -> s32): rows 0..3 of the A operand hold the four digits of
 // the 32 weights, the B operand holds the 32 gathered byte rows (8 columns per instruction, 32 instructions per
@@ -818,7 +818,7 @@ constexpr int kWinW = kWinData + 128;                         // float[2][32]: t
 constexpr int kWinInfo = kWinData + 384;                      // int4: descriptor, scale bits
 constexpr int kWinBytes = kWinData + 384 + 32;
 constexpr int kStagePitch = 324;                              // ints per digit in the recombination buffer (16 chunks of 20)
-constexpr int kSegHeadroom = 3;                               // S = 2^(3+1) times the power of two below the first window's largest weight
+constexpr int kSegHeadroom = 2;                               // S = 2^(2+1) times the power of two below the first window's largest weight
 constexpr int kSegMaxWindows = 2048;
 enum : int { kWinCnt = 63, kWinLast = 64, kWinFirst = 128, kWinValid = 256, kWinSegEnd = 512 };
 
@@ -999,7 +999,7 @@ __device__ __forceinline__ void stream_rows_imma(const SpmmDev& p, unsigned char
             }
             ++seg_windows;
             const float inv = __int_as_float((284 - es_lim) << 23);           // 2^31 / S
-            const int q = __float2int_rz(wa * inv);                           // |q| < 2^30 (2^28 in a segment's first window)
+            const int q = __float2int_rz(wa * inv);                           // |q| < 2^30 (2^29 in a segment's first window)
             *reinterpret_cast<uint32_t*>(slot + kWinQ + 4 * lane) = ((uint32_t)q + 0x00808080u) ^ 0x00808080u;   // balanced digits
             if (kHalf) {
                 float* wf = reinterpret_cast<float*>(slot + kWinW);
