@@ -796,13 +796,13 @@ __device__ __forceinline__ void stream_rows_multi(const SpmmDev& p, uint4* ring,
 // products: within a segment of a row the weights are written in fixed point against a common power of two S
 // (q_e = trunc(w_e 2^31 / S), |q_e| < 2^30, at least 29 significant bits for the largest weight of the segment's
 // first window), q_e is split into four balanced base-256 digits, and a window of up to 32 stored entries of ONE row
-// becomes one K = 32 step of mma.sync.m16n8k32 (s8 x s8 -> s32): rows 0..3 of the A operand hold the four digits of
-// the 32 weights, the B operand holds the 32 gathered byte rows (8 columns per instruction, 32 instructions per
-// window for 256 columns), rows 0..3 of the accumulator hold the four digit sums.  When a row (or a segment) ends,
+// becomes one K = 32 step of mma.sync.m16n8k32 (s8 x s8 -> s32): the A operand holds 16 columns of the 32 gathered
+// byte rows (16 instructions per window for 256 columns), columns 0..3 of the B operand hold the four digits of the
+// 32 weights, columns 0..3 of the accumulator hold the four digit sums of the 16 columns.  When a row (or a segment) ends,
 // the digit sums are recombined in fp32 and scaled by S 2^-31.  The gathered rows never pass through a byte -> float
 // conversion: per stored entry the kernel issues about a third of the instructions of the FMA stream.
 //
-// The B fragment wants, in one register, the same column of four consecutive entries; the gathered rows sit in
+// The A fragment wants, in one register, the same column of four consecutive entries; the gathered rows sit in
 // shared memory entry by entry, so a lane reads 16 columns of four entries (4 x 16 bytes) and transposes 4 x 4 bytes
 // with byte permutes.  Which accumulator a column lands in is a fixed permutation that the recombination undoes.
 // A window's slot holds 32 rows of 256 bytes; 16-byte chunk c of entry e sits at chunk c ^ (2 ((e / 4) % 4)), which
@@ -822,12 +822,11 @@ constexpr int kSegHeadroom = 2;                               // S = 2^(2+1) tim
 constexpr int kSegMaxWindows = 2048;
 enum : int { kWinCnt = 63, kWinLast = 64, kWinFirst = 128, kWinValid = 256, kWinSegEnd = 512 };
 
-__device__ __forceinline__ void mma_s8_k32(int (&c)[2], uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi)
+__device__ __forceinline__ void mma_s8_k32(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
 {
-    int unused0, unused1;                                     // rows 8..15 of the tile: the A operand has zeros there
-    asm("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %10, %10};\n"
-        : "+r"(c[0]), "+r"(c[1]), "=r"(unused0), "=r"(unused1)
-        : "r"(a_lo), "r"(0), "r"(a_hi), "r"(0), "r"(b_lo), "r"(b_hi), "r"(0));
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};\n"
+        : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 // out[c] = (r0.byte c, r1.byte c, r2.byte c, r3.byte c)
@@ -874,11 +873,9 @@ __device__ __forceinline__ void stream_rows_imma(const SpmmDev& p, unsigned char
     int es_lim = 0, seg_windows = 0;
     // retire side
     int rr = row_lo;
-    int C[2][16][2];
+    int C[16][4];                                             // tile t: columns 16 x + t; [0], [1]: x = g, [2], [3]: x = g + 8
 #pragma unroll
-    for (int a = 0; a < 2; ++a)
-#pragma unroll
-        for (int t = 0; t < 16; ++t) C[a][t][0] = C[a][t][1] = 0;
+    for (int t = 0; t < 16; ++t) C[t][0] = C[t][1] = C[t][2] = C[t][3] = 0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) accf[0][i] = 0.f;
     float wsum = 0.f, wsgn = 0.f;
@@ -893,31 +890,42 @@ __device__ __forceinline__ void stream_rows_imma(const SpmmDev& p, unsigned char
             cp_async_wait<NG - 1>();
             __syncwarp();
             const int2 info = *reinterpret_cast<const int2*>(slot + kWinInfo);
-            uint32_t a_lo, a_hi;
+            uint32_t b_lo, b_hi;                              // B operand: column n = digit n of the 32 weights (n < 4)
             {
                 const uint4 q0 = *reinterpret_cast<const uint4*>(slot + kWinQ + 16 * qq);
                 const uint4 q1 = *reinterpret_cast<const uint4*>(slot + kWinQ + 64 + 16 * qq);
                 const uint32_t sel = (uint32_t)(g & 3) | ((uint32_t)(4 + (g & 3)) << 4);   // digit g of two words
-                a_lo = __byte_perm(__byte_perm(q0.x, q0.y, sel), __byte_perm(q0.z, q0.w, sel), 0x5410);
-                a_hi = __byte_perm(__byte_perm(q1.x, q1.y, sel), __byte_perm(q1.z, q1.w, sel), 0x5410);
-                if (g >= 4) a_lo = a_hi = 0u;
+                b_lo = __byte_perm(__byte_perm(q0.x, q0.y, sel), __byte_perm(q0.z, q0.w, sel), 0x5410);
+                b_hi = __byte_perm(__byte_perm(q1.x, q1.y, sel), __byte_perm(q1.z, q1.w, sel), 0x5410);
+                if (g >= 4) b_lo = b_hi = 0u;
             }
+            {
+                // A operand (16 columns x 32 entries): row g = a column of chunk g, row g + 8 = a column of chunk g + 8
+                uint4 r[2][2][4];                             // [chunk g / g + 8][entries 4 qq.. / 16 + 4 qq..][entry]
 #pragma unroll
-            for (int hx = 0; hx < 2; ++hx) {
-                uint32_t bf[2][16];
+                for (int hx = 0; hx < 2; ++hx)
 #pragma unroll
-                for (int kh = 0; kh < 2; ++kh) {
-                    uint4 r[4];
+                    for (int kh = 0; kh < 2; ++kh)
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        r[j] = *reinterpret_cast<const uint4*>(slot + frag_off + hx * 128 + kh * 4096 + j * 256);
-                    transpose_4x4_bytes(r[0].x, r[1].x, r[2].x, r[3].x, &bf[kh][0]);
-                    transpose_4x4_bytes(r[0].y, r[1].y, r[2].y, r[3].y, &bf[kh][4]);
-                    transpose_4x4_bytes(r[0].z, r[1].z, r[2].z, r[3].z, &bf[kh][8]);
-                    transpose_4x4_bytes(r[0].w, r[1].w, r[2].w, r[3].w, &bf[kh][12]);
+                        for (int j = 0; j < 4; ++j)
+                            r[hx][kh][j] = *reinterpret_cast<const uint4*>(slot + frag_off + hx * 128 + kh * 4096 + j * 256);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {                 // four columns of each chunk at a time
+                    uint32_t a[2][2][4];
+#pragma unroll
+                    for (int hx = 0; hx < 2; ++hx)
+#pragma unroll
+                        for (int kh = 0; kh < 2; ++kh) {
+                            const uint4* v = r[hx][kh];
+                            if (c == 0) transpose_4x4_bytes(v[0].x, v[1].x, v[2].x, v[3].x, a[hx][kh]);
+                            else if (c == 1) transpose_4x4_bytes(v[0].y, v[1].y, v[2].y, v[3].y, a[hx][kh]);
+                            else if (c == 2) transpose_4x4_bytes(v[0].z, v[1].z, v[2].z, v[3].z, a[hx][kh]);
+                            else transpose_4x4_bytes(v[0].w, v[1].w, v[2].w, v[3].w, a[hx][kh]);
+                        }
+#pragma unroll
+                    for (int tt = 0; tt < 4; ++tt)
+                        mma_s8_k32(C[4 * c + tt], a[0][0][tt], a[1][0][tt], a[0][1][tt], a[1][1][tt], b_lo, b_hi);
                 }
-#pragma unroll
-                for (int t = 0; t < 16; ++t) mma_s8_k32(C[hx][t], a_lo, a_hi, bf[0][t], bf[1][t]);
             }
             if (kHalf) {
                 const float* wf = reinterpret_cast<const float*>(slot + kWinW);
@@ -928,16 +936,16 @@ __device__ __forceinline__ void stream_rows_imma(const SpmmDev& p, unsigned char
                 // ---- the segment ends: recombine the digit sums (through the window's data area, free now)
                 __syncwarp();
                 int* stage = reinterpret_cast<int*>(slot);
-                if (g < 4) {
+                if (qq < 2) {                                 // these lanes hold digits 2 qq and 2 qq + 1
 #pragma unroll
                     for (int hx = 0; hx < 2; ++hx)
 #pragma unroll
                         for (int b = 0; b < 2; ++b) {
-                            int* dst = stage + g * kStagePitch + (2 * qq + b + 8 * hx) * 20;
+                            int* dst = stage + (2 * qq + b) * kStagePitch + (g + 8 * hx) * 20;
 #pragma unroll
                             for (int i = 0; i < 4; ++i)
                                 *reinterpret_cast<int4*>(dst + 4 * i) =
-                                    make_int4(C[hx][4 * i][b], C[hx][4 * i + 1][b], C[hx][4 * i + 2][b], C[hx][4 * i + 3][b]);
+                                    make_int4(C[4 * i][2 * hx + b], C[4 * i + 1][2 * hx + b], C[4 * i + 2][2 * hx + b], C[4 * i + 3][2 * hx + b]);
                         }
                 }
                 __syncwarp();
@@ -957,9 +965,7 @@ __device__ __forceinline__ void stream_rows_imma(const SpmmDev& p, unsigned char
                     accf[0][i] = fmaf(scale, f, accf[0][i]);
                 }
 #pragma unroll
-                for (int a = 0; a < 2; ++a)
-#pragma unroll
-                    for (int t = 0; t < 16; ++t) C[a][t][0] = C[a][t][1] = 0;
+                for (int t = 0; t < 16; ++t) C[t][0] = C[t][1] = C[t][2] = C[t][3] = 0;
                 if (info.x & kWinLast) {                      // the row is complete
                     if (kHalf) {
 #pragma unroll
