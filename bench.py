@@ -41,6 +41,8 @@ def parse_args():
                          "entropy: side benchmark of the binning entropy estimator; backward: side benchmark of Algorithm 1 "
                          "for the hidden layer of the workload")
     ap.add_argument("--zeta-format", type=int, default=0, help="0 auto, 1 fp32, 2 int16, 3 int8, 4 fp16, 5 half-dot bytes")
+    ap.add_argument("--byte-aggregation", type=int, default=0,
+                    help="rows of 129..256 bytes: 0 / 1 the fp32 FMA stream (default), 2 integer tensor-core products")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--graph", action="store_true", help="also time the forward replayed as one CUDA graph")
@@ -227,6 +229,8 @@ def run_ours(args):
     ctx = binding.BiGCN(local)
     if args.zeta_format:
         ctx.set_option(binding.OPT_ZETA_FORMAT, args.zeta_format)
+    if args.byte_aggregation:
+        ctx.set_option(binding.OPT_BYTE_AGGREGATION, args.byte_aggregation)
     G = ctx.normalize_adjacency(wl.rowptr, wl.colidx)
     n, nnz = G.n, G.nnz
     deg = torch.sort(torch.diff(G.rowptr), descending=True).values
@@ -354,6 +358,21 @@ def run_ours(args):
                 extras["spmm_fp16_rows_ms"] = "failed: %r" % (exc,)
             finally:
                 ctx.set_option(binding.OPT_ZETA_FORMAT, 0)
+        # byte rows aggregated as integer products on the tensor cores (the library's other path), for comparison
+        if args.zeta_format == 0 and args.byte_aggregation == 0:
+            try:
+                ctx.set_option(binding.OPT_BYTE_AGGREGATION, 2)
+                alt = [[] for _ in range(L)]
+                for k in range(3 + min(args.steps, 5)):
+                    _, st = ctx.forward(G, layers, X, logits, stats=True)
+                    if k >= 3:
+                        for l in range(L):
+                            alt[l].append(st.ms_spmm[l])
+                extras["spmm_integer_products_ms"] = [sum(v) / len(v) for v in alt]
+            except Exception as exc:
+                extras["spmm_integer_products_ms"] = "failed: %r" % (exc,)
+            finally:
+                ctx.set_option(binding.OPT_BYTE_AGGREGATION, 0)
         # the same contraction on the XOR / bit-count pipe (the library's other path), for comparison
         try:
             ctx.set_option(binding.OPT_CONTRACTION, 1)

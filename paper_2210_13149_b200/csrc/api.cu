@@ -20,7 +20,7 @@ struct bigcn_ctx {
     int zeta_format;             // 0 = auto
     int64_t long_row;            // 0 = default
     int contraction;             // 0 = auto, 1 = bit-count pipe, 2 = tensor cores wherever covered
-    int byte_path;               // aggregation of 129..256 byte columns: 0 / 2 = integer tensor-core products, 1 = fp32 FMA stream
+    int byte_path;               // aggregation of 129..256 byte columns: 0 / 1 = fp32 FMA stream, 2 = integer tensor-core products
     cudaEvent_t ev[2 * BIGCN_MAX_LAYERS + 2];
     bool ev_ready;
 };

@@ -54,7 +54,7 @@ struct SpmmArgs {
     const float* col_w;      // integer formats: per-column factor (alpha), applied once per output
     const float* col_b0 = nullptr;   // half-dot bytes (kZetaI8H): per-column first weight sign (0 when d_in is odd)
     bool half_dots = false;          // zeta holds s = (dot' - 1) / 2 and node_w carries the first feature sign
-    int byte_path = 0;               // rows of 129..256 bytes: 0 auto (integer tensor-core products), 1 the fp32 FMA stream, 2 tensor cores
+    int byte_path = 0;               // rows of 129..256 bytes: 0 auto (the fp32 FMA stream), 1 the fp32 FMA stream, 2 integer tensor-core products
     const float* add = nullptr;   // optional fp32 [n x ld_add] added to every aggregated row (Bi-GraphSAGE self term)
     int64_t ld_add = 0;
     float* h_out;            // nullable

@@ -99,7 +99,7 @@ struct SpmmDev {
     const float* col_w;      // nullable
     const float* col_b0;     // half-dot bytes only: per-column first weight sign (0 where none)
     int half_dots;           // zeta holds s = (dot' - 1) / 2; node_w carries the first feature sign
-    int byte_path;           // 129..256 byte columns: 0 / 2 integer tensor-core products, 1 the FMA stream
+    int byte_path;           // 129..256 byte columns: 0 / 1 the FMA stream, 2 integer tensor-core products
     const float* add;        // nullable: fp32 [n x ld_add] added to the aggregated row (after col_w)
     int64_t ld_add;
     float* h_out;
@@ -1298,7 +1298,7 @@ cudaError_t dispatch(cudaStream_t s, const SpmmDev& p, double mean_row)
     if (nv <= 8) return launch_one<T, 1, 8>(s, p);
     if (nv <= 16) {
         if constexpr (sizeof(T) == 1) {
-            if (nv > 8 && p.byte_path != 1) {                  // integer tensor-core products
+            if (nv > 8 && p.byte_path == 2) {                  // integer tensor-core products
                 if (p.half_dots) return nv == 16 ? launch_imma<true, true>(s, p) : launch_imma<false, true>(s, p);
                 return nv == 16 ? launch_imma<true, false>(s, p) : launch_imma<false, false>(s, p);
             }

@@ -184,10 +184,10 @@ BYTE_ROW_SHAPES = [(3, 500, 6000, 100, 200), (3, 300, 3000, 127, 256), (3, 40000
 
 
 @pytest.mark.parametrize("fmt,n,e,d_in,d_out", BYTE_ROW_SHAPES)
-def test_byte_rows_on_the_fma_stream(ctx, B, fmt, n, e, d_in, d_out):
-    """The library's other aggregation of 129..256 byte columns (bytes converted to fp32, packed FMAs) beside the
-    default integer tensor-core products."""
-    ctx.set_option(B.OPT_BYTE_AGGREGATION, 1)
+def test_byte_rows_as_integer_products(ctx, B, fmt, n, e, d_in, d_out):
+    """The library's other aggregation of 129..256 byte columns (exact integer products on the tensor cores with
+    fixed-point edge weights) beside the default fp32 FMA stream."""
+    ctx.set_option(B.OPT_BYTE_AGGREGATION, 2)
     try:
         check_layer_forward(ctx, B, fmt, n, e, d_in, d_out)
     finally:
@@ -207,10 +207,14 @@ def test_byte_rows_signed_edge_values_of_wide_range(ctx, B, fmt, d_in, span):
     W = (rng.standard_normal((d_in, d_out)) * d_in ** -0.5).astype(np.float32)
     t = oracle.layer_forward(g, oracle.Layer(W), H)
     ctx.set_option(B.OPT_ZETA_FORMAT, fmt)
+    ctx.set_option(B.OPT_BYTE_AGGREGATION, 2)
     G = device_graph(B, g)
     layer = B.make_layer(d_in, d_out, bits_to_dev(t.bitsT), dev(t.alpha))
-    out = ctx.layer_forward(G, layer, bits_to_dev(t.bits), dev(t.beta), want_h=True, debug=True)
-    ctx.sync_check()
+    try:
+        out = ctx.layer_forward(G, layer, bits_to_dev(t.bits), dev(t.beta), want_h=True, debug=True)
+        ctx.sync_check()
+    finally:
+        ctx.set_option(B.OPT_BYTE_AGGREGATION, 0)
     assert np.array_equal(out["dot"].cpu().numpy(), t.dot)
     ref = t.H_out
     got = out["h"].cpu().numpy().astype(np.float64)
@@ -242,7 +246,7 @@ def test_half_dot_bytes_hub_row_split_across_the_block(ctx, B):
     ctx.set_option(B.OPT_ZETA_FORMAT, 5)
     G = device_graph(B, g)
     layer = B.make_layer(d_in, d_out, bits_to_dev(t.bitsT), dev(t.alpha))
-    for path in (0, 1):
+    for path in (1, 2):
         ctx.set_option(B.OPT_BYTE_AGGREGATION, path)
         try:
             for thr in (0, 8, 100000):
