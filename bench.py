@@ -460,11 +460,11 @@ def run_ours(args):
     for l in range(L):
         f = args.zeta_format                      # the library's rule for the storage of zeta, layer by layer
         wide = 128 < dims[l + 1] <= 256
-        half_ok = wide and 128 <= dims[l] <= 256 and n >= 64
+        half_ok = dims[l + 1] <= 256 and 128 <= dims[l] <= 256 and n >= 64
         if f == 0:
             if wide and dims[l] <= 127:
                 f = binding.ZETA_I8
-            elif half_ok and n * dims[l + 1] >= (1 << 20):
+            elif half_ok and wide and n * dims[l + 1] >= (1 << 20):
                 f = binding.ZETA_I8H
             else:
                 f = binding.ZETA_F16

@@ -67,7 +67,8 @@ enum {
      * 3 = as 2 but int8 (layers with d_in <= 127 only; others fall back to 4);
      * 4 = as 2 but the integers held as fp16, which is exact for |dot| <= 2048 (layers with
      *     d_in <= 2048 only; others fall back to 2);
-     * 5 = signed bytes for 128 <= d_in <= 256 and 129..256 output columns (other layers as 0): the byte is
+     * 5 = signed bytes for 128 <= d_in <= 256 and up to 256 output columns (other layers as 0; the automatic
+     *     choice takes it for 129..256 output columns only -- narrower rows measured level with 4): the byte is
      *     s = (dot' - 1) / 2, dot' the dot without its first position when d_in is even (so that dot' is
      *     odd and s fits a byte exactly); the aggregation adds back sum_k w_k (1 + f_k0 b_0j), two per-row
      *     sums that ride along with the edge weights.  Exact in the integers; on the tensor-core contraction. */

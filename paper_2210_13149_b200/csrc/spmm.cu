@@ -73,15 +73,17 @@ template <> struct Elt<int16_t> {
 };
 template <> struct Elt<int8_t> {
     static constexpr int kPerVec = 16;
+    // Without the conversion unit: b ^ 0x80 placed in the low mantissa byte of 2^23 is the float 2^23 + 128 + b;
+    // one subtraction gives b exactly.
     static __device__ __forceinline__ void unpack(const uint4& v, float (&f)[16])
     {
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        const uint32_t w[4] = {v.x ^ 0x80808080u, v.y ^ 0x80808080u, v.z ^ 0x80808080u, v.w ^ 0x80808080u};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            f[4 * i] = (float)(int8_t)(w[i] & 0xffu);
-            f[4 * i + 1] = (float)(int8_t)((w[i] >> 8) & 0xffu);
-            f[4 * i + 2] = (float)(int8_t)((w[i] >> 16) & 0xffu);
-            f[4 * i + 3] = (float)((int32_t)w[i] >> 24);
+            f[4 * i] = __uint_as_float(__byte_perm(w[i], 0x4B000000u, 0x7540)) - 8388736.f;
+            f[4 * i + 1] = __uint_as_float(__byte_perm(w[i], 0x4B000000u, 0x7541)) - 8388736.f;
+            f[4 * i + 2] = __uint_as_float(__byte_perm(w[i], 0x4B000000u, 0x7542)) - 8388736.f;
+            f[4 * i + 3] = __uint_as_float(__byte_perm(w[i], 0x4B000000u, 0x7543)) - 8388736.f;
         }
     }
 };
@@ -264,7 +266,11 @@ struct Pipe {
 //                     row is written as its last entry is consumed.
 //   kPartial = true : the entries are a slice of one long row; the slice's sum is left in `acc`
 //                     (already combined over the lane groups).
-template <typename T, int NCH, int LPR, bool kPartial>
+__device__ __forceinline__ void fma_bytes16(float w, const uint4& v, float (&acc)[16]);
+
+// kHalf (rows of signed bytes only): half-dot bytes -- the weights' sign carries the source's first feature sign; the
+// row's plain and signed weight sums ride along and the epilogue reconstructs the dots (see finish_row).
+template <typename T, int NCH, int LPR, bool kPartial, bool kHalf = false>
 __device__ __forceinline__ void stream_entries(const SpmmDev& p, uint4* ring, float* wfifo, const float* ctab, int lane,
                                                int64_t e0, int n_ent, int64_t warp_row0, int row_lo,
                                                int row_hi, int rp_rel,
@@ -298,6 +304,7 @@ __device__ __forceinline__ void stream_entries(const SpmmDev& p, uint4* ring, fl
     int rt = row_lo;                                          // row being accumulated (local index)
     int row_end = kPartial ? n_ent : __shfl_sync(0xffffffffu, rp_rel, rt + 1);
     zero_acc<NCH, EPV>(acc);
+    float wsum = 0.f, wsgn = 0.f;                             // half-dot bytes: sum of the row's weights, plain and signed
 
     for (int it = 0; it < n_groups + NG; ++it) {
         const int gslot = (it % NG) * PB;                     // first slot of the group handled now
@@ -317,16 +324,23 @@ __device__ __forceinline__ void stream_entries(const SpmmDev& p, uint4* ring, fl
             if (off0 + PB * G < row_end) {
                 // the whole group lies inside the current row: no boundary logic
 #pragma unroll
-                for (int b = 0; b < PB; ++b)
+                for (int b = 0; b < PB; ++b) {
+                    const float wa = kHalf ? fabsf(w[b]) : w[b];
+                    if (kHalf) { wsum += wa; wsgn += w[b]; }
 #pragma unroll
                     for (int c = 0; c < NCH; ++c) {
-                        float f[EPV];
-                        Elt<T>::unpack(v[b][c], f);
-                        if (NCH == 1 || active[c]) {
+                        if constexpr (sizeof(T) == 1) {
+                            if (NCH == 1 || active[c]) fma_bytes16(wa, v[b][c], acc[c]);
+                        } else {
+                            float f[EPV];
+                            Elt<T>::unpack(v[b][c], f);
+                            if (NCH == 1 || active[c]) {
 #pragma unroll
-                            for (int i = 0; i < EPV; ++i) acc[c][i] = fmaf(w[b], f[i], acc[c][i]);
+                                for (int i = 0; i < EPV; ++i) acc[c][i] = fmaf(wa, f[i], acc[c][i]);
+                            }
                         }
                     }
+                }
             } else {
 #pragma unroll
                 for (int b = 0; b < PB; ++b) {
@@ -341,18 +355,39 @@ __device__ __forceinline__ void stream_entries(const SpmmDev& p, uint4* ring, fl
                         const int rem = row_end - eb;         // entries of the position before the row's end
                         const int upto = rem < nb ? rem : nb;
                         if (g >= done && g < upto) {
+                            const float wa = kHalf ? fabsf(w[b]) : w[b];
+                            if (kHalf) { wsum += wa; wsgn += w[b]; }
 #pragma unroll
                             for (int c = 0; c < NCH; ++c)
                                 if (active[c]) {
 #pragma unroll
-                                    for (int i = 0; i < EPV; ++i) acc[c][i] = fmaf(w[b], f[c][i], acc[c][i]);
+                                    for (int i = 0; i < EPV; ++i) acc[c][i] = fmaf(wa, f[c][i], acc[c][i]);
                                 }
                         }
                         if (rem > nb) break;                  // the row continues in a later position
                         reduce_groups<NCH, EPV, LPR>(acc);
-                        if (kPartial) return;                 // slice complete (only at the last position)
-                        finish_row<T, NCH, LPR>(p, ctab, warp_row0 + rt, lane, acc);
+                        if (kHalf) {
+#pragma unroll
+                            for (int o = LPR; o < kWarp; o <<= 1) {
+                                wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
+                                wsgn += __shfl_xor_sync(0xffffffffu, wsgn, o);
+                            }
+                        }
+                        if (kPartial) {                       // slice complete (only at the last position)
+                            if (kHalf) {                      // hand back the reconstructed partial sums
+                                constexpr int kCols = NCH * LPR * EPV;
+#pragma unroll
+                                for (int c = 0; c < NCH; ++c)
+#pragma unroll
+                                    for (int i = 0; i < EPV; ++i)
+                                        acc[c][i] = fmaf(2.f, acc[c][i], fmaf(ctab[3 * kCols + (c * LPR + l) * EPV + i], wsgn, wsum));
+                            }
+                            return;
+                        }
+                        finish_row<T, NCH, LPR, kHalf>(p, ctab, warp_row0 + rt, lane, acc, wsum, wsgn);
                         zero_acc<NCH, EPV>(acc);
+                        wsum = 0.f;
+                        wsgn = 0.f;
                         if (upto > done) done = upto;
                         ++rt;
                         if (rt == row_hi) break;
@@ -1155,20 +1190,21 @@ cudaError_t launch_imma(cudaStream_t s, SpmmDev p)
 }
 
 // Thread blocks per SM the kernel is compiled for (register budget) and launched with (grid size).
-template <int NCH, int LPR, bool kAligned>
+template <int NCH, int LPR, bool kAligned, int kEltBytes>
 constexpr int spmm_blocks_per_sm()
 {
-    return NCH == 1 ? ((LPR == 32 || kAligned) ? 3 : 4) : (NCH == 2 ? 2 : 1);
+    // (a lane of the general stream holds 16 accumulators for byte rows, 4 or 8 otherwise)
+    return NCH == 1 ? ((LPR == 32 || kAligned || kEltBytes == 1) ? 3 : 4) : (NCH == 2 ? 2 : 1);
 }
 
 // kAligned (rows of 8 or 16 vectors only): the row-aligned multi-entry stream instead of the general one.
-// kHalf: half-dot bytes (aligned byte stream only).
+// kHalf: half-dot bytes (rows of signed bytes; either stream).
 template <typename T, int NCH, int LPR, bool kFull, bool kAligned, bool kHalf = false>
-__global__ void __launch_bounds__(kSpmmThreads, spmm_blocks_per_sm<NCH, LPR, kAligned>())
+__global__ void __launch_bounds__(kSpmmThreads, spmm_blocks_per_sm<NCH, LPR, kAligned, (int)sizeof(T)>())
 spmm_kernel(const SpmmDev p, int rows_per_warp)
 {
-    static_assert(!kHalf || (kAligned && sizeof(T) == 1), "half-dot bytes take the aligned byte stream");
-    static_assert(!kAligned || ((NCH == 1 || NCH == 2) && (LPR == 8 || LPR == 16)), "the multi-entry stream: 8 or 16 lanes per row, one or two vectors per lane");
+    static_assert(!kHalf || (sizeof(T) == 1 && LPR < 32), "half-dot bytes: rows of up to 256 signed bytes");
+    static_assert(!kAligned || ((NCH == 1 || NCH == 2) && (LPR == 4 || LPR == 8 || LPR == 16)), "the multi-entry stream: 4, 8 or 16 lanes per row, one or two vectors per lane");
     using P = Pipe<NCH, LPR, kAligned>;
     constexpr int EPV = Elt<T>::kPerVec;
     constexpr int G = P::G;
@@ -1219,7 +1255,7 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
                     stream_rows_multi<T, kWarp / LPR, NCH, kFull, false, kHalf>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
                                                                     (int)(rp_reg - e0), acc);
                 else
-                    stream_entries<T, NCH, LPR, false>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
+                    stream_entries<T, NCH, LPR, false, kHalf>(p, ring, wfifo, ctab, lane, e0, (int)(e1 - e0), warp_row0, ra, rl,
                                                        (int)(rp_reg - e0), acc);
             }
             ra = rl + 1;
@@ -1238,7 +1274,7 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
         else if constexpr (kAligned)
             stream_rows_multi<T, kWarp / LPR, NCH, kFull, true, kHalf>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
         else
-            stream_entries<T, NCH, LPR, true>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
+            stream_entries<T, NCH, LPR, true, kHalf>(p, ring, wfifo, ctab, lane, s0, (int)(s1 - s0), 0, 0, 1, 0, acc);
         __syncthreads();                                      // every ring is idle: reuse them for the partial sums
         const int l = lane % LPR;
         if (lane < LPR) {
@@ -1278,7 +1314,7 @@ cudaError_t launch_one(cudaStream_t s, const SpmmDev& p)
     if (e != cudaSuccess) return e;
     // one wave of resident blocks; the warps pull runs of rows until none are left
     const int64_t wanted = ceil_div(ceil_div(p.n, rows_per_warp), kSpmmWarps);
-    const unsigned grid = (unsigned)std::min<int64_t>(wanted, 148 * spmm_blocks_per_sm<NCH, LPR, kAligned>());
+    const unsigned grid = (unsigned)std::min<int64_t>(wanted, 148 * spmm_blocks_per_sm<NCH, LPR, kAligned, (int)sizeof(T)>());
     spmm_kernel<T, NCH, LPR, kFull, kAligned, kHalf><<<grid, kSpmmThreads, smem, s>>>(p, rows_per_warp);
     return cudaGetLastError();
 }
@@ -1292,6 +1328,21 @@ template <typename T>
 cudaError_t dispatch(cudaStream_t s, const SpmmDev& p, double mean_row)
 {
     const int nv = p.nv;
+    if constexpr (sizeof(T) == 1) {
+        if (p.half_dots && nv <= 8) {                         // narrow rows of half-dot bytes
+            if (nv <= 1) return launch_one<T, 1, 1, false, false, true>(s, p);
+            if (nv <= 2) return launch_one<T, 1, 2, false, false, true>(s, p);
+            // rows of 3..8 vectors: the row-aligned stream (8 or 4 entries per position, groups of 32 or 16 entries)
+            // unless the rows are known to be much shorter than a group
+            const bool short_rows = mean_row > 0.0 && mean_row < 8.0;
+            if (nv <= 4) {
+                if (short_rows) return launch_one<T, 1, 4, false, false, true>(s, p);
+                return nv == 4 ? launch_one<T, 1, 4, true, true, true>(s, p) : launch_one<T, 1, 4, false, true, true>(s, p);
+            }
+            if (short_rows) return launch_one<T, 1, 8, false, false, true>(s, p);
+            return nv == 8 ? launch_one<T, 1, 8, true, true, true>(s, p) : launch_one<T, 1, 8, false, true, true>(s, p);
+        }
+    }
     if (nv <= 1) return launch_one<T, 1, 1>(s, p);
     if (nv <= 2) return launch_one<T, 1, 2>(s, p);
     if (nv <= 4) return launch_one<T, 1, 4>(s, p);
@@ -1344,7 +1395,7 @@ cudaError_t launch_spmm(cudaStream_t s, const SpmmArgs& a, int* launches)
     p.col_b0 = a.half_dots ? a.col_b0 : nullptr;
     p.half_dots = a.half_dots ? 1 : 0;
     p.byte_path = a.byte_path;
-    if (a.half_dots && (a.fmt != kZetaI8 || p.nv > 16 || p.nv <= 8 || !a.col_b0 || !a.node_w)) return cudaErrorInvalidValue;   // 129..256 byte columns only
+    if (a.half_dots && (a.fmt != kZetaI8 || p.nv > 16 || !a.col_b0 || !a.node_w)) return cudaErrorInvalidValue;   // up to 256 byte columns
     p.ld_add = a.ld_add;
     p.h_out = a.h_out;
     p.ldh = a.ldh;

@@ -158,6 +158,18 @@ def test_layer_forward_half_dot_bytes(ctx, B, n, e, d_in, d_out):
     check_layer_forward(ctx, B, 5, n, e, d_in, d_out)
 
 
+# half-dot bytes in rows of 1, 2, 3, 4, 7 and 8 sixteen-byte vectors (the general stream): short and long rows,
+# both parities of d_in, rows that end inside a group of positions
+HALF_NARROW_SHAPES = [(64, 300, 128, 5), (500, 6000, 129, 16), (700, 9000, 200, 17), (300, 4000, 255, 32),
+                      (3000, 30000, 256, 47), (2000, 120000, 256, 47), (40000, 300000, 256, 47), (900, 9000, 254, 64),
+                      (1500, 40000, 256, 100), (5000, 60000, 256, 128), (600, 2400, 256, 41), (2000, 6000, 256, 100)]
+
+
+@pytest.mark.parametrize("n,e,d_in,d_out", HALF_NARROW_SHAPES)
+def test_layer_forward_half_dot_bytes_narrow_rows(ctx, B, n, e, d_in, d_out):
+    check_layer_forward(ctx, B, 5, n, e, d_in, d_out)
+
+
 def test_half_dot_bytes_at_the_ends_of_the_byte_range(ctx, B):
     """Rows equal to a weight column (dot = +256) and to its complement (dot = -256): the stored bytes reach
     +127 and -128; the reconstructed sums must still be exact."""
@@ -231,9 +243,10 @@ def test_byte_rows_signed_edge_values_of_wide_range(ctx, B, fmt, d_in, span):
     assert np.all(np.abs(got - ref) <= 1e-5 * np.abs(ref) + 4e-6 * bound + 2.0 ** -27 * fixed + 1e-30)
 
 
-def test_half_dot_bytes_hub_row_split_across_the_block(ctx, B):
+@pytest.mark.parametrize("d_out", [256, 47])
+def test_half_dot_bytes_hub_row_split_across_the_block(ctx, B, d_out):
     """One row with n entries under half-dot bytes: slices of a long row hand back reconstructed partial sums."""
-    n, d_in, d_out = 3000, 256, 256
+    n, d_in = 3000, 256
     rng = np.random.default_rng(78)
     rp, ci = synth.power_law_graph(n, 30000, 78)
     src, dst = synth.edge_list(rp, ci)
