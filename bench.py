@@ -165,7 +165,11 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64-accumulate (CPU oracle)", "data": "synthetic",
-            "config": {"workload": "CPU oracle on a sample of " + args.config, "sample": sample},
+            "config": {"workload": ("%s: %d-layer Bi-GCN forward, synthetic power-law graph, %d nodes, about %d stored entries of "
+                                    "A_tilde, widths %s, %s features (the CPU oracle, timed on a sample of it)"
+                                    % (spec.name, len(spec.dims) - 1, spec.n, spec.e_dir + spec.n,
+                                       "-".join(str(d) for d in spec.dims), spec.features)),
+                       "sample": sample},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
