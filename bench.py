@@ -463,7 +463,7 @@ def run_ours(args):
     dom = max(range(L), key=lambda l: spmm_ms[l])
     for l in range(L):
         f = args.zeta_format                      # the library's rule for the storage of zeta, layer by layer
-        wide = 128 < dims[l + 1] <= 256
+        wide = 128 < dims[l + 1] <= 256 or (l == L - 1 and 32 < dims[l + 1] <= 64)   # (a last layer: fp32 output only)
         half_ok = dims[l + 1] <= 256 and 128 <= dims[l] <= 256 and n >= 64
         if f == 0:
             if wide and dims[l] <= 127:

@@ -63,10 +63,12 @@ size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 // Asked for by option, half-dot bytes also serve narrower rows (up to 128 columns); the automatic choice leaves those
 // in fp16: with rows that short the aggregation is bound by instructions per entry, not bytes, and measured level
 // (47 columns on 126 M entries: 3.69 + 0.21 ms against 3.72 + 0.16 ms for aggregation + contraction).
-int pick_format(const bigcn_ctx* ctx, int d_in, int d_out, int64_t n, bool allow_half = false)
+// `fp32_only`: the layer's result is only written out as fp32 (a network's last layer); then 33..64 columns also take
+// bytes, for which the aggregation has a stream with one stored entry per lane (c4 layer 1: 2.8 -> 1.8 ms).
+int pick_format(const bigcn_ctx* ctx, int d_in, int d_out, int64_t n, bool allow_half = false, bool fp32_only = false)
 {
     int f = ctx->zeta_format;
-    const bool wide = d_out > 128 && d_out <= 256;
+    const bool wide = (d_out > 128 && d_out <= 256) || (fp32_only && d_out > 32 && d_out <= 64);
     const bool half_ok = allow_half && d_out <= 256 && d_in >= 128 && d_in <= 256 && n >= 64 && ctx->contraction != 1;
     if (f == 0) {
         if (wide && d_in <= 127) f = kZetaI8;
@@ -127,7 +129,7 @@ bigcn_status run_layer(bigcn_ctx* ctx, const bigcn_graph* g, const bigcn_layer* 
                        float* next_beta, int32_t* dbg_dot, float* dbg_zeta,
                        cudaEvent_t ev_mid /*nullable*/)
 {
-    const int fmt = pick_format(ctx, layer->d_in, layer->d_out, g->n, /*allow_half=*/true);
+    const int fmt = pick_format(ctx, layer->d_in, layer->d_out, g->n, /*allow_half=*/true, /*fp32_only=*/next == nullptr && h_out != nullptr);
     const bool half = fmt == kZetaI8H;
     const int64_t ldz = zeta_ld(layer->d_out, fmt);
     const int64_t stride_in = bigcn_packed_stride_words(layer->d_in);

@@ -1189,6 +1189,261 @@ cudaError_t launch_imma(cudaStream_t s, SpmmDev p)
     return cudaGetLastError();
 }
 
+// ---- narrow rows of signed bytes, one stored entry per lane ------------------------------------------------------
+//
+// For rows of 3 or 4 sixteen-byte vectors (33..64 byte columns) whose result is only written out as fp32 (a
+// network's last layer).  The streams above give a lane one vector of an entry, so a warp handles 8 entries per
+// instruction and every row end costs a reduction over the lane groups; here a lane owns a whole stored entry:
+// it loads the entry's column, value and node factor itself (no shuffles), fetches the NV vectors of the operand
+// row straight into registers and accumulates all 16 NV columns.  A pass is up to 32 entries of one row; the
+// passes of a run of rows form one stream (column indices two passes ahead, gathers one pass ahead), so that the
+// latencies of a row's first pass hide behind the previous row.  When a row ends the 32 lanes' partial sums are
+// added through a per-warp shared-memory buffer (a lane reads four columns of sixteen lanes, two half-sums meet
+// by one shuffle) and lanes 0 .. 4 NV - 1 write four columns each.
+constexpr int kLaneWarps = 8;
+constexpr int kLaneThreads = kLaneWarps * kWarp;
+constexpr int kLanePitch = 68;                                // floats per lane in the reduction buffer (64 + 4: 16-byte stores of 8 lanes fall into distinct banks)
+
+// Streams rows [row_lo, row_hi) of a run (kPartial: the stored entries [e0, e0 + n_ent) as one row, whose sums are
+// handed back in `out` / `wsum` / `wsgn` instead of being written).
+template <int NV, bool kHalf, bool kPartial>
+__device__ __forceinline__ void stream_rows_lane(const SpmmDev& p, float* red, int lane, int64_t e0, int n_ent,
+                                                 int64_t warp_row0, int row_lo, int row_hi, int rp_rel,
+                                                 const float (&al)[4], const float (&b0)[4], float4& out, float& wsum_out, float& wsgn_out)
+{
+    constexpr int NG4 = 4 * NV;                               // groups of four columns
+    const int32_t* cols = p.colidx + e0;
+    const float* vals = p.val + e0;
+    const char* zeta = reinterpret_cast<const char*>(p.zeta);
+    auto row_start = [&](int r) { return kPartial ? 0 : __shfl_sync(0xffffffffu, rp_rel, r); };
+    auto row_end = [&](int r) { return kPartial ? n_ent : __shfl_sync(0xffffffffu, rp_rel, r + 1); };
+
+    int ir = row_lo, io = 0;                                  // index cursor: row, offset of the next pass inside it
+    auto fetch_indices = [&](int& c, float& w) {
+        c = -1;
+        w = 0.f;
+        if (ir < row_hi) {
+            const int rs = row_start(ir), re = row_end(ir);
+            const int idx = rs + io + lane;
+            if (idx < re) {
+                c = __ldg(cols + idx);
+                w = __ldg(vals + idx);
+            }
+            io += 32;
+            if (rs + io >= re) {
+                ++ir;
+                io = 0;
+            }
+        }
+    };
+    uint4 vn[NV];
+    float nwn = 1.f;
+    auto gather = [&](int c) {
+        if (c >= 0) {
+            nwn = p.node_w ? __ldg(p.node_w + c) : 1.f;
+            const uint4* src = reinterpret_cast<const uint4*>(zeta + (uint64_t)(uint32_t)c * (uint32_t)(NV * 16));
+#pragma unroll
+            for (int q = 0; q < NV; ++q) vn[q] = __ldg(src + q);
+        }
+    };
+    int c1, c2;
+    float w1, w2;
+#pragma unroll
+    for (int q = 0; q < NV; ++q) vn[q] = make_uint4(0u, 0u, 0u, 0u);
+    fetch_indices(c1, w1);
+    fetch_indices(c2, w2);
+    gather(c1);
+
+    float acc[NV][16];
+    zero_acc<NV, 16>(acc);
+    float ws = 0.f, wg = 0.f;
+    int cr = row_lo, co = 0;                                  // consume cursor
+    while (cr < row_hi) {
+        uint4 v[NV];
+#pragma unroll
+        for (int q = 0; q < NV; ++q) v[q] = vn[q];
+        const float wt = c1 >= 0 ? w1 * nwn : 0.f;            // lanes past the row's end add nothing
+        c1 = c2;
+        w1 = w2;
+        gather(c1);                                           // the next pass's operand rows
+        fetch_indices(c2, w2);                                // the indices of the pass after that
+        const float wa = kHalf ? fabsf(wt) : wt;              // half-dot bytes: the sign carries the source's first feature sign
+        if (kHalf) { ws += wa; wg += wt; }
+#pragma unroll
+        for (int q = 0; q < NV; ++q) fma_bytes16(wa, v[q], acc[q]);
+        const int rs = row_start(cr), re = row_end(cr);
+        co += 32;
+        if (rs + co >= re) {
+            // ---- the row is complete: add the lanes' sums
+            float* mine = red + lane * kLanePitch;
+#pragma unroll
+            for (int q = 0; q < NV; ++q)
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    *reinterpret_cast<float4*>(mine + 16 * q + 4 * i) = make_float4(acc[q][4 * i], acc[q][4 * i + 1], acc[q][4 * i + 2], acc[q][4 * i + 3]);
+            __syncwarp();
+            const int cg = lane % NG4, jh = lane / NG4;       // four columns, one half of the lanes (jh = 2: idle)
+            float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (jh < 2) {
+                const float* src = red + (16 * jh) * kLanePitch + 4 * cg;
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float4 u = *reinterpret_cast<const float4*>(src + j * kLanePitch);
+                    t.x += u.x, t.y += u.y, t.z += u.z, t.w += u.w;
+                }
+            }
+            __syncwarp();
+            t.x += __shfl_down_sync(0xffffffffu, t.x, NG4);
+            t.y += __shfl_down_sync(0xffffffffu, t.y, NG4);
+            t.z += __shfl_down_sync(0xffffffffu, t.z, NG4);
+            t.w += __shfl_down_sync(0xffffffffu, t.w, NG4);
+            if (kHalf) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    ws += __shfl_xor_sync(0xffffffffu, ws, o);
+                    wg += __shfl_xor_sync(0xffffffffu, wg, o);
+                }
+            }
+            if (kPartial) {
+                out = t;
+                wsum_out = ws;
+                wsgn_out = wg;
+                return;
+            }
+            if (lane < NG4) {
+                float x[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (kHalf) x[i] = fmaf(2.f, x[i], fmaf(b0[i], wg, ws));
+                    x[i] *= al[i];
+                }
+                float* dst = p.h_out + (warp_row0 + cr) * p.ldh + 4 * cg;
+                if (p.h_vec && 4 * cg + 3 < p.d_out) {
+                    *reinterpret_cast<float4*>(dst) = make_float4(x[0], x[1], x[2], x[3]);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        if (4 * cg + i < p.d_out) dst[i] = x[i];
+                }
+            }
+            zero_acc<NV, 16>(acc);
+            ws = 0.f;
+            wg = 0.f;
+            ++cr;
+            co = 0;
+        }
+    }
+    if (kPartial) {                                           // empty slice
+        out = make_float4(0.f, 0.f, 0.f, 0.f);
+        wsum_out = 0.f;
+        wsgn_out = 0.f;
+    }
+}
+
+template <int NV, bool kHalf>
+__global__ void __launch_bounds__(kLaneThreads, 2)
+spmm_lane_kernel(const SpmmDev p, int rows_per_warp)
+{
+    constexpr int NG4 = 4 * NV;
+    extern __shared__ __align__(16) float lsm[];
+    __shared__ int64_t long_rows[kLongQueue];
+    __shared__ int n_long;
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    float* red = lsm + (size_t)warp * 32 * kLanePitch;
+    float* part = lsm + (size_t)kLaneWarps * 32 * kLanePitch;       // [kLaneWarps][NG4 * 4 + 4]: slices of a long row
+    constexpr int kPartPitch = NG4 * 4 + 4;
+    const int cg = lane % NG4;
+    float al[4], b0[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int col = 4 * cg + i;
+        const bool in = lane < NG4 && col < p.d_out;
+        al[i] = in ? (p.col_w ? __ldg(p.col_w + col) : 1.f) : 0.f;
+        b0[i] = (in && kHalf && p.col_b0) ? __ldg(p.col_b0 + col) : 0.f;
+    }
+    if (threadIdx.x == 0) n_long = 0;
+    __syncthreads();
+
+    const int64_t n_runs = ceil_div(p.n, rows_per_warp);
+    float4 t;
+    float ws, wg;
+    for (;;) {
+        int64_t run = 0;
+        if (lane == 0) run = atomicAdd(p.run_counter, 1);
+        run = __shfl_sync(0xffffffffu, run, 0);
+        if (run >= n_runs) break;
+        const int64_t warp_row0 = run * rows_per_warp;
+        const int n_rows = (int)min((int64_t)rows_per_warp, p.n - warp_row0);
+        const int64_t rp_reg = __ldg(p.rowptr + warp_row0 + min(lane, n_rows));
+        const int64_t rp_next = __shfl_down_sync(0xffffffffu, rp_reg, 1);
+        bool is_long = lane < n_rows && p.long_row > 0 && (rp_next - rp_reg) > p.long_row;
+        if (is_long) {                                        // queue it for the block; if the queue is full, stream it here
+            const int slot = atomicAdd(&n_long, 1);
+            if (slot < kLongQueue) long_rows[slot] = warp_row0 + lane;
+            else is_long = false;
+        }
+        const unsigned long_mask = __ballot_sync(0xffffffffu, is_long);
+        int ra = 0;
+        while (ra < n_rows) {                                 // runs of rows between the long ones
+            const unsigned rest = long_mask >> ra;
+            const int rl = rest ? ra + (__ffs(rest) - 1) : n_rows;
+            if (rl > ra) {
+                const int64_t e0 = __shfl_sync(0xffffffffu, rp_reg, ra);
+                stream_rows_lane<NV, kHalf, false>(p, red, lane, e0, 0, warp_row0, ra, rl, (int)(rp_reg - e0), al, b0, t, ws, wg);
+            }
+            ra = rl + 1;
+        }
+    }
+    __syncthreads();
+    const int nl = min(n_long, kLongQueue);
+    for (int q = 0; q < nl; ++q) {                            // long rows of this block, each by all warps together
+        const int64_t lrow = long_rows[q];
+        const int64_t ls = __ldg(p.rowptr + lrow), le = __ldg(p.rowptr + lrow + 1);
+        const int64_t slice = round_up(ceil_div(le - ls, kLaneWarps), 32);
+        const int64_t s0 = min(le, ls + warp * slice), s1 = min(le, s0 + slice);
+        stream_rows_lane<NV, kHalf, true>(p, red, lane, s0, (int)(s1 - s0), 0, 0, (s1 > s0) ? 1 : 0, 0, al, b0, t, ws, wg);
+        if (lane < NG4) *reinterpret_cast<float4*>(part + warp * kPartPitch + 4 * cg) = t;
+        if (lane == 0) {
+            part[warp * kPartPitch + NG4 * 4] = ws;
+            part[warp * kPartPitch + NG4 * 4 + 1] = wg;
+        }
+        __syncthreads();
+        if (warp == 0 && lane < NG4) {
+            float x[4] = {0.f, 0.f, 0.f, 0.f};
+            float sws = 0.f, swg = 0.f;
+            for (int w = 0; w < kLaneWarps; ++w) {
+                const float4 u = *reinterpret_cast<const float4*>(part + w * kPartPitch + 4 * cg);
+                x[0] += u.x, x[1] += u.y, x[2] += u.z, x[3] += u.w;
+                sws += part[w * kPartPitch + NG4 * 4];
+                swg += part[w * kPartPitch + NG4 * 4 + 1];
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (kHalf) x[i] = fmaf(2.f, x[i], fmaf(b0[i], swg, sws));
+                x[i] *= al[i];
+                if (4 * cg + i < p.d_out) p.h_out[lrow * p.ldh + 4 * cg + i] = x[i];
+            }
+        }
+        __syncthreads();
+    }
+}
+
+template <int NV, bool kHalf>
+cudaError_t launch_lane(cudaStream_t s, const SpmmDev& p)
+{
+    constexpr size_t smem = ((size_t)kLaneWarps * 32 * kLanePitch + (size_t)kLaneWarps * (NV * 16 + 4)) * sizeof(float);
+    const int rows_per_warp = (int)std::min<int64_t>(kMaxRowsPerWarp, std::max<int64_t>(1, p.n / (kLaneWarps * 148 * 8)));
+    cudaError_t e = cudaFuncSetAttribute(spmm_lane_kernel<NV, kHalf>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(p.run_counter, 0, sizeof(int), s);
+    if (e != cudaSuccess) return e;
+    const int64_t wanted = ceil_div(ceil_div(p.n, rows_per_warp), kLaneWarps);
+    const unsigned grid = (unsigned)std::min<int64_t>(wanted, 148 * 2);
+    spmm_lane_kernel<NV, kHalf><<<grid, kLaneThreads, smem, s>>>(p, rows_per_warp);
+    return cudaGetLastError();
+}
+
 // Thread blocks per SM the kernel is compiled for (register budget) and launched with (grid size).
 template <int NCH, int LPR, bool kAligned, int kEltBytes>
 constexpr int spmm_blocks_per_sm()
@@ -1329,6 +1584,11 @@ cudaError_t dispatch(cudaStream_t s, const SpmmDev& p, double mean_row)
 {
     const int nv = p.nv;
     if constexpr (sizeof(T) == 1) {
+        // 33..64 byte columns, fp32 output only (a last layer), rows not much shorter than a pass: one entry per lane
+        if ((nv == 3 || nv == 4) && p.h_out && !p.next_bits && !p.add && p.byte_path != 2 && !(mean_row > 0.0 && mean_row < 8.0)) {
+            if (p.half_dots) return nv == 3 ? launch_lane<3, true>(s, p) : launch_lane<4, true>(s, p);
+            return nv == 3 ? launch_lane<3, false>(s, p) : launch_lane<4, false>(s, p);
+        }
         if (p.half_dots && nv <= 8) {                         // narrow rows of half-dot bytes
             if (nv <= 1) return launch_one<T, 1, 1, false, false, true>(s, p);
             if (nv <= 2) return launch_one<T, 1, 2, false, false, true>(s, p);

@@ -243,6 +243,30 @@ def test_byte_rows_signed_edge_values_of_wide_range(ctx, B, fmt, d_in, span):
     assert np.all(np.abs(got - ref) <= 1e-5 * np.abs(ref) + 4e-6 * bound + 2.0 ** -27 * fixed + 1e-30)
 
 
+# a network's last layer (fp32 output only) with 33..64 byte columns: the stream with one stored entry per lane
+LAST_LAYER_SHAPES = [(5, 3000, 30000, 256, 47), (5, 2000, 120000, 256, 47), (5, 40000, 400000, 256, 41), (5, 900, 9000, 129, 33),
+                     (5, 900, 9000, 254, 64), (5, 1500, 40000, 200, 48), (3, 3000, 30000, 100, 47), (3, 900, 20000, 127, 64),
+                     (5, 64, 300, 256, 47), (5, 2000, 5000, 256, 47)]
+
+
+@pytest.mark.parametrize("fmt,n,e,d_in,d_out", LAST_LAYER_SHAPES)
+def test_last_layer_narrow_byte_rows(ctx, B, fmt, n, e, d_in, d_out):
+    rng = np.random.default_rng(n + d_in + d_out)
+    _, _, g = small_graph(n, e, 300 + n)
+    H = rng.standard_normal((n, d_in)).astype(np.float32)
+    W = (rng.standard_normal((d_in, d_out)) * d_in ** -0.5).astype(np.float32)
+    t = oracle.layer_forward(g, oracle.Layer(W), H)
+    ctx.set_option(B.OPT_ZETA_FORMAT, fmt)
+    G = device_graph(B, g)
+    layer = B.make_layer(d_in, d_out, bits_to_dev(t.bitsT), dev(t.alpha))
+    out = ctx.layer_forward(G, layer, bits_to_dev(t.bits), dev(t.beta), want_h=True, debug=True)
+    ctx.sync_check()
+    assert np.array_equal(out["dot"].cpu().numpy(), t.dot)
+    assert_close(out["h"], t.H_out, "H' (last layer, format %d)" % fmt)
+    again = ctx.layer_forward(G, layer, bits_to_dev(t.bits), dev(t.beta), want_h=True)["h"]
+    assert torch.equal(again, out["h"])                       # run-to-run deterministic
+
+
 @pytest.mark.parametrize("d_out", [256, 47])
 def test_half_dot_bytes_hub_row_split_across_the_block(ctx, B, d_out):
     """One row with n entries under half-dot bytes: slices of a long row hand back reconstructed partial sums."""
