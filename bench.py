@@ -26,7 +26,8 @@ if ROOT not in sys.path:
 
 METRIC = "bigcn_forward_nodes_per_s"
 UNIT = "nodes/s"
-DTYPE = "u32-xor-popc+f32"
+DTYPE = "u32-xor-popc+f32"                # contraction on the XOR / bit-count pipe, fp32 aggregation
+DTYPE_TC = "b1-as-s8-tcgen05-s32+f32"     # contraction as int8 tensor-core products of the +-1 bits (int32 sums), fp32 aggregation
 
 
 def parse_args():
@@ -527,9 +528,11 @@ def run_ours(args):
         except Exception as exc:      # the oracle is optional equipment for the bench
             cpu = {"value": None, "unit": UNIT, "cores": 0, "kind": "oracle", "sample": "failed: %r" % (exc,)}
 
+    on_tc_layers = [kernels["bitgemm_l%d" % l]["path"].startswith("tcgen05") for l in range(L)]
+    dtype = DTYPE_TC if all(on_tc_layers) else (DTYPE if not any(on_tc_layers) else DTYPE_TC + " / " + DTYPE)
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": DTYPE, "data": "synthetic",
+            "vs_baseline": None, "dtype": dtype, "data": "synthetic",
             "config": {"workload": workload_description(spec, n, nnz), "l2": "inputs_exceed_l2",
                        "parallelism": "replicas" if world > 1 else "single-gpu",
                        "zeta_format": {0: "auto", 1: "f32", 2: "i16", 3: "i8", 4: "f16", 5: "i8h"}[args.zeta_format]},
