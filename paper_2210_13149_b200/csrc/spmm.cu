@@ -151,16 +151,28 @@ __device__ __forceinline__ void reduce_groups(float (&acc)[NCH][EPV])
 // Per-column constants of the row epilogue, staged once per thread block: four arrays of kCols
 // floats -- the column factor (0 for padding columns, 1 when there is none), the next layer's shift and
 // scale (0 and 1 where there are none, so that applying them changes nothing), and the first weight
-// sign of the column (half-dot bytes only, else 0).
-template <int kCols>
+// sign of the column (half-dot bytes only, else 0).  Inside an array the 16-byte chunks are ordered so that the
+// lanes' reads in the row epilogue are contiguous: a lane holds EPV consecutive columns (EPV / 4 chunks) and reads
+// its q-th chunk together with the other lanes, so chunk q of vector v sits at position q * (kCols / EPV) + v
+// (in column order the reads of 8- and 16-column vectors fall 32 and 64 bytes apart: 2- and 4-way bank conflicts).
+template <int kCols, int EPV>
+__device__ __forceinline__ int ctab_at(int col)
+{
+    constexpr int Q = EPV / 4, NVEC = kCols / EPV;
+    const int ch = col >> 2;
+    return 4 * ((ch % Q) * NVEC + ch / Q) + (col & 3);
+}
+
+template <int kCols, int EPV>
 __device__ __forceinline__ void fill_col_table(const SpmmDev& p, float* ctab)
 {
     for (int col = threadIdx.x; col < kCols; col += blockDim.x) {
         const bool in = col < p.d_out;
-        ctab[col] = in ? (p.col_w ? __ldg(p.col_w + col) : 1.f) : 0.f;
-        ctab[kCols + col] = (in && p.next_shift) ? __ldg(p.next_shift + col) : 0.f;
-        ctab[2 * kCols + col] = (in && p.next_shift) ? __ldg(p.next_scale + col) : 1.f;
-        ctab[3 * kCols + col] = (in && p.col_b0) ? __ldg(p.col_b0 + col) : 0.f;
+        const int at = ctab_at<kCols, EPV>(col);
+        ctab[at] = in ? (p.col_w ? __ldg(p.col_w + col) : 1.f) : 0.f;
+        ctab[kCols + at] = (in && p.next_shift) ? __ldg(p.next_shift + col) : 0.f;
+        ctab[2 * kCols + at] = (in && p.next_shift) ? __ldg(p.next_scale + col) : 1.f;
+        ctab[3 * kCols + at] = (in && p.col_b0) ? __ldg(p.col_b0 + col) : 0.f;
     }
 }
 
@@ -185,10 +197,10 @@ __device__ __forceinline__ void finish_row(const SpmmDev& p, const float* ctab, 
         float x[EPV], sh[EPV], sc[EPV];
 #pragma unroll
         for (int q = 0; q < EPV / 4; ++q) {
-            const float4 a = *reinterpret_cast<const float4*>(ctab + col0 + 4 * q);
+            const float4 a = *reinterpret_cast<const float4*>(ctab + ctab_at<kCols, EPV>(col0 + 4 * q));
             float t[4] = {acc[c][4 * q], acc[c][4 * q + 1], acc[c][4 * q + 2], acc[c][4 * q + 3]};
             if constexpr (kHalf) {
-                const float4 b0 = *reinterpret_cast<const float4*>(ctab + 3 * kCols + col0 + 4 * q);
+                const float4 b0 = *reinterpret_cast<const float4*>(ctab + 3 * kCols + ctab_at<kCols, EPV>(col0 + 4 * q));
                 t[0] = fmaf(2.f, t[0], fmaf(b0.x, wsgn, wsum));
                 t[1] = fmaf(2.f, t[1], fmaf(b0.y, wsgn, wsum));
                 t[2] = fmaf(2.f, t[2], fmaf(b0.z, wsgn, wsum));
@@ -217,8 +229,8 @@ __device__ __forceinline__ void finish_row(const SpmmDev& p, const float* ctab, 
         if (p.next_bits) {
 #pragma unroll
             for (int q = 0; q < EPV / 4; ++q) {
-                const float4 a = *reinterpret_cast<const float4*>(ctab + kCols + col0 + 4 * q);
-                const float4 b = *reinterpret_cast<const float4*>(ctab + 2 * kCols + col0 + 4 * q);
+                const float4 a = *reinterpret_cast<const float4*>(ctab + kCols + ctab_at<kCols, EPV>(col0 + 4 * q));
+                const float4 b = *reinterpret_cast<const float4*>(ctab + 2 * kCols + ctab_at<kCols, EPV>(col0 + 4 * q));
                 sh[4 * q] = a.x, sh[4 * q + 1] = a.y, sh[4 * q + 2] = a.z, sh[4 * q + 3] = a.w;
                 sc[4 * q] = b.x, sc[4 * q + 1] = b.y, sc[4 * q + 2] = b.z, sc[4 * q + 3] = b.w;
             }
@@ -380,7 +392,7 @@ __device__ __forceinline__ void stream_entries(const SpmmDev& p, uint4* ring, fl
                                 for (int c = 0; c < NCH; ++c)
 #pragma unroll
                                     for (int i = 0; i < EPV; ++i)
-                                        acc[c][i] = fmaf(2.f, acc[c][i], fmaf(ctab[3 * kCols + (c * LPR + l) * EPV + i], wsgn, wsum));
+                                        acc[c][i] = fmaf(2.f, acc[c][i], fmaf(ctab[3 * kCols + ctab_at<kCols, EPV>((c * LPR + l) * EPV + i)], wsgn, wsum));
                             }
                             return;
                         }
@@ -752,7 +764,7 @@ __device__ __forceinline__ void stream_rows_multi(const SpmmDev& p, uint4* ring,
                         for (int c = 0; c < NV; ++c)
 #pragma unroll
                             for (int i = 0; i < EPV; ++i)
-                                acc[c][i] = fmaf(2.f, acc[c][i], fmaf(ctab[3 * kCols + (c * LPR + l) * EPV + i], wsgn, wsum));
+                                acc[c][i] = fmaf(2.f, acc[c][i], fmaf(ctab[3 * kCols + ctab_at<kCols, EPV>((c * LPR + l) * EPV + i)], wsgn, wsum));
                     }
                     return;
                 }
@@ -1013,7 +1025,7 @@ __device__ __forceinline__ void stream_rows_imma(const SpmmDev& p, unsigned char
                         if (kHalf) {                          // a slice of a long row: hand back the reconstructed partial sums
 #pragma unroll
                             for (int i = 0; i < 8; ++i)
-                                accf[0][i] = fmaf(2.f, accf[0][i], fmaf(ctab[3 * 256 + 8 * lane + i], wsgn, wsum));
+                                accf[0][i] = fmaf(2.f, accf[0][i], fmaf(ctab[3 * 256 + ctab_at<256, 8>(8 * lane + i)], wsgn, wsum));
                         }
                         return;
                     }
@@ -1114,7 +1126,7 @@ spmm_imma_kernel(const SpmmDev p, int rows_per_warp)
     unsigned char* ring = dsmem + (size_t)warp * kImmaNG * kWinBytes;
     float* part = reinterpret_cast<float*>(dsmem);           // [kImmaWarps][kCols], reuses the rings
     float* ctab = reinterpret_cast<float*>(dsmem + (size_t)kImmaWarps * kImmaNG * kWinBytes);   // [4][kCols]
-    fill_col_table<kCols>(p, ctab);
+    fill_col_table<kCols, 8>(p, ctab);
     if (threadIdx.x == 0) n_long = 0;
     __syncthreads();
 
@@ -1474,7 +1486,7 @@ spmm_kernel(const SpmmDev p, int rows_per_warp)
     float* part = reinterpret_cast<float*>(dsmem);           // [kSpmmWarps][kCols], reuses the rings (see below)
     static_assert((size_t)kSpmmWarps * kCols * 4 <= (size_t)kSpmmWarps * P::RING * NCH * 512, "partials must fit the rings");
     float* ctab = reinterpret_cast<float*>(dsmem + (size_t)kSpmmWarps * P::kWarpBytes);   // [3][kCols]
-    fill_col_table<kCols>(p, ctab);
+    fill_col_table<kCols, EPV>(p, ctab);
     if (threadIdx.x == 0) n_long = 0;
     __syncthreads();
 
