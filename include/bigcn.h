@@ -39,6 +39,11 @@ extern "C" {
 #endif
 
 #define BIGCN_MAX_LAYERS 16
+/* Widest layer the contraction kernels serve: the packed K extent of a tile of feature rows and of the
+ * weight panel is kept in shared memory.  A layer with d_in above this, or d_out above
+ * BIGCN_MAX_D_OUT, is refused with BIGCN_ERR_UNSUPPORTED before anything is launched. */
+#define BIGCN_MAX_D_IN 16384
+#define BIGCN_MAX_D_OUT 512
 
 typedef enum {
     BIGCN_OK = 0,
@@ -160,7 +165,8 @@ bigcn_status bigcn_pack_weights(bigcn_ctx* ctx, const float* W, int32_t d_in, in
 
 /* One binarized layer's parameters: packed weights from bigcn_pack_weights() with
  * stride bigcn_packed_stride_words(d_in), and the optional batch-norm constants of the layer's
- * INPUT (fp32 [d_in], both or neither; Sec. 4.4). */
+ * INPUT (fp32 [d_in], both or neither; Sec. 4.4).  1 <= d_in <= BIGCN_MAX_D_IN,
+ * 1 <= d_out <= BIGCN_MAX_D_OUT. */
 typedef struct {
     int32_t d_in;
     int32_t d_out;
@@ -331,12 +337,18 @@ bigcn_status bigcn_measure_popc_peak(bigcn_ctx* ctx, double* word_steps_per_s /*
  * or any allocating routine.
  *   cuda_stream  the cudaStream_t to enqueue on (0 = default stream); the device that owns it
  *                must be the calling thread's current device.
- *   other arguments and results: exactly as bigcn_layer_forward(), default option values, without
- *   the debug taps.  Results are the same as that call's.
+ *   other arguments and results: as bigcn_layer_forward(), without the debug taps.  The integer
+ *   dots are the same; between the contraction and the aggregation they are always kept as 16-bit
+ *   values here, whereas bigcn_layer_forward() picks narrower rows for some widths and so adds the
+ *   same fp32 terms in another order: H' and next_beta agree with that call within fp32 rounding
+ *   (inside the library's tolerance 1e-4 + 1e-5 |x|), and a re-binarized bit can differ where the
+ *   value under the sign sits at the threshold within that rounding.
  * Limits and rules:
- *   - n * round_up(d_out, 8) * 2 bytes (4 bytes per element and round_up(d_out, 4) when d_in > 32767)
- *     must not exceed BIGCN_NOALLOC_SCRATCH_BYTES - 256; a larger problem is refused with
- *     BIGCN_ERR_WORKSPACE before anything is launched.
+ *   - n * round_up(d_out, 8) * 2 bytes must not exceed BIGCN_NOALLOC_SCRATCH_BYTES - 256; a larger
+ *     problem is refused with BIGCN_ERR_WORKSPACE before anything is launched.
+ *   - A bounded wait inside the tensor-core contraction that runs out makes that kernel stop early
+ *     and raise a device flag; with no context here, the flag is only reported by
+ *     bigcn_sync_check() on some context of the same device.
  *   - The first call on a device looks up the array's device address (once per device); make that
  *     first call before starting any stream capture on that device.
  *   - All calls in a process share the one array, and it keeps what the previous call left; the call

@@ -282,6 +282,22 @@ def layer_forward(g: Graph, layer: Layer, H: np.ndarray, use_pm1: bool = False) 
     return LayerTrace(F, beta, bits, bitsT, alpha, dot, zeta, H_out)
 
 
+def layer_forward_packed(g: Graph, layer: Layer, bits: np.ndarray, beta: np.ndarray) -> LayerTrace:
+    """The same layer from an input that is already binary (Sec. 5.2: packed signs F and one
+    scalar beta_i per node): sign / alpha of the weights -> F (*) B -> rescale -> A_tilde zeta.
+    The layer's batch-norm constants are not used: they act before the binarization."""
+    d_in = layer.W.shape[0]
+    bits = _arr(bits, np.uint32)
+    beta = _arr(beta, np.float32)
+    F = unpack_rows(bits, d_in)
+    B, alpha = binarize_cols(layer.W)
+    bitsT = pack_cols(B)
+    dot = dot_popc(pack_rows(F), bitsT, d_in)
+    zeta = rescale(dot, beta, alpha)
+    H_out = spmm(g, zeta)
+    return LayerTrace(F, beta, bits, bitsT, alpha, dot, zeta, H_out)
+
+
 def forward(g: Graph, layers: List[Layer], X: np.ndarray, keep_trace: bool = True):
     """L stacked layers, H^(0) = X; the last layer's output is the logits (Sec. 3.2)."""
     H = X

@@ -7,8 +7,7 @@
  * helper, no table.  Only the test-suite, the smoke check and the timed CPU
  * baseline of the benchmark may call it; the product never does.
  *
- * Conventions taken where the paper is silent or misprinted (each is also
- * listed in the design notes):
+ * Conventions taken where the paper is silent or misprinted:
  *   - sign(x) = +1 iff x >= 0 (so +0.0 and -0.0 give +1), else -1; a NaN gives -1.
  *   - the scalar of a bucket of t values is ||.||_1 / t with t = d_in for both
  *     the weight columns (Eq. "alpha", printed with 1/d_out) and the feature

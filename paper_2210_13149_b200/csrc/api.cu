@@ -69,7 +69,12 @@ int pick_format(const bigcn_ctx* ctx, int d_in, int d_out, int64_t n, bool allow
 {
     int f = ctx->zeta_format;
     const bool wide = (d_out > 128 && d_out <= 256) || (fp32_only && d_out > 32 && d_out <= 64);
-    const bool half_ok = allow_half && d_out <= 256 && d_in >= 128 && d_in <= 256 && n >= 64 && ctx->contraction != 1;
+    // half-dot bytes keep two side arrays (n node factors, d_out first weight signs) behind the byte rows inside
+    // the zeta scratch, which is sized for fp32 rows: they must fit there (they do not for d_out <= 4, where an fp32
+    // row is no longer than a byte row)
+    const bool side_fits = up((size_t)n * (size_t)zeta_ld(d_out, kZetaI8H)) + up((size_t)n * 4) + (size_t)d_out * 4
+                           <= (size_t)n * (size_t)zeta_ld(d_out, kZetaF32) * 4;
+    const bool half_ok = allow_half && d_out <= 256 && d_in >= 128 && d_in <= 256 && n >= 64 && ctx->contraction != 1 && side_fits;
     if (f == 0) {
         if (wide && d_in <= 127) f = kZetaI8;
         else if (half_ok && wide && n * (int64_t)d_out >= (int64_t(1) << 20)) f = kZetaI8H;
@@ -115,7 +120,8 @@ bigcn_status check_layer(bigcn_ctx* ctx, const bigcn_layer* l, const char* name)
 {
     if (!l) return fail(ctx, BIGCN_ERR_NULL, "%s is null", name);
     if (l->d_in < 1 || l->d_out < 1) return fail(ctx, BIGCN_ERR_SHAPE, "%s: d_in=%d d_out=%d must be >= 1", name, l->d_in, l->d_out);
-    if (l->d_out > 512) return fail(ctx, BIGCN_ERR_UNSUPPORTED, "%s: d_out=%d > 512 is not supported", name, l->d_out);
+    if (l->d_out > BIGCN_MAX_D_OUT) return fail(ctx, BIGCN_ERR_UNSUPPORTED, "%s: d_out=%d > %d is not supported", name, l->d_out, BIGCN_MAX_D_OUT);
+    if (l->d_in > BIGCN_MAX_D_IN) return fail(ctx, BIGCN_ERR_UNSUPPORTED, "%s: d_in=%d > %d is not supported", name, l->d_in, BIGCN_MAX_D_IN);
     if (!l->w_bitsT || !l->alpha) return fail(ctx, BIGCN_ERR_NULL, "%s: w_bitsT/alpha are null", name);
     if ((l->in_shift == nullptr) != (l->in_scale == nullptr)) return fail(ctx, BIGCN_ERR_NULL, "%s: in_shift and in_scale go together", name);
     if (!aligned(l->w_bitsT, 16)) return fail(ctx, BIGCN_ERR_ALIGN, "%s: w_bitsT must be 16-byte aligned", name);

@@ -662,7 +662,7 @@ cudaError_t launch_grad_h_tc(cudaStream_t s, const float* gz, int64_t ldz, const
     const size_t smem = 3 * 128 * 128 + (size_t)N * 128;
     cudaError_t e = cudaFuncSetAttribute(grad_h_tc_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, 128), 148 * 2);
+    const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, 128), sm_count() * 2);
     grad_h_tc_kernel<N><<<grid, kBwThreads, smem, s>>>(gz, ldz, alpha, W, ldw, n, d_in, d_out, g_h, ldh);
     return cudaGetLastError();
 }
@@ -710,7 +710,7 @@ int64_t pad4(int64_t d) { return (d + 3) / 4 * 4; }
 int wt_splits(int64_t n, int d_in, int d_out)
 {
     const int64_t tiles = ceil_div(d_in, kMmaTile) * ceil_div(d_out, kMmaTile);
-    const int64_t want = std::max<int64_t>(1, (148 * 4) / tiles);               // about four blocks per SM in all
+    const int64_t want = std::max<int64_t>(1, (sm_count() * 4) / tiles);               // about four blocks per SM in all
     return (int)std::max<int64_t>(1, std::min<int64_t>(want, ceil_div(n, 4 * kMmaK)));
 }
 
@@ -760,7 +760,7 @@ cudaError_t launch_layer_backward(cudaStream_t s, int64_t n, const int64_t* rowp
     // step 1a: G_zeta = A_tilde^T G' (A_tilde is symmetric: the forward aggregation on fp32 rows)
     const float* g_src = g_out;
     if (ldg != ldz || reinterpret_cast<uintptr_t>(g_out) % 16 != 0) {            // rows must be 16-byte vectors
-        pad_rows_kernel<<<(unsigned)std::min<int64_t>(ceil_div(n * ldz, 256), 148 * 16), 256, 0, s>>>(g_out, n, d_out, ldg, g_pad, ldz);
+        pad_rows_kernel<<<(unsigned)std::min<int64_t>(ceil_div(n * ldz, 256), sm_count() * 16), 256, 0, s>>>(g_out, n, d_out, ldg, g_pad, ldz);
         ++*launches;
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;

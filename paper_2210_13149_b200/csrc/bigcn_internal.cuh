@@ -25,6 +25,10 @@ inline int64_t zeta_ld(int d_out, int fmt)
 }
 inline int zeta_elt_bytes(int fmt) { return fmt == kZetaF32 ? 4 : ((fmt == kZetaI8 || fmt == kZetaI8H) ? 1 : 2); }
 
+// Number of multiprocessors of the calling thread's current device (queried once per device; 1 if the query
+// fails, so that a grid derived from it stays valid).  Persistent grids are sized from it.
+int sm_count();
+
 // ---- launchers (each returns the launch status; all asynchronous on `s`) ------------------------
 
 cudaError_t launch_pack_rows(cudaStream_t s, const float* H, int64_t n, int d, int64_t ld,

@@ -140,7 +140,7 @@ cudaError_t launch_inst(cudaStream_t s, const uint32_t* A, int64_t stride_a, con
     }
     const int64_t n_tiles = ceil_div(n, kTileRows);
     const unsigned gy = (unsigned)ceil_div(d_out, TN * 32);
-    const unsigned gx = (unsigned)std::min<int64_t>(n_tiles, 148 * 8);
+    const unsigned gx = (unsigned)std::min<int64_t>(n_tiles, sm_count() * 8);
     bitgemm_kernel<TN, FMT, DBG><<<dim3(gx, gy), kGemmThreads, smem_bytes, s>>>(
         A, stride_a, BT, stride_b, n, d_in, d_out, kw, ldb, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta);
     return cudaGetLastError();

@@ -321,10 +321,13 @@ cudaError_t launch_tc_inst(cudaStream_t s, const uint32_t* A, int64_t stride_a, 
                            int32_t* dbg_dot, float* dbg_zeta, float* nws, float* col_b0)
 {
     // operands: weight panel N x K bytes, feature tile 128 x K bytes (at least the 32 KB the epilogue's scratch needs)
-    const size_t smem = (size_t)N * stride_a * 32 + std::max<size_t>((size_t)kTcRows * stride_a * 32, 32 * 1024);
+    size_t smem = (size_t)N * stride_a * 32 + std::max<size_t>((size_t)kTcRows * stride_a * 32, 32 * 1024);
+    // a CTA holds 256 of the SM's 512 tensor-memory columns when N > 128: ask for enough shared memory that a third
+    // CTA can never become resident on an SM and sit in tcgen05.alloc until a neighbour leaves
+    if (N > 128) smem = std::max<size_t>(smem, 78 * 1024);
     cudaError_t e = cudaFuncSetAttribute(bitgemm_tc_kernel<N, FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, kTcRows), 148 * 2);
+    const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, kTcRows), sm_count() * 2);
     bitgemm_tc_kernel<N, FMT><<<grid, kTcThreads, smem, s>>>(A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0);
     return cudaGetLastError();
 }

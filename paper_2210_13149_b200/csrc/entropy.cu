@@ -167,7 +167,7 @@ cudaError_t launch_histogram(cudaStream_t s, const float* H, int64_t n, int d, i
     const unsigned gy = (unsigned)ceil_div(d, CW);
     const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(8, (200 * 1024) / std::max<size_t>(smem, 1)));
     // about one resident wave of blocks over both grid dimensions; every block takes a contiguous range of rows
-    const int64_t gx = std::max<int64_t>(1, std::min<int64_t>(ceil_div(n, 1024), ceil_div((int64_t)148 * per_sm, gy)));
+    const int64_t gx = std::max<int64_t>(1, std::min<int64_t>(ceil_div(n, 1024), ceil_div((int64_t)sm_count() * per_sm, gy)));
     const int64_t rows_per_block = ceil_div(n, gx);
     histogram_kernel<CW><<<dim3((unsigned)gx, gy), kEntThreads, smem, s>>>(H, n, d, ld, n_bins, rows_per_block, key_min,
                                                                          key_max, col_min, col_max, counts);
@@ -192,7 +192,7 @@ cudaError_t launch_entropy_bins(cudaStream_t s, const float* H, int64_t n, int d
     if (e != cudaSuccess) return e;
     {
         const unsigned gy = (unsigned)ceil_div(d, 32);
-        const int64_t gx = std::max<int64_t>(1, std::min<int64_t>(ceil_div(n, 256), ceil_div((int64_t)148 * 8, gy)));
+        const int64_t gx = std::max<int64_t>(1, std::min<int64_t>(ceil_div(n, 256), ceil_div((int64_t)sm_count() * 8, gy)));
         range_kernel<<<dim3((unsigned)gx, gy), kEntThreads, 0, s>>>(H, n, d, ld, ceil_div(n, gx), key_min, key_max);
         ++*launches;
         if ((e = cudaGetLastError()) != cudaSuccess) return e;

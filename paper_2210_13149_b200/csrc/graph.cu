@@ -179,13 +179,17 @@ col_partial_kernel(const float* __restrict__ H, int64_t n, int d, int64_t ld, in
     const int j = blockIdx.x * 32 + tx;
     const int64_t r0 = (int64_t)blockIdx.y * rows_per_chunk;
     const int64_t r1 = min(n, r0 + rows_per_chunk);
+    // sums of (x - pivot) and (x - pivot)^2 around the column's first value: the variance formed from them does
+    // not cancel for a column with a large offset, and is exactly 0 for a constant one
     double s = 0.0, q = 0.0;
-    if (j < d)
+    if (j < d) {
+        const double pivot = (double)__ldg(H + j);
         for (int64_t r = r0 + ty; r < r1; r += 8) {
-            const double x = (double)__ldg(H + r * ld + j);
+            const double x = (double)__ldg(H + r * ld + j) - pivot;
             s += x;
             q += x * x;
         }
+    }
     s_sum[ty][tx] = s;
     s_sq[ty][tx] = q;
     __syncthreads();
@@ -197,7 +201,7 @@ col_partial_kernel(const float* __restrict__ H, int64_t n, int d, int64_t ld, in
     }
 }
 
-__global__ void col_final_kernel(const double* __restrict__ partial, int chunks, int d, int64_t n, double eps,
+__global__ void col_final_kernel(const float* __restrict__ H, const double* __restrict__ partial, int chunks, int d, int64_t n, double eps,
                                  float* __restrict__ shift, float* __restrict__ scale)
 {
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
@@ -207,8 +211,9 @@ __global__ void col_final_kernel(const double* __restrict__ partial, int chunks,
         s += partial[((int64_t)c * d + j) * 2];
         q += partial[((int64_t)c * d + j) * 2 + 1];
     }
-    const double mean = n > 0 ? s / (double)n : 0.0;
-    double var = n > 0 ? q / (double)n - mean * mean : 0.0;
+    const double off = n > 0 ? s / (double)n : 0.0;                       // mean of x - pivot
+    const double mean = n > 0 ? (double)__ldg(H + j) + off : 0.0;
+    double var = n > 0 ? q / (double)n - off * off : 0.0;
     if (var < 0.0) var = 0.0;
     shift[j] = (float)mean;
     scale[j] = (float)(1.0 / sqrt(var + eps));
@@ -255,7 +260,7 @@ cudaError_t launch_col_stats(cudaStream_t s, const float* H, int64_t n, int d, i
     ++*launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    col_final_kernel<<<(unsigned)ceil_div(d, 128), 128, 0, s>>>(partial, chunks, d, n, (double)eps, shift, scale);
+    col_final_kernel<<<(unsigned)ceil_div(d, 128), 128, 0, s>>>(H, partial, chunks, d, n, (double)eps, shift, scale);
     ++*launches;
     return cudaGetLastError();
 }

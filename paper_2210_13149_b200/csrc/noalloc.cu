@@ -57,7 +57,7 @@ extern "C" bigcn_status bigcn_layer_forward_noalloc(void* cuda_stream, const big
     if (!graph || !layer) return BIGCN_ERR_NULL;
     if (graph->n < 0 || graph->n >= (int64_t(1) << 31) || graph->nnz < 0) return BIGCN_ERR_SHAPE;
     if (layer->d_in < 1 || layer->d_out < 1) return BIGCN_ERR_SHAPE;
-    if (layer->d_out > 512) return BIGCN_ERR_UNSUPPORTED;
+    if (layer->d_out > BIGCN_MAX_D_OUT || layer->d_in > BIGCN_MAX_D_IN) return BIGCN_ERR_UNSUPPORTED;
     if (!layer->w_bitsT || !layer->alpha) return BIGCN_ERR_NULL;
     if (next && next->d_in != layer->d_out) return BIGCN_ERR_SHAPE;
     if (next && ((next->in_shift == nullptr) != (next->in_scale == nullptr))) return BIGCN_ERR_NULL;
@@ -69,8 +69,8 @@ extern "C" bigcn_status bigcn_layer_forward_noalloc(void* cuda_stream, const big
     if (next && (!next_bits || !next_beta)) return BIGCN_ERR_NULL;
     if (!aligned16(in_bits) || !aligned16(layer->w_bitsT)) return BIGCN_ERR_ALIGN;
 
-    // zeta as integers coded in fp16 (int16 / fp32 beyond their exact ranges): 2 bytes per element decide the size limit
-    const int fmt = layer->d_in <= 2048 ? kZetaF16 : (layer->d_in <= 32767 ? kZetaI16 : kZetaF32);
+    // zeta as integers coded in fp16 (int16 beyond fp16's exact range): 2 bytes per element decide the size limit
+    const int fmt = layer->d_in <= 2048 ? kZetaF16 : kZetaI16;
     const int64_t ldz = zeta_ld(layer->d_out, fmt);
     const size_t zeta_bytes = (size_t)graph->n * (size_t)ldz * zeta_elt_bytes(fmt);
     if (zeta_bytes > BIGCN_NOALLOC_SCRATCH_BYTES - kCounterBytes) return BIGCN_ERR_WORKSPACE;   // problem too large for the built-in scratch

@@ -287,7 +287,7 @@ cudaError_t launch_pack_rows(cudaStream_t s, const float* H, int64_t n, int d, i
     }
     const int kw = (d + 31) / 32;
     const int rows = kw <= 4 ? 8 : (kw <= 8 ? 4 : (kw <= 32 ? 2 : 1));     // rows a warp packs at a time
-    const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, (int64_t)kPackWarpsPerBlock * rows), 148 * 8);
+    const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, (int64_t)kPackWarpsPerBlock * rows), sm_count() * 8);
     const dim3 block(kPackWarpsPerBlock * kWarp);
 #define BIGCN_PACK_LAUNCH(NORM, R, WC) \
     pack_rows_kernel<NORM, R, WC><<<grid, block, 0, s>>>(H, n, d, ld, shift, scale, bits, stride, beta)

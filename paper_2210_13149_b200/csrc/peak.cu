@@ -34,13 +34,13 @@ popc_peak_kernel(uint32_t* out, int iters, uint32_t seed)
 
 }  // namespace
 
-size_t popc_peak_scratch_bytes() { return (size_t)148 * 8 * 256 * sizeof(uint32_t); }
+size_t popc_peak_scratch_bytes() { return (size_t)sm_count() * 8 * 256 * sizeof(uint32_t); }
 
 // Runs the loop three times and returns the best rate in 32-bit word steps (one XOR, one bit count,
 // one add on 32 bits) per second.  Synchronises the stream.
 cudaError_t measure_popc_peak(cudaStream_t s, void* scratch, double* word_steps_per_s, int* launches)
 {
-    const int blocks = 148 * 8, iters = 20000;
+    const int blocks = sm_count() * 8, iters = 20000;
     cudaEvent_t e0, e1;
     cudaError_t e = cudaEventCreate(&e0);
     if (e != cudaSuccess) return e;

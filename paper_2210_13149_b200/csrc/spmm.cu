@@ -1190,13 +1190,13 @@ cudaError_t launch_imma(cudaStream_t s, SpmmDev p)
 {
     constexpr size_t smem = (size_t)kImmaWarps * kImmaNG * kWinBytes + 4 * 256 * sizeof(float);
     p.nv_fin = 2 * p.nv;                                      // the row epilogue works on groups of 8 columns
-    const int rows_per_warp = (int)std::min<int64_t>(kMaxRowsPerWarp, std::max<int64_t>(1, p.n / (kImmaWarps * 148 * 8)));
+    const int rows_per_warp = (int)std::min<int64_t>(kMaxRowsPerWarp, std::max<int64_t>(1, p.n / (kImmaWarps * sm_count() * 8)));
     cudaError_t e = cudaFuncSetAttribute(spmm_imma_kernel<kFull, kHalf>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     e = cudaMemsetAsync(p.run_counter, 0, sizeof(int), s);
     if (e != cudaSuccess) return e;
     const int64_t wanted = ceil_div(ceil_div(p.n, rows_per_warp), kImmaWarps);
-    const unsigned grid = (unsigned)std::min<int64_t>(wanted, 148);
+    const unsigned grid = (unsigned)std::min<int64_t>(wanted, sm_count());
     spmm_imma_kernel<kFull, kHalf><<<grid, kImmaThreads, smem, s>>>(p, rows_per_warp);
     return cudaGetLastError();
 }
@@ -1445,13 +1445,13 @@ template <int NV, bool kHalf>
 cudaError_t launch_lane(cudaStream_t s, const SpmmDev& p)
 {
     constexpr size_t smem = ((size_t)kLaneWarps * 32 * kLanePitch + (size_t)kLaneWarps * (NV * 16 + 4)) * sizeof(float);
-    const int rows_per_warp = (int)std::min<int64_t>(kMaxRowsPerWarp, std::max<int64_t>(1, p.n / (kLaneWarps * 148 * 8)));
+    const int rows_per_warp = (int)std::min<int64_t>(kMaxRowsPerWarp, std::max<int64_t>(1, p.n / (kLaneWarps * sm_count() * 8)));
     cudaError_t e = cudaFuncSetAttribute(spmm_lane_kernel<NV, kHalf>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     e = cudaMemsetAsync(p.run_counter, 0, sizeof(int), s);
     if (e != cudaSuccess) return e;
     const int64_t wanted = ceil_div(ceil_div(p.n, rows_per_warp), kLaneWarps);
-    const unsigned grid = (unsigned)std::min<int64_t>(wanted, 148 * 2);
+    const unsigned grid = (unsigned)std::min<int64_t>(wanted, sm_count() * 2);
     spmm_lane_kernel<NV, kHalf><<<grid, kLaneThreads, smem, s>>>(p, rows_per_warp);
     return cudaGetLastError();
 }
@@ -1572,7 +1572,7 @@ cudaError_t launch_one(cudaStream_t s, const SpmmDev& p)
     constexpr int kCols = NCH * (LPR < 32 ? LPR : 32) * Elt<T>::kPerVec;
     constexpr size_t smem = kSpmmWarps * Pipe<NCH, LPR, kAligned>::kWarpBytes + 4 * kCols * sizeof(float);   // rings, weights, column table
     // enough thread blocks to fill the machine on small graphs, long runs of rows on large ones
-    const int rows_per_warp = (int)std::min<int64_t>(kMaxRowsPerWarp, std::max<int64_t>(1, p.n / (kSpmmWarps * 148 * 8)));
+    const int rows_per_warp = (int)std::min<int64_t>(kMaxRowsPerWarp, std::max<int64_t>(1, p.n / (kSpmmWarps * sm_count() * 8)));
     if (smem > 40 * 1024) {                                   // above the default limit: opt in
         cudaError_t e = cudaFuncSetAttribute(spmm_kernel<T, NCH, LPR, kFull, kAligned, kHalf>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -1581,7 +1581,7 @@ cudaError_t launch_one(cudaStream_t s, const SpmmDev& p)
     if (e != cudaSuccess) return e;
     // one wave of resident blocks; the warps pull runs of rows until none are left
     const int64_t wanted = ceil_div(ceil_div(p.n, rows_per_warp), kSpmmWarps);
-    const unsigned grid = (unsigned)std::min<int64_t>(wanted, 148 * spmm_blocks_per_sm<NCH, LPR, kAligned, (int)sizeof(T)>());
+    const unsigned grid = (unsigned)std::min<int64_t>(wanted, sm_count() * spmm_blocks_per_sm<NCH, LPR, kAligned, (int)sizeof(T)>());
     spmm_kernel<T, NCH, LPR, kFull, kAligned, kHalf><<<grid, kSpmmThreads, smem, s>>>(p, rows_per_warp);
     return cudaGetLastError();
 }

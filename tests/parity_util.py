@@ -103,24 +103,50 @@ def unpack_signs_dev(bits: torch.Tensor, d: int) -> torch.Tensor:
 
 
 def end_to_end_with_flip_accounting(ctx, G, layers, run: OracleRun, X: torch.Tensor):
-    """Runs the network layer by layer on the GPU's own intermediate results and checks it against
-    the oracle: every fp32 output row that is not downstream of a re-binarization disagreement must be
-    within tolerance, and every disagreement that is not itself downstream of an earlier one must sit
-    at the threshold (the oracle's pre-sign value within the fp32 tolerance of it).
+    """Runs the network layer by layer on the GPU's own intermediate results and checks EVERY row of
+    EVERY layer against the oracle -- no row is exempt:
 
-    Returns a dict with the counts that are reported: threshold flips per layer, share of output rows
-    downstream of a flip, share of logits outside tolerance overall, argmax agreement."""
+    * layer 0 gets the same packed input on both sides (asserted bit for bit), so its output is
+      compared with the oracle's own layer 0;
+    * every later layer is compared with the oracle's layer fed the GPU's own packed input (the
+      re-binarized bits unpacked by the oracle, and the GPU's beta): all rows of H' within the
+      tolerance, re-binarized bits equal to the sign of that reference except where the reference
+      lies within the tolerance of the threshold, the next beta within the tolerance.
+
+    Beside that it keeps the accounting against the oracle's own end-to-end run (whose later layers
+    see the oracle's bits, so a threshold flip moves the rows downstream of it): threshold flips per
+    layer, share of logit rows downstream of a flip, share of logits outside tolerance, argmax
+    agreement.  Those figures are reported, not asserted, except that a flip which is not itself
+    downstream of an earlier one must sit at the threshold."""
     n = G.n
     A = torch.sparse_csr_tensor(G.rowptr, G.colidx.long(), torch.ones_like(G.val), size=(n, n))
     L = len(layers)
     bits, beta = ctx.pack_features(X, layers[0].in_shift, layers[0].in_scale)
     assert torch.equal(bits, bits_to_dev(run.traces[0].bits)), "first-layer packed bits differ from the oracle"
     dirty = torch.zeros(n, dtype=torch.bool, device=X.device)          # rows whose packed input differs
-    report = {"origin_flips": [], "dirty_rows": []}
+    report = {"origin_flips": [], "dirty_rows": [], "own_fed_flips": [], "own_fed_worst_ratio": []}
     for l in range(L):
         t = run.traces[l]
         nxt = layers[l + 1] if l + 1 < L else None
         out = ctx.layer_forward(G, layers[l], bits, beta, want_h=True, next_layer=nxt)
+        # ---- the complete check: the oracle's layer on the very input the GPU's layer saw
+        if l == 0:
+            own_H = t.H_out
+        else:
+            own_H = oracle.layer_forward_packed(run.graph, run.layers[l], bits_from_dev(bits), beta.cpu().numpy()).H_out
+        ok, ratio, mx = within_tol(out["h"], torch.from_numpy(own_H))
+        assert ok, "layer %d on the GPU's own input: H' error / allowance = %.3g (max abs %.3g)" % (l, ratio, mx)
+        report["own_fed_worst_ratio"].append(ratio)
+        if nxt is not None:
+            nl = run.layers[l + 1]
+            own_F, own_beta = oracle.binarize_rows(own_H, nl.in_shift, nl.in_scale)
+            flips, bad, total = flip_report(bits_from_dev(out["next_bits"]), own_F, own_H, nl.in_shift)
+            assert bad == 0, "layer %d on the GPU's own input: %d of %d sign flips away from the threshold" % (l, bad, flips)
+            report["own_fed_flips"].append(flips)
+            np.testing.assert_allclose(out["next_beta"].cpu().numpy(), own_beta, rtol=RTOL, atol=ATOL)
+            del own_F, own_beta
+        del own_H
+        # ---- accounting against the oracle's own end-to-end run
         tainted = (A @ dirty.to(torch.float32).unsqueeze(1)).squeeze(1) > 0    # rows that gather a differing row
         ref = dev(t.H_out)
         err = (out["h"].double() - ref.double()).abs()

@@ -82,3 +82,25 @@ def test_null_context_is_rejected(lib):
     assert lib.bigcn_sync_check(None) != 0
     assert lib.bigcn_launch_count(None) == 0
     assert lib.bigcn_last_error(None) == b"context is null"
+
+
+def test_layer_width_limits_are_refused_on_the_host(lib):
+    """A layer wider than the contraction kernels serve (their shared-memory tiles hold the whole packed K extent)
+    is refused as unsupported by argument validation, before any GPU work: checked through the entry point that needs
+    no context.  The header states the limits."""
+    from paper_2210_13149_b200 import binding
+    text = open(HEADER).read()
+    max_in = int(re.search(r"#define BIGCN_MAX_D_IN (\d+)", text).group(1))
+    max_out = int(re.search(r"#define BIGCN_MAX_D_OUT (\d+)", text).group(1))
+    assert max_in * 384 // 32 + 1024 <= 200 * 1024          # 96 words of tile and panel per 32 inputs + slack fit the kernel's shared memory
+    g = binding.bigcn_graph(n=4, nnz=4, rowptr=None, colidx=None, val=None, dinv=None)
+    fake = ctypes.c_void_p(256)                             # never dereferenced: validation fails first
+
+    def call(d_in, d_out):
+        layer = binding.bigcn_layer(d_in=d_in, d_out=d_out, w_bitsT=fake, alpha=fake, in_shift=None, in_scale=None)
+        return lib.bigcn_layer_forward_noalloc(None, ctypes.byref(g), ctypes.byref(layer), fake, fake, fake, d_out, None, None, None)
+
+    assert call(max_in + 1, 8) == 7                         # BIGCN_ERR_UNSUPPORTED
+    assert call(8, max_out + 1) == 7
+    assert call(0, 8) == 2                                  # BIGCN_ERR_SHAPE
+    assert call(max_in, max_out) == 1                       # passes the width checks; the null rowptr is caught next

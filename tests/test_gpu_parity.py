@@ -125,13 +125,24 @@ def test_pack_weights(ctx, d_in, d_out):
     np.testing.assert_allclose(ga.cpu().numpy(), alpha, rtol=1e-6)
 
 
-def test_col_stats(ctx):
-    rng = np.random.default_rng(9)
-    H = (rng.standard_normal((5000, 77)) * 3 + 1.5).astype(np.float32)
+@pytest.mark.parametrize("n,d,pad", [(1, 5, 0), (2, 47, 3), (5000, 77, 0), (4099, 256, 8), (700, 1433, 0), (300, 3703, 5),
+                                     (40000, 1, 0), (2449029, 3, 1)])
+def test_col_stats(ctx, n, d, pad):
+    """Batch statistics of Sec. 4.4 against the oracle (two passes in double): any width, rows with a leading
+    dimension larger than the width, a single row, a constant column (variance exactly 0, scale = eps^-1/2) and a
+    column with an offset a thousand times its spread."""
+    rng = np.random.default_rng(9 + n + d)
+    H = (rng.standard_normal((n, d)) * 3 + 1.5).astype(np.float32)
+    H[:, 0] = 3.25                                              # constant
+    if d > 2:
+        H[:, 2] = (1000.0 + rng.standard_normal(n)).astype(np.float32)
     shift, scale = oracle.col_stats(H)
-    gs, gc = ctx.col_stats(dev(H))
+    buf = np.full((n, d + pad), np.float32(7e9))                # whatever lies beyond a row's d columns is not read
+    buf[:, :d] = H
+    gs, gc = ctx.col_stats(dev(buf)[:, :d])
     np.testing.assert_allclose(gs.cpu().numpy(), shift, rtol=1e-6, atol=1e-7)
     np.testing.assert_allclose(gc.cpu().numpy(), scale, rtol=1e-6)
+    assert gc[0].item() == pytest.approx(1e-5 ** -0.5, rel=1e-6)
 
 
 # --------------------------------------------------------------------------- one layer, oracle-fed
@@ -350,7 +361,7 @@ def check_layer_forward(ctx, B, fmt, n, e, d_in, d_out):
     if d_out % 32:
         assert (nb[:, d_out // 32] >> (d_out % 32) == 0).all()
     assert (nb[:, (d_out + 31) // 32:] == 0).all()
-    np.testing.assert_allclose(out["next_beta"].cpu().numpy(), beta_n, rtol=1e-4, atol=1e-5)
+    np.testing.assert_allclose(out["next_beta"].cpu().numpy(), beta_n, rtol=RTOL, atol=ATOL)
 
 
 @pytest.mark.parametrize("fmt", FORMATS)
@@ -481,7 +492,7 @@ def test_network_layer_by_layer_oracle_fed(B, net, fmt):
             tn = net.traces[l + 1]
             flips, bad, total = flip_report(bits_from_dev(out["next_bits"]), tn.F, t.H_out, net.layers[l + 1].in_shift)
             assert bad == 0 and flips <= max(2, total // 2000), (flips, bad, total)
-            np.testing.assert_allclose(out["next_beta"].cpu().numpy(), tn.beta, rtol=1e-4, atol=1e-5)
+            np.testing.assert_allclose(out["next_beta"].cpu().numpy(), tn.beta, rtol=RTOL, atol=ATOL)
     ctx.sync_check()
     ctx.close()
 

@@ -5,7 +5,7 @@ import torch
 
 import oracle
 from paper_2210_13149_b200 import synth
-from parity_util import assert_close, bits_from_dev, bits_to_dev, dev, flip_report
+from parity_util import ATOL, RTOL, assert_close, bits_from_dev, bits_to_dev, dev, flip_report
 
 pytestmark = pytest.mark.gpu
 
@@ -32,9 +32,13 @@ def test_mean_adjacency_is_bit_exact(ctx, n, e, seed):
     assert np.array_equal(got.dinv.cpu().numpy(), g.dinv)
 
 
-@pytest.mark.parametrize("fmt", [1, 2, 4])
+# storage of the neighbours' dots between contraction and aggregation: 0 = the automatic choice (bytes for 129..256
+# columns when d_in <= 127), 1 fp32, 2 int16, 3 bytes, 4 fp16, 5 half-dot bytes (not offered to this layer: falls back);
+# the (4200, .., 256, 256) case has 2^20 outputs, from where the contraction runs on the tensor cores
+@pytest.mark.parametrize("fmt", [0, 1, 2, 3, 4, 5])
 @pytest.mark.parametrize("n,e,d_in,d_out", [(300, 2500, 33, 7), (500, 6000, 100, 256), (400, 5000, 602, 256),
-                                             (600, 9000, 256, 47), (450, 4000, 64, 6), (350, 3000, 1433, 64)])
+                                             (600, 9000, 256, 47), (450, 4000, 64, 6), (350, 3000, 1433, 64),
+                                             (4200, 50000, 256, 256)])
 def test_sage_layer_against_oracle(ctx, fmt, n, e, d_in, d_out):
     from paper_2210_13149_b200 import binding as B
     rng = np.random.default_rng(n + 5 * d_in + 11 * d_out)
@@ -58,7 +62,7 @@ def test_sage_layer_against_oracle(ctx, fmt, n, e, d_in, d_out):
     assert_close(out["h"], t.H_out, "Bi-GraphSAGE layer output")
     flips, bad, total = flip_report(bits_from_dev(out["next_bits"]), Fn, t.H_out, nshift)
     assert bad == 0 and flips <= max(2, total // 2000), (flips, bad, total)
-    np.testing.assert_allclose(out["next_beta"].cpu().numpy(), beta_n, rtol=1e-4, atol=1e-5)
+    np.testing.assert_allclose(out["next_beta"].cpu().numpy(), beta_n, rtol=RTOL, atol=ATOL)
 
 
 def test_sage_layer_on_pm1_inputs_is_the_graphsage_mean_layer(ctx):
@@ -101,10 +105,16 @@ def test_two_sage_layers_chain_through_the_fused_rebinarization(ctx):
     assert np.array_equal(bits_from_dev(bits), t0.bits)
     o0 = ctx.sage_layer_forward(G, layers[0][0], layers[0][1], bits, beta, want_h=True, next_layer=layers[1][0])
     assert_close(o0["h"], t0.H_out, "layer 0")
-    flips = int((oracle.unpack_rows(bits_from_dev(o0["next_bits"]), dims[1]) != t1.F).sum())
+    # the re-binarized bits differ from the oracle's only at the threshold
+    flips, bad, total = flip_report(bits_from_dev(o0["next_bits"]), t1.F, t0.H_out, None)
+    assert bad == 0 and flips <= 4, (flips, bad, total)
     o1 = ctx.sage_layer_forward(G, layers[1][0], layers[1][1], o0["next_bits"], o0["next_beta"], want_h=True)
+    # every row of the second layer against the oracle's steps on the very input it saw (the GPU's own bits and beta)
+    own_bits, own_beta = bits_from_dev(o0["next_bits"]), o0["next_beta"].cpu().numpy()
+    Bs, a_s = oracle.binarize_cols(W[1][0])
+    Bn, a_n = oracle.binarize_cols(W[1][1])
+    z_s = oracle.rescale(oracle.dot_popc(own_bits, oracle.pack_cols(Bs), dims[1]), own_beta, a_s)
+    z_n = oracle.rescale(oracle.dot_popc(own_bits, oracle.pack_cols(Bn), dims[1]), own_beta, a_n)
+    assert_close(o1["h"], oracle.spmm_add(g, z_n, z_s), "logits on the GPU's own second-layer input")
     if flips == 0:
         assert_close(o1["h"], t1.H_out, "logits")
-    else:
-        agree = float((o1["h"].cpu().argmax(1) == torch.from_numpy(t1.H_out).argmax(1)).double().mean())
-        assert flips <= 4 and agree > 0.99

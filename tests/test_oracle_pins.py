@@ -306,6 +306,36 @@ def test_layer_is_the_l2_optimal_binary_approximation_chain():
     np.testing.assert_allclose(t.H_out, dense @ (H_tilde @ W_tilde), rtol=1e-5, atol=1e-6)
 
 
+def test_layer_from_packed_input_is_the_dense_product_of_its_own_input():
+    """The layer that starts from an input that is already binary (packed signs and one scalar per node, Sec. 5.2):
+    against the dense product A_tilde (diag(beta) F) (B diag(alpha)) formed with numpy from bits written by hand
+    (np.packbits layout, not the oracle's packer), with beta an arbitrary vector that is NOT the row mean of
+    anything; and equal, bit for bit, to the layer that binarizes the fp32 input itself when given that layer's bits."""
+    rng = np.random.default_rng(24)
+    n, d, c = 14, 45, 6
+    pairs = random_pairs(rng, n, 35)
+    g = oracle.normalize_adjacency(n, pairs[:, 0], pairs[:, 1])
+    W = rng.standard_normal((d, c)).astype(np.float32)
+    F = rng.choice(np.array([-1, 1], np.int8), size=(n, d))
+    beta = (rng.random(n) * 2 + 0.1).astype(np.float32)
+    stride = oracle.stride_words(d)
+    padded = np.zeros((n, stride * 32), np.uint8)
+    padded[:, :d] = F > 0
+    bits = np.packbits(padded, axis=1, bitorder="little").view("<u4").reshape(n, stride)
+    t = oracle.layer_forward_packed(g, oracle.Layer(W), bits, beta)
+    alpha = np.abs(W).astype(np.float64).mean(0)
+    dense, _ = dense_norm_adj(n, pairs.tolist())
+    want = dense @ ((beta.astype(np.float64)[:, None] * F) @ (np.where(W >= 0, 1.0, -1.0) * alpha[None, :]))
+    np.testing.assert_allclose(t.H_out, want, rtol=1e-5, atol=1e-6)
+    assert np.array_equal(t.dot, F.astype(np.int64) @ np.where(W >= 0, 1, -1))
+    # a transposed or mis-scaled operand would show: beta scales rows, alpha columns
+    assert not np.allclose(t.H_out, dense @ ((F @ np.where(W >= 0, 1.0, -1.0)) * alpha[None, :]), rtol=1e-3)
+    H = rng.standard_normal((n, d)).astype(np.float32)
+    t1 = oracle.layer_forward(g, oracle.Layer(W), H)
+    t2 = oracle.layer_forward_packed(g, oracle.Layer(W), t1.bits, t1.beta)
+    assert np.array_equal(t1.H_out, t2.H_out) and np.array_equal(t1.dot, t2.dot) and np.array_equal(t1.zeta, t2.zeta)
+
+
 def test_batchnorm_apply_balances_bits():
     rng = np.random.default_rng(31)
     H = (rng.random((400, 13)) < 0.05).astype(np.float32) * 3 + 2    # far from zero-centred
