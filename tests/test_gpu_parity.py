@@ -3,6 +3,8 @@
 Packed bits and integer dot products must match exactly; fp32 outputs within
 |gpu - oracle| <= 1e-4 + 1e-5 |oracle| when the layer is fed the oracle's own input.
 """
+import ctypes
+
 import numpy as np
 import pytest
 import torch
@@ -255,6 +257,37 @@ def test_byte_rows_signed_edge_values_of_wide_range(ctx, B, fmt, d_in, span):
 
 
 # a network's last layer (fp32 output only) with 33..64 byte columns: the stream with one stored entry per lane
+@pytest.mark.parametrize("d_in", [128, 256])
+@pytest.mark.parametrize("d_out", [1, 4, 5, 8, 16])
+def test_half_dot_bytes_asked_for_on_tiny_widths_stay_inside_an_exactly_sized_workspace(B, d_in, d_out):
+    """Half-dot bytes keep two side arrays behind the byte rows inside the zeta scratch.  For d_out <= 4 they do not
+    fit there (an fp32 row is no longer than a byte row), so the format falls back; from d_out = 5 they fit.  Either
+    way the layer must match the oracle and must not write past a workspace of exactly bigcn_workspace_bytes()."""
+    n = 300
+    rng = np.random.default_rng(17 * d_in + d_out)
+    _, _, g = small_graph(n, 2500, 77)
+    H = rng.standard_normal((n, d_in)).astype(np.float32)
+    W = (rng.standard_normal((d_in, d_out)) * d_in ** -0.5).astype(np.float32)
+    t = oracle.layer_forward(g, oracle.Layer(W), H)
+    ctx = B.BiGCN(0)
+    ctx.set_option(B.OPT_ZETA_FORMAT, 5)
+    need = ctx.workspace_bytes(n, g.nnz, [d_in, d_out])
+    guard = 1 << 16
+    buf = torch.full((need + guard,), 0xAB, dtype=torch.uint8, device="cuda")
+    ctx.workspace = buf                                         # keeps the tensor alive; the library sees `need` bytes only
+    ctx._check(ctx.lib.bigcn_set_workspace(ctx.h, ctypes.c_void_p(buf.data_ptr()), need))
+    G = device_graph(B, g)
+    layer = B.make_layer(d_in, d_out, bits_to_dev(t.bitsT), dev(t.alpha))
+    for _ in range(2):                                          # the second call finds the first one's leftovers
+        out = ctx.layer_forward(G, layer, bits_to_dev(t.bits), dev(t.beta), want_h=True, debug=True)
+        ctx.sync_check()
+        assert ctx.workspace is buf
+        assert np.array_equal(out["dot"].cpu().numpy(), t.dot)
+        assert_close(out["h"], t.H_out, "H'")
+        assert bool((buf[need:] == 0xAB).all()), "bytes behind the workspace were written"
+    ctx.close()
+
+
 LAST_LAYER_SHAPES = [(5, 3000, 30000, 256, 47), (5, 2000, 120000, 256, 47), (5, 40000, 400000, 256, 41), (5, 900, 9000, 129, 33),
                      (5, 900, 9000, 254, 64), (5, 1500, 40000, 200, 48), (3, 3000, 30000, 100, 47), (3, 900, 20000, 127, 64),
                      (5, 64, 300, 256, 47), (5, 2000, 5000, 256, 47)]
