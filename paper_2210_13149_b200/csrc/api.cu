@@ -5,6 +5,7 @@
 #include <new>
 
 #include "bigcn_internal.cuh"
+#include "spmm_dev.cuh"
 
 using namespace bigcn;
 
@@ -357,7 +358,7 @@ bigcn_status bigcn_set_option(bigcn_ctx* ctx, int32_t option, int64_t value)
             ctx->contraction = (int)value;
             return BIGCN_OK;
         case BIGCN_OPT_BYTE_AGGREGATION:
-            if (value < 0 || value > 2) return fail(ctx, BIGCN_ERR_SHAPE, "byte aggregation path %lld not in 0..2", (long long)value);
+            if (value < 0 || value > 3) return fail(ctx, BIGCN_ERR_SHAPE, "byte aggregation path %lld not in 0..3", (long long)value);
             ctx->byte_path = (int)value;
             return BIGCN_OK;
     }
@@ -374,6 +375,7 @@ bigcn_status bigcn_sync_check(bigcn_ctx* ctx)
     BIGCN_CUDA(ctx, cudaGetLastError());
     if (bitgemm_tc_timeouts() != 0) return fail(ctx, BIGCN_ERR_INTERNAL, "a bounded wait on the tensor cores ran out (contraction kernel)");
     if (backward_tc_timeouts() != 0) return fail(ctx, BIGCN_ERR_INTERNAL, "a bounded wait on the tensor cores ran out (backward kernel)");
+    if (spmm_tc_timeouts() != 0) return fail(ctx, BIGCN_ERR_INTERNAL, "a bounded wait ran out (tensor-core aggregation kernel)");
     return BIGCN_OK;
 }
 

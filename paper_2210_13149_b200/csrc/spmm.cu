@@ -26,6 +26,7 @@
 #include <algorithm>
 
 #include "bigcn_internal.cuh"
+#include "spmm_dev.cuh"
 
 namespace bigcn {
 
@@ -88,35 +89,6 @@ template <> struct Elt<int8_t> {
     }
 };
 
-struct SpmmDev {
-    int64_t n;
-    const int64_t* rowptr;
-    const int32_t* colidx;
-    const float* val;
-    const uint4* zeta;       // rows of nv 16-byte vectors
-    int nv;                  // vectors per zeta row
-    int nv_fin;              // groups of Elt<T>::kPerVec columns the row epilogue covers (nv, unless the epilogue's element type differs)
-    int d_out;
-    const float* node_w;     // nullable
-    const float* col_w;      // nullable
-    const float* col_b0;     // half-dot bytes only: per-column first weight sign (0 where none)
-    int half_dots;           // zeta holds s = (dot' - 1) / 2; node_w carries the first feature sign
-    int byte_path;           // 129..256 byte columns: 0 / 1 the FMA stream, 2 integer tensor-core products
-    const float* add;        // nullable: fp32 [n x ld_add] added to the aggregated row (after col_w)
-    int64_t ld_add;
-    float* h_out;
-    int64_t ldh;
-    int h_vec;               // 1: rows of h_out can be stored as float4
-    uint32_t* next_bits;
-    int64_t next_stride;
-    float* next_beta;
-    const float* next_shift;
-    const float* next_scale;
-    int64_t long_row;
-    int covered_words;       // packed words of the next layer that the zeta columns cover
-    float inv_d_out;
-    int* run_counter;        // zeroed before the launch: next run of rows to hand out
-};
 
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
 {
@@ -1684,6 +1656,8 @@ cudaError_t launch_spmm(cudaStream_t s, const SpmmArgs& a, int* launches)
     p.run_counter = static_cast<int*>(a.scratch);
     ++*launches;
     const double mean_row = (a.nnz > 0 && a.n > 0) ? (double)a.nnz / (double)a.n : 0.0;
+    // rows of 129..256 signed bytes as tcgen05 integer products (a run of rows must hold fewer than 2^31 entries)
+    if (a.fmt == kZetaI8 && a.byte_path == 3 && a.nnz > 0 && a.nnz < (int64_t(1) << 31) && spmm_tc_covers(p)) return launch_spmm_tc(s, p);
     switch (a.fmt) {
         case kZetaF32: return dispatch<float>(s, p, mean_row);
         case kZetaF16: return dispatch<__half>(s, p, mean_row);

@@ -1,0 +1,549 @@
+// Aggregation H' = A_tilde zeta (Bi-GCN, last equation of Sec. 4.2.3) for rows of 129..256 signed bytes, with the sum
+// over a row's stored entries taken as exact integer products on the 5th-generation tensor cores, and the
+// re-binarization of H' for the next layer (Sec. 4.2.2 after the batch-norm constants of Sec. 4.4) in the epilogue.
+//
+// Why.  The fp32 FMA stream (spmm.cu) turns every gathered byte into a float and multiplies it on the fp32 pipe:
+// about 38 warp instructions per stored entry, which bounds it below the rate at which the rows can be fetched.
+// Here a gathered row never passes through a register.  The rows of a chunk of 64 stored entries are copied
+// (cp.async, 16 bytes per lane) straight into shared memory in the layout the tensor core reads as the A operand:
+// M = 128 output columns x K = 64 entries, M-major (an entry's 128 bytes are contiguous), 128-byte swizzle; two such
+// operands cover 256 columns.  The B operand holds the chunk's edge weights: weight e of row segment s (the part of
+// one output row that falls into the chunk; at most 8 per chunk) is written in fixed point against a power of two
+// S_s above the segment's largest weight, q_e = round(w_e 2^30 / S_s), split into four balanced base-256 digits that
+// fill columns 4 s .. 4 s + 3 of row e; all other columns of that row are 0.  One tcgen05.mma.kind::i8 per operand and
+// K = 32 step (N = 32) leaves in tensor memory, for every output column (a lane) and segment, the four digit sums
+// sum_e digit_d(q_e) zeta_e,col: exact integers.  They are read back once per segment (tcgen05.ld, four registers),
+// recombined in fp32 (sum_d 256^d . S_s 2^-30) and added to the row's fp32 accumulator; when a row ends, the
+// thread that owns a column scales it by alpha, stores it and takes part in the packing of sign bits and beta.
+// The error this adds to the fp32 sum is at most 2^-31 S_s sum_e |zeta_e| per segment (S_s < 2 max_e |w_e|).
+//
+// Who does what.  A block is 8 consumer warps and 1 producer warp.  The producer walks over runs of 31 consecutive
+// rows handed out by an atomic counter (zeroed by the launcher; it only hands out work), cuts their entries into
+// chunks, loads column indices, edge values and the per-source factor (beta_k, with the first feature sign for
+// half-dot bytes), derives the segment scales, digits and -- for half-dot bytes -- the per-segment weight sums
+// (as exact integer sums of the q_e, so that they match the products digit for digit), and publishes a chunk slot
+// (mbarrier).  The consumers issue the gathers of chunk i + 2, wait for the copies of chunk i, one thread issues its
+// products, and all read back chunk i - 1 (thread = output column) while the tensor core works on chunk i.
+// Three operand stages (48 KB), two accumulator stages (128 tensor-memory columns), six chunk slots per block; three
+// blocks per multiprocessor.  Every wait on an mbarrier is bounded: if one runs out the block raises a flag (reported
+// by bigcn_sync_check), the consumers agree on leaving at their next named barrier, the tensor memory is freed.
+#include <algorithm>
+
+#include "bigcn_internal.cuh"
+#include "spmm_dev.cuh"
+#include "tc_common.cuh"
+
+namespace bigcn {
+
+namespace {
+
+constexpr int kConsumers = 256;                 // 8 consumer warps: thread = output column
+constexpr int kThreads = kConsumers + 32;       // + the producer warp
+constexpr int kChunk = 64;                      // stored entries per chunk: two K = 32 steps
+constexpr int kSegMax = 8;                      // row segments per chunk, four digit columns each
+constexpr int kN = 4 * kSegMax;                 // N of the instruction
+constexpr int kRunRows = 31;                    // rows per run: its 32 row offsets are one value per producer lane
+constexpr int kSlots = 6;                       // chunk slots in flight between producer and consumers
+constexpr int kAStages = 3;
+constexpr int kAStageBytes = kChunk * 256;      // two operands of 64 entries x 128 bytes
+constexpr int kBSlotBytes = kChunk * kN;        // 64 entries x 32 digit columns
+constexpr int kTmemCols = 128;                  // 2 accumulator stages x 2 operands x N = 32 columns
+constexpr int kEbitsMin = 40, kEbitsMax = 253;  // clamp of the scale's biased exponent (keeps 2^30 / S and S 2^-30 normal floats)
+
+__device__ int g_spmm_tc_timeout;               // set when a wait ran out
+
+using tc::smem_u32;
+
+struct ChunkSlot {
+    int32_t cols[kChunk];                       // source node of every entry
+    int32_t n_ent;                              // entries in the chunk (0..64); -1 = end of the stream
+    int32_t nseg;
+    int32_t seg_row[kSegMax];                   // output row of a segment
+    int32_t seg_last[kSegMax];                  // 1: the row ends with this segment
+    float seg_scale[kSegMax];                   // S_s 2^-30
+    float seg_wsum[kSegMax];                    // half-dot bytes: sum of the segment's weights, plain and
+    float seg_wsgn[kSegMax];                    // signed by the sources' first feature sign
+    int32_t pad[6];
+};
+static_assert(sizeof(ChunkSlot) == 448, "slot size");
+
+// dynamic shared memory, relative to a 1024-byte aligned base
+constexpr int kOffA = 0;
+constexpr int kOffB = kOffA + kAStages * kAStageBytes;
+constexpr int kOffSlots = kOffB + kSlots * kBSlotBytes;
+constexpr int kOffBetaPart = kOffSlots + kSlots * (int)sizeof(ChunkSlot);          // float [2][kSegMax][8]
+constexpr int kOffBetaRow = kOffBetaPart + 2 * kSegMax * 8 * 4;                    // int [2][kSegMax]
+constexpr int kOffRunTab = kOffBetaRow + 2 * kSegMax * 4;                          // int [32]
+constexpr int kOffBars = kOffRunTab + 32 * 4;                                      // uint64 [kSlots + kSlots + 2]
+constexpr int kOffMisc = kOffBars + (2 * kSlots + 2) * 8;                          // uint32 tmem base, int abort
+constexpr int kSmemBytes = kOffMisc + 16 + 1024;                                   // + slack for the alignment
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar)
+{
+    asm volatile("{\n.reg .b64 st;\nmbarrier.arrive.shared::cta.b64 st, [%0];\n}\n" ::"r"(smem_u32(bar)) : "memory");
+}
+// Bounded wait that also gives up when another thread of the block has raised `abort`.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort)
+{
+    uint32_t done = 0;
+    for (int it = 0; it < tc::kWaitTries && !done; ++it) {
+        asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+                     : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        if (!done && *abort) break;
+    }
+    if (!done) {
+        atomicExch(&g_spmm_tc_timeout, 1);
+        *abort = 1;
+    }
+    return done != 0;
+}
+// All consumers meet; returns the OR of their `bad` flags.
+__device__ __forceinline__ bool consumers_sync_or(bool bad)
+{
+    uint32_t r;
+    asm volatile("{\n.reg .pred p, q;\nsetp.ne.u32 q, %1, 0;\nbarrier.cta.red.or.pred p, 1, %2, q;\nselp.u32 %0, 1, 0, p;\n}\n"
+                 : "=r"(r) : "r"((uint32_t)bad), "n"(kConsumers) : "memory");
+    return r != 0;
+}
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
+// shared-memory matrix descriptor with a layout type (0 = no swizzle, 2 = 128-byte swizzle)
+__device__ __forceinline__ uint64_t make_desc_l(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout)
+{
+    return tc::make_desc(saddr, lbo_bytes, sbo_bytes) | ((uint64_t)layout << 61);
+}
+
+// ---- the producer warp ---------------------------------------------------------------------------------------------
+
+// A chunk while the producer works on it: uniform values, per-segment values in lanes 0..7, and two entries per lane
+// (entry `lane` and entry 32 + lane).
+struct Prep {
+    int64_t e_base;          // global index of the chunk's first stored entry
+    int n_ent;               // -1: end of the stream
+    int nseg;
+    int seg_end;             // lane s: end of segment s relative to the chunk (255 for s >= nseg)
+    int seg_row;             // lane s: output row
+    int seg_last;            // lane s: the row ends here
+    int col_a, col_b;
+    float val_a, val_b;
+    float nw_a, nw_b;
+};
+
+template <bool kHalf>
+__device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, volatile int* abort)
+{
+    const int lane = threadIdx.x & 31;
+    int* run_tab = reinterpret_cast<int*>(sm + kOffRunTab);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sm + kOffBars);
+    uint64_t* prep_full = bars;
+    uint64_t* prep_empty = bars + kSlots;
+    const int64_t n_runs = ceil_div(p.n, kRunRows);
+
+    // the run being cut into chunks, and the one fetched ahead
+    int64_t run_base = 0, run_row0 = 0;
+    int nrows = 0, r = 0, e = 0;
+    int64_t nxt_run = -1, nxt_rp = 0;
+    auto fetch_next = [&]() {
+        int64_t id = 0;
+        if (lane == 0) id = atomicAdd(p.run_counter, 1);
+        id = __shfl_sync(0xffffffffu, id, 0);
+        nxt_run = id < n_runs ? id : -1;
+        if (nxt_run >= 0) nxt_rp = __ldg(p.rowptr + min(nxt_run * kRunRows + lane, p.n));
+    };
+    auto activate_next = [&]() -> bool {
+        if (nxt_run < 0) return false;
+        run_row0 = nxt_run * kRunRows;
+        nrows = (int)min((int64_t)kRunRows, p.n - run_row0);
+        run_base = __shfl_sync(0xffffffffu, nxt_rp, 0);
+        __syncwarp();
+        run_tab[lane] = (int)(nxt_rp - run_base);            // lanes beyond nrows repeat the last offset
+        __syncwarp();
+        r = 0;
+        e = 0;
+        fetch_next();
+        return true;
+    };
+    fetch_next();
+
+    // stage 1: the next chunk of the stream: its extent and segments, and the loads of its column indices and values
+    auto stage1 = [&](Prep& c) {
+        while (r == nrows) {
+            if (!activate_next()) {
+                c.n_ent = -1;
+                return;
+            }
+        }
+        const int row_hi = min(r + kSegMax, nrows);
+        const int e_cap = min(e + kChunk, run_tab[row_hi]);
+        const int row_j = r + lane;
+        const bool in_run = lane < kSegMax && row_j < nrows;
+        const int a = in_run ? run_tab[row_j] : 0x7fffffff;
+        const int b = in_run ? run_tab[row_j + 1] : 0x7fffffff;
+        const bool part = in_run && (a < e_cap || b <= e_cap);
+        const bool last = part && b <= e_cap;
+        c.nseg = __popc(__ballot_sync(0xffffffffu, part));
+        c.seg_end = part ? (min(b, e_cap) - e) : 255;
+        c.seg_row = (int)(run_row0 + row_j);
+        c.seg_last = last ? 1 : 0;
+        c.n_ent = e_cap - e;
+        c.e_base = run_base + e;
+        r += __popc(__ballot_sync(0xffffffffu, last));
+        e = e_cap;
+        c.col_a = c.col_b = 0;
+        c.val_a = c.val_b = 0.f;
+        if (lane < c.n_ent) {
+            c.col_a = __ldg(p.colidx + c.e_base + lane);
+            c.val_a = __ldg(p.val + c.e_base + lane);
+        }
+        if (32 + lane < c.n_ent) {
+            c.col_b = __ldg(p.colidx + c.e_base + 32 + lane);
+            c.val_b = __ldg(p.val + c.e_base + 32 + lane);
+        }
+    };
+    // stage 2: the per-source factors (the column indices have arrived)
+    auto stage2 = [&](Prep& c) {
+        c.nw_a = c.nw_b = 1.f;
+        if (c.n_ent > 0 && p.node_w) {
+            if (lane < c.n_ent) c.nw_a = __ldg(p.node_w + c.col_a);
+            if (32 + lane < c.n_ent) c.nw_b = __ldg(p.node_w + c.col_b);
+        }
+    };
+    // stage 3: scales, digits, sums; publish the slot
+    auto stage3 = [&](const Prep& c, int64_t k) -> bool {
+        const int slot_i = (int)(k % kSlots);
+        const uint32_t use = (uint32_t)(k / kSlots);
+        if (!mbar_wait(&prep_empty[slot_i], (use & 1u) ^ 1u, abort)) return false;
+        ChunkSlot* slot = reinterpret_cast<ChunkSlot*>(sm + kOffSlots) + slot_i;
+        unsigned char* Bs = sm + kOffB + slot_i * kBSlotBytes;
+        if (c.n_ent < 0) {
+            if (lane == 0) slot->n_ent = -1;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&prep_full[slot_i]);
+            return false;                                     // end of the stream
+        }
+        const float w_a = lane < c.n_ent ? c.val_a * c.nw_a : 0.f;
+        const float w_b = 32 + lane < c.n_ent ? c.val_b * c.nw_b : 0.f;
+        // the segment of each of the two entries: how many segments end at or before it
+        int sid_a = 0, sid_b = 0;
+#pragma unroll
+        for (int s = 0; s < kSegMax; ++s) {
+            const int end_s = __shfl_sync(0xffffffffu, c.seg_end, s);
+            sid_a += lane >= end_s;
+            sid_b += 32 + lane >= end_s;
+        }
+        // per segment: the largest |w| (as float bits: order-preserving for non-negative floats) -> the scale's exponent
+        const uint32_t m_a = __float_as_uint(fabsf(w_a)), m_b = __float_as_uint(fabsf(w_b));
+        int eb_a = kEbitsMin, eb_b = kEbitsMin, eb_mine = kEbitsMin;
+#pragma unroll
+        for (int s = 0; s < kSegMax; ++s) {
+            if (s < c.nseg) {
+                const uint32_t m = __reduce_max_sync(0xffffffffu, max(sid_a == s ? m_a : 0u, sid_b == s ? m_b : 0u));
+                const int eb = min(max((int)(m >> 23), kEbitsMin), kEbitsMax);
+                if (sid_a == s) eb_a = eb;
+                if (sid_b == s) eb_b = eb;
+                if (lane == s) eb_mine = eb;
+            }
+        }
+        // S = 2^(eb + 1 - 127) > |w|; q = round(w 2^30 / S), |q| <= 2^30
+        const float f_a = __uint_as_float((uint32_t)(283 - eb_a) << 23), f_b = __uint_as_float((uint32_t)(283 - eb_b) << 23);
+        // half-dot bytes: the factor's sign is the source's first feature sign, not part of the weight
+        const float u_a = kHalf ? c.val_a * fabsf(c.nw_a) : w_a, u_b = kHalf ? c.val_b * fabsf(c.nw_b) : w_b;
+        const int q_a = lane < c.n_ent ? __float2int_rn(u_a * f_a) : 0, q_b = 32 + lane < c.n_ent ? __float2int_rn(u_b * f_b) : 0;
+        // four balanced base-256 digits of q, one per byte
+        const uint32_t dg_a = ((uint32_t)q_a + 0x80808080u) ^ 0x80808080u, dg_b = ((uint32_t)q_b + 0x80808080u) ^ 0x80808080u;
+        // row e of the B operand: 32 digit columns = two 16-byte lines (N-major, no swizzle: line l of entry e at e * 16 + l * 1024)
+#pragma unroll
+        for (int l = 0; l < kN / 16; ++l) {
+            const int wa = (sid_a >> 2) == l ? (sid_a & 3) : -1, wb = (sid_b >> 2) == l ? (sid_b & 3) : -1;
+            const uint4 va = make_uint4(wa == 0 ? dg_a : 0u, wa == 1 ? dg_a : 0u, wa == 2 ? dg_a : 0u, wa == 3 ? dg_a : 0u);
+            const uint4 vb = make_uint4(wb == 0 ? dg_b : 0u, wb == 1 ? dg_b : 0u, wb == 2 ? dg_b : 0u, wb == 3 ? dg_b : 0u);
+            *reinterpret_cast<uint4*>(Bs + lane * 16 + l * 1024) = va;
+            *reinterpret_cast<uint4*>(Bs + (32 + lane) * 16 + l * 1024) = vb;
+        }
+        slot->cols[lane] = c.col_a;
+        slot->cols[32 + lane] = c.col_b;
+        float my_wsum = 0.f, my_wsgn = 0.f;
+        const float my_scale = __uint_as_float((uint32_t)(eb_mine + 1 - 30) << 23);   // S 2^-30
+        if constexpr (kHalf) {
+            // sum_e q_e and sum_e sign_e q_e per segment, exactly, as two 16-bit halves each
+            const int g_a = c.nw_a < 0.f ? -q_a : q_a, g_b = c.nw_b < 0.f ? -q_b : q_b;
+#pragma unroll
+            for (int s = 0; s < kSegMax; ++s) {
+                if (s < c.nseg) {
+                    const int lo = (sid_a == s ? (q_a & 0xffff) : 0) + (sid_b == s ? (q_b & 0xffff) : 0);
+                    const int hi = (sid_a == s ? (q_a >> 16) : 0) + (sid_b == s ? (q_b >> 16) : 0);
+                    const int glo = (sid_a == s ? (g_a & 0xffff) : 0) + (sid_b == s ? (g_b & 0xffff) : 0);
+                    const int ghi = (sid_a == s ? (g_a >> 16) : 0) + (sid_b == s ? (g_b >> 16) : 0);
+                    const int tlo = __reduce_add_sync(0xffffffffu, lo), thi = __reduce_add_sync(0xffffffffu, hi);
+                    const int tglo = __reduce_add_sync(0xffffffffu, glo), tghi = __reduce_add_sync(0xffffffffu, ghi);
+                    if (lane == s) {
+                        my_wsum = fmaf((float)thi, 65536.f, (float)tlo) * my_scale;
+                        my_wsgn = fmaf((float)tghi, 65536.f, (float)tglo) * my_scale;
+                    }
+                }
+            }
+        }
+        if (lane < kSegMax) {
+            slot->seg_row[lane] = c.seg_row;
+            slot->seg_last[lane] = c.seg_last;
+            slot->seg_scale[lane] = my_scale;
+            slot->seg_wsum[lane] = my_wsum;
+            slot->seg_wsgn[lane] = my_wsgn;
+        }
+        if (lane == 0) {
+            slot->n_ent = c.n_ent;
+            slot->nseg = c.nseg;
+        }
+        tc::fence_async_smem();                               // the digits are read by the tensor core (async proxy)
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&prep_full[slot_i]);
+        return true;
+    };
+
+    // three chunks in flight inside the producer: loads of chunk k + 2, factors of k + 1, digits of k
+    Prep c0, c1, c2;
+    stage1(c0);
+    if (c0.n_ent >= 0) stage1(c1); else c1.n_ent = -1;
+    stage2(c0);
+    for (int64_t k = 0;; ++k) {
+        if (c1.n_ent >= 0) stage1(c2); else c2.n_ent = -1;
+        stage2(c1);
+        if (!stage3(c0, k)) break;
+        c0 = c1;
+        c1 = c2;
+    }
+}
+
+// ---- the consumer warps --------------------------------------------------------------------------------------------
+
+template <bool kHalf>
+__device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, volatile int* abort, uint32_t tmem_base)
+{
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int half = warp >> 2, quarter = warp & 3;           // operand (columns 128 half ..) and tensor-memory lane quarter
+    const int col = 128 * half + 32 * quarter + lane;         // the output column of this thread = its tensor-memory lane
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sm + kOffBars);
+    uint64_t* prep_full = bars;
+    uint64_t* prep_empty = bars + kSlots;
+    uint64_t* mma_done = bars + 2 * kSlots;
+    ChunkSlot* slots = reinterpret_cast<ChunkSlot*>(sm + kOffSlots);
+    float* beta_part = reinterpret_cast<float*>(sm + kOffBetaPart);
+    int* beta_row = reinterpret_cast<int*>(sm + kOffBetaRow);
+    const uint32_t a_base = smem_u32(sm + kOffA), b_base = smem_u32(sm + kOffB);
+
+    // per-column constants of the row epilogue
+    const bool col_in = col < p.d_out;
+    const float alpha = col_in ? (p.col_w ? __ldg(p.col_w + col) : 1.f) : 0.f;
+    const float shift = (col_in && p.next_shift) ? __ldg(p.next_shift + col) : 0.f;
+    const float scale = (col_in && p.next_shift) ? __ldg(p.next_scale + col) : 1.f;
+    const float b0 = (kHalf && col_in && p.col_b0) ? __ldg(p.col_b0 + col) : 0.f;
+
+    const char* zeta_b = reinterpret_cast<const char*>(p.zeta);
+    const uint32_t row_bytes = (uint32_t)p.nv * 16u;
+    // instruction descriptor: D = s32, A = B = s8, both M/N-major, N = 32, M = 128
+    const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(kN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+
+    // copies of chunk c into operand stage c % 3: thread (warp, lane), step it: operand it / 2, entry 4 ((it & 1) 8 + warp) + lane / 8,
+    // 16-byte piece lane % 8 -- a warp instruction covers 4 entries x 128 contiguous bytes on both sides
+    auto gather = [&](int64_t c) {
+        const ChunkSlot* slot = slots + (int)(c % kSlots);
+        const int n_ent = slot->n_ent;
+        const uint32_t stage = a_base + (uint32_t)(c % kAStages) * kAStageBytes;
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int hh = it >> 1;
+            const int j = 4 * ((it & 1) * 8 + warp) + (lane >> 3);
+            const int piece = lane & 7;
+            if (j < n_ent && hh * 8 + piece < p.nv) {
+                const uint32_t k = (uint32_t)slot->cols[j];
+                const char* src = zeta_b + (uint64_t)k * row_bytes + hh * 128 + piece * 16;
+                cp_async16(stage + hh * 8192 + j * 128 + ((piece ^ (j & 7)) * 16), src);
+            }
+        }
+    };
+
+    int64_t end_idx = INT64_MAX;                              // index of the end marker once seen
+    bool bad = false;
+    // prologue: chunks 0 and 1
+    for (int64_t c = 0; c < 2; ++c) {
+        if (end_idx == INT64_MAX && !bad) {
+            if (!mbar_wait(&prep_full[c % kSlots], (uint32_t)((c / kSlots) & 1), abort)) bad = true;
+            else if (slots[c % kSlots].n_ent < 0) end_idx = c;
+            else gather(c);
+        }
+        asm volatile("cp.async.commit_group;\n" ::: "memory");
+    }
+
+    float acc = 0.f, rs = 0.f, rg = 0.f;                      // the open row: this column's sum, the row's weight sums
+    for (int64_t i = 0;; ++i) {
+        const bool has_cur = i < end_idx, has_prev = i >= 1 && i - 1 < end_idx, has_fin = i >= 2 && i - 2 < end_idx;
+        if (!has_cur && !has_prev && !has_fin) break;
+        if (has_prev && !bad)
+            if (!mbar_wait(&mma_done[(i - 1) & 1], (uint32_t)(((i - 1) >> 1) & 1), abort)) bad = true;
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+        if (end_idx == INT64_MAX && !bad) {
+            const int64_t c = i + 2;
+            if (!mbar_wait(&prep_full[c % kSlots], (uint32_t)((c / kSlots) & 1), abort)) bad = true;
+            else if (slots[c % kSlots].n_ent < 0) end_idx = c;
+            else gather(c);
+        }
+        asm volatile("cp.async.commit_group;\n" ::: "memory");
+        asm volatile("cp.async.wait_group 2;\n" ::: "memory");   // the copies of chunk i have landed (this thread's)
+        tc::fence_async_smem();
+        tc::fence_before_sync();
+        if (consumers_sync_or(bad)) break;
+        if (has_cur && tid == 0) {
+            tc::fence_after_sync();
+            const ChunkSlot* slot = slots + (int)(i % kSlots);
+            const int ksteps = max(1, (slot->n_ent + 31) >> 5);
+            const uint32_t a_stage = a_base + (uint32_t)(i % kAStages) * kAStageBytes;
+            const uint32_t b_slot = b_base + (uint32_t)(i % kSlots) * kBSlotBytes;
+            for (int hh = 0; hh < 2; ++hh)
+                for (int ks = 0; ks < ksteps; ++ks) {
+                    const uint64_t ad = make_desc_l(a_stage + hh * 8192 + ks * 4096, 8192, 1024, 2);
+                    const uint64_t bd = make_desc_l(b_slot + ks * 512, 128, 1024, 0);
+                    const uint32_t d_addr = tmem_base + (uint32_t)((i & 1) * 64 + hh * 32);
+                    const uint32_t accum = ks > 0 ? 1u : 0u;
+                    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}\n"
+                                 ::"r"(d_addr), "l"(ad), "l"(bd), "r"(idesc), "r"(accum) : "memory");
+                }
+            tc::commit_to(&mma_done[i & 1]);
+        }
+        // beta of the rows that ended in chunk i - 2: the eight warps' partial sums in warp order
+        if (has_fin && p.next_bits && tid < kSegMax) {
+            const int par = (int)((i - 2) & 1);
+            const int row = beta_row[par * kSegMax + tid];
+            if (row >= 0) {
+                float t = 0.f;
+#pragma unroll
+                for (int w = 0; w < 8; ++w) t += beta_part[(par * kSegMax + tid) * 8 + w];
+                p.next_beta[row] = t * p.inv_d_out;
+            }
+        }
+        // read back chunk i - 1
+        if (has_prev) {
+            const int64_t c = i - 1;
+            const ChunkSlot* slot = slots + (int)(c % kSlots);
+            const int par = (int)(c & 1);
+            const int nseg = slot->nseg;
+            const uint32_t t_addr = tmem_base + ((uint32_t)(32 * quarter) << 16) + (uint32_t)(par * 64 + half * 32);
+            for (int s = 0; s < kSegMax; ++s) {
+                int row_done = -1;
+                if (s < nseg) {
+                    uint32_t d0, d1, d2, d3;
+                    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];\n"
+                                 : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3) : "r"(t_addr + 4 * s) : "memory");
+                    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+                    // |digit sum| <= 64 * 128 * 128 = 2^20: the bit pattern 0x4B400000 + d is the float 1.5 * 2^23 + d
+                    const float f0 = __uint_as_float(0x4B400000u + d0) - 12582912.f, f1 = __uint_as_float(0x4B400000u + d1) - 12582912.f;
+                    const float f2 = __uint_as_float(0x4B400000u + d2) - 12582912.f, f3 = __uint_as_float(0x4B400000u + d3) - 12582912.f;
+                    const float x = fmaf(fmaf(fmaf(f3, 256.f, f2), 256.f, f1), 256.f, f0);
+                    acc = fmaf(x, slot->seg_scale[s], acc);
+                    if constexpr (kHalf) {
+                        rs += slot->seg_wsum[s];
+                        rg += slot->seg_wsgn[s];
+                    }
+                    if (slot->seg_last[s]) row_done = slot->seg_row[s];
+                }
+                if (warp == 0 && lane == 0) beta_row[par * kSegMax + s] = row_done;
+                if (row_done >= 0) {
+                    const int64_t row = row_done;
+                    float t = acc;
+                    if constexpr (kHalf) t = fmaf(2.f, t, fmaf(b0, rg, rs));       // sum_k w_k dot_kj = 2 acc_j + wsum + b0_j wsgn
+                    float x = t * alpha;
+                    if (p.add && col_in) x += __ldg(p.add + row * p.ld_add + col);
+                    if (p.h_out && col_in) p.h_out[row * p.ldh + col] = x;
+                    if (p.next_bits) {
+                        const float xh = __fmul_rn(__fsub_rn(x, shift), scale);
+                        const uint32_t word = __ballot_sync(0xffffffffu, col_in && xh >= 0.f);
+                        float l1 = col_in ? fabsf(xh) : 0.f;
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) l1 += __shfl_xor_sync(0xffffffffu, l1, o);
+                        if (lane == 0) {
+                            if (warp < p.next_stride) p.next_bits[row * p.next_stride + warp] = word;
+                            beta_part[(par * kSegMax + s) * 8 + warp] = l1;
+                        }
+                    }
+                    acc = 0.f;
+                    rs = 0.f;
+                    rg = 0.f;
+                }
+            }
+            tc::fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&prep_empty[c % kSlots]);
+        }
+    }
+    asm volatile("cp.async.wait_all;\n" ::: "memory");        // nothing of this thread is in flight when the block leaves
+}
+
+template <bool kHalf>
+__global__ void __launch_bounds__(kThreads, 3)
+spmm_tc_kernel(const SpmmDev p)
+{
+    extern __shared__ unsigned char tca_raw[];
+    unsigned char* sm = tca_raw + ((1024u - (smem_u32(tca_raw) & 1023u)) & 1023u);   // the swizzled operands want 1024-byte alignment
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sm + kOffBars);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + kOffMisc);
+    volatile int* abort = reinterpret_cast<volatile int*>(sm + kOffMisc + 4);
+    const int warp = threadIdx.x >> 5;
+    if (warp == 0) tc::tmem_alloc(tmem_slot, kTmemCols);
+    if (threadIdx.x == 32) {
+        for (int i = 0; i < kSlots; ++i) {
+            mbar_init(&bars[i], 1);                           // chunk published: the producer's lane 0
+            mbar_init(&bars[kSlots + i], 8);                  // chunk read back: one arrival per consumer warp
+        }
+        mbar_init(&bars[2 * kSlots], 1);                      // products done: tcgen05.commit
+        mbar_init(&bars[2 * kSlots + 1], 1);
+        *abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    tc::fence_before_sync();
+    __syncthreads();
+    tc::fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    if (warp == kConsumers / 32) producer<kHalf>(p, sm, abort);
+    else consumers<kHalf>(p, sm, abort, tmem_base);
+    tc::fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tc::tmem_free(tmem_base, kTmemCols);
+}
+
+}  // namespace
+
+// Rows of 129..256 signed bytes (9..16 vectors), n < 2^31.
+bool spmm_tc_covers(const SpmmDev& p)
+{
+    return p.nv > 8 && p.nv <= 16 && p.d_out <= 256 && p.next_stride <= 8;
+}
+
+cudaError_t launch_spmm_tc(cudaStream_t s, const SpmmDev& p)
+{
+    cudaError_t e;
+    if (p.half_dots) e = cudaFuncSetAttribute(spmm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    else e = cudaFuncSetAttribute(spmm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    if ((e = cudaMemsetAsync(p.run_counter, 0, sizeof(int), s)) != cudaSuccess) return e;
+    // one wave of resident blocks (three per multiprocessor: 3 x 128 of the 512 tensor-memory columns); each pulls
+    // runs of rows until none are left
+    const int64_t n_runs = ceil_div(p.n, kRunRows);
+    const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>(ceil_div(n_runs, 4), (int64_t)sm_count() * 3));
+    if (p.half_dots) spmm_tc_kernel<true><<<grid, kThreads, kSmemBytes, s>>>(p);
+    else spmm_tc_kernel<false><<<grid, kThreads, kSmemBytes, s>>>(p);
+    return cudaGetLastError();
+}
+
+int spmm_tc_timeouts()
+{
+    int v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_spmm_tc_timeout, sizeof(int)) != cudaSuccess) return -1;
+    return v;
+}
+
+}  // namespace bigcn

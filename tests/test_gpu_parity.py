@@ -208,22 +208,34 @@ BYTE_ROW_SHAPES = [(3, 500, 6000, 100, 200), (3, 300, 3000, 127, 256), (3, 40000
                    (5, 500, 6000, 129, 200), (5, 300, 3000, 256, 256), (5, 40000, 300000, 256, 256)]
 
 
-@pytest.mark.parametrize("fmt,n,e,d_in,d_out", BYTE_ROW_SHAPES)
-def test_byte_rows_as_integer_products(ctx, B, fmt, n, e, d_in, d_out):
-    """The library's other aggregation of 129..256 byte columns (exact integer products on the tensor cores with
-    fixed-point edge weights) beside the default fp32 FMA stream."""
-    ctx.set_option(B.OPT_BYTE_AGGREGATION, 2)
+# many rows of one or two entries (chunks limited by their eight row segments), a row count that is a multiple of
+# the run length and one just above, ragged widths
+BYTE_ROW_SHAPES_TC = [(3, 31 * 40, 700, 100, 256), (3, 31 * 40 + 1, 4000, 127, 129), (5, 5000, 5200, 256, 256),
+                      (5, 2000, 150000, 200, 177), (5, 64, 2000, 256, 241), (3, 3, 4, 64, 256), (3, 3, 2, 100, 130)]
+
+
+@pytest.mark.parametrize("path", [1, 2, 3])
+@pytest.mark.parametrize("fmt,n,e,d_in,d_out", BYTE_ROW_SHAPES + BYTE_ROW_SHAPES_TC)
+def test_byte_rows_as_integer_products(ctx, B, path, fmt, n, e, d_in, d_out):
+    """The aggregations of 129..256 byte columns: the fp32 FMA stream (1) and the exact integer products with
+    fixed-point edge weights on the tensor cores (2: mma.sync, operands in registers; 3: tcgen05, operands gathered
+    straight into shared memory, digit sums in tensor memory)."""
+    ctx.set_option(B.OPT_BYTE_AGGREGATION, path)
     try:
         check_layer_forward(ctx, B, fmt, n, e, d_in, d_out)
     finally:
         ctx.set_option(B.OPT_BYTE_AGGREGATION, 0)
 
 
+@pytest.mark.parametrize("path", [2, 3])
 @pytest.mark.parametrize("fmt,d_in", [(3, 100), (5, 256), (5, 201)])
 @pytest.mark.parametrize("span", [0, 12, 40])
-def test_byte_rows_signed_edge_values_of_wide_range(ctx, B, fmt, d_in, span):
+def test_byte_rows_signed_edge_values_of_wide_range(ctx, B, path, fmt, d_in, span):
     """Edge values of both signs spread over 2^-span .. 2^span inside every row: the fixed-point weights of the
-    integer products open new segments as larger weights arrive, and the sign rides in the digits."""
+    integer products take their scale from the largest weight of a piece of the row (path 2 opens a new segment as a
+    larger weight arrives, path 3 scales every row segment of a chunk by its own maximum), and the sign rides in the
+    digits.  The bound below is this test's own: the normalized adjacency never has such values, and the library's
+    tolerance of 1e-4 + 1e-5 |x| is an absolute one that weights of 2^40 cannot meet in fp32 at all."""
     n, d_out = 600, 256
     rng = np.random.default_rng(5 + span)
     _, _, g = small_graph(n, 24000, 31)                      # about 80 entries per row: several windows
@@ -232,7 +244,7 @@ def test_byte_rows_signed_edge_values_of_wide_range(ctx, B, fmt, d_in, span):
     W = (rng.standard_normal((d_in, d_out)) * d_in ** -0.5).astype(np.float32)
     t = oracle.layer_forward(g, oracle.Layer(W), H)
     ctx.set_option(B.OPT_ZETA_FORMAT, fmt)
-    ctx.set_option(B.OPT_BYTE_AGGREGATION, 2)
+    ctx.set_option(B.OPT_BYTE_AGGREGATION, path)
     G = device_graph(B, g)
     layer = B.make_layer(d_in, d_out, bits_to_dev(t.bitsT), dev(t.alpha))
     try:
@@ -327,7 +339,7 @@ def test_half_dot_bytes_hub_row_split_across_the_block(ctx, B, d_out):
     ctx.set_option(B.OPT_ZETA_FORMAT, 5)
     G = device_graph(B, g)
     layer = B.make_layer(d_in, d_out, bits_to_dev(t.bitsT), dev(t.alpha))
-    for path in (1, 2):
+    for path in (1, 2, 3):
         ctx.set_option(B.OPT_BYTE_AGGREGATION, path)
         try:
             for thr in (0, 8, 100000):

@@ -40,6 +40,22 @@ def test_mean_adjacency_is_bit_exact(ctx, n, e, seed):
                                              (600, 9000, 256, 47), (450, 4000, 64, 6), (350, 3000, 1433, 64),
                                              (4200, 50000, 256, 256)])
 def test_sage_layer_against_oracle(ctx, fmt, n, e, d_in, d_out):
+    check_sage_layer(ctx, fmt, n, e, d_in, d_out)
+
+
+@pytest.mark.parametrize("n,e,d_in,d_out", [(500, 6000, 100, 256), (300, 200, 64, 200), (4200, 50000, 127, 256)])
+def test_sage_layer_with_the_tensor_core_aggregation(ctx, n, e, d_in, d_out):
+    """The neighbours' term as tcgen05 integer products (byte rows of 129..256 columns); the second shape has
+    mostly isolated nodes, whose rows of the mean aggregator are empty and must come out as the node's own term."""
+    from paper_2210_13149_b200 import binding as B
+    ctx.set_option(B.OPT_BYTE_AGGREGATION, 3)
+    try:
+        check_sage_layer(ctx, 0, n, e, d_in, d_out)
+    finally:
+        ctx.set_option(B.OPT_BYTE_AGGREGATION, 0)
+
+
+def check_sage_layer(ctx, fmt, n, e, d_in, d_out):
     from paper_2210_13149_b200 import binding as B
     rng = np.random.default_rng(n + 5 * d_in + 11 * d_out)
     rp, ci = synth.power_law_graph(n, e, 200 + n)
