@@ -17,13 +17,14 @@
 // thread that owns a column scales it by alpha, stores it and takes part in the packing of sign bits and beta.
 // The error this adds to the fp32 sum is at most 2^-31 S_s sum_e |zeta_e| per segment (S_s < 2 max_e |w_e|).
 //
-// Who does what.  A block is 8 consumer warps and 1 producer warp.  The producer walks over runs of 31 consecutive
-// rows handed out by an atomic counter (zeroed by the launcher; it only hands out work), cuts their entries into
-// chunks, loads column indices, edge values and the per-source factor (beta_k, with the first feature sign for
-// half-dot bytes), derives the segment scales, digits and -- for half-dot bytes -- the per-segment weight sums
-// (as exact integer sums of the q_e, so that they match the products digit for digit), and publishes a chunk slot
-// (mbarrier).  The consumers issue the gathers of chunk i + 2, wait for the copies of chunk i, one thread issues its
-// products, and all read back chunk i - 1 (thread = output column) while the tensor core works on chunk i.
+// Who does what.  A block is 8 consumer warps and 1 producer warp.  The rows are split over the blocks once, by
+// cost (stored entries plus a constant per row).  The producer streams its block's row offsets, column indices, edge
+// values and per-source factors (beta_k, with the first feature sign for half-dot bytes) through shared-memory rings
+// with asynchronous copies issued several loop iterations ahead, cuts the entries into chunks, derives the segment
+// scales, digits and -- for half-dot bytes -- the per-segment weight sums (as exact integer sums of the q_e, so that
+// they match the products digit for digit), and publishes a chunk slot (mbarrier).  The consumers issue the gathers of
+// chunk i + 2, wait for the copies of chunk i, one thread issues its products, and all read back chunk i - 1
+// (thread = output column) while the tensor core works on chunk i.
 // Three operand stages (48 KB), two accumulator stages (128 tensor-memory columns), six chunk slots per block; three
 // blocks per multiprocessor.  Every wait on an mbarrier is bounded: if one runs out the block raises a flag (reported
 // by bigcn_sync_check), the consumers agree on leaving at their next named barrier, the tensor memory is freed.
@@ -38,11 +39,13 @@ namespace bigcn {
 namespace {
 
 constexpr int kConsumers = 256;                 // 8 consumer warps: thread = output column
-constexpr int kThreads = kConsumers + 32;       // + the producer warp
+constexpr int kThreads = kConsumers + 64;       // + the producer warp and the issuer warp
 constexpr int kChunk = 64;                      // stored entries per chunk: two K = 32 steps
 constexpr int kSegMax = 8;                      // row segments per chunk, four digit columns each
 constexpr int kN = 4 * kSegMax;                 // N of the instruction
-constexpr int kRunRows = 31;                    // rows per run: its 32 row offsets are one value per producer lane
+constexpr int kEntRing = 768;                   // producer's ring of stored entries (column, value, factor): 2 kLag + 1 blocks of 64 and slack
+constexpr int kRowRing = 128;                   // producer's ring of row offsets
+constexpr int kLag = 4;                         // producer loop iterations between issuing a copy and using its data
 constexpr int kSlots = 6;                       // chunk slots in flight between producer and consumers
 constexpr int kAStages = 3;
 constexpr int kAStageBytes = kChunk * 256;      // two operands of 64 entries x 128 bytes
@@ -73,9 +76,10 @@ constexpr int kOffB = kOffA + kAStages * kAStageBytes;
 constexpr int kOffSlots = kOffB + kSlots * kBSlotBytes;
 constexpr int kOffBetaPart = kOffSlots + kSlots * (int)sizeof(ChunkSlot);          // float [2][kSegMax][8]
 constexpr int kOffBetaRow = kOffBetaPart + 2 * kSegMax * 8 * 4;                    // int [2][kSegMax]
-constexpr int kOffRunTab = kOffBetaRow + 2 * kSegMax * 4;                          // int [32]
-constexpr int kOffBars = kOffRunTab + 32 * 4;                                      // uint64 [kSlots + kSlots + 2]
-constexpr int kOffMisc = kOffBars + (2 * kSlots + 2) * 8;                          // uint32 tmem base, int abort
+constexpr int kOffEntRing = kOffBetaRow + 2 * kSegMax * 4;                         // producer: int32 / float / float [kEntRing]
+constexpr int kOffRowRing = kOffEntRing + 3 * kEntRing * 4;                        // producer: int64 [kRowRing]
+constexpr int kOffBars = kOffRowRing + kRowRing * 8;                               // uint64: published [kSlots], read back [kSlots], products done [2], accumulators read [2], rows landed [kAStages]
+constexpr int kOffMisc = kOffBars + (2 * kSlots + 4 + kAStages) * 8;               // uint32 tmem base, int abort
 constexpr int kSmemBytes = kOffMisc + 16 + 1024;                                   // + slack for the alignment
 
 __device__ __forceinline__ void mbar_init(uint64_t* bar, int count)
@@ -93,7 +97,8 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     for (int it = 0; it < tc::kWaitTries && !done; ++it) {
         asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
                      : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-        if (!done && *abort) break;
+        if (done || *abort) break;
+        __nanosleep(32);                                      // polling must not eat the issue slots of the warps that work
     }
     if (!done) {
         atomicExch(&g_spmm_tc_timeout, 1);
@@ -121,119 +126,145 @@ __device__ __forceinline__ uint64_t make_desc_l(uint32_t saddr, uint32_t lbo_byt
 
 // ---- the producer warp ---------------------------------------------------------------------------------------------
 
-// A chunk while the producer works on it: uniform values, per-segment values in lanes 0..7, and two entries per lane
-// (entry `lane` and entry 32 + lane).
-struct Prep {
-    int64_t e_base;          // global index of the chunk's first stored entry
-    int n_ent;               // -1: end of the stream
-    int nseg;
-    int seg_end;             // lane s: end of segment s relative to the chunk (255 for s >= nseg)
-    int seg_row;             // lane s: output row
-    int seg_last;            // lane s: the row ends here
-    int col_a, col_b;
-    float val_a, val_b;
-    float nw_a, nw_b;
-};
+// The rows of the matrix are split over the blocks once, by position in a cost scale on which a row counts its stored
+// entries plus kRowCost (the row epilogue): block b takes the rows whose cost offsets fall into the b-th of gridDim.x
+// equal parts.  Returns the first row whose offset reaches `target` (32 probes per step, all lanes).
+constexpr int kRowCost = 8;
+__device__ __forceinline__ int64_t first_row_at_cost(const SpmmDev& p, int64_t target, int lane)
+{
+    int64_t lo = 0, hi = p.n;                                 // answer in [lo, hi]; cost(hi) >= target or hi == n
+    while (hi - lo > 0) {
+        const int64_t span = hi - lo;
+        const int64_t probe = lo + (span * (lane + 1)) / 33;  // lo <= probe <= hi, non-decreasing in lane, probe < hi when span >= 1
+        const bool ge = __ldg(p.rowptr + probe) + kRowCost * probe >= target;
+        const unsigned m = __ballot_sync(0xffffffffu, ge);
+        const int first = m ? __ffs(m) - 1 : 32;              // first lane whose probe is at or above the target
+        const int64_t new_hi = first < 32 ? __shfl_sync(0xffffffffu, probe, first) : hi;
+        const int64_t new_lo = first > 0 ? __shfl_sync(0xffffffffu, probe, first - 1) + 1 : lo;
+        lo = new_lo;
+        hi = new_hi;
+    }
+    return lo;
+}
 
+__device__ __forceinline__ void cp_async4(void* smem_dst, const void* gmem_src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(smem_u32(smem_dst)), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async8(void* smem_dst, const void* gmem_src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(smem_u32(smem_dst)), "l"(gmem_src) : "memory");
+}
+
+// The producer streams its block's part of the matrix -- row offsets, column indices, edge values, and the
+// per-source factors the column indices point at -- through rings in shared memory with asynchronous copies issued
+// kLag loop iterations before their data is used (the factors are a dependent fetch: their copies are issued once the
+// column indices have landed, and used kLag iterations after that).  Every iteration issues at most one block of
+// 64 entries of each kind, commits one copy group, and cuts and publishes at most one chunk.
 template <bool kHalf>
 __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, volatile int* abort)
 {
     const int lane = threadIdx.x & 31;
-    int* run_tab = reinterpret_cast<int*>(sm + kOffRunTab);
     uint64_t* bars = reinterpret_cast<uint64_t*>(sm + kOffBars);
     uint64_t* prep_full = bars;
     uint64_t* prep_empty = bars + kSlots;
-    const int64_t n_runs = ceil_div(p.n, kRunRows);
+    int32_t* col_ring = reinterpret_cast<int32_t*>(sm + kOffEntRing);
+    float* val_ring = reinterpret_cast<float*>(sm + kOffEntRing + kEntRing * 4);
+    float* nw_ring = reinterpret_cast<float*>(sm + kOffEntRing + kEntRing * 8);
+    int64_t* row_ring = reinterpret_cast<int64_t*>(sm + kOffRowRing);
 
-    // the run being cut into chunks, and the one fetched ahead
-    int64_t run_base = 0, run_row0 = 0;
-    int nrows = 0, r = 0, e = 0;
-    int64_t nxt_run = -1, nxt_rp = 0;
-    auto fetch_next = [&]() {
-        int64_t id = 0;
-        if (lane == 0) id = atomicAdd(p.run_counter, 1);
-        id = __shfl_sync(0xffffffffu, id, 0);
-        nxt_run = id < n_runs ? id : -1;
-        if (nxt_run >= 0) nxt_rp = __ldg(p.rowptr + min(nxt_run * kRunRows + lane, p.n));
-    };
-    auto activate_next = [&]() -> bool {
-        if (nxt_run < 0) return false;
-        run_row0 = nxt_run * kRunRows;
-        nrows = (int)min((int64_t)kRunRows, p.n - run_row0);
-        run_base = __shfl_sync(0xffffffffu, nxt_rp, 0);
-        __syncwarp();
-        run_tab[lane] = (int)(nxt_rp - run_base);            // lanes beyond nrows repeat the last offset
-        __syncwarp();
-        r = 0;
-        e = 0;
-        fetch_next();
-        return true;
-    };
-    fetch_next();
+    // this block's rows [R0, R1) and stored entries [E0, E0 + total)
+    const int64_t cost_all = __ldg(p.rowptr + p.n) + kRowCost * p.n;
+    const int64_t R0 = first_row_at_cost(p, (cost_all * blockIdx.x) / gridDim.x, lane);
+    const int64_t R1 = blockIdx.x + 1 == gridDim.x ? p.n : first_row_at_cost(p, (cost_all * (blockIdx.x + 1)) / gridDim.x, lane);
+    const int nrows = (int)(R1 - R0);
+    const int64_t E0 = __ldg(p.rowptr + R0);
+    const int total = (int)(__ldg(p.rowptr + R1) - E0);
 
-    // stage 1: the next chunk of the stream: its extent and segments, and the loads of its column indices and values
-    auto stage1 = [&](Prep& c) {
-        while (r == nrows) {
-            if (!activate_next()) {
-                c.n_ent = -1;
-                return;
+    int r = 0, e = 0;                                         // the cutter: next row, next entry (relative to R0, E0)
+    int ci = 0, ni = 0, ri = 0;                               // entries / rows whose copies have been issued (blocks of 64 / 16)
+    int ci_h[kLag], ni_h[kLag], ri_h[kLag];                   // the same counters after each of the last kLag iterations
+#pragma unroll
+    for (int q = 0; q < kLag; ++q) ci_h[q] = ni_h[q] = ri_h[q] = 0;
+
+    for (int64_t k = 0;;) {                                   // k: chunks published so far
+        asm volatile("cp.async.wait_group %0;\n" ::"n"(kLag - 1) : "memory");
+        __syncwarp();
+        const int ci_done = ci_h[kLag - 1], ni_done = ni_h[kLag - 1], ri_done = ri_h[kLag - 1];
+        // ---- issue: column indices and values of the next block of entries
+        if (ci < total && ci + 64 <= e + kEntRing) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int x = ci + 32 * h + lane;
+                if (x < total) {
+                    cp_async4(col_ring + (x % kEntRing), p.colidx + E0 + x);
+                    cp_async4(val_ring + (x % kEntRing), p.val + E0 + x);
+                }
             }
+            ci += 64;
         }
-        const int row_hi = min(r + kSegMax, nrows);
-        const int e_cap = min(e + kChunk, run_tab[row_hi]);
-        const int row_j = r + lane;
-        const bool in_run = lane < kSegMax && row_j < nrows;
-        const int a = in_run ? run_tab[row_j] : 0x7fffffff;
-        const int b = in_run ? run_tab[row_j + 1] : 0x7fffffff;
-        const bool part = in_run && (a < e_cap || b <= e_cap);
-        const bool last = part && b <= e_cap;
-        c.nseg = __popc(__ballot_sync(0xffffffffu, part));
-        c.seg_end = part ? (min(b, e_cap) - e) : 255;
-        c.seg_row = (int)(run_row0 + row_j);
-        c.seg_last = last ? 1 : 0;
-        c.n_ent = e_cap - e;
-        c.e_base = run_base + e;
-        r += __popc(__ballot_sync(0xffffffffu, last));
-        e = e_cap;
-        c.col_a = c.col_b = 0;
-        c.val_a = c.val_b = 0.f;
-        if (lane < c.n_ent) {
-            c.col_a = __ldg(p.colidx + c.e_base + lane);
-            c.val_a = __ldg(p.val + c.e_base + lane);
+        // ---- issue: the factors of a block whose column indices have landed
+        if (ni < ci_done) {
+            if (p.node_w) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int x = ni + 32 * h + lane;
+                    if (x < total) cp_async4(nw_ring + (x % kEntRing), p.node_w + col_ring[x % kEntRing]);
+                }
+            }
+            ni += 64;
         }
-        if (32 + lane < c.n_ent) {
-            c.col_b = __ldg(p.colidx + c.e_base + 32 + lane);
-            c.val_b = __ldg(p.val + c.e_base + 32 + lane);
+        // ---- issue: row offsets
+        if (ri <= nrows && ri + 16 <= r + kRowRing) {
+            const int j = ri + lane;
+            if (lane < 16 && j <= nrows) cp_async8(row_ring + (j % kRowRing), p.rowptr + R0 + j);
+            ri += 16;
         }
-    };
-    // stage 2: the per-source factors (the column indices have arrived)
-    auto stage2 = [&](Prep& c) {
-        c.nw_a = c.nw_b = 1.f;
-        if (c.n_ent > 0 && p.node_w) {
-            if (lane < c.n_ent) c.nw_a = __ldg(p.node_w + c.col_a);
-            if (32 + lane < c.n_ent) c.nw_b = __ldg(p.node_w + c.col_b);
-        }
-    };
-    // stage 3: scales, digits, sums; publish the slot
-    auto stage3 = [&](const Prep& c, int64_t k) -> bool {
+        asm volatile("cp.async.commit_group;\n" ::: "memory");
+#pragma unroll
+        for (int q = kLag - 1; q > 0; --q) { ci_h[q] = ci_h[q - 1]; ni_h[q] = ni_h[q - 1]; ri_h[q] = ri_h[q - 1]; }
+        ci_h[0] = ci; ni_h[0] = ni; ri_h[0] = ri;
+
+        // ---- cut the next chunk if everything it can touch has landed
+        const bool finished = r == nrows;
+        if (!finished && !(min(r + kSegMax + 1, nrows + 1) <= ri_done && min(e + kChunk, total) <= ni_done)) continue;
         const int slot_i = (int)(k % kSlots);
-        const uint32_t use = (uint32_t)(k / kSlots);
-        if (!mbar_wait(&prep_empty[slot_i], (use & 1u) ^ 1u, abort)) return false;
+        if (!mbar_wait(&prep_empty[slot_i], ((uint32_t)(k / kSlots) & 1u) ^ 1u, abort)) break;
         ChunkSlot* slot = reinterpret_cast<ChunkSlot*>(sm + kOffSlots) + slot_i;
         unsigned char* Bs = sm + kOffB + slot_i * kBSlotBytes;
-        if (c.n_ent < 0) {
+        if (finished) {                                       // end of the stream
             if (lane == 0) slot->n_ent = -1;
             __syncwarp();
             if (lane == 0) mbar_arrive(&prep_full[slot_i]);
-            return false;                                     // end of the stream
+            break;
         }
-        const float w_a = lane < c.n_ent ? c.val_a * c.nw_a : 0.f;
-        const float w_b = 32 + lane < c.n_ent ? c.val_b * c.nw_b : 0.f;
+        // segments: the rows r .. r + 7 as far as they start before the chunk's end (or are empty and sit at it)
+        const int rp_rel = (lane <= kSegMax && r + lane <= nrows) ? (int)(row_ring[(r + lane) % kRowRing] - E0) : 0x7fffffff;
+        const int row_hi = min(r + kSegMax, nrows);
+        const int e_cap = min(e + kChunk, __shfl_sync(0xffffffffu, rp_rel, row_hi - r));
+        const int a = rp_rel, b = __shfl_down_sync(0xffffffffu, rp_rel, 1);
+        const bool in_run = lane < kSegMax && r + lane < nrows;
+        const bool part = in_run && (a < e_cap || b <= e_cap);
+        const bool last = part && b <= e_cap;
+        const int nseg = __popc(__ballot_sync(0xffffffffu, part));
+        const int seg_end = part ? (min(b, e_cap) - e) : 255;
+        const int seg_row = (int)(R0 + r + lane);
+        const int n_ent = e_cap - e;
+        // the chunk's entries: two per lane
+        const bool in_a = lane < n_ent, in_b = 32 + lane < n_ent;
+        const int xa = (e + lane) % kEntRing, xb = (e + 32 + lane) % kEntRing;
+        const int col_a = in_a ? col_ring[xa] : 0, col_b = in_b ? col_ring[xb] : 0;
+        const float val_a = in_a ? val_ring[xa] : 0.f, val_b = in_b ? val_ring[xb] : 0.f;
+        const float nw_a = (in_a && p.node_w) ? nw_ring[xa] : 1.f, nw_b = (in_b && p.node_w) ? nw_ring[xb] : 1.f;
+        r += __popc(__ballot_sync(0xffffffffu, last));
+        e = e_cap;
+
+        const float w_a = in_a ? val_a * nw_a : 0.f, w_b = in_b ? val_b * nw_b : 0.f;
         // the segment of each of the two entries: how many segments end at or before it
         int sid_a = 0, sid_b = 0;
 #pragma unroll
         for (int s = 0; s < kSegMax; ++s) {
-            const int end_s = __shfl_sync(0xffffffffu, c.seg_end, s);
+            const int end_s = __shfl_sync(0xffffffffu, seg_end, s);
             sid_a += lane >= end_s;
             sid_b += 32 + lane >= end_s;
         }
@@ -242,7 +273,7 @@ __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, vo
         int eb_a = kEbitsMin, eb_b = kEbitsMin, eb_mine = kEbitsMin;
 #pragma unroll
         for (int s = 0; s < kSegMax; ++s) {
-            if (s < c.nseg) {
+            if (s < nseg) {
                 const uint32_t m = __reduce_max_sync(0xffffffffu, max(sid_a == s ? m_a : 0u, sid_b == s ? m_b : 0u));
                 const int eb = min(max((int)(m >> 23), kEbitsMin), kEbitsMax);
                 if (sid_a == s) eb_a = eb;
@@ -253,8 +284,8 @@ __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, vo
         // S = 2^(eb + 1 - 127) > |w|; q = round(w 2^30 / S), |q| <= 2^30
         const float f_a = __uint_as_float((uint32_t)(283 - eb_a) << 23), f_b = __uint_as_float((uint32_t)(283 - eb_b) << 23);
         // half-dot bytes: the factor's sign is the source's first feature sign, not part of the weight
-        const float u_a = kHalf ? c.val_a * fabsf(c.nw_a) : w_a, u_b = kHalf ? c.val_b * fabsf(c.nw_b) : w_b;
-        const int q_a = lane < c.n_ent ? __float2int_rn(u_a * f_a) : 0, q_b = 32 + lane < c.n_ent ? __float2int_rn(u_b * f_b) : 0;
+        const float u_a = kHalf ? val_a * fabsf(nw_a) : w_a, u_b = kHalf ? val_b * fabsf(nw_b) : w_b;
+        const int q_a = in_a ? __float2int_rn(u_a * f_a) : 0, q_b = in_b ? __float2int_rn(u_b * f_b) : 0;
         // four balanced base-256 digits of q, one per byte
         const uint32_t dg_a = ((uint32_t)q_a + 0x80808080u) ^ 0x80808080u, dg_b = ((uint32_t)q_b + 0x80808080u) ^ 0x80808080u;
         // row e of the B operand: 32 digit columns = two 16-byte lines (N-major, no swizzle: line l of entry e at e * 16 + l * 1024)
@@ -266,16 +297,16 @@ __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, vo
             *reinterpret_cast<uint4*>(Bs + lane * 16 + l * 1024) = va;
             *reinterpret_cast<uint4*>(Bs + (32 + lane) * 16 + l * 1024) = vb;
         }
-        slot->cols[lane] = c.col_a;
-        slot->cols[32 + lane] = c.col_b;
+        slot->cols[lane] = col_a;
+        slot->cols[32 + lane] = col_b;
         float my_wsum = 0.f, my_wsgn = 0.f;
         const float my_scale = __uint_as_float((uint32_t)(eb_mine + 1 - 30) << 23);   // S 2^-30
         if constexpr (kHalf) {
             // sum_e q_e and sum_e sign_e q_e per segment, exactly, as two 16-bit halves each
-            const int g_a = c.nw_a < 0.f ? -q_a : q_a, g_b = c.nw_b < 0.f ? -q_b : q_b;
+            const int g_a = nw_a < 0.f ? -q_a : q_a, g_b = nw_b < 0.f ? -q_b : q_b;
 #pragma unroll
             for (int s = 0; s < kSegMax; ++s) {
-                if (s < c.nseg) {
+                if (s < nseg) {
                     const int lo = (sid_a == s ? (q_a & 0xffff) : 0) + (sid_b == s ? (q_b & 0xffff) : 0);
                     const int hi = (sid_a == s ? (q_a >> 16) : 0) + (sid_b == s ? (q_b >> 16) : 0);
                     const int glo = (sid_a == s ? (g_a & 0xffff) : 0) + (sid_b == s ? (g_b & 0xffff) : 0);
@@ -290,34 +321,110 @@ __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, vo
             }
         }
         if (lane < kSegMax) {
-            slot->seg_row[lane] = c.seg_row;
-            slot->seg_last[lane] = c.seg_last;
+            slot->seg_row[lane] = seg_row;
+            slot->seg_last[lane] = last ? 1 : 0;
             slot->seg_scale[lane] = my_scale;
             slot->seg_wsum[lane] = my_wsum;
             slot->seg_wsgn[lane] = my_wsgn;
         }
         if (lane == 0) {
-            slot->n_ent = c.n_ent;
-            slot->nseg = c.nseg;
+            slot->n_ent = n_ent;
+            slot->nseg = nseg;
         }
         tc::fence_async_smem();                               // the digits are read by the tensor core (async proxy)
         __syncwarp();
         if (lane == 0) mbar_arrive(&prep_full[slot_i]);
+        ++k;
+    }
+    asm volatile("cp.async.wait_all;\n" ::: "memory");
+}
+
+// ---- the issuer warp: gathers and products ------------------------------------------------------------------------
+
+// Lane 0 polls, every lane gets the outcome.
+__device__ __forceinline__ bool wait_bcast(uint64_t* bar, uint32_t parity, volatile int* abort, int lane)
+{
+    int ok = 1;
+    if (lane == 0) ok = mbar_wait(bar, parity, abort) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
+// The copies of chunk c + 2 are issued before the products of chunk c: two chunks of rows are in flight while a
+// third is multiplied.  A lane's copies of a chunk report to the stage's mbarrier when they have landed
+// (cp.async.mbarrier.arrive), so nobody waits for them but the one thread that issues the products.
+__device__ __forceinline__ void issuer(const SpmmDev& p, unsigned char* sm, volatile int* abort, uint32_t tmem_base)
+{
+    const int lane = threadIdx.x & 31;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sm + kOffBars);
+    uint64_t* prep_full = bars;
+    uint64_t* mma_done = bars + 2 * kSlots;
+    uint64_t* tmem_empty = bars + 2 * kSlots + 2;
+    uint64_t* a_full = bars + 2 * kSlots + 4;
+    const ChunkSlot* slots = reinterpret_cast<const ChunkSlot*>(sm + kOffSlots);
+    const uint32_t a_base = smem_u32(sm + kOffA), b_base = smem_u32(sm + kOffB);
+    const char* zeta_b = reinterpret_cast<const char*>(p.zeta);
+    const uint32_t row_bytes = (uint32_t)p.nv * 16u;
+    // instruction descriptor: D = s32, A = B = s8, both M/N-major, N = 32, M = 128
+    const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(kN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+    const int sub = lane >> 3, piece = lane & 7;              // a warp instruction copies 4 entries x 128 contiguous bytes
+
+    // copies of chunk c into operand stage c % 3 (the slot has been published); false at the end marker
+    auto gather = [&](int64_t c) -> bool {
+        const ChunkSlot* slot = slots + (int)(c % kSlots);
+        const int n_ent = slot->n_ent;
+        if (n_ent < 0) return false;
+        const uint32_t stage = a_base + (uint32_t)(c % kAStages) * kAStageBytes;
+#pragma unroll 4
+        for (int g = 0; g < kChunk / 4; ++g) {
+            const int j = 4 * g + sub;
+            if (j < n_ent) {
+                const char* src = zeta_b + (uint64_t)(uint32_t)slot->cols[j] * row_bytes + piece * 16;
+                const uint32_t dst = stage + j * 128 + ((piece ^ (j & 7)) * 16);
+                if (piece < p.nv) cp_async16(dst, src);
+                if (8 + piece < p.nv) cp_async16(dst + 8192, src + 128);
+            }
+        }
+        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(smem_u32(&a_full[c % kAStages])) : "memory");
         return true;
     };
 
-    // three chunks in flight inside the producer: loads of chunk k + 2, factors of k + 1, digits of k
-    Prep c0, c1, c2;
-    stage1(c0);
-    if (c0.n_ent >= 0) stage1(c1); else c1.n_ent = -1;
-    stage2(c0);
-    for (int64_t k = 0;; ++k) {
-        if (c1.n_ent >= 0) stage1(c2); else c2.n_ent = -1;
-        stage2(c1);
-        if (!stage3(c0, k)) break;
-        c0 = c1;
-        c1 = c2;
+    int64_t end_idx = INT64_MAX;
+    for (int64_t c = 0; c < 2 && end_idx == INT64_MAX; ++c) {
+        if (!wait_bcast(&prep_full[c % kSlots], (uint32_t)((c / kSlots) & 1), abort, lane)) return;
+        if (!gather(c)) end_idx = c;
     }
+    for (int64_t c = 0; c < end_idx; ++c) {
+        if (end_idx == INT64_MAX) {
+            const int64_t g = c + 2;
+            if (!wait_bcast(&prep_full[g % kSlots], (uint32_t)((g / kSlots) & 1), abort, lane)) return;
+            // its stage was read by the products of chunk c - 1
+            if (c >= 1 && !wait_bcast(&mma_done[(c - 1) & 1], (uint32_t)(((c - 1) >> 1) & 1), abort, lane)) return;
+            if (!gather(g)) end_idx = g;
+        }
+        // products of chunk c: its rows have landed, its accumulator stage has been read back (chunk c - 2)
+        if (!wait_bcast(&a_full[c % kAStages], (uint32_t)((c / kAStages) & 1), abort, lane)) return;
+        if (c >= 2 && !wait_bcast(&tmem_empty[c & 1], (uint32_t)(((c >> 1) - 1) & 1), abort, lane)) return;
+        if (lane == 0) {
+            tc::fence_async_smem();                           // the copied rows become visible to the tensor core
+            tc::fence_after_sync();
+            const ChunkSlot* slot = slots + (int)(c % kSlots);
+            const int ksteps = max(1, (slot->n_ent + 31) >> 5);
+            const uint32_t a_stage = a_base + (uint32_t)(c % kAStages) * kAStageBytes;
+            const uint32_t b_slot = b_base + (uint32_t)(c % kSlots) * kBSlotBytes;
+            for (int hh = 0; hh < 2; ++hh)
+                for (int ks = 0; ks < ksteps; ++ks) {
+                    const uint64_t ad = make_desc_l(a_stage + hh * 8192 + ks * 4096, 8192, 1024, 2);
+                    const uint64_t bd = make_desc_l(b_slot + ks * 512, 128, 1024, 0);
+                    const uint32_t d_addr = tmem_base + (uint32_t)((c & 1) * 64 + hh * 32);
+                    const uint32_t accum = ks > 0 ? 1u : 0u;
+                    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}\n"
+                                 ::"r"(d_addr), "l"(ad), "l"(bd), "r"(idesc), "r"(accum) : "memory");
+                }
+            tc::commit_to(&mma_done[c & 1]);
+        }
+        __syncwarp();
+    }
+    asm volatile("cp.async.wait_all;\n" ::: "memory");
 }
 
 // ---- the consumer warps --------------------------------------------------------------------------------------------
@@ -332,10 +439,10 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
     uint64_t* prep_full = bars;
     uint64_t* prep_empty = bars + kSlots;
     uint64_t* mma_done = bars + 2 * kSlots;
+    uint64_t* tmem_empty = bars + 2 * kSlots + 2;
     ChunkSlot* slots = reinterpret_cast<ChunkSlot*>(sm + kOffSlots);
     float* beta_part = reinterpret_cast<float*>(sm + kOffBetaPart);
     int* beta_row = reinterpret_cast<int*>(sm + kOffBetaRow);
-    const uint32_t a_base = smem_u32(sm + kOffA), b_base = smem_u32(sm + kOffB);
 
     // per-column constants of the row epilogue
     const bool col_in = col < p.d_out;
@@ -344,80 +451,20 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
     const float scale = (col_in && p.next_shift) ? __ldg(p.next_scale + col) : 1.f;
     const float b0 = (kHalf && col_in && p.col_b0) ? __ldg(p.col_b0 + col) : 0.f;
 
-    const char* zeta_b = reinterpret_cast<const char*>(p.zeta);
-    const uint32_t row_bytes = (uint32_t)p.nv * 16u;
-    // instruction descriptor: D = s32, A = B = s8, both M/N-major, N = 32, M = 128
-    const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(kN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-
-    // copies of chunk c into operand stage c % 3: thread (warp, lane), step it: operand it / 2, entry 4 ((it & 1) 8 + warp) + lane / 8,
-    // 16-byte piece lane % 8 -- a warp instruction covers 4 entries x 128 contiguous bytes on both sides
-    auto gather = [&](int64_t c) {
-        const ChunkSlot* slot = slots + (int)(c % kSlots);
-        const int n_ent = slot->n_ent;
-        const uint32_t stage = a_base + (uint32_t)(c % kAStages) * kAStageBytes;
-#pragma unroll
-        for (int it = 0; it < 4; ++it) {
-            const int hh = it >> 1;
-            const int j = 4 * ((it & 1) * 8 + warp) + (lane >> 3);
-            const int piece = lane & 7;
-            if (j < n_ent && hh * 8 + piece < p.nv) {
-                const uint32_t k = (uint32_t)slot->cols[j];
-                const char* src = zeta_b + (uint64_t)k * row_bytes + hh * 128 + piece * 16;
-                cp_async16(stage + hh * 8192 + j * 128 + ((piece ^ (j & 7)) * 16), src);
-            }
-        }
-    };
-
-    int64_t end_idx = INT64_MAX;                              // index of the end marker once seen
-    bool bad = false;
-    // prologue: chunks 0 and 1
-    for (int64_t c = 0; c < 2; ++c) {
-        if (end_idx == INT64_MAX && !bad) {
-            if (!mbar_wait(&prep_full[c % kSlots], (uint32_t)((c / kSlots) & 1), abort)) bad = true;
-            else if (slots[c % kSlots].n_ent < 0) end_idx = c;
-            else gather(c);
-        }
-        asm volatile("cp.async.commit_group;\n" ::: "memory");
-    }
-
     float acc = 0.f, rs = 0.f, rg = 0.f;                      // the open row: this column's sum, the row's weight sums
+    bool bad = false;
     for (int64_t i = 0;; ++i) {
-        const bool has_cur = i < end_idx, has_prev = i >= 1 && i - 1 < end_idx, has_fin = i >= 2 && i - 2 < end_idx;
-        if (!has_cur && !has_prev && !has_fin) break;
-        if (has_prev && !bad)
-            if (!mbar_wait(&mma_done[(i - 1) & 1], (uint32_t)(((i - 1) >> 1) & 1), abort)) bad = true;
-        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-        if (end_idx == INT64_MAX && !bad) {
-            const int64_t c = i + 2;
-            if (!mbar_wait(&prep_full[c % kSlots], (uint32_t)((c / kSlots) & 1), abort)) bad = true;
-            else if (slots[c % kSlots].n_ent < 0) end_idx = c;
-            else gather(c);
+        // one thread polls (the chunk is published; its products are done); the others wait at the named barrier
+        if (tid == 0) {
+            if (!mbar_wait(&prep_full[i % kSlots], (uint32_t)((i / kSlots) & 1), abort)) bad = true;
+            else if (slots[i % kSlots].n_ent >= 0 && !mbar_wait(&mma_done[i & 1], (uint32_t)((i >> 1) & 1), abort)) bad = true;
         }
-        asm volatile("cp.async.commit_group;\n" ::: "memory");
-        asm volatile("cp.async.wait_group 2;\n" ::: "memory");   // the copies of chunk i have landed (this thread's)
-        tc::fence_async_smem();
         tc::fence_before_sync();
         if (consumers_sync_or(bad)) break;
-        if (has_cur && tid == 0) {
-            tc::fence_after_sync();
-            const ChunkSlot* slot = slots + (int)(i % kSlots);
-            const int ksteps = max(1, (slot->n_ent + 31) >> 5);
-            const uint32_t a_stage = a_base + (uint32_t)(i % kAStages) * kAStageBytes;
-            const uint32_t b_slot = b_base + (uint32_t)(i % kSlots) * kBSlotBytes;
-            for (int hh = 0; hh < 2; ++hh)
-                for (int ks = 0; ks < ksteps; ++ks) {
-                    const uint64_t ad = make_desc_l(a_stage + hh * 8192 + ks * 4096, 8192, 1024, 2);
-                    const uint64_t bd = make_desc_l(b_slot + ks * 512, 128, 1024, 0);
-                    const uint32_t d_addr = tmem_base + (uint32_t)((i & 1) * 64 + hh * 32);
-                    const uint32_t accum = ks > 0 ? 1u : 0u;
-                    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}\n"
-                                 ::"r"(d_addr), "l"(ad), "l"(bd), "r"(idesc), "r"(accum) : "memory");
-                }
-            tc::commit_to(&mma_done[i & 1]);
-        }
-        // beta of the rows that ended in chunk i - 2: the eight warps' partial sums in warp order
-        if (has_fin && p.next_bits && tid < kSegMax) {
-            const int par = (int)((i - 2) & 1);
+        tc::fence_after_sync();
+        // beta of the rows that ended in chunk i - 1: the eight warps' partial sums in warp order
+        if (i >= 1 && p.next_bits && tid < kSegMax) {
+            const int par = (int)((i - 1) & 1);
             const int row = beta_row[par * kSegMax + tid];
             if (row >= 0) {
                 float t = 0.f;
@@ -426,61 +473,62 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
                 p.next_beta[row] = t * p.inv_d_out;
             }
         }
-        // read back chunk i - 1
-        if (has_prev) {
-            const int64_t c = i - 1;
-            const ChunkSlot* slot = slots + (int)(c % kSlots);
-            const int par = (int)(c & 1);
-            const int nseg = slot->nseg;
-            const uint32_t t_addr = tmem_base + ((uint32_t)(32 * quarter) << 16) + (uint32_t)(par * 64 + half * 32);
-            for (int s = 0; s < kSegMax; ++s) {
-                int row_done = -1;
-                if (s < nseg) {
-                    uint32_t d0, d1, d2, d3;
-                    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];\n"
-                                 : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3) : "r"(t_addr + 4 * s) : "memory");
-                    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-                    // |digit sum| <= 64 * 128 * 128 = 2^20: the bit pattern 0x4B400000 + d is the float 1.5 * 2^23 + d
-                    const float f0 = __uint_as_float(0x4B400000u + d0) - 12582912.f, f1 = __uint_as_float(0x4B400000u + d1) - 12582912.f;
-                    const float f2 = __uint_as_float(0x4B400000u + d2) - 12582912.f, f3 = __uint_as_float(0x4B400000u + d3) - 12582912.f;
-                    const float x = fmaf(fmaf(fmaf(f3, 256.f, f2), 256.f, f1), 256.f, f0);
-                    acc = fmaf(x, slot->seg_scale[s], acc);
-                    if constexpr (kHalf) {
-                        rs += slot->seg_wsum[s];
-                        rg += slot->seg_wsgn[s];
-                    }
-                    if (slot->seg_last[s]) row_done = slot->seg_row[s];
-                }
-                if (warp == 0 && lane == 0) beta_row[par * kSegMax + s] = row_done;
-                if (row_done >= 0) {
-                    const int64_t row = row_done;
-                    float t = acc;
-                    if constexpr (kHalf) t = fmaf(2.f, t, fmaf(b0, rg, rs));       // sum_k w_k dot_kj = 2 acc_j + wsum + b0_j wsgn
-                    float x = t * alpha;
-                    if (p.add && col_in) x += __ldg(p.add + row * p.ld_add + col);
-                    if (p.h_out && col_in) p.h_out[row * p.ldh + col] = x;
-                    if (p.next_bits) {
-                        const float xh = __fmul_rn(__fsub_rn(x, shift), scale);
-                        const uint32_t word = __ballot_sync(0xffffffffu, col_in && xh >= 0.f);
-                        float l1 = col_in ? fabsf(xh) : 0.f;
+        const ChunkSlot* slot = slots + (int)(i % kSlots);
+        if (slot->n_ent < 0) break;                           // end of the stream
+        // read back chunk i: the four digit sums of every segment (16 columns at a time)
+        const int par = (int)(i & 1);
+        const int nseg = slot->nseg;
+        const uint32_t t_addr = tmem_base + ((uint32_t)(32 * quarter) << 16) + (uint32_t)(par * 64 + half * 32);
+        uint32_t d[32];
+        tc::tmem_ld16_nowait(t_addr, *reinterpret_cast<uint32_t(*)[16]>(&d[0]));
+        if (nseg > 4) tc::tmem_ld16_nowait(t_addr + 16, *reinterpret_cast<uint32_t(*)[16]>(&d[16]));
+        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
 #pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) l1 += __shfl_xor_sync(0xffffffffu, l1, o);
-                        if (lane == 0) {
-                            if (warp < p.next_stride) p.next_bits[row * p.next_stride + warp] = word;
-                            beta_part[(par * kSegMax + s) * 8 + warp] = l1;
-                        }
-                    }
-                    acc = 0.f;
-                    rs = 0.f;
-                    rg = 0.f;
+        for (int s = 0; s < kSegMax; ++s) {
+            int row_done = -1;
+            if (s < nseg) {
+                // |digit sum| <= 64 * 128 * 128 = 2^20: the bit pattern 0x4B400000 + d is the float 1.5 * 2^23 + d
+                const float f0 = __uint_as_float(0x4B400000u + d[4 * s]) - 12582912.f, f1 = __uint_as_float(0x4B400000u + d[4 * s + 1]) - 12582912.f;
+                const float f2 = __uint_as_float(0x4B400000u + d[4 * s + 2]) - 12582912.f, f3 = __uint_as_float(0x4B400000u + d[4 * s + 3]) - 12582912.f;
+                const float x = fmaf(fmaf(fmaf(f3, 256.f, f2), 256.f, f1), 256.f, f0);
+                acc = fmaf(x, slot->seg_scale[s], acc);
+                if constexpr (kHalf) {
+                    rs += slot->seg_wsum[s];
+                    rg += slot->seg_wsgn[s];
                 }
+                if (slot->seg_last[s]) row_done = slot->seg_row[s];
             }
-            tc::fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&prep_empty[c % kSlots]);
+            if (warp == 0 && lane == 0) beta_row[par * kSegMax + s] = row_done;
+            if (row_done >= 0) {
+                const int64_t row = row_done;
+                float t = acc;
+                if constexpr (kHalf) t = fmaf(2.f, t, fmaf(b0, rg, rs));       // sum_k w_k dot_kj = 2 acc_j + wsum + b0_j wsgn
+                float x = t * alpha;
+                if (p.add && col_in) x += __ldg(p.add + row * p.ld_add + col);
+                if (p.h_out && col_in) p.h_out[row * p.ldh + col] = x;
+                if (p.next_bits) {
+                    const float xh = __fmul_rn(__fsub_rn(x, shift), scale);
+                    const uint32_t word = __ballot_sync(0xffffffffu, col_in && xh >= 0.f);
+                    float l1 = col_in ? fabsf(xh) : 0.f;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) l1 += __shfl_xor_sync(0xffffffffu, l1, o);
+                    if (lane == 0) {
+                        if (warp < p.next_stride) p.next_bits[row * p.next_stride + warp] = word;
+                        beta_part[(par * kSegMax + s) * 8 + warp] = l1;
+                    }
+                }
+                acc = 0.f;
+                rs = 0.f;
+                rg = 0.f;
+            }
+        }
+        tc::fence_before_sync();
+        __syncwarp();
+        if (lane == 0) {
+            mbar_arrive(&tmem_empty[par]);
+            mbar_arrive(&prep_empty[i % kSlots]);
         }
     }
-    asm volatile("cp.async.wait_all;\n" ::: "memory");        // nothing of this thread is in flight when the block leaves
 }
 
 template <bool kHalf>
@@ -499,8 +547,11 @@ spmm_tc_kernel(const SpmmDev p)
             mbar_init(&bars[i], 1);                           // chunk published: the producer's lane 0
             mbar_init(&bars[kSlots + i], 8);                  // chunk read back: one arrival per consumer warp
         }
-        mbar_init(&bars[2 * kSlots], 1);                      // products done: tcgen05.commit
-        mbar_init(&bars[2 * kSlots + 1], 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&bars[2 * kSlots + i], 1);              // products done: tcgen05.commit
+            mbar_init(&bars[2 * kSlots + 2 + i], 8);          // accumulator stage read back: one arrival per consumer warp
+        }
+        for (int i = 0; i < kAStages; ++i) mbar_init(&bars[2 * kSlots + 4 + i], 32);   // rows landed: every lane of the issuer warp
         *abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -509,6 +560,7 @@ spmm_tc_kernel(const SpmmDev p)
     tc::fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     if (warp == kConsumers / 32) producer<kHalf>(p, sm, abort);
+    else if (warp == kConsumers / 32 + 1) issuer(p, sm, abort, tmem_base);
     else consumers<kHalf>(p, sm, abort, tmem_base);
     tc::fence_before_sync();
     __syncthreads();
@@ -529,11 +581,9 @@ cudaError_t launch_spmm_tc(cudaStream_t s, const SpmmDev& p)
     if (p.half_dots) e = cudaFuncSetAttribute(spmm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     else e = cudaFuncSetAttribute(spmm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    if ((e = cudaMemsetAsync(p.run_counter, 0, sizeof(int), s)) != cudaSuccess) return e;
-    // one wave of resident blocks (three per multiprocessor: 3 x 128 of the 512 tensor-memory columns); each pulls
-    // runs of rows until none are left
-    const int64_t n_runs = ceil_div(p.n, kRunRows);
-    const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>(ceil_div(n_runs, 4), (int64_t)sm_count() * 3));
+    // one wave of resident blocks (three per multiprocessor: 3 x 128 of the 512 tensor-memory columns); the rows are
+    // split over them by cost inside the kernel
+    const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>(ceil_div(p.n, 64), (int64_t)sm_count() * 3));
     if (p.half_dots) spmm_tc_kernel<true><<<grid, kThreads, kSmemBytes, s>>>(p);
     else spmm_tc_kernel<false><<<grid, kThreads, kSmemBytes, s>>>(p);
     return cudaGetLastError();
