@@ -17,14 +17,16 @@
 // thread that owns a column scales it by alpha, stores it and takes part in the packing of sign bits and beta.
 // The error this adds to the fp32 sum is at most 2^-31 S_s sum_e |zeta_e| per segment (S_s < 2 max_e |w_e|).
 //
-// Who does what.  A block is 8 consumer warps and 1 producer warp.  The rows are split over the blocks once, by
+// Who does what.  A block is 4 consumer warps, 1 producer warp and 1 issuer warp.  The rows are split over the blocks once, by
 // cost (stored entries plus a constant per row).  The producer streams its block's row offsets, column indices, edge
 // values and per-source factors (beta_k, with the first feature sign for half-dot bytes) through shared-memory rings
 // with asynchronous copies issued several loop iterations ahead, cuts the entries into chunks, derives the segment
 // scales, digits and -- for half-dot bytes -- the per-segment weight sums (as exact integer sums of the q_e, so that
-// they match the products digit for digit), and publishes a chunk slot (mbarrier).  The consumers issue the gathers of
-// chunk i + 2, wait for the copies of chunk i, one thread issues its products, and all read back chunk i - 1
-// (thread = output column) while the tensor core works on chunk i.
+// they match the products digit for digit), and publishes a chunk slot (mbarrier).  The consumers (a thread owns one
+// tensor-memory lane = output columns t and 128 + t) copy the rows of chunk i + 3 into the operand stage the products
+// of chunk i have released -- the copies report to the stage's mbarrier when they have landed, nobody waits for them
+// but the issuer -- and read back chunk i; the issuer's one thread issues the products of a chunk as soon as it is
+// published, its rows have landed and its accumulator stage has been read back.
 // Three operand stages (48 KB), two accumulator stages (128 tensor-memory columns), six chunk slots per block; three
 // blocks per multiprocessor.  Every wait on an mbarrier is bounded: if one runs out the block raises a flag (reported
 // by bigcn_sync_check), the consumers agree on leaving at their next named barrier, the tensor memory is freed.
@@ -38,20 +40,23 @@ namespace bigcn {
 
 namespace {
 
-constexpr int kConsumers = 256;                 // 8 consumer warps: thread = output column
+constexpr int kConsumers = 128;                 // 4 consumer warps: thread = tensor-memory lane = output columns lane and 128 + lane
 constexpr int kThreads = kConsumers + 64;       // + the producer warp and the issuer warp
 constexpr int kChunk = 64;                      // stored entries per chunk: two K = 32 steps
 constexpr int kSegMax = 8;                      // row segments per chunk, four digit columns each
 constexpr int kN = 4 * kSegMax;                 // N of the instruction
-constexpr int kEntRing = 768;                   // producer's ring of stored entries (column, value, factor): 2 kLag + 1 blocks of 64 and slack
+constexpr int kEntRing = 512;                   // producer's ring of stored entries (column, value, factor): 2 kLag + 1 blocks of 64 and slack
 constexpr int kRowRing = 128;                   // producer's ring of row offsets
-constexpr int kLag = 4;                         // producer loop iterations between issuing a copy and using its data
+constexpr int kLag = 3;                         // producer loop iterations between issuing a copy and using its data
 constexpr int kSlots = 6;                       // chunk slots in flight between producer and consumers
 constexpr int kAStages = 3;
 constexpr int kAStageBytes = kChunk * 256;      // two operands of 64 entries x 128 bytes
 constexpr int kBSlotBytes = kChunk * kN;        // 64 entries x 32 digit columns
 constexpr int kTmemCols = 128;                  // 2 accumulator stages x 2 operands x N = 32 columns
 constexpr int kEbitsMin = 40, kEbitsMax = 253;  // clamp of the scale's biased exponent (keeps 2^30 / S and S 2^-30 normal floats)
+
+constexpr int kTries = 1 << 20;                 // bound of every mbarrier wait: tries of up to kSuspendNs each
+constexpr uint32_t kSuspendNs = 1000;
 
 __device__ int g_spmm_tc_timeout;               // set when a wait ran out
 
@@ -74,7 +79,7 @@ static_assert(sizeof(ChunkSlot) == 448, "slot size");
 constexpr int kOffA = 0;
 constexpr int kOffB = kOffA + kAStages * kAStageBytes;
 constexpr int kOffSlots = kOffB + kSlots * kBSlotBytes;
-constexpr int kOffBetaPart = kOffSlots + kSlots * (int)sizeof(ChunkSlot);          // float [2][kSegMax][8]
+constexpr int kOffBetaPart = kOffSlots + kSlots * (int)sizeof(ChunkSlot);          // float [2][kSegMax][8] (one per consumer warp; 4 used)
 constexpr int kOffBetaRow = kOffBetaPart + 2 * kSegMax * 8 * 4;                    // int [2][kSegMax]
 constexpr int kOffEntRing = kOffBetaRow + 2 * kSegMax * 4;                         // producer: int32 / float / float [kEntRing]
 constexpr int kOffRowRing = kOffEntRing + 3 * kEntRing * 4;                        // producer: int64 [kRowRing]
@@ -91,14 +96,14 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar)
     asm volatile("{\n.reg .b64 st;\nmbarrier.arrive.shared::cta.b64 st, [%0];\n}\n" ::"r"(smem_u32(bar)) : "memory");
 }
 // Bounded wait that also gives up when another thread of the block has raised `abort`.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort)
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort, unsigned backoff_ns = 0)
 {
     uint32_t done = 0;
-    for (int it = 0; it < tc::kWaitTries && !done; ++it) {
-        asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
-                     : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    for (int it = 0; it < kTries && !done; ++it) {
+        asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}\n"
+                     : "=r"(done) : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendNs) : "memory");   // the thread may be parked for up to the hint
         if (done || *abort) break;
-        __nanosleep(32);                                      // polling must not eat the issue slots of the warps that work
+        if (backoff_ns) __nanosleep(backoff_ns);
     }
     if (!done) {
         atomicExch(&g_spmm_tc_timeout, 1);
@@ -229,7 +234,7 @@ __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, vo
         const bool finished = r == nrows;
         if (!finished && !(min(r + kSegMax + 1, nrows + 1) <= ri_done && min(e + kChunk, total) <= ni_done)) continue;
         const int slot_i = (int)(k % kSlots);
-        if (!mbar_wait(&prep_empty[slot_i], ((uint32_t)(k / kSlots) & 1u) ^ 1u, abort)) break;
+        if (!mbar_wait(&prep_empty[slot_i], ((uint32_t)(k / kSlots) & 1u) ^ 1u, abort, 200)) break;
         ChunkSlot* slot = reinterpret_cast<ChunkSlot*>(sm + kOffSlots) + slot_i;
         unsigned char* Bs = sm + kOffB + slot_i * kBSlotBytes;
         if (finished) {                                       // end of the stream
@@ -262,8 +267,7 @@ __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, vo
         const float w_a = in_a ? val_a * nw_a : 0.f, w_b = in_b ? val_b * nw_b : 0.f;
         // the segment of each of the two entries: how many segments end at or before it
         int sid_a = 0, sid_b = 0;
-#pragma unroll
-        for (int s = 0; s < kSegMax; ++s) {
+        for (int s = 0; s < nseg; ++s) {
             const int end_s = __shfl_sync(0xffffffffu, seg_end, s);
             sid_a += lane >= end_s;
             sid_b += 32 + lane >= end_s;
@@ -271,15 +275,12 @@ __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, vo
         // per segment: the largest |w| (as float bits: order-preserving for non-negative floats) -> the scale's exponent
         const uint32_t m_a = __float_as_uint(fabsf(w_a)), m_b = __float_as_uint(fabsf(w_b));
         int eb_a = kEbitsMin, eb_b = kEbitsMin, eb_mine = kEbitsMin;
-#pragma unroll
-        for (int s = 0; s < kSegMax; ++s) {
-            if (s < nseg) {
-                const uint32_t m = __reduce_max_sync(0xffffffffu, max(sid_a == s ? m_a : 0u, sid_b == s ? m_b : 0u));
-                const int eb = min(max((int)(m >> 23), kEbitsMin), kEbitsMax);
-                if (sid_a == s) eb_a = eb;
-                if (sid_b == s) eb_b = eb;
-                if (lane == s) eb_mine = eb;
-            }
+        for (int s = 0; s < nseg; ++s) {
+            const uint32_t m = __reduce_max_sync(0xffffffffu, max(sid_a == s ? m_a : 0u, sid_b == s ? m_b : 0u));
+            const int eb = min(max((int)(m >> 23), kEbitsMin), kEbitsMax);
+            if (sid_a == s) eb_a = eb;
+            if (sid_b == s) eb_b = eb;
+            if (lane == s) eb_mine = eb;
         }
         // S = 2^(eb + 1 - 127) > |w|; q = round(w 2^30 / S), |q| <= 2^30
         const float f_a = __uint_as_float((uint32_t)(283 - eb_a) << 23), f_b = __uint_as_float((uint32_t)(283 - eb_b) << 23);
@@ -304,19 +305,16 @@ __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, vo
         if constexpr (kHalf) {
             // sum_e q_e and sum_e sign_e q_e per segment, exactly, as two 16-bit halves each
             const int g_a = nw_a < 0.f ? -q_a : q_a, g_b = nw_b < 0.f ? -q_b : q_b;
-#pragma unroll
-            for (int s = 0; s < kSegMax; ++s) {
-                if (s < nseg) {
-                    const int lo = (sid_a == s ? (q_a & 0xffff) : 0) + (sid_b == s ? (q_b & 0xffff) : 0);
-                    const int hi = (sid_a == s ? (q_a >> 16) : 0) + (sid_b == s ? (q_b >> 16) : 0);
-                    const int glo = (sid_a == s ? (g_a & 0xffff) : 0) + (sid_b == s ? (g_b & 0xffff) : 0);
-                    const int ghi = (sid_a == s ? (g_a >> 16) : 0) + (sid_b == s ? (g_b >> 16) : 0);
-                    const int tlo = __reduce_add_sync(0xffffffffu, lo), thi = __reduce_add_sync(0xffffffffu, hi);
-                    const int tglo = __reduce_add_sync(0xffffffffu, glo), tghi = __reduce_add_sync(0xffffffffu, ghi);
-                    if (lane == s) {
-                        my_wsum = fmaf((float)thi, 65536.f, (float)tlo) * my_scale;
-                        my_wsgn = fmaf((float)tghi, 65536.f, (float)tglo) * my_scale;
-                    }
+            for (int s = 0; s < nseg; ++s) {
+                const int lo = (sid_a == s ? (q_a & 0xffff) : 0) + (sid_b == s ? (q_b & 0xffff) : 0);
+                const int hi = (sid_a == s ? (q_a >> 16) : 0) + (sid_b == s ? (q_b >> 16) : 0);
+                const int glo = (sid_a == s ? (g_a & 0xffff) : 0) + (sid_b == s ? (g_b & 0xffff) : 0);
+                const int ghi = (sid_a == s ? (g_a >> 16) : 0) + (sid_b == s ? (g_b >> 16) : 0);
+                const int tlo = __reduce_add_sync(0xffffffffu, lo), thi = __reduce_add_sync(0xffffffffu, hi);
+                const int tglo = __reduce_add_sync(0xffffffffu, glo), tghi = __reduce_add_sync(0xffffffffu, ghi);
+                if (lane == s) {
+                    my_wsum = fmaf((float)thi, 65536.f, (float)tlo) * my_scale;
+                    my_wsgn = fmaf((float)tghi, 65536.f, (float)tglo) * my_scale;
                 }
             }
         }
@@ -339,19 +337,18 @@ __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, vo
     asm volatile("cp.async.wait_all;\n" ::: "memory");
 }
 
-// ---- the issuer warp: gathers and products ------------------------------------------------------------------------
+// ---- the issuer warp: products ------------------------------------------------------------------------------------
 
 // Lane 0 polls, every lane gets the outcome.
 __device__ __forceinline__ bool wait_bcast(uint64_t* bar, uint32_t parity, volatile int* abort, int lane)
 {
     int ok = 1;
-    if (lane == 0) ok = mbar_wait(bar, parity, abort) ? 1 : 0;
+    if (lane == 0) ok = mbar_wait(bar, parity, abort, 100) ? 1 : 0;
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
-// The copies of chunk c + 2 are issued before the products of chunk c: two chunks of rows are in flight while a
-// third is multiplied.  A lane's copies of a chunk report to the stage's mbarrier when they have landed
-// (cp.async.mbarrier.arrive), so nobody waits for them but the one thread that issues the products.
+// Chunk after chunk: once the chunk is published, its rows have landed (the consumers' copies report to the stage's
+// mbarrier) and its accumulator stage has been read back (chunk c - 2), one thread issues the products.
 __device__ __forceinline__ void issuer(const SpmmDev& p, unsigned char* sm, volatile int* abort, uint32_t tmem_base)
 {
     const int lane = threadIdx.x & 31;
@@ -362,53 +359,19 @@ __device__ __forceinline__ void issuer(const SpmmDev& p, unsigned char* sm, vola
     uint64_t* a_full = bars + 2 * kSlots + 4;
     const ChunkSlot* slots = reinterpret_cast<const ChunkSlot*>(sm + kOffSlots);
     const uint32_t a_base = smem_u32(sm + kOffA), b_base = smem_u32(sm + kOffB);
-    const char* zeta_b = reinterpret_cast<const char*>(p.zeta);
-    const uint32_t row_bytes = (uint32_t)p.nv * 16u;
     // instruction descriptor: D = s32, A = B = s8, both M/N-major, N = 32, M = 128
     const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(kN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-    const int sub = lane >> 3, piece = lane & 7;              // a warp instruction copies 4 entries x 128 contiguous bytes
-
-    // copies of chunk c into operand stage c % 3 (the slot has been published); false at the end marker
-    auto gather = [&](int64_t c) -> bool {
+    for (int64_t c = 0;; ++c) {
+        if (!wait_bcast(&prep_full[c % kSlots], (uint32_t)((c / kSlots) & 1), abort, lane)) return;
         const ChunkSlot* slot = slots + (int)(c % kSlots);
         const int n_ent = slot->n_ent;
-        if (n_ent < 0) return false;
-        const uint32_t stage = a_base + (uint32_t)(c % kAStages) * kAStageBytes;
-#pragma unroll 4
-        for (int g = 0; g < kChunk / 4; ++g) {
-            const int j = 4 * g + sub;
-            if (j < n_ent) {
-                const char* src = zeta_b + (uint64_t)(uint32_t)slot->cols[j] * row_bytes + piece * 16;
-                const uint32_t dst = stage + j * 128 + ((piece ^ (j & 7)) * 16);
-                if (piece < p.nv) cp_async16(dst, src);
-                if (8 + piece < p.nv) cp_async16(dst + 8192, src + 128);
-            }
-        }
-        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(smem_u32(&a_full[c % kAStages])) : "memory");
-        return true;
-    };
-
-    int64_t end_idx = INT64_MAX;
-    for (int64_t c = 0; c < 2 && end_idx == INT64_MAX; ++c) {
-        if (!wait_bcast(&prep_full[c % kSlots], (uint32_t)((c / kSlots) & 1), abort, lane)) return;
-        if (!gather(c)) end_idx = c;
-    }
-    for (int64_t c = 0; c < end_idx; ++c) {
-        if (end_idx == INT64_MAX) {
-            const int64_t g = c + 2;
-            if (!wait_bcast(&prep_full[g % kSlots], (uint32_t)((g / kSlots) & 1), abort, lane)) return;
-            // its stage was read by the products of chunk c - 1
-            if (c >= 1 && !wait_bcast(&mma_done[(c - 1) & 1], (uint32_t)(((c - 1) >> 1) & 1), abort, lane)) return;
-            if (!gather(g)) end_idx = g;
-        }
-        // products of chunk c: its rows have landed, its accumulator stage has been read back (chunk c - 2)
+        if (n_ent < 0) return;                                // end of the stream
         if (!wait_bcast(&a_full[c % kAStages], (uint32_t)((c / kAStages) & 1), abort, lane)) return;
         if (c >= 2 && !wait_bcast(&tmem_empty[c & 1], (uint32_t)(((c >> 1) - 1) & 1), abort, lane)) return;
         if (lane == 0) {
             tc::fence_async_smem();                           // the copied rows become visible to the tensor core
             tc::fence_after_sync();
-            const ChunkSlot* slot = slots + (int)(c % kSlots);
-            const int ksteps = max(1, (slot->n_ent + 31) >> 5);
+            const int ksteps = max(1, (n_ent + 31) >> 5);
             const uint32_t a_stage = a_base + (uint32_t)(c % kAStages) * kAStageBytes;
             const uint32_t b_slot = b_base + (uint32_t)(c % kSlots) * kBSlotBytes;
             for (int hh = 0; hh < 2; ++hh)
@@ -424,100 +387,154 @@ __device__ __forceinline__ void issuer(const SpmmDev& p, unsigned char* sm, vola
         }
         __syncwarp();
     }
-    asm volatile("cp.async.wait_all;\n" ::: "memory");
 }
 
 // ---- the consumer warps --------------------------------------------------------------------------------------------
 
+// One segment's four digit sums -> sum_e q_e zeta_e: the two low and the two high digits are combined as integers
+// (|digit sum| <= 64 * 128 * 128 = 2^20, so each pair fits 32 bits), then two conversions and one FMA.
+__device__ __forceinline__ float digits_to_float(uint32_t d0, uint32_t d1, uint32_t d2, uint32_t d3)
+{
+    const int lo = (int)d0 + ((int)d1 << 8), hi = (int)d2 + ((int)d3 << 8);
+    return fmaf((float)hi, 65536.f, (float)lo);
+}
+
 template <bool kHalf>
 __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, volatile int* abort, uint32_t tmem_base)
 {
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int half = warp >> 2, quarter = warp & 3;           // operand (columns 128 half ..) and tensor-memory lane quarter
-    const int col = 128 * half + 32 * quarter + lane;         // the output column of this thread = its tensor-memory lane
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;      // warp = tensor-memory lane quarter
     uint64_t* bars = reinterpret_cast<uint64_t*>(sm + kOffBars);
     uint64_t* prep_full = bars;
     uint64_t* prep_empty = bars + kSlots;
     uint64_t* mma_done = bars + 2 * kSlots;
     uint64_t* tmem_empty = bars + 2 * kSlots + 2;
+    uint64_t* a_full = bars + 2 * kSlots + 4;
     ChunkSlot* slots = reinterpret_cast<ChunkSlot*>(sm + kOffSlots);
     float* beta_part = reinterpret_cast<float*>(sm + kOffBetaPart);
     int* beta_row = reinterpret_cast<int*>(sm + kOffBetaRow);
+    const uint32_t a_base = smem_u32(sm + kOffA);
 
-    // per-column constants of the row epilogue
-    const bool col_in = col < p.d_out;
-    const float alpha = col_in ? (p.col_w ? __ldg(p.col_w + col) : 1.f) : 0.f;
-    const float shift = (col_in && p.next_shift) ? __ldg(p.next_shift + col) : 0.f;
-    const float scale = (col_in && p.next_shift) ? __ldg(p.next_scale + col) : 1.f;
-    const float b0 = (kHalf && col_in && p.col_b0) ? __ldg(p.col_b0 + col) : 0.f;
+    // per-column constants of the row epilogue: this thread owns columns tid (operand 0) and 128 + tid (operand 1)
+    float alpha[2], shift[2], scale[2], b0[2];
+    bool col_in[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int col = 128 * h + tid;
+        col_in[h] = col < p.d_out;
+        alpha[h] = col_in[h] ? (p.col_w ? __ldg(p.col_w + col) : 1.f) : 0.f;
+        shift[h] = (col_in[h] && p.next_shift) ? __ldg(p.next_shift + col) : 0.f;
+        scale[h] = (col_in[h] && p.next_shift) ? __ldg(p.next_scale + col) : 1.f;
+        b0[h] = (kHalf && col_in[h] && p.col_b0) ? __ldg(p.col_b0 + col) : 0.f;
+    }
 
-    float acc = 0.f, rs = 0.f, rg = 0.f;                      // the open row: this column's sum, the row's weight sums
+    const char* zeta_b = reinterpret_cast<const char*>(p.zeta);
+    const uint32_t row_bytes = (uint32_t)p.nv * 16u;
+    const int sub = lane >> 3, piece = lane & 7;              // a warp instruction copies 4 entries x 128 contiguous bytes
+    // copies of chunk c into operand stage c % 3: warp w takes the entries 16 w .. 16 w + 15, both operands; they
+    // report to the stage's mbarrier when they have landed
+    auto gather = [&](int64_t c) {
+        const ChunkSlot* slot = slots + (int)(c % kSlots);
+        const int n_ent = slot->n_ent;
+        const uint32_t stage = a_base + (uint32_t)(c % kAStages) * kAStageBytes;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const int j = 16 * warp + 4 * g + sub;
+            if (j < n_ent) {
+                const char* src = zeta_b + (uint64_t)(uint32_t)slot->cols[j] * row_bytes + piece * 16;
+                const uint32_t dst = stage + j * 128 + ((piece ^ (j & 7)) * 16);
+                if (piece < p.nv) cp_async16(dst, src);
+                if (8 + piece < p.nv) cp_async16(dst + 8192, src + 128);
+            }
+        }
+        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(smem_u32(&a_full[c % kAStages])) : "memory");
+    };
+
+    int64_t end_idx = INT64_MAX;                              // index of the end marker once seen
     bool bad = false;
-    for (int64_t i = 0;; ++i) {
-        // one thread polls (the chunk is published; its products are done); the others wait at the named barrier
+    // prologue: the rows of chunks 0, 1 and 2 (only one thread polls; the others wait at the named barrier)
+    for (int64_t c = 0; c < kAStages && end_idx == INT64_MAX && !bad; ++c) {
+        if (tid == 0 && !mbar_wait(&prep_full[c % kSlots], (uint32_t)((c / kSlots) & 1), abort)) bad = true;
+        bad = consumers_sync_or(bad);
+        if (!bad) {
+            if (slots[c % kSlots].n_ent < 0) end_idx = c;
+            else gather(c);
+        }
+    }
+
+    float acc[2] = {0.f, 0.f};                                // the open row: this thread's two column sums
+    float rs = 0.f, rg = 0.f;                                 // and the row's weight sums (half-dot bytes)
+    for (int64_t i = 0; !bad; ++i) {
+        const bool has_cur = i < end_idx, need_next = end_idx == INT64_MAX;
         if (tid == 0) {
-            if (!mbar_wait(&prep_full[i % kSlots], (uint32_t)((i / kSlots) & 1), abort)) bad = true;
-            else if (slots[i % kSlots].n_ent >= 0 && !mbar_wait(&mma_done[i & 1], (uint32_t)((i >> 1) & 1), abort)) bad = true;
+            if (has_cur && !mbar_wait(&mma_done[i & 1], (uint32_t)((i >> 1) & 1), abort)) bad = true;
+            if (!bad && need_next && !mbar_wait(&prep_full[(i + kAStages) % kSlots], (uint32_t)(((i + kAStages) / kSlots) & 1), abort)) bad = true;
         }
         tc::fence_before_sync();
         if (consumers_sync_or(bad)) break;
         tc::fence_after_sync();
-        // beta of the rows that ended in chunk i - 1: the eight warps' partial sums in warp order
+        // beta of the rows that ended in chunk i - 1: the four warps' partial sums in warp order
         if (i >= 1 && p.next_bits && tid < kSegMax) {
             const int par = (int)((i - 1) & 1);
             const int row = beta_row[par * kSegMax + tid];
             if (row >= 0) {
-                float t = 0.f;
-#pragma unroll
-                for (int w = 0; w < 8; ++w) t += beta_part[(par * kSegMax + tid) * 8 + w];
-                p.next_beta[row] = t * p.inv_d_out;
+                const float* bp = beta_part + (par * kSegMax + tid) * 8;
+                p.next_beta[row] = (((bp[0] + bp[1]) + bp[2]) + bp[3]) * p.inv_d_out;
             }
         }
+        if (!has_cur) break;
+        // the rows of chunk i + 3 go into the stage the products of chunk i have just released
+        if (need_next) {
+            if (slots[(i + kAStages) % kSlots].n_ent < 0) end_idx = i + kAStages;
+            else gather(i + kAStages);
+        }
+        // read back chunk i: the four digit sums of every segment, both operands
         const ChunkSlot* slot = slots + (int)(i % kSlots);
-        if (slot->n_ent < 0) break;                           // end of the stream
-        // read back chunk i: the four digit sums of every segment (16 columns at a time)
         const int par = (int)(i & 1);
         const int nseg = slot->nseg;
-        const uint32_t t_addr = tmem_base + ((uint32_t)(32 * quarter) << 16) + (uint32_t)(par * 64 + half * 32);
-        uint32_t d[32];
-        tc::tmem_ld16_nowait(t_addr, *reinterpret_cast<uint32_t(*)[16]>(&d[0]));
-        if (nseg > 4) tc::tmem_ld16_nowait(t_addr + 16, *reinterpret_cast<uint32_t(*)[16]>(&d[16]));
-        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-#pragma unroll
-        for (int s = 0; s < kSegMax; ++s) {
+        const uint32_t t_addr = tmem_base + ((uint32_t)(32 * warp) << 16) + (uint32_t)(par * 64);
+        for (int s = 0; s < kSegMax; ++s) {                    // a run-time loop: small code, the same for every segment
             int row_done = -1;
-            if (s < nseg) {
-                // |digit sum| <= 64 * 128 * 128 = 2^20: the bit pattern 0x4B400000 + d is the float 1.5 * 2^23 + d
-                const float f0 = __uint_as_float(0x4B400000u + d[4 * s]) - 12582912.f, f1 = __uint_as_float(0x4B400000u + d[4 * s + 1]) - 12582912.f;
-                const float f2 = __uint_as_float(0x4B400000u + d[4 * s + 2]) - 12582912.f, f3 = __uint_as_float(0x4B400000u + d[4 * s + 3]) - 12582912.f;
-                const float x = fmaf(fmaf(fmaf(f3, 256.f, f2), 256.f, f1), 256.f, f0);
-                acc = fmaf(x, slot->seg_scale[s], acc);
+            if (s < nseg) {                                   // uniform over the consumers
+                uint32_t a0, a1, a2, a3, c0, c1, c2, c3;
+                asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];\n"
+                             : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(t_addr + 4 * s) : "memory");
+                asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];\n"
+                             : "=r"(c0), "=r"(c1), "=r"(c2), "=r"(c3) : "r"(t_addr + 32 + 4 * s) : "memory");
+                asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+                const float sc = slot->seg_scale[s];
+                acc[0] = fmaf(digits_to_float(a0, a1, a2, a3), sc, acc[0]);
+                acc[1] = fmaf(digits_to_float(c0, c1, c2, c3), sc, acc[1]);
                 if constexpr (kHalf) {
                     rs += slot->seg_wsum[s];
                     rg += slot->seg_wsgn[s];
                 }
                 if (slot->seg_last[s]) row_done = slot->seg_row[s];
             }
-            if (warp == 0 && lane == 0) beta_row[par * kSegMax + s] = row_done;
+            if (tid == 0) beta_row[par * kSegMax + s] = row_done;
             if (row_done >= 0) {
                 const int64_t row = row_done;
-                float t = acc;
-                if constexpr (kHalf) t = fmaf(2.f, t, fmaf(b0, rg, rs));       // sum_k w_k dot_kj = 2 acc_j + wsum + b0_j wsgn
-                float x = t * alpha;
-                if (p.add && col_in) x += __ldg(p.add + row * p.ld_add + col);
-                if (p.h_out && col_in) p.h_out[row * p.ldh + col] = x;
+                float l1 = 0.f;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    float t = acc[h];
+                    if constexpr (kHalf) t = fmaf(2.f, t, fmaf(b0[h], rg, rs));   // sum_k w_k dot_kj = 2 acc_j + wsum + b0_j wsgn
+                    float x = t * alpha[h];
+                    const int col = 128 * h + tid;
+                    if (p.add && col_in[h]) x += __ldg(p.add + row * p.ld_add + col);
+                    if (p.h_out && col_in[h]) p.h_out[row * p.ldh + col] = x;
+                    if (p.next_bits) {
+                        const float xh = __fmul_rn(__fsub_rn(x, shift[h]), scale[h]);
+                        const uint32_t word = __ballot_sync(0xffffffffu, col_in[h] && xh >= 0.f);
+                        if (lane == 0 && 4 * h + warp < p.next_stride) p.next_bits[row * p.next_stride + 4 * h + warp] = word;
+                        l1 += col_in[h] ? fabsf(xh) : 0.f;
+                    }
+                    acc[h] = 0.f;
+                }
                 if (p.next_bits) {
-                    const float xh = __fmul_rn(__fsub_rn(x, shift), scale);
-                    const uint32_t word = __ballot_sync(0xffffffffu, col_in && xh >= 0.f);
-                    float l1 = col_in ? fabsf(xh) : 0.f;
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) l1 += __shfl_xor_sync(0xffffffffu, l1, o);
-                    if (lane == 0) {
-                        if (warp < p.next_stride) p.next_bits[row * p.next_stride + warp] = word;
-                        beta_part[(par * kSegMax + s) * 8 + warp] = l1;
-                    }
+                    if (lane == 0) beta_part[(par * kSegMax + s) * 8 + warp] = l1;
                 }
-                acc = 0.f;
                 rs = 0.f;
                 rg = 0.f;
             }
@@ -529,6 +546,7 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
             mbar_arrive(&prep_empty[i % kSlots]);
         }
     }
+    asm volatile("cp.async.wait_all;\n" ::: "memory");        // nothing of this thread is in flight when the block leaves
 }
 
 template <bool kHalf>
@@ -545,13 +563,13 @@ spmm_tc_kernel(const SpmmDev p)
     if (threadIdx.x == 32) {
         for (int i = 0; i < kSlots; ++i) {
             mbar_init(&bars[i], 1);                           // chunk published: the producer's lane 0
-            mbar_init(&bars[kSlots + i], 8);                  // chunk read back: one arrival per consumer warp
+            mbar_init(&bars[kSlots + i], kConsumers / 32);   // chunk read back: one arrival per consumer warp
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&bars[2 * kSlots + i], 1);              // products done: tcgen05.commit
-            mbar_init(&bars[2 * kSlots + 2 + i], 8);          // accumulator stage read back: one arrival per consumer warp
+            mbar_init(&bars[2 * kSlots + 2 + i], kConsumers / 32);   // accumulator stage read back: one arrival per consumer warp
         }
-        for (int i = 0; i < kAStages; ++i) mbar_init(&bars[2 * kSlots + 4 + i], 32);   // rows landed: every lane of the issuer warp
+        for (int i = 0; i < kAStages; ++i) mbar_init(&bars[2 * kSlots + 4 + i], kConsumers);   // rows landed: every consumer thread's copies
         *abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
