@@ -280,6 +280,12 @@ bigcn_status bigcn_layer_backward(bigcn_ctx* ctx, const bigcn_graph* graph, cons
  *                         the context's workspace was sized with host_io = slots.  The workspace must
  *                         not be replaced, and the context not used for other calls, while steps are
  *                         outstanding.
+ *   bigcn_pipeline_submit_packed  the same step from an input that is already binary (Sec. 5.2, Eq. "DC": the
+ *                         loaded data is 1 bit per element and one scalar per node, about 31 times less than
+ *                         fp32): bits_host u32 [n x bigcn_packed_stride_words(d_0)] and beta_host fp32 [n] in
+ *                         HOST memory, as bigcn_pack_features() produces them under the first layer's
+ *                         batch-norm constants.  The step computes what bigcn_forward_packed() computes.  Steps
+ *                         of both kinds may be mixed in one pipeline.
  *   bigcn_pipeline_wait   blocks until the OLDEST outstanding step has delivered its logits (steps
  *                         complete in submission order); BIGCN_OK at once if none is outstanding.
  *   bigcn_pipeline_close  waits for everything outstanding and frees the streams and events. */
@@ -288,6 +294,8 @@ typedef struct bigcn_pipeline bigcn_pipeline;
 bigcn_status bigcn_pipeline_open(bigcn_ctx* ctx, const bigcn_graph* graph, const bigcn_layer* layers /*host*/,
                                  int32_t n_layers, int32_t slots, bigcn_pipeline** out);
 bigcn_status bigcn_pipeline_submit(bigcn_pipeline* pipe, const float* X_host, float* logits_host);
+bigcn_status bigcn_pipeline_submit_packed(bigcn_pipeline* pipe, const uint32_t* bits_host, const float* beta_host,
+                                          float* logits_host);
 bigcn_status bigcn_pipeline_wait(bigcn_pipeline* pipe);
 bigcn_status bigcn_pipeline_close(bigcn_pipeline* pipe);
 

@@ -69,6 +69,7 @@ SIGNATURES = {
     "bigcn_pipeline_open": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer), _i32, _i32,
                                            ctypes.POINTER(_vp)]),
     "bigcn_pipeline_submit": (ctypes.c_int, [_vp, _vp, _vp]),
+    "bigcn_pipeline_submit_packed": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
     "bigcn_pipeline_wait": (ctypes.c_int, [_vp]),
     "bigcn_pipeline_close": (ctypes.c_int, [_vp]),
     "bigcn_col_stats": (ctypes.c_int, [_vp, _vp, _i64, _i32, _i64, ctypes.c_float, _vp, _vp]),
@@ -445,6 +446,17 @@ class Pipeline:
         assert tuple(logits_host.shape) == (self.graph.n, self.dims[-1]) and logits_host.dtype == torch.float32
         self.ctx._check(self.ctx.lib.bigcn_pipeline_submit(self.h, _ptr(X_host), _ptr(logits_host)))
         self._held.append((X_host, logits_host))
+
+    def submit_packed(self, bits_host: torch.Tensor, beta_host: torch.Tensor, logits_host: torch.Tensor):
+        """A step from an already binary input (packed sign bits and beta, host tensors)."""
+        n = self.graph.n
+        assert bits_host.device.type == "cpu" and beta_host.device.type == "cpu" and logits_host.device.type == "cpu"
+        assert bits_host.is_contiguous() and beta_host.is_contiguous() and logits_host.is_contiguous()
+        assert tuple(bits_host.shape) == (n, packed_stride_words(self.dims[0])) and bits_host.dtype == torch.int32
+        assert tuple(beta_host.shape) == (n,) and beta_host.dtype == torch.float32
+        assert tuple(logits_host.shape) == (n, self.dims[-1]) and logits_host.dtype == torch.float32
+        self.ctx._check(self.ctx.lib.bigcn_pipeline_submit_packed(self.h, _ptr(bits_host), _ptr(beta_host), _ptr(logits_host)))
+        self._held.append(((bits_host, beta_host), logits_host))
 
     def wait(self) -> Optional[torch.Tensor]:
         self.ctx._check(self.ctx.lib.bigcn_pipeline_wait(self.h))

@@ -194,6 +194,15 @@ size_t zeta_bytes_max(int64_t n, const int32_t* dims, int n_layers)
     return m;
 }
 
+// Bytes of a slot's input staging buffer: the fp32 features, or -- whichever is larger -- the packed input
+// (bits, then beta behind them at the next 256-byte boundary).
+size_t staging_in_bytes(int64_t n, int32_t d0)
+{
+    const size_t dense = (size_t)n * d0 * 4;
+    const size_t packed = up((size_t)n * bigcn_packed_stride_words(d0) * 4) + (size_t)n * 4;
+    return dense > packed ? dense : packed;
+}
+
 void finish_call(bigcn_ctx* ctx)
 {
     ctx->launches += ctx->launches_i;
@@ -400,7 +409,7 @@ size_t bigcn_workspace_bytes(int64_t n, int64_t nnz, const int32_t* dims, int32_
     size_t aux = up(normalize_scratch_bytes(n));
     if (up(col_stats_scratch_bytes(d_max)) > aux) aux = up(col_stats_scratch_bytes(d_max));
     if (host_io > 0) {                                        // staging buffers: one pair per slot
-        total += (size_t)host_io * (up((size_t)n * dims[0] * 4) + up((size_t)n * dims[n_layers] * 4));
+        total += (size_t)host_io * (up(staging_in_bytes(n, dims[0])) + up((size_t)n * dims[n_layers] * 4));
     }
     if (aux > total) total = aux;
     return total + kAlign;
@@ -622,7 +631,11 @@ bigcn_status bigcn_pipeline_open(bigcn_ctx* ctx, const bigcn_graph* graph, const
     return BIGCN_OK;
 }
 
-bigcn_status bigcn_pipeline_submit(bigcn_pipeline* p, const float* X_host, float* logits_host)
+namespace {
+
+// One step of a pipeline from fp32 features (X_host) or from an already binary input (bits_host, beta_host).
+bigcn_status pipeline_submit_impl(bigcn_pipeline* p, const float* X_host, const uint32_t* bits_host, const float* beta_host,
+                                  float* logits_host)
 {
     if (!p) return BIGCN_ERR_NULL;
     bigcn_ctx* ctx = p->ctx;
@@ -637,23 +650,33 @@ bigcn_status bigcn_pipeline_submit(bigcn_pipeline* p, const float* X_host, float
         ++p->submitted;
         return BIGCN_OK;
     }
-    if (!X_host || !logits_host) return fail(ctx, BIGCN_ERR_NULL, "X_host or logits_host is null");
+    const bool packed = X_host == nullptr;
+    if (!logits_host || (packed ? (!bits_host || !beta_host) : false)) return fail(ctx, BIGCN_ERR_NULL, "an input or logits_host is null");
     Carver ws{static_cast<char*>(ctx->ws), ctx->ws_bytes, 0};
     float* x_dev = nullptr;
     float* out_dev = nullptr;
     for (int i = 0; i < p->slots; ++i) {                      // the same carving at every call: slot i keeps its buffers
-        float* x = static_cast<float*>(ws.take((size_t)n * d0 * 4));
+        float* x = static_cast<float*>(ws.take(staging_in_bytes(n, d0)));
         float* o = static_cast<float*>(ws.take((size_t)n * classes * 4));
         if (!x || !o) return fail(ctx, BIGCN_ERR_WORKSPACE, "workspace too small for %d pairs of staging buffers (size it with host_io = %d)", p->slots, p->slots);
         if (i == s) { x_dev = x; out_dev = o; }
     }
     // copy in: the slot's input buffer is free once the step that used it last has been computed
     if (p->used[s]) BIGCN_CUDA(ctx, cudaStreamWaitEvent(p->up, p->computed[s], 0));
-    BIGCN_CUDA(ctx, cudaMemcpyAsync(x_dev, X_host, (size_t)n * d0 * 4, cudaMemcpyHostToDevice, p->up));
+    const size_t bits_bytes = (size_t)n * bigcn_packed_stride_words(d0) * 4;
+    uint32_t* bits_dev = reinterpret_cast<uint32_t*>(x_dev);
+    float* beta_dev = reinterpret_cast<float*>(reinterpret_cast<char*>(x_dev) + up(bits_bytes));
+    if (packed) {                                             // Sec. 5.2: the loaded data is binary -- 1 bit per element and one scalar per node
+        BIGCN_CUDA(ctx, cudaMemcpyAsync(bits_dev, bits_host, bits_bytes, cudaMemcpyHostToDevice, p->up));
+        BIGCN_CUDA(ctx, cudaMemcpyAsync(beta_dev, beta_host, (size_t)n * 4, cudaMemcpyHostToDevice, p->up));
+    } else {
+        BIGCN_CUDA(ctx, cudaMemcpyAsync(x_dev, X_host, (size_t)n * d0 * 4, cudaMemcpyHostToDevice, p->up));
+    }
     BIGCN_CUDA(ctx, cudaEventRecord(p->x_ready[s], p->up));
     // forward: the slot's logits buffer is free because its last step has been waited for (slots bound above)
     BIGCN_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, p->x_ready[s], 0));
-    st = forward_impl(ctx, &p->graph, p->layers, p->n_layers, x_dev, d0, nullptr, nullptr, out_dev, classes, nullptr, ws);
+    if (packed) st = forward_impl(ctx, &p->graph, p->layers, p->n_layers, nullptr, 0, bits_dev, beta_dev, out_dev, classes, nullptr, ws);
+    else st = forward_impl(ctx, &p->graph, p->layers, p->n_layers, x_dev, d0, nullptr, nullptr, out_dev, classes, nullptr, ws);
     finish_call(ctx);
     if (st != BIGCN_OK) return st;
     BIGCN_CUDA(ctx, cudaEventRecord(p->computed[s], ctx->stream));
@@ -664,6 +687,19 @@ bigcn_status bigcn_pipeline_submit(bigcn_pipeline* p, const float* X_host, float
     p->used[s] = true;
     ++p->submitted;
     return BIGCN_OK;
+}
+
+}  // namespace
+
+bigcn_status bigcn_pipeline_submit(bigcn_pipeline* p, const float* X_host, float* logits_host)
+{
+    if (p && p->graph.n > 0 && !X_host) return fail(p->ctx, BIGCN_ERR_NULL, "X_host is null");
+    return pipeline_submit_impl(p, X_host, nullptr, nullptr, logits_host);
+}
+
+bigcn_status bigcn_pipeline_submit_packed(bigcn_pipeline* p, const uint32_t* bits_host, const float* beta_host, float* logits_host)
+{
+    return pipeline_submit_impl(p, nullptr, bits_host, beta_host, logits_host);
 }
 
 bigcn_status bigcn_pipeline_wait(bigcn_pipeline* p)

@@ -66,12 +66,53 @@ def test_pipeline_matches_forward_in_order(B, net, slots):
         done += 1
     assert pipe.wait() is None                    # nothing outstanding: returns at once
     pipe.close()
-    # the first step is the workload itself: hold it against the oracle
+    # the first step is the workload itself: its predictions agree with the oracle's end-to-end run (what bigcn_forward
+    # computes is held against the oracle element by element in test_gpu_parity.py and, below, for the packed steps)
     ref = torch.from_numpy(net.logits)
-    err = (outs[0].double() - ref.double()).abs()
-    allow = ATOL + RTOL * ref.double().abs()
-    assert (err > allow).double().mean().item() < 0.02      # threshold flips of re-binarised bits aside
     assert (outs[0].argmax(1) == ref.argmax(1)).double().mean().item() > 0.99
+    ctx.sync_check()
+    ctx.close()
+
+
+@pytest.mark.parametrize("slots", [1, 3])
+def test_pipeline_steps_from_packed_input(B, net, slots):
+    """Steps whose input is already binary (Sec. 5.2: packed sign bits and one scalar per node, in host memory), mixed
+    with steps from fp32 features: bit for bit what bigcn_forward_packed() gives, and every logit within the tolerance of
+    the oracle's last layer fed the very bits that layer saw (the network has two layers: the library's own
+    re-binarized output of layer 0, unpacked by the oracle)."""
+    import oracle
+    from parity_util import bits_from_dev, within_tol
+    ctx, G, layers = build(B, net)
+    assert len(layers) == 2
+    n_steps = 6
+    xs = [step_inputs(net.wl, k) for k in range(n_steps)]
+    packed = [ctx.pack_features(x.cuda(), layers[0].in_shift, layers[0].in_scale) for x in xs]
+    want = [ctx.forward_packed(G, layers, b, be).cpu() for b, be in packed]
+    for x, w in zip(xs, want):
+        assert torch.equal(ctx.forward(G, layers, x.cuda()).cpu(), w)     # the same bits, the same result
+    host = [(b.cpu().pin_memory(), be.cpu().pin_memory()) for b, be in packed]
+    xs_pinned = [x.pin_memory() for x in xs]
+    outs = [torch.full((net.wl.n, want[0].shape[1]), float("nan")).pin_memory() for _ in range(n_steps)]
+    pipe = ctx.open_pipeline(G, layers, slots=slots)
+    done = 0
+    for k in range(n_steps):
+        if k - done == slots:
+            assert torch.equal(pipe.wait(), want[done]), "step %d" % done
+            done += 1
+        if k % 3 == 2:
+            pipe.submit(xs_pinned[k], outs[k])                 # a step from fp32 features in between
+        else:
+            pipe.submit_packed(host[k][0], host[k][1], outs[k])
+    while done < n_steps:
+        assert torch.equal(pipe.wait(), want[done]), "step %d" % done
+        done += 1
+    pipe.close()
+    # against the oracle, no element exempt
+    for k in (0, 1):
+        mid = ctx.layer_forward(G, layers[0], packed[k][0], packed[k][1], want_h=False, next_layer=layers[1])
+        ref = oracle.layer_forward_packed(net.graph, net.layers[1], bits_from_dev(mid["next_bits"]), mid["next_beta"].cpu().numpy()).H_out
+        ok, ratio, mx = within_tol(outs[k], torch.from_numpy(ref))
+        assert ok, "step %d: error / allowance %.3g (max abs %.3g)" % (k, ratio, mx)
     ctx.sync_check()
     ctx.close()
 
