@@ -132,6 +132,19 @@ typedef struct {
     const float* dinv;
 } bigcn_graph;
 
+/* Set-up from a raw list of node pairs (Sec. 3.1: an undirected graph; A_hat = A + I).  src, dst int32 [m] in DEVICE
+ * memory, node ids in [0, n): any order, either or both directions, repeats and self pairs allowed.  Every pair
+ * (u, v) with u != v contributes the entries (u, v) and (v, u); repeats and self pairs are dropped (the one self-loop
+ * per node is added by bigcn_normalize_adjacency()).  Output: the pattern of A as the CSR that
+ * bigcn_normalize_adjacency() takes -- rowptr_A int64 [n + 1], colidx_A int32 with room for 2 m entries (ascending
+ * and unique within a row, symmetric, no diagonal); *nnz_out = entries written.  m < 2^30.
+ * Needs bigcn_edges_workspace_bytes(n, m) of workspace (about 32 m bytes: two buffers of 64-bit sort keys and the
+ * scratch of the CUDA toolkit's device-wide sort and de-duplication, which this set-up step uses).  SYNCHRONOUS.
+ * BIGCN_ERR_GRAPH if a node id lies outside [0, n). */
+size_t bigcn_edges_workspace_bytes(int64_t n, int64_t m);
+bigcn_status bigcn_adjacency_from_edges(bigcn_ctx* ctx, int64_t n, int64_t m, const int32_t* src, const int32_t* dst,
+                                        int64_t* rowptr_A, int32_t* colidx_A, int64_t* nnz_out /*host*/);
+
 /* Set-up step, once per graph (Sec. 3.1, Eq. 1).  Input: CSR of the adjacency A of an undirected
  * graph: symmetric pattern, columns ascending and unique within a row; diagonal entries in the
  * input are ignored and exactly one self-loop per node is added (A_hat = A + I).

@@ -56,6 +56,8 @@ SIGNATURES = {
     "bigcn_set_workspace": (ctypes.c_int, [_vp, _vp, _sz]),
     "bigcn_normalize_adjacency": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp,
                                                  ctypes.POINTER(_i64)]),
+    "bigcn_edges_workspace_bytes": (_sz, [_i64, _i64]),
+    "bigcn_adjacency_from_edges": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp, _vp, ctypes.POINTER(_i64)]),
     "bigcn_pack_features": (ctypes.c_int, [_vp, _vp, _i64, _i32, _i64, _vp, _vp, _vp, _i64, _vp]),
     "bigcn_pack_weights": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i64, _vp, _i64, _vp]),
     "bigcn_layer_forward": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer),
@@ -260,6 +262,18 @@ class BiGCN:
                                                        ctypes.byref(nnz)))
         k = int(nnz.value)
         return make_graph(rowptr, colidx[:k], val[:k], dinv)
+
+    def adjacency_from_edges(self, n: int, src: torch.Tensor, dst: torch.Tensor):
+        """Canonical CSR pattern of A (rowptr int64, colidx int32) from a raw list of node pairs (device int32)."""
+        m = src.numel()
+        assert src.dtype == torch.int32 and dst.dtype == torch.int32 and dst.numel() == m
+        self.ensure_workspace(int(self.lib.bigcn_edges_workspace_bytes(n, m)))
+        rowptr = self._empty(n + 1, torch.int64)
+        colidx = self._empty(max(2 * m, 1), torch.int32)
+        nnz = _i64(0)
+        self._check(self.lib.bigcn_adjacency_from_edges(self.h, n, m, _ptr(src), _ptr(dst), _ptr(rowptr), _ptr(colidx),
+                                                        ctypes.byref(nnz)))
+        return rowptr, colidx[:int(nnz.value)]
 
     def pack_features(self, H: torch.Tensor, shift: Optional[torch.Tensor] = None,
                       scale: Optional[torch.Tensor] = None, stride_words: Optional[int] = None):

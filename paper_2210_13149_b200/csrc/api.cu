@@ -461,6 +461,35 @@ bigcn_status bigcn_normalize_adjacency(bigcn_ctx* ctx, int64_t n, int64_t nnz_in
     return BIGCN_OK;
 }
 
+size_t bigcn_edges_workspace_bytes(int64_t n, int64_t m)
+{
+    if (n < 0 || m < 0 || m >= (int64_t(1) << 30)) return 0;
+    return edges_scratch_bytes(m) + kAlign;
+}
+
+bigcn_status bigcn_adjacency_from_edges(bigcn_ctx* ctx, int64_t n, int64_t m, const int32_t* src, const int32_t* dst,
+                                        int64_t* rowptr_A, int32_t* colidx_A, int64_t* nnz_out)
+{
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    if (n < 0 || n >= (int64_t(1) << 31) || m < 0 || m >= (int64_t(1) << 30)) return fail(ctx, BIGCN_ERR_SHAPE, "n=%lld m=%lld out of range", (long long)n, (long long)m);
+    if (!nnz_out || !rowptr_A) return fail(ctx, BIGCN_ERR_NULL, "nnz_out or rowptr_A is null");
+    *nnz_out = 0;
+    if (m > 0 && (!src || !dst || !colidx_A)) return fail(ctx, BIGCN_ERR_NULL, "src, dst or colidx_A is null");
+    if (m > 0 && (!ctx->ws || ctx->ws_bytes < edges_scratch_bytes(m))) return fail(ctx, BIGCN_ERR_WORKSPACE, "needs %zu bytes of workspace (bigcn_edges_workspace_bytes)", edges_scratch_bytes(m));
+    cudaError_t e = launch_adjacency_from_edges(ctx->stream, n, m, src, dst, rowptr_A, colidx_A, ctx->ws, ctx->d_flag, &ctx->launches_i);
+    finish_call(ctx);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "adjacency_from_edges");
+    int flag = 0;
+    int64_t total = 0;
+    BIGCN_CUDA(ctx, cudaMemcpyAsync(&flag, ctx->d_flag, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+    BIGCN_CUDA(ctx, cudaMemcpyAsync(&total, rowptr_A + n, sizeof(int64_t), cudaMemcpyDeviceToHost, ctx->stream));
+    BIGCN_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (flag) return fail(ctx, BIGCN_ERR_GRAPH, "edge list rejected: a node id lies outside [0, n)");
+    *nnz_out = total;
+    return BIGCN_OK;
+}
+
 bigcn_status bigcn_pack_features(bigcn_ctx* ctx, const float* H, int64_t n, int32_t d, int64_t ld,
                                  const float* col_shift, const float* col_scale,
                                  uint32_t* bits_out, int64_t stride_words, float* beta_out)

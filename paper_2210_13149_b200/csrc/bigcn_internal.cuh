@@ -81,6 +81,11 @@ cudaError_t launch_normalize_adjacency(cudaStream_t s, int64_t n, int64_t nnz_in
                                        void* scratch, int* d_flag, int* launches, bool mean = false);
 size_t normalize_scratch_bytes(int64_t n);
 
+// Canonical CSR pattern of A from a raw list of node pairs (edges.cu).
+cudaError_t launch_adjacency_from_edges(cudaStream_t s, int64_t n, int64_t m, const int32_t* src, const int32_t* dst,
+                                        int64_t* rowptr, int32_t* colidx, void* scratch, int* flag, int* launches);
+size_t edges_scratch_bytes(int64_t m);
+
 cudaError_t launch_col_stats(cudaStream_t s, const float* H, int64_t n, int d, int64_t ld, float eps,
                              float* shift, float* scale, void* scratch, int* launches);
 size_t col_stats_scratch_bytes(int d);

@@ -52,6 +52,46 @@ def test_normalize_adjacency_is_bit_exact(ctx, n, e, seed):
     assert np.array_equal(got.val.cpu().numpy(), g.val)
 
 
+@pytest.mark.parametrize("n,m,seed", [(1, 0, 1), (5, 0, 2), (2, 7, 3), (60, 500, 4), (3000, 40000, 5), (200000, 1500000, 6)])
+def test_adjacency_from_a_raw_edge_list(ctx, B, n, m, seed):
+    """The set-up from node pairs as a data set lists them -- one direction or both, repeated, some joining a node to
+    itself, many nodes isolated -- followed by the normalisation: structure and values bit for bit what the oracle
+    builds from the same list (Sec. 3.1; the oracle symmetrises, de-duplicates and drops self pairs itself)."""
+    rng = np.random.default_rng(seed)
+    hi = max(n // 2, 1)                                              # the upper half of the ids stays isolated
+    src = rng.integers(0, hi, m).astype(np.int32)
+    dst = rng.integers(0, hi, m).astype(np.int32)
+    if m > 10:
+        src[: m // 5], dst[: m // 5] = dst[m // 5: 2 * (m // 5)].copy(), src[m // 5: 2 * (m // 5)].copy()   # reversed copies
+        src[-(m // 10):] = src[: m // 10]                            # exact repeats
+        dst[-(m // 10):] = dst[: m // 10]
+    g = oracle.normalize_adjacency(n, src, dst)
+    rp, ci = ctx.adjacency_from_edges(n, dev(src), dev(dst))
+    # the pattern of A: the oracle's A_hat without its diagonal
+    keep = g.colidx != np.repeat(np.arange(n), np.diff(g.rowptr))
+    assert np.array_equal(ci.cpu().numpy(), g.colidx[keep])
+    assert np.array_equal(rp.cpu().numpy(), g.rowptr - np.arange(n + 1))
+    got = ctx.normalize_adjacency(rp, ci)
+    assert got.nnz == g.nnz
+    assert np.array_equal(got.rowptr.cpu().numpy(), g.rowptr)
+    assert np.array_equal(got.colidx.cpu().numpy(), g.colidx)
+    assert np.array_equal(got.val.cpu().numpy(), g.val)
+    assert np.array_equal(got.dinv.cpu().numpy(), g.dinv)
+
+
+def test_adjacency_from_edges_rejects_ids_out_of_range(ctx, B):
+    src = dev(np.array([0, 1, 5], np.int32))
+    dst = dev(np.array([1, 2, 0], np.int32))
+    with pytest.raises(B.BigcnError) as e:
+        ctx.adjacency_from_edges(5, src, dst)                        # node 5 of 5
+    assert e.value.status == 4                                       # BIGCN_ERR_GRAPH
+    with pytest.raises(B.BigcnError) as e:
+        ctx.adjacency_from_edges(5, dev(np.array([-1], np.int32)), dev(np.array([0], np.int32)))
+    assert e.value.status == 4
+    rp, ci = ctx.adjacency_from_edges(6, src, dst)                   # fine with one more node
+    assert rp.cpu().tolist() == [0, 2, 4, 5, 5, 5, 6] and ci.cpu().tolist() == [1, 5, 0, 2, 1, 0]
+
+
 def test_normalize_adjacency_drops_input_diagonal(ctx):
     # path 0-1-2 with self-loops already present on 0 and 2
     rp = torch.tensor([0, 2, 4, 6], dtype=torch.int64)
