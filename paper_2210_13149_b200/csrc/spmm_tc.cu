@@ -23,12 +23,13 @@
 // with asynchronous copies issued several loop iterations ahead, cuts the entries into chunks, derives the segment
 // scales, digits and -- for half-dot bytes -- the per-segment weight sums (as exact integer sums of the q_e, so that
 // they match the products digit for digit), and publishes a chunk slot (mbarrier).  The consumers (a thread owns one
-// tensor-memory lane = output columns t and 128 + t) copy the rows of chunk i + 3 into the operand stage the products
+// tensor-memory lane = output columns t and 128 + t) copy the rows of chunk i + 2 into the operand stage the products
 // of chunk i have released -- the copies report to the stage's mbarrier when they have landed, nobody waits for them
 // but the issuer -- and read back chunk i; the issuer's one thread issues the products of a chunk as soon as it is
 // published, its rows have landed and its accumulator stage has been read back.
-// Three operand stages (48 KB), two accumulator stages (128 tensor-memory columns), six chunk slots per block; three
-// blocks per multiprocessor.  Every wait on an mbarrier is bounded: if one runs out the block raises a flag (reported
+// Two operand stages (32 KB), two accumulator stages (128 tensor-memory columns), four chunk slots per block; four
+// blocks per multiprocessor (what bounds the kernel is the latency of each block's chain of dependent steps per chunk,
+// so the number of blocks that fit counts for more than the depth of one block's pipeline).  Every wait on an mbarrier is bounded: if one runs out the block raises a flag (reported
 // by bigcn_sync_check), the consumers agree on leaving at their next named barrier, the tensor memory is freed.
 #include <algorithm>
 
@@ -48,8 +49,8 @@ constexpr int kN = 4 * kSegMax;                 // N of the instruction
 constexpr int kEntRing = 512;                   // producer's ring of stored entries (column, value, factor): 2 kLag + 1 blocks of 64 and slack
 constexpr int kRowRing = 128;                   // producer's ring of row offsets
 constexpr int kLag = 3;                         // producer loop iterations between issuing a copy and using its data
-constexpr int kSlots = 6;                       // chunk slots in flight between producer and consumers
-constexpr int kAStages = 3;
+constexpr int kSlots = 4;                       // chunk slots in flight between producer and consumers
+constexpr int kAStages = 2;
 constexpr int kAStageBytes = kChunk * 256;      // two operands of 64 entries x 128 bytes
 constexpr int kBSlotBytes = kChunk * kN;        // 64 entries x 32 digit columns
 constexpr int kTmemCols = 128;                  // 2 accumulator stages x 2 operands x N = 32 columns
@@ -430,7 +431,7 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
     const char* zeta_b = reinterpret_cast<const char*>(p.zeta);
     const uint32_t row_bytes = (uint32_t)p.nv * 16u;
     const int sub = lane >> 3, piece = lane & 7;              // a warp instruction copies 4 entries x 128 contiguous bytes
-    // copies of chunk c into operand stage c % 3: warp w takes the entries 16 w .. 16 w + 15, both operands; they
+    // copies of chunk c into operand stage c % kAStages: warp w takes the entries 16 w .. 16 w + 15, both operands; they
     // report to the stage's mbarrier when they have landed
     auto gather = [&](int64_t c) {
         const ChunkSlot* slot = slots + (int)(c % kSlots);
@@ -451,7 +452,7 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
 
     int64_t end_idx = INT64_MAX;                              // index of the end marker once seen
     bool bad = false;
-    // prologue: the rows of chunks 0, 1 and 2 (only one thread polls; the others wait at the named barrier)
+    // prologue: the rows of the first kAStages chunks (only one thread polls; the others wait at the named barrier)
     for (int64_t c = 0; c < kAStages && end_idx == INT64_MAX && !bad; ++c) {
         if (tid == 0 && !mbar_wait(&prep_full[c % kSlots], (uint32_t)((c / kSlots) & 1), abort)) bad = true;
         bad = consumers_sync_or(bad);
@@ -482,7 +483,7 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
             }
         }
         if (!has_cur) break;
-        // the rows of chunk i + 3 go into the stage the products of chunk i have just released
+        // the rows of chunk i + kAStages go into the stage the products of chunk i have just released
         if (need_next) {
             if (slots[(i + kAStages) % kSlots].n_ent < 0) end_idx = i + kAStages;
             else gather(i + kAStages);
@@ -550,7 +551,7 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
 }
 
 template <bool kHalf>
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kThreads, 4)
 spmm_tc_kernel(const SpmmDev p)
 {
     extern __shared__ unsigned char tca_raw[];
@@ -599,9 +600,9 @@ cudaError_t launch_spmm_tc(cudaStream_t s, const SpmmDev& p)
     if (p.half_dots) e = cudaFuncSetAttribute(spmm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     else e = cudaFuncSetAttribute(spmm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    // one wave of resident blocks (three per multiprocessor: 3 x 128 of the 512 tensor-memory columns); the rows are
+    // one wave of resident blocks (four per multiprocessor: 4 x 128 = all 512 tensor-memory columns); the rows are
     // split over them by cost inside the kernel
-    const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>(ceil_div(p.n, 64), (int64_t)sm_count() * 3));
+    const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>(ceil_div(p.n, 64), (int64_t)sm_count() * 4));
     if (p.half_dots) spmm_tc_kernel<true><<<grid, kThreads, kSmemBytes, s>>>(p);
     else spmm_tc_kernel<false><<<grid, kThreads, kSmemBytes, s>>>(p);
     return cudaGetLastError();
