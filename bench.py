@@ -537,6 +537,10 @@ def run_ours(args):
         per16 = 16 // elt
         ldz = (dims[l + 1] + per16 - 1) // per16 * per16
         last = (l == L - 1)
+        # a last layer of 33..60 byte columns on the tensor-core contraction: 64-byte rows that carry the node factor
+        on_tc = dims[l] <= 256 and dims[l + 1] <= 256 and (f == binding.ZETA_I8H or n * dims[l + 1] >= (1 << 20))
+        if last and elt == 1 and 32 < dims[l + 1] <= 60 and on_tc:
+            ldz = 64
         out_bytes = n * dims[l + 1] * 4.0 if last else n * (binding.packed_stride_words(dims[l + 1]) * 4.0 + 4.0)
         lower, upper, expected = spmm_bytes_model(n, nnz, ldz * elt, out_bytes, deg_cum)
         t = spmm_ms[l] * 1e-3

@@ -138,8 +138,12 @@ bigcn_status run_layer(bigcn_ctx* ctx, const bigcn_graph* g, const bigcn_layer* 
 {
     const int fmt = pick_format(ctx, layer->d_in, layer->d_out, g->n, /*allow_half=*/true, /*fp32_only=*/next == nullptr && h_out != nullptr);
     const bool half = fmt == kZetaI8H;
-    const int64_t ldz = zeta_ld(layer->d_out, fmt);
     const int64_t stride_in = bigcn_packed_stride_words(layer->d_in);
+    // a last layer of 33..60 byte columns on the tensor-core contraction: 64-byte rows that carry the node factor in
+    // their last four bytes, so that the aggregation's lane-per-entry stream needs two lookups per entry, not four or five
+    const bool row_tail = (fmt == kZetaI8 || half) && next == nullptr && h_out != nullptr && layer->d_out > 32 && layer->d_out <= 60 &&
+                          bitgemm_takes_tc(fmt, half ? 2 : ctx->contraction, g->n, layer->d_in, layer->d_out, stride_in, stride_in);
+    const int64_t ldz = row_tail ? 64 : zeta_ld(layer->d_out, fmt);
     // half-dot bytes: the node factors carrying the first feature sign and the columns' first weight signs follow
     // the byte rows inside the zeta scratch (which is sized for fp32 rows, four times as much)
     float* nws = nullptr;
@@ -151,7 +155,7 @@ bigcn_status run_layer(bigcn_ctx* ctx, const bigcn_graph* g, const bigcn_layer* 
     }
     cudaError_t e = launch_bitgemm(ctx->stream, in_bits, stride_in, layer->w_bitsT, stride_in, g->n,
                                    layer->d_in, layer->d_out, in_beta, layer->alpha, fmt, zeta, ldz,
-                                   dbg_dot, dbg_zeta, &ctx->launches_i, half ? 2 : ctx->contraction, nws, col_b0);
+                                   dbg_dot, dbg_zeta, &ctx->launches_i, half ? 2 : ctx->contraction, nws, col_b0, row_tail ? 1 : 0);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "bit-GEMM launch");
     if (ev_mid) BIGCN_CUDA(ctx, cudaEventRecord(ev_mid, ctx->stream));
     SpmmArgs a;
@@ -168,6 +172,7 @@ bigcn_status run_layer(bigcn_ctx* ctx, const bigcn_graph* g, const bigcn_layer* 
     a.col_w = layer->alpha;
     a.half_dots = half;
     a.byte_path = ctx->byte_path;
+    a.row_tail = row_tail;
     a.col_b0 = col_b0;
     a.h_out = h_out;
     a.ldh = ldh;

@@ -42,7 +42,10 @@ cudaError_t launch_bitgemm(cudaStream_t s, const uint32_t* A, int64_t stride_a,
                            const uint32_t* BT, int64_t stride_b, int64_t n, int d_in, int d_out,
                            const float* beta, const float* alpha, int fmt, void* zeta, int64_t ldz,
                            int32_t* dbg_dot, float* dbg_zeta, int* launches, int path = 0 /* 0 auto, 1 bit-count pipe, 2 tensor cores wherever covered */,
-                           float* nws = nullptr /* kZetaI8H: [n] beta_i times the first sign */, float* col_b0 = nullptr /* kZetaI8H: [d_out] */);
+                           float* nws = nullptr /* kZetaI8H: [n] beta_i times the first sign */, float* col_b0 = nullptr /* kZetaI8H: [d_out] */,
+                           int row_tail = 0 /* byte formats on the tensor-core path, ldz = 64: the row's node factor in its last four bytes */);
+// Whether launch_bitgemm will take the tensor-core path for these arguments.
+bool bitgemm_takes_tc(int fmt, int path, int64_t n, int d_in, int d_out, int64_t stride_a, int64_t stride_b);
 
 struct SpmmArgs {
     int64_t n;
@@ -59,6 +62,7 @@ struct SpmmArgs {
     const float* col_b0 = nullptr;   // half-dot bytes (kZetaI8H): per-column first weight sign (0 when d_in is odd)
     bool half_dots = false;          // zeta holds s = (dot' - 1) / 2 and node_w carries the first feature sign
     int byte_path = 0;               // rows of 129..256 bytes: 0 auto (the fp32 FMA stream), 1 the fp32 FMA stream, 2 integer tensor-core products
+    bool row_tail = false;           // byte rows of 64 bytes whose last four bytes hold the source's node factor (see bitgemm_tc.cu)
     const float* add = nullptr;   // optional fp32 [n x ld_add] added to every aggregated row (Bi-GraphSAGE self term)
     int64_t ld_add = 0;
     float* h_out;            // nullable
@@ -97,7 +101,7 @@ size_t popc_peak_scratch_bytes();
 bool bitgemm_tc_covers(int d_in, int d_out, int64_t stride_a, int64_t stride_b);
 cudaError_t launch_bitgemm_tc(cudaStream_t s, const uint32_t* A, int64_t stride_a, const uint32_t* BT, int64_t stride_b,
                               int64_t n, int d_in, int d_out, const float* beta, const float* alpha, int fmt, void* zeta,
-                              int64_t ldz, int32_t* dbg_dot, float* dbg_zeta, float* nws = nullptr, float* col_b0 = nullptr);
+                              int64_t ldz, int32_t* dbg_dot, float* dbg_zeta, float* nws = nullptr, float* col_b0 = nullptr, int row_tail = 0);
 int bitgemm_tc_timeouts();
 
 // Binning entropy estimate (entropy.cu): scratch = 2 * d uint32.

@@ -167,23 +167,30 @@ cudaError_t launch_tn(cudaStream_t s, const uint32_t* A, int64_t stride_a, const
 
 }  // namespace
 
+bool bitgemm_takes_tc(int fmt, int path, int64_t n, int d_in, int d_out, int64_t stride_a, int64_t stride_b)
+{
+    if (!bitgemm_tc_covers(d_in, d_out, stride_a, stride_b)) return false;
+    if (fmt == kZetaI8H) return true;
+    return path != 1 && (path == 2 || n * (int64_t)d_out >= (int64_t(1) << 20));
+}
+
 cudaError_t launch_bitgemm(cudaStream_t s, const uint32_t* A, int64_t stride_a,
                            const uint32_t* BT, int64_t stride_b, int64_t n, int d_in, int d_out,
                            const float* beta, const float* alpha, int fmt, void* zeta, int64_t ldz,
-                           int32_t* dbg_dot, float* dbg_zeta, int* launches, int path, float* nws, float* col_b0)
+                           int32_t* dbg_dot, float* dbg_zeta, int* launches, int path, float* nws, float* col_b0, int row_tail)
 {
     if (n == 0) return cudaSuccess;
     if (fmt == kZetaI8H) {                                 // half-dot bytes exist on the tensor-core path only
         if (!bitgemm_tc_covers(d_in, d_out, stride_a, stride_b)) return cudaErrorInvalidValue;
         ++*launches;
-        return launch_bitgemm_tc(s, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, fmt, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0);
+        return launch_bitgemm_tc(s, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, fmt, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0, row_tail);
     }
     // the int8 tensor-core path: for covered shapes, by default from a million outputs on (below that the two
     // paths are level and the bit-count kernel has less fixed cost)
     const bool big = n * (int64_t)d_out >= (int64_t(1) << 20);
     if (path != 1 && (path == 2 || big) && bitgemm_tc_covers(d_in, d_out, stride_a, stride_b)) {
         ++*launches;
-        return launch_bitgemm_tc(s, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, fmt, zeta, ldz, dbg_dot, dbg_zeta);
+        return launch_bitgemm_tc(s, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, fmt, zeta, ldz, dbg_dot, dbg_zeta, nullptr, nullptr, row_tail);
     }
     const int kw = (d_in + 31) / 32;
     const int ldb = kw | 1;

@@ -139,8 +139,11 @@ __global__ void __launch_bounds__(kTcThreads, 2)
 bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32_t* __restrict__ BT, int64_t stride_b,
                   int64_t n, int d_in, int d_out, const float* __restrict__ beta, const float* __restrict__ alpha,
                   void* __restrict__ zeta, int64_t ldz, int32_t* __restrict__ dbg_dot, float* __restrict__ dbg_zeta,
-                  float* __restrict__ nws, float* __restrict__ col_b0)
+                  float* __restrict__ nws, float* __restrict__ col_b0, int row_tail)
 {
+    // row_tail (byte formats, N = 64, d_out <= 60): a row of zeta is 64 bytes and its last four bytes hold the row's
+    // node factor as a float (beta_i, with the first feature sign for half-dot bytes), so that the aggregation of a
+    // last layer fetches an entry's dots and its factor with one pair of 32-byte loads
     using Out = TcOut<FMT>;
     constexpr int kElt = Out::kElt;                         // bytes per stored element = 16-byte pieces per chunk of 16 columns
     extern __shared__ __align__(128) unsigned char tc_smem[];
@@ -244,13 +247,15 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
         const int64_t row0 = tile_row0(i) + lane_base;
         const int64_t row = row0 + lane;
         const bool row_in = row < n;
-        const float be = (row_in && (FMT == kZetaF32 || FMT == kZetaI8H || dbg_zeta)) ? __ldg(beta + row) : 0.f;
+        const float be = (row_in && (FMT == kZetaF32 || FMT == kZetaI8H || dbg_zeta || row_tail)) ? __ldg(beta + row) : 0.f;
+        float row_fac = be;                                 // the node factor the aggregation multiplies the edge value by
         int f0 = 0;                                         // half-dot bytes: the row's first sign (0 when d_in is odd)
         if constexpr (FMT == kZetaI8H) {
             if (row_in) {
                 const int sgn = (__ldg(A + row * stride_a) & 1u) ? 1 : -1;
                 f0 = (d_in & 1) ? 0 : sgn;
-                if (warp < 4) nws[row] = (d_in & 1) ? be : be * (float)sgn;      // beta_i carrying the first sign
+                row_fac = (d_in & 1) ? be : be * (float)sgn;                     // beta_i carrying the first sign
+                if (warp < 4) nws[row] = row_fac;
             }
         }
 #pragma unroll 1
@@ -278,6 +283,9 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
                 }
                 uint4 out[kElt];
                 Out::pack(dot, be, al_s + c0, out);
+                if constexpr (kElt == 1) {
+                    if (row_tail && c0 == 48) out[0].w = __float_as_uint(row_fac);
+                }
 #pragma unroll
                 for (int u = 0; u < kElt; ++u) {
                     const int piece = ch * kElt + u;
@@ -318,7 +326,7 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
 template <int N, int FMT>
 cudaError_t launch_tc_inst(cudaStream_t s, const uint32_t* A, int64_t stride_a, const uint32_t* BT, int64_t stride_b,
                            int64_t n, int d_in, int d_out, const float* beta, const float* alpha, void* zeta, int64_t ldz,
-                           int32_t* dbg_dot, float* dbg_zeta, float* nws, float* col_b0)
+                           int32_t* dbg_dot, float* dbg_zeta, float* nws, float* col_b0, int row_tail)
 {
     // operands: weight panel N x K bytes, feature tile 128 x K bytes (at least the 32 KB the epilogue's scratch needs)
     size_t smem = (size_t)N * stride_a * 32 + std::max<size_t>((size_t)kTcRows * stride_a * 32, 32 * 1024);
@@ -328,16 +336,16 @@ cudaError_t launch_tc_inst(cudaStream_t s, const uint32_t* A, int64_t stride_a, 
     cudaError_t e = cudaFuncSetAttribute(bitgemm_tc_kernel<N, FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, kTcRows), sm_count() * 2);
-    bitgemm_tc_kernel<N, FMT><<<grid, kTcThreads, smem, s>>>(A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0);
+    bitgemm_tc_kernel<N, FMT><<<grid, kTcThreads, smem, s>>>(A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0, row_tail);
     return cudaGetLastError();
 }
 
 template <int N>
 cudaError_t launch_tc_n(cudaStream_t s, int fmt, const uint32_t* A, int64_t stride_a, const uint32_t* BT, int64_t stride_b,
                         int64_t n, int d_in, int d_out, const float* beta, const float* alpha, void* zeta, int64_t ldz,
-                        int32_t* dbg_dot, float* dbg_zeta, float* nws, float* col_b0)
+                        int32_t* dbg_dot, float* dbg_zeta, float* nws, float* col_b0, int row_tail)
 {
-#define BIGCN_TC_CALL(FMT) launch_tc_inst<N, FMT>(s, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0)
+#define BIGCN_TC_CALL(FMT) launch_tc_inst<N, FMT>(s, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0, (N == 64 && ldz == 64) ? row_tail : 0)
     switch (fmt) {
         case kZetaF32: return BIGCN_TC_CALL(kZetaF32);
         case kZetaF16: return BIGCN_TC_CALL(kZetaF16);
@@ -358,12 +366,12 @@ bool bitgemm_tc_covers(int d_in, int d_out, int64_t stride_a, int64_t stride_b)
 
 cudaError_t launch_bitgemm_tc(cudaStream_t s, const uint32_t* A, int64_t stride_a, const uint32_t* BT, int64_t stride_b,
                               int64_t n, int d_in, int d_out, const float* beta, const float* alpha, int fmt, void* zeta,
-                              int64_t ldz, int32_t* dbg_dot, float* dbg_zeta, float* nws, float* col_b0)
+                              int64_t ldz, int32_t* dbg_dot, float* dbg_zeta, float* nws, float* col_b0, int row_tail)
 {
     // the instruction's N: the output channels rounded up to 64 / 128 / 256 (16 would do; fewer variants to build)
-    if (d_out <= 64) return launch_tc_n<64>(s, fmt, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0);
-    if (d_out <= 128) return launch_tc_n<128>(s, fmt, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0);
-    return launch_tc_n<256>(s, fmt, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0);
+    if (d_out <= 64) return launch_tc_n<64>(s, fmt, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0, row_tail);
+    if (d_out <= 128) return launch_tc_n<128>(s, fmt, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0, 0);
+    return launch_tc_n<256>(s, fmt, A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0, 0);
 }
 
 // Number of waits that ran out since the library was loaded on the current device (0 = none).

@@ -1190,7 +1190,9 @@ constexpr int kLanePitch = 68;                                // floats per lane
 
 // Streams rows [row_lo, row_hi) of a run (kPartial: the stored entries [e0, e0 + n_ent) as one row, whose sums are
 // handed back in `out` / `wsum` / `wsgn` instead of being written).
-template <int NV, bool kHalf, bool kPartial>
+// kTail: a row of zeta is 64 bytes, 32-byte aligned, and carries its node factor in its last four bytes: an entry's
+// dots and factor come with one pair of 32-byte loads (two tag lookups per entry instead of NV + 1).
+template <int NV, bool kHalf, bool kPartial, bool kTail = false>
 __device__ __forceinline__ void stream_rows_lane(const SpmmDev& p, float* red, int lane, int64_t e0, int n_ent,
                                                  int64_t warp_row0, int row_lo, int row_hi, int rp_rel,
                                                  const float (&al)[4], const float (&b0)[4], float4& out, float& wsum_out, float& wsgn_out)
@@ -1224,10 +1226,22 @@ __device__ __forceinline__ void stream_rows_lane(const SpmmDev& p, float* red, i
     float nwn = 1.f;
     auto gather = [&](int c) {
         if (c >= 0) {
-            nwn = p.node_w ? __ldg(p.node_w + c) : 1.f;
-            const uint4* src = reinterpret_cast<const uint4*>(zeta + (uint64_t)(uint32_t)c * (uint32_t)(NV * 16));
+            if constexpr (kTail) {
+                const char* src = zeta + (uint64_t)(uint32_t)c * 64u;
+                uint32_t w[16];
+                asm volatile("ld.global.nc.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];\n"
+                             : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]) : "l"(src));
+                asm volatile("ld.global.nc.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];\n"
+                             : "=r"(w[8]), "=r"(w[9]), "=r"(w[10]), "=r"(w[11]), "=r"(w[12]), "=r"(w[13]), "=r"(w[14]), "=r"(w[15]) : "l"(src + 32));
 #pragma unroll
-            for (int q = 0; q < NV; ++q) vn[q] = __ldg(src + q);
+                for (int q = 0; q < NV; ++q) vn[q] = make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+                nwn = __uint_as_float(w[15]);
+            } else {
+                nwn = p.node_w ? __ldg(p.node_w + c) : 1.f;
+                const uint4* src = reinterpret_cast<const uint4*>(zeta + (uint64_t)(uint32_t)c * (uint32_t)(NV * 16));
+#pragma unroll
+                for (int q = 0; q < NV; ++q) vn[q] = __ldg(src + q);
+            }
         }
     };
     int c1, c2;
@@ -1324,7 +1338,7 @@ __device__ __forceinline__ void stream_rows_lane(const SpmmDev& p, float* red, i
     }
 }
 
-template <int NV, bool kHalf>
+template <int NV, bool kHalf, bool kTail = false>
 __global__ void __launch_bounds__(kLaneThreads, 2)
 spmm_lane_kernel(const SpmmDev p, int rows_per_warp)
 {
@@ -1374,7 +1388,7 @@ spmm_lane_kernel(const SpmmDev p, int rows_per_warp)
             const int rl = rest ? ra + (__ffs(rest) - 1) : n_rows;
             if (rl > ra) {
                 const int64_t e0 = __shfl_sync(0xffffffffu, rp_reg, ra);
-                stream_rows_lane<NV, kHalf, false>(p, red, lane, e0, 0, warp_row0, ra, rl, (int)(rp_reg - e0), al, b0, t, ws, wg);
+                stream_rows_lane<NV, kHalf, false, kTail>(p, red, lane, e0, 0, warp_row0, ra, rl, (int)(rp_reg - e0), al, b0, t, ws, wg);
             }
             ra = rl + 1;
         }
@@ -1386,7 +1400,7 @@ spmm_lane_kernel(const SpmmDev p, int rows_per_warp)
         const int64_t ls = __ldg(p.rowptr + lrow), le = __ldg(p.rowptr + lrow + 1);
         const int64_t slice = round_up(ceil_div(le - ls, kLaneWarps), 32);
         const int64_t s0 = min(le, ls + warp * slice), s1 = min(le, s0 + slice);
-        stream_rows_lane<NV, kHalf, true>(p, red, lane, s0, (int)(s1 - s0), 0, 0, (s1 > s0) ? 1 : 0, 0, al, b0, t, ws, wg);
+        stream_rows_lane<NV, kHalf, true, kTail>(p, red, lane, s0, (int)(s1 - s0), 0, 0, (s1 > s0) ? 1 : 0, 0, al, b0, t, ws, wg);
         if (lane < NG4) *reinterpret_cast<float4*>(part + warp * kPartPitch + 4 * cg) = t;
         if (lane == 0) {
             part[warp * kPartPitch + NG4 * 4] = ws;
@@ -1413,18 +1427,18 @@ spmm_lane_kernel(const SpmmDev p, int rows_per_warp)
     }
 }
 
-template <int NV, bool kHalf>
+template <int NV, bool kHalf, bool kTail = false>
 cudaError_t launch_lane(cudaStream_t s, const SpmmDev& p)
 {
     constexpr size_t smem = ((size_t)kLaneWarps * 32 * kLanePitch + (size_t)kLaneWarps * (NV * 16 + 4)) * sizeof(float);
     const int rows_per_warp = (int)std::min<int64_t>(kMaxRowsPerWarp, std::max<int64_t>(1, p.n / (kLaneWarps * sm_count() * 8)));
-    cudaError_t e = cudaFuncSetAttribute(spmm_lane_kernel<NV, kHalf>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(spmm_lane_kernel<NV, kHalf, kTail>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     e = cudaMemsetAsync(p.run_counter, 0, sizeof(int), s);
     if (e != cudaSuccess) return e;
     const int64_t wanted = ceil_div(ceil_div(p.n, rows_per_warp), kLaneWarps);
     const unsigned grid = (unsigned)std::min<int64_t>(wanted, sm_count() * 2);
-    spmm_lane_kernel<NV, kHalf><<<grid, kLaneThreads, smem, s>>>(p, rows_per_warp);
+    spmm_lane_kernel<NV, kHalf, kTail><<<grid, kLaneThreads, smem, s>>>(p, rows_per_warp);
     return cudaGetLastError();
 }
 
@@ -1570,6 +1584,11 @@ cudaError_t dispatch(cudaStream_t s, const SpmmDev& p, double mean_row)
     if constexpr (sizeof(T) == 1) {
         // 33..64 byte columns, fp32 output only (a last layer), rows not much shorter than a pass: one entry per lane
         if ((nv == 3 || nv == 4) && p.h_out && !p.next_bits && !p.add && p.byte_path != 2 && !(mean_row > 0.0 && mean_row < 8.0)) {
+            if (p.row_tail && nv == 4) {                      // 64-byte rows that carry their node factor: 3 or 4 vectors of columns
+                const bool three = p.d_out <= 48;
+                if (p.half_dots) return three ? launch_lane<3, true, true>(s, p) : launch_lane<4, true, true>(s, p);
+                return three ? launch_lane<3, false, true>(s, p) : launch_lane<4, false, true>(s, p);
+            }
             if (p.half_dots) return nv == 3 ? launch_lane<3, true>(s, p) : launch_lane<4, true>(s, p);
             return nv == 3 ? launch_lane<3, false>(s, p) : launch_lane<4, false>(s, p);
         }
@@ -1639,6 +1658,7 @@ cudaError_t launch_spmm(cudaStream_t s, const SpmmArgs& a, int* launches)
     p.col_b0 = a.half_dots ? a.col_b0 : nullptr;
     p.half_dots = a.half_dots ? 1 : 0;
     p.byte_path = a.byte_path;
+    p.row_tail = (a.row_tail && a.fmt == kZetaI8 && a.ldz == 64 && a.d_out <= 60) ? 1 : 0;
     if (a.half_dots && (a.fmt != kZetaI8 || p.nv > 16 || !a.col_b0 || !a.node_w)) return cudaErrorInvalidValue;   // up to 256 byte columns
     p.ld_add = a.ld_add;
     p.h_out = a.h_out;

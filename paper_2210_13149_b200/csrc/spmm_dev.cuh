@@ -20,6 +20,7 @@ struct SpmmDev {
     const float* col_b0;     // half-dot bytes only: per-column first weight sign (0 where none)
     int half_dots;           // zeta holds s = (dot' - 1) / 2; node_w carries the first feature sign
     int byte_path;           // 129..256 byte columns: 0 / 1 the FMA stream, 2 integer tensor-core products
+    int row_tail;            // rows of 64 bytes whose last four bytes hold the source's node factor as a float
     const float* add;        // nullable: fp32 [n x ld_add] added to the aggregated row (after col_w)
     int64_t ld_add;
     float* h_out;
