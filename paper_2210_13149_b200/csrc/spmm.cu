@@ -1195,7 +1195,8 @@ constexpr int kLanePitch = 68;                                // floats per lane
 template <int NV, bool kHalf, bool kPartial, bool kTail = false>
 __device__ __forceinline__ void stream_rows_lane(const SpmmDev& p, float* red, int lane, int64_t e0, int n_ent,
                                                  int64_t warp_row0, int row_lo, int row_hi, int rp_rel,
-                                                 const float (&al)[4], const float (&b0)[4], float4& out, float& wsum_out, float& wsgn_out)
+                                                 const float (&al)[4], const float (&b0)[4], float4& out, float& wsum_out, float& wsgn_out,
+                                                 const float (&al2)[4], const float (&b02)[4])
 {
     constexpr int NG4 = 4 * NV;                               // groups of four columns
     const int32_t* cols = p.colidx + e0;
@@ -1271,8 +1272,60 @@ __device__ __forceinline__ void stream_rows_lane(const SpmmDev& p, float* red, i
         for (int q = 0; q < NV; ++q) fma_bytes16(wa, v[q], acc[q]);
         const int rs = row_start(cr), re = row_end(cr);
         co += 32;
-        if (rs + co >= re) {
-            // ---- the row is complete: add the lanes' sums
+        if (!kPartial && rs + co >= re) {
+            // ---- the row is complete: add the 32 lanes' sums in registers.  Five exchange steps, each halving what a
+            // lane holds: a lane keeps the half of its columns that its bit of the lane index selects and sends the other
+            // half to its partner (16 NV shuffles in all); afterwards lanes 2 j and 2 j + 1 both hold the totals of
+            // columns 16 q + j, q < NV.  (Through shared memory the same reduction moved 12 KB per row, more than the
+            // row's gathered operands, and kept the L1 data path, not the gathers, the busiest unit.)
+            float x[NV];
+#pragma unroll
+            for (int q = 0; q < NV; ++q) {
+                float t8[8], t4[4], t2[2];
+                const bool h16 = (lane & 16) != 0, h8 = (lane & 8) != 0, h4 = (lane & 4) != 0, h2 = (lane & 2) != 0;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float send = h16 ? acc[q][i] : acc[q][8 + i], keep = h16 ? acc[q][8 + i] : acc[q][i];
+                    t8[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float send = h8 ? t8[i] : t8[4 + i], keep = h8 ? t8[4 + i] : t8[i];
+                    t4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+                }
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const float send = h4 ? t4[i] : t4[2 + i], keep = h4 ? t4[2 + i] : t4[i];
+                    t2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+                }
+                const float send = h2 ? t2[0] : t2[1], keep = h2 ? t2[1] : t2[0];
+                const float t1 = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+                x[q] = t1 + __shfl_xor_sync(0xffffffffu, t1, 1);
+            }
+            if (kHalf) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    ws += __shfl_xor_sync(0xffffffffu, ws, o);
+                    wg += __shfl_xor_sync(0xffffffffu, wg, o);
+                }
+            }
+            if ((lane & 1) == 0) {
+                const int j = lane >> 1;                      // this lane's column inside every group of 16
+                float* dst = p.h_out + (warp_row0 + cr) * p.ldh + j;
+#pragma unroll
+                for (int q = 0; q < NV; ++q) {
+                    float v = x[q];
+                    if (kHalf) v = fmaf(2.f, v, fmaf(b02[q], wg, ws));
+                    if (16 * q + j < p.d_out) dst[16 * q] = v * al2[q];
+                }
+            }
+            zero_acc<NV, 16>(acc);
+            ws = 0.f;
+            wg = 0.f;
+            ++cr;
+            co = 0;
+        } else if (kPartial && rs + co >= re) {
+            // ---- a slice of a long row is complete: add the lanes' sums through shared memory and hand them back
             float* mine = red + lane * kLanePitch;
 #pragma unroll
             for (int q = 0; q < NV; ++q)
@@ -1302,33 +1355,10 @@ __device__ __forceinline__ void stream_rows_lane(const SpmmDev& p, float* red, i
                     wg += __shfl_xor_sync(0xffffffffu, wg, o);
                 }
             }
-            if (kPartial) {
-                out = t;
-                wsum_out = ws;
-                wsgn_out = wg;
-                return;
-            }
-            if (lane < NG4) {
-                float x[4] = {t.x, t.y, t.z, t.w};
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    if (kHalf) x[i] = fmaf(2.f, x[i], fmaf(b0[i], wg, ws));
-                    x[i] *= al[i];
-                }
-                float* dst = p.h_out + (warp_row0 + cr) * p.ldh + 4 * cg;
-                if (p.h_vec && 4 * cg + 3 < p.d_out) {
-                    *reinterpret_cast<float4*>(dst) = make_float4(x[0], x[1], x[2], x[3]);
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i)
-                        if (4 * cg + i < p.d_out) dst[i] = x[i];
-                }
-            }
-            zero_acc<NV, 16>(acc);
-            ws = 0.f;
-            wg = 0.f;
-            ++cr;
-            co = 0;
+            out = t;
+            wsum_out = ws;
+            wsgn_out = wg;
+            return;
         }
     }
     if (kPartial) {                                           // empty slice
@@ -1360,6 +1390,14 @@ spmm_lane_kernel(const SpmmDev p, int rows_per_warp)
         al[i] = in ? (p.col_w ? __ldg(p.col_w + col) : 1.f) : 0.f;
         b0[i] = (in && kHalf && p.col_b0) ? __ldg(p.col_b0 + col) : 0.f;
     }
+    float al2[4], b02[4];                                     // the same constants for the columns 16 q + lane / 2 (rows finished in registers)
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const int col = 16 * q + (lane >> 1);
+        const bool in = q < NV && col < p.d_out;
+        al2[q] = in ? (p.col_w ? __ldg(p.col_w + col) : 1.f) : 0.f;
+        b02[q] = (in && kHalf && p.col_b0) ? __ldg(p.col_b0 + col) : 0.f;
+    }
     if (threadIdx.x == 0) n_long = 0;
     __syncthreads();
 
@@ -1388,7 +1426,7 @@ spmm_lane_kernel(const SpmmDev p, int rows_per_warp)
             const int rl = rest ? ra + (__ffs(rest) - 1) : n_rows;
             if (rl > ra) {
                 const int64_t e0 = __shfl_sync(0xffffffffu, rp_reg, ra);
-                stream_rows_lane<NV, kHalf, false, kTail>(p, red, lane, e0, 0, warp_row0, ra, rl, (int)(rp_reg - e0), al, b0, t, ws, wg);
+                stream_rows_lane<NV, kHalf, false, kTail>(p, red, lane, e0, 0, warp_row0, ra, rl, (int)(rp_reg - e0), al, b0, t, ws, wg, al2, b02);
             }
             ra = rl + 1;
         }
@@ -1400,7 +1438,7 @@ spmm_lane_kernel(const SpmmDev p, int rows_per_warp)
         const int64_t ls = __ldg(p.rowptr + lrow), le = __ldg(p.rowptr + lrow + 1);
         const int64_t slice = round_up(ceil_div(le - ls, kLaneWarps), 32);
         const int64_t s0 = min(le, ls + warp * slice), s1 = min(le, s0 + slice);
-        stream_rows_lane<NV, kHalf, true, kTail>(p, red, lane, s0, (int)(s1 - s0), 0, 0, (s1 > s0) ? 1 : 0, 0, al, b0, t, ws, wg);
+        stream_rows_lane<NV, kHalf, true, kTail>(p, red, lane, s0, (int)(s1 - s0), 0, 0, (s1 > s0) ? 1 : 0, 0, al, b0, t, ws, wg, al2, b02);
         if (lane < NG4) *reinterpret_cast<float4*>(part + warp * kPartPitch + 4 * cg) = t;
         if (lane == 0) {
             part[warp * kPartPitch + NG4 * 4] = ws;
