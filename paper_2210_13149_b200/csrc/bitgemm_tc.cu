@@ -105,8 +105,11 @@ template <> struct TcOut<kZetaI8> {
     {
         uint32_t b[4];
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
-            b[q] = ((uint32_t)dot[4 * q] & 0xffu) | (((uint32_t)dot[4 * q + 1] & 0xffu) << 8) | (((uint32_t)dot[4 * q + 2] & 0xffu) << 16) | ((uint32_t)dot[4 * q + 3] << 24);
+        for (int q = 0; q < 4; ++q) {                       // the low bytes of four ints in one word: three byte permutes
+            const uint32_t lo = __byte_perm((uint32_t)dot[4 * q], (uint32_t)dot[4 * q + 1], 0x0040);
+            const uint32_t hi = __byte_perm((uint32_t)dot[4 * q + 2], (uint32_t)dot[4 * q + 3], 0x0040);
+            b[q] = __byte_perm(lo, hi, 0x5410);
+        }
         out[0] = make_uint4(b[0], b[1], b[2], b[3]);
     }
 };
@@ -151,6 +154,7 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
     __shared__ uint32_t tmem_base_s;
     __shared__ float al_s[N];
     __shared__ int b0_s[FMT == kZetaI8H ? N : 1];          // half-dot bytes: first sign of every weight column (0 when d_in is odd)
+    __shared__ __align__(16) int hd_s[FMT == kZetaI8H ? 3 * N : 4];   // 1 + f b0_j for the row signs f = -1, 0, +1: what a half-dot subtracts
     constexpr int kCols = N <= 32 ? 32 : (N <= 64 ? 64 : (N <= 128 ? 128 : 256));   // tensor-memory columns of the accumulator
     const int K = (int)stride_a * 32;                       // bytes per expanded row (padding included)
     const int pad = K - d_in;                               // padding positions: each contributes +1
@@ -172,6 +176,9 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
         for (int j = threadIdx.x; j < N; j += kTcThreads) {
             const int b0 = (even && j < d_out) ? ((__ldg(BT + (int64_t)j * stride_b) & 1u) ? 1 : -1) : 0;
             b0_s[j] = b0;
+            hd_s[j] = 1 - b0;
+            hd_s[N + j] = 1;
+            hd_s[2 * N + j] = 1 + b0;
             if (blockIdx.x == 0 && j < d_out) col_b0[j] = (float)b0;
         }
     }
@@ -271,15 +278,33 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
                              : "r"(taddr) : "memory");
                 asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
                 int dot[16];
+                const bool whole = c0 + 16 <= d_out;        // every column of the chunk exists: no per-column tests
+                if (whole) {
 #pragma unroll
-                for (int e = 0; e < 16; ++e) dot[e] = (c0 + e < d_out) ? (int)v[e] - pad : 0;   // padding columns of zeta stay 0
+                    for (int e = 0; e < 16; ++e) dot[e] = (int)v[e] - pad;
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) dot[e] = (c0 + e < d_out) ? (int)v[e] - pad : 0;   // padding columns of zeta stay 0
+                }
                 int full[16];                               // the true dots, for the debug taps
 #pragma unroll
                 for (int e = 0; e < 16; ++e) full[e] = dot[e];
-                if constexpr (FMT == kZetaI8H) {
+                if constexpr (FMT == kZetaI8H) {            // s = (dot - f0 b0_j - 1) / 2: odd by construction, exact
+                    const int4* hd = reinterpret_cast<const int4*>(hd_s + (f0 + 1) * N + c0);
+                    int sub[16];
 #pragma unroll
-                    for (int e = 0; e < 16; ++e)
-                        if (c0 + e < d_out) dot[e] = (dot[e] - f0 * b0_s[c0 + e] - 1) >> 1;       // odd by construction: exact
+                    for (int q = 0; q < 4; ++q) {
+                        const int4 t = hd[q];
+                        sub[4 * q] = t.x, sub[4 * q + 1] = t.y, sub[4 * q + 2] = t.z, sub[4 * q + 3] = t.w;
+                    }
+                    if (whole) {
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) dot[e] = (dot[e] - sub[e]) >> 1;
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 16; ++e)
+                            if (c0 + e < d_out) dot[e] = (dot[e] - sub[e]) >> 1;
+                    }
                 }
                 uint4 out[kElt];
                 Out::pack(dot, be, al_s + c0, out);
