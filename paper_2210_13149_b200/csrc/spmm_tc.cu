@@ -193,7 +193,7 @@ __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, vo
 #pragma unroll
     for (int q = 0; q < kLag; ++q) ci_h[q] = ni_h[q] = ri_h[q] = 0;
 
-    for (int64_t k = 0;;) {                                   // k: chunks published so far
+    for (uint32_t k = 0;;) {                                  // k: chunks published so far
         asm volatile("cp.async.wait_group %0;\n" ::"n"(kLag - 1) : "memory");
         __syncwarp();
         const int ci_done = ci_h[kLag - 1], ni_done = ni_h[kLag - 1], ri_done = ri_h[kLag - 1];
@@ -235,7 +235,7 @@ __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, vo
         const bool finished = r == nrows;
         if (!finished && !(min(r + kSegMax + 1, nrows + 1) <= ri_done && min(e + kChunk, total) <= ni_done)) continue;
         const int slot_i = (int)(k % kSlots);
-        if (!mbar_wait(&prep_empty[slot_i], ((uint32_t)(k / kSlots) & 1u) ^ 1u, abort, 200)) break;
+        if (!mbar_wait(&prep_empty[slot_i], ((k / kSlots) & 1u) ^ 1u, abort, 400)) break;
         ChunkSlot* slot = reinterpret_cast<ChunkSlot*>(sm + kOffSlots) + slot_i;
         unsigned char* Bs = sm + kOffB + slot_i * kBSlotBytes;
         if (finished) {                                       // end of the stream
@@ -344,7 +344,7 @@ __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, vo
 __device__ __forceinline__ bool wait_bcast(uint64_t* bar, uint32_t parity, volatile int* abort, int lane)
 {
     int ok = 1;
-    if (lane == 0) ok = mbar_wait(bar, parity, abort, 100) ? 1 : 0;
+    if (lane == 0) ok = mbar_wait(bar, parity, abort, 250) ? 1 : 0;
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
@@ -362,29 +362,29 @@ __device__ __forceinline__ void issuer(const SpmmDev& p, unsigned char* sm, vola
     const uint32_t a_base = smem_u32(sm + kOffA), b_base = smem_u32(sm + kOffB);
     // instruction descriptor: D = s32, A = B = s8, both M/N-major, N = 32, M = 128
     const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(kN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-    for (int64_t c = 0;; ++c) {
-        if (!wait_bcast(&prep_full[c % kSlots], (uint32_t)((c / kSlots) & 1), abort, lane)) return;
-        const ChunkSlot* slot = slots + (int)(c % kSlots);
+    for (uint32_t c = 0;; ++c) {
+        if (!wait_bcast(&prep_full[c % kSlots], (c / kSlots) & 1u, abort, lane)) return;
+        const ChunkSlot* slot = slots + (c % kSlots);
         const int n_ent = slot->n_ent;
         if (n_ent < 0) return;                                // end of the stream
-        if (!wait_bcast(&a_full[c % kAStages], (uint32_t)((c / kAStages) & 1), abort, lane)) return;
-        if (c >= 2 && !wait_bcast(&tmem_empty[c & 1], (uint32_t)(((c >> 1) - 1) & 1), abort, lane)) return;
+        if (!wait_bcast(&a_full[c % kAStages], (c / kAStages) & 1u, abort, lane)) return;
+        if (c >= 2 && !wait_bcast(&tmem_empty[c & 1u], ((c >> 1) - 1u) & 1u, abort, lane)) return;
         if (lane == 0) {
             tc::fence_async_smem();                           // the copied rows become visible to the tensor core
             tc::fence_after_sync();
             const int ksteps = max(1, (n_ent + 31) >> 5);
-            const uint32_t a_stage = a_base + (uint32_t)(c % kAStages) * kAStageBytes;
-            const uint32_t b_slot = b_base + (uint32_t)(c % kSlots) * kBSlotBytes;
+            const uint32_t a_stage = a_base + (c % kAStages) * kAStageBytes;
+            const uint32_t b_slot = b_base + (c % kSlots) * kBSlotBytes;
             for (int hh = 0; hh < 2; ++hh)
                 for (int ks = 0; ks < ksteps; ++ks) {
                     const uint64_t ad = make_desc_l(a_stage + hh * 8192 + ks * 4096, 8192, 1024, 2);
                     const uint64_t bd = make_desc_l(b_slot + ks * 512, 128, 1024, 0);
-                    const uint32_t d_addr = tmem_base + (uint32_t)((c & 1) * 64 + hh * 32);
+                    const uint32_t d_addr = tmem_base + (c & 1u) * 64u + (uint32_t)(hh * 32);
                     const uint32_t accum = ks > 0 ? 1u : 0u;
                     asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}\n"
                                  ::"r"(d_addr), "l"(ad), "l"(bd), "r"(idesc), "r"(accum) : "memory");
                 }
-            tc::commit_to(&mma_done[c & 1]);
+            tc::commit_to(&mma_done[c & 1u]);
         }
         __syncwarp();
     }
@@ -431,30 +431,37 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
     const char* zeta_b = reinterpret_cast<const char*>(p.zeta);
     const uint32_t row_bytes = (uint32_t)p.nv * 16u;
     const int sub = lane >> 3, piece = lane & 7;              // a warp instruction copies 4 entries x 128 contiguous bytes
+    const bool lo_in = piece < p.nv, hi_in = 8 + piece < p.nv;   // this lane's 16-byte piece exists in operand 0 / 1
+    const char* zeta_l = zeta_b + piece * 16;
+    uint32_t dst_off[4];                                      // where this lane's piece of entry 16 warp + 4 g + sub goes inside a stage
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        const int j = 16 * warp + 4 * g + sub;
+        dst_off[g] = (uint32_t)(j * 128 + ((piece ^ (j & 7)) * 16));
+    }
     // copies of chunk c into operand stage c % kAStages: warp w takes the entries 16 w .. 16 w + 15, both operands; they
-    // report to the stage's mbarrier when they have landed
-    auto gather = [&](int64_t c) {
-        const ChunkSlot* slot = slots + (int)(c % kSlots);
+    // report to the stage's mbarrier when they have landed.  (Chunk counters are 32-bit: a block sees far fewer than 2^31.)
+    auto gather = [&](uint32_t c) {
+        const ChunkSlot* slot = slots + (c % kSlots);
         const int n_ent = slot->n_ent;
-        const uint32_t stage = a_base + (uint32_t)(c % kAStages) * kAStageBytes;
+        const uint32_t stage = a_base + (c % kAStages) * kAStageBytes;
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
             const int j = 16 * warp + 4 * g + sub;
             if (j < n_ent) {
-                const char* src = zeta_b + (uint64_t)(uint32_t)slot->cols[j] * row_bytes + piece * 16;
-                const uint32_t dst = stage + j * 128 + ((piece ^ (j & 7)) * 16);
-                if (piece < p.nv) cp_async16(dst, src);
-                if (8 + piece < p.nv) cp_async16(dst + 8192, src + 128);
+                const char* src = zeta_l + (uint64_t)(uint32_t)slot->cols[j] * row_bytes;
+                if (lo_in) cp_async16(stage + dst_off[g], src);
+                if (hi_in) cp_async16(stage + dst_off[g] + 8192, src + 128);
             }
         }
         asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(smem_u32(&a_full[c % kAStages])) : "memory");
     };
 
-    int64_t end_idx = INT64_MAX;                              // index of the end marker once seen
+    uint32_t end_idx = 0xffffffffu;                           // index of the end marker once seen
     bool bad = false;
     // prologue: the rows of the first kAStages chunks (only one thread polls; the others wait at the named barrier)
-    for (int64_t c = 0; c < kAStages && end_idx == INT64_MAX && !bad; ++c) {
-        if (tid == 0 && !mbar_wait(&prep_full[c % kSlots], (uint32_t)((c / kSlots) & 1), abort)) bad = true;
+    for (uint32_t c = 0; c < kAStages && end_idx == 0xffffffffu && !bad; ++c) {
+        if (tid == 0 && !mbar_wait(&prep_full[c % kSlots], (c / kSlots) & 1u, abort)) bad = true;
         bad = consumers_sync_or(bad);
         if (!bad) {
             if (slots[c % kSlots].n_ent < 0) end_idx = c;
@@ -464,18 +471,19 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
 
     float acc[2] = {0.f, 0.f};                                // the open row: this thread's two column sums
     float rs = 0.f, rg = 0.f;                                 // and the row's weight sums (half-dot bytes)
-    for (int64_t i = 0; !bad; ++i) {
-        const bool has_cur = i < end_idx, need_next = end_idx == INT64_MAX;
+    int prev_nseg = 0;                                        // segments of chunk i - 1
+    for (uint32_t i = 0; !bad; ++i) {
+        const bool has_cur = i < end_idx, need_next = end_idx == 0xffffffffu;
         if (tid == 0) {
-            if (has_cur && !mbar_wait(&mma_done[i & 1], (uint32_t)((i >> 1) & 1), abort)) bad = true;
-            if (!bad && need_next && !mbar_wait(&prep_full[(i + kAStages) % kSlots], (uint32_t)(((i + kAStages) / kSlots) & 1), abort)) bad = true;
+            if (has_cur && !mbar_wait(&mma_done[i & 1u], (i >> 1) & 1u, abort)) bad = true;
+            if (!bad && need_next && !mbar_wait(&prep_full[(i + kAStages) % kSlots], ((i + kAStages) / kSlots) & 1u, abort)) bad = true;
         }
         tc::fence_before_sync();
         if (consumers_sync_or(bad)) break;
         tc::fence_after_sync();
         // beta of the rows that ended in chunk i - 1: the four warps' partial sums in warp order
-        if (i >= 1 && p.next_bits && tid < kSegMax) {
-            const int par = (int)((i - 1) & 1);
+        if (p.next_bits && tid < prev_nseg) {
+            const int par = (int)((i - 1u) & 1u);
             const int row = beta_row[par * kSegMax + tid];
             if (row >= 0) {
                 const float* bp = beta_part + (par * kSegMax + tid) * 8;
@@ -489,13 +497,14 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
             else gather(i + kAStages);
         }
         // read back chunk i: the four digit sums of every segment, both operands
-        const ChunkSlot* slot = slots + (int)(i % kSlots);
-        const int par = (int)(i & 1);
+        const ChunkSlot* slot = slots + (i % kSlots);
+        const int par = (int)(i & 1u);
         const int nseg = slot->nseg;
+        prev_nseg = nseg;
         const uint32_t t_addr = tmem_base + ((uint32_t)(32 * warp) << 16) + (uint32_t)(par * 64);
-        for (int s = 0; s < kSegMax; ++s) {                    // a run-time loop: small code, the same for every segment
+        for (int s = 0; s < nseg; ++s) {                       // a run-time loop (uniform over the readers): small code, the same for every segment
             int row_done = -1;
-            if (s < nseg) {                                   // uniform over the consumers
+            {
                 uint32_t a0, a1, a2, a3, c0, c1, c2, c3;
                 asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];\n"
                              : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(t_addr + 4 * s) : "memory");
