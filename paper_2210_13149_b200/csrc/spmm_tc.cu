@@ -96,15 +96,16 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar)
 {
     asm volatile("{\n.reg .b64 st;\nmbarrier.arrive.shared::cta.b64 st, [%0];\n}\n" ::"r"(smem_u32(bar)) : "memory");
 }
-// Bounded wait that also gives up when another thread of the block has raised `abort`.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort, unsigned backoff_ns = 0)
+// Bounded wait that also gives up when another thread of the block has raised `abort`.  No sleep between tries: the
+// try itself parks the thread (measured: next to no failed tries), and every sleep added to it showed up in the chain
+// of hand-offs that bounds the kernel.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort)
 {
     uint32_t done = 0;
     for (int it = 0; it < kTries && !done; ++it) {
         asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}\n"
                      : "=r"(done) : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendNs) : "memory");   // the thread may be parked for up to the hint
         if (done || *abort) break;
-        if (backoff_ns) __nanosleep(backoff_ns);
     }
     if (!done) {
         atomicExch(&g_spmm_tc_timeout, 1);
@@ -235,7 +236,7 @@ __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, vo
         const bool finished = r == nrows;
         if (!finished && !(min(r + kSegMax + 1, nrows + 1) <= ri_done && min(e + kChunk, total) <= ni_done)) continue;
         const int slot_i = (int)(k % kSlots);
-        if (!mbar_wait(&prep_empty[slot_i], ((k / kSlots) & 1u) ^ 1u, abort, 400)) break;
+        if (!mbar_wait(&prep_empty[slot_i], ((k / kSlots) & 1u) ^ 1u, abort)) break;
         ChunkSlot* slot = reinterpret_cast<ChunkSlot*>(sm + kOffSlots) + slot_i;
         unsigned char* Bs = sm + kOffB + slot_i * kBSlotBytes;
         if (finished) {                                       // end of the stream
@@ -344,7 +345,7 @@ __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, vo
 __device__ __forceinline__ bool wait_bcast(uint64_t* bar, uint32_t parity, volatile int* abort, int lane)
 {
     int ok = 1;
-    if (lane == 0) ok = mbar_wait(bar, parity, abort, 250) ? 1 : 0;
+    if (lane == 0) ok = mbar_wait(bar, parity, abort) ? 1 : 0;
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
