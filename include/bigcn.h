@@ -91,8 +91,12 @@ enum {
      * as those of the normalized adjacency are); 2 = as exact integer products on the tensor cores (mma.sync
      * s8 x s8 -> s32: the edge weights of up to 32 stored entries of a row in 28..31-bit fixed point against a
      * common power of two, split into four signed base-256 digits; the digit sums recombined in fp32 when the row
-     * ends; edge values of either sign).  The FMA stream is the default because it measured faster (6.0 / 6.4 ms
-     * against 8.0 / 8.3 ms on the two 256-column layers of a 2.4 M-node, 126 M-entry graph). */
+     * ends; edge values of either sign); 3 = the same fixed-point digits on the 5th-generation tensor cores
+     * (tcgen05.mma kind::i8: the gathered rows of 64 stored entries go by asynchronous copies straight into shared
+     * memory as the swizzled A operand, the digits of the edge weights are the B operand, the digit sums are read back
+     * from tensor memory once per row segment; graphs of fewer than 2^31 stored entries, otherwise the FMA stream
+     * runs).  The FMA stream is the default because it measured fastest (5.7-5.9 / 5.9-6.1 ms against 8.0 / 8.3 ms
+     * for 2 and 6.3 / 6.7 ms for 3 on the two 256-column layers of a 2.4 M-node, 126 M-entry graph). */
     BIGCN_OPT_BYTE_AGGREGATION = 4
 };
 
