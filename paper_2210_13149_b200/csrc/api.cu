@@ -66,10 +66,12 @@ size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 // (47 columns on 126 M entries: 3.69 + 0.21 ms against 3.72 + 0.16 ms for aggregation + contraction).
 // `fp32_only`: the layer's result is only written out as fp32 (a network's last layer); then 33..64 columns also take
 // bytes, for which the aggregation has a stream with one stored entry per lane (c4 layer 1: 2.8 -> 1.8 ms).
-int pick_format(const bigcn_ctx* ctx, int d_in, int d_out, int64_t n, bool allow_half = false, bool fp32_only = false)
+// narrow_bytes: rows of 33..64 columns may be stored as bytes too (the aggregation then has its one-entry-per-lane
+// stream: a last layer written as fp32, or a hidden layer of a graph whose rows are not much shorter than a pass)
+int pick_format(const bigcn_ctx* ctx, int d_in, int d_out, int64_t n, bool allow_half = false, bool narrow_bytes = false)
 {
     int f = ctx->zeta_format;
-    const bool wide = (d_out > 128 && d_out <= 256) || (fp32_only && d_out > 32 && d_out <= 64);
+    const bool wide = (d_out > 128 && d_out <= 256) || (narrow_bytes && d_out > 32 && d_out <= 64);
     // half-dot bytes keep two side arrays (n node factors, d_out first weight signs) behind the byte rows inside
     // the zeta scratch, which is sized for fp32 rows: they must fit there (they do not for d_out <= 4, where an fp32
     // row is no longer than a byte row)
@@ -136,12 +138,13 @@ bigcn_status run_layer(bigcn_ctx* ctx, const bigcn_graph* g, const bigcn_layer* 
                        float* next_beta, int32_t* dbg_dot, float* dbg_zeta,
                        cudaEvent_t ev_mid /*nullable*/)
 {
-    const int fmt = pick_format(ctx, layer->d_in, layer->d_out, g->n, /*allow_half=*/true, /*fp32_only=*/next == nullptr && h_out != nullptr);
+    const bool lane_stream = (next == nullptr && h_out != nullptr) || (next != nullptr && g->nnz >= 8 * g->n);
+    const int fmt = pick_format(ctx, layer->d_in, layer->d_out, g->n, /*allow_half=*/true, /*narrow_bytes=*/lane_stream);
     const bool half = fmt == kZetaI8H;
     const int64_t stride_in = bigcn_packed_stride_words(layer->d_in);
-    // a last layer of 33..60 byte columns on the tensor-core contraction: 64-byte rows that carry the node factor in
-    // their last four bytes, so that the aggregation's lane-per-entry stream needs two lookups per entry, not four or five
-    const bool row_tail = (fmt == kZetaI8 || half) && next == nullptr && h_out != nullptr && layer->d_out > 32 && layer->d_out <= 60 &&
+    // 33..60 byte columns for the lane-per-entry stream, on the tensor-core contraction: 64-byte rows that carry the node
+    // factor in their last four bytes, so that the aggregation needs two lookups per entry, not four or five
+    const bool row_tail = (fmt == kZetaI8 || half) && lane_stream && layer->d_out > 32 && layer->d_out <= 60 &&
                           bitgemm_takes_tc(fmt, half ? 2 : ctx->contraction, g->n, layer->d_in, layer->d_out, stride_in, stride_in);
     const int64_t ldz = row_tail ? 64 : zeta_ld(layer->d_out, fmt);
     // half-dot bytes: the node factors carrying the first feature sign and the columns' first weight signs follow

@@ -1175,8 +1175,8 @@ cudaError_t launch_imma(cudaStream_t s, SpmmDev p)
 
 // ---- narrow rows of signed bytes, one stored entry per lane ------------------------------------------------------
 //
-// For rows of 3 or 4 sixteen-byte vectors (33..64 byte columns) whose result is only written out as fp32 (a
-// network's last layer).  The streams above give a lane one vector of an entry, so a warp handles 8 entries per
+// For rows of 3 or 4 sixteen-byte vectors (33..64 byte columns): a network's last layer (fp32 out) or, with kNext,
+// a hidden layer whose result is re-binarized for the next one (more columns do not fit: a lane holds 16 NV sums).  The streams above give a lane one vector of an entry, so a warp handles 8 entries per
 // instruction and every row end costs a reduction over the lane groups; here a lane owns a whole stored entry:
 // it loads the entry's column, value and node factor itself (no shuffles), fetches the NV vectors of the operand
 // row straight into registers and accumulates all 16 NV columns.  A pass is up to 32 entries of one row; the
@@ -1192,7 +1192,7 @@ constexpr int kLanePitch = 68;                                // floats per lane
 // handed back in `out` / `wsum` / `wsgn` instead of being written).
 // kTail: a row of zeta is 64 bytes, 32-byte aligned, and carries its node factor in its last four bytes: an entry's
 // dots and factor come with one pair of 32-byte loads (two tag lookups per entry instead of NV + 1).
-template <int NV, bool kHalf, bool kPartial, bool kTail = false>
+template <int NV, bool kHalf, bool kPartial, bool kTail = false, bool kNext = false>
 __device__ __forceinline__ void stream_rows_lane(const SpmmDev& p, float* red, int lane, int64_t e0, int n_ent,
                                                  int64_t warp_row0, int row_lo, int row_hi, int rp_rel,
                                                  const float (&al)[4], const float (&b0)[4], float4& out, float& wsum_out, float& wsgn_out,
@@ -1309,15 +1309,45 @@ __device__ __forceinline__ void stream_rows_lane(const SpmmDev& p, float* red, i
                     wg += __shfl_xor_sync(0xffffffffu, wg, o);
                 }
             }
-            if ((lane & 1) == 0) {
-                const int j = lane >> 1;                      // this lane's column inside every group of 16
+            const int j = lane >> 1;                          // this lane's column inside every group of 16
+#pragma unroll
+            for (int q = 0; q < NV; ++q) {
+                if (kHalf) x[q] = fmaf(2.f, x[q], fmaf(b02[q], wg, ws));
+                x[q] *= al2[q];
+            }
+            if ((!kNext || p.h_out) && (lane & 1) == 0) {
                 float* dst = p.h_out + (warp_row0 + cr) * p.ldh + j;
 #pragma unroll
+                for (int q = 0; q < NV; ++q)
+                    if (16 * q + j < p.d_out) dst[16 * q] = x[q];
+            }
+            if constexpr (kNext) {
+                // ---- re-binarization for the next layer: the lanes 2 j and 2 j + 1 hold column 16 q + j; a packed word
+                // wants column 32 w + l in lane l, i.e. group 2 w from lane 2 l for l < 16, group 2 w + 1 from lane
+                // 2 (l - 16) otherwise: two shuffles and a ballot per word
+                const int64_t row = warp_row0 + cr;
+                float xh[NV], l1 = 0.f;
+#pragma unroll
                 for (int q = 0; q < NV; ++q) {
-                    float v = x[q];
-                    if (kHalf) v = fmaf(2.f, v, fmaf(b02[q], wg, ws));
-                    if (16 * q + j < p.d_out) dst[16 * q] = v * al2[q];
+                    const int col = 16 * q + j;
+                    const bool in = col < p.d_out;
+                    const float sh = (in && p.next_shift) ? __ldg(p.next_shift + col) : 0.f;
+                    const float sc = (in && p.next_shift) ? __ldg(p.next_scale + col) : 1.f;
+                    xh[q] = in ? __fmul_rn(__fsub_rn(x[q], sh), sc) : -1.f;    // columns past d_out pack as 0
+                    if (in && (lane & 1) == 0) l1 += fabsf(xh[q]);
                 }
+                const int src = 2 * (lane & 15);
+#pragma unroll
+                for (int w = 0; w < (NV + 1) / 2; ++w) {
+                    const float a = __shfl_sync(0xffffffffu, xh[2 * w], src);
+                    const float b = (2 * w + 1 < NV) ? __shfl_sync(0xffffffffu, xh[(2 * w + 1 < NV) ? 2 * w + 1 : 0], src) : -1.f;
+                    const uint32_t word = __ballot_sync(0xffffffffu, (lane < 16 ? a : b) >= 0.f);
+                    if (lane == 0 && w < p.next_stride) p.next_bits[row * p.next_stride + w] = word;
+                }
+                for (int w = (NV + 1) / 2 + lane; w < p.next_stride; w += 32) p.next_bits[row * p.next_stride + w] = 0u;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) l1 += __shfl_xor_sync(0xffffffffu, l1, o);
+                if (lane == 0) p.next_beta[row] = l1 * p.inv_d_out;
             }
             zero_acc<NV, 16>(acc);
             ws = 0.f;
@@ -1368,7 +1398,7 @@ __device__ __forceinline__ void stream_rows_lane(const SpmmDev& p, float* red, i
     }
 }
 
-template <int NV, bool kHalf, bool kTail = false>
+template <int NV, bool kHalf, bool kTail = false, bool kNext = false>
 __global__ void __launch_bounds__(kLaneThreads, 2)
 spmm_lane_kernel(const SpmmDev p, int rows_per_warp)
 {
@@ -1426,7 +1456,7 @@ spmm_lane_kernel(const SpmmDev p, int rows_per_warp)
             const int rl = rest ? ra + (__ffs(rest) - 1) : n_rows;
             if (rl > ra) {
                 const int64_t e0 = __shfl_sync(0xffffffffu, rp_reg, ra);
-                stream_rows_lane<NV, kHalf, false, kTail>(p, red, lane, e0, 0, warp_row0, ra, rl, (int)(rp_reg - e0), al, b0, t, ws, wg, al2, b02);
+                stream_rows_lane<NV, kHalf, false, kTail, kNext>(p, red, lane, e0, 0, warp_row0, ra, rl, (int)(rp_reg - e0), al, b0, t, ws, wg, al2, b02);
             }
             ra = rl + 1;
         }
@@ -1445,38 +1475,65 @@ spmm_lane_kernel(const SpmmDev p, int rows_per_warp)
             part[warp * kPartPitch + NG4 * 4 + 1] = wg;
         }
         __syncthreads();
-        if (warp == 0 && lane < NG4) {
+        if (warp == 0) {
             float x[4] = {0.f, 0.f, 0.f, 0.f};
             float sws = 0.f, swg = 0.f;
-            for (int w = 0; w < kLaneWarps; ++w) {
-                const float4 u = *reinterpret_cast<const float4*>(part + w * kPartPitch + 4 * cg);
-                x[0] += u.x, x[1] += u.y, x[2] += u.z, x[3] += u.w;
-                sws += part[w * kPartPitch + NG4 * 4];
-                swg += part[w * kPartPitch + NG4 * 4 + 1];
-            }
+            if (lane < NG4) {
+                for (int w = 0; w < kLaneWarps; ++w) {
+                    const float4 u = *reinterpret_cast<const float4*>(part + w * kPartPitch + 4 * cg);
+                    x[0] += u.x, x[1] += u.y, x[2] += u.z, x[3] += u.w;
+                    sws += part[w * kPartPitch + NG4 * 4];
+                    swg += part[w * kPartPitch + NG4 * 4 + 1];
+                }
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                if (kHalf) x[i] = fmaf(2.f, x[i], fmaf(b0[i], swg, sws));
-                x[i] *= al[i];
-                if (4 * cg + i < p.d_out) p.h_out[lrow * p.ldh + 4 * cg + i] = x[i];
+                for (int i = 0; i < 4; ++i) {
+                    if (kHalf) x[i] = fmaf(2.f, x[i], fmaf(b0[i], swg, sws));
+                    x[i] *= al[i];
+                    if ((!kNext || p.h_out) && 4 * cg + i < p.d_out) p.h_out[lrow * p.ldh + 4 * cg + i] = x[i];
+                }
+            }
+            if constexpr (kNext) {                            // lane l < NG4 holds columns 4 l .. 4 l + 3: eight lanes per packed word
+                uint32_t bits = 0u;
+                float l1 = 0.f;
+                if (lane < NG4) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int col = 4 * lane + i;
+                        if (col < p.d_out) {
+                            const float sh = p.next_shift ? __ldg(p.next_shift + col) : 0.f;
+                            const float sc = p.next_shift ? __ldg(p.next_scale + col) : 1.f;
+                            const float xh = __fmul_rn(__fsub_rn(x[i], sh), sc);
+                            if (xh >= 0.f) bits |= 1u << i;
+                            l1 += fabsf(xh);
+                        }
+                    }
+                }
+                uint32_t word = bits << ((4 * lane) & 31);
+#pragma unroll
+                for (int o = 1; o < 8; o <<= 1) word |= __shfl_xor_sync(0xffffffffu, word, o);
+                if ((lane & 7) == 0 && lane < NG4 && (lane >> 3) < p.next_stride) p.next_bits[lrow * p.next_stride + (lane >> 3)] = word;
+                for (int w = (NV + 1) / 2 + lane; w < p.next_stride; w += 32) p.next_bits[lrow * p.next_stride + w] = 0u;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) l1 += __shfl_xor_sync(0xffffffffu, l1, o);
+                if (lane == 0) p.next_beta[lrow] = l1 * p.inv_d_out;
             }
         }
         __syncthreads();
     }
 }
 
-template <int NV, bool kHalf, bool kTail = false>
+template <int NV, bool kHalf, bool kTail = false, bool kNext = false>
 cudaError_t launch_lane(cudaStream_t s, const SpmmDev& p)
 {
     constexpr size_t smem = ((size_t)kLaneWarps * 32 * kLanePitch + (size_t)kLaneWarps * (NV * 16 + 4)) * sizeof(float);
     const int rows_per_warp = (int)std::min<int64_t>(kMaxRowsPerWarp, std::max<int64_t>(1, p.n / (kLaneWarps * sm_count() * 8)));
-    cudaError_t e = cudaFuncSetAttribute(spmm_lane_kernel<NV, kHalf, kTail>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(spmm_lane_kernel<NV, kHalf, kTail, kNext>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     e = cudaMemsetAsync(p.run_counter, 0, sizeof(int), s);
     if (e != cudaSuccess) return e;
     const int64_t wanted = ceil_div(ceil_div(p.n, rows_per_warp), kLaneWarps);
     const unsigned grid = (unsigned)std::min<int64_t>(wanted, sm_count() * 2);
-    spmm_lane_kernel<NV, kHalf, kTail><<<grid, kLaneThreads, smem, s>>>(p, rows_per_warp);
+    spmm_lane_kernel<NV, kHalf, kTail, kNext><<<grid, kLaneThreads, smem, s>>>(p, rows_per_warp);
     return cudaGetLastError();
 }
 
@@ -1620,8 +1677,18 @@ cudaError_t dispatch(cudaStream_t s, const SpmmDev& p, double mean_row)
 {
     const int nv = p.nv;
     if constexpr (sizeof(T) == 1) {
-        // 33..64 byte columns, fp32 output only (a last layer), rows not much shorter than a pass: one entry per lane
-        if ((nv == 3 || nv == 4) && p.h_out && !p.next_bits && !p.add && p.byte_path != 2 && !(mean_row > 0.0 && mean_row < 8.0)) {
+        // 33..64 byte columns, written out as fp32 (a last layer) or re-binarized (a hidden layer), rows not much
+        // shorter than a pass: one entry per lane
+        if ((nv == 3 || nv == 4) && (p.h_out || p.next_bits) && !p.add && p.byte_path != 2 && !(mean_row > 0.0 && mean_row < 8.0)) {
+            if (p.next_bits) {
+                if (p.row_tail && nv == 4) {
+                    const bool three = p.d_out <= 48;
+                    if (p.half_dots) return three ? launch_lane<3, true, true, true>(s, p) : launch_lane<4, true, true, true>(s, p);
+                    return three ? launch_lane<3, false, true, true>(s, p) : launch_lane<4, false, true, true>(s, p);
+                }
+                if (p.half_dots) return nv == 3 ? launch_lane<3, true, false, true>(s, p) : launch_lane<4, true, false, true>(s, p);
+                return nv == 3 ? launch_lane<3, false, false, true>(s, p) : launch_lane<4, false, false, true>(s, p);
+            }
             if (p.row_tail && nv == 4) {                      // 64-byte rows that carry their node factor: 3 or 4 vectors of columns
                 const bool three = p.d_out <= 48;
                 if (p.half_dots) return three ? launch_lane<3, true, true>(s, p) : launch_lane<4, true, true>(s, p);

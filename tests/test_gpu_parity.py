@@ -363,6 +363,77 @@ def test_last_layer_narrow_byte_rows(ctx, B, fmt, n, e, d_in, d_out):
     assert torch.equal(again, out["h"])                       # run-to-run deterministic
 
 
+# hidden layers of 33..64 columns (re-binarized for a next layer) on graphs whose rows are not much shorter than a pass:
+# byte rows and the one-entry-per-lane stream by default; 64-byte rows that carry the node factor where the
+# tensor-core contraction runs (n * d_out >= 2^20); both byte formats; with and without the fp32 output
+HIDDEN_NARROW_SHAPES = [(0, 900, 9000, 254, 64), (0, 3000, 30000, 100, 47), (0, 40000, 400000, 256, 47), (0, 40000, 400000, 100, 64),
+                        (0, 40000, 400000, 127, 33), (0, 24000, 400000, 200, 60), (5, 1500, 40000, 256, 48), (3, 900, 20000, 127, 61),
+                        (0, 2000, 5000, 256, 47)]
+
+
+@pytest.mark.parametrize("fmt,n,e,d_in,d_out", HIDDEN_NARROW_SHAPES)
+def test_hidden_layer_narrow_byte_rows(ctx, B, fmt, n, e, d_in, d_out):
+    check_layer_forward(ctx, B, fmt, n, e, d_in, d_out)
+    # the same layer without the fp32 output: bits and beta only
+    rng = np.random.default_rng(n + 3 * d_in + 7 * d_out)
+    _, _, g = small_graph(n, e, 100 + n)
+    H = rng.standard_normal((n, d_in)).astype(np.float32)
+    W = (rng.standard_normal((d_in, d_out)) * d_in ** -0.5).astype(np.float32)
+    W2 = rng.standard_normal((d_out, 4)).astype(np.float32)
+    t = oracle.layer_forward(g, oracle.Layer(W), H)
+    nshift, nscale = oracle.col_stats(t.H_out)
+    Fn, beta_n = oracle.binarize_rows(t.H_out, nshift, nscale)
+    G = device_graph(B, g)
+    layer = B.make_layer(d_in, d_out, bits_to_dev(t.bitsT), dev(t.alpha))
+    nxt = B.make_layer(d_out, 4, bits_to_dev(oracle.pack_cols(oracle.binarize_cols(W2)[0])), dev(np.ones(4, np.float32)),
+                       dev(nshift), dev(nscale))
+    out = ctx.layer_forward(G, layer, bits_to_dev(t.bits), dev(t.beta), want_h=False, next_layer=nxt)
+    ctx.sync_check()
+    flips, bad, total = flip_report(bits_from_dev(out["next_bits"]), Fn, t.H_out, nshift)
+    assert bad == 0 and flips <= max(2, total // 2000)
+    nb = bits_from_dev(out["next_bits"])
+    if d_out % 32:
+        assert (nb[:, d_out // 32] >> (d_out % 32) == 0).all()
+    assert (nb[:, (d_out + 31) // 32:] == 0).all()
+    np.testing.assert_allclose(out["next_beta"].cpu().numpy(), beta_n, rtol=RTOL, atol=ATOL)
+
+
+@pytest.mark.parametrize("fmt,d_in", [(5, 256), (3, 100)])
+def test_hidden_layer_narrow_byte_rows_hub_row(ctx, B, fmt, d_in):
+    """One row with n entries in a hidden layer of 47 columns: the block finishes the row and re-binarizes it."""
+    n, d_out = 3000, 47
+    rng = np.random.default_rng(79)
+    rp, ci = synth.power_law_graph(n, 30000, 79)
+    src, dst = synth.edge_list(rp, ci)
+    src = np.concatenate([src, np.zeros(n - 1, np.int32)])
+    dst = np.concatenate([dst, np.arange(1, n, dtype=np.int32)])
+    g = oracle.normalize_adjacency(n, src, dst)
+    H = rng.standard_normal((n, d_in)).astype(np.float32)
+    W = (rng.standard_normal((d_in, d_out)) * 0.1).astype(np.float32)
+    W2 = rng.standard_normal((d_out, 4)).astype(np.float32)
+    t = oracle.layer_forward(g, oracle.Layer(W), H)
+    nshift, nscale = oracle.col_stats(t.H_out)
+    Fn, beta_n = oracle.binarize_rows(t.H_out, nshift, nscale)
+    ctx.set_option(B.OPT_ZETA_FORMAT, fmt)
+    G = device_graph(B, g)
+    layer = B.make_layer(d_in, d_out, bits_to_dev(t.bitsT), dev(t.alpha))
+    nxt = B.make_layer(d_out, 4, bits_to_dev(oracle.pack_cols(oracle.binarize_cols(W2)[0])), dev(np.ones(4, np.float32)),
+                       dev(nshift), dev(nscale))
+    try:
+        for thr in (0, 8, 100000):
+            ctx.set_option(B.OPT_LONG_ROW, thr)
+            out = ctx.layer_forward(G, layer, bits_to_dev(t.bits), dev(t.beta), want_h=True, next_layer=nxt)
+            ctx.sync_check()
+            assert_close(out["h"], t.H_out, "H' (threshold %d)" % thr)
+            flips, bad, total = flip_report(bits_from_dev(out["next_bits"]), Fn, t.H_out, nshift)
+            assert bad == 0 and flips <= max(2, total // 2000)
+            nb = bits_from_dev(out["next_bits"])
+            assert (nb[:, 1] >> 15 == 0).all() and (nb[:, 2:] == 0).all()
+            np.testing.assert_allclose(out["next_beta"].cpu().numpy(), beta_n, rtol=RTOL, atol=ATOL)
+    finally:
+        ctx.set_option(B.OPT_LONG_ROW, 0)
+
+
 @pytest.mark.parametrize("d_out", [256, 47])
 def test_half_dot_bytes_hub_row_split_across_the_block(ctx, B, d_out):
     """One row with n entries under half-dot bytes: slices of a long row hand back reconstructed partial sums."""
