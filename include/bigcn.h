@@ -96,7 +96,7 @@ enum {
      * memory as the swizzled A operand, the digits of the edge weights are the B operand, the digit sums are read back
      * from tensor memory once per row segment; graphs of fewer than 2^31 stored entries, otherwise the FMA stream
      * runs).  The FMA stream is the default because it measured fastest (5.7-5.9 / 5.9-6.1 ms against 8.0 / 8.3 ms
-     * for 2 and 6.3 / 6.7 ms for 3 on the two 256-column layers of a 2.4 M-node, 126 M-entry graph). */
+     * for 2 and 6.0 / 6.5 ms for 3 on the two 256-column layers of a 2.4 M-node, 126 M-entry graph). */
     BIGCN_OPT_BYTE_AGGREGATION = 4
 };
 

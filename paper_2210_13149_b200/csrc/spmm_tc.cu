@@ -22,15 +22,21 @@
 // values and per-source factors (beta_k, with the first feature sign for half-dot bytes) through shared-memory rings
 // with asynchronous copies issued several loop iterations ahead, cuts the entries into chunks, derives the segment
 // scales, digits and -- for half-dot bytes -- the per-segment weight sums (as exact integer sums of the q_e, so that
-// they match the products digit for digit), and publishes a chunk slot (mbarrier).  The consumers (a thread owns one
+// they match the products digit for digit), and publishes a chunk slot.  The consumers (a thread owns one
 // tensor-memory lane = output columns t and 128 + t) copy the rows of chunk i + 2 into the operand stage the products
 // of chunk i have released -- the copies report to the stage's mbarrier when they have landed, nobody waits for them
 // but the issuer -- and read back chunk i; the issuer's one thread issues the products of a chunk as soon as it is
 // published, its rows have landed and its accumulator stage has been read back.
 // Two operand stages (32 KB), two accumulator stages (128 tensor-memory columns), four chunk slots per block; four
 // blocks per multiprocessor (what bounds the kernel is the latency of each block's chain of dependent steps per chunk,
-// so the number of blocks that fit counts for more than the depth of one block's pipeline).  Every wait on an mbarrier is bounded: if one runs out the block raises a flag (reported
-// by bigcn_sync_check), the consumers agree on leaving at their next named barrier, the tensor memory is freed.
+// so the number of blocks that fit counts for more than the depth of one block's pipeline).
+// Hand-offs.  Between warps -- chunk published (producer -> consumers, producer -> issuer), chunk read back (consumers
+// -> producer), accumulator stage read back (consumers -> issuer) -- through named barriers: the side that hands over
+// arrives, the side that takes over syncs (15 of the block's 16 barriers; a hop measured 50 cycles against 190 through
+// an mbarrier).  Where an asynchronous unit reports -- the row copies, tcgen05.commit -- through mbarriers, and every
+// wait on those is bounded: if one runs out the block raises a flag (reported by bigcn_sync_check) and from then on
+// every role only passes its barriers, without copies' results or products, until the stream of chunks has ended;
+// nobody is left waiting, the tensor memory is freed.
 #include <algorithm>
 
 #include "bigcn_internal.cuh"
@@ -84,17 +90,13 @@ constexpr int kOffBetaPart = kOffSlots + kSlots * (int)sizeof(ChunkSlot);       
 constexpr int kOffBetaRow = kOffBetaPart + 2 * kSegMax * 8 * 4;                    // int [2][kSegMax]
 constexpr int kOffEntRing = kOffBetaRow + 2 * kSegMax * 4;                         // producer: int32 / float / float [kEntRing]
 constexpr int kOffRowRing = kOffEntRing + 3 * kEntRing * 4;                        // producer: int64 [kRowRing]
-constexpr int kOffBars = kOffRowRing + kRowRing * 8;                               // uint64: published [kSlots], read back [kSlots], products done [2], accumulators read [2], rows landed [kAStages]
-constexpr int kOffMisc = kOffBars + (2 * kSlots + 4 + kAStages) * 8;               // uint32 tmem base, int abort
+constexpr int kOffBars = kOffRowRing + kRowRing * 8;                               // uint64 mbarriers: products done [2], rows landed [kAStages]
+constexpr int kOffMisc = kOffBars + (2 + kAStages) * 8;               // uint32 tmem base, int abort
 constexpr int kSmemBytes = kOffMisc + 16 + 1024;                                   // + slack for the alignment
 
 __device__ __forceinline__ void mbar_init(uint64_t* bar, int count)
 {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar)
-{
-    asm volatile("{\n.reg .b64 st;\nmbarrier.arrive.shared::cta.b64 st, [%0];\n}\n" ::"r"(smem_u32(bar)) : "memory");
 }
 // Bounded wait that also gives up when another thread of the block has raised `abort`.  No sleep between tries: the
 // try itself parks the thread (measured: next to no failed tries), and every sleep added to it showed up in the chain
@@ -112,6 +114,19 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         *abort = 1;
     }
     return done != 0;
+}
+// Hand-offs between the roles go through named barriers (a round trip through two of them was measured at 100 cycles,
+// through two mbarriers at 350-400): the side that hands over arrives, the side that takes over syncs; `count` is the
+// number of threads of both sides.  Whole warps execute these.
+constexpr int kBarPR = 2, kBarPI = 2 + kSlots, kBarRP = 2 + 2 * kSlots, kBarRI = 2 + 3 * kSlots;   // + slot, + slot, + slot, + stage
+static_assert(kBarRI + 2 <= 16, "named barriers");
+__device__ __forceinline__ void bar_arrive(int id, int count)
+{
+    asm volatile("barrier.cta.arrive.aligned %0, %1;\n" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void bar_sync(int id, int count)
+{
+    asm volatile("barrier.cta.sync.aligned %0, %1;\n" ::"r"(id), "r"(count) : "memory");
 }
 // All consumers meet; returns the OR of their `bad` flags.
 __device__ __forceinline__ bool consumers_sync_or(bool bad)
@@ -172,9 +187,6 @@ template <bool kHalf>
 __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, volatile int* abort)
 {
     const int lane = threadIdx.x & 31;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sm + kOffBars);
-    uint64_t* prep_full = bars;
-    uint64_t* prep_empty = bars + kSlots;
     int32_t* col_ring = reinterpret_cast<int32_t*>(sm + kOffEntRing);
     float* val_ring = reinterpret_cast<float*>(sm + kOffEntRing + kEntRing * 4);
     float* nw_ring = reinterpret_cast<float*>(sm + kOffEntRing + kEntRing * 8);
@@ -236,13 +248,14 @@ __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, vo
         const bool finished = r == nrows;
         if (!finished && !(min(r + kSegMax + 1, nrows + 1) <= ri_done && min(e + kChunk, total) <= ni_done)) continue;
         const int slot_i = (int)(k % kSlots);
-        if (!mbar_wait(&prep_empty[slot_i], ((k / kSlots) & 1u) ^ 1u, abort)) break;
+        if (k >= kSlots) bar_sync(kBarRP + slot_i, kConsumers + 32);      // the consumers have read chunk k - kSlots
         ChunkSlot* slot = reinterpret_cast<ChunkSlot*>(sm + kOffSlots) + slot_i;
         unsigned char* Bs = sm + kOffB + slot_i * kBSlotBytes;
         if (finished) {                                       // end of the stream
             if (lane == 0) slot->n_ent = -1;
             __syncwarp();
-            if (lane == 0) mbar_arrive(&prep_full[slot_i]);
+            bar_arrive(kBarPR + slot_i, kConsumers + 32);
+            bar_arrive(kBarPI + slot_i, 64);
             break;
         }
         // segments: the rows r .. r + 7 as far as they start before the chunk's end (or are empty and sit at it)
@@ -333,7 +346,8 @@ __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, vo
         }
         tc::fence_async_smem();                               // the digits are read by the tensor core (async proxy)
         __syncwarp();
-        if (lane == 0) mbar_arrive(&prep_full[slot_i]);
+        bar_arrive(kBarPR + slot_i, kConsumers + 32);
+        bar_arrive(kBarPI + slot_i, 64);
         ++k;
     }
     asm volatile("cp.async.wait_all;\n" ::: "memory");
@@ -355,21 +369,20 @@ __device__ __forceinline__ void issuer(const SpmmDev& p, unsigned char* sm, vola
 {
     const int lane = threadIdx.x & 31;
     uint64_t* bars = reinterpret_cast<uint64_t*>(sm + kOffBars);
-    uint64_t* prep_full = bars;
-    uint64_t* mma_done = bars + 2 * kSlots;
-    uint64_t* tmem_empty = bars + 2 * kSlots + 2;
-    uint64_t* a_full = bars + 2 * kSlots + 4;
+    uint64_t* mma_done = bars;
+    uint64_t* a_full = bars + 2;
     const ChunkSlot* slots = reinterpret_cast<const ChunkSlot*>(sm + kOffSlots);
     const uint32_t a_base = smem_u32(sm + kOffA), b_base = smem_u32(sm + kOffB);
     // instruction descriptor: D = s32, A = B = s8, both M/N-major, N = 32, M = 128
     const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(kN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
     for (uint32_t c = 0;; ++c) {
-        if (!wait_bcast(&prep_full[c % kSlots], (c / kSlots) & 1u, abort, lane)) return;
+        bar_sync(kBarPI + (int)(c % kSlots), 64);             // chunk c is published
         const ChunkSlot* slot = slots + (c % kSlots);
         const int n_ent = slot->n_ent;
         if (n_ent < 0) return;                                // end of the stream
-        if (!wait_bcast(&a_full[c % kAStages], (c / kAStages) & 1u, abort, lane)) return;
-        if (c >= 2 && !wait_bcast(&tmem_empty[c & 1u], ((c >> 1) - 1u) & 1u, abort, lane)) return;
+        // a wait that runs out raises the block's flag; every role then keeps passing its barriers without work
+        wait_bcast(&a_full[c % kAStages], (c / kAStages) & 1u, abort, lane);
+        if (c >= 2) bar_sync(kBarRI + (int)(c & 1u), kConsumers + 32);     // the accumulator stage has been read back
         if (lane == 0) {
             tc::fence_async_smem();                           // the copied rows become visible to the tensor core
             tc::fence_after_sync();
@@ -406,11 +419,8 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;      // warp = tensor-memory lane quarter
     uint64_t* bars = reinterpret_cast<uint64_t*>(sm + kOffBars);
-    uint64_t* prep_full = bars;
-    uint64_t* prep_empty = bars + kSlots;
-    uint64_t* mma_done = bars + 2 * kSlots;
-    uint64_t* tmem_empty = bars + 2 * kSlots + 2;
-    uint64_t* a_full = bars + 2 * kSlots + 4;
+    uint64_t* mma_done = bars;
+    uint64_t* a_full = bars + 2;
     ChunkSlot* slots = reinterpret_cast<ChunkSlot*>(sm + kOffSlots);
     float* beta_part = reinterpret_cast<float*>(sm + kOffBetaPart);
     int* beta_row = reinterpret_cast<int*>(sm + kOffBetaRow);
@@ -462,28 +472,23 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
     bool bad = false;
     // prologue: the rows of the first kAStages chunks (only one thread polls; the others wait at the named barrier)
     for (uint32_t c = 0; c < kAStages && end_idx == 0xffffffffu && !bad; ++c) {
-        if (tid == 0 && !mbar_wait(&prep_full[c % kSlots], (c / kSlots) & 1u, abort)) bad = true;
-        bad = consumers_sync_or(bad);
-        if (!bad) {
-            if (slots[c % kSlots].n_ent < 0) end_idx = c;
-            else gather(c);
-        }
+        bar_sync(kBarPR + (int)(c % kSlots), kConsumers + 32);
+        if (slots[c % kSlots].n_ent < 0) end_idx = c;
+        else gather(c);
     }
 
     float acc[2] = {0.f, 0.f};                                // the open row: this thread's two column sums
     float rs = 0.f, rg = 0.f;                                 // and the row's weight sums (half-dot bytes)
     int prev_nseg = 0;                                        // segments of chunk i - 1
-    for (uint32_t i = 0; !bad; ++i) {
+    for (uint32_t i = 0;; ++i) {
         const bool has_cur = i < end_idx, need_next = end_idx == 0xffffffffu;
-        if (tid == 0) {
-            if (has_cur && !mbar_wait(&mma_done[i & 1u], (i >> 1) & 1u, abort)) bad = true;
-            if (!bad && need_next && !mbar_wait(&prep_full[(i + kAStages) % kSlots], ((i + kAStages) / kSlots) & 1u, abort)) bad = true;
-        }
+        if (need_next) bar_sync(kBarPR + (int)((i + kAStages) % kSlots), kConsumers + 32);   // chunk i + kAStages is published
+        if (tid == 0 && has_cur && !mbar_wait(&mma_done[i & 1u], (i >> 1) & 1u, abort)) bad = true;
         tc::fence_before_sync();
-        if (consumers_sync_or(bad)) break;
+        bad = consumers_sync_or(bad || *abort != 0);          // from here on the block only passes its barriers
         tc::fence_after_sync();
         // beta of the rows that ended in chunk i - 1: the four warps' partial sums in warp order
-        if (p.next_bits && tid < prev_nseg) {
+        if (!bad && p.next_bits && tid < prev_nseg) {
             const int par = (int)((i - 1u) & 1u);
             const int row = beta_row[par * kSegMax + tid];
             if (row >= 0) {
@@ -500,7 +505,7 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
         // read back chunk i: the four digit sums of every segment, both operands
         const ChunkSlot* slot = slots + (i % kSlots);
         const int par = (int)(i & 1u);
-        const int nseg = slot->nseg;
+        const int nseg = bad ? 0 : slot->nseg;
         prev_nseg = nseg;
         const uint32_t t_addr = tmem_base + ((uint32_t)(32 * warp) << 16) + (uint32_t)(par * 64);
         for (int s = 0; s < nseg; ++s) {                       // a run-time loop (uniform over the readers): small code, the same for every segment
@@ -552,10 +557,8 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
         }
         tc::fence_before_sync();
         __syncwarp();
-        if (lane == 0) {
-            mbar_arrive(&tmem_empty[par]);
-            mbar_arrive(&prep_empty[i % kSlots]);
-        }
+        bar_arrive(kBarRI + par, kConsumers + 32);
+        bar_arrive(kBarRP + (int)(i % kSlots), kConsumers + 32);
     }
     asm volatile("cp.async.wait_all;\n" ::: "memory");        // nothing of this thread is in flight when the block leaves
 }
@@ -572,15 +575,8 @@ spmm_tc_kernel(const SpmmDev p)
     const int warp = threadIdx.x >> 5;
     if (warp == 0) tc::tmem_alloc(tmem_slot, kTmemCols);
     if (threadIdx.x == 32) {
-        for (int i = 0; i < kSlots; ++i) {
-            mbar_init(&bars[i], 1);                           // chunk published: the producer's lane 0
-            mbar_init(&bars[kSlots + i], kConsumers / 32);   // chunk read back: one arrival per consumer warp
-        }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(&bars[2 * kSlots + i], 1);              // products done: tcgen05.commit
-            mbar_init(&bars[2 * kSlots + 2 + i], kConsumers / 32);   // accumulator stage read back: one arrival per consumer warp
-        }
-        for (int i = 0; i < kAStages; ++i) mbar_init(&bars[2 * kSlots + 4 + i], kConsumers);   // rows landed: every consumer thread's copies
+        for (int i = 0; i < 2; ++i) mbar_init(&bars[i], 1);                        // products done: tcgen05.commit
+        for (int i = 0; i < kAStages; ++i) mbar_init(&bars[2 + i], kConsumers);   // rows landed: every consumer thread's copies
         *abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
