@@ -65,7 +65,9 @@ enum {
     /* Storage of the rescaled contraction zeta between the bit-GEMM and the aggregation.
      * 0 = choose per layer (default: for 129..256 output columns, where the aggregation streams 256-byte
      *     rows, and for 33..64 output columns of a layer whose result is only written out as fp32 (no next
-     *     layer), 3 when d_in <= 127 and 5 when 128 <= d_in <= 256 and the layer has at least 2^20 outputs;
+     *     layer) or of a hidden layer on a graph whose rows average at least 8 stored entries (the aggregation
+     *     then streams one stored entry per lane), 3 when d_in <= 127 and 5 when 128 <= d_in <= 256 and the
+     *     layer has at least 2^20 outputs;
      *     otherwise 4 when d_in <= 2048, else 2);
      * 1 = fp32 zeta_ij = (beta_i alpha_j) dot_ij, exactly Eq. "cdot-op";
      * 2 = the integer dot products as int16, with beta folded into the edge weights and alpha
@@ -74,7 +76,7 @@ enum {
      * 4 = as 2 but the integers held as fp16, which is exact for |dot| <= 2048 (layers with
      *     d_in <= 2048 only; others fall back to 2);
      * 5 = signed bytes for 128 <= d_in <= 256 and up to 256 output columns (other layers as 0; the automatic
-     *     choice takes it for 129..256 output columns, and for 33..64 of a last layer): the byte is
+     *     choice takes it for 129..256 output columns, and for 33..64 as described under 0): the byte is
      *     s = (dot' - 1) / 2, dot' the dot without its first position when d_in is even (so that dot' is
      *     odd and s fits a byte exactly); the aggregation adds back sum_k w_k (1 + f_k0 b_0j), two per-row
      *     sums that ride along with the edge weights.  Exact in the integers; on the tensor-core contraction. */
