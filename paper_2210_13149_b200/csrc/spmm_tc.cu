@@ -38,6 +38,7 @@
 // every role only passes its barriers, without copies' results or products, until the stream of chunks has ended;
 // nobody is left waiting, the tensor memory is freed.
 #include <algorithm>
+#include <cstddef>
 
 #include "bigcn_internal.cuh"
 #include "spmm_dev.cuh"
@@ -69,26 +70,27 @@ __device__ int g_spmm_tc_timeout;               // set when a wait ran out
 
 using tc::smem_u32;
 
+struct SegRec {                                 // one row segment of a chunk
+    float scale;                                // S_s 2^-30
+    float wsum, wsgn;                           // half-dot bytes: sum of the segment's weights, plain and signed by the sources' first feature sign
+    int32_t row_done;                           // the output row if it ends with this segment, else -1
+};
 struct ChunkSlot {
     int32_t cols[kChunk];                       // source node of every entry
+    SegRec seg[kSegMax];
     int32_t n_ent;                              // entries in the chunk (0..64); -1 = end of the stream
     int32_t nseg;
-    int32_t seg_row[kSegMax];                   // output row of a segment
-    int32_t seg_last[kSegMax];                  // 1: the row ends with this segment
-    float seg_scale[kSegMax];                   // S_s 2^-30
-    float seg_wsum[kSegMax];                    // half-dot bytes: sum of the segment's weights, plain and
-    float seg_wsgn[kSegMax];                    // signed by the sources' first feature sign
-    int32_t pad[6];
+    int32_t pad[14];
 };
-static_assert(sizeof(ChunkSlot) == 448, "slot size");
+static_assert(sizeof(ChunkSlot) == 448 && offsetof(ChunkSlot, seg) % 16 == 0, "slot size");
 
 // dynamic shared memory, relative to a 1024-byte aligned base
 constexpr int kOffA = 0;
 constexpr int kOffB = kOffA + kAStages * kAStageBytes;
 constexpr int kOffSlots = kOffB + kSlots * kBSlotBytes;
-constexpr int kOffBetaPart = kOffSlots + kSlots * (int)sizeof(ChunkSlot);          // float [2][kSegMax][8] (one per consumer warp; 4 used)
-constexpr int kOffBetaRow = kOffBetaPart + 2 * kSegMax * 8 * 4;                    // int [2][kSegMax]
-constexpr int kOffEntRing = kOffBetaRow + 2 * kSegMax * 4;                         // producer: int32 / float / float [kEntRing]
+constexpr int kOffBetaPart = kOffSlots + kSlots * (int)sizeof(ChunkSlot);          // float [4][kSegMax][4]: per chunk (index & 3) and segment, one partial sum per consumer warp
+constexpr int kOffBetaRow = kOffBetaPart + 4 * kSegMax * 4 * 4;                    // int [4][kSegMax]: the row that ended with the segment, or -1; [4]: segments of the chunk
+constexpr int kOffEntRing = kOffBetaRow + 4 * kSegMax * 4 + 16;                         // producer: int32 / float / float [kEntRing]
 constexpr int kOffRowRing = kOffEntRing + 3 * kEntRing * 4;                        // producer: int64 [kRowRing]
 constexpr int kOffBars = kOffRowRing + kRowRing * 8;                               // uint64 mbarriers: products done [2], rows landed [kAStages]
 constexpr int kOffMisc = kOffBars + (2 + kAStages) * 8;               // uint32 tmem base, int abort
@@ -305,8 +307,7 @@ __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, vo
         // four balanced base-256 digits of q, one per byte
         const uint32_t dg_a = ((uint32_t)q_a + 0x80808080u) ^ 0x80808080u, dg_b = ((uint32_t)q_b + 0x80808080u) ^ 0x80808080u;
         // row e of the B operand: 32 digit columns = two 16-byte lines (N-major, no swizzle: line l of entry e at e * 16 + l * 1024)
-#pragma unroll
-        for (int l = 0; l < kN / 16; ++l) {
+        for (int l = 0; l < (nseg > 4 ? 2 : 1); ++l) {
             const int wa = (sid_a >> 2) == l ? (sid_a & 3) : -1, wb = (sid_b >> 2) == l ? (sid_b & 3) : -1;
             const uint4 va = make_uint4(wa == 0 ? dg_a : 0u, wa == 1 ? dg_a : 0u, wa == 2 ? dg_a : 0u, wa == 3 ? dg_a : 0u);
             const uint4 vb = make_uint4(wb == 0 ? dg_b : 0u, wb == 1 ? dg_b : 0u, wb == 2 ? dg_b : 0u, wb == 3 ? dg_b : 0u);
@@ -333,13 +334,8 @@ __device__ __forceinline__ void producer(const SpmmDev& p, unsigned char* sm, vo
                 }
             }
         }
-        if (lane < kSegMax) {
-            slot->seg_row[lane] = seg_row;
-            slot->seg_last[lane] = last ? 1 : 0;
-            slot->seg_scale[lane] = my_scale;
-            slot->seg_wsum[lane] = my_wsum;
-            slot->seg_wsgn[lane] = my_wsgn;
-        }
+        if (lane < kSegMax)
+            *reinterpret_cast<float4*>(&slot->seg[lane]) = make_float4(my_scale, my_wsum, my_wsgn, __int_as_float(last ? seg_row : -1));
         if (lane == 0) {
             slot->n_ent = n_ent;
             slot->nseg = nseg;
@@ -364,22 +360,44 @@ __device__ __forceinline__ bool wait_bcast(uint64_t* bar, uint32_t parity, volat
 }
 
 // Chunk after chunk: once the chunk is published, its rows have landed (the consumers' copies report to the stage's
-// mbarrier) and its accumulator stage has been read back (chunk c - 2), one thread issues the products.
+// mbarrier) and its accumulator stage has been read back (chunk c - 2), one thread issues the products.  The warp
+// then finishes beta of the rows that ended in chunk c - 2, whose read-back it has just waited for: the four consumer
+// warps' partial sums, in warp order (the partials sit in four buffers, chunk index & 3, so that the consumers, who
+// cannot be more than two chunks ahead of this warp, never write the one being read here).
 __device__ __forceinline__ void issuer(const SpmmDev& p, unsigned char* sm, volatile int* abort, uint32_t tmem_base)
 {
     const int lane = threadIdx.x & 31;
+    const float* beta_part = reinterpret_cast<const float*>(sm + kOffBetaPart);
+    const int* beta_row = reinterpret_cast<const int*>(sm + kOffBetaRow);
+    auto finish_beta = [&](uint32_t d) {
+        if (!p.next_bits || *abort) return;
+        const int bq = (int)(d & 3u);
+        if (lane < beta_row[4 * kSegMax + bq]) {
+            const int row = beta_row[bq * kSegMax + lane];
+            if (row >= 0) {
+                const float4 bp = *reinterpret_cast<const float4*>(beta_part + (bq * kSegMax + lane) * 4);
+                p.next_beta[row] = (((bp.x + bp.y) + bp.z) + bp.w) * p.inv_d_out;
+            }
+        }
+    };
     uint64_t* bars = reinterpret_cast<uint64_t*>(sm + kOffBars);
     uint64_t* mma_done = bars;
     uint64_t* a_full = bars + 2;
     const ChunkSlot* slots = reinterpret_cast<const ChunkSlot*>(sm + kOffSlots);
     const uint32_t a_base = smem_u32(sm + kOffA), b_base = smem_u32(sm + kOffB);
     // instruction descriptor: D = s32, A = B = s8, both M/N-major, N = 32, M = 128
-    const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(kN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+    const uint32_t idesc0 = (2u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(128 >> 4) << 24);
     for (uint32_t c = 0;; ++c) {
         bar_sync(kBarPI + (int)(c % kSlots), 64);             // chunk c is published
         const ChunkSlot* slot = slots + (c % kSlots);
         const int n_ent = slot->n_ent;
-        if (n_ent < 0) return;                                // end of the stream
+        if (n_ent < 0) {                                      // end of the stream: the last two chunks' rows
+            for (uint32_t d = c >= 2 ? c - 2 : 0; d < c; ++d) {
+                bar_sync(kBarRI + (int)(d & 1u), kConsumers + 32);
+                finish_beta(d);
+            }
+            return;
+        }
         // a wait that runs out raises the block's flag; every role then keeps passing its barriers without work
         wait_bcast(&a_full[c % kAStages], (c / kAStages) & 1u, abort, lane);
         if (c >= 2) bar_sync(kBarRI + (int)(c & 1u), kConsumers + 32);     // the accumulator stage has been read back
@@ -387,6 +405,7 @@ __device__ __forceinline__ void issuer(const SpmmDev& p, unsigned char* sm, vola
             tc::fence_async_smem();                           // the copied rows become visible to the tensor core
             tc::fence_after_sync();
             const int ksteps = max(1, (n_ent + 31) >> 5);
+            const uint32_t idesc = idesc0 | ((uint32_t)((slot->nseg > 4 ? 32 : 16) >> 3) << 17);
             const uint32_t a_stage = a_base + (c % kAStages) * kAStageBytes;
             const uint32_t b_slot = b_base + (c % kSlots) * kBSlotBytes;
             for (int hh = 0; hh < 2; ++hh)
@@ -401,6 +420,7 @@ __device__ __forceinline__ void issuer(const SpmmDev& p, unsigned char* sm, vola
             tc::commit_to(&mma_done[c & 1u]);
         }
         __syncwarp();
+        if (c >= 2) finish_beta(c - 2);
     }
 }
 
@@ -479,7 +499,6 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
 
     float acc[2] = {0.f, 0.f};                                // the open row: this thread's two column sums
     float rs = 0.f, rg = 0.f;                                 // and the row's weight sums (half-dot bytes)
-    int prev_nseg = 0;                                        // segments of chunk i - 1
     for (uint32_t i = 0;; ++i) {
         const bool has_cur = i < end_idx, need_next = end_idx == 0xffffffffu;
         if (need_next) bar_sync(kBarPR + (int)((i + kAStages) % kSlots), kConsumers + 32);   // chunk i + kAStages is published
@@ -487,15 +506,6 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
         tc::fence_before_sync();
         bad = consumers_sync_or(bad || *abort != 0);          // from here on the block only passes its barriers
         tc::fence_after_sync();
-        // beta of the rows that ended in chunk i - 1: the four warps' partial sums in warp order
-        if (!bad && p.next_bits && tid < prev_nseg) {
-            const int par = (int)((i - 1u) & 1u);
-            const int row = beta_row[par * kSegMax + tid];
-            if (row >= 0) {
-                const float* bp = beta_part + (par * kSegMax + tid) * 8;
-                p.next_beta[row] = (((bp[0] + bp[1]) + bp[2]) + bp[3]) * p.inv_d_out;
-            }
-        }
         if (!has_cur) break;
         // the rows of chunk i + kAStages go into the stage the products of chunk i have just released
         if (need_next) {
@@ -506,7 +516,8 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
         const ChunkSlot* slot = slots + (i % kSlots);
         const int par = (int)(i & 1u);
         const int nseg = bad ? 0 : slot->nseg;
-        prev_nseg = nseg;
+        const int bq = (int)(i & 3u);                         // beta partials of this chunk: finished by the issuer warp
+        if (tid == 0) beta_row[4 * kSegMax + bq] = nseg;
         const uint32_t t_addr = tmem_base + ((uint32_t)(32 * warp) << 16) + (uint32_t)(par * 64);
         for (int s = 0; s < nseg; ++s) {                       // a run-time loop (uniform over the readers): small code, the same for every segment
             int row_done = -1;
@@ -517,16 +528,16 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
                 asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];\n"
                              : "=r"(c0), "=r"(c1), "=r"(c2), "=r"(c3) : "r"(t_addr + 32 + 4 * s) : "memory");
                 asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-                const float sc = slot->seg_scale[s];
-                acc[0] = fmaf(digits_to_float(a0, a1, a2, a3), sc, acc[0]);
-                acc[1] = fmaf(digits_to_float(c0, c1, c2, c3), sc, acc[1]);
+                const float4 rec = *reinterpret_cast<const float4*>(&slot->seg[s]);
+                acc[0] = fmaf(digits_to_float(a0, a1, a2, a3), rec.x, acc[0]);
+                acc[1] = fmaf(digits_to_float(c0, c1, c2, c3), rec.x, acc[1]);
                 if constexpr (kHalf) {
-                    rs += slot->seg_wsum[s];
-                    rg += slot->seg_wsgn[s];
+                    rs += rec.y;
+                    rg += rec.z;
                 }
-                if (slot->seg_last[s]) row_done = slot->seg_row[s];
+                row_done = __float_as_int(rec.w);
             }
-            if (tid == 0) beta_row[par * kSegMax + s] = row_done;
+            if (tid == 0) beta_row[bq * kSegMax + s] = row_done;
             if (row_done >= 0) {
                 const int64_t row = row_done;
                 float l1 = 0.f;
@@ -549,7 +560,7 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
                 if (p.next_bits) {
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) l1 += __shfl_xor_sync(0xffffffffu, l1, o);
-                    if (lane == 0) beta_part[(par * kSegMax + s) * 8 + warp] = l1;
+                    if (lane == 0) beta_part[(bq * kSegMax + s) * 4 + warp] = l1;
                 }
                 rs = 0.f;
                 rg = 0.f;
