@@ -434,7 +434,8 @@ __device__ __forceinline__ float digits_to_float(uint32_t d0, uint32_t d1, uint3
     return fmaf((float)hi, 65536.f, (float)lo);
 }
 
-template <bool kHalf>
+// kBitsOnly: the launch wants only the next layer's sign bits and beta (no fp32 output, nothing added to the rows)
+template <bool kHalf, bool kBitsOnly>
 __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, volatile int* abort, uint32_t tmem_base)
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;      // warp = tensor-memory lane quarter
@@ -547,9 +548,11 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
                     if constexpr (kHalf) t = fmaf(2.f, t, fmaf(b0[h], rg, rs));   // sum_k w_k dot_kj = 2 acc_j + wsum + b0_j wsgn
                     float x = t * alpha[h];
                     const int col = 128 * h + tid;
-                    if (p.add && col_in[h]) x += __ldg(p.add + row * p.ld_add + col);
-                    if (p.h_out && col_in[h]) p.h_out[row * p.ldh + col] = x;
-                    if (p.next_bits) {
+                    if constexpr (!kBitsOnly) {
+                        if (p.add && col_in[h]) x += __ldg(p.add + row * p.ld_add + col);
+                        if (p.h_out && col_in[h]) p.h_out[row * p.ldh + col] = x;
+                    }
+                    if (kBitsOnly || p.next_bits) {
                         const float xh = __fmul_rn(__fsub_rn(x, shift[h]), scale[h]);
                         const uint32_t word = __ballot_sync(0xffffffffu, col_in[h] && xh >= 0.f);
                         if (lane == 0 && 4 * h + warp < p.next_stride) p.next_bits[row * p.next_stride + 4 * h + warp] = word;
@@ -557,7 +560,7 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
                     }
                     acc[h] = 0.f;
                 }
-                if (p.next_bits) {
+                if (kBitsOnly || p.next_bits) {
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) l1 += __shfl_xor_sync(0xffffffffu, l1, o);
                     if (lane == 0) beta_part[(bq * kSegMax + s) * 4 + warp] = l1;
@@ -574,7 +577,7 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
     asm volatile("cp.async.wait_all;\n" ::: "memory");        // nothing of this thread is in flight when the block leaves
 }
 
-template <bool kHalf>
+template <bool kHalf, bool kBitsOnly>
 __global__ void __launch_bounds__(kThreads, 4)
 spmm_tc_kernel(const SpmmDev p)
 {
@@ -597,7 +600,7 @@ spmm_tc_kernel(const SpmmDev p)
     const uint32_t tmem_base = *tmem_slot;
     if (warp == kConsumers / 32) producer<kHalf>(p, sm, abort);
     else if (warp == kConsumers / 32 + 1) issuer(p, sm, abort, tmem_base);
-    else consumers<kHalf>(p, sm, abort, tmem_base);
+    else consumers<kHalf, kBitsOnly>(p, sm, abort, tmem_base);
     tc::fence_before_sync();
     __syncthreads();
     if (warp == 0) tc::tmem_free(tmem_base, kTmemCols);
@@ -613,16 +616,18 @@ bool spmm_tc_covers(const SpmmDev& p)
 
 cudaError_t launch_spmm_tc(cudaStream_t s, const SpmmDev& p)
 {
-    cudaError_t e;
-    if (p.half_dots) e = cudaFuncSetAttribute(spmm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    else e = cudaFuncSetAttribute(spmm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return e;
     // one wave of resident blocks (four per multiprocessor: 4 x 128 = all 512 tensor-memory columns); the rows are
     // split over them by cost inside the kernel
     const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>(ceil_div(p.n, 64), (int64_t)sm_count() * 4));
-    if (p.half_dots) spmm_tc_kernel<true><<<grid, kThreads, kSmemBytes, s>>>(p);
-    else spmm_tc_kernel<false><<<grid, kThreads, kSmemBytes, s>>>(p);
-    return cudaGetLastError();
+    const bool bits_only = p.next_bits && !p.h_out && !p.add;
+    auto launch = [&](auto kernel) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+        kernel<<<grid, kThreads, kSmemBytes, s>>>(p);
+        return cudaGetLastError();
+    };
+    if (p.half_dots) return bits_only ? launch(spmm_tc_kernel<true, true>) : launch(spmm_tc_kernel<true, false>);
+    return bits_only ? launch(spmm_tc_kernel<false, true>) : launch(spmm_tc_kernel<false, false>);
 }
 
 int spmm_tc_timeouts()
