@@ -383,21 +383,23 @@ def run_ours(args):
                 extras["spmm_fp16_rows_ms"] = "failed: %r" % (exc,)
             finally:
                 ctx.set_option(binding.OPT_ZETA_FORMAT, 0)
-        # byte rows aggregated as integer products on the tensor cores (the library's other path), for comparison
+        # byte rows aggregated by the library's other paths, for comparison: the fp32 FMA stream (1) and integer
+        # products on mma.sync (2); the default for a hidden layer of 129..256 byte columns is tcgen05 products (3)
         if args.zeta_format == 0 and args.byte_aggregation == 0:
-            try:
-                ctx.set_option(binding.OPT_BYTE_AGGREGATION, 2)
-                alt = [[] for _ in range(L)]
-                for k in range(3 + min(args.steps, 5)):
-                    _, st = ctx.forward(G, layers, X, logits, stats=True)
-                    if k >= 3:
-                        for l in range(L):
-                            alt[l].append(st.ms_spmm[l])
-                extras["spmm_integer_products_ms"] = [sum(v) / len(v) for v in alt]
-            except Exception as exc:
-                extras["spmm_integer_products_ms"] = "failed: %r" % (exc,)
-            finally:
-                ctx.set_option(binding.OPT_BYTE_AGGREGATION, 0)
+            for opt, key in ((1, "spmm_fma_stream_ms"), (2, "spmm_integer_products_ms")):
+                try:
+                    ctx.set_option(binding.OPT_BYTE_AGGREGATION, opt)
+                    alt = [[] for _ in range(L)]
+                    for k in range(3 + min(args.steps, 5)):
+                        _, st = ctx.forward(G, layers, X, logits, stats=True)
+                        if k >= 3:
+                            for l in range(L):
+                                alt[l].append(st.ms_spmm[l])
+                    extras[key] = [sum(v) / len(v) for v in alt]
+                except Exception as exc:
+                    extras[key] = "failed: %r" % (exc,)
+                finally:
+                    ctx.set_option(binding.OPT_BYTE_AGGREGATION, 0)
         # the same contraction on the XOR / bit-count pipe (the library's other path), for comparison
         try:
             ctx.set_option(binding.OPT_CONTRACTION, 1)
@@ -544,7 +546,12 @@ def run_ours(args):
         out_bytes = n * dims[l + 1] * 4.0 if last else n * (binding.packed_stride_words(dims[l + 1]) * 4.0 + 4.0)
         lower, upper, expected = spmm_bytes_model(n, nnz, ldz * elt, out_bytes, deg_cum)
         t = spmm_ms[l] * 1e-3
-        kernels["spmm_l%d" % l] = {"ms": spmm_ms[l], "GBps_cached_model": expected / t / 1e9,
+        # the library's rule for the aggregation kernel: tcgen05 products for a hidden layer (only bits and beta wanted) of
+        # 129..256 byte columns on a graph whose rows average at least 8 stored entries, unless another path is asked for
+        on_tc_agg = (elt == 1 and 128 < dims[l + 1] <= 256 and not last and nnz < (1 << 31)
+                     and (args.byte_aggregation == 3 or (args.byte_aggregation == 0 and nnz >= 8 * n)))
+        agg_name = "spmm_tc_kernel" if on_tc_agg else ("spmm_lane_kernel" if (last and elt == 1 and 32 < dims[l + 1] <= 64 and nnz >= 8 * n) else "spmm_kernel")
+        kernels["spmm_l%d" % l] = {"ms": spmm_ms[l], "kernel": agg_name, "GBps_cached_model": expected / t / 1e9,
                                    "GBps_lower_model": lower / t / 1e9, "GBps_no_reuse_model": upper / t / 1e9,
                                    "bytes_cached_model": expected, "row_bytes": ldz * elt, "zeta_format": {1: "f32", 2: "i16", 3: "i8", 4: "f16", 5: "i8h"}[f]}
         ops = 2.0 * n * dims[l] * dims[l + 1]
@@ -565,14 +572,16 @@ def run_ours(args):
     kernels["pack_features"] = {"ms": pack_ms, "GBps": pack_bytes / (pack_ms * 1e-3) / 1e9,
                                 "frac_of_hbm_peak": pack_bytes / (pack_ms * 1e-3) / 1e9 / peak}
     achieved = kernels["spmm_l%d" % dom]["GBps_cached_model"]
-    dom_key = "spmm_kernel/%s/%s/l%d" % (spec.name, kernels["spmm_l%d" % dom]["zeta_format"], dom)
-    roofline = {"kernel": "spmm_kernel (layer %d: %d -> %d columns)" % (dom, dims[dom], dims[dom + 1]),
+    dom_name = kernels["spmm_l%d" % dom]["kernel"]
+    dom_key = "%s/%s/%s/l%d" % (dom_name, spec.name, kernels["spmm_l%d" % dom]["zeta_format"], dom)
+    roofline = {"kernel": "%s (layer %d: %d -> %d columns)" % (dom_name, dom, dims[dom], dims[dom + 1]),
                 "bound": "hbm", "achieved": achieved, "peak": peak, "peak_kind": "%s copy bandwidth" % peak_kind,
                 "unit": "GB/s", "frac": achieved / peak, "traffic": traffic_record(dom_key),
                 "algorithmic_bytes": kernels["spmm_l%d" % dom]["bytes_cached_model"],
                 "note": "byte rows (i8 / i8h) halve the DRAM traffic of the 256-column aggregations and leave them bound by "
-                        "instruction issue, not HBM; with fp16 rows (--zeta-format 4) the same layer is HBM-bound: see "
-                        "extras.spmm_fp16_rows_ms and kernels.*",
+                        "the per-chunk chain of hand-offs (tcgen05 products, the default) or by instruction issue (the fp32 "
+                        "FMA stream, extras.spmm_fma_stream_ms), not HBM; with fp16 rows (--zeta-format 4) the same layer is "
+                        "HBM-bound: see extras.spmm_fp16_rows_ms and kernels.*",
                 "model": "per launch: 8 B per stored entry (column, value) + rowptr + node weights + output + every "
                          "operand row once + one operand row per further stored entry whose source is not among the "
                          "highest-degree rows an ideal 126 MB cache would hold"}

@@ -88,17 +88,21 @@ enum {
      * d_out <= 256 and at least 2^20 outputs, on the XOR / bit-count pipe otherwise; 1 = always on the
      * XOR / bit-count pipe; 2 = tensor cores for every layer with d_in <= 256 and d_out <= 256. */
     BIGCN_OPT_CONTRACTION = 3,
-    /* How rows of 129..256 signed bytes (zeta formats 3 and 5) are aggregated.  0 = default and 1: the fp32 FMA
-     * stream (bytes converted to fp32 one by one; with format 5 this stream takes the edge values as non-negative,
-     * as those of the normalized adjacency are); 2 = as exact integer products on the tensor cores (mma.sync
-     * s8 x s8 -> s32: the edge weights of up to 32 stored entries of a row in 28..31-bit fixed point against a
-     * common power of two, split into four signed base-256 digits; the digit sums recombined in fp32 when the row
-     * ends; edge values of either sign); 3 = the same fixed-point digits on the 5th-generation tensor cores
-     * (tcgen05.mma kind::i8: the gathered rows of 64 stored entries go by asynchronous copies straight into shared
-     * memory as the swizzled A operand, the digits of the edge weights are the B operand, the digit sums are read back
-     * from tensor memory once per row segment; graphs of fewer than 2^31 stored entries, otherwise the FMA stream
-     * runs).  The FMA stream is the default because it measured fastest (5.7-5.9 / 5.9-6.1 ms against 8.0 / 8.3 ms
-     * for 2 and 6.0 / 6.5 ms for 3 on the two 256-column layers of a 2.4 M-node, 126 M-entry graph). */
+    /* How rows of 129..256 signed bytes (zeta formats 3 and 5) are aggregated.
+     * 1 = the fp32 FMA stream (bytes converted to fp32 one by one; with format 5 this stream takes the edge values
+     *     as non-negative, as those of the normalized adjacency are);
+     * 2 = exact integer products on the tensor cores through mma.sync (s8 x s8 -> s32: the edge weights of up to 32
+     *     stored entries of a row in 28..31-bit fixed point against a common power of two, split into four signed
+     *     base-256 digits; the digit sums recombined in fp32 when the row ends; edge values of either sign);
+     * 3 = the same fixed-point digits on the 5th-generation tensor cores (tcgen05.mma kind::i8: the gathered rows
+     *     of 64 stored entries go by asynchronous copies straight into shared memory as the swizzled A operand, the
+     *     digits of the edge weights are the B operand, the digit sums are read back from tensor memory once per
+     *     row segment; graphs of fewer than 2^31 stored entries, otherwise the FMA stream runs);
+     * 0 = default: 3 for a launch that wants only the next layer's sign bits and beta (a hidden layer inside
+     *     bigcn_forward) on a graph whose rows average at least 8 stored entries, 1 otherwise.  Measured on the two
+     *     256-column layers of a 2.4 M-node, 126 M-entry graph, bits and beta only: 5.1 / 5.5 ms for 3,
+     *     5.7-5.9 / 5.9-6.1 ms for 1, 8.0 / 8.3 ms for 2.  All paths meet the same tolerance; their fp32 sums differ
+     *     in rounding, so a re-binarized bit at the threshold may differ between them. */
     BIGCN_OPT_BYTE_AGGREGATION = 4
 };
 

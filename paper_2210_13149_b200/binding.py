@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libbigcn.so")
 MAX_LAYERS = 16
 OPT_ZETA_FORMAT = 1
 OPT_LONG_ROW = 2
-OPT_BYTE_AGGREGATION = 4   # rows of 129..256 bytes: 0 = default, 1 = fp32 FMA stream, 2 = integer products (mma.sync), 3 = integer products (tcgen05)
+OPT_BYTE_AGGREGATION = 4   # rows of 129..256 bytes: 0 = default (3 where only bits and beta are wanted, else 1), 1 = fp32 FMA stream, 2 = integer products (mma.sync), 3 = integer products (tcgen05)
 OPT_CONTRACTION = 3     # 0 = auto (default), 1 = XOR / bit-count pipe, 2 = tensor cores wherever the shape is covered
 ZETA_AUTO, ZETA_F32, ZETA_I16, ZETA_I8, ZETA_F16, ZETA_I8H = 0, 1, 2, 3, 4, 5
 

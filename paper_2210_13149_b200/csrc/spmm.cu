@@ -1781,8 +1781,11 @@ cudaError_t launch_spmm(cudaStream_t s, const SpmmArgs& a, int* launches)
     p.run_counter = static_cast<int*>(a.scratch);
     ++*launches;
     const double mean_row = (a.nnz > 0 && a.n > 0) ? (double)a.nnz / (double)a.n : 0.0;
-    // rows of 129..256 signed bytes as tcgen05 integer products (a run of rows must hold fewer than 2^31 entries)
-    if (a.fmt == kZetaI8 && a.byte_path == 3 && a.nnz > 0 && a.nnz < (int64_t(1) << 31) && spmm_tc_covers(p)) return launch_spmm_tc(s, p);
+    // rows of 129..256 signed bytes as tcgen05 integer products (a block's rows must hold fewer than 2^31 entries): when
+    // asked for, and by default where that kernel measured faster than the FMA stream -- a hidden layer of which only
+    // the sign bits and beta are wanted, on a graph whose rows are not much shorter than its chunks' eight segments allow
+    const bool tc_default = a.byte_path == 0 && a.next_bits && !a.h_out && !a.add && mean_row >= 8.0;
+    if (a.fmt == kZetaI8 && (a.byte_path == 3 || tc_default) && a.nnz > 0 && a.nnz < (int64_t(1) << 31) && spmm_tc_covers(p)) return launch_spmm_tc(s, p);
     switch (a.fmt) {
         case kZetaF32: return dispatch<float>(s, p, mean_row);
         case kZetaF16: return dispatch<__half>(s, p, mean_row);

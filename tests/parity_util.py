@@ -111,7 +111,9 @@ def end_to_end_with_flip_accounting(ctx, G, layers, run: OracleRun, X: torch.Ten
     * every later layer is compared with the oracle's layer fed the GPU's own packed input (the
       re-binarized bits unpacked by the oracle, and the GPU's beta): all rows of H' within the
       tolerance, re-binarized bits equal to the sign of that reference except where the reference
-      lies within the tolerance of the threshold, the next beta within the tolerance.
+      lies within the tolerance of the threshold, the next beta within the tolerance -- for the launch
+      that also writes H' and for the launch that wants only bits and beta (what bigcn_forward runs
+      for a hidden layer; its outputs feed the next layer here as they do there).
 
     Beside that it keeps the accounting against the oracle's own end-to-end run (whose later layers
     see the oracle's bits, so a threshold flip moves the rows downstream of it): threshold flips per
@@ -142,9 +144,16 @@ def end_to_end_with_flip_accounting(ctx, G, layers, run: OracleRun, X: torch.Ten
             own_F, own_beta = oracle.binarize_rows(own_H, nl.in_shift, nl.in_scale)
             flips, bad, total = flip_report(bits_from_dev(out["next_bits"]), own_F, own_H, nl.in_shift)
             assert bad == 0, "layer %d on the GPU's own input: %d of %d sign flips away from the threshold" % (l, bad, flips)
-            report["own_fed_flips"].append(flips)
             np.testing.assert_allclose(out["next_beta"].cpu().numpy(), own_beta, rtol=RTOL, atol=ATOL)
-            del own_F, own_beta
+            # the same layer as bigcn_forward launches it -- only the sign bits and beta wanted, which may run another
+            # aggregation kernel -- held to the same reference; its outputs are the ones carried to the next layer
+            carried = ctx.layer_forward(G, layers[l], bits, beta, want_h=False, next_layer=nxt)
+            flips, bad, total = flip_report(bits_from_dev(carried["next_bits"]), own_F, own_H, nl.in_shift)
+            assert bad == 0, "layer %d (bits only) on the GPU's own input: %d of %d sign flips away from the threshold" % (l, bad, flips)
+            report["own_fed_flips"].append(flips)
+            np.testing.assert_allclose(carried["next_beta"].cpu().numpy(), own_beta, rtol=RTOL, atol=ATOL)
+            out["next_bits"], out["next_beta"] = carried["next_bits"], carried["next_beta"]
+            del own_F, own_beta, carried
         del own_H
         # ---- accounting against the oracle's own end-to-end run
         tainted = (A @ dirty.to(torch.float32).unsqueeze(1)).squeeze(1) > 0    # rows that gather a differing row

@@ -518,6 +518,18 @@ def check_layer_forward(ctx, B, fmt, n, e, d_in, d_out):
         assert (nb[:, d_out // 32] >> (d_out % 32) == 0).all()
     assert (nb[:, (d_out + 31) // 32:] == 0).all()
     np.testing.assert_allclose(out["next_beta"].cpu().numpy(), beta_n, rtol=RTOL, atol=ATOL)
+    # the same layer with only the sign bits and beta wanted (how a hidden layer runs inside bigcn_forward; for byte
+    # rows of 129..256 columns that launch takes the tcgen05 aggregation by default)
+    outb = ctx.layer_forward(G, layer, bits_to_dev(t.bits), dev(t.beta), want_h=False, next_layer=nxt)
+    ctx.sync_check()
+    nb = bits_from_dev(outb["next_bits"])
+    flips, bad, total = flip_report(nb, Fn, t.H_out, nshift)
+    assert bad == 0, "bits only: %d sign flips away from the threshold (of %d flips, %d bits)" % (bad, flips, total)
+    assert flips <= max(2, total // 2000)
+    if d_out % 32:
+        assert (nb[:, d_out // 32] >> (d_out % 32) == 0).all()
+    assert (nb[:, (d_out + 31) // 32:] == 0).all()
+    np.testing.assert_allclose(outb["next_beta"].cpu().numpy(), beta_n, rtol=RTOL, atol=ATOL)
 
 
 @pytest.mark.parametrize("fmt", FORMATS)
