@@ -435,7 +435,8 @@ __device__ __forceinline__ float digits_to_float(uint32_t d0, uint32_t d1, uint3
 }
 
 // kBitsOnly: the launch wants only the next layer's sign bits and beta (no fp32 output, nothing added to the rows)
-template <bool kHalf, bool kBitsOnly>
+// kFull: rows of exactly 256 bytes, all of them columns (no piece of a row and no column needs a test)
+template <bool kHalf, bool kBitsOnly, bool kFull>
 __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, volatile int* abort, uint32_t tmem_base)
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;      // warp = tensor-memory lane quarter
@@ -453,7 +454,7 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const int col = 128 * h + tid;
-        col_in[h] = col < p.d_out;
+        col_in[h] = kFull || col < p.d_out;
         alpha[h] = col_in[h] ? (p.col_w ? __ldg(p.col_w + col) : 1.f) : 0.f;
         shift[h] = (col_in[h] && p.next_shift) ? __ldg(p.next_shift + col) : 0.f;
         scale[h] = (col_in[h] && p.next_shift) ? __ldg(p.next_scale + col) : 1.f;
@@ -463,7 +464,7 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
     const char* zeta_b = reinterpret_cast<const char*>(p.zeta);
     const uint32_t row_bytes = (uint32_t)p.nv * 16u;
     const int sub = lane >> 3, piece = lane & 7;              // a warp instruction copies 4 entries x 128 contiguous bytes
-    const bool lo_in = piece < p.nv, hi_in = 8 + piece < p.nv;   // this lane's 16-byte piece exists in operand 0 / 1
+    const bool lo_in = kFull || piece < p.nv, hi_in = kFull || 8 + piece < p.nv;   // this lane's 16-byte piece exists in operand 0 / 1
     const char* zeta_l = zeta_b + piece * 16;
     uint32_t dst_off[4];                                      // where this lane's piece of entry 16 warp + 4 g + sub goes inside a stage
 #pragma unroll
@@ -577,7 +578,7 @@ __device__ __forceinline__ void consumers(const SpmmDev& p, unsigned char* sm, v
     asm volatile("cp.async.wait_all;\n" ::: "memory");        // nothing of this thread is in flight when the block leaves
 }
 
-template <bool kHalf, bool kBitsOnly>
+template <bool kHalf, bool kBitsOnly, bool kFull>
 __global__ void __launch_bounds__(kThreads, 4)
 spmm_tc_kernel(const SpmmDev p)
 {
@@ -600,7 +601,7 @@ spmm_tc_kernel(const SpmmDev p)
     const uint32_t tmem_base = *tmem_slot;
     if (warp == kConsumers / 32) producer<kHalf>(p, sm, abort);
     else if (warp == kConsumers / 32 + 1) issuer(p, sm, abort, tmem_base);
-    else consumers<kHalf, kBitsOnly>(p, sm, abort, tmem_base);
+    else consumers<kHalf, kBitsOnly, kFull>(p, sm, abort, tmem_base);
     tc::fence_before_sync();
     __syncthreads();
     if (warp == 0) tc::tmem_free(tmem_base, kTmemCols);
@@ -626,8 +627,13 @@ cudaError_t launch_spmm_tc(cudaStream_t s, const SpmmDev& p)
         kernel<<<grid, kThreads, kSmemBytes, s>>>(p);
         return cudaGetLastError();
     };
-    if (p.half_dots) return bits_only ? launch(spmm_tc_kernel<true, true>) : launch(spmm_tc_kernel<true, false>);
-    return bits_only ? launch(spmm_tc_kernel<false, true>) : launch(spmm_tc_kernel<false, false>);
+    const bool full = p.nv == 16 && p.d_out == 256;
+    if (p.half_dots) {
+        if (bits_only) return full ? launch(spmm_tc_kernel<true, true, true>) : launch(spmm_tc_kernel<true, true, false>);
+        return full ? launch(spmm_tc_kernel<true, false, true>) : launch(spmm_tc_kernel<true, false, false>);
+    }
+    if (bits_only) return full ? launch(spmm_tc_kernel<false, true, true>) : launch(spmm_tc_kernel<false, true, false>);
+    return full ? launch(spmm_tc_kernel<false, false, true>) : launch(spmm_tc_kernel<false, false, false>);
 }
 
 int spmm_tc_timeouts()
