@@ -100,7 +100,7 @@ enum {
      *     row segment; graphs of fewer than 2^31 stored entries, otherwise the FMA stream runs);
      * 0 = default: 3 for a launch that wants only the next layer's sign bits and beta (a hidden layer inside
      *     bigcn_forward) on a graph whose rows average at least 8 stored entries, 1 otherwise.  Measured on the two
-     *     256-column layers of a 2.4 M-node, 126 M-entry graph, bits and beta only: 5.1 / 5.5 ms for 3,
+     *     256-column layers of a 2.4 M-node, 126 M-entry graph, bits and beta only: 4.9 / 5.2 ms for 3,
      *     5.7-5.9 / 5.9-6.1 ms for 1, 8.0 / 8.3 ms for 2.  All paths meet the same tolerance; their fp32 sums differ
      *     in rounding, so a re-binarized bit at the threshold may differ between them. */
     BIGCN_OPT_BYTE_AGGREGATION = 4
