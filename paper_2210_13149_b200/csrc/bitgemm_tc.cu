@@ -137,8 +137,10 @@ template <> struct TcOut<kZetaF32> {
 // memory (the feature tile's space, free once the products are done): a thread owns one row of the
 // accumulators, and rows are far apart in zeta, so each warp first collects 32 rows x 128 bytes and
 // then stores them as whole 128-byte row segments.
-template <int N, int FMT>
-__global__ void __launch_bounds__(kTcThreads, 2)
+// kDebug: the debug taps (the integer dots and the literal fp32 zeta of every element) are wanted.
+// Blocks per SM: two where the accumulator takes 256 of the 512 tensor-memory columns or the taps are on, three otherwise.
+template <int N, int FMT, bool kDebug>
+__global__ void __launch_bounds__(kTcThreads, (N > 128 || kDebug) ? 2 : 3)
 bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32_t* __restrict__ BT, int64_t stride_b,
                   int64_t n, int d_in, int d_out, const float* __restrict__ beta, const float* __restrict__ alpha,
                   void* __restrict__ zeta, int64_t ldz, int32_t* __restrict__ dbg_dot, float* __restrict__ dbg_zeta,
@@ -254,7 +256,7 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
         const int64_t row0 = tile_row0(i) + lane_base;
         const int64_t row = row0 + lane;
         const bool row_in = row < n;
-        const float be = (row_in && (FMT == kZetaF32 || FMT == kZetaI8H || dbg_zeta || row_tail)) ? __ldg(beta + row) : 0.f;
+        const float be = (row_in && (FMT == kZetaF32 || FMT == kZetaI8H || (kDebug && dbg_zeta) || row_tail)) ? __ldg(beta + row) : 0.f;
         float row_fac = be;                                 // the node factor the aggregation multiplies the edge value by
         int f0 = 0;                                         // half-dot bytes: the row's first sign (0 when d_in is odd)
         if constexpr (FMT == kZetaI8H) {
@@ -286,9 +288,11 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
 #pragma unroll
                     for (int e = 0; e < 16; ++e) dot[e] = (c0 + e < d_out) ? (int)v[e] - pad : 0;   // padding columns of zeta stay 0
                 }
-                int full[16];                               // the true dots, for the debug taps
+                int full[kDebug ? 16 : 1];                  // the true dots, for the debug taps
+                if constexpr (kDebug) {
 #pragma unroll
-                for (int e = 0; e < 16; ++e) full[e] = dot[e];
+                    for (int e = 0; e < 16; ++e) full[e] = dot[e];
+                }
                 if constexpr (FMT == kZetaI8H) {            // s = (dot - f0 b0_j - 1) / 2: odd by construction, exact
                     const int4* hd = reinterpret_cast<const int4*>(hd_s + (f0 + 1) * N + c0);
                     int sub[16];
@@ -316,13 +320,15 @@ bitgemm_tc_kernel(const uint32_t* __restrict__ A, int64_t stride_a, const uint32
                     const int piece = ch * kElt + u;
                     *reinterpret_cast<uint4*>(scr + lane * 128 + ((piece ^ (lane & 7)) * 16)) = out[u];
                 }
-                if (row_in && (dbg_dot || dbg_zeta)) {
+                if constexpr (kDebug) {
+                    if (row_in) {
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        const int c = c0 + e;
-                        if (c < d_out) {
-                            if (dbg_dot) dbg_dot[row * (int64_t)d_out + c] = full[e];
-                            if (dbg_zeta) dbg_zeta[row * (int64_t)d_out + c] = __fmul_rn(__fmul_rn(be, al_s[c]), (float)full[e]);
+                        for (int e = 0; e < 16; ++e) {
+                            const int c = c0 + e;
+                            if (c < d_out) {
+                                if (dbg_dot) dbg_dot[row * (int64_t)d_out + c] = full[e];
+                                if (dbg_zeta) dbg_zeta[row * (int64_t)d_out + c] = __fmul_rn(__fmul_rn(be, al_s[c]), (float)full[e]);
+                            }
                         }
                     }
                 }
@@ -358,11 +364,18 @@ cudaError_t launch_tc_inst(cudaStream_t s, const uint32_t* A, int64_t stride_a, 
     // a CTA holds 256 of the SM's 512 tensor-memory columns when N > 128: ask for enough shared memory that a third
     // CTA can never become resident on an SM and sit in tcgen05.alloc until a neighbour leaves
     if (N > 128) smem = std::max<size_t>(smem, 78 * 1024);
-    cudaError_t e = cudaFuncSetAttribute(bitgemm_tc_kernel<N, FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, kTcRows), sm_count() * 2);
-    bitgemm_tc_kernel<N, FMT><<<grid, kTcThreads, smem, s>>>(A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0, row_tail);
-    return cudaGetLastError();
+    const bool debug = dbg_dot || dbg_zeta;
+    auto launch = [&](auto kernel, int blocks_per_sm) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        // persistent blocks: as many as stay resident (tensor-memory columns, registers, and shared memory: 227 KB per SM)
+        const int fit = (int)std::max<size_t>(1, std::min<size_t>((size_t)blocks_per_sm, (size_t)(227 * 1024) / (smem + 2048)));
+        const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n, kTcRows), (int64_t)sm_count() * fit);
+        kernel<<<grid, kTcThreads, smem, s>>>(A, stride_a, BT, stride_b, n, d_in, d_out, beta, alpha, zeta, ldz, dbg_dot, dbg_zeta, nws, col_b0, row_tail);
+        return cudaGetLastError();
+    };
+    if (debug) return launch(bitgemm_tc_kernel<N, FMT, true>, 2);
+    return launch(bitgemm_tc_kernel<N, FMT, false>, N > 128 ? 2 : 3);
 }
 
 template <int N>
