@@ -400,6 +400,12 @@ def run_ours(args):
                     extras[key] = "failed: %r" % (exc,)
                 finally:
                     ctx.set_option(binding.OPT_BYTE_AGGREGATION, 0)
+        # the gather of the aggregations alone (no weights, no sums, no output): what the memory system needs for the
+        # row sizes this network's layers store
+        try:
+            extras["gather_only_ms"] = {str(rb): ctx.measure_gather_peak(G, rb) for rb in (256, 64)}
+        except Exception as exc:
+            extras["gather_only_ms"] = "failed: %r" % (exc,)
         # the same contraction on the XOR / bit-count pipe (the library's other path), for comparison
         try:
             ctx.set_option(binding.OPT_CONTRACTION, 1)

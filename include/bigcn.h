@@ -358,6 +358,15 @@ bigcn_status bigcn_sage_layer_forward(bigcn_ctx* ctx, const bigcn_graph* mean_gr
  * Needs 1.2 MB of workspace.  SYNCHRONOUS. */
 bigcn_status bigcn_measure_popc_peak(bigcn_ctx* ctx, double* word_steps_per_s /*host*/);
 
+/* Measurement aid: the time the memory system alone needs for the access pattern of the aggregation
+ * H' = A_tilde zeta (last equation of Sec. 4.2.3) on graph g -- for every stored entry, the row colidx[e] of a
+ * row-major matrix of `row_bytes` bytes per row (a power of two, 16..512) is read, 16 bytes per lane, and
+ * discarded; no weights, no sums, no output.  *ms (host) receives the best of three runs in milliseconds:
+ * the ceiling an aggregation kernel over rows of that size can be held against.  The rows read are the
+ * first n * row_bytes bytes of the workspace (contents irrelevant); needs that much workspace + 256 bytes.
+ * SYNCHRONOUS. */
+bigcn_status bigcn_measure_gather_peak(bigcn_ctx* ctx, const bigcn_graph* g, int32_t row_bytes, double* ms /*host*/);
+
 /* One layer without any allocation (the paper has no counterpart of this call; it is a packaging of
  * bigcn_layer_forward() for callers that must not allocate device memory: a process whose own pool
  * took the whole GPU at start-up, so that cudaMalloc would fail, or a latency-critical loop that

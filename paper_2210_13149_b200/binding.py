@@ -85,6 +85,7 @@ SIGNATURES = {
     "bigcn_layer_backward": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer), _vp, _i64,
                                             _vp, _vp, _vp, _i64, _vp, _i64, _vp, _i64]),
     "bigcn_measure_popc_peak": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_double)]),
+    "bigcn_measure_gather_peak": (ctypes.c_int, [_vp, _vp, ctypes.c_int32, ctypes.POINTER(ctypes.c_double)]),
     "bigcn_layer_forward_noalloc": (ctypes.c_int, [_vp, ctypes.POINTER(bigcn_graph), ctypes.POINTER(bigcn_layer),
                                                    _vp, _vp, _vp, _i64, ctypes.POINTER(bigcn_layer), _vp, _vp]),
 }
@@ -433,6 +434,14 @@ class BiGCN:
         self.ensure_workspace(2 << 20)
         out = ctypes.c_double(0.0)
         self._check(self.lib.bigcn_measure_popc_peak(self.h, ctypes.byref(out)))
+        return float(out.value)
+
+    def measure_gather_peak(self, G, row_bytes: int) -> float:
+        """Milliseconds the memory system alone needs to read, for every stored entry of G, the row of
+        `row_bytes` bytes its column index names (the aggregation's gather without any arithmetic)."""
+        self.ensure_workspace(G.n * row_bytes + (1 << 20))
+        out = ctypes.c_double(0.0)
+        self._check(self.lib.bigcn_measure_gather_peak(self.h, ctypes.byref(G.c), int(row_bytes), ctypes.byref(out)))
         return float(out.value)
 
     # -- convenience built only from the calls above

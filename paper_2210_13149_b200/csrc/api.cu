@@ -858,6 +858,24 @@ bigcn_status bigcn_measure_popc_peak(bigcn_ctx* ctx, double* word_steps_per_s)
     return BIGCN_OK;
 }
 
+bigcn_status bigcn_measure_gather_peak(bigcn_ctx* ctx, const bigcn_graph* g, int32_t row_bytes, double* ms)
+{
+    bigcn_status st = bind_device(ctx);
+    if (st != BIGCN_OK) return st;
+    if ((st = check_graph(ctx, g)) != BIGCN_OK) return st;
+    if (!ms) return fail(ctx, BIGCN_ERR_NULL, "ms is null");
+    if (row_bytes < 16 || row_bytes > 512 || (row_bytes & (row_bytes - 1))) return fail(ctx, BIGCN_ERR_SHAPE, "row_bytes=%d must be a power of two in 16..512", row_bytes);
+    const size_t need = up((size_t)g->n * (size_t)row_bytes) + 256;
+    if (!ctx->ws || ctx->ws_bytes < need) return fail(ctx, BIGCN_ERR_WORKSPACE, "needs %zu bytes of workspace", need);
+    *ms = 0.0;
+    if (g->n == 0 || g->nnz == 0) return BIGCN_OK;
+    cudaError_t e = measure_gather_peak(ctx->stream, g->colidx, g->nnz, ctx->ws, row_bytes,
+                                        static_cast<char*>(ctx->ws) + up((size_t)g->n * (size_t)row_bytes), ms, &ctx->launches_i);
+    finish_call(ctx);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "gather measurement");
+    return BIGCN_OK;
+}
+
 bigcn_status bigcn_mean_adjacency(bigcn_ctx* ctx, int64_t n, int64_t nnz_in,
                                   const int64_t* rowptr_A, const int32_t* colidx_A,
                                   int64_t* rowptr, int32_t* colidx, float* val, float* inv_deg,

@@ -96,6 +96,8 @@ size_t col_stats_scratch_bytes(int d);
 
 cudaError_t measure_popc_peak(cudaStream_t s, void* scratch, double* word_steps_per_s, int* launches);
 size_t popc_peak_scratch_bytes();
+cudaError_t measure_gather_peak(cudaStream_t s, const int32_t* colidx, int64_t nnz, const void* rows, int row_bytes,
+                                void* scratch, double* ms_out, int* launches);
 
 // The same contraction as tcgen05 int8 products (bitgemm_tc.cu): shapes with d_in, d_out <= 256.
 bool bitgemm_tc_covers(int d_in, int d_out, int64_t stride_a, int64_t stride_b);

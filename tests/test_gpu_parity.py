@@ -598,6 +598,18 @@ def test_isolated_nodes_and_empty_graph(ctx, B):
     assert logits.shape == (0, d_out)
 
 
+def test_gather_only_probe(ctx, B):
+    """The measurement aid that reads every stored entry's operand row and nothing else: runs, times, validates."""
+    _, _, g = small_graph(5000, 60000, 11)
+    G = device_graph(B, g)
+    for rb in (16, 64, 256, 512):
+        assert ctx.measure_gather_peak(G, rb) > 0.0
+    for bad in (0, 8, 48, 1024):
+        with pytest.raises(B.BigcnError):
+            ctx.measure_gather_peak(G, bad)
+    ctx.sync_check()
+
+
 def test_argument_errors_are_reported_not_launched(ctx, B):
     import ctypes
     n, d_in, d_out = 10, 40, 5
