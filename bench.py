@@ -592,6 +592,13 @@ def run_ours(args):
                          "operand row once + one operand row per further stored entry whose source is not among the "
                          "highest-degree rows an ideal 126 MB cache would hold"}
 
+    # the same launch against the gather alone (no arithmetic): how close the kernel is to what the memory system can do
+    go = extras.get("gather_only_ms")
+    if isinstance(go, dict) and str(kernels["spmm_l%d" % dom]["row_bytes"]) in go:
+        g_ms = go[str(kernels["spmm_l%d" % dom]["row_bytes"])]
+        roofline["gather_only_ms"] = g_ms
+        roofline["gather_only_over_kernel"] = g_ms / spmm_ms[dom]
+
     cpu = None
     if not args.no_cpu_baseline:
         try:
