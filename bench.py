@@ -43,7 +43,8 @@ def parse_args():
                          "for the hidden layer of the workload")
     ap.add_argument("--zeta-format", type=int, default=0, help="0 auto, 1 fp32, 2 int16, 3 int8, 4 fp16, 5 half-dot bytes")
     ap.add_argument("--byte-aggregation", type=int, default=0,
-                    help="rows of 129..256 bytes: 0 / 1 the fp32 FMA stream (default), 2 integer tensor-core products")
+                    help="rows of 129..256 bytes: 0 the library's choice (tcgen05 products for hidden layers), 1 the fp32 FMA stream, "
+                         "2 integer products on mma.sync, 3 tcgen05 products wherever they apply")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--graph", action="store_true", help="also time the forward replayed as one CUDA graph")
